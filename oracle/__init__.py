@@ -1,0 +1,222 @@
+"""fp64 CPU oracle for the Fork-dLLM sampling step -- TEST INFRASTRUCTURE ONLY.
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import this package.
+The product package never does, and this package never imports the product package.
+
+It is a ctypes wrapper around ``fork_oracle.c`` (plain C, fp64), which states Algorithm 2
+(Fork-dLLM), the softmax confidence / entropy / log-probability definitions of Section 2 and
+Section 3.2, and the semi-autoregressive loop of Section 4.1 (Setup) as directly as possible.
+
+Arrays are numpy: bf16 logits are ``uint16`` bit patterns, fp32 logits are ``float32``.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "fork_oracle.c")
+_LIB = os.path.join(_HERE, "libfork_oracle.so")
+
+BF16, F32 = 0, 1
+OK, ERR_ARG, ERR_MAX_STEPS, ERR_PROVIDER = 0, -1, -4, -5
+ROW_BAD, ROW_BAD_TOKEN = 1, 2
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc if the shared object is missing or older than its source."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-pthread",
+                               "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+class _StepArgs(C.Structure):
+    _fields_ = [
+        ("logits", C.c_void_p), ("stride_b", C.c_int64), ("stride_l", C.c_int64), ("pos0", C.c_int32),
+        ("B", C.c_int32), ("Lt", C.c_int32), ("Ll", C.c_int32), ("V", C.c_int32), ("dtype", C.c_int32),
+        ("tokens", C.c_void_p), ("mask", C.c_void_p), ("blk_lo", C.c_void_p), ("blk_hi", C.c_void_p),
+        ("threshold", C.c_float), ("step", C.c_int32),
+        ("conf", C.c_void_p), ("cand", C.c_void_p), ("entropy", C.c_void_p), ("logp", C.c_void_p),
+        ("commit_step", C.c_void_p), ("commit_fallback", C.c_void_p), ("commit_logp", C.c_void_p),
+        ("n_unmasked", C.c_void_p), ("is_fallback", C.c_void_p), ("fallback_pos", C.c_void_p),
+        ("nfe", C.c_void_p), ("n_fallback", C.c_void_p),
+        ("row_status", C.c_void_p),
+        ("nthreads", C.c_int32),
+    ]
+
+
+_PROVIDER = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                        C.c_void_p)
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(build())
+        L.fork_oracle_row_stats.restype = None
+        L.fork_oracle_row_stats.argtypes = [C.c_void_p, C.c_int32, C.c_int32] + [C.c_void_p] * 8
+        L.fork_oracle_row_logp.restype = C.c_double
+        L.fork_oracle_row_logp.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
+        L.fork_oracle_step.restype = C.c_int
+        L.fork_oracle_step.argtypes = [C.POINTER(_StepArgs)]
+        L.fork_oracle_logprob.restype = C.c_int
+        L.fork_oracle_logprob.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_int32,
+                                          C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                                          C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32]
+        L.fork_oracle_block_cursors.restype = None
+        L.fork_oracle_block_cursors.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                                C.c_int32, C.c_void_p, C.c_void_p]
+        L.fork_oracle_decode_loop.restype = C.c_int
+        L.fork_oracle_decode_loop.argtypes = [C.POINTER(_StepArgs), C.c_int32, C.c_int32, C.c_int32,
+                                              _PROVIDER, C.c_void_p, C.c_int32, C.c_void_p]
+        L.fork_oracle_threads_used.restype = C.c_int
+        L.fork_oracle_threads_used.argtypes = [C.c_int32, C.c_int64]
+        _lib = L
+    return _lib
+
+
+def _dtype_of(a: np.ndarray) -> int:
+    if a.dtype == np.uint16:
+        return BF16
+    if a.dtype == np.float32:
+        return F32
+    raise TypeError("logits must be uint16 (bf16 bits) or float32, got %s" % a.dtype)
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data
+
+
+def threads_used(nthreads: int, n_rows: int) -> int:
+    return int(lib().fork_oracle_threads_used(nthreads, n_rows))
+
+
+def row_stats(row: np.ndarray) -> dict:
+    """conf, cand, entropy, logp of the candidate, and (m, s, t) for one contiguous logits row."""
+    row = np.ascontiguousarray(row)
+    conf, ent, lp, m, s, t = (C.c_double() for _ in range(6))
+    cand, st = C.c_int32(), C.c_uint32()
+    lib().fork_oracle_row_stats(row.ctypes.data, row.shape[0], _dtype_of(row),
+                                C.addressof(conf), C.addressof(cand), C.addressof(ent), C.addressof(lp),
+                                C.addressof(m), C.addressof(s), C.addressof(t), C.addressof(st))
+    return dict(conf=conf.value, cand=cand.value, entropy=ent.value, logp=lp.value,
+                m=m.value, s=s.value, t=t.value, status=st.value)
+
+
+def row_logp(row: np.ndarray, tok: int):
+    row = np.ascontiguousarray(row)
+    st = C.c_uint32()
+    v = lib().fork_oracle_row_logp(row.ctypes.data, row.shape[0], _dtype_of(row), int(tok), C.addressof(st))
+    return float(v), int(st.value)
+
+
+class StepState:
+    """Host buffers of one batch: the sequence, its mask, and every output of the step."""
+
+    def __init__(self, B: int, Lt: int, tokens=None, mask=None):
+        self.B, self.Lt = B, Lt
+        self.tokens = np.zeros((B, Lt), np.int32) if tokens is None else np.ascontiguousarray(tokens, np.int32).copy()
+        self.mask = np.ones((B, Lt), np.uint8) if mask is None else np.ascontiguousarray(mask, np.uint8).copy()
+        self.conf = np.full((B, Lt), np.nan, np.float64)
+        self.cand = np.full((B, Lt), -1, np.int32)
+        self.entropy = np.full((B, Lt), np.nan, np.float64)
+        self.logp = np.full((B, Lt), np.nan, np.float64)
+        self.commit_step = np.full((B, Lt), -1, np.int32)
+        self.commit_fallback = np.full((B, Lt), 255, np.uint8)
+        self.commit_logp = np.full((B, Lt), np.nan, np.float64)
+        self.n_unmasked = np.zeros(B, np.int32)
+        self.is_fallback = np.zeros(B, np.uint8)
+        self.fallback_pos = np.full(B, -1, np.int32)
+        self.nfe = np.zeros(B, np.int32)
+        self.n_fallback = np.zeros(B, np.int32)
+        self.row_status = np.zeros((B, Lt), np.uint32)
+
+
+def _fill_args(st: StepState, logits: np.ndarray, lo, hi, threshold, step, pos0, nthreads) -> _StepArgs:
+    assert logits.ndim == 3 and logits.flags.c_contiguous
+    B, Ll, V = logits.shape
+    assert B == st.B
+    a = _StepArgs()
+    a.logits = logits.ctypes.data
+    a.stride_b, a.stride_l, a.pos0 = Ll * V, V, pos0
+    a.B, a.Lt, a.Ll, a.V, a.dtype = B, st.Lt, Ll, V, _dtype_of(logits)
+    a.tokens, a.mask = st.tokens.ctypes.data, st.mask.ctypes.data
+    a.blk_lo, a.blk_hi = _ptr(lo), _ptr(hi)
+    a.threshold, a.step = float(threshold), int(step)
+    a.conf, a.cand, a.entropy, a.logp = (x.ctypes.data for x in (st.conf, st.cand, st.entropy, st.logp))
+    a.commit_step, a.commit_fallback, a.commit_logp = (x.ctypes.data for x in
+                                                        (st.commit_step, st.commit_fallback, st.commit_logp))
+    a.n_unmasked, a.is_fallback, a.fallback_pos = (x.ctypes.data for x in
+                                                   (st.n_unmasked, st.is_fallback, st.fallback_pos))
+    a.nfe, a.n_fallback = st.nfe.ctypes.data, st.n_fallback.ctypes.data
+    a.row_status = st.row_status.ctypes.data
+    a.nthreads = nthreads
+    return a
+
+
+def step(st: StepState, logits: np.ndarray, lo: np.ndarray, hi: np.ndarray, threshold: float,
+         step_id: int = 0, pos0: int = 0, nthreads: int = 0) -> int:
+    """One Fork-dLLM sampling step (Algorithm 2) on host buffers; ``st`` is updated in place."""
+    lo = np.ascontiguousarray(lo, np.int32)
+    hi = np.ascontiguousarray(hi, np.int32)
+    a = _fill_args(st, logits, lo, hi, threshold, step_id, pos0, nthreads)
+    return int(lib().fork_oracle_step(C.byref(a)))
+
+
+def logprob(logits: np.ndarray, tokens: np.ndarray, select: np.ndarray, pos0: int = 0, nthreads: int = 0):
+    """Per-token log-likelihood at selected positions and its per-sequence sum (Section 3.2)."""
+    assert logits.ndim == 3 and logits.flags.c_contiguous
+    B, Ll, V = logits.shape
+    tokens = np.ascontiguousarray(tokens, np.int32)
+    select = np.ascontiguousarray(select, np.uint8)
+    Lt = tokens.shape[1]
+    lp = np.zeros((B, Lt), np.float64)
+    ssum = np.zeros(B, np.float64)
+    scnt = np.zeros(B, np.int32)
+    status = np.zeros((B, Lt), np.uint32)
+    rc = lib().fork_oracle_logprob(logits.ctypes.data, Ll * V, V, pos0, B, Lt, Ll, V, _dtype_of(logits),
+                                   tokens.ctypes.data, select.ctypes.data, lp.ctypes.data, ssum.ctypes.data,
+                                   scnt.ctypes.data, status.ctypes.data, nthreads)
+    return int(rc), lp, ssum, scnt, status
+
+
+def block_cursors(mask: np.ndarray, gen_lo: int, gen_hi: int, block_len: int, lo=None, hi=None):
+    mask = np.ascontiguousarray(mask, np.uint8)
+    B, Lt = mask.shape
+    if lo is None:
+        lo = np.full(B, gen_lo, np.int32)
+        hi = np.full(B, gen_lo, np.int32)
+    lib().fork_oracle_block_cursors(mask.ctypes.data, B, Lt, gen_lo, gen_hi, block_len,
+                                    lo.ctypes.data, hi.ctypes.data)
+    return lo, hi
+
+
+def decode_loop(st: StepState, logits: np.ndarray, block_len: int, gen_lo: int, gen_hi: int, provider,
+                threshold: float, max_steps: int, step0: int = 0, pos0: int = 0, nthreads: int = 0):
+    """Run the semi-autoregressive loop.  ``provider(step, tokens, mask, lo, hi, logits)`` fills
+    ``logits`` (numpy views of the live host buffers) and returns 0, or non-zero to abort."""
+    B, Lt = st.B, st.Lt
+
+    def _cb(_ctx, step_id, _tok, _mask, lo_p, hi_p, _out):
+        lo = np.ctypeslib.as_array(C.cast(lo_p, C.POINTER(C.c_int32)), shape=(B,))
+        hi = np.ctypeslib.as_array(C.cast(hi_p, C.POINTER(C.c_int32)), shape=(B,))
+        try:
+            return int(provider(int(step_id), st.tokens, st.mask, lo, hi, logits) or 0)
+        except Exception:  # a Python error must not unwind through C
+            import traceback
+            traceback.print_exc()
+            return 1
+
+    a = _fill_args(st, logits, None, None, threshold, step0, pos0, nthreads)
+    steps = C.c_int32(0)
+    rc = lib().fork_oracle_decode_loop(C.byref(a), block_len, gen_lo, gen_hi, _PROVIDER(_cb), None,
+                                       max_steps, C.addressof(steps))
+    return int(rc), int(steps.value)
