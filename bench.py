@@ -1,0 +1,520 @@
+#!/usr/bin/env python
+"""Benchmark of the Fork-dLLM confidence pass (fork_step) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload b8|passk|sweep]
+
+A "step" is one fork_step call (active-set kernel + streaming reduce/select/commit kernel) on a
+batch whose active block is fully masked: B*block_len live rows, each V logits read once.
+Prints ONE JSON line (rank 0).  `value` is masked positions per second with the logits already in
+HBM; `e2e` is the same metric through fork_step_host with pinned HOST buffers (H2D of the logits
+window and D2H of every output inside the timed region); `roofline` is the streaming kernel's
+algorithmic bytes over its own CUDA-event duration against the measured HBM peak; `cpu_baseline`
+is the fp64 oracle timed on the host cores on one full-block step's rows.
+
+With `--impl reference` the oracle itself is the timed arm (rank 0 only, host cores).
+Multi-GPU (torchrun, one rank per GPU): sequences are independent, so every rank runs its own
+batch (different seed) with no data-path collective; timing is the max over ranks (weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes as C
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "masked positions/s (fork_step; HBM GB/s and fraction of peak in `roofline`)"
+UNIT = "positions/s"
+L2_BYTES = 126 * 1024 * 1024
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json, copy bandwidth)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
+
+
+def rank_info():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+
+
+def shard_seed(base_seed: int, rank: int) -> int:
+    """Every rank decodes its own, different batch of sequences (weak scaling over B)."""
+    return (base_seed + 0x9E3779B1 * rank) & 0xFFFFFFFFFFFF
+
+
+def aggregate(rows_per_rank_step: int, steps: int, world: int, max_ms: float) -> float:
+    """Whole-job throughput: rows processed by all ranks over the slowest rank's time."""
+    return rows_per_rank_step * steps * world / (max_ms * 1e-3)
+
+
+def max_over_ranks(value: float, device) -> float:
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return value
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons while the GPU is under the benchmark's load."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap,utilization.gpu")
+
+    def __init__(self, index: int):
+        self.samples = []
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, smmax, reasons, power = [], [], set(), []
+        for s in self.samples:
+            f = [x.strip() for x in s.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                util = float(f[7])
+                if util < 20:          # keep only samples taken under load
+                    continue
+                sm.append(float(f[0])); smmax.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smmax) if smmax else None,
+                "power_w_max": max(power) if power else None, "samples_under_load": len(sm),
+                "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------------
+def full_block_setup(w, seed, n_buf, n_state, device):
+    """Rotating block-window logits buffers (together larger than 2x L2) filled by the device
+    generator, and a pool of fresh all-masked states."""
+    import torch
+    import fork_synth as fs
+    import paper_2609_39859_b200 as pkg
+    cfg = w.cfg()
+    cfg.seed = seed
+    BL = w.block_len
+    tdt = torch.bfloat16 if w.dtype == fs.BF16 else torch.float32
+    lo = torch.zeros(w.B, dtype=torch.int32, device=device)
+    hi = torch.full((w.B,), BL, dtype=torch.int32, device=device)
+    ones = torch.ones((w.B, w.Lt), dtype=torch.uint8, device=device)
+    bufs = []
+    for i in range(n_buf):
+        t = torch.empty((w.B, BL, w.V), dtype=tdt, device=device)
+        fs.cuda_fill(cfg, i, ones.data_ptr(), lo.data_ptr(), hi.data_ptr(), t.data_ptr(), BL * w.V, w.V, 0, BL,
+                     stream_ptr=torch.cuda.current_stream().cuda_stream)
+        bufs.append(t)
+    states = [pkg.ForkState(w.B, w.Lt, device=device) for _ in range(n_state)]
+    pool = torch.ones((n_state, w.B, w.Lt), dtype=torch.uint8, device=device)
+    for i, s in enumerate(states):          # all masks in one tensor: one fill re-arms the whole pool
+        s.mask = pool[i]
+    states[0].pool_mask = pool
+    torch.cuda.synchronize()
+    return cfg, bufs, states, lo, hi
+
+
+def reset_states(states):
+    states[0].pool_mask[:len(states)].fill_(1)
+
+
+def time_full_block(w, seed, steps, warmup, device, use_graph=True):
+    """Times `steps` fork_step calls (after `warmup`), each on B*block_len live rows.  The timed
+    steps are replayed from one CUDA graph when `use_graph` (host launch cost would otherwise bound
+    a ~10 us step); a second, un-graphed pass brackets each step's streaming kernel with events."""
+    import torch
+    import paper_2609_39859_b200 as pkg
+    rows = w.B * w.block_len
+    row_bytes = w.V * w.es
+    n_buf = max(2, -(-2 * L2_BYTES // (rows * row_bytes)) + 1)
+    n_state = min(max(steps, warmup), 64)
+    cfg, bufs, states, lo, hi = full_block_setup(w, seed, n_buf, n_state, device)
+    L = pkg.lib()
+    cache = {}
+
+    def call(i, sp):
+        s, b = i % n_state, i % n_buf
+        a = cache.get((s, b))
+        if a is None:
+            a = cache[(s, b)] = pkg.make_step_args(states[s], bufs[b], lo, hi, w.threshold, step=0)
+        rc = L.fork_step(C.byref(a), C.c_void_p(states[s].ws_ptr), states[s].ws_bytes, sp)
+        if rc != 0:
+            raise RuntimeError("fork_step: " + pkg.fork_status_string(rc))
+
+    def run(n, first, sp):
+        """n steps; the state pool is re-armed (masks set back to 1) every n_state steps"""
+        done = 0
+        while done < n:
+            chunk = min(n_state, n - done)
+            reset_states(states[:chunk])
+            for j in range(chunk):
+                call(first + done + j, sp)
+            done += chunk
+
+    stream = torch.cuda.current_stream()
+    sp = C.c_void_p(stream.cuda_stream)
+    run(warmup, 0, sp)
+    torch.cuda.synchronize()
+    launches0 = pkg.fork_kernel_launches()
+    graph = None
+    if use_graph:
+        try:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                run(steps, warmup, C.c_void_p(torch.cuda.current_stream().cuda_stream))
+        except Exception as e:                      # fall back to plain launches, and say so
+            sys.stderr.write("bench: CUDA graph capture failed (%r); timing plain launches\n" % (e,))
+            graph = None
+            torch.cuda.synchronize()
+    launches = pkg.fork_kernel_launches() - launches0 if graph is not None else None
+    stream = torch.cuda.current_stream()
+    sp = C.c_void_p(stream.cuda_stream)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    host_t0 = time.perf_counter()
+    if graph is not None:
+        e0.record(stream)
+        graph.replay()
+        e1.record(stream)
+    else:
+        launches0 = pkg.fork_kernel_launches()
+        e0.record(stream)
+        run(steps, warmup, sp)
+        e1.record(stream)
+        launches = pkg.fork_kernel_launches() - launches0
+    host_submit_ms = (time.perf_counter() - host_t0) * 1e3
+    torch.cuda.synchronize()
+    total_ms = e0.elapsed_time(e1)
+    # second pass: events around each step's streaming kernel (plain launches)
+    n = min(steps, n_state)
+    reset_states(states[:n])
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+    for a, b in evs:                                 # creates the CUDA events the library will re-record
+        a.record(stream)
+        b.record(stream)
+    torch.cuda.synchronize()
+    for j in range(n):
+        L.fork_set_timing_events(C.c_void_p(evs[j][0].cuda_event), C.c_void_p(evs[j][1].cuda_event))
+        call(warmup + j, sp)
+    torch.cuda.synchronize()
+    kernel_ms = sum(a.elapsed_time(b) for a, b in evs) / n
+    return dict(rows=rows, row_bytes=row_bytes, total_ms=total_ms, ms_per_step=total_ms / steps,
+                kernel_ms=kernel_ms, launches=launches, n_buf=n_buf, graph=graph is not None,
+                host_submit_ms=host_submit_ms, setup=(cfg, bufs, states, lo, hi), keep=graph)
+
+
+def time_e2e(w, setup, steps, warmup, device):
+    """fork_step_host: pinned host buffers in, every output back out, inside the timed region."""
+    import torch
+    import paper_2609_39859_b200 as pkg
+    cfg, bufs, states, lo, hi = setup
+    B, Lt, BL, V = w.B, w.Lt, w.block_len, w.V
+    L = pkg.lib()
+    h_logits = torch.empty(bufs[0].shape, dtype=bufs[0].dtype).pin_memory()
+    h_logits.copy_(bufs[0])
+    pin = lambda *shape, dt: torch.zeros(shape, dtype=dt).pin_memory()
+    h = dict(tokens=pin(B, Lt, dt=torch.int32), mask=pin(B, Lt, dt=torch.uint8), lo=pin(B, dt=torch.int32),
+             hi=pin(B, dt=torch.int32), conf=pin(B, Lt, dt=torch.float32), cand=pin(B, Lt, dt=torch.int32),
+             entropy=pin(B, Lt, dt=torch.float32), logp=pin(B, Lt, dt=torch.float32),
+             row_status=pin(B, Lt, dt=torch.int32), commit_step=pin(B, Lt, dt=torch.int32),
+             commit_fallback=pin(B, Lt, dt=torch.uint8), commit_logp=pin(B, Lt, dt=torch.float32),
+             n_unmasked=pin(B, dt=torch.int32), is_fallback=pin(B, dt=torch.uint8), fallback_pos=pin(B, dt=torch.int32),
+             nfe=pin(B, dt=torch.int32), n_fallback=pin(B, dt=torch.int32))
+    h["hi"].fill_(BL)
+    a = pkg.fork_step_args()
+    a.logits = h_logits.data_ptr()
+    a.stride_b, a.stride_l, a.pos0 = BL * V, V, 0
+    a.B, a.Lt, a.Ll, a.V, a.dtype = B, Lt, BL, V, (pkg.FORK_BF16 if w.es == 2 else pkg.FORK_F32)
+    a.tokens, a.mask, a.blk_lo, a.blk_hi = h["tokens"].data_ptr(), h["mask"].data_ptr(), h["lo"].data_ptr(), h["hi"].data_ptr()
+    a.threshold, a.step = w.threshold, 0
+    for name in ("conf", "cand", "entropy", "logp", "row_status", "commit_step", "commit_fallback", "commit_logp",
+                 "n_unmasked", "is_fallback", "fallback_pos", "nfe", "n_fallback"):
+        setattr(a, name, h[name].data_ptr())
+    nbytes = L.fork_staging_bytes(C.byref(a))
+    staging = torch.empty(nbytes + 256, dtype=torch.uint8, device=device)
+    sp = staging.data_ptr() + (-staging.data_ptr()) % 256
+    st = states[0]
+    stream = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    n_pos = B * Lt
+    h2d = h_logits.numel() * h_logits.element_size() + n_pos * (4 + 1) + B * 8 + B * 8 + n_pos * (4 * 4 + 4 + 4 + 1 + 4)
+    d2h = n_pos * (4 + 1) + n_pos * (4 * 4 + 4 + 4 + 1 + 4) + B * (4 + 1 + 4 + 4 + 4)
+
+    def one():
+        h["mask"].fill_(1)
+        rc = L.fork_step_host(C.byref(a), C.c_void_p(sp), nbytes, C.c_void_p(st.ws_ptr), st.ws_bytes, stream)
+        if rc != 0:
+            raise RuntimeError("fork_step_host: " + pkg.fork_status_string(rc))
+    for _ in range(max(1, min(warmup, 3))):
+        one()
+    n = max(1, min(steps, 20))
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(n):
+        one()                         # synchronises the stream itself: wall clock spans copies + kernels
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    assert int(h["n_unmasked"].sum()) > 0
+    return dict(ms_per_step=dt * 1e3 / n, steps=n, h2d=int(h2d), d2h=int(d2h))
+
+
+def time_logprob(device, peak):
+    """ForkGRPO scoring shape: B=128 fp32, ~20% of positions selected (one call)."""
+    import torch
+    import fork_synth as fs
+    import paper_2609_39859_b200 as pkg
+    w = fs.workload("grpo")
+    cfg = w.cfg()
+    tokens, select = fs.scoring_inputs(w, cfg)
+    t = torch.empty((w.B, w.Lt, w.V), dtype=torch.float32, device=device)
+    sel_d = torch.from_numpy(select).to(device)
+    tok_d = torch.from_numpy(tokens).to(device)
+    fs.cuda_fill(cfg, 0, sel_d.data_ptr(), None, None, t.data_ptr(), w.Lt * w.V, w.V, 0, w.Lt,
+                 stream_ptr=torch.cuda.current_stream().cuda_stream)
+    st = pkg.ForkState(w.B, w.Lt, device=device)
+    for _ in range(3):
+        pkg.fork_logprob(t, tok_d, sel_d, st)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n = 5
+    e0.record()
+    for _ in range(n):
+        pkg.fork_logprob(t, tok_d, sel_d, st)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / n
+    rows = int(select.sum())
+    gbs = rows * w.V * 4 / (ms * 1e-3) / 1e9
+    del t
+    torch.cuda.empty_cache()
+    return {"workload": "grpo: fork_logprob B=128 Lt=256 V=126464 f32, %d selected rows (3.3 GB >> L2)" % rows,
+            "positions_per_s": rows / (ms * 1e-3), "ms": ms, "hbm_gbs": gbs, "frac_of_measured_peak": gbs / peak}
+
+
+def cpu_baseline(w, seed, target_cpu_seconds=12.0):
+    """The oracle, as it stands, on one full-block step's rows generated on the host."""
+    import fork_synth as fs
+    import oracle
+    cfg = w.cfg()
+    cfg.seed = seed
+    B, BL, V = w.B, w.block_len, w.V
+    logits = np.empty((B, BL, V), w.np_dtype)
+    mask = np.ones((B, w.Lt), np.uint8)
+    lo, hi = np.zeros(B, np.int32), np.full(B, BL, np.int32)
+    fs.fill_host(cfg, 0, mask, lo, hi, logits)
+    rows = B * BL
+    cores = oracle.threads_used(0, rows)
+    st = oracle.StepState(B, w.Lt)
+    t0 = time.perf_counter()
+    oracle.step(st, logits, lo, hi, w.threshold)
+    one = time.perf_counter() - t0
+    reps = int(max(1, min(40, target_cpu_seconds / max(one * cores, 1e-6))))
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        st = oracle.StepState(B, w.Lt)
+        oracle.step(st, logits, lo, hi, w.threshold)
+    dt = time.perf_counter() - t0
+    return {"value": rows * reps / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "%d full-block steps of workload %s (%d rows each, V=%d) on host-generated logits" %
+                      (reps, w.name, rows, V)}
+
+
+def reference_arm(args):
+    """--impl reference: the fp64 oracle is the timed arm (host cores, rank 0 only)."""
+    rank, _, world = rank_info()
+    if rank != 0:
+        return 0
+    import fork_synth as fs
+    import oracle
+    w = fs.workload(args.workload)
+    cfg = w.cfg()
+    B, BL, V = w.B, w.block_len, w.V
+    logits = np.empty((B, BL, V), w.np_dtype)
+    mask = np.ones((B, w.Lt), np.uint8)
+    lo, hi = np.zeros(B, np.int32), np.full(B, BL, np.int32)
+    fs.fill_host(cfg, 0, mask, lo, hi, logits)
+    rows = B * BL
+    cores = oracle.threads_used(0, rows)
+    steps = max(1, min(args.steps, 40))
+    warm = max(1, min(args.warmup, 3))
+    for _ in range(warm):
+        oracle.step(oracle.StepState(B, w.Lt), logits, lo, hi, w.threshold)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle.step(oracle.StepState(B, w.Lt), logits, lo, hi, w.threshold)
+    dt = time.perf_counter() - t0
+    value = rows * steps / dt
+    sample = "%d full-block steps (%d rows each) of workload %s on the host cores" % (steps, rows, w.name)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": warm, "ms_per_step": dt * 1e3 / steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w, rows),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+    return 0
+
+
+def workload_config(w, rows):
+    return {"workload": "%s: B=%d, block %d of Lt=%d, V=%d %s logits, threshold %.2f, all %d block positions live "
+                        "(full-block fork_step)" % (w.name, w.B, w.block_len, w.Lt, w.V,
+                                                     "bf16" if w.es == 2 else "f32", w.threshold, rows),
+            "B": w.B, "block_len": w.block_len, "gen_len": w.Lt, "V": w.V,
+            "logits_dtype": "bf16" if w.es == 2 else "f32", "live_rows_per_step": rows,
+            "bytes_per_row": w.V * w.es}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="own", choices=["own", "reference"])
+    ap.add_argument("--workload", default="b8", choices=["b8", "passk", "sweep"])
+    ap.add_argument("--no-extras", action="store_true", help="skip the other shapes, e2e and the CPU baseline")
+    ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of one CUDA graph")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return reference_arm(args)
+
+    import torch
+    import torch.distributed as dist
+    import fork_synth as fs
+    import paper_2609_39859_b200 as pkg
+    rank, local_rank, world = rank_info()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA library is the only implementation of the path")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    steps, warmup = max(1, args.steps), max(3, args.warmup)
+    w = fs.workload(args.workload)
+    seed = shard_seed(w.seed, rank)
+    peak, peak_src = measured_peak()
+    fs.cuda_init()
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    r = time_full_block(w, seed, steps, warmup, device, use_graph=not args.no_graph)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    max_ms = max_over_ranks(r["total_ms"], device)
+    # keep the same load running so that nvidia-smi (100 ms period) samples clocks under it
+    t_end = time.time() + 1.5
+    while time.time() < t_end:
+        time_full_block_again(r, w, pkg)
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if sampler else None
+
+    rows, row_bytes = r["rows"], r["row_bytes"]
+    value = aggregate(rows, steps, world, max_ms)
+    step_gbs = rows * row_bytes / (r["ms_per_step"] * 1e-3) / 1e9
+    kern_gbs = rows * row_bytes / (r["kernel_ms"] * 1e-3) / 1e9
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": max_ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": dict(workload_config(w, rows),
+                       l2="inputs rotate over %d logits buffers (%.0f MB in total, > 2x the 126 MB L2)" %
+                          (r["n_buf"], r["n_buf"] * rows * row_bytes / 1e6)),
+        "launch": ("one CUDA graph of the K steps" if r["graph"] else "plain stream launches"),
+        "hbm_gbs_per_gpu": step_gbs, "frac_of_8TBs_nominal": step_gbs / NOMINAL_HBM_GBS,
+        "gpu_launches": int(r["launches"]),
+        "roofline": {"bound": "hbm", "kernel": "reduce_select_kernel<bf16,step>" if w.es == 2 else "reduce_select_kernel<f32,step>",
+                     "achieved": kern_gbs, "peak": peak, "unit": "GB/s", "frac": kern_gbs / peak,
+                     "peak_source": peak_src, "traffic": None,
+                     "algorithmic_bytes_per_launch": rows * row_bytes, "kernel_ms": r["kernel_ms"],
+                     "whole_step_gbs": step_gbs, "whole_step_frac": step_gbs / peak,
+                     "frac_of_8TBs_nominal": kern_gbs / NOMINAL_HBM_GBS},
+        "clocks": clocks,
+    }
+    if rank == 0 and not args.no_extras:
+        e = time_e2e(w, r["setup"], steps, warmup, device)
+        out["e2e"] = {"value": rows * world / (e["ms_per_step"] * 1e-3), "unit": UNIT,
+                      "h2d_bytes_per_step": e["h2d"], "d2h_bytes_per_step": e["d2h"], "ms_per_step": e["ms_per_step"],
+                      "steps": e["steps"], "api": "fork_step_host (pinned host buffers, copies inside the timed region)"}
+    r.pop("setup", None)
+    r.pop("keep", None)
+    torch.cuda.empty_cache()
+    if rank == 0 and not args.no_extras and world == 1:
+        also = []
+        for name in ("b8", "passk", "sweep"):
+            if name == args.workload:
+                continue
+            w2 = fs.workload(name)
+            r2 = time_full_block(w2, w2.seed, min(steps, 50), 5, device)
+            r2.pop("setup", None)
+            r2.pop("keep", None)
+            torch.cuda.empty_cache()
+            g2 = r2["rows"] * r2["row_bytes"] / (r2["kernel_ms"] * 1e-3) / 1e9
+            s2 = r2["rows"] * r2["row_bytes"] / (r2["ms_per_step"] * 1e-3) / 1e9
+            also.append({"workload": workload_config(w2, r2["rows"])["workload"],
+                         "positions_per_s": r2["rows"] / (r2["ms_per_step"] * 1e-3), "ms_per_step": r2["ms_per_step"],
+                         "whole_step_gbs": s2, "whole_step_frac_of_measured_peak": s2 / peak,
+                         "kernel_gbs": g2, "kernel_frac_of_measured_peak": g2 / peak,
+                         "kernel_frac_of_8TBs_nominal": g2 / NOMINAL_HBM_GBS})
+        also.append(time_logprob(device, peak))
+        out["also"] = also
+        out["cpu_baseline"] = cpu_baseline(w, seed)
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+def time_full_block_again(r, w, pkg):
+    """Untimed repeat of the benchmark's own steps (keeps the GPU under the same load)."""
+    import torch
+    cfg, bufs, states, lo, hi = r["setup"]
+    n = len(states)
+    reset_states(states)
+    for j in range(n):
+        pkg.fork_step(states[j], bufs[j % len(bufs)], lo, hi, w.threshold)
+    torch.cuda.synchronize()
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -111,11 +111,64 @@ def cuda():
         L.fork_synth_provider_destroy.argtypes = [C.c_void_p]
         L.fork_synth_provider_calls.restype = C.c_int64
         L.fork_synth_provider_calls.argtypes = [C.c_void_p]
+        L.fork_synth_provider_fail_at.restype = None
+        L.fork_synth_provider_fail_at.argtypes = [C.c_void_p, C.c_int32]
         tm, tt = C.c_void_p(), C.c_void_p()
         cpu().fork_synth_tables(C.byref(tm), C.byref(tt))
         L._tables = (tm, tt)
         _cuda = L
     return _cuda
+
+
+def provider_address() -> int:
+    """Address of the C callback `fork_synth_provider` (has the decode loop's fork_logits_fn signature)."""
+    return C.cast(cuda().fork_synth_provider, C.c_void_p).value
+
+
+class Provider:
+    """Owns a generator context for the decode loop: `address` + `ctx` go to fork_decode_loop."""
+
+    def __init__(self, cfg: Cfg, stride_b: int, stride_l: int, pos0: int, Ll: int, nonce=None):
+        L = cuda_init()
+        arr = None if nonce is None else np.ascontiguousarray(nonce, np.uint32)
+        self._L = L
+        self.ctx = L.fork_synth_provider_create(C.byref(cfg), stride_b, stride_l, pos0, Ll,
+                                                None if arr is None else arr.ctypes.data,
+                                                0 if arr is None else len(arr))
+        self.address = provider_address()
+
+    @property
+    def calls(self) -> int:
+        return int(self._L.fork_synth_provider_calls(self.ctx))
+
+    def fail_at(self, step: int):
+        self._L.fork_synth_provider_fail_at(self.ctx, step)
+
+    def close(self):
+        if self.ctx:
+            self._L.fork_synth_provider_destroy(self.ctx)
+            self.ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def cuda_fill(cfg: Cfg, step: int, mask_ptr: int, lo_ptr, hi_ptr, logits_ptr: int, stride_b: int, stride_l: int,
+              pos0: int, Ll: int, stream_ptr: int = 0, nonce: int = 0):
+    """Enqueue the fill of every live row of a device logits buffer (raw device pointers)."""
+    rc = cuda_init().fork_synth_cuda_fill(C.byref(cfg), nonce, step, mask_ptr, lo_ptr, hi_ptr, logits_ptr,
+                                          stride_b, stride_l, pos0, Ll, stream_ptr)
+    if rc != 0:
+        raise RuntimeError("fork_synth_cuda_fill: CUDA error %d" % rc)
+
+
+def cuda_canary(logits_ptr: int, n_elems: int, dtype: int, stream_ptr: int = 0):
+    rc = cuda().fork_synth_cuda_canary(logits_ptr, n_elems, dtype, stream_ptr)
+    if rc != 0:
+        raise RuntimeError("fork_synth_cuda_canary: CUDA error %d" % rc)
 
 
 def cuda_init():

@@ -1,0 +1,188 @@
+/*
+ * fork_dllm.h — C ABI of the Fork-dLLM confidence pass for NVIDIA B200 (sm_100a).
+ *
+ * One sampling step of a masked diffusion language model, as Fork-dLLM defines it
+ * (Algorithm 2 of the paper; Section 2, "Sampling in masked dLLMs"):
+ *   M_t   = still-masked positions (here: mask[b,k] != 0 inside the sequence's active block),
+ *   x_0^k = candidate token at temperature 0 = arg-max of the position's distribution,
+ *   c_t^k = q_theta^k(x_0^k | x_t) = largest softmax probability of the position's logits,
+ *   U_t   = {k in M_t : c_t^k > lambda}; if U_t is empty, U_t = {leftmost(M_t)}   (the Fork fallback),
+ *   x_{t-1}^k = x_0^k for k in U_t.
+ * Besides the commit, the step emits per position the confidence, candidate, token entropy
+ * (Section 3.1) and log-probability, and per sequence whether the step was a fallback step
+ * (the set F_i of Section 3.2), which is what ForkGRPO scores.
+ *
+ * Conventions for every entry point
+ *   - All data pointers are DEVICE pointers owned by the caller unless a comment says "host".
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  fork_step and
+ *     fork_logprob only enqueue work on it and return; results are in device memory once the
+ *     stream reaches that point.  They never synchronise, allocate or free.
+ *   - `workspace` is device scratch of at least fork_workspace_bytes(B, Lt) bytes, 256-byte
+ *     aligned, private to one call at a time on one stream; its contents need not be kept
+ *     between calls (fork_decode_loop keeps its block cursors there while it runs).
+ *   - Argument errors are found on the host before anything is launched and return
+ *     FORK_ERR_INVALID_ARG / FORK_ERR_WORKSPACE; a failed launch returns FORK_ERR_CUDA.
+ *   - Logits rows are contiguous in V.  Row (b,k) starts at element
+ *       b*stride_b + (k - pos0)*stride_l
+ *     of `logits`; the buffer covers positions pos0 .. pos0+Ll-1 (pos0 = 0 and Ll = Lt for a
+ *     full [B,Lt,V] tensor, or one block's window).  Rows that are not live are never read, so
+ *     they may hold anything.  The fast path needs the base pointer and both strides to be
+ *     multiples of 16 bytes; otherwise a slower scalar path runs (same results).
+ *   - Vocabulary ties go to the lowest index.  A logit of -inf has probability 0.  A row that
+ *     holds NaN or +inf, or only -inf, gets FORK_ROW_NONFINITE in row_status, confidence 0,
+ *     NaN entropy / log-probability, and as candidate the lowest index of the maximum over
+ *     its non-NaN entries (0 if it has none).
+ */
+#ifndef FORK_DLLM_H
+#define FORK_DLLM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum fork_status {
+  FORK_OK = 0,
+  FORK_ERR_INVALID_ARG = -1,
+  FORK_ERR_CUDA = -2,
+  FORK_ERR_WORKSPACE = -3,
+  FORK_ERR_MAX_STEPS = -4,
+  FORK_ERR_PROVIDER = -5
+} fork_status;
+
+typedef enum fork_dtype { FORK_BF16 = 0, FORK_F32 = 1 } fork_dtype;
+
+/* bits of row_status[b,k] */
+#define FORK_ROW_NONFINITE 1u /* NaN or +inf in the row, or nothing but -inf */
+#define FORK_ROW_BAD_TOKEN 2u /* fork_logprob: token id outside [0,V) */
+
+/* bits of the device status word (fork_device_status) */
+#define FORK_DEV_WINDOW_CLAMPED 1u /* a block [lo,hi) reached outside [pos0,pos0+Ll) or [0,Lt) and was clipped */
+
+/*
+ * Arguments of one sampling step (Algorithm 2; inputs x_t, q_theta, lambda -> x_{t-1}).
+ * Output pointers marked "optional" may be NULL.
+ */
+typedef struct fork_step_args {
+  const void* logits;        /* model output q_theta(.|x_t) as logits; see the layout rule above */
+  int64_t stride_b, stride_l;/* in elements; stride_l >= V */
+  int32_t pos0;              /* sequence position of logits row 0 */
+  int32_t B, Lt, Ll, V;      /* sequences, sequence-buffer length, logits rows per sequence, vocabulary */
+  int32_t dtype;             /* fork_dtype of the logits */
+  int32_t* tokens;           /* [B,Lt] in/out: x_t -> x_{t-1}; written only at committed positions */
+  uint8_t* mask;             /* [B,Lt] in/out: 1 = still [MASK]; cleared at committed positions */
+  const int32_t* blk_lo;     /* [B] active block, half open [lo,hi), absolute positions; */
+  const int32_t* blk_hi;     /*     lo == hi means the sequence takes no part in this step */
+  float threshold;           /* lambda; commit iff confidence > lambda (strict) */
+  int32_t step;              /* id written into commit_step */
+  /* per position, written for every live position (masked and inside the block); all optional */
+  float* conf;               /* [B,Lt] c_t^k */
+  int32_t* cand;             /* [B,Lt] x_0^k */
+  float* entropy;            /* [B,Lt] token entropy of q_theta^k in nats */
+  float* logp;               /* [B,Lt] log q_theta^k(x_0^k | x_t) = ln conf */
+  uint32_t* row_status;      /* [B,Lt] FORK_ROW_* bits */
+  /* per position, written only at positions committed by this step; all optional.
+     (conf/entropy/logp are last written at the step that commits the position, so after a
+     decode loop they hold the values at commit time.) */
+  int32_t* commit_step;      /* [B,Lt] */
+  uint8_t* commit_fallback;  /* [B,Lt] 1 if committed by the leftmost fallback (a step in F_i) */
+  float* commit_logp;        /* [B,Lt] log-probability of the committed token (old-policy term of the ForkGRPO ratio) */
+  /* per sequence; all optional */
+  int32_t* n_unmasked;       /* [B] |U_t| (0 if the sequence had no live position) */
+  uint8_t* is_fallback;      /* [B] 1 if U_t was empty and the leftmost position was taken */
+  int32_t* fallback_pos;     /* [B] that position, else -1 */
+  int32_t* nfe;              /* [B] += 1 if the sequence had a live position (model evaluations used) */
+  int32_t* n_fallback;       /* [B] += is_fallback */
+} fork_step_args;
+
+/*
+ * Arguments of the log-likelihood scoring used by ForkGRPO (Section 3.2): for every selected
+ * position (select[b,k] != 0, normally the fallback steps' positions k_{i,t}) the log-probability
+ * of the given token under the given logits, log q_theta^k(x^k | .) = x_tok - max - ln sum exp.
+ */
+typedef struct fork_logprob_args {
+  const void* logits; int64_t stride_b, stride_l; int32_t pos0;
+  int32_t B, Lt, Ll, V; int32_t dtype;
+  const int32_t* tokens;     /* [B,Lt] token whose likelihood is wanted */
+  const uint8_t* select;     /* [B,Lt] */
+  float* logp;               /* [B,Lt] out: log-probability where selected, 0 elsewhere */
+  float* seq_sum;            /* [B] out, optional: sum of logp over the sequence's selected positions */
+  int32_t* seq_cnt;          /* [B] out, optional: number of selected positions (|F_i|) */
+  uint32_t* row_status;      /* [B,Lt] out, optional: FORK_ROW_* bits at selected positions.
+                                A token outside [0,V) sets FORK_ROW_BAD_TOKEN and scores 0. */
+} fork_logprob_args;
+
+/* Device scratch needed by any entry point for a batch of B sequences of buffer length Lt. */
+size_t fork_workspace_bytes(int32_t B, int32_t Lt);
+
+/* One sampling step (Algorithm 2) for all B sequences.  Asynchronous on `stream`. */
+fork_status fork_step(const fork_step_args* args, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Log-likelihood of given tokens at selected positions (Section 3.2).  Asynchronous on `stream`. */
+fork_status fork_logprob(const fork_logprob_args* args, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Model-forward callback of the decode loop: must enqueue on `stream` the work that fills
+ * `logits_out` (the buffer given as proto->logits) for the live positions of step `step`,
+ * given the current device-side tokens / mask / block cursors.  Returns 0 on success.
+ * One call = one model evaluation (NFE, Section 4.1).
+ */
+typedef int (*fork_logits_fn)(void* ctx, int32_t step, const int32_t* tokens, const uint8_t* mask,
+                              const int32_t* blk_lo, const int32_t* blk_hi, void* logits_out, void* stream);
+
+/*
+ * Semi-autoregressive decoding (Section 2: repeat sampling steps until nothing is masked;
+ * Section 4.1: blocks of block_len inside the generation window [gen_lo,gen_hi)).
+ * Every sequence keeps its own block cursor: the first block that still holds a masked
+ * position.  Each iteration calls provider once, runs fork_step on every unfinished sequence's
+ * block (step ids proto->step, proto->step+1, ...), advances the cursors and reads one int back
+ * to the host to test for termination (one stream synchronisation per step).
+ * proto->blk_lo / blk_hi are ignored.  *steps_taken (host) receives the number of provider
+ * calls.  Returns FORK_ERR_MAX_STEPS if masked positions remain after max_steps steps, and
+ * FORK_ERR_PROVIDER if the callback fails; device state then reflects the steps completed.
+ */
+fork_status fork_decode_loop(const fork_step_args* proto, int32_t block_len, int32_t gen_lo, int32_t gen_hi,
+                             fork_logits_fn provider, void* ctx, int32_t max_steps, int32_t* steps_taken,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * fork_step for callers whose buffers live in HOST memory (pinned memory recommended): every
+ * pointer in `host_args` is a host pointer.  The call copies the logits window, tokens, mask
+ * and block bounds into `staging` (device, at least fork_staging_bytes(host_args) bytes), runs
+ * fork_step, copies every non-NULL output back and synchronises `stream` before returning.
+ */
+size_t fork_staging_bytes(const fork_step_args* host_args);
+fork_status fork_step_host(const fork_step_args* host_args, void* staging, size_t staging_bytes,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+/* Copies the device status word of the last call that used `workspace` to *host_out
+   (FORK_DEV_* bits) and synchronises `stream`. */
+fork_status fork_device_status(const void* workspace, uint32_t* host_out, void* stream);
+
+/* Human-readable name of a status code. */
+const char* fork_status_string(int status);
+
+/*
+ * Tuning knobs (process wide; intended for benchmarking).  Keys:
+ *   FORK_TUNE_VARIANT       0 = automatic, 1 = direct vector loads, 2 = bulk-copy shared-memory ring
+ *   FORK_TUNE_CTAS_PER_SM   0 = automatic, else resident CTAs per SM used to size the grid
+ *   FORK_TUNE_PDL           1 = chain the two kernels of a step with programmatic dependent launch
+ * Returns the previous value, or -1 for an unknown key.
+ */
+enum { FORK_TUNE_VARIANT = 0, FORK_TUNE_CTAS_PER_SM = 1, FORK_TUNE_PDL = 2, FORK_TUNE_COUNT_ = 3 };
+int32_t fork_set_tuning(int32_t key, int32_t value);
+
+/* Profiling hook: the next fork_step / fork_logprob call made by this host thread records the two
+   CUDA events (cudaEvent_t passed as void*) on its stream immediately before and after its
+   streaming kernel (not around the active-set kernel), then forgets them. */
+void fork_set_timing_events(void* start, void* stop);
+
+/* Number of kernels this library has launched since it was loaded (all entry points). */
+int64_t fork_kernel_launches(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FORK_DLLM_H */

@@ -1,0 +1,257 @@
+"""Thin ctypes binding of libfork_dllm.so: argument marshalling only.
+
+Every function here has the name and the meaning of the C entry point it forwards to
+(see include/fork_dllm.h); all computation happens in the CUDA kernels behind them.  PyTorch is
+used for device memory and streams.  There is no CPU fallback: if the library cannot be loaded
+the import fails.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+from . import _build
+
+FORK_OK, FORK_ERR_INVALID_ARG, FORK_ERR_CUDA, FORK_ERR_WORKSPACE, FORK_ERR_MAX_STEPS, FORK_ERR_PROVIDER = \
+    0, -1, -2, -3, -4, -5
+FORK_BF16, FORK_F32 = 0, 1
+FORK_ROW_NONFINITE, FORK_ROW_BAD_TOKEN = 1, 2
+FORK_DEV_WINDOW_CLAMPED = 1
+FORK_TUNE_VARIANT, FORK_TUNE_CTAS_PER_SM, FORK_TUNE_PDL = 0, 1, 2
+
+
+class fork_step_args(C.Structure):
+    _fields_ = [
+        ("logits", C.c_void_p), ("stride_b", C.c_int64), ("stride_l", C.c_int64), ("pos0", C.c_int32),
+        ("B", C.c_int32), ("Lt", C.c_int32), ("Ll", C.c_int32), ("V", C.c_int32), ("dtype", C.c_int32),
+        ("tokens", C.c_void_p), ("mask", C.c_void_p), ("blk_lo", C.c_void_p), ("blk_hi", C.c_void_p),
+        ("threshold", C.c_float), ("step", C.c_int32),
+        ("conf", C.c_void_p), ("cand", C.c_void_p), ("entropy", C.c_void_p), ("logp", C.c_void_p),
+        ("row_status", C.c_void_p),
+        ("commit_step", C.c_void_p), ("commit_fallback", C.c_void_p), ("commit_logp", C.c_void_p),
+        ("n_unmasked", C.c_void_p), ("is_fallback", C.c_void_p), ("fallback_pos", C.c_void_p),
+        ("nfe", C.c_void_p), ("n_fallback", C.c_void_p),
+    ]
+
+
+class fork_logprob_args(C.Structure):
+    _fields_ = [
+        ("logits", C.c_void_p), ("stride_b", C.c_int64), ("stride_l", C.c_int64), ("pos0", C.c_int32),
+        ("B", C.c_int32), ("Lt", C.c_int32), ("Ll", C.c_int32), ("V", C.c_int32), ("dtype", C.c_int32),
+        ("tokens", C.c_void_p), ("select", C.c_void_p), ("logp", C.c_void_p), ("seq_sum", C.c_void_p),
+        ("seq_cnt", C.c_void_p), ("row_status", C.c_void_p),
+    ]
+
+
+fork_logits_fn = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                             C.c_void_p, C.c_void_p)
+
+EXPORTS = ("fork_workspace_bytes", "fork_step", "fork_logprob", "fork_decode_loop", "fork_staging_bytes",
+           "fork_step_host", "fork_device_status", "fork_status_string", "fork_set_tuning",
+           "fork_kernel_launches", "fork_set_timing_events")
+
+_lib = None
+
+
+def lib():
+    """Load (building first if the shared object is missing or stale) the C-ABI library."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    try:
+        path = _build.build()
+    except Exception as e:  # no silent fallback: the CUDA library IS the product
+        if not os.path.exists(_build.LIB):
+            raise ImportError("libfork_dllm.so is missing and could not be built with nvcc: %r" % (e,)) from e
+        path = _build.LIB
+    L = C.CDLL(path)
+    L.fork_workspace_bytes.restype = C.c_size_t
+    L.fork_workspace_bytes.argtypes = [C.c_int32, C.c_int32]
+    L.fork_step.restype = C.c_int
+    L.fork_step.argtypes = [C.POINTER(fork_step_args), C.c_void_p, C.c_size_t, C.c_void_p]
+    L.fork_logprob.restype = C.c_int
+    L.fork_logprob.argtypes = [C.POINTER(fork_logprob_args), C.c_void_p, C.c_size_t, C.c_void_p]
+    L.fork_decode_loop.restype = C.c_int
+    L.fork_decode_loop.argtypes = [C.POINTER(fork_step_args), C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
+                                   C.c_void_p, C.c_int32, C.POINTER(C.c_int32), C.c_void_p, C.c_size_t, C.c_void_p]
+    L.fork_staging_bytes.restype = C.c_size_t
+    L.fork_staging_bytes.argtypes = [C.POINTER(fork_step_args)]
+    L.fork_step_host.restype = C.c_int
+    L.fork_step_host.argtypes = [C.POINTER(fork_step_args), C.c_void_p, C.c_size_t, C.c_void_p, C.c_size_t, C.c_void_p]
+    L.fork_device_status.restype = C.c_int
+    L.fork_device_status.argtypes = [C.c_void_p, C.POINTER(C.c_uint32), C.c_void_p]
+    L.fork_status_string.restype = C.c_char_p
+    L.fork_status_string.argtypes = [C.c_int]
+    L.fork_set_tuning.restype = C.c_int32
+    L.fork_set_tuning.argtypes = [C.c_int32, C.c_int32]
+    L.fork_kernel_launches.restype = C.c_int64
+    L.fork_kernel_launches.argtypes = []
+    L.fork_set_timing_events.restype = None
+    L.fork_set_timing_events.argtypes = [C.c_void_p, C.c_void_p]
+    _lib = L
+    return L
+
+
+class ForkError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: %s" % (where, fork_status_string(status)))
+
+
+def fork_status_string(status: int) -> str:
+    return lib().fork_status_string(int(status)).decode()
+
+
+def fork_workspace_bytes(B: int, Lt: int) -> int:
+    return int(lib().fork_workspace_bytes(B, Lt))
+
+
+def fork_set_tuning(key: int, value: int) -> int:
+    return int(lib().fork_set_tuning(key, value))
+
+
+def fork_kernel_launches() -> int:
+    return int(lib().fork_kernel_launches())
+
+
+def _p(t):
+    return None if t is None else t.data_ptr()
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return FORK_BF16
+    if t.dtype == torch.float32:
+        return FORK_F32
+    raise TypeError("logits must be bfloat16 or float32, got %s" % t.dtype)
+
+
+class ForkState:
+    """Device buffers of one batch: the sequence and its mask, every output of fork_step, and the
+    scratch workspace.  Plain tensors; nothing here computes."""
+
+    PER_POS = (("conf", torch.float32, float("nan")), ("cand", torch.int32, -1),
+               ("entropy", torch.float32, float("nan")), ("logp", torch.float32, float("nan")),
+               ("row_status", torch.int32, 0), ("commit_step", torch.int32, -1),
+               ("commit_fallback", torch.uint8, 255), ("commit_logp", torch.float32, float("nan")))
+    PER_SEQ = (("n_unmasked", torch.int32, 0), ("is_fallback", torch.uint8, 0), ("fallback_pos", torch.int32, -1),
+               ("nfe", torch.int32, 0), ("n_fallback", torch.int32, 0))
+
+    def __init__(self, B: int, Lt: int, device="cuda", tokens=None, mask=None):
+        self.B, self.Lt, self.device = B, Lt, torch.device(device)
+        dev = self.device
+        self.tokens = (torch.zeros((B, Lt), dtype=torch.int32, device=dev) if tokens is None
+                       else torch.as_tensor(tokens, dtype=torch.int32).to(dev).contiguous().clone())
+        self.mask = (torch.ones((B, Lt), dtype=torch.uint8, device=dev) if mask is None
+                     else torch.as_tensor(mask, dtype=torch.uint8).to(dev).contiguous().clone())
+        for name, dt, fill in self.PER_POS:
+            setattr(self, name, torch.full((B, Lt), fill, dtype=dt, device=dev))
+        for name, dt, fill in self.PER_SEQ:
+            setattr(self, name, torch.full((B,), fill, dtype=dt, device=dev))
+        nbytes = fork_workspace_bytes(B, Lt)
+        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=dev)
+        off = (-self.workspace.data_ptr()) % 256
+        self.ws_ptr, self.ws_bytes = self.workspace.data_ptr() + off, nbytes
+
+    def host(self) -> dict:
+        names = ["tokens", "mask"] + [n for n, _, _ in self.PER_POS] + [n for n, _, _ in self.PER_SEQ]
+        return {n: getattr(self, n).cpu().numpy() for n in names}
+
+
+def make_step_args(st: ForkState, logits: torch.Tensor, blk_lo, blk_hi, threshold: float, step: int = 0,
+                   pos0: int = 0) -> fork_step_args:
+    assert logits.dim() == 3 and logits.stride(2) == 1, "logits must be [B, Ll, V] with V contiguous"
+    B, Ll, V = logits.shape
+    assert B == st.B
+    a = fork_step_args()
+    a.logits = logits.data_ptr()
+    a.stride_b, a.stride_l, a.pos0 = logits.stride(0), logits.stride(1), pos0
+    a.B, a.Lt, a.Ll, a.V, a.dtype = B, st.Lt, Ll, V, _dtype_code(logits)
+    a.tokens, a.mask = st.tokens.data_ptr(), st.mask.data_ptr()
+    a.blk_lo, a.blk_hi = _p(blk_lo), _p(blk_hi)
+    a.threshold, a.step = float(threshold), int(step)
+    for name, _, _ in ForkState.PER_POS + ForkState.PER_SEQ:
+        setattr(a, name, getattr(st, name).data_ptr())
+    return a
+
+
+def fork_step(st: ForkState, logits: torch.Tensor, blk_lo: torch.Tensor, blk_hi: torch.Tensor, threshold: float,
+              step: int = 0, pos0: int = 0, stream=None) -> None:
+    """One Fork-dLLM sampling step on device buffers (asynchronous on the stream)."""
+    a = make_step_args(st, logits, blk_lo, blk_hi, threshold, step, pos0)
+    rc = lib().fork_step(C.byref(a), C.c_void_p(st.ws_ptr), st.ws_bytes, _stream_ptr(stream))
+    if rc != FORK_OK:
+        raise ForkError(rc, "fork_step")
+
+
+def fork_logprob(logits: torch.Tensor, tokens: torch.Tensor, select: torch.Tensor, st: ForkState, pos0: int = 0,
+                 stream=None):
+    """Log-likelihood of `tokens` at the selected positions; returns (logp [B,Lt], seq_sum [B],
+    seq_cnt [B], row_status [B,Lt]) as device tensors (asynchronous on the stream)."""
+    assert logits.dim() == 3 and logits.stride(2) == 1
+    B, Ll, V = logits.shape
+    Lt = tokens.shape[1]
+    dev = logits.device
+    logp = torch.empty((B, Lt), dtype=torch.float32, device=dev)
+    seq_sum = torch.empty((B,), dtype=torch.float32, device=dev)
+    seq_cnt = torch.empty((B,), dtype=torch.int32, device=dev)
+    status = torch.zeros((B, Lt), dtype=torch.int32, device=dev)
+    a = fork_logprob_args()
+    a.logits = logits.data_ptr()
+    a.stride_b, a.stride_l, a.pos0 = logits.stride(0), logits.stride(1), pos0
+    a.B, a.Lt, a.Ll, a.V, a.dtype = B, Lt, Ll, V, _dtype_code(logits)
+    assert tokens.dtype == torch.int32 and select.dtype == torch.uint8 and tokens.is_contiguous() and select.is_contiguous()
+    a.tokens, a.select = tokens.data_ptr(), select.data_ptr()
+    a.logp, a.seq_sum, a.seq_cnt, a.row_status = logp.data_ptr(), seq_sum.data_ptr(), seq_cnt.data_ptr(), status.data_ptr()
+    rc = lib().fork_logprob(C.byref(a), C.c_void_p(st.ws_ptr), st.ws_bytes, _stream_ptr(stream))
+    if rc != FORK_OK:
+        raise ForkError(rc, "fork_logprob")
+    return logp, seq_sum, seq_cnt, status
+
+
+def fork_decode_loop(st: ForkState, logits: torch.Tensor, block_len: int, gen_lo: int, gen_hi: int, provider,
+                     ctx, threshold: float, max_steps: int, step0: int = 0, pos0: int = 0, stream=None,
+                     raise_on_error: bool = True):
+    """Semi-autoregressive decoding.  `provider` is either a C function pointer (int address or
+    ctypes function) with the fork_logits_fn signature plus its `ctx` pointer, or a Python callable
+    ``provider(step, lo_ptr, hi_ptr, stream_ptr) -> int`` that enqueues the work filling `logits`.
+    Returns (status, steps_taken)."""
+    a = make_step_args(st, logits, None, None, threshold, step0, pos0)
+    keep = None
+    if callable(provider) and not isinstance(provider, (int, C._CFuncPtr)):
+        def _tramp(_ctx, step, _tok, _mask, lo, hi, _out, stream_p):
+            try:
+                return int(provider(int(step), lo, hi, stream_p) or 0)
+            except Exception:
+                import traceback
+                traceback.print_exc()
+                return 1
+        keep = fork_logits_fn(_tramp)
+        fn_ptr = C.cast(keep, C.c_void_p)
+    elif isinstance(provider, int):
+        fn_ptr = C.c_void_p(provider)
+    else:
+        fn_ptr = C.cast(provider, C.c_void_p)
+    steps = C.c_int32(0)
+    rc = lib().fork_decode_loop(C.byref(a), block_len, gen_lo, gen_hi, fn_ptr, C.c_void_p(ctx or 0), max_steps,
+                                C.byref(steps), C.c_void_p(st.ws_ptr), st.ws_bytes, _stream_ptr(stream))
+    del keep
+    if rc != FORK_OK and raise_on_error:
+        raise ForkError(rc, "fork_decode_loop")
+    return int(rc), int(steps.value)
+
+
+def fork_device_status(st: ForkState, stream=None) -> int:
+    out = C.c_uint32(0)
+    rc = lib().fork_device_status(C.c_void_p(st.ws_ptr), C.byref(out), _stream_ptr(stream))
+    if rc != FORK_OK:
+        raise ForkError(rc, "fork_device_status")
+    return int(out.value)

@@ -1,0 +1,93 @@
+"""Shared test plumbing: comparing the CUDA path's buffers with the oracle's, and running the oracle's
+decode loop on generator inputs while keeping every confidence away from the threshold."""
+import copy
+
+import numpy as np
+
+import fork_synth as fs
+import oracle
+
+RTOL, ATOL = 1e-4, 1e-5          # |gpu - oracle| <= ATOL + RTOL * |oracle| for conf, entropy, log-prob
+
+
+def assert_close(name, got, want, where=None):
+    got = np.asarray(got, np.float64)
+    want = np.asarray(want, np.float64)
+    if where is not None:
+        got, want = got[where], want[where]
+    both_nan = np.isnan(got) & np.isnan(want)
+    both_inf = np.isinf(want) & (got == want)
+    ok = both_nan | both_inf | (np.abs(got - want) <= ATOL + RTOL * np.abs(want))
+    if not ok.all():
+        i = np.flatnonzero(~ok.ravel())[:5]
+        raise AssertionError("%s: %d of %d outside tolerance; first got=%s want=%s" %
+                             (name, (~ok).sum(), ok.size, got.ravel()[i], want.ravel()[i]))
+
+
+def assert_equal(name, got, want, where=None):
+    got = np.asarray(got)
+    want = np.asarray(want)
+    if where is not None:
+        got, want = got[where], want[where]
+    if not (got.astype(np.int64) == want.astype(np.int64)).all():
+        bad = np.flatnonzero((got.astype(np.int64) != want.astype(np.int64)).ravel())[:8]
+        raise AssertionError("%s differs at %s: got=%s want=%s" % (name, bad, got.ravel()[bad], want.ravel()[bad]))
+
+
+def compare_step_state(g: dict, o: "oracle.StepState", nseq=None):
+    """Bit-exact integers, floats within tolerance.  `g` is ForkState.host(); compares the first
+    `nseq` sequences (all by default).  Positions never written keep their initial fill on both
+    sides (-1 / 255 / NaN), so whole arrays can be compared."""
+    n = o.B if nseq is None else nseq
+    for name in ("tokens", "mask", "cand", "commit_step", "commit_fallback", "row_status"):
+        assert_equal(name, g[name][:n], getattr(o, name)[:n])
+    for name in ("n_unmasked", "is_fallback", "fallback_pos", "nfe", "n_fallback"):
+        assert_equal(name, g[name][:n], getattr(o, name)[:n])
+    for name in ("conf", "entropy", "logp", "commit_logp"):
+        assert_close(name, g[name][:n], getattr(o, name)[:n])
+
+
+def live_mask(mask, lo, hi):
+    B, Lt = mask.shape
+    k = np.arange(Lt)[None, :]
+    return (mask != 0) & (k >= np.asarray(lo)[:, None]) & (k < np.asarray(hi)[:, None])
+
+
+def oracle_reference_loop(w: "fs.Workload", nseq: int, threshold: float, margin: float = 1e-4,
+                          max_steps: int = 100000, nthreads: int = 0):
+    """The oracle's semi-autoregressive loop on the first `nseq` sequences of workload `w`, with
+    host-generated logits.  At every step the nonce is bumped until no live confidence lies within
+    `margin` of the threshold, so fp32 and fp64 cannot disagree on the unmask decision.
+    Returns (final StepState, per-step nonces, steps taken, per-step live-row counts)."""
+    cfg = w.cfg(B=nseq)
+    st = oracle.StepState(nseq, w.Lt)
+    logits = np.empty((nseq, w.Lt, w.V), w.np_dtype)
+    fs.canary_host(logits)
+    lo, hi = oracle.block_cursors(st.mask, 0, w.Lt, w.block_len)
+    nonces, live_counts = [], []
+    step = 0
+    while (lo < hi).any():
+        assert step < max_steps
+        live = live_mask(st.mask, lo, hi)
+        nonce = 0
+        while True:
+            fs.fill_host(cfg, step, st.mask, lo, hi, logits, nonce=nonce, nthreads=nthreads)
+            trial = copy.deepcopy(st)
+            assert oracle.step(trial, logits, lo, hi, threshold, step_id=step, nthreads=nthreads) == 0
+            if (np.abs(trial.conf[live] - np.float64(np.float32(threshold))) >= margin).all():
+                break
+            nonce += 1
+            assert nonce < 64
+        st = trial
+        nonces.append(nonce)
+        live_counts.append(int(live.sum()))
+        step += 1
+        lo, hi = oracle.block_cursors(st.mask, 0, w.Lt, w.block_len, lo, hi)
+    return st, np.asarray(nonces, np.uint32), step, live_counts
+
+
+def to_torch_logits(arr: np.ndarray, device="cuda"):
+    import torch
+    if arr.dtype == np.uint16:
+        return torch.from_numpy(arr.view(np.int16)).to(device).view(torch.bfloat16)
+    return torch.from_numpy(arr).to(device)

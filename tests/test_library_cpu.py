@@ -1,0 +1,133 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports every symbol the header
+declares, rejects bad arguments before touching CUDA, and its work partition is consistent."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+import paper_2609_39859_b200 as pkg
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "fork_dllm.h")
+
+
+def declared_functions():
+    src = open(HEADER).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    names = set(re.findall(r"\b(fork_[a-z_]+)\s*\(", src))
+    names.discard("fork_logits_fn")
+    return sorted(names)
+
+
+def test_library_exports_every_declared_symbol():
+    L = pkg.lib()
+    names = declared_functions()
+    assert {"fork_step", "fork_logprob", "fork_decode_loop", "fork_workspace_bytes", "fork_step_host"} <= set(names)
+    for n in names:
+        assert hasattr(L, n), n
+    assert set(pkg.binding.EXPORTS) == set(names)
+
+
+def test_status_strings_and_workspace_size():
+    assert pkg.fork_status_string(0) == "FORK_OK"
+    assert pkg.fork_status_string(-4) == "FORK_ERR_MAX_STEPS"
+    assert pkg.fork_status_string(99) == "FORK_UNKNOWN_STATUS"
+    a, b = pkg.fork_workspace_bytes(8, 256), pkg.fork_workspace_bytes(64, 256)
+    assert 0 < a < b and a % 256 == 0
+    assert pkg.fork_workspace_bytes(-1, 256) == 0 and pkg.fork_workspace_bytes(4, 0) == 0
+
+
+def good_step_args():
+    a = pkg.fork_step_args()
+    a.logits = 0x1000
+    a.stride_b, a.stride_l, a.pos0 = 32 * 1024, 1024, 0
+    a.B, a.Lt, a.Ll, a.V, a.dtype = 2, 32, 32, 1024, pkg.FORK_BF16
+    a.tokens, a.mask, a.blk_lo, a.blk_hi = 0x2000, 0x3000, 0x4000, 0x5000
+    a.threshold, a.step = 0.9, 0
+    return a
+
+
+def test_invalid_arguments_are_rejected_on_the_host():
+    """None of these reach a CUDA call (the pointers are fake, and this machine has no GPU)."""
+    L = pkg.lib()
+    ws, nbytes = C.c_void_p(0x100000), pkg.fork_workspace_bytes(2, 32)
+    assert L.fork_step(None, ws, nbytes, None) == pkg.FORK_ERR_INVALID_ARG
+    for field, value in (("logits", None), ("tokens", None), ("mask", None), ("blk_lo", None), ("blk_hi", None),
+                         ("V", 0), ("Lt", 0), ("Ll", 0), ("B", -1), ("dtype", 7), ("stride_l", 100), ("pos0", -1),
+                         ("threshold", float("nan"))):
+        a = good_step_args()
+        setattr(a, field, value)
+        assert L.fork_step(C.byref(a), ws, nbytes, None) == pkg.FORK_ERR_INVALID_ARG, field
+    a = good_step_args()
+    assert L.fork_step(C.byref(a), None, nbytes, None) == pkg.FORK_ERR_WORKSPACE
+    assert L.fork_step(C.byref(a), ws, nbytes - 1, None) == pkg.FORK_ERR_WORKSPACE
+    assert L.fork_step(C.byref(a), C.c_void_p(0x100010), nbytes, None) == pkg.FORK_ERR_WORKSPACE   # not 256-aligned
+    a.B = 0
+    assert L.fork_step(C.byref(a), ws, nbytes, None) == pkg.FORK_OK                                # nothing to do
+    # decode loop
+    steps = C.c_int32(-1)
+    a = good_step_args()
+    assert L.fork_decode_loop(C.byref(a), 32, 0, 32, None, None, 10, C.byref(steps), ws, nbytes, None) == pkg.FORK_ERR_INVALID_ARG
+    fn = C.c_void_p(0x1234)
+    for bl, glo, ghi, ms in ((0, 0, 32, 10), (32, -1, 32, 10), (32, 0, 33, 10), (32, 8, 4, 10), (32, 0, 32, -1)):
+        assert L.fork_decode_loop(C.byref(a), bl, glo, ghi, fn, None, ms, C.byref(steps), ws, nbytes, None) == pkg.FORK_ERR_INVALID_ARG
+    assert steps.value == 0
+    # scoring
+    lp = pkg.fork_logprob_args()
+    assert L.fork_logprob(None, ws, nbytes, None) == pkg.FORK_ERR_INVALID_ARG
+    lp.logits, lp.stride_b, lp.stride_l, lp.B, lp.Lt, lp.Ll, lp.V, lp.dtype = 0x1000, 32 * 1024, 1024, 2, 32, 32, 1024, 1
+    lp.tokens, lp.select, lp.logp = 0x2000, 0x3000, None
+    assert L.fork_logprob(C.byref(lp), ws, nbytes, None) == pkg.FORK_ERR_INVALID_ARG
+    # host entry point
+    a = good_step_args()
+    assert L.fork_staging_bytes(C.byref(a)) > 2 * 32 * 1024 * 2
+    assert L.fork_step_host(C.byref(a), None, 1 << 30, ws, nbytes, None) == pkg.FORK_ERR_WORKSPACE
+    a.stride_b = 32 * 1024 + 8
+    assert L.fork_step_host(C.byref(a), C.c_void_p(0x200000), 1 << 30, ws, nbytes, None) == pkg.FORK_ERR_INVALID_ARG
+    assert L.fork_device_status(None, None, None) == pkg.FORK_ERR_INVALID_ARG
+
+
+def test_tuning_knobs_round_trip():
+    assert pkg.fork_set_tuning(99, 1) == -1
+    old = pkg.fork_set_tuning(pkg.FORK_TUNE_CTAS_PER_SM, 2)
+    assert pkg.fork_set_tuning(pkg.FORK_TUNE_CTAS_PER_SM, old) == 2
+    assert pkg.fork_kernel_launches() >= 0
+
+
+def test_partition_is_a_partition():
+    """Brute force: CTA ranges tile [0,U) in order, the owner formula inverts them, the number of
+    parts per row matches a direct count, and the slot r+g is unique and below R+G."""
+    L = pkg.lib()
+    L.fork_debug_part_begin.restype = C.c_int64
+    L.fork_debug_part_begin.argtypes = [C.c_int64, C.c_int32, C.c_int32]
+    L.fork_debug_part_owner.restype = C.c_int32
+    L.fork_debug_part_owner.argtypes = [C.c_int64, C.c_int32, C.c_int64]
+    L.fork_debug_row_parts.restype = C.c_int32
+    L.fork_debug_row_parts.argtypes = [C.c_int64, C.c_int32, C.c_int32, C.c_int64]
+    assert L.fork_debug_chunk() == 2048
+    L.fork_debug_effective_grid.restype = C.c_int32
+    L.fork_debug_effective_grid.argtypes = [C.c_int64, C.c_int32]
+    for R in (1, 2, 3, 8, 31, 32, 33, 256, 700):
+        for Cc in (1, 2, 5, 62, 75):
+            for G0 in (1, 3, 148, 592, 2048):
+                U = R * Cc
+                G = L.fork_debug_effective_grid(U, G0)
+                assert G == min(G0, U)
+                begins = [L.fork_debug_part_begin(U, G, g) for g in range(G + 1)]
+                assert begins[0] == 0 and begins[-1] == U and all(x <= y for x, y in zip(begins, begins[1:]))
+                assert max(y - x for x, y in zip(begins, begins[1:])) - min(y - x for x, y in zip(begins, begins[1:])) <= 1
+                slots = set()
+                for r in range(R):
+                    owners = sorted({L.fork_debug_part_owner(U, G, u) for u in range(r * Cc, (r + 1) * Cc)})
+                    for u in (r * Cc, (r + 1) * Cc - 1):
+                        g = L.fork_debug_part_owner(U, G, u)
+                        assert begins[g] <= u < begins[g + 1]
+                    assert owners == list(range(owners[0], owners[-1] + 1))
+                    assert L.fork_debug_row_parts(U, G, Cc, r) == len(owners)
+                    for g in owners:
+                        assert (r + g) not in slots and r + g < R + G
+                        slots.add(r + g)
+    # sizes of the real workloads: no overflow in the 64-bit arithmetic
+    U = 32768 * 75
+    assert L.fork_debug_part_begin(U, 2048, 2048) == U and L.fork_debug_part_owner(U, 2048, U - 1) == 2047
