@@ -83,8 +83,9 @@ def test_device_generator_is_bit_identical_to_host_generator():
             mask = np.ones((B, wl.Lt), np.uint8)
             mask[0, 2] = 0
             lo, hi = np.zeros(B, np.int32), np.full(B, Ll, np.int32)
-            fs.cuda_fill(cfg, 3, torch.from_numpy(mask).cuda().data_ptr(), torch.from_numpy(lo).cuda().data_ptr(),
-                         torch.from_numpy(hi).cuda().data_ptr(), t.data_ptr(), Ll * wl.V, wl.V, 0, Ll, nonce=5)
+            mask_d, lo_d, hi_d = (torch.from_numpy(a).cuda() for a in (mask, lo, hi))   # kept alive until the sync
+            fs.cuda_fill(cfg, 3, mask_d.data_ptr(), lo_d.data_ptr(), hi_d.data_ptr(), t.data_ptr(), Ll * wl.V, wl.V,
+                         0, Ll, nonce=5)
             torch.cuda.synchronize()
             got = (t.view(torch.int16) if wl.dtype == fs.BF16 else t).cpu().numpy()
             got = got.view(np.uint16) if wl.dtype == fs.BF16 else got
@@ -126,7 +127,7 @@ def test_b8_full_decode_loop(variant):
     ost, nonces, osteps, _ = oracle_reference_loop(w, nseq, w.threshold)
     rc, steps, calls, h = gpu_loop(w, w.threshold, nonces)
     assert rc == 0 and steps == calls and steps >= osteps
-    compare_step_state(h, ost, nseq=nseq)
+    compare_step_state(h, ost, nseq=nseq, last_step_outputs=(steps == osteps))
     check_loop_invariants(h, w, steps)
     if variant == "literal":            # almost nothing clears 0.9: close to pure left-to-right decoding
         assert steps > 0.8 * w.Lt and h["commit_fallback"].mean() > 0.8
@@ -142,7 +143,7 @@ def test_passk_decode_loop_prefix_exact_rest_by_invariants():
     ost, nonces, osteps, _ = oracle_reference_loop(w, nseq, w.threshold)
     rc, steps, calls, h = gpu_loop(w, w.threshold, nonces)
     assert rc == 0 and steps == calls
-    compare_step_state(h, ost, nseq=nseq)
+    compare_step_state(h, ost, nseq=nseq, last_step_outputs=(steps == osteps))
     check_loop_invariants(h, w, steps)
     assert steps < w.Lt                      # parallel decoding: fewer model evaluations than tokens
     assert 0.05 < h["commit_fallback"].mean() < 0.16
@@ -170,7 +171,7 @@ def test_sweep_decode_loop(lam):
     ost, nonces, osteps, _ = oracle_reference_loop(w, nseq, lam)
     rc, steps, calls, h = gpu_loop(w, lam, nonces)
     assert rc == 0 and steps == calls
-    compare_step_state(h, ost, nseq=nseq)
+    compare_step_state(h, ost, nseq=nseq, last_step_outputs=(steps == osteps))
     check_loop_invariants(h, w, steps)
 
 
