@@ -410,6 +410,10 @@ def main():
     ap.add_argument("--workload", default="b8", choices=["b8", "passk", "sweep"])
     ap.add_argument("--no-extras", action="store_true", help="skip the other shapes, e2e and the CPU baseline")
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of one CUDA graph")
+    ap.add_argument("--variant", type=int, default=0, help="0 auto, 1 direct loads, 2 bulk-copy shared-memory ring")
+    ap.add_argument("--ctas-per-sm", type=int, default=0)
+    ap.add_argument("--stages", type=int, default=0)
+    ap.add_argument("--pdl", type=int, default=-1, help="1/0: programmatic dependent launch between a step's two kernels")
     args = ap.parse_args()
     if args.impl == "reference":
         return reference_arm(args)
@@ -430,6 +434,11 @@ def main():
     seed = shard_seed(w.seed, rank)
     peak, peak_src = measured_peak()
     fs.cuda_init()
+    pkg.fork_set_tuning(pkg.FORK_TUNE_VARIANT, args.variant)
+    pkg.fork_set_tuning(pkg.FORK_TUNE_CTAS_PER_SM, args.ctas_per_sm)
+    pkg.fork_set_tuning(pkg.FORK_TUNE_STAGES, args.stages)
+    if args.pdl >= 0:
+        pkg.fork_set_tuning(pkg.FORK_TUNE_PDL, args.pdl)
 
     sampler = ClockSampler(local_rank) if rank == 0 else None
     if world > 1:

@@ -60,6 +60,7 @@ typedef enum fork_dtype { FORK_BF16 = 0, FORK_F32 = 1 } fork_dtype;
 
 /* bits of the device status word (fork_device_status) */
 #define FORK_DEV_WINDOW_CLAMPED 1u /* a block [lo,hi) reached outside [pos0,pos0+Ll) or [0,Lt) and was clipped */
+#define FORK_DEV_TIMEOUT 2u        /* a bounded in-kernel wait gave up; the results of that call are not valid */
 
 /*
  * Arguments of one sampling step (Algorithm 2; inputs x_t, q_theta, lambda -> x_{t-1}).
@@ -169,9 +170,10 @@ const char* fork_status_string(int status);
  *   FORK_TUNE_VARIANT       0 = automatic, 1 = direct vector loads, 2 = bulk-copy shared-memory ring
  *   FORK_TUNE_CTAS_PER_SM   0 = automatic, else resident CTAs per SM used to size the grid
  *   FORK_TUNE_PDL           1 = chain the two kernels of a step with programmatic dependent launch
+ *   FORK_TUNE_STAGES        0 = automatic, else shared-memory stages (16 KB each) per CTA of variant 2
  * Returns the previous value, or -1 for an unknown key.
  */
-enum { FORK_TUNE_VARIANT = 0, FORK_TUNE_CTAS_PER_SM = 1, FORK_TUNE_PDL = 2, FORK_TUNE_COUNT_ = 3 };
+enum { FORK_TUNE_VARIANT = 0, FORK_TUNE_CTAS_PER_SM = 1, FORK_TUNE_PDL = 2, FORK_TUNE_STAGES = 3, FORK_TUNE_COUNT_ = 4 };
 int32_t fork_set_tuning(int32_t key, int32_t value);
 
 /* Profiling hook: the next fork_step / fork_logprob call made by this host thread records the two

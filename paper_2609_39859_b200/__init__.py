@@ -1,9 +1,9 @@
 """B200-native Fork-dLLM confidence pass: a C-ABI CUDA library (csrc/, include/fork_dllm.h) and a
 thin ctypes binding with the same entry-point names."""
 from .binding import (  # noqa: F401
-    FORK_BF16, FORK_DEV_WINDOW_CLAMPED, FORK_ERR_CUDA, FORK_ERR_INVALID_ARG, FORK_ERR_MAX_STEPS,
+    FORK_BF16, FORK_DEV_TIMEOUT, FORK_DEV_WINDOW_CLAMPED, FORK_ERR_CUDA, FORK_ERR_INVALID_ARG, FORK_ERR_MAX_STEPS,
     FORK_ERR_PROVIDER, FORK_ERR_WORKSPACE, FORK_F32, FORK_OK, FORK_ROW_BAD_TOKEN, FORK_ROW_NONFINITE,
-    FORK_TUNE_CTAS_PER_SM, FORK_TUNE_PDL, FORK_TUNE_VARIANT, ForkError, ForkState, fork_decode_loop,
+    FORK_TUNE_CTAS_PER_SM, FORK_TUNE_PDL, FORK_TUNE_STAGES, FORK_TUNE_VARIANT, ForkError, ForkState, fork_decode_loop,
     fork_device_status, fork_kernel_launches, fork_logits_fn, fork_logprob, fork_logprob_args, fork_set_tuning,
     fork_status_string, fork_step, fork_step_args, fork_workspace_bytes, lib, make_step_args,
 )

@@ -18,8 +18,8 @@ FORK_OK, FORK_ERR_INVALID_ARG, FORK_ERR_CUDA, FORK_ERR_WORKSPACE, FORK_ERR_MAX_S
     0, -1, -2, -3, -4, -5
 FORK_BF16, FORK_F32 = 0, 1
 FORK_ROW_NONFINITE, FORK_ROW_BAD_TOKEN = 1, 2
-FORK_DEV_WINDOW_CLAMPED = 1
-FORK_TUNE_VARIANT, FORK_TUNE_CTAS_PER_SM, FORK_TUNE_PDL = 0, 1, 2
+FORK_DEV_WINDOW_CLAMPED, FORK_DEV_TIMEOUT = 1, 2
+FORK_TUNE_VARIANT, FORK_TUNE_CTAS_PER_SM, FORK_TUNE_PDL, FORK_TUNE_STAGES = 0, 1, 2, 3
 
 
 class fork_step_args(C.Structure):
@@ -60,8 +60,9 @@ def lib():
     global _lib
     if _lib is not None:
         return _lib
+    override = os.environ.get("FORK_DLLM_LIB")          # developer hook: load an experimental build instead
     try:
-        path = _build.build()
+        path = override if override else _build.build()
     except Exception as e:  # no silent fallback: the CUDA library IS the product
         if not os.path.exists(_build.LIB):
             raise ImportError("libfork_dllm.so is missing and could not be built with nvcc: %r" % (e,)) from e

@@ -105,6 +105,25 @@ __device__ __forceinline__ const T* row_ptr(const RowSource& s, int b, int k) {
 
 __device__ __forceinline__ float4 ld_cg_f4(const float4* p) { return __ldcg(p); }
 
+/* ---- the partition as the kernels see it ---------------------------------------------------- */
+struct PartitionCtx {
+  long long U; int G; int C;
+  bool small;                                    /* (U+1)*G < 2^32: 32-bit division is exact */
+  __device__ __forceinline__ int owner(long long x) const {
+    if (small) return (int)((((uint32_t)x + 1u) * (uint32_t)G - 1u) / (uint32_t)U);
+    return fork_part_owner(U, G, x);
+  }
+};
+
+__device__ __forceinline__ PartitionCtx make_partition(int R, int C, int grid) {
+  PartitionCtx c;
+  c.U = (long long)R * C;
+  c.G = fork_effective_grid(c.U, grid);
+  c.C = C;
+  c.small = (unsigned long long)(c.U + 1) * (unsigned long long)c.G < 0xffffffffull;
+  return c;
+}
+
 /* ---- kernel 1: the active set -------------------------------------------------------------- */
 /* One CTA.  live(b,k) = flags[b,k] != 0 and k inside the sequence's window (block bounds clipped
    to the sequence buffer and to the positions the logits buffer covers). */
@@ -129,11 +148,15 @@ __device__ __forceinline__ void seq_window(const SetupParams& p, int b, int& lo,
   if (hi < lo) hi = lo;
 }
 
+constexpr int kSetupMaxB = 4096;     /* sequences whose counts fit in shared memory (more: counts go through global memory) */
+
 __global__ void __launch_bounds__(kSetupNT, 1) active_set_kernel(SetupParams p) {
   asm volatile("griddepcontrol.launch_dependents;");
+  __shared__ int sh_cnt[kSetupMaxB + 1];          /* sh_cnt[b+1] = live rows of b, then their inclusive scan */
   __shared__ int sh_warp[kSetupNT / 32];
   __shared__ int sh_carry;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = kSetupNT / 32;
+  int* cnt = (p.B <= kSetupMaxB) ? sh_cnt : p.seq_off;       /* cnt[0..B] */
   unsigned clipped_any = 0;
 
   /* pass 1: live rows per sequence */
@@ -141,22 +164,21 @@ __global__ void __launch_bounds__(kSetupNT, 1) active_set_kernel(SetupParams p) 
     int lo, hi; bool clipped;
     seq_window(p, b, lo, hi, clipped);
     clipped_any |= clipped ? 1u : 0u;
-    int cnt = 0;
+    int n = 0;
     for (int k0 = lo; k0 < hi; k0 += 32) {
       int k = k0 + lane;
       bool live = (k < hi) && p.flags[(size_t)b * p.Lt + k] != 0;
-      cnt += __popc(__ballot_sync(0xffffffffu, live));
+      n += __popc(__ballot_sync(0xffffffffu, live));
     }
-    if (lane == 0) { p.seq_off[b + 1] = cnt; p.expected[b] = 0; p.ticket[b] = 0; }
+    if (lane == 0) { cnt[b + 1] = n; p.ticket[b] = 0; }
   }
-  if (tid == 0) { p.seq_off[0] = 0; sh_carry = 0; }
+  if (tid == 0) { cnt[0] = 0; sh_carry = 0; }
   __syncthreads();
 
   /* pass 2: inclusive scan of the counts, kSetupNT sequences at a time */
   for (int base = 0; base < p.B; base += kSetupNT) {
     int b = base + tid;
-    int v = (b < p.B) ? p.seq_off[b + 1] : 0;
-    int x = v;
+    int x = (b < p.B) ? cnt[b + 1] : 0;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) { int y = __shfl_up_sync(0xffffffffu, x, o); if (lane >= o) x += y; }
     if (lane == 31) sh_warp[warp] = x;
@@ -170,23 +192,22 @@ __global__ void __launch_bounds__(kSetupNT, 1) active_set_kernel(SetupParams p) 
     }
     __syncthreads();
     int incl = sh_carry + sh_warp[warp] + x;
-    if (b < p.B) p.seq_off[b + 1] = incl;
+    if (b < p.B) cnt[b + 1] = incl;
     __syncthreads();
     if (tid == kSetupNT - 1) sh_carry = incl;
     __syncthreads();
   }
   const int R = sh_carry;
-  const long long U = (long long)R * p.C;
-  const int G = fork_effective_grid(U, p.G);
+  const PartitionCtx c = make_partition(R, p.C, p.G);
   if (tid == 0) {
-    p.hdr->R = R; p.hdr->C = p.C; p.hdr->G = G;
+    p.hdr->R = R; p.hdr->C = p.C; p.hdr->G = c.G;
   }
 
   /* pass 3: row list, expected part counts, outputs of idle sequences */
   for (int b = warp; b < p.B; b += nwarp) {
     int lo, hi; bool clipped;
     seq_window(p, b, lo, hi, clipped);
-    const int r0 = p.seq_off[b], r1 = p.seq_off[b + 1];
+    const int r0 = cnt[b], r1 = cnt[b + 1];
     int run = r0;
     for (int k0 = lo; k0 < hi; k0 += 32) {
       int k = k0 + lane;
@@ -196,11 +217,13 @@ __global__ void __launch_bounds__(kSetupNT, 1) active_set_kernel(SetupParams p) 
       run += __popc(bal);
     }
     int parts = 0;
-    for (int r = r0 + lane; r < r1; r += 32) parts += fork_row_parts(U, G, p.C, r);
+    for (int r = r0 + lane; r < r1; r += 32)
+      parts += c.owner((long long)(r + 1) * c.C - 1) - c.owner((long long)r * c.C) + 1;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) parts += __shfl_down_sync(0xffffffffu, parts, o);
     if (lane == 0) {
       p.expected[b] = parts;
+      if (cnt == sh_cnt) { p.seq_off[b + 1] = r1; if (b == 0) p.seq_off[0] = 0; }
       if (r0 == r1) {
         if (p.n_unmasked) p.n_unmasked[b] = 0;
         if (p.is_fallback) p.is_fallback[b] = 0;
@@ -214,119 +237,208 @@ __global__ void __launch_bounds__(kSetupNT, 1) active_set_kernel(SetupParams p) 
   if (tid == 0) p.hdr->dev_status = clipped_any ? FORK_DEV_WINDOW_CLAMPED : 0u;
 }
 
-/* ---- kernel 2: stream, reduce, select, commit --------------------------------------------- */
-struct Smem {
-  Part parts[kNT / 32];
-  float fl[kNT / 32];
-  int flag;
-  int pick;
-  int count;
-};
+/* ---- shared by both streaming kernels: merging parts, the unmask rule, scoring ------------- */
+__device__ __forceinline__ Part part_from(const float4& v) { return Part{v.x, v.y, v.z, __float_as_int(v.w)}; }
 
-/* all parts of row r, merged in ascending CTA order */
-__device__ __forceinline__ Part merge_row_parts(const ReduceParams& p, long long U, int G, int r) {
-  const int g0 = fork_part_owner(U, G, (long long)r * p.C);
-  const int g1 = fork_part_owner(U, G, (long long)(r + 1) * p.C - 1);
-  Part acc = part_empty();
-  for (int g = g0; g <= g1; ++g) {
-    float4 v = ld_cg_f4(p.parts + (r + g));
-    Part q{v.x, v.y, v.z, __float_as_int(v.w)};
-    acc = (g == g0) ? q : part_merge(acc, q);
+constexpr int kLaneMergeMax = 24;
+/* Parts of row r, by one lane, loaded four at a time and merged in ascending CTA order.  `n`
+   returns how many parts the row has; rows with more than kLaneMergeMax (very few live rows, the
+   whole grid on them) are merged by merge_row_parts_warp instead. */
+__device__ __forceinline__ Part merge_row_parts(const ReduceParams& p, const PartitionCtx& c, int r, int& g0, int& n) {
+  g0 = c.owner((long long)r * c.C);
+  const int g1 = c.owner((long long)(r + 1) * c.C - 1);
+  n = g1 - g0 + 1;
+  const float4* q = p.parts + (r + g0);
+  const float4 v0 = ld_cg_f4(q);
+  float4 v1 = v0, v2 = v0, v3 = v0;
+  if (n > 1) v1 = ld_cg_f4(q + 1);
+  if (n > 2) v2 = ld_cg_f4(q + 2);
+  if (n > 3) v3 = ld_cg_f4(q + 3);
+  Part acc = part_from(v0);
+  if (n > 1) acc = part_merge(acc, part_from(v1));
+  if (n > 2) acc = part_merge(acc, part_from(v2));
+  if (n > 3) acc = part_merge(acc, part_from(v3));
+  if (n <= kLaneMergeMax) {                                  /* a moderate number: this lane goes on, four loads at a time */
+    for (int j = 4; j < n; j += 4) {
+      const float4 w0 = ld_cg_f4(q + j);
+      float4 w1 = w0, w2 = w0, w3 = w0;
+      if (j + 1 < n) w1 = ld_cg_f4(q + j + 1);
+      if (j + 2 < n) w2 = ld_cg_f4(q + j + 2);
+      if (j + 3 < n) w3 = ld_cg_f4(q + j + 3);
+      acc = part_merge(acc, part_from(w0));
+      if (j + 1 < n) acc = part_merge(acc, part_from(w1));
+      if (j + 2 < n) acc = part_merge(acc, part_from(w2));
+      if (j + 3 < n) acc = part_merge(acc, part_from(w3));
+    }
   }
   return acc;
 }
 
-/* Row statistics of a batch of up to kNT rows starting at `base`, one row per thread; rows whose
-   streamed result is not finite are re-read by the whole CTA with the guarded routine. */
-template <typename T>
-__device__ __forceinline__ RowOut finalize_rows(const ReduceParams& p, Smem& sm, long long U, int G,
-                                                int base, int r1, Part& merged) {
-  const int r = base + threadIdx.x;
-  const bool valid = r < r1;
-  bool redo = false;
-  merged = part_empty();
-  if (valid) { merged = merge_row_parts(p, U, G, r); redo = part_needs_careful(merged); }
-  RowOut o = row_out_from(merged, false);
-  if (__syncthreads_or(redo ? 1 : 0)) {
-    for (;;) {
-      if (threadIdx.x == 0) sm.pick = kIdxNone;
-      __syncthreads();
-      if (redo) atomicMin(&sm.pick, r);
-      __syncthreads();
-      const int pick = sm.pick;
-      if (pick == kIdxNone) break;
-      const int2 bk = p.rows[pick];
-      bool bad;
-      Part c = careful_segment<T, kNT>(row_ptr<T>(p.src, bk.x, bk.y), 0, p.src.V, sm.parts, sm.fl, bad);
-      if (r == pick) { merged = c; o = row_out_from(c, bad); redo = false; }
-      __syncthreads();
+/* A row cut into many parts (few live rows, many CTAs): the whole warp loads 32 parts at a time
+   and tree-merges them; every lane returns the same Part. */
+__device__ __forceinline__ Part merge_row_parts_warp(const ReduceParams& p, int r, int g0, int n) {
+  const int lane = threadIdx.x & 31;
+  const float4* q = p.parts + (r + g0);
+  Part acc = part_empty();
+  for (int j0 = 0; j0 < n; j0 += 32) {
+    Part x = (j0 + lane < n) ? part_from(ld_cg_f4(q + j0 + lane)) : part_empty();
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      Part y;
+      y.m = __shfl_xor_sync(0xffffffffu, x.m, o); y.s = __shfl_xor_sync(0xffffffffu, x.s, o);
+      y.t = __shfl_xor_sync(0xffffffffu, x.t, o); y.idx = __shfl_xor_sync(0xffffffffu, x.idx, o);
+      const bool low = (lane & o) == 0;                      /* both partners compute merge(lower, upper) */
+      x = low ? part_merge(x, y) : part_merge(y, x);
     }
+    acc = part_merge(acc, x);
   }
-  return o;
+  return acc;
 }
 
+/* Guarded scalar reduction of a whole row by ONE warp (every lane returns the same Part). */
 template <typename T>
-__device__ void finalize_step_sequence(const ReduceParams& p, Smem& sm, long long U, int G, int b) {
+__device__ Part careful_row_warp(const T* row, int V, bool& bad) {
+  const int lane = threadIdx.x & 31;
+  float m = -INFINITY;
+  int idx = -1, isbad = 0;
+  for (int i = lane; i < V; i += 32) {
+    const float x = to_f32(row[i]);
+    if (x != x) { isbad = 1; continue; }
+    if (x == INFINITY) isbad = 1;
+    if (idx < 0 || x > m) { m = x; idx = i; }
+  }
+  if (idx < 0) idx = kIdxNone;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float om = __shfl_xor_sync(0xffffffffu, m, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+    const bool take = (oi != kIdxNone) && (idx == kIdxNone || om > m || (om == m && oi < idx));
+    if (take) { m = om; idx = oi; }
+  }
+  isbad = __any_sync(0xffffffffu, isbad);
+  if (isbad || idx == kIdxNone || m == -INFINITY) {
+    bad = true;
+    return Part{m, __int_as_float(0x7fc00000), __int_as_float(0x7fc00000), idx == kIdxNone ? 0 : idx};
+  }
+  bad = false;
+  float s = 0.f, t = 0.f;
+  for (int i = lane; i < V; i += 32) {
+    const float x = to_f32(row[i]);
+    if (x == -INFINITY) continue;
+    const float y = (x - m) * kLog2e;
+    const float e = exp2f(y);
+    s += e;
+    if (e > 0.f) t = fmaf(y, e, t);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) { s += __shfl_xor_sync(0xffffffffu, s, o); t += __shfl_xor_sync(0xffffffffu, t, o); }
+  return Part{m, s, t, idx};
+}
+
+/* Final statistics of up to 32 rows (one per lane) of sequence b starting at row `base`.
+   Rows whose streamed result is not finite are re-read by the whole warp with the guarded routine. */
+template <typename T, bool WANT_INDEX>
+__device__ __forceinline__ RowOut finalize_rows_warp(const ReduceParams& p, const PartitionCtx& c, int b, int base,
+                                                     int r1, Part& merged, int& k) {
+  const int lane = threadIdx.x & 31;
+  const int r = base + lane;
+  const bool valid = r < r1;
+  bool redo = false, bad = false;
+  merged = part_empty();
+  k = 0;
+  int g0 = 0, nparts = 0;
+  if (valid) { k = p.rows[r].y; merged = merge_row_parts(p, c, r, g0, nparts); }
+  unsigned many = __ballot_sync(0xffffffffu, valid && nparts > kLaneMergeMax);
+  while (many) {                                             /* rows cut into very many parts: all lanes help */
+    const int src = __ffs(many) - 1;
+    many &= many - 1;
+    const Part m = merge_row_parts_warp(p, __shfl_sync(0xffffffffu, r, src), __shfl_sync(0xffffffffu, g0, src),
+                                        __shfl_sync(0xffffffffu, nparts, src));
+    if (lane == src) merged = m;
+  }
+  if (valid) redo = part_needs_careful(merged);
+  unsigned todo = __ballot_sync(0xffffffffu, valid && redo);
+  while (todo) {
+    const int src = __ffs(todo) - 1;
+    todo &= todo - 1;
+    const int kk = __shfl_sync(0xffffffffu, k, src);
+    bool bd;
+    const Part cp = careful_row_warp<T>(row_ptr<T>(p.src, b, kk), p.src.V, bd);
+    if (lane == src) { merged = cp; bad = bd; }
+  }
+  if (valid && WANT_INDEX && !bad) merged.idx = resolve_index<T>(row_ptr<T>(p.src, b, k), merged.idx, p.src.V, merged.m);
+  return row_out_from(merged, bad);
+}
+
+/* The unmask rule for one sequence, run by one warp once every part of the sequence has arrived
+   (Algorithm 2 lines 6-9): commit every live position whose confidence exceeds lambda, or the
+   leftmost live position when none does; write tokens, mask and the per-token records. */
+template <typename T>
+__device__ void finalize_step_sequence(const ReduceParams& p, const PartitionCtx& c, int b) {
+  const int lane = threadIdx.x & 31;
   const int r0 = p.seq_off[b], r1 = p.seq_off[b + 1];
+  const bool one_batch = (r1 - r0) <= 32;                    /* the usual case: results stay in registers */
   int any = 0;
-  for (int base = r0; base < r1; base += kNT) {
-    Part merged;
-    RowOut o = finalize_rows<T>(p, sm, U, G, base, r1, merged);
-    const int r = base + threadIdx.x;
+  float4 keep = make_float4(0.f, 0.f, 0.f, 0.f);
+  int keep_k = 0;
+  for (int base = r0; base < r1; base += 32) {
+    Part merged; int k;
+    const RowOut o = finalize_rows_warp<T, true>(p, c, b, base, r1, merged, k);
+    const int r = base + lane;
     if (r < r1) {
-      const size_t at = (size_t)b * p.Lt + p.rows[r].y;
+      const size_t at = (size_t)b * p.Lt + k;
       if (p.conf) p.conf[at] = o.conf;
       if (p.cand) p.cand[at] = o.cand;
       if (p.entropy) p.entropy[at] = o.entropy;
       if (p.logp) p.logp[at] = o.logp;
       if (p.row_status) p.row_status[at] = o.status;
-      p.final_rec[r] = make_float4(o.conf, o.logp, __int_as_float(o.cand), 0.f);
+      keep = make_float4(o.conf, o.logp, __int_as_float(o.cand), 0.f);
+      keep_k = k;
+      if (!one_batch) p.final_rec[r] = keep;
       any |= (o.conf > p.threshold) ? 1 : 0;                 /* U_t non-empty (Algorithm 2, line 6) */
     }
   }
-  any = __syncthreads_or(any);
+  any = __any_sync(0xffffffffu, any);
   const int fb = any ? 0 : 1;                                /* fallback step: max_k c <= lambda */
   int count = 0;
-  for (int base = r0; base < r1; base += kNT) {
-    const int r = base + threadIdx.x;
+  for (int base = r0; base < r1; base += 32) {
+    const int r = base + lane;
+    bool commit = false;
     if (r < r1) {
-      const float4 f = p.final_rec[r];                       /* written by this same thread above */
-      const bool commit = fb ? (r == r0) : (f.x > p.threshold);   /* leftmost(M_t), or the threshold set */
+      const float4 f = one_batch ? keep : p.final_rec[r];    /* written by this same lane above */
+      commit = fb ? (r == r0) : (f.x > p.threshold);         /* leftmost(M_t), or the threshold set */
       if (commit) {
-        const size_t at = (size_t)b * p.Lt + p.rows[r].y;
+        const size_t at = (size_t)b * p.Lt + (one_batch ? keep_k : p.rows[r].y);
         p.tokens[at] = __float_as_int(f.z);
         p.mask[at] = 0;
         if (p.commit_step) p.commit_step[at] = p.step;
         if (p.commit_fallback) p.commit_fallback[at] = (uint8_t)fb;
         if (p.commit_logp) p.commit_logp[at] = f.y;
-        ++count;
       }
     }
+    count += __popc(__ballot_sync(0xffffffffu, commit));
   }
-  if (threadIdx.x == 0) sm.count = 0;
-  __syncthreads();
-  if (count) atomicAdd(&sm.count, count);
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    if (p.n_unmasked) p.n_unmasked[b] = sm.count;
+  if (lane == 0) {
+    if (p.n_unmasked) p.n_unmasked[b] = count;
     if (p.is_fallback) p.is_fallback[b] = (uint8_t)fb;
-    if (p.fallback_pos) p.fallback_pos[b] = fb ? p.rows[r0].y : -1;
+    if (p.fallback_pos) p.fallback_pos[b] = fb ? (one_batch ? keep_k : p.rows[r0].y) : -1;
     if (p.nfe) p.nfe[b] += 1;
     if (p.n_fallback) p.n_fallback[b] += fb;
   }
-  __syncthreads();
 }
 
+/* Scoring for one sequence by one warp: log q(token) = x_tok - m - ln s at every selected position
+   and their sum (Section 3.2 of the paper: the likelihood terms of the ForkGRPO ratio). */
 template <typename T>
-__device__ void finalize_logprob_sequence(const ReduceParams& p, Smem& sm, long long U, int G, int b) {
+__device__ void finalize_logprob_sequence(const ReduceParams& p, const PartitionCtx& c, int b) {
+  const int lane = threadIdx.x & 31;
   const int r0 = p.seq_off[b], r1 = p.seq_off[b + 1];
   float local = 0.f;
-  for (int base = r0; base < r1; base += kNT) {
-    Part merged;
-    RowOut o = finalize_rows<T>(p, sm, U, G, base, r1, merged);
-    const int r = base + threadIdx.x;
+  for (int base = r0; base < r1; base += 32) {
+    Part merged; int k;
+    const RowOut o = finalize_rows_warp<T, false>(p, c, b, base, r1, merged, k);
+    const int r = base + lane;
     if (r < r1) {
-      const int k = p.rows[r].y;
       const size_t at = (size_t)b * p.Lt + k;
       const int tok = p.lp_tokens[at];
       uint32_t st = o.status;
@@ -339,13 +451,56 @@ __device__ void finalize_logprob_sequence(const ReduceParams& p, Smem& sm, long 
       local += lp;
     }
   }
-  const float total = block_sum_f32<kNT>(local, sm.fl);
-  if (threadIdx.x == 0) {
-    if (p.seq_sum) p.seq_sum[b] = total;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) local += __shfl_xor_sync(0xffffffffu, local, o);
+  if (lane == 0) {
+    if (p.seq_sum) p.seq_sum[b] = local;
     if (p.seq_cnt) p.seq_cnt[b] = r1 - r0;
   }
-  __syncthreads();
 }
+
+/* Lane 0 of the calling warp publishes one part of row r (sequence b) and takes a ticket; returns
+   (to every lane) whether this was the last part the sequence was waiting for. */
+__device__ __forceinline__ bool publish_part(const ReduceParams& p, const Part& part, int r, int g, int b) {
+  int last = 0;
+  if ((threadIdx.x & 31) == 0) {
+    const int want = p.expected[b];
+    p.parts[r + g] = make_float4(part.m, part.s, part.t, __int_as_float(part.idx));
+    int old;                                 /* release our part, acquire everybody else's */
+    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(p.ticket + b) : "memory");
+    last = (old + 1 == want) ? 1 : 0;
+  }
+  return __shfl_sync(0xffffffffu, last, 0) != 0;
+}
+
+/* The rows a CTA works on: its contiguous unit range cut at row boundaries. */
+struct Segment { int r, e0, e1; };
+struct SegmentIter {
+  long long u, u1; int C, V;
+  __device__ __forceinline__ void init(const PartitionCtx& c, int g, int V_) {
+    u = fork_part_begin(c.U, c.G, g); u1 = fork_part_begin(c.U, c.G, g + 1); C = c.C; V = V_;
+  }
+  __device__ __forceinline__ bool next(Segment& s) {
+    if (u >= u1) return false;
+    s.r = (int)(u / C);
+    const int c0 = (int)(u - (long long)s.r * C);
+    long long uend = (long long)(s.r + 1) * C;
+    if (uend > u1) uend = u1;
+    const int c1 = (int)(uend - (long long)s.r * C);
+    s.e0 = c0 * FORK_CHUNK;
+    s.e1 = c1 * FORK_CHUNK;
+    if (s.e1 > V) s.e1 = V;
+    u = uend;
+    return true;
+  }
+};
+
+/* ---- kernel 2a: direct 128-bit loads (also the path for buffers that are not 16-byte aligned) -- */
+struct Smem {
+  Part parts[kNT / 32];
+  float fl[kNT / 32];
+  int flag;
+};
 
 template <typename T, int MODE>
 __global__ void __launch_bounds__(kNT, 4) reduce_select_kernel(ReduceParams p) {
@@ -354,50 +509,284 @@ __global__ void __launch_bounds__(kNT, 4) reduce_select_kernel(ReduceParams p) {
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const int R = p.hdr->R;
   if (R <= 0) return;
-  const int g = blockIdx.x, C = p.C;
-  const long long U = (long long)R * C;
-  const int G = fork_effective_grid(U, (int)gridDim.x);     /* CTAs beyond the number of units have no work */
-  if (g >= G) return;
-  long long u = fork_part_begin(U, G, g);
-  const long long u1 = fork_part_begin(U, G, g + 1);
-
-  while (u < u1) {
-    const int r = (int)(u / C);
-    const int c0 = (int)(u - (long long)r * C);
-    long long uend = (long long)(r + 1) * C;
-    if (uend > u1) uend = u1;
-    const int c1 = (int)(uend - (long long)r * C);
-    const int e0 = c0 * FORK_CHUNK;
-    int e1 = c1 * FORK_CHUNK;
-    if (e1 > p.src.V) e1 = p.src.V;
-    const int2 bk = p.rows[r];
+  const PartitionCtx c = make_partition(R, p.C, (int)gridDim.x);
+  const int g = blockIdx.x;
+  if (g >= c.G) return;                                     /* CTAs beyond the number of units have no work */
+  SegmentIter it;
+  it.init(c, g, p.src.V);
+  Segment sg;
+  bool sticky = false;
+  while (it.next(sg)) {
+    const int2 bk = p.rows[sg.r];
     const T* row = row_ptr<T>(p.src, bk.x, bk.y);
-
     Part part;
     if (p.fast) {
-      Acc<WITH_T> acc;
-      acc.init();
-      stream_direct<T, WITH_T, kNT, kUnroll>(acc, row, e0, e1);
-      part = part_block_reduce<kNT>(acc.part(), sm.parts);
+      part = part_block_reduce<kNT>(
+          stream_thread<T, WITH_T, kNT, kUnroll>(row, sg.e0, sg.e1, threadIdx.x, threadIdx.x == 0, sticky), sm.parts);
     } else {
       bool bad;
-      part = careful_segment<T, kNT>(row, e0, e1, sm.parts, sm.fl, bad);
+      part = careful_segment<T, kNT>(row, sg.e0, sg.e1, sm.parts, sm.fl, bad);
     }
-    if (threadIdx.x == 0) {
-      p.parts[r + g] = make_float4(part.m, part.s, part.t, __int_as_float(part.idx));
-      __threadfence();
-      const int old = atomicAdd(p.ticket + bk.x, 1);
-      sm.flag = (old + 1 == p.expected[bk.x]) ? 1 : 0;
+    if (threadIdx.x < 32) {
+      const bool last = publish_part(p, part, sg.r, g, bk.x);
+      if (last) {                                           /* every part of sequence b has been delivered */
+        if (MODE == kModeStep) finalize_step_sequence<T>(p, c, bk.x);
+        else finalize_logprob_sequence<T>(p, c, bk.x);
+      }
     }
-    __syncthreads();
-    const int last = sm.flag;
-    __syncthreads();
-    if (last) {                                   /* every part of sequence b has been delivered */
-      __threadfence();
-      if (MODE == kModeStep) finalize_step_sequence<T>(p, sm, U, G, bk.x);
-      else finalize_logprob_sequence<T>(p, sm, U, G, bk.x);
+  }
+}
+
+/* ---- kernel 2b: bulk-copy (TMA) shared-memory ring, warp-specialised --------------------------
+ * Warps 0..kCW-1 consume, warp kCW produces, warp kCW+1 finalises.
+ *   producer : one lane walks the CTA's segments and issues cp.async.bulk copies of up to one stage
+ *              (kStageBytes) into a ring of shared-memory stages, each guarded by a full/empty
+ *              mbarrier pair; it runs ahead of the consumers by the depth of the ring, across row
+ *              boundaries, so HBM requests never drain while rows are being wrapped up.
+ *   consumers: wait for a stage, read their 128-bit vectors from shared memory, accumulate, release
+ *              the stage; at the end of a row segment each warp shuffle-reduces its threads' Parts
+ *              and hands ONE Part to the finaliser through a small mbarrier-guarded mailbox, then
+ *              goes straight on to the next segment.
+ *   finaliser: merges the kCW warp Parts, publishes the CTA's part of the row, takes the sequence's
+ *              ticket and, if it was the last, applies the unmask rule for that sequence.
+ * Every mbarrier wait is bounded: after kSpinLimit failed polls the thread records
+ * FORK_DEV_TIMEOUT in the workspace header and leaves its loop.                                   */
+constexpr int kCW = 8;
+constexpr int kCT = kCW * 32;
+constexpr int kStageVecs = kCT * kUnroll;                  /* 128-bit vectors per stage */
+constexpr int kStageBytes = kStageVecs * 16;               /* 16 KB */
+constexpr int kMail = 4;                                   /* mailbox depth (row segments in flight to the finaliser) */
+constexpr int kMaxStages = 13;
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+struct RingSmem {
+  unsigned long long full[kMaxStages], empty[kMaxStages], mfull[kMail], mempty[kMail];
+  Part mail[kMail][kCW];
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+/* bounded wait; false (and a status bit in the workspace header) if the phase never completed */
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity, const ReduceParams& p) {
+  for (uint32_t i = 0; i < kSpinLimit; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  atomicOr(const_cast<uint32_t*>(&p.hdr->dev_status), FORK_DEV_TIMEOUT);
+  return false;
+}
+__device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               :: "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
+#ifdef FORK_EXP_TRACE
+__device__ unsigned long long g_trace[FORK_MAX_GRID][16];
+__device__ __forceinline__ void trace(int slot) {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  g_trace[blockIdx.x][slot] = t;
+}
+#define FORK_TRACE(slot) trace(slot)
+#else
+#define FORK_TRACE(slot)
+#endif
+
+template <typename T, int MODE>
+__global__ void __launch_bounds__((kCW + 2) * 32, 2) reduce_select_ring_kernel(ReduceParams p, int n_stages) {
+  constexpr bool WITH_T = (MODE == kModeStep);
+  constexpr int VEC = 16 / (int)sizeof(T);
+  extern __shared__ __align__(1024) unsigned char dyn_smem[];
+  unsigned char* ring = dyn_smem;
+  RingSmem& rs = *reinterpret_cast<RingSmem*>(dyn_smem + (size_t)n_stages * kStageBytes);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) FORK_TRACE(0);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < n_stages; ++s) { mbar_init(&rs.full[s], 1); mbar_init(&rs.empty[s], kCW); }
+    for (int d = 0; d < kMail; ++d) { mbar_init(&rs.mfull[d], kCW); mbar_init(&rs.mempty[d], 1); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int R = p.hdr->R;
+  if (R <= 0) return;
+  if (threadIdx.x == 0) FORK_TRACE(1);
+  const PartitionCtx c = make_partition(R, p.C, (int)gridDim.x);
+  const int g = blockIdx.x;
+  if (g >= c.G) return;
+  SegmentIter it;
+  it.init(c, g, p.src.V);
+  Segment sg;
+  if (threadIdx.x == 0) FORK_TRACE(2);
+
+  if (warp == kCW) {
+    /* ---------------- producer ---------------- */
+    if (lane != 0) return;
+    uint32_t n = 0, s = 0, ph = 0;                           /* stages issued, ring slot, its phase */
+    bool ok = true;
+    while (ok && it.next(sg)) {
+      const int2 bk = p.rows[sg.r];
+      const char* src = reinterpret_cast<const char*>(row_ptr<T>(p.src, bk.x, bk.y) + sg.e0);
+      const uint32_t total = (uint32_t)((sg.e1 - sg.e0) / VEC) * 16u;
+      for (uint32_t off = 0; off < total; off += kStageBytes, ++n) {
+        const uint32_t bytes = (total - off < (uint32_t)kStageBytes) ? (total - off) : (uint32_t)kStageBytes;
+        if (!mbar_wait(&rs.empty[s], ph ^ 1u, p)) { ok = false; break; }
+        mbar_arrive_expect_tx(&rs.full[s], bytes);
+        bulk_copy_g2s(ring + (size_t)s * kStageBytes, src + off, bytes, &rs.full[s]);
+        if (n == 0) FORK_TRACE(3);
+        if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1u; }
+      }
     }
-    u = uend;
+    if (!ok) {                                               /* do not leave with copies still landing */
+      const uint32_t first = n > (uint32_t)n_stages ? n - (uint32_t)n_stages : 0u;
+      for (uint32_t q = first; q < n; ++q)
+        mbar_wait(&rs.full[q % (uint32_t)n_stages], (q / (uint32_t)n_stages) & 1u, p);
+    }
+    FORK_TRACE(4);
+    return;
+  }
+
+  if (warp < kCW) {
+    /* ---------------- consumers ---------------- */
+    const int ctid = threadIdx.x;                           /* 0 .. kCT-1 */
+    uint32_t s = 0, ph = 0, nseg = 0;                       /* ring slot, its phase, segments done */
+    bool sticky = false;                                    /* this thread has met a -inf logit before */
+#ifdef FORK_EXP_TRACE
+    unsigned long long tw = 0, tt = 0, ta = 0, tn = 0;
+    const long long cstart = clock64();
+#endif
+    while (it.next(sg)) {
+      Acc<T, WITH_T, false> a;
+      a.init();
+      const int nvec = (sg.e1 - sg.e0) / VEC;
+      for (int voff = 0; voff < nvec; voff += kStageVecs) {
+#ifdef FORK_EXP_TRACE
+        const long long c0 = clock64();
+#endif
+        if (!mbar_wait(&rs.full[s], ph, p)) return;
+#ifdef FORK_EXP_TRACE
+        const long long c1 = clock64();
+#endif
+        if (ctid == 0 && nseg == 0 && voff == 0) FORK_TRACE(5);
+        const uint4* sp = reinterpret_cast<const uint4*>(ring + (size_t)s * kStageBytes);
+        const int nv = nvec - voff;
+#ifndef FORK_EXP_NO_COMPUTE
+        if (nv >= kStageVecs) {
+          /* a full stage: kUnroll vectors per thread; the stage is handed back to the producer as
+             soon as the values sit in registers (track() has consumed every loaded word) */
+          uint4 v[kUnroll];
+#pragma unroll
+          for (int j = 0; j < kUnroll; ++j) v[j] = sp[ctid + j * kCT];
+          if (!sticky) a.template track<kUnroll>(v, sg.e0 + (voff + ctid) * VEC, kCT * VEC);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&rs.empty[s]);
+#ifdef FORK_EXP_TRACE
+          const long long c2 = clock64();
+#endif
+          if (!sticky) a.template accumulate<kUnroll>(v);
+#ifdef FORK_EXP_TRACE
+          {
+            const long long c3 = clock64();
+            tw += (unsigned long long)(c1 - c0); tt += (unsigned long long)(c2 - c1); ta += (unsigned long long)(c3 - c2); tn += 1ull;
+          }
+#endif
+        } else {
+          if (!sticky) {
+            for (int i = ctid; i < nv; i += kCT) {
+              uint4 v[1];
+              v[0] = sp[i];
+              a.template group<1>(v, sg.e0 + (voff + i) * VEC, 0);
+            }
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&rs.empty[s]);
+        }
+#else
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&rs.empty[s]);
+#endif
+        if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1u; }
+      }
+      const bool tail = (ctid == 0) && (sg.e0 + nvec * VEC < sg.e1);   /* fewer than VEC trailing elements */
+      Part pt;
+      if (!sticky) {
+        if (tail) {
+          const int2 bk = p.rows[sg.r];
+          const T* row = row_ptr<T>(p.src, bk.x, bk.y);
+          for (int e = sg.e0 + nvec * VEC; e < sg.e1; ++e) a.one(to_f32(row[e]), e);
+        }
+        pt = a.part();
+#ifndef FORK_EXP_NO_COMPUTE
+        if (!part_is_finite(pt)) sticky = true;
+#endif
+      }
+      /* a thread that met -inf (now or earlier) takes its own vectors again from global memory, clamped */
+      if (sticky) {
+        const int2 bk = p.rows[sg.r];
+        pt = stream_thread_clamped<T, WITH_T, kCT>(row_ptr<T>(p.src, bk.x, bk.y), sg.e0, sg.e1, ctid, ctid == 0);
+      }
+#ifdef FORK_EXP_NO_COMPUTE
+      pt = Part{1.f, 1.f, 0.f, sg.e0};
+#endif
+      __syncwarp();
+      pt = part_warp_reduce(pt);
+      if (ctid == 0) FORK_TRACE(6);
+      if (lane == 0) {
+        const uint32_t d = nseg % kMail, mph = (nseg / kMail) & 1u;
+        if (mbar_wait(&rs.mempty[d], mph ^ 1u, p)) {
+          rs.mail[d][warp] = pt;
+          mbar_arrive(&rs.mfull[d]);
+        }
+      }
+      if (ctid == 0) FORK_TRACE(7);
+      ++nseg;
+    }
+#ifdef FORK_EXP_TRACE
+    if (lane == 0 && warp == 3) {
+      g_trace[blockIdx.x][12] = tw; g_trace[blockIdx.x][13] = tt; g_trace[blockIdx.x][14] = ta; g_trace[blockIdx.x][15] = tn;
+      g_trace[blockIdx.x][11] = (unsigned long long)(clock64() - cstart);
+    }
+#endif
+    return;
+  }
+
+  /* ---------------- finaliser ---------------- */
+  uint32_t nseg = 0;
+  while (it.next(sg)) {
+    const uint32_t d = nseg % kMail, ph = (nseg / kMail) & 1u;
+    if (!mbar_wait(&rs.mfull[d], ph, p)) return;
+    Part pt = (lane < kCW) ? rs.mail[d][lane] : part_empty();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&rs.mempty[d]);
+    pt = part_warp_reduce(pt);
+    const int b = p.rows[sg.r].x;
+    if (lane == 0) FORK_TRACE(8);
+#ifndef FORK_EXP_NO_PUBLISH
+    if (publish_part(p, pt, sg.r, g, b)) {
+      if (lane == 0) FORK_TRACE(9);
+#ifndef FORK_EXP_NO_FINALIZE
+      if (MODE == kModeStep) finalize_step_sequence<T>(p, c, b);
+      else finalize_logprob_sequence<T>(p, c, b);
+#endif
+      if (lane == 0) FORK_TRACE(11);
+    }
+    if (lane == 0) FORK_TRACE(10);
+#endif
+    ++nseg;
   }
 }
 
@@ -446,7 +835,20 @@ using namespace forkd;
 static std::atomic<long long> g_launches{0};
 static std::atomic<int> g_tune[FORK_TUNE_COUNT_];
 
-struct DeviceInfo { int sms = 0; int occ[2][2] = {{0, 0}, {0, 0}}; };
+static size_t ring_smem_bytes(int n_stages) { return (size_t)n_stages * kStageBytes + sizeof(RingSmem); }
+
+static void ring_config(int* ctas_per_sm, int* n_stages) {
+  int per_sm = g_tune[FORK_TUNE_CTAS_PER_SM].load();
+  if (per_sm <= 0 || per_sm > 3) per_sm = 2;
+  int st = g_tune[FORK_TUNE_STAGES].load();
+  const int max_st = (int)((220 * 1024 / per_sm - sizeof(RingSmem) - 1024) / kStageBytes);
+  if (st <= 0 || st > max_st) st = max_st;
+  if (st > kMaxStages) st = kMaxStages;
+  if (st < 2) st = 2;
+  *ctas_per_sm = per_sm; *n_stages = st;
+}
+
+struct DeviceInfo { int sms = 0; int occ[2][2] = {{0, 0}, {0, 0}}; bool ring_ready = false; };
 static DeviceInfo g_dev[64];
 
 template <typename T, int MODE>
@@ -467,13 +869,26 @@ static bool device_info(DeviceInfo** out) {
     d.occ[0][1] = occupancy_of<bf16_t, kModeLogprob>();
     d.occ[1][0] = occupancy_of<float, kModeStep>();
     d.occ[1][1] = occupancy_of<float, kModeLogprob>();
+    const int max_dyn = (int)ring_smem_bytes(kMaxStages);
+    d.ring_ready =
+        cudaFuncSetAttribute(reduce_select_ring_kernel<bf16_t, kModeStep>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn) == cudaSuccess &&
+        cudaFuncSetAttribute(reduce_select_ring_kernel<bf16_t, kModeLogprob>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn) == cudaSuccess &&
+        cudaFuncSetAttribute(reduce_select_ring_kernel<float, kModeStep>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn) == cudaSuccess &&
+        cudaFuncSetAttribute(reduce_select_ring_kernel<float, kModeLogprob>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn) == cudaSuccess;
+    if (!d.ring_ready) return false;
     d.sms = sms;
   }
   *out = &d;
   return true;
 }
 
-static int grid_size(const DeviceInfo& d, int dtype, int mode) {
+static int grid_size(const DeviceInfo& d, int dtype, int mode, bool fast) {
+  const int variant = g_tune[FORK_TUNE_VARIANT].load();
+  if (fast && (variant == 0 || variant == 2)) {
+    int per, stages;
+    ring_config(&per, &stages);
+    return d.sms * per;
+  }
   int per_sm = g_tune[FORK_TUNE_CTAS_PER_SM].load();
   int occ = d.occ[dtype][mode];
   if (occ <= 0) occ = 1;
@@ -527,8 +942,41 @@ static cudaError_t launch_reduce(const ReduceParams& rp, int dtype, int mode, in
   return e;
 }
 
+template <typename T, int MODE>
+static cudaError_t launch_ring(const ReduceParams& rp, int G, int n_stages, bool pdl, cudaStream_t st) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(G); cfg.blockDim = dim3((kCW + 2) * 32); cfg.dynamicSmemBytes = ring_smem_bytes(n_stages);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  if (pdl) {
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+  }
+  cudaError_t e = cudaLaunchKernelEx(&cfg, reduce_select_ring_kernel<T, MODE>, rp, n_stages);
+  if (e == cudaSuccess) g_launches.fetch_add(1);
+  return e;
+}
+
+/* variant 2 (bulk-copy ring) needs 16-byte aligned rows; everything else takes variant 1 */
+static bool use_ring(const ReduceParams& rp) {
+  const int v = g_tune[FORK_TUNE_VARIANT].load();
+  return rp.fast && (v == 0 || v == 2);
+}
+
 static cudaError_t launch_reduce_inner(const ReduceParams& rp, int dtype, int mode, int G, cudaStream_t st) {
   const bool pdl = g_tune[FORK_TUNE_PDL].load() != 0;
+  if (use_ring(rp)) {
+    int per_sm, n_stages;
+    ring_config(&per_sm, &n_stages);
+    if (dtype == FORK_BF16) {
+      if (mode == kModeStep) return launch_ring<bf16_t, kModeStep>(rp, G, n_stages, pdl, st);
+      return launch_ring<bf16_t, kModeLogprob>(rp, G, n_stages, pdl, st);
+    }
+    if (mode == kModeStep) return launch_ring<float, kModeStep>(rp, G, n_stages, pdl, st);
+    return launch_ring<float, kModeLogprob>(rp, G, n_stages, pdl, st);
+  }
   if (dtype == FORK_BF16) {
     if (mode == kModeStep) return launch(reduce_select_kernel<bf16_t, kModeStep>, dim3(G), dim3(kNT), st, pdl, rp);
     return launch(reduce_select_kernel<bf16_t, kModeLogprob>, dim3(G), dim3(kNT), st, pdl, rp);
@@ -578,7 +1026,8 @@ static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const i
   if (!device_info(&dev)) return FORK_ERR_CUDA;
   WsView w = ws_view(ws, a->B, a->Lt);
   const int mode = kModeStep;
-  const int G = grid_size(*dev, a->dtype, mode);
+  const bool fast = source_is_vector_aligned(a->logits, a->stride_b, a->stride_l, a->dtype);
+  const int G = grid_size(*dev, a->dtype, mode, fast);
   const int C = (a->V + FORK_CHUNK - 1) / FORK_CHUNK;
 
   SetupParams sp;
@@ -593,7 +1042,7 @@ static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const i
   memset(&rp, 0, sizeof(rp));
   rp.src = RowSource{a->logits, (long long)a->stride_b, (long long)a->stride_l, a->pos0, a->Ll, a->V};
   rp.B = a->B; rp.Lt = a->Lt; rp.C = C;
-  rp.fast = source_is_vector_aligned(a->logits, a->stride_b, a->stride_l, a->dtype) ? 1 : 0;
+  rp.fast = fast ? 1 : 0;
   rp.hdr = w.hdr; rp.seq_off = w.seq_off; rp.expected = w.expected; rp.ticket = w.ticket;
   rp.rows = w.rows; rp.final_rec = w.final_rec; rp.parts = w.parts;
   rp.tokens = a->tokens; rp.mask = a->mask; rp.threshold = a->threshold; rp.step = a->step;
@@ -637,7 +1086,8 @@ extern "C" fork_status fork_logprob(const fork_logprob_args* a, void* ws, size_t
   if (!device_info(&dev)) return FORK_ERR_CUDA;
   WsView w = ws_view(ws, a->B, a->Lt);
   const int mode = kModeLogprob;
-  const int G = grid_size(*dev, a->dtype, mode);
+  const bool fast = source_is_vector_aligned(a->logits, a->stride_b, a->stride_l, a->dtype);
+  const int G = grid_size(*dev, a->dtype, mode, fast);
   const int C = (a->V + FORK_CHUNK - 1) / FORK_CHUNK;
   if (cudaMemsetAsync(a->logp, 0, sizeof(float) * (size_t)a->B * a->Lt, st) != cudaSuccess) return FORK_ERR_CUDA;
 
@@ -653,7 +1103,7 @@ extern "C" fork_status fork_logprob(const fork_logprob_args* a, void* ws, size_t
   memset(&rp, 0, sizeof(rp));
   rp.src = RowSource{a->logits, (long long)a->stride_b, (long long)a->stride_l, a->pos0, a->Ll, a->V};
   rp.B = a->B; rp.Lt = a->Lt; rp.C = C;
-  rp.fast = source_is_vector_aligned(a->logits, a->stride_b, a->stride_l, a->dtype) ? 1 : 0;
+  rp.fast = fast ? 1 : 0;
   rp.hdr = w.hdr; rp.seq_off = w.seq_off; rp.expected = w.expected; rp.ticket = w.ticket;
   rp.rows = w.rows; rp.final_rec = w.final_rec; rp.parts = w.parts;
   rp.lp_tokens = a->tokens; rp.lp_out = a->logp; rp.seq_sum = a->seq_sum; rp.seq_cnt = a->seq_cnt;
@@ -801,4 +1251,13 @@ extern "C" int64_t fork_debug_part_begin(int64_t U, int32_t G, int32_t g) { retu
 extern "C" int32_t fork_debug_part_owner(int64_t U, int32_t G, int64_t x) { return fork_part_owner(U, G, x); }
 extern "C" int32_t fork_debug_row_parts(int64_t U, int32_t G, int32_t C, int64_t r) { return fork_row_parts(U, G, C, r); }
 extern "C" int32_t fork_debug_chunk(void) { return FORK_CHUNK; }
+#ifdef FORK_EXP_TRACE
+extern "C" int fork_debug_trace(void* host_out) {
+  return (int)cudaMemcpyFromSymbol(host_out, g_trace, sizeof(unsigned long long) * FORK_MAX_GRID * 16);
+}
+extern "C" int fork_debug_trace_clear(void) {
+  static unsigned long long z[FORK_MAX_GRID][16];
+  return (int)cudaMemcpyToSymbol(g_trace, z, sizeof(z));
+}
+#endif
 extern "C" int32_t fork_debug_effective_grid(int64_t U, int32_t G) { return fork_effective_grid(U, G); }

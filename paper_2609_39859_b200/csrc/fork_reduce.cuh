@@ -92,6 +92,24 @@ __device__ __forceinline__ Part part_merge(const Part& a, const Part& b) {
   return o;
 }
 
+/* Reduce one Part per lane over the warp; every lane returns the result.  Cheaper than a tree of
+   part_merge: one max-reduction, ONE rebase per lane, then plain sums (fixed shape, deterministic). */
+__device__ __forceinline__ Part part_warp_reduce(const Part& p) {
+  float M = p.m;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+  float s, t;
+  part_rebase(p, M, s, t);
+  int idx = (p.m == M) ? p.idx : kIdxNone;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    s += __shfl_xor_sync(0xffffffffu, s, o);
+    t += __shfl_xor_sync(0xffffffffu, t, o);
+    idx = min(idx, __shfl_xor_sync(0xffffffffu, idx, o));
+  }
+  return Part{M, s, t, idx};
+}
+
 __device__ __forceinline__ Part part_shfl_down(const Part& p, int delta) {
   Part q;
   q.m = __shfl_down_sync(0xffffffffu, p.m, delta);
@@ -107,132 +125,316 @@ template <int NT>
 __device__ __forceinline__ Part part_block_reduce(Part p, Part* sh) {
   constexpr int NW = NT / 32;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) p = part_merge(p, part_shfl_down(p, o));
+  p = part_warp_reduce(p);
   __syncthreads();                         /* previous users of sh are done */
   if (lane == 0) sh[warp] = p;
   __syncthreads();
-  if (warp == 0) {
-    p = (lane < NW) ? sh[lane] : part_empty();
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) p = part_merge(p, part_shfl_down(p, o));
-  }
+  if (warp == 0) p = part_warp_reduce((lane < NW) ? sh[lane] : part_empty());
   return p;
 }
 
 /* ------------------------------------------------------------------------------------------ */
-/* Per-thread streaming accumulator with a lazily raised reference max and 4 independent lanes. */
-template <bool WITH_T>
-struct Acc {
-  float m, nmL;          /* reference max and -m*L */
-  int idx;
-  float s[4], t[4];
+/* Per-thread streaming accumulator.
+ *
+ * The exponentials are taken against a per-thread REFERENCE that is not the running maximum: any
+ * reference within a few dozen nats of the true maximum gives the same relative precision in fp32,
+ * so the reference is set from the thread's first group of vectors and raised again only if the
+ * running maximum exceeds it by more than kRaiseNats (overflow guard) -- a branch that is uniform
+ * at the start of a segment and practically never taken afterwards, so warps do not diverge.
+ * The true maximum is tracked separately with packed NaN-propagating max instructions.  The index
+ * of its first occurrence is tracked per 128-bit vector, not per element: for each half of the
+ * packed maximum the accumulator remembers the vector in which it last rose (predicated selects,
+ * no branch).  Vectors of different threads are disjoint and ordered, so "lowest vector start"
+ * orders candidates exactly; the Part therefore carries the START of the winning vector in `idx`
+ * and whoever finalises the row reads those few elements once to find the exact position.
+ * `part()` re-expresses (s, t) against the thread's true maximum.                                  */
+constexpr float kRaiseNats = 32.f;
 
-  __device__ __forceinline__ void init() {
-    m = -INFINITY; nmL = INFINITY; idx = kIdxNone;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) { s[j] = 0.f; t[j] = 0.f; }
+/* lo/hi halves of a that are greater than b's select `code` into g_lo / g_hi */
+__device__ __forceinline__ void track_rise_bf16x2(uint32_t a, uint32_t b, int code, int& g_lo, int& g_hi) {
+  asm("{\n\t.reg .pred p, q;\n\tsetp.gt.bf16x2 p|q, %2, %3;\n\tselp.s32 %0, %4, %0, p;\n\tselp.s32 %1, %4, %1, q;\n\t}"
+      : "+r"(g_lo), "+r"(g_hi) : "r"(a), "r"(b), "r"(code));
+}
+__device__ __forceinline__ bool any_gt_bf16x2(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("{\n\t.reg .pred p, q;\n\tsetp.gt.bf16x2 p|q, %1, %2;\n\tor.pred p, p, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r) : "r"(a), "r"(b));
+  return r != 0;
+}
+
+template <typename T, bool WITH_T, bool CLAMP>
+struct Acc;
+
+/* Shared arithmetic: four accumulator lanes held as two f32x2 pairs, so that y = x*L - ref*L,
+   s += e and t += y*e each take ONE packed instruction (fma.rn.f32x2 / add.rn.f32x2, sm_100)
+   per pair of logits; the two exp2 of a pair stay scalar (MUFU has no packed form). */
+template <bool WITH_T>
+struct AccCore {
+  float ref;                   /* reference, -inf before the first group */
+  float2 nrefL2;               /* (-ref*L, -ref*L) */
+  float2 s2[2], t2[2];
+
+  __device__ __forceinline__ void init_core() {
+    ref = -INFINITY; nrefL2 = make_float2(INFINITY, INFINITY);
+    s2[0] = s2[1] = t2[0] = t2[1] = make_float2(0.f, 0.f);
   }
-  /* raise the reference to newm (> m): s *= w, t = w (t + d s) with d = (m-newm) L */
-  __device__ __forceinline__ void raise(float newm) {
-    if (m <= kClamp) {
+  __device__ __forceinline__ void rescale(float newref) {
+    if (ref <= kClamp) {                     /* nothing but -inf so far: weight 0 (NaN is kept) */
 #pragma unroll
-      for (int j = 0; j < 4; ++j) { s[j] *= 0.f; if (WITH_T) t[j] *= 0.f; }
+      for (int j = 0; j < 2; ++j) {
+        s2[j].x *= 0.f; s2[j].y *= 0.f;
+        if (WITH_T) { t2[j].x *= 0.f; t2[j].y *= 0.f; }
+      }
     } else {
-      float d = (m - newm) * kLog2e;
-      float w = ex2_approx(d);
+      const float d = (ref - newref) * kLog2e;
+      const float w = ex2_approx(d);
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        if (WITH_T) t[j] = w * fmaf(d, s[j], t[j]);
-        s[j] *= w;
+      for (int j = 0; j < 2; ++j) {
+        if (WITH_T) { t2[j].x = w * fmaf(d, s2[j].x, t2[j].x); t2[j].y = w * fmaf(d, s2[j].y, t2[j].y); }
+        s2[j].x *= w; s2[j].y *= w;
       }
     }
-    m = newm;
-    nmL = -newm * kLog2e;
+    ref = newref;
+    const float n = -newref * kLog2e;
+    nrefL2 = make_float2(n, n);
   }
-  __device__ __forceinline__ void add(int j, float x) {
-    float y = fmaf(x, kLog2e, nmL);
-    float e = ex2_approx(y);
-    s[j] += e;
-    if (WITH_T) t[j] = fmaf(y, e, t[j]);
+  /* two logits into pair k */
+  __device__ __forceinline__ void add2(int k, float xa, float xb) {
+    const float2 y = __ffma2_rn(make_float2(xa, xb), make_float2(kLog2e, kLog2e), nrefL2);
+    const float2 e = make_float2(ex2_approx(y.x), ex2_approx(y.y));
+    s2[k] = __fadd2_rn(s2[k], e);
+    if (WITH_T) t2[k] = __ffma2_rn(y, e, t2[k]);
   }
-  /* one element (already clamped), at vocabulary index i; used for ragged tails */
-  __device__ __forceinline__ void one(float x, int i) {
-    if (x > m) { idx = i; raise(x); }
-    add(0, x);
+  __device__ __forceinline__ void add1(float x) {
+    const float y = fmaf(x, kLog2e, nrefL2.x);
+    const float e = ex2_approx(y);
+    s2[0].x += e;
+    if (WITH_T) t2[0].x = fmaf(y, e, t2[0].x);
   }
-  __device__ __forceinline__ Part part() const {
-    Part p;
-    p.m = m; p.idx = idx;
-    p.s = (s[0] + s[1]) + (s[2] + s[3]);
-    p.t = WITH_T ? (t[0] + t[1]) + (t[2] + t[3]) : 0.f;
-    return p;
+  /* (s, t) re-expressed against the true maximum m >= ref */
+  __device__ __forceinline__ void totals(float m, float& ss, float& tt) const {
+    ss = (s2[0].x + s2[0].y) + (s2[1].x + s2[1].y);
+    tt = WITH_T ? (t2[0].x + t2[0].y) + (t2[1].x + t2[1].y) : 0.f;
+    if (ref != m && ref > kClamp) {
+      const float d = (ref - m) * kLog2e;
+      const float w = ex2_approx(d);
+      tt = WITH_T ? w * fmaf(d, ss, tt) : 0.f;
+      ss *= w;
+    }
   }
 };
 
-/* 8 bf16 logits starting at vocabulary index base */
-template <bool WITH_T>
-__device__ __forceinline__ void acc_vec(Acc<WITH_T>& a, uint4 v, int base, bf16_t) {
-  v.x = max_nan_bf16x2(v.x, kClampBf16x2);
-  v.y = max_nan_bf16x2(v.y, kClampBf16x2);
-  v.z = max_nan_bf16x2(v.z, kClampBf16x2);
-  v.w = max_nan_bf16x2(v.w, kClampBf16x2);
-  const float x0 = bf16_lo(v.x), x1 = bf16_hi(v.x), x2 = bf16_lo(v.y), x3 = bf16_hi(v.y);
-  const float x4 = bf16_lo(v.z), x5 = bf16_hi(v.z), x6 = bf16_lo(v.w), x7 = bf16_hi(v.w);
-  const float vmax = fmaxf(fmaxf(fmaxf(x0, x1), fmaxf(x2, x3)), fmaxf(fmaxf(x4, x5), fmaxf(x6, x7)));
-  if (vmax > a.m) {                      /* rare after the first few vectors */
-    int j = 7;
-    if (x6 == vmax) j = 6;
-    if (x5 == vmax) j = 5;
-    if (x4 == vmax) j = 4;
-    if (x3 == vmax) j = 3;
-    if (x2 == vmax) j = 2;
-    if (x1 == vmax) j = 1;
-    if (x0 == vmax) j = 0;
-    a.idx = base + j;
-    a.raise(vmax);
+/* ---- bf16: 8 logits per 128-bit vector --------------------------------------------------------
+ * CLAMP = false is the normal path: -inf logits are NOT clamped, so a thread that meets one ends
+ * with a NaN in t (0 * -inf) and redoes its own vectors with CLAMP = true (see stream_thread). */
+template <bool WITH_T, bool CLAMP>
+struct Acc<bf16_t, WITH_T, CLAMP> : AccCore<WITH_T> {
+  static constexpr int VEC = 8;
+  uint32_t thr2;               /* packed bf16x2 (ref + kRaiseNats): a running max above it raises the reference */
+  uint32_t pm;                 /* running packed maximum of the logits */
+  int g_lo, g_hi;              /* element index of the start of the vector where each half last rose */
+  float tail_m; int tail_idx;  /* scalar tail elements */
+
+  __device__ __forceinline__ void init() {
+    this->init_core();
+    thr2 = 0xFF80FF80u; pm = 0xFF80FF80u; g_lo = kIdxNone; g_hi = kIdxNone;
+    tail_m = -INFINITY; tail_idx = kIdxNone;
   }
-  a.add(0, x0); a.add(1, x1); a.add(2, x2); a.add(3, x3);
-  a.add(0, x4); a.add(1, x5); a.add(2, x6); a.add(3, x7);
+  __device__ __forceinline__ void raise(float newref) {
+    this->rescale(newref);
+    const uint32_t tb = __float_as_uint(newref + kRaiseNats) >> 16;
+    thr2 = tb | (tb << 16);
+  }
+  /* N vectors; vector j starts at vocabulary index base + j*stride.  track() touches every loaded
+     word (so the loads have landed once it has issued) and updates the maximum; accumulate() does
+     the exponentials. */
+  template <int N>
+  __device__ __forceinline__ void track(uint4 (&v)[N], int base, int stride) {
+#pragma unroll
+    for (int j = 0; j < N; ++j) {
+      if (CLAMP) {
+        v[j].x = max_nan_bf16x2(v[j].x, kClampBf16x2); v[j].y = max_nan_bf16x2(v[j].y, kClampBf16x2);
+        v[j].z = max_nan_bf16x2(v[j].z, kClampBf16x2); v[j].w = max_nan_bf16x2(v[j].w, kClampBf16x2);
+      }
+      const uint32_t vm = max_nan_bf16x2(max_nan_bf16x2(v[j].x, v[j].y), max_nan_bf16x2(v[j].z, v[j].w));
+      track_rise_bf16x2(vm, pm, base + j * stride, g_lo, g_hi);
+      pm = max_nan_bf16x2(pm, vm);
+    }
+    if (any_gt_bf16x2(pm, thr2)) raise(fmaxf(bf16_lo(pm), bf16_hi(pm)));
+  }
+  template <int N>
+  __device__ __forceinline__ void group(uint4 (&v)[N], int base, int stride) {
+    track<N>(v, base, stride);
+    accumulate<N>(v);
+  }
+  template <int N>
+  __device__ __forceinline__ void accumulate(const uint4 (&v)[N]) {
+#pragma unroll
+    for (int j = 0; j < N; ++j) {
+      this->add2(0, bf16_lo(v[j].x), bf16_hi(v[j].x)); this->add2(1, bf16_lo(v[j].y), bf16_hi(v[j].y));
+      this->add2(0, bf16_lo(v[j].z), bf16_hi(v[j].z)); this->add2(1, bf16_lo(v[j].w), bf16_hi(v[j].w));
+    }
+  }
+  /* one trailing element at vocabulary index idx (after all of the thread's vectors) */
+  __device__ __forceinline__ void one(float x, int idx) {
+    if (CLAMP) x = max_nan_f32(x, kClamp);
+    if (x > tail_m) { tail_m = x; tail_idx = idx; }
+    if (x > this->ref + kRaiseNats || this->ref == -INFINITY) raise(fmaxf(x, this->ref));
+    this->add1(x);
+  }
+  __device__ __forceinline__ Part part() const {
+    Part r;
+    const float ml = bf16_lo(pm), mh = bf16_hi(pm);
+    float m = fmaxf(ml, mh);
+    int idx = (ml == m && (mh != m || g_lo <= g_hi)) ? g_lo : g_hi;
+    if (g_lo == kIdxNone && g_hi == kIdxNone) m = -INFINITY;      /* no vector seen */
+    if (tail_m > m) { m = tail_m; idx = tail_idx; }
+    r.m = m; r.idx = idx;
+    this->totals(m, r.s, r.t);
+    return r;
+  }
+};
+
+/* ---- fp32: 4 logits per 128-bit vector -------------------------------------------------------- */
+template <bool WITH_T, bool CLAMP>
+struct Acc<float, WITH_T, CLAMP> : AccCore<WITH_T> {
+  static constexpr int VEC = 4;
+  float thr;
+  float fm;                    /* running maximum of the logits */
+  int g;                       /* element index of the start of the vector where fm last rose */
+  float tail_m; int tail_idx;
+
+  __device__ __forceinline__ void init() {
+    this->init_core();
+    thr = -INFINITY; fm = -INFINITY; g = kIdxNone;
+    tail_m = -INFINITY; tail_idx = kIdxNone;
+  }
+  __device__ __forceinline__ void raise(float newref) {
+    this->rescale(newref);
+    thr = newref + kRaiseNats;
+  }
+  template <int N>
+  __device__ __forceinline__ void track(uint4 (&v)[N], int base, int stride) {
+#pragma unroll
+    for (int j = 0; j < N; ++j) {
+      if (CLAMP) {
+        v[j].x = __float_as_uint(max_nan_f32(__uint_as_float(v[j].x), kClamp));
+        v[j].y = __float_as_uint(max_nan_f32(__uint_as_float(v[j].y), kClamp));
+        v[j].z = __float_as_uint(max_nan_f32(__uint_as_float(v[j].z), kClamp));
+        v[j].w = __float_as_uint(max_nan_f32(__uint_as_float(v[j].w), kClamp));
+      }
+      const float vm = fmaxf(fmaxf(__uint_as_float(v[j].x), __uint_as_float(v[j].y)),
+                             fmaxf(__uint_as_float(v[j].z), __uint_as_float(v[j].w)));
+      g = (vm > fm) ? (base + j * stride) : g;
+      fm = fmaxf(fm, vm);
+    }
+    if (fm > thr) raise(fm);
+  }
+  template <int N>
+  __device__ __forceinline__ void accumulate(const uint4 (&v)[N]) {
+#pragma unroll
+    for (int j = 0; j < N; ++j) {
+      this->add2(0, __uint_as_float(v[j].x), __uint_as_float(v[j].y));
+      this->add2(1, __uint_as_float(v[j].z), __uint_as_float(v[j].w));
+    }
+  }
+  template <int N>
+  __device__ __forceinline__ void group(uint4 (&v)[N], int base, int stride) {
+    track<N>(v, base, stride);
+    accumulate<N>(v);
+  }
+  __device__ __forceinline__ void one(float x, int idx) {
+    if (CLAMP) x = max_nan_f32(x, kClamp);
+    if (x > tail_m) { tail_m = x; tail_idx = idx; }
+    if (x > this->ref + kRaiseNats || this->ref == -INFINITY) raise(fmaxf(x, this->ref));
+    this->add1(x);
+  }
+  __device__ __forceinline__ Part part() const {
+    Part r;
+    float m = (g == kIdxNone) ? -INFINITY : fm;
+    int idx = g;
+    if (tail_m > m) { m = tail_m; idx = tail_idx; }
+    r.m = m; r.idx = idx;
+    this->totals(m, r.s, r.t);
+    return r;
+  }
+};
+
+__device__ __forceinline__ bool part_is_finite(const Part& p) { return isfinite(p.s) && isfinite(p.t); }
+
+/* The exact position of the row maximum M, given the start `idx` of the vector that holds its
+   first occurrence (or the exact position): look at one vector's worth of elements.  All loads are
+   issued before any comparison (one 128-bit load when the window is aligned), because this sits
+   on the critical path at the end of a step. */
+template <typename T>
+__device__ __forceinline__ int resolve_index(const T* row, int idx, int V, float M) {
+  constexpr int VEC = 16 / (int)sizeof(T);
+  if (idx < 0 || idx >= V) return 0;
+  float x[VEC];
+  if (idx + VEC <= V && (reinterpret_cast<uintptr_t>(row + idx) & 15u) == 0) {
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(row + idx));
+    if (sizeof(T) == 2) {
+      x[0] = bf16_lo(v.x); x[1] = bf16_hi(v.x); x[2 % VEC] = bf16_lo(v.y); x[3 % VEC] = bf16_hi(v.y);
+      x[4 % VEC] = bf16_lo(v.z); x[5 % VEC] = bf16_hi(v.z); x[6 % VEC] = bf16_lo(v.w); x[7 % VEC] = bf16_hi(v.w);
+    } else {
+      x[0] = __uint_as_float(v.x); x[1] = __uint_as_float(v.y); x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) x[j] = (idx + j < V) ? to_f32(row[idx + j]) : __int_as_float(0x7fc00000);
+  }
+  int best = idx;
+#pragma unroll
+  for (int j = VEC - 1; j >= 0; --j)
+    if (max_nan_f32(x[j], kClamp) == M) best = idx + j;
+  return best;
 }
 
-/* 4 fp32 logits starting at vocabulary index base */
-template <bool WITH_T>
-__device__ __forceinline__ void acc_vec(Acc<WITH_T>& a, uint4 v, int base, float) {
-  const float x0 = max_nan_f32(__uint_as_float(v.x), kClamp), x1 = max_nan_f32(__uint_as_float(v.y), kClamp);
-  const float x2 = max_nan_f32(__uint_as_float(v.z), kClamp), x3 = max_nan_f32(__uint_as_float(v.w), kClamp);
-  const float vmax = fmaxf(fmaxf(x0, x1), fmaxf(x2, x3));
-  if (vmax > a.m) {
-    int j = 3;
-    if (x2 == vmax) j = 2;
-    if (x1 == vmax) j = 1;
-    if (x0 == vmax) j = 0;
-    a.idx = base + j;
-    a.raise(vmax);
-  }
-  a.add(0, x0); a.add(1, x1); a.add(2, x2); a.add(3, x3);
-}
-
-/* Stream elements [e0,e1) of one row with 128-bit loads; e0 is a multiple of the vector width and
-   the row base is 16-byte aligned.  Threads take vectors tid, tid+NT, ... so each thread sees
-   ascending indices (strict '>' then keeps the lowest arg-max). */
-template <typename T, bool WITH_T, int NT, int UNROLL>
-__device__ __forceinline__ void stream_direct(Acc<WITH_T>& a, const T* row, int e0, int e1) {
+/* One thread's share of elements [e0,e1) of a row, read with 128-bit loads straight from global
+   memory: vectors tid, tid+NT, tid+2NT, ... (ascending indices), in groups of UNROLL; the thread
+   with `tail` also takes the fewer-than-a-vector trailing elements.  e0 is a multiple of the vector
+   width and the row base is 16-byte aligned. */
+template <typename T, bool WITH_T, bool CLAMP, int NT, int UNROLL>
+__device__ __forceinline__ Part stream_thread_once(const T* row, int e0, int e1, int tid, bool tail) {
+  Acc<T, WITH_T, CLAMP> a;
+  a.init();
   constexpr int VEC = 16 / (int)sizeof(T);
   const uint4* p = reinterpret_cast<const uint4*>(row + e0);
   const int nvec = (e1 - e0) / VEC;
-  int i = threadIdx.x;
+  int i = tid;
   for (; i + (UNROLL - 1) * NT < nvec; i += UNROLL * NT) {
     uint4 v[UNROLL];
 #pragma unroll
     for (int j = 0; j < UNROLL; ++j) v[j] = ld_stream(p + i + j * NT);
-#pragma unroll
-    for (int j = 0; j < UNROLL; ++j) acc_vec(a, v[j], e0 + (i + j * NT) * VEC, T{});
+    a.template group<UNROLL>(v, e0 + i * VEC, NT * VEC);
   }
-  for (; i < nvec; i += NT) acc_vec(a, ld_stream(p + i), e0 + i * VEC, T{});
-  if (threadIdx.x == 0) {                                  /* fewer than VEC trailing elements */
-    for (int e = e0 + nvec * VEC; e < e1; ++e) a.one(max_nan_f32(to_f32(row[e]), kClamp), e);
+  for (; i < nvec; i += NT) {
+    uint4 v[1];
+    v[0] = ld_stream(p + i);
+    a.template group<1>(v, e0 + i * VEC, NT * VEC);
   }
+  if (tail) {
+    for (int e = e0 + nvec * VEC; e < e1; ++e) a.one(to_f32(row[e]), e);
+  }
+  return a.part();
+}
+
+/* The same share again with -inf clamped, for a thread whose unclamped pass came out non-finite
+   (it met a -inf logit, or the row really holds NaN / +inf and will be flagged by the finaliser). */
+template <typename T, bool WITH_T, int NT>
+__device__ __noinline__ Part stream_thread_clamped(const T* row, int e0, int e1, int tid, bool tail) {
+  return stream_thread_once<T, WITH_T, true, NT, 1>(row, e0, e1, tid, tail);
+}
+
+/* `sticky` remembers that this thread has met a -inf before and starts clamped from then on. */
+template <typename T, bool WITH_T, int NT, int UNROLL>
+__device__ __forceinline__ Part stream_thread(const T* row, int e0, int e1, int tid, bool tail, bool& sticky) {
+  if (!sticky) {
+    const Part pt = stream_thread_once<T, WITH_T, false, NT, UNROLL>(row, e0, e1, tid, tail);
+    if (part_is_finite(pt)) return pt;
+    sticky = true;
+  }
+  return stream_thread_clamped<T, WITH_T, NT>(row, e0, e1, tid, tail);
 }
 
 /* ------------------------------------------------------------------------------------------ */
