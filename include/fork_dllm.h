@@ -125,6 +125,30 @@ fork_status fork_step(const fork_step_args* args, void* workspace, size_t worksp
 fork_status fork_logprob(const fork_logprob_args* args, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * fork_step without a workspace argument, for callers that have no device memory to give and
+ * cannot allocate any.  (The paper has no counterpart of this entry point; it exists for
+ * deployment.)  Typical callers: an inference server whose memory pool already owns the whole
+ * device, so that a cudaMalloc made on its behalf would fail or fragment the pool; and code on a
+ * latency-critical path, where the implicit device synchronisation of cudaMalloc / cudaFree is not
+ * acceptable.  This call allocates nothing and frees nothing, neither with the CUDA runtime nor
+ * through any library: the scratch is a fixed array of FORK_STATIC_SCRATCH_BYTES inside the library's
+ * device image (every GPU that loads the library holds that much until the process exits).
+ *
+ *   - Same arguments, results and asynchrony as fork_step.
+ *   - Batches whose scratch need, fork_workspace_bytes(B, Lt), exceeds FORK_STATIC_SCRATCH_BYTES are
+ *     rejected with FORK_ERR_WORKSPACE before anything is launched (B*Lt up to about 50,000
+ *     positions fits).
+ *   - The first call on each device looks up the array's device address (one cudaGetSymbolAddress,
+ *     with that device current) and caches it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which simply keeps what the previous call left:
+ *     the step's first kernel re-initialises everything it reads (row list, offsets, ticket
+ *     counters are cleared), so back-to-back calls on one stream are fine, but two calls that can
+ *     overlap on the GPU (different streams, or different threads without ordering) race on it.
+ */
+#define FORK_STATIC_SCRATCH_BYTES (2u * 1024u * 1024u)
+fork_status fork_step_static(const fork_step_args* args, void* stream);
+
+/*
  * Model-forward callback of the decode loop: must enqueue on `stream` the work that fills
  * `logits_out` (the buffer given as proto->logits) for the live positions of step `step`,
  * given the current device-side tokens / mask / block cursors.  Returns 0 on success.

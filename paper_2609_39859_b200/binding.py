@@ -48,7 +48,7 @@ class fork_logprob_args(C.Structure):
 fork_logits_fn = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                              C.c_void_p, C.c_void_p)
 
-EXPORTS = ("fork_workspace_bytes", "fork_step", "fork_logprob", "fork_decode_loop", "fork_staging_bytes",
+EXPORTS = ("fork_workspace_bytes", "fork_step", "fork_step_static", "fork_logprob", "fork_decode_loop", "fork_staging_bytes",
            "fork_step_host", "fork_device_status", "fork_status_string", "fork_set_tuning",
            "fork_kernel_launches", "fork_set_timing_events")
 
@@ -72,6 +72,8 @@ def lib():
     L.fork_workspace_bytes.argtypes = [C.c_int32, C.c_int32]
     L.fork_step.restype = C.c_int
     L.fork_step.argtypes = [C.POINTER(fork_step_args), C.c_void_p, C.c_size_t, C.c_void_p]
+    L.fork_step_static.restype = C.c_int
+    L.fork_step_static.argtypes = [C.POINTER(fork_step_args), C.c_void_p]
     L.fork_logprob.restype = C.c_int
     L.fork_logprob.argtypes = [C.POINTER(fork_logprob_args), C.c_void_p, C.c_size_t, C.c_void_p]
     L.fork_decode_loop.restype = C.c_int
@@ -191,6 +193,20 @@ def fork_step(st: ForkState, logits: torch.Tensor, blk_lo: torch.Tensor, blk_hi:
     rc = lib().fork_step(C.byref(a), C.c_void_p(st.ws_ptr), st.ws_bytes, _stream_ptr(stream))
     if rc != FORK_OK:
         raise ForkError(rc, "fork_step")
+
+
+FORK_STATIC_SCRATCH_BYTES = 2 * 1024 * 1024
+
+
+def fork_step_static(st: ForkState, logits: torch.Tensor, blk_lo: torch.Tensor, blk_hi: torch.Tensor,
+                     threshold: float, step: int = 0, pos0: int = 0, stream=None) -> None:
+    """fork_step on the library's built-in scratch: for callers that cannot allocate device memory
+    (a server whose pool owns the device, a latency-critical path).  `st.workspace` is not used.
+    Raises ForkError(FORK_ERR_WORKSPACE) when the batch needs more than FORK_STATIC_SCRATCH_BYTES."""
+    a = make_step_args(st, logits, blk_lo, blk_hi, threshold, step, pos0)
+    rc = lib().fork_step_static(C.byref(a), _stream_ptr(stream))
+    if rc != FORK_OK:
+        raise ForkError(rc, "fork_step_static")
 
 
 def fork_logprob(logits: torch.Tensor, tokens: torch.Tensor, select: torch.Tensor, st: ForkState, pos0: int = 0,

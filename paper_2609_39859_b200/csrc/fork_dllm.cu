@@ -1159,6 +1159,42 @@ extern "C" fork_status fork_device_status(const void* ws, uint32_t* host_out, vo
   return FORK_OK;
 }
 
+/* ---- fork_step on the library's own scratch ------------------------------------------------- */
+/* The scratch that fork_step normally receives from its caller, held instead in a fixed array that
+   is part of this library's device image: every GPU that loads the library carries these bytes
+   until the process exits.  In host code the NAME of a __device__ array is only a host-side
+   stand-in, not a device address, so the address the kernels get is looked up once per device with
+   cudaGetSymbolAddress and cached. */
+static __device__ __align__(256) unsigned char g_static_scratch[FORK_STATIC_SCRATCH_BYTES];
+static void* g_static_scratch_ptr[64];
+static std::atomic<int> g_static_scratch_ready[64];
+
+static fork_status static_scratch(void** out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FORK_ERR_CUDA;
+  if (!g_static_scratch_ready[dev].load(std::memory_order_acquire)) {
+    void* ptr = nullptr;                       /* set-up, once per device, with that device current */
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) return FORK_ERR_CUDA;
+    g_static_scratch_ptr[dev] = ptr;           /* every thread that gets here stores the same address */
+    g_static_scratch_ready[dev].store(1, std::memory_order_release);
+  }
+  *out = g_static_scratch_ptr[dev];
+  return FORK_OK;
+}
+
+extern "C" fork_status fork_step_static(const fork_step_args* a, void* stream) {
+  fork_status s = check_step_args(a, true);
+  if (s != FORK_OK) return s;
+  if (fork_workspace_bytes(a->B, a->Lt) > (size_t)FORK_STATIC_SCRATCH_BYTES) return FORK_ERR_WORKSPACE;
+  if (a->B == 0) return FORK_OK;
+  void* ws = nullptr;
+  s = static_scratch(&ws);
+  if (s != FORK_OK) return s;
+  /* nothing in the scratch has to survive from call to call: the active-set kernel rewrites the
+     row list and offsets and clears the per-sequence ticket counters at the start of every step */
+  return step_impl(a, a->blk_lo, a->blk_hi, ws, (cudaStream_t)stream);
+}
+
 /* ---- host-buffer entry point --------------------------------------------------------------- */
 struct StagingView {
   char* logits; int32_t* tokens; uint8_t* mask; int32_t* lo; int32_t* hi;
