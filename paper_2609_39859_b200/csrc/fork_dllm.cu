@@ -482,7 +482,7 @@ struct SegmentIter {
   }
   __device__ __forceinline__ bool next(Segment& s) {
     if (u >= u1) return false;
-    s.r = (int)(u / C);
+    s.r = (u < 0x7fffffffLL) ? (int)((uint32_t)u / (uint32_t)C) : (int)(u / C);
     const int c0 = (int)(u - (long long)s.r * C);
     long long uend = (long long)(s.r + 1) * C;
     if (uend > u1) uend = u1;
@@ -551,17 +551,15 @@ __global__ void __launch_bounds__(kNT, 4) reduce_select_kernel(ReduceParams p) {
  *              ticket and, if it was the last, applies the unmask rule for that sequence.
  * Every mbarrier wait is bounded: after kSpinLimit failed polls the thread records
  * FORK_DEV_TIMEOUT in the workspace header and leaves its loop.                                   */
-constexpr int kCW = 8;
-constexpr int kCT = kCW * 32;
-constexpr int kStageVecs = kCT * kUnroll;                  /* 128-bit vectors per stage */
-constexpr int kStageBytes = kStageVecs * 16;               /* 16 KB */
+constexpr int kMaxCW = 16;                                 /* consumer warps: 8 (two CTAs per SM) or 16 (one CTA per SM) */
 constexpr int kMail = 4;                                   /* mailbox depth (row segments in flight to the finaliser) */
 constexpr int kMaxStages = 13;
 constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr int ring_stage_bytes(int cw) { return cw * 32 * kUnroll * 16; }   /* 16 KB (8 warps) or 32 KB (16 warps) */
 
 struct RingSmem {
   unsigned long long full[kMaxStages], empty[kMaxStages], mfull[kMail], mempty[kMail];
-  Part mail[kMail][kCW];
+  Part mail[kMail][kMaxCW];
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -604,10 +602,13 @@ __device__ __forceinline__ void trace(int slot) {
 #define FORK_TRACE(slot)
 #endif
 
-template <typename T, int MODE>
-__global__ void __launch_bounds__((kCW + 2) * 32, 2) reduce_select_ring_kernel(ReduceParams p, int n_stages) {
+template <typename T, int MODE, int kCW>
+__global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_select_ring_kernel(ReduceParams p, int n_stages) {
   constexpr bool WITH_T = (MODE == kModeStep);
   constexpr int VEC = 16 / (int)sizeof(T);
+  constexpr int kCT = kCW * 32;                              /* consumer threads */
+  constexpr int kStageVecs = kCT * kUnroll;                  /* 128-bit vectors per stage */
+  constexpr int kStageBytes = kStageVecs * 16;
   extern __shared__ __align__(1024) unsigned char dyn_smem[];
   unsigned char* ring = dyn_smem;
   RingSmem& rs = *reinterpret_cast<RingSmem*>(dyn_smem + (size_t)n_stages * kStageBytes);
@@ -666,8 +667,9 @@ __global__ void __launch_bounds__((kCW + 2) * 32, 2) reduce_select_ring_kernel(R
     uint32_t s = 0, ph = 0, nseg = 0;                       /* ring slot, its phase, segments done */
     bool sticky = false;                                    /* this thread has met a -inf logit before */
 #ifdef FORK_EXP_TRACE
-    unsigned long long tw = 0, tt = 0, ta = 0, tn = 0;
+    unsigned long long tw = 0, tt = 0, ta = 0, tn = 0, tloop = 0, trow = 0, nrow = 0;
     const long long cstart = clock64();
+    long long cprev = cstart; bool prev_same_seg = false;
 #endif
     while (it.next(sg)) {
       Acc<T, WITH_T, false> a;
@@ -676,6 +678,7 @@ __global__ void __launch_bounds__((kCW + 2) * 32, 2) reduce_select_ring_kernel(R
       for (int voff = 0; voff < nvec; voff += kStageVecs) {
 #ifdef FORK_EXP_TRACE
         const long long c0 = clock64();
+        if (prev_same_seg) tloop += (unsigned long long)(c0 - cprev); else { trow += (unsigned long long)(c0 - cprev); nrow += 1; }
 #endif
         if (!mbar_wait(&rs.full[s], ph, p)) return;
 #ifdef FORK_EXP_TRACE
@@ -702,18 +705,24 @@ __global__ void __launch_bounds__((kCW + 2) * 32, 2) reduce_select_ring_kernel(R
           {
             const long long c3 = clock64();
             tw += (unsigned long long)(c1 - c0); tt += (unsigned long long)(c2 - c1); ta += (unsigned long long)(c3 - c2); tn += 1ull;
+            cprev = c3; prev_same_seg = true;
           }
 #endif
         } else {
-          if (!sticky) {
-            for (int i = ctid; i < nv; i += kCT) {
-              uint4 v[1];
-              v[0] = sp[i];
-              a.template group<1>(v, sg.e0 + (voff + i) * VEC, 0);
-            }
-          }
+          /* the last, partly filled stage of a segment: same unrolled code, vectors past the end
+             replaced by the clamp value (contributes 2^-huge = 0 and never wins the maximum
+             against a finite logit; an all -inf row is re-read by the finaliser anyway) */
+          uint4 v[kUnroll];
+#pragma unroll
+          for (int j = 0; j < kUnroll; ++j)
+            v[j] = (ctid + j * kCT < nv) ? sp[ctid + j * kCT] : neutral_vector(T{});
+          if (!sticky) a.template track<kUnroll>(v, sg.e0 + (voff + ctid) * VEC, kCT * VEC);
           __syncwarp();
           if (lane == 0) mbar_arrive(&rs.empty[s]);
+          if (!sticky) a.template accumulate<kUnroll>(v);
+#ifdef FORK_EXP_TRACE
+          { const long long c3 = clock64(); tw += (unsigned long long)(c1 - c0); ta += (unsigned long long)(c3 - c1); cprev = c3; prev_same_seg = true; }
+#endif
         }
 #else
         __syncwarp();
@@ -754,10 +763,16 @@ __global__ void __launch_bounds__((kCW + 2) * 32, 2) reduce_select_ring_kernel(R
       }
       if (ctid == 0) FORK_TRACE(7);
       ++nseg;
+#ifdef FORK_EXP_TRACE
+      prev_same_seg = false;
+#endif
     }
 #ifdef FORK_EXP_TRACE
     if (lane == 0 && warp == 3) {
+      unsigned smid; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+      g_trace[blockIdx.x][4] = smid;
       g_trace[blockIdx.x][12] = tw; g_trace[blockIdx.x][13] = tt; g_trace[blockIdx.x][14] = ta; g_trace[blockIdx.x][15] = tn;
+      g_trace[blockIdx.x][1] = tloop; g_trace[blockIdx.x][2] = trow; g_trace[blockIdx.x][3] = nrow;
       g_trace[blockIdx.x][11] = (unsigned long long)(clock64() - cstart);
     }
 #endif
@@ -835,17 +850,19 @@ using namespace forkd;
 static std::atomic<long long> g_launches{0};
 static std::atomic<int> g_tune[FORK_TUNE_COUNT_];
 
-static size_t ring_smem_bytes(int n_stages) { return (size_t)n_stages * kStageBytes + sizeof(RingSmem); }
+static size_t ring_smem_bytes(int n_stages, int cw) { return (size_t)n_stages * ring_stage_bytes(cw) + sizeof(RingSmem); }
 
-static void ring_config(int* ctas_per_sm, int* n_stages) {
+/* one CTA per SM with 16 consumer warps (default), or two with 8 each */
+static void ring_config(int* ctas_per_sm, int* n_stages, int* cw) {
   int per_sm = g_tune[FORK_TUNE_CTAS_PER_SM].load();
-  if (per_sm <= 0 || per_sm > 3) per_sm = 2;
+  if (per_sm != 2) per_sm = 1;
+  const int warps = (per_sm == 1) ? 16 : 8;
   int st = g_tune[FORK_TUNE_STAGES].load();
-  const int max_st = (int)((220 * 1024 / per_sm - sizeof(RingSmem) - 1024) / kStageBytes);
+  const int max_st = (int)((220 * 1024 / per_sm - sizeof(RingSmem) - 1024) / ring_stage_bytes(warps));
   if (st <= 0 || st > max_st) st = max_st;
   if (st > kMaxStages) st = kMaxStages;
   if (st < 2) st = 2;
-  *ctas_per_sm = per_sm; *n_stages = st;
+  *ctas_per_sm = per_sm; *n_stages = st; *cw = warps;
 }
 
 struct DeviceInfo { int sms = 0; int occ[2][2] = {{0, 0}, {0, 0}}; bool ring_ready = false; };
@@ -869,12 +886,13 @@ static bool device_info(DeviceInfo** out) {
     d.occ[0][1] = occupancy_of<bf16_t, kModeLogprob>();
     d.occ[1][0] = occupancy_of<float, kModeStep>();
     d.occ[1][1] = occupancy_of<float, kModeLogprob>();
-    const int max_dyn = (int)ring_smem_bytes(kMaxStages);
+    const int max_dyn = 220 * 1024;
+    auto allow = [&](const void* fn) { return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn) == cudaSuccess; };
     d.ring_ready =
-        cudaFuncSetAttribute(reduce_select_ring_kernel<bf16_t, kModeStep>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn) == cudaSuccess &&
-        cudaFuncSetAttribute(reduce_select_ring_kernel<bf16_t, kModeLogprob>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn) == cudaSuccess &&
-        cudaFuncSetAttribute(reduce_select_ring_kernel<float, kModeStep>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn) == cudaSuccess &&
-        cudaFuncSetAttribute(reduce_select_ring_kernel<float, kModeLogprob>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn) == cudaSuccess;
+        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeStep, 8>) && allow((const void*)reduce_select_ring_kernel<bf16_t, kModeLogprob, 8>) &&
+        allow((const void*)reduce_select_ring_kernel<float, kModeStep, 8>) && allow((const void*)reduce_select_ring_kernel<float, kModeLogprob, 8>) &&
+        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeStep, 16>) && allow((const void*)reduce_select_ring_kernel<bf16_t, kModeLogprob, 16>) &&
+        allow((const void*)reduce_select_ring_kernel<float, kModeStep, 16>) && allow((const void*)reduce_select_ring_kernel<float, kModeLogprob, 16>);
     if (!d.ring_ready) return false;
     d.sms = sms;
   }
@@ -885,8 +903,8 @@ static bool device_info(DeviceInfo** out) {
 static int grid_size(const DeviceInfo& d, int dtype, int mode, bool fast) {
   const int variant = g_tune[FORK_TUNE_VARIANT].load();
   if (fast && (variant == 0 || variant == 2)) {
-    int per, stages;
-    ring_config(&per, &stages);
+    int per, stages, cw;
+    ring_config(&per, &stages, &cw);
     return d.sms * per;
   }
   int per_sm = g_tune[FORK_TUNE_CTAS_PER_SM].load();
@@ -942,11 +960,11 @@ static cudaError_t launch_reduce(const ReduceParams& rp, int dtype, int mode, in
   return e;
 }
 
-template <typename T, int MODE>
+template <typename T, int MODE, int CW>
 static cudaError_t launch_ring(const ReduceParams& rp, int G, int n_stages, bool pdl, cudaStream_t st) {
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
-  cfg.gridDim = dim3(G); cfg.blockDim = dim3((kCW + 2) * 32); cfg.dynamicSmemBytes = ring_smem_bytes(n_stages);
+  cfg.gridDim = dim3(G); cfg.blockDim = dim3((CW + 2) * 32); cfg.dynamicSmemBytes = ring_smem_bytes(n_stages, CW);
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   if (pdl) {
@@ -954,7 +972,7 @@ static cudaError_t launch_ring(const ReduceParams& rp, int G, int n_stages, bool
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
   }
-  cudaError_t e = cudaLaunchKernelEx(&cfg, reduce_select_ring_kernel<T, MODE>, rp, n_stages);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, reduce_select_ring_kernel<T, MODE, CW>, rp, n_stages);
   if (e == cudaSuccess) g_launches.fetch_add(1);
   return e;
 }
@@ -968,14 +986,22 @@ static bool use_ring(const ReduceParams& rp) {
 static cudaError_t launch_reduce_inner(const ReduceParams& rp, int dtype, int mode, int G, cudaStream_t st) {
   const bool pdl = g_tune[FORK_TUNE_PDL].load() != 0;
   if (use_ring(rp)) {
-    int per_sm, n_stages;
-    ring_config(&per_sm, &n_stages);
-    if (dtype == FORK_BF16) {
-      if (mode == kModeStep) return launch_ring<bf16_t, kModeStep>(rp, G, n_stages, pdl, st);
-      return launch_ring<bf16_t, kModeLogprob>(rp, G, n_stages, pdl, st);
+    int per_sm, n_stages, cw;
+    ring_config(&per_sm, &n_stages, &cw);
+    if (cw == 16) {
+      if (dtype == FORK_BF16) {
+        if (mode == kModeStep) return launch_ring<bf16_t, kModeStep, 16>(rp, G, n_stages, pdl, st);
+        return launch_ring<bf16_t, kModeLogprob, 16>(rp, G, n_stages, pdl, st);
+      }
+      if (mode == kModeStep) return launch_ring<float, kModeStep, 16>(rp, G, n_stages, pdl, st);
+      return launch_ring<float, kModeLogprob, 16>(rp, G, n_stages, pdl, st);
     }
-    if (mode == kModeStep) return launch_ring<float, kModeStep>(rp, G, n_stages, pdl, st);
-    return launch_ring<float, kModeLogprob>(rp, G, n_stages, pdl, st);
+    if (dtype == FORK_BF16) {
+      if (mode == kModeStep) return launch_ring<bf16_t, kModeStep, 8>(rp, G, n_stages, pdl, st);
+      return launch_ring<bf16_t, kModeLogprob, 8>(rp, G, n_stages, pdl, st);
+    }
+    if (mode == kModeStep) return launch_ring<float, kModeStep, 8>(rp, G, n_stages, pdl, st);
+    return launch_ring<float, kModeLogprob, 8>(rp, G, n_stages, pdl, st);
   }
   if (dtype == FORK_BF16) {
     if (mode == kModeStep) return launch(reduce_select_kernel<bf16_t, kModeStep>, dim3(G), dim3(kNT), st, pdl, rp);

@@ -55,6 +55,9 @@ __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u 
 __device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
 
 struct bf16_t { uint16_t bits; };                   /* storage type tag for bf16 logits */
+/* a 128-bit vector of logits that changes nothing: every element is the clamp value (about -1e38) */
+__device__ __forceinline__ uint4 neutral_vector(bf16_t) { return make_uint4(0xFE96FE96u, 0xFE96FE96u, 0xFE96FE96u, 0xFE96FE96u); }
+__device__ __forceinline__ uint4 neutral_vector(float) { return make_uint4(0xFE960000u, 0xFE960000u, 0xFE960000u, 0xFE960000u); }
 __device__ __forceinline__ float to_f32(bf16_t v) { return __uint_as_float(((uint32_t)v.bits) << 16); }
 __device__ __forceinline__ float to_f32(float v) { return v; }
 
