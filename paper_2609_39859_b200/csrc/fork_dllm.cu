@@ -339,7 +339,7 @@ __device__ Part careful_row_warp(const T* row, int V, bool& bad) {
    Rows whose streamed result is not finite are re-read by the whole warp with the guarded routine. */
 template <typename T, bool WANT_INDEX>
 __device__ __forceinline__ RowOut finalize_rows_warp(const ReduceParams& p, const PartitionCtx& c, int b, int base,
-                                                     int r1, Part& merged, int& k) {
+                                                     int r1, Part& merged, int& k, int k_hint) {
   const int lane = threadIdx.x & 31;
   const int r = base + lane;
   const bool valid = r < r1;
@@ -347,7 +347,7 @@ __device__ __forceinline__ RowOut finalize_rows_warp(const ReduceParams& p, cons
   merged = part_empty();
   k = 0;
   int g0 = 0, nparts = 0;
-  if (valid) { k = p.rows[r].y; merged = merge_row_parts(p, c, r, g0, nparts); }
+  if (valid) { k = (k_hint >= 0) ? k_hint : p.rows[r].y; merged = merge_row_parts(p, c, r, g0, nparts); }
   unsigned many = __ballot_sync(0xffffffffu, valid && nparts > kLaneMergeMax);
   while (many) {                                             /* rows cut into very many parts: all lanes help */
     const int src = __ffs(many) - 1;
@@ -370,20 +370,31 @@ __device__ __forceinline__ RowOut finalize_rows_warp(const ReduceParams& p, cons
   return row_out_from(merged, bad);
 }
 
+/* What a finaliser can load about a sequence BEFORE its last part arrives (it idles until then):
+   the sequence's row range and this lane's position among its first 32 rows. */
+struct SeqHint { int r0, r1, k; };
+__device__ __forceinline__ SeqHint load_seq_hint(const ReduceParams& p, int b) {
+  SeqHint h;
+  h.r0 = p.seq_off[b]; h.r1 = p.seq_off[b + 1];
+  const int r = h.r0 + (int)(threadIdx.x & 31);
+  h.k = (r < h.r1) ? p.rows[r].y : -1;
+  return h;
+}
+
 /* The unmask rule for one sequence, run by one warp once every part of the sequence has arrived
    (Algorithm 2 lines 6-9): commit every live position whose confidence exceeds lambda, or the
    leftmost live position when none does; write tokens, mask and the per-token records. */
 template <typename T>
-__device__ void finalize_step_sequence(const ReduceParams& p, const PartitionCtx& c, int b) {
+__device__ void finalize_step_sequence(const ReduceParams& p, const PartitionCtx& c, int b, const SeqHint& h) {
   const int lane = threadIdx.x & 31;
-  const int r0 = p.seq_off[b], r1 = p.seq_off[b + 1];
+  const int r0 = h.r0, r1 = h.r1;
   const bool one_batch = (r1 - r0) <= 32;                    /* the usual case: results stay in registers */
   int any = 0;
   float4 keep = make_float4(0.f, 0.f, 0.f, 0.f);
   int keep_k = 0;
   for (int base = r0; base < r1; base += 32) {
     Part merged; int k;
-    const RowOut o = finalize_rows_warp<T, true>(p, c, b, base, r1, merged, k);
+    const RowOut o = finalize_rows_warp<T, true>(p, c, b, base, r1, merged, k, base == r0 ? h.k : -1);
     const int r = base + lane;
     if (r < r1) {
       const size_t at = (size_t)b * p.Lt + k;
@@ -430,13 +441,13 @@ __device__ void finalize_step_sequence(const ReduceParams& p, const PartitionCtx
 /* Scoring for one sequence by one warp: log q(token) = x_tok - m - ln s at every selected position
    and their sum (Section 3.2 of the paper: the likelihood terms of the ForkGRPO ratio). */
 template <typename T>
-__device__ void finalize_logprob_sequence(const ReduceParams& p, const PartitionCtx& c, int b) {
+__device__ void finalize_logprob_sequence(const ReduceParams& p, const PartitionCtx& c, int b, const SeqHint& h) {
   const int lane = threadIdx.x & 31;
-  const int r0 = p.seq_off[b], r1 = p.seq_off[b + 1];
+  const int r0 = h.r0, r1 = h.r1;
   float local = 0.f;
   for (int base = r0; base < r1; base += 32) {
     Part merged; int k;
-    const RowOut o = finalize_rows_warp<T, false>(p, c, b, base, r1, merged, k);
+    const RowOut o = finalize_rows_warp<T, false>(p, c, b, base, r1, merged, k, base == r0 ? h.k : -1);
     const int r = base + lane;
     if (r < r1) {
       const size_t at = (size_t)b * p.Lt + k;
@@ -461,10 +472,9 @@ __device__ void finalize_logprob_sequence(const ReduceParams& p, const Partition
 
 /* Lane 0 of the calling warp publishes one part of row r (sequence b) and takes a ticket; returns
    (to every lane) whether this was the last part the sequence was waiting for. */
-__device__ __forceinline__ bool publish_part(const ReduceParams& p, const Part& part, int r, int g, int b) {
+__device__ __forceinline__ bool publish_part(const ReduceParams& p, const Part& part, int r, int g, int b, int want) {
   int last = 0;
   if ((threadIdx.x & 31) == 0) {
-    const int want = p.expected[b];
     p.parts[r + g] = make_float4(part.m, part.s, part.t, __int_as_float(part.idx));
     int old;                                 /* release our part, acquire everybody else's */
     asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(p.ticket + b) : "memory");
@@ -528,10 +538,11 @@ __global__ void __launch_bounds__(kNT, 4) reduce_select_kernel(ReduceParams p) {
       part = careful_segment<T, kNT>(row, sg.e0, sg.e1, sm.parts, sm.fl, bad);
     }
     if (threadIdx.x < 32) {
-      const bool last = publish_part(p, part, sg.r, g, bk.x);
+      const bool last = publish_part(p, part, sg.r, g, bk.x, p.expected[bk.x]);
       if (last) {                                           /* every part of sequence b has been delivered */
-        if (MODE == kModeStep) finalize_step_sequence<T>(p, c, bk.x);
-        else finalize_logprob_sequence<T>(p, c, bk.x);
+        const SeqHint h = load_seq_hint(p, bk.x);
+        if (MODE == kModeStep) finalize_step_sequence<T>(p, c, bk.x, h);
+        else finalize_logprob_sequence<T>(p, c, bk.x, h);
       }
     }
   }
@@ -782,20 +793,23 @@ __global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_sel
   /* ---------------- finaliser ---------------- */
   uint32_t nseg = 0;
   while (it.next(sg)) {
+    /* everything that does not depend on the parts is fetched while the consumers still stream */
+    const int b = p.rows[sg.r].x;
+    const int want = p.expected[b];
+    const SeqHint h = load_seq_hint(p, b);
     const uint32_t d = nseg % kMail, ph = (nseg / kMail) & 1u;
     if (!mbar_wait(&rs.mfull[d], ph, p)) return;
     Part pt = (lane < kCW) ? rs.mail[d][lane] : part_empty();
     __syncwarp();
     if (lane == 0) mbar_arrive(&rs.mempty[d]);
     pt = part_warp_reduce(pt);
-    const int b = p.rows[sg.r].x;
     if (lane == 0) FORK_TRACE(8);
 #ifndef FORK_EXP_NO_PUBLISH
-    if (publish_part(p, pt, sg.r, g, b)) {
+    if (publish_part(p, pt, sg.r, g, b, want)) {
       if (lane == 0) FORK_TRACE(9);
 #ifndef FORK_EXP_NO_FINALIZE
-      if (MODE == kModeStep) finalize_step_sequence<T>(p, c, b);
-      else finalize_logprob_sequence<T>(p, c, b);
+      if (MODE == kModeStep) finalize_step_sequence<T>(p, c, b, h);
+      else finalize_logprob_sequence<T>(p, c, b, h);
 #endif
       if (lane == 0) FORK_TRACE(11);
     }
@@ -852,10 +866,10 @@ static std::atomic<int> g_tune[FORK_TUNE_COUNT_];
 
 static size_t ring_smem_bytes(int n_stages, int cw) { return (size_t)n_stages * ring_stage_bytes(cw) + sizeof(RingSmem); }
 
-/* one CTA per SM with 16 consumer warps (default), or two with 8 each */
+/* two CTAs per SM with 8 consumer warps each (default), or one with 16 */
 static void ring_config(int* ctas_per_sm, int* n_stages, int* cw) {
   int per_sm = g_tune[FORK_TUNE_CTAS_PER_SM].load();
-  if (per_sm != 2) per_sm = 1;
+  if (per_sm != 1) per_sm = 2;
   const int warps = (per_sm == 1) ? 16 : 8;
   int st = g_tune[FORK_TUNE_STAGES].load();
   const int max_st = (int)((220 * 1024 / per_sm - sizeof(RingSmem) - 1024) / ring_stage_bytes(warps));
