@@ -37,6 +37,9 @@ METRIC = "masked positions/s (fork_step; HBM GB/s and fraction of peak in `roofl
 UNIT = "positions/s"
 L2_BYTES = 126 * 1024 * 1024
 NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the streaming kernel, from the committed
+# ncu captures (profiles/reduce_select_ring_bf16_b8_and_passk.md)
+NCU_TRAFFIC_BYTES = {"b8": 64_889_344, "passk": 522_844_928}
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -472,7 +475,7 @@ def main():
         "gpu_launches": int(r["launches"]),
         "roofline": {"bound": "hbm", "kernel": "reduce_select_kernel<bf16,step>" if w.es == 2 else "reduce_select_kernel<f32,step>",
                      "achieved": kern_gbs, "peak": peak, "unit": "GB/s", "frac": kern_gbs / peak,
-                     "peak_source": peak_src, "traffic": None,
+                     "peak_source": peak_src, "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
                      "algorithmic_bytes_per_launch": rows * row_bytes, "kernel_ms": r["kernel_ms"],
                      "whole_step_gbs": step_gbs, "whole_step_frac": step_gbs / peak,
                      "frac_of_8TBs_nominal": kern_gbs / NOMINAL_HBM_GBS},
