@@ -156,6 +156,35 @@ def test_nonfinite_rows(dtype):
     assert g["is_fallback"][0] == 1 and g["fallback_pos"][0] == 0 and g["mask"][0].tolist() == [0, 1, 1, 1]
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_banned_token_ranges_of_minus_inf_at_full_vocabulary(dtype):
+    """Many rows with ranges of -inf logits (banned tokens) at V=126464+3 on a padded pitch: the
+    streaming path first runs unclamped, the threads that met -inf redo their vectors clamped and
+    stay clamped for later rows; several stages, a partly filled last stage and a scalar tail."""
+    rng = np.random.default_rng(21)
+    B, Lt, V, pitch = 3, 24, 126467, 126472
+    x = (rng.standard_normal((B, Lt, V)) * 3).astype(np.float32)
+    x[np.arange(B)[:, None], np.arange(Lt)[None, :], rng.integers(0, V, size=(B, Lt))] += 25.0
+    for b in range(B):
+        for l in range(Lt):
+            kind = (b * Lt + l) % 4
+            if kind == 0:
+                x[b, l, :2000] = -np.inf                       # reserved ids at the start
+            elif kind == 1:
+                a = int(rng.integers(0, V - 30000))
+                x[b, l, a:a + 30000] = -np.inf                 # a long range in the middle
+            elif kind == 2:
+                x[b, l, V - 300:] = -np.inf                    # padding ids at the end, incl. the scalar tail
+    xs = x if dtype == "f32" else fs.f32_to_bf16_bits(x)
+    buf = np.full((B, Lt, pitch), np.nan if dtype == "f32" else 0x7FC0, xs.dtype)
+    buf[..., :V] = xs
+    lt = to_torch_logits(buf)[..., :V]
+    mask = np.ones((B, Lt), np.uint8)
+    g, o = run_both(xs, mask, np.zeros(B, np.int32), np.full(B, Lt, np.int32), 0.9, logits_t=lt)
+    compare_step_state(g, o)
+    assert (g["row_status"] == 0).all()
+
+
 def test_threshold_extremes_and_strictness():
     rng = np.random.default_rng(4)
     x = make_rows(rng, (3, 12), 300, "f32")
