@@ -330,6 +330,39 @@ def time_logprob(device, peak):
             "positions_per_s": rows / (ms * 1e-3), "ms": ms, "hbm_gbs": gbs, "frac_of_measured_peak": gbs / peak}
 
 
+def loop_stats(device):
+    """Full semi-autoregressive decode loops of the configurations (generator as the model): model
+    evaluations used versus tokens, share of tokens committed at fallback steps, live rows."""
+    import torch
+    import fork_synth as fs
+    import paper_2609_39859_b200 as pkg
+    out = []
+    for name, lams in (("tiny", None), ("b8", None), ("passk", None), ("sweep", "all")):
+        w = fs.workload(name)
+        for lam in (w.thresholds if lams == "all" else (w.threshold,)):
+            cfg = w.cfg()
+            tdt = torch.bfloat16 if w.dtype == fs.BF16 else torch.float32
+            logits = torch.empty((w.B, w.Lt, w.V), dtype=tdt, device=device)
+            fs.cuda_canary(logits.data_ptr(), logits.numel(), w.dtype, torch.cuda.current_stream().cuda_stream)
+            st = pkg.ForkState(w.B, w.Lt, device=device)
+            prov = fs.Provider(cfg, w.Lt * w.V, w.V, 0, w.Lt)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            rc, steps = pkg.fork_decode_loop(st, logits, w.block_len, 0, w.Lt, prov.address, prov.ctx, lam, 100000)
+            torch.cuda.synchronize()
+            dt = time.perf_counter() - t0
+            prov.close()
+            h = st.host()
+            out.append({"workload": name, "threshold": lam, "B": w.B, "tokens_per_sequence": w.Lt,
+                        "steps_taken": steps, "nfe_mean": float(h["nfe"].mean()),
+                        "fallback_token_share": float(h["commit_fallback"].mean()),
+                        "tokens_committed": int((h["commit_step"] >= 0).sum()),
+                        "wall_ms_incl_generator": dt * 1e3})
+            del logits
+            torch.cuda.empty_cache()
+    return out
+
+
 def cpu_baseline(w, seed, target_cpu_seconds=12.0):
     """The oracle, as it stands, on one full-block step's rows generated on the host."""
     import fork_synth as fs
@@ -412,6 +445,7 @@ def main():
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
     ap.add_argument("--workload", default="b8", choices=["b8", "passk", "sweep"])
     ap.add_argument("--no-extras", action="store_true", help="skip the other shapes, e2e and the CPU baseline")
+    ap.add_argument("--loops", action="store_true", help="also run the full decode loops of the configurations and report their statistics")
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of one CUDA graph")
     ap.add_argument("--variant", type=int, default=0, help="0 auto, 1 direct loads, 2 bulk-copy shared-memory ring")
     ap.add_argument("--ctas-per-sm", type=int, default=0)
@@ -473,7 +507,7 @@ def main():
         "launch": ("one CUDA graph of the K steps" if r["graph"] else "plain stream launches"),
         "hbm_gbs_per_gpu": step_gbs, "frac_of_8TBs_nominal": step_gbs / NOMINAL_HBM_GBS,
         "gpu_launches": int(r["launches"]),
-        "roofline": {"bound": "hbm", "kernel": "reduce_select_kernel<bf16,step>" if w.es == 2 else "reduce_select_kernel<f32,step>",
+        "roofline": {"bound": "hbm", "kernel": "reduce_select_ring_kernel<%s,step,8>" % ("bf16" if w.es == 2 else "f32"),
                      "achieved": kern_gbs, "peak": peak, "unit": "GB/s", "frac": kern_gbs / peak,
                      "peak_source": peak_src, "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
                      "algorithmic_bytes_per_launch": rows * row_bytes, "kernel_ms": r["kernel_ms"],
@@ -509,6 +543,8 @@ def main():
         also.append(time_logprob(device, peak))
         out["also"] = also
         out["cpu_baseline"] = cpu_baseline(w, seed)
+        if args.loops:
+            out["loops"] = loop_stats(device)
     if rank == 0:
         print(json.dumps(out))
     if world > 1:
