@@ -151,6 +151,10 @@ __device__ __forceinline__ void seq_window(const SetupParams& p, int b, int& lo,
 constexpr int kSetupMaxB = 4096;     /* sequences whose counts fit in shared memory (more: counts go through global memory) */
 
 __global__ void __launch_bounds__(kSetupNT, 1) active_set_kernel(SetupParams p) {
+  /* with programmatic dependent launch this grid may already be resident while the kernel before
+     it in the stream (normally the previous step) is still running: nothing is read or written
+     before that kernel has completed; the streaming kernel of this step may be made resident now */
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;");
   __shared__ int sh_cnt[kSetupMaxB + 1];          /* sh_cnt[b+1] = live rows of b, then their inclusive scan */
   __shared__ int sh_warp[kSetupNT / 32];
@@ -634,6 +638,7 @@ __global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_sel
   }
   __syncthreads();
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;");          /* the next kernel in the stream may take free SM slots */
   const int R = p.hdr->R;
   if (R <= 0) return;
   if (threadIdx.x == 0) FORK_TRACE(1);
@@ -998,7 +1003,7 @@ static bool use_ring(const ReduceParams& rp) {
 }
 
 static cudaError_t launch_reduce_inner(const ReduceParams& rp, int dtype, int mode, int G, cudaStream_t st) {
-  const bool pdl = g_tune[FORK_TUNE_PDL].load() != 0;
+  const bool pdl = g_tune[FORK_TUNE_PDL].load() >= 0;
   if (use_ring(rp)) {
     int per_sm, n_stages, cw;
     ring_config(&per_sm, &n_stages, &cw);
@@ -1076,7 +1081,7 @@ static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const i
   sp.B = a->B; sp.Lt = a->Lt; sp.pos0 = a->pos0; sp.Ll = a->Ll; sp.C = C; sp.G = G;
   sp.hdr = w.hdr; sp.seq_off = w.seq_off; sp.expected = w.expected; sp.ticket = w.ticket; sp.rows = w.rows;
   sp.n_unmasked = a->n_unmasked; sp.is_fallback = a->is_fallback; sp.fallback_pos = a->fallback_pos;
-  if (launch(active_set_kernel, dim3(1), dim3(kSetupNT), st, false, sp) != cudaSuccess) return FORK_ERR_CUDA;
+  if (launch(active_set_kernel, dim3(1), dim3(kSetupNT), st, g_tune[FORK_TUNE_PDL].load() >= 0, sp) != cudaSuccess) return FORK_ERR_CUDA;
 
   ReduceParams rp;
   memset(&rp, 0, sizeof(rp));
@@ -1137,7 +1142,7 @@ extern "C" fork_status fork_logprob(const fork_logprob_args* a, void* ws, size_t
   sp.B = a->B; sp.Lt = a->Lt; sp.pos0 = a->pos0; sp.Ll = a->Ll; sp.C = C; sp.G = G;
   sp.hdr = w.hdr; sp.seq_off = w.seq_off; sp.expected = w.expected; sp.ticket = w.ticket; sp.rows = w.rows;
   sp.seq_sum = a->seq_sum; sp.seq_cnt = a->seq_cnt;
-  if (launch(active_set_kernel, dim3(1), dim3(kSetupNT), st, false, sp) != cudaSuccess) return FORK_ERR_CUDA;
+  if (launch(active_set_kernel, dim3(1), dim3(kSetupNT), st, g_tune[FORK_TUNE_PDL].load() >= 0, sp) != cudaSuccess) return FORK_ERR_CUDA;
 
   ReduceParams rp;
   memset(&rp, 0, sizeof(rp));
