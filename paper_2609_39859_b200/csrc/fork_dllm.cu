@@ -605,17 +605,6 @@ __device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32
                :: "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
-#ifdef FORK_EXP_TRACE
-__device__ unsigned long long g_trace[FORK_MAX_GRID][16];
-__device__ __forceinline__ void trace(int slot) {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  g_trace[blockIdx.x][slot] = t;
-}
-#define FORK_TRACE(slot) trace(slot)
-#else
-#define FORK_TRACE(slot)
-#endif
 
 template <typename T, int MODE, int kCW>
 __global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_select_ring_kernel(ReduceParams p, int n_stages) {
@@ -628,7 +617,6 @@ __global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_sel
   unsigned char* ring = dyn_smem;
   RingSmem& rs = *reinterpret_cast<RingSmem*>(dyn_smem + (size_t)n_stages * kStageBytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (threadIdx.x == 0) FORK_TRACE(0);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < n_stages; ++s) { mbar_init(&rs.full[s], 1); mbar_init(&rs.empty[s], kCW); }
@@ -641,14 +629,12 @@ __global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_sel
   asm volatile("griddepcontrol.launch_dependents;");          /* the next kernel in the stream may take free SM slots */
   const int R = p.hdr->R;
   if (R <= 0) return;
-  if (threadIdx.x == 0) FORK_TRACE(1);
   const PartitionCtx c = make_partition(R, p.C, (int)gridDim.x);
   const int g = blockIdx.x;
   if (g >= c.G) return;
   SegmentIter it;
   it.init(c, g, p.src.V);
   Segment sg;
-  if (threadIdx.x == 0) FORK_TRACE(2);
 
   if (warp == kCW) {
     /* ---------------- producer ---------------- */
@@ -664,7 +650,6 @@ __global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_sel
         if (!mbar_wait(&rs.empty[s], ph ^ 1u, p)) { ok = false; break; }
         mbar_arrive_expect_tx(&rs.full[s], bytes);
         bulk_copy_g2s(ring + (size_t)s * kStageBytes, src + off, bytes, &rs.full[s]);
-        if (n == 0) FORK_TRACE(3);
         if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1u; }
       }
     }
@@ -673,7 +658,6 @@ __global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_sel
       for (uint32_t q = first; q < n; ++q)
         mbar_wait(&rs.full[q % (uint32_t)n_stages], (q / (uint32_t)n_stages) & 1u, p);
     }
-    FORK_TRACE(4);
     return;
   }
 
@@ -682,28 +666,14 @@ __global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_sel
     const int ctid = threadIdx.x;                           /* 0 .. kCT-1 */
     uint32_t s = 0, ph = 0, nseg = 0;                       /* ring slot, its phase, segments done */
     bool sticky = false;                                    /* this thread has met a -inf logit before */
-#ifdef FORK_EXP_TRACE
-    unsigned long long tw = 0, tt = 0, ta = 0, tn = 0, tloop = 0, trow = 0, nrow = 0;
-    const long long cstart = clock64();
-    long long cprev = cstart; bool prev_same_seg = false;
-#endif
     while (it.next(sg)) {
       Acc<T, WITH_T, false> a;
       a.init();
       const int nvec = (sg.e1 - sg.e0) / VEC;
       for (int voff = 0; voff < nvec; voff += kStageVecs) {
-#ifdef FORK_EXP_TRACE
-        const long long c0 = clock64();
-        if (prev_same_seg) tloop += (unsigned long long)(c0 - cprev); else { trow += (unsigned long long)(c0 - cprev); nrow += 1; }
-#endif
         if (!mbar_wait(&rs.full[s], ph, p)) return;
-#ifdef FORK_EXP_TRACE
-        const long long c1 = clock64();
-#endif
-        if (ctid == 0 && nseg == 0 && voff == 0) FORK_TRACE(5);
         const uint4* sp = reinterpret_cast<const uint4*>(ring + (size_t)s * kStageBytes);
         const int nv = nvec - voff;
-#ifndef FORK_EXP_NO_COMPUTE
         if (nv >= kStageVecs) {
           /* a full stage: kUnroll vectors per thread; the stage is handed back to the producer as
              soon as the values sit in registers (track() has consumed every loaded word) */
@@ -713,17 +683,7 @@ __global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_sel
           if (!sticky) a.template track<kUnroll>(v, sg.e0 + (voff + ctid) * VEC, kCT * VEC);
           __syncwarp();
           if (lane == 0) mbar_arrive(&rs.empty[s]);
-#ifdef FORK_EXP_TRACE
-          const long long c2 = clock64();
-#endif
           if (!sticky) a.template accumulate<kUnroll>(v);
-#ifdef FORK_EXP_TRACE
-          {
-            const long long c3 = clock64();
-            tw += (unsigned long long)(c1 - c0); tt += (unsigned long long)(c2 - c1); ta += (unsigned long long)(c3 - c2); tn += 1ull;
-            cprev = c3; prev_same_seg = true;
-          }
-#endif
         } else {
           /* the last, partly filled stage of a segment: same unrolled code, vectors past the end
              replaced by the clamp value (contributes 2^-huge = 0 and never wins the maximum
@@ -736,14 +696,7 @@ __global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_sel
           __syncwarp();
           if (lane == 0) mbar_arrive(&rs.empty[s]);
           if (!sticky) a.template accumulate<kUnroll>(v);
-#ifdef FORK_EXP_TRACE
-          { const long long c3 = clock64(); tw += (unsigned long long)(c1 - c0); ta += (unsigned long long)(c3 - c1); cprev = c3; prev_same_seg = true; }
-#endif
         }
-#else
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&rs.empty[s]);
-#endif
         if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1u; }
       }
       const bool tail = (ctid == 0) && (sg.e0 + nvec * VEC < sg.e1);   /* fewer than VEC trailing elements */
@@ -755,21 +708,15 @@ __global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_sel
           for (int e = sg.e0 + nvec * VEC; e < sg.e1; ++e) a.one(to_f32(row[e]), e);
         }
         pt = a.part();
-#ifndef FORK_EXP_NO_COMPUTE
         if (!part_is_finite(pt)) sticky = true;
-#endif
       }
       /* a thread that met -inf (now or earlier) takes its own vectors again from global memory, clamped */
       if (sticky) {
         const int2 bk = p.rows[sg.r];
         pt = stream_thread_clamped<T, WITH_T, kCT>(row_ptr<T>(p.src, bk.x, bk.y), sg.e0, sg.e1, ctid, ctid == 0);
       }
-#ifdef FORK_EXP_NO_COMPUTE
-      pt = Part{1.f, 1.f, 0.f, sg.e0};
-#endif
       __syncwarp();
       pt = part_warp_reduce(pt);
-      if (ctid == 0) FORK_TRACE(6);
       if (lane == 0) {
         const uint32_t d = nseg % kMail, mph = (nseg / kMail) & 1u;
         if (mbar_wait(&rs.mempty[d], mph ^ 1u, p)) {
@@ -777,21 +724,8 @@ __global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_sel
           mbar_arrive(&rs.mfull[d]);
         }
       }
-      if (ctid == 0) FORK_TRACE(7);
       ++nseg;
-#ifdef FORK_EXP_TRACE
-      prev_same_seg = false;
-#endif
     }
-#ifdef FORK_EXP_TRACE
-    if (lane == 0 && warp == 3) {
-      unsigned smid; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-      g_trace[blockIdx.x][4] = smid;
-      g_trace[blockIdx.x][12] = tw; g_trace[blockIdx.x][13] = tt; g_trace[blockIdx.x][14] = ta; g_trace[blockIdx.x][15] = tn;
-      g_trace[blockIdx.x][1] = tloop; g_trace[blockIdx.x][2] = trow; g_trace[blockIdx.x][3] = nrow;
-      g_trace[blockIdx.x][11] = (unsigned long long)(clock64() - cstart);
-    }
-#endif
     return;
   }
 
@@ -808,18 +742,10 @@ __global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_sel
     __syncwarp();
     if (lane == 0) mbar_arrive(&rs.mempty[d]);
     pt = part_warp_reduce(pt);
-    if (lane == 0) FORK_TRACE(8);
-#ifndef FORK_EXP_NO_PUBLISH
     if (publish_part(p, pt, sg.r, g, b, want)) {
-      if (lane == 0) FORK_TRACE(9);
-#ifndef FORK_EXP_NO_FINALIZE
       if (MODE == kModeStep) finalize_step_sequence<T>(p, c, b, h);
       else finalize_logprob_sequence<T>(p, c, b, h);
-#endif
-      if (lane == 0) FORK_TRACE(11);
     }
-    if (lane == 0) FORK_TRACE(10);
-#endif
     ++nseg;
   }
 }
@@ -1332,13 +1258,4 @@ extern "C" int64_t fork_debug_part_begin(int64_t U, int32_t G, int32_t g) { retu
 extern "C" int32_t fork_debug_part_owner(int64_t U, int32_t G, int64_t x) { return fork_part_owner(U, G, x); }
 extern "C" int32_t fork_debug_row_parts(int64_t U, int32_t G, int32_t C, int64_t r) { return fork_row_parts(U, G, C, r); }
 extern "C" int32_t fork_debug_chunk(void) { return FORK_CHUNK; }
-#ifdef FORK_EXP_TRACE
-extern "C" int fork_debug_trace(void* host_out) {
-  return (int)cudaMemcpyFromSymbol(host_out, g_trace, sizeof(unsigned long long) * FORK_MAX_GRID * 16);
-}
-extern "C" int fork_debug_trace_clear(void) {
-  static unsigned long long z[FORK_MAX_GRID][16];
-  return (int)cudaMemcpyToSymbol(g_trace, z, sizeof(z));
-}
-#endif
 extern "C" int32_t fork_debug_effective_grid(int64_t U, int32_t G) { return fork_effective_grid(U, G); }

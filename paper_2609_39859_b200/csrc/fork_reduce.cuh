@@ -152,9 +152,6 @@ __device__ __forceinline__ Part part_block_reduce(Part p, Part* sh) {
  * and whoever finalises the row reads those few elements once to find the exact position.
  * `part()` re-expresses (s, t) against the thread's true maximum.                                  */
 constexpr float kRaiseNats = 32.f;
-#ifndef FORK_POLY_WORDS
-#define FORK_POLY_WORDS 0      /* bf16: words per 128-bit vector whose exp2 runs on the FMA pipe */
-#endif
 
 /* lo/hi halves of a that are greater than b's select `code` into g_lo / g_hi */
 __device__ __forceinline__ void track_rise_bf16x2(uint32_t a, uint32_t b, int code, int& g_lo, int& g_hi) {
@@ -208,28 +205,6 @@ struct AccCore {
   __device__ __forceinline__ void add2(int k, float xa, float xb) {
     const float2 y = __ffma2_rn(make_float2(xa, xb), make_float2(kLog2e, kLog2e), nrefL2);
     const float2 e = make_float2(ex2_approx(y.x), ex2_approx(y.y));
-    s2[k] = __fadd2_rn(s2[k], e);
-    if (WITH_T) t2[k] = __ffma2_rn(y, e, t2[k]);
-  }
-  /* two logits into pair k with 2^y evaluated on the FMA pipe instead of the special-function unit:
-     y = n + f with n = round(y), 2^f by a degree-4 polynomial on [-0.5, 0.5] (max relative error
-     3e-6, exact at f = 0), 2^n by an add into the exponent field.  y is floored at -126, where the
-     term is 1e-38 and vanishes against the row maximum's 1. */
-  __device__ __forceinline__ void add2_poly(int k, float xa, float xb) {
-    const float kMagic = 12582912.f;                                   /* 1.5 * 2^23 */
-    float2 y = __ffma2_rn(make_float2(xa, xb), make_float2(kLog2e, kLog2e), nrefL2);
-    y.x = fmaxf(y.x, -126.f); y.y = fmaxf(y.y, -126.f);
-    const float2 r = __fadd2_rn(y, make_float2(kMagic, kMagic));
-    const float2 n = __fadd2_rn(r, make_float2(-kMagic, -kMagic));
-    const float2 f = __ffma2_rn(n, make_float2(-1.f, -1.f), y);
-    float2 q = make_float2(0.00960039533674717f, 0.00960039533674717f);
-    q = __ffma2_rn(q, f, make_float2(0.05591689422726631f, 0.05591689422726631f));
-    q = __ffma2_rn(q, f, make_float2(0.24023719131946564f, 0.24023719131946564f));
-    q = __ffma2_rn(q, f, make_float2(0.6931219696998596f, 0.6931219696998596f));
-    q = __ffma2_rn(q, f, make_float2(1.f, 1.f));
-    float2 e;
-    e.x = __int_as_float(__float_as_int(q.x) + (__float_as_int(r.x) << 23));
-    e.y = __int_as_float(__float_as_int(q.y) + (__float_as_int(r.y) << 23));
     s2[k] = __fadd2_rn(s2[k], e);
     if (WITH_T) t2[k] = __ffma2_rn(y, e, t2[k]);
   }
@@ -299,11 +274,10 @@ struct Acc<bf16_t, WITH_T, CLAMP> : AccCore<WITH_T> {
   __device__ __forceinline__ void accumulate(const uint4 (&v)[N]) {
 #pragma unroll
     for (int j = 0; j < N; ++j) {
-      /* FORK_POLY_WORDS of the four 32-bit words of every vector take the polynomial route */
-      if (FORK_POLY_WORDS > 0) this->add2_poly(0, bf16_lo(v[j].x), bf16_hi(v[j].x)); else this->add2(0, bf16_lo(v[j].x), bf16_hi(v[j].x));
-      if (FORK_POLY_WORDS > 1) this->add2_poly(1, bf16_lo(v[j].y), bf16_hi(v[j].y)); else this->add2(1, bf16_lo(v[j].y), bf16_hi(v[j].y));
-      if (FORK_POLY_WORDS > 2) this->add2_poly(0, bf16_lo(v[j].z), bf16_hi(v[j].z)); else this->add2(0, bf16_lo(v[j].z), bf16_hi(v[j].z));
-      if (FORK_POLY_WORDS > 3) this->add2_poly(1, bf16_lo(v[j].w), bf16_hi(v[j].w)); else this->add2(1, bf16_lo(v[j].w), bf16_hi(v[j].w));
+      this->add2(0, bf16_lo(v[j].x), bf16_hi(v[j].x));
+      this->add2(1, bf16_lo(v[j].y), bf16_hi(v[j].y));
+      this->add2(0, bf16_lo(v[j].z), bf16_hi(v[j].z));
+      this->add2(1, bf16_lo(v[j].w), bf16_hi(v[j].w));
     }
   }
   /* one trailing element at vocabulary index idx (after all of the thread's vectors) */
