@@ -24,6 +24,7 @@ _LIB = os.path.join(_HERE, "libfork_oracle.so")
 BF16, F32 = 0, 1
 OK, ERR_ARG, ERR_MAX_STEPS, ERR_PROVIDER = 0, -1, -4, -5
 ROW_BAD, ROW_BAD_TOKEN = 1, 2
+FB_LEFTMOST, FB_MAX_CONF, FB_MIN_CONF, FB_MAX_ENTROPY, FB_RANDOM = 0, 1, 2, 3, 4
 
 
 def build(force: bool = False) -> str:
@@ -48,6 +49,9 @@ class _StepArgs(C.Structure):
         ("nfe", C.c_void_p), ("n_fallback", C.c_void_p),
         ("row_status", C.c_void_p),
         ("nthreads", C.c_int32),
+        ("fallback_mode", C.c_int32), ("fallback_rand", C.c_void_p),
+        ("temperature", C.c_float), ("sample_seed", C.c_uint64),
+        ("fallback_margin", C.c_void_p), ("sample_margin", C.c_void_p),
     ]
 
 
@@ -79,6 +83,18 @@ def lib():
                                               _PROVIDER, C.c_void_p, C.c_int32, C.c_void_p]
         L.fork_oracle_threads_used.restype = C.c_int
         L.fork_oracle_threads_used.argtypes = [C.c_int32, C.c_int64]
+        L.fork_oracle_noise.restype = None
+        L.fork_oracle_noise.argtypes = [C.c_uint64, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+        L.fork_oracle_select_top_entropy.restype = C.c_int
+        L.fork_oracle_select_top_entropy.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float,
+                                                     C.c_void_p, C.c_void_p]
+        L.fork_oracle_grpo_loss.restype = C.c_int
+        L.fork_oracle_grpo_loss.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                            C.c_void_p, C.c_float, C.c_float] + [C.c_void_p] * 6
+        L.fork_oracle_row_logp_grad.restype = C.c_int
+        L.fork_oracle_row_logp_grad.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_double, C.c_void_p]
+        L.fork_oracle_row_lse.restype = C.c_double
+        L.fork_oracle_row_lse.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
         _lib = L
     return _lib
 
@@ -138,9 +154,12 @@ class StepState:
         self.nfe = np.zeros(B, np.int32)
         self.n_fallback = np.zeros(B, np.int32)
         self.row_status = np.zeros((B, Lt), np.uint32)
+        self.fallback_margin = np.full(B, np.inf, np.float64)
+        self.sample_margin = np.full((B, Lt), np.inf, np.float64)
 
 
-def _fill_args(st: StepState, logits: np.ndarray, lo, hi, threshold, step, pos0, nthreads) -> _StepArgs:
+def _fill_args(st: StepState, logits: np.ndarray, lo, hi, threshold, step, pos0, nthreads,
+               fallback_mode=FB_LEFTMOST, fallback_rand=None, temperature=0.0, sample_seed=0) -> _StepArgs:
     assert logits.ndim == 3 and logits.flags.c_contiguous
     B, Ll, V = logits.shape
     assert B == st.B
@@ -159,15 +178,27 @@ def _fill_args(st: StepState, logits: np.ndarray, lo, hi, threshold, step, pos0,
     a.nfe, a.n_fallback = st.nfe.ctypes.data, st.n_fallback.ctypes.data
     a.row_status = st.row_status.ctypes.data
     a.nthreads = nthreads
+    a.fallback_mode = int(fallback_mode)
+    a.fallback_rand = _ptr(fallback_rand)
+    a.temperature = float(temperature)
+    a.sample_seed = int(sample_seed)
+    a.fallback_margin = st.fallback_margin.ctypes.data
+    a.sample_margin = st.sample_margin.ctypes.data
     return a
 
 
 def step(st: StepState, logits: np.ndarray, lo: np.ndarray, hi: np.ndarray, threshold: float,
-         step_id: int = 0, pos0: int = 0, nthreads: int = 0) -> int:
-    """One Fork-dLLM sampling step (Algorithm 2) on host buffers; ``st`` is updated in place."""
+         step_id: int = 0, pos0: int = 0, nthreads: int = 0, fallback_mode: int = FB_LEFTMOST,
+         fallback_rand=None, temperature: float = 0.0, sample_seed: int = 0) -> int:
+    """One sampling step on host buffers; ``st`` is updated in place.  The defaults give Fork-dLLM
+    (Algorithm 2) with arg-max candidates; ``fallback_mode`` selects Fast-dLLM's order (Algorithm 1)
+    or an ablation order, ``temperature`` > 0 draws the candidates (noise stream ``sample_seed``)."""
     lo = np.ascontiguousarray(lo, np.int32)
     hi = np.ascontiguousarray(hi, np.int32)
-    a = _fill_args(st, logits, lo, hi, threshold, step_id, pos0, nthreads)
+    if fallback_rand is not None:
+        fallback_rand = np.ascontiguousarray(fallback_rand, np.uint32)
+    a = _fill_args(st, logits, lo, hi, threshold, step_id, pos0, nthreads, fallback_mode, fallback_rand,
+                   temperature, sample_seed)
     return int(lib().fork_oracle_step(C.byref(a)))
 
 
@@ -200,7 +231,9 @@ def block_cursors(mask: np.ndarray, gen_lo: int, gen_hi: int, block_len: int, lo
 
 
 def decode_loop(st: StepState, logits: np.ndarray, block_len: int, gen_lo: int, gen_hi: int, provider,
-                threshold: float, max_steps: int, step0: int = 0, pos0: int = 0, nthreads: int = 0):
+                threshold: float, max_steps: int, step0: int = 0, pos0: int = 0, nthreads: int = 0,
+                fallback_mode: int = FB_LEFTMOST, fallback_rand=None, temperature: float = 0.0,
+                sample_seed: int = 0):
     """Run the semi-autoregressive loop.  ``provider(step, tokens, mask, lo, hi, logits)`` fills
     ``logits`` (numpy views of the live host buffers) and returns 0, or non-zero to abort."""
     B, Lt = st.B, st.Lt
@@ -215,8 +248,66 @@ def decode_loop(st: StepState, logits: np.ndarray, block_len: int, gen_lo: int, 
             traceback.print_exc()
             return 1
 
-    a = _fill_args(st, logits, None, None, threshold, step0, pos0, nthreads)
+    a = _fill_args(st, logits, None, None, threshold, step0, pos0, nthreads, fallback_mode, fallback_rand,
+                   temperature, sample_seed)
     steps = C.c_int32(0)
     rc = lib().fork_oracle_decode_loop(C.byref(a), block_len, gen_lo, gen_hi, _PROVIDER(_cb), None,
                                        max_steps, C.addressof(steps))
     return int(rc), int(steps.value)
+
+
+def noise(seed: int, step_id: int, b: int, k: int, v: int):
+    """(u, g): the uniform and the standard Gumbel variate of vocabulary entry v of row (step, b, k)."""
+    u, g = C.c_double(), C.c_double()
+    lib().fork_oracle_noise(int(seed), step_id, b, k, v, C.addressof(u), C.addressof(g))
+    return u.value, g.value
+
+
+def select_top_entropy(entropy: np.ndarray, eligible: np.ndarray, ratio: float):
+    """JustGRPO-Fast's selection: per rollout the floor(ratio*n) eligible positions of highest entropy."""
+    entropy = np.ascontiguousarray(entropy, np.float32)
+    eligible = np.ascontiguousarray(eligible, np.uint8)
+    B, Lt = entropy.shape
+    select = np.zeros((B, Lt), np.uint8)
+    cnt = np.zeros(B, np.int32)
+    rc = lib().fork_oracle_select_top_entropy(entropy.ctypes.data, eligible.ctypes.data, B, Lt, float(ratio),
+                                              select.ctypes.data, cnt.ctypes.data)
+    return int(rc), select, cnt
+
+
+def grpo_loss(logp_new: np.ndarray, logp_old: np.ndarray, select: np.ndarray, reward: np.ndarray, group: int,
+              eps_lo: float, eps_hi: float) -> dict:
+    """The ForkGRPO objective (Eq. 2) and its derivative with respect to logp_new."""
+    logp_new = np.ascontiguousarray(logp_new, np.float32)
+    logp_old = np.ascontiguousarray(logp_old, np.float32)
+    select = np.ascontiguousarray(select, np.uint8)
+    reward = np.ascontiguousarray(reward, np.float32)
+    B, Lt = logp_new.shape
+    adv = np.zeros(B, np.float64)
+    ratio = np.zeros((B, Lt), np.float64)
+    seq_obj = np.zeros(B, np.float64)
+    obj = np.zeros(1, np.float64)
+    dlogp = np.zeros((B, Lt), np.float64)
+    skipped = np.zeros(max(B // max(group, 1), 1), np.uint8)
+    rc = lib().fork_oracle_grpo_loss(B, Lt, group, logp_new.ctypes.data, logp_old.ctypes.data, select.ctypes.data,
+                                     reward.ctypes.data, float(eps_lo), float(eps_hi), adv.ctypes.data,
+                                     ratio.ctypes.data, seq_obj.ctypes.data, obj.ctypes.data, dlogp.ctypes.data,
+                                     skipped.ctypes.data)
+    return dict(rc=int(rc), adv=adv, ratio=ratio, seq_obj=seq_obj, objective=float(obj[0]), dlogp=dlogp,
+                skipped=skipped)
+
+
+def row_logp_grad(row: np.ndarray, tok: int, w: float = 1.0) -> np.ndarray:
+    """d(w * log q(tok))/d logits of one row."""
+    row = np.ascontiguousarray(row)
+    g = np.zeros(row.shape[0], np.float64)
+    rc = lib().fork_oracle_row_logp_grad(row.ctypes.data, row.shape[0], _dtype_of(row), int(tok), float(w),
+                                         g.ctypes.data)
+    if rc != 0:
+        raise ValueError("row_logp_grad: bad arguments")
+    return g
+
+
+def row_lse(row: np.ndarray) -> float:
+    row = np.ascontiguousarray(row)
+    return float(lib().fork_oracle_row_lse(row.ctypes.data, row.shape[0], _dtype_of(row)))

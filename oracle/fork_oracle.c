@@ -18,6 +18,17 @@
  *   - semi-autoregressive blocks of length BL inside the generation window (Section 4.1 Setup).
  *   - token entropy of q_theta^k (Section 3.1 / Figure 2), in nats, of the untempered softmax.
  *
+ *   - candidates at temperature tau > 0: x_0^k ~ q_theta^k(. | x_t; tau)  (Section 2; Algorithm 2
+ *       line 4), drawn as arg-max_v (x_v/tau + g_v) with g_v standard Gumbel noise from a stated
+ *       counter-based generator; the confidence stays the UNtempered probability of the drawn token
+ *       (Algorithm 2 line 5 has no tau).
+ *   - the fallback orders the paper compares with: highest confidence (Algorithm 1, Fast-dLLM) and
+ *       the lowest-confidence / highest-entropy / random ablations (Section 4.1, ablations).
+ *   - top-entropy position selection of JustGRPO-Fast (Section 3.2, last paragraph).
+ *   - the ForkGRPO objective (Eq. 2): ratio rho, group-standardised advantage, clipped minimum,
+ *       mean over the fallback steps of a rollout, mean over rollouts; and its derivative with
+ *       respect to the logits of a selected row.
+ *
  * Softmax quantities are written out from their definitions with the usual max shift:
  *   m = max_v x_v,  a = min{v : x_v = m},  s = sum_v exp(x_v - m),  t = sum_v (x_v - m) exp(x_v - m)
  *   p_v = exp(x_v - m)/s,  conf = p_a = 1/s,
@@ -33,7 +44,10 @@
  *
  * Parity pins (tests, CPU only): brute force without the max shift on tiny V, the one-peak /
  * k-way-tie closed forms, hand-worked rows and steps, library log-sum-exp/entropy, invariants,
- * AR and whole-block special cases of the loop.
+ * AR and whole-block special cases of the loop; for the variants: moments and a chi-square of
+ * the noise stream, scipy's softmax(x/tau) for the drawn candidates, hand-worked fallback choices
+ * of Algorithm 1 against Algorithm 2, numpy sorting for both selections, hand-worked advantages
+ * and clipping cases of Eq. 2, finite differences for both derivatives.
  *
  * Build: gcc -O2 -std=c11 -fPIC -shared -pthread fork_oracle.c -lm
  */
@@ -70,7 +84,39 @@ typedef struct {
   double m, s, t;      /* max, sum exp(x-m), sum (x-m) exp(x-m) */
   int32_t a;           /* lowest arg-max */
   uint32_t status;
+  /* temperature > 0 only */
+  int32_t a_s;         /* drawn token */
+  double x_s;          /* its logit */
+  double key_margin;   /* best perturbed key minus the best strictly smaller one (+inf if none) */
 } row_red;
+
+/* ---- the noise stream of stochastic candidates -------------------------------------------------
+ * One 64-bit key per (seed, step, b, k); one 32-bit hash per vocabulary entry; a uniform on the
+ * 2^-23 grid of midpoints, u = ((h >> 9) + 1/2) 2^-23 in (0,1); standard Gumbel g = -ln(-ln u).
+ * The draw arg-max_v (x_v/tau + g_v) is then a sample of softmax(x/tau) (Gumbel-max), up to the
+ * grid of u (largest g = 16.6).  The CUDA path implements the same integer recipe on its own. */
+static uint64_t mix64(uint64_t z) {
+  z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ULL; z ^= z >> 27; z *= 0x94D049BB133111EBULL; z ^= z >> 31;
+  return z;
+}
+static uint64_t noise_row_key(uint64_t seed, int32_t step, int32_t b, int32_t k) {
+  uint64_t z = mix64(seed + 0x9E3779B97F4A7C15ULL * (uint64_t)((uint32_t)step + 1u));
+  return mix64(z ^ (((uint64_t)(uint32_t)b << 32) | (uint64_t)(uint32_t)k));
+}
+static uint32_t noise_hash(uint64_t row_key, uint32_t v) {
+  uint32_t x = (v ^ (uint32_t)(row_key >> 32)) * 0x9E3779B1u + (uint32_t)row_key;
+  x ^= x >> 16; x *= 0x21F0AAADu; x ^= x >> 15; x *= 0x735A2D97u; x ^= x >> 15;
+  return x;
+}
+static double noise_uniform(uint32_t h) { return ((double)(h >> 9) + 0.5) * (1.0 / 8388608.0); }
+static double noise_gumbel(uint32_t h) { return -log(-log(noise_uniform(h))); }
+
+/* Exported for the pins: the uniform and the Gumbel variate of entry v of row (seed, step, b, k). */
+void fork_oracle_noise(uint64_t seed, int32_t step, int32_t b, int32_t k, int32_t v, double* u, double* g) {
+  uint32_t h = noise_hash(noise_row_key(seed, step, b, k), (uint32_t)v);
+  if (u) *u = noise_uniform(h);
+  if (g) *g = noise_gumbel(h);
+}
 
 /* m, a, s, t of one row, straight from the definitions */
 static void reduce_row(const void* row, int32_t V, int dtype, row_red* out) {
@@ -92,6 +138,23 @@ static void reduce_row(const void* row, int32_t V, int dtype, row_red* out) {
     nsum_add(&s, e); nsum_add(&t, d * e);
   }
   out->s = nsum_get(&s); out->t = nsum_get(&t);
+}
+
+/* x_0 ~ q(. ; tau) for tau > 0 (Algorithm 2 line 4) by Gumbel-max over the row; ties in the
+   perturbed key go to the lowest index.  Rows flagged bad keep the greedy candidate. */
+static void sample_row(const void* row, int32_t V, int dtype, double tau, uint64_t row_key, row_red* out) {
+  out->a_s = out->a; out->x_s = out->m; out->key_margin = INFINITY;
+  if (out->status & ORA_ROW_BAD) return;
+  double best = -INFINITY, second = -INFINITY; int32_t arg = -1;
+  for (int32_t v = 0; v < V; ++v) {
+    double x = load_logit(row, v, dtype);
+    if (isinf(x)) continue;                          /* probability 0 */
+    double key = x / tau + noise_gumbel(noise_hash(row_key, (uint32_t)v));
+    if (arg < 0 || key > best) { if (arg >= 0 && best > second) second = best; best = key; arg = v; }
+    else if (key < best && key > second) second = key;
+  }
+  out->a_s = arg; out->x_s = load_logit(row, arg, dtype);
+  out->key_margin = best - second;
 }
 
 /* Exported: statistics of a single row. Any output pointer may be NULL. */
@@ -133,13 +196,27 @@ typedef struct fork_oracle_step_args {
   int32_t* nfe; int32_t* n_fallback;                                   /* [B], accumulated */
   uint32_t* row_status;                                                /* [B,Lt], written on the active set */
   int32_t nthreads;                                                    /* <=0: all host cores */
+  /* --- the variants the paper compares with; all-zero values give Algorithm 2 at temperature 0 --- */
+  int32_t fallback_mode;                                               /* ORA_FB_* */
+  const uint32_t* fallback_rand;                                       /* [B], ORA_FB_RANDOM only */
+  float temperature;                                                   /* tau; 0 = arg-max candidates */
+  uint64_t sample_seed;                                                /* noise stream of tau > 0 */
+  double* fallback_margin;   /* [B] test aid: gap between the chosen fallback position's key and the runner-up */
+  double* sample_margin;     /* [B,Lt] test aid: gap between the winning perturbed key and the runner-up */
 } fork_oracle_step_args;
+
+/* Which position a fallback step commits.  LEFTMOST is Fork-dLLM (Algorithm 2); MAX_CONF is
+   Fast-dLLM (Algorithm 1, arg-max_k c); MIN_CONF, MAX_ENTROPY and RANDOM are the ablations of
+   Section 4.1.  Ties go to the lowest position; rows flagged bad are passed over unless every
+   live row is bad, in which case the leftmost is taken. */
+enum { ORA_FB_LEFTMOST = 0, ORA_FB_MAX_CONF = 1, ORA_FB_MIN_CONF = 2, ORA_FB_MAX_ENTROPY = 3, ORA_FB_RANDOM = 4 };
 
 typedef struct { int32_t b, k; row_red red; } live_row;
 
 typedef struct {
   const void* logits; int64_t stride_b, stride_l; int32_t pos0; int32_t V, dtype; size_t es;
   live_row* rows; int64_t n; int64_t next; pthread_mutex_t mu;
+  double tau; uint64_t seed; int32_t step;
 } reduce_job;
 
 static void* reduce_worker(void* p) {
@@ -151,6 +228,8 @@ static void* reduce_worker(void* p) {
     const char* row = (const char*)J->logits +
         ((int64_t)lr->b * J->stride_b + (int64_t)(lr->k - J->pos0) * J->stride_l) * (int64_t)J->es;
     reduce_row(row, J->V, J->dtype, &lr->red);
+    if (J->tau > 0.0)
+      sample_row(row, J->V, J->dtype, J->tau, noise_row_key(J->seed, J->step, lr->b, lr->k), &lr->red);
   }
   return NULL;
 }
@@ -174,10 +253,28 @@ static void reduce_rows_parallel(reduce_job* J, int nthreads) {
 
 int fork_oracle_threads_used(int32_t nthreads, int64_t n_rows) { return host_threads(nthreads, n_rows); }
 
+/* per-row outputs.  The candidate x_0^k is the arg-max (temperature 0) or the drawn token; its
+   confidence c_t^k is its probability under the untempered softmax (Algorithm 2 lines 4-5). */
+static int32_t row_cand(const row_red* q, int sampled) { return sampled ? q->a_s : q->a; }
+static double row_logp(const row_red* q, int sampled) {
+  if (q->status & ORA_ROW_BAD) return NAN;
+  return (sampled ? q->x_s - q->m : 0.0) - log(q->s);
+}
+static double row_conf(const row_red* q, int sampled) {
+  if (q->status & ORA_ROW_BAD) return 0.0;
+  return sampled ? exp(q->x_s - q->m) / q->s : 1.0 / q->s;
+}
+static double row_entropy(const row_red* q) {
+  return (q->status & ORA_ROW_BAD) ? NAN : log(q->s) - q->t / q->s;
+}
+
 int fork_oracle_step(const fork_oracle_step_args* A) {
   if (!A || !A->logits || !A->tokens || !A->mask || !A->blk_lo || !A->blk_hi) return ORA_ERR_ARG;
   if (A->B < 0 || A->Lt <= 0 || A->V <= 0 || A->Ll <= 0) return ORA_ERR_ARG;
   if (A->threshold != A->threshold) return ORA_ERR_ARG;
+  if (A->fallback_mode < ORA_FB_LEFTMOST || A->fallback_mode > ORA_FB_RANDOM) return ORA_ERR_ARG;
+  if (A->fallback_mode == ORA_FB_RANDOM && !A->fallback_rand) return ORA_ERR_ARG;
+  if (!(A->temperature >= 0.0f) || isinf(A->temperature)) return ORA_ERR_ARG;
   const int32_t B = A->B, Lt = A->Lt;
   /* M_t restricted to each sequence's active block (Algorithm 2 line 3; semi-AR blocks) */
   live_row* rows = (live_row*)malloc(sizeof(live_row) * (size_t)((int64_t)B * Lt + 1));
@@ -195,7 +292,9 @@ int fork_oracle_step(const fork_oracle_step_args* A) {
   /* q_theta^k for every k in the active set: the only O(V) work */
   reduce_job J; J.logits = A->logits; J.stride_b = A->stride_b; J.stride_l = A->stride_l; J.pos0 = A->pos0;
   J.V = A->V; J.dtype = A->dtype; J.es = (A->dtype == ORA_BF16) ? 2 : 4; J.rows = rows; J.n = n;
+  J.tau = (double)A->temperature; J.seed = A->sample_seed; J.step = A->step;
   reduce_rows_parallel(&J, A->nthreads);
+  const int sampled = A->temperature > 0.0f;
 
   const double lambda = (double)A->threshold;
   for (int32_t b = 0; b < B; ++b) {
@@ -209,31 +308,45 @@ int fork_oracle_step(const fork_oracle_step_args* A) {
     int any_above = 0;
     for (int64_t r = r0; r < r1; ++r) {
       const row_red* q = &rows[r].red; int64_t at = (int64_t)b * Lt + rows[r].k;
-      int bad = (q->status & ORA_ROW_BAD) != 0;
-      double c = bad ? 0.0 : 1.0 / q->s;                         /* c_t^k (Algorithm 2 line 5) */
-      if (A->conf) A->conf[at] = c;
-      if (A->cand) A->cand[at] = q->a;                           /* x_0^k at temperature 0 */
-      if (A->entropy) A->entropy[at] = bad ? NAN : log(q->s) - q->t / q->s;
-      if (A->logp) A->logp[at] = bad ? NAN : -log(q->s);
+      if (A->conf) A->conf[at] = row_conf(q, sampled);
+      if (A->cand) A->cand[at] = row_cand(q, sampled);
+      if (A->entropy) A->entropy[at] = row_entropy(q);
+      if (A->logp) A->logp[at] = row_logp(q, sampled);
       if (A->row_status) A->row_status[at] = q->status;
-      if (c > lambda) any_above = 1;                             /* U_t non-empty (line 6) */
+      if (A->sample_margin) A->sample_margin[at] = sampled ? q->key_margin : INFINITY;
+      if (row_conf(q, sampled) > lambda) any_above = 1;          /* U_t non-empty (line 6) */
     }
     int fb = !any_above;                                         /* fallback step: max_k c <= lambda */
+    int64_t pick = r0;                                           /* the row a fallback step commits */
+    double margin = INFINITY;
+    if (fb && A->fallback_mode == ORA_FB_RANDOM) {
+      pick = r0 + (int64_t)(A->fallback_rand[b] % (uint32_t)(r1 - r0));
+    } else if (fb && A->fallback_mode != ORA_FB_LEFTMOST) {
+      double best = 0.0, second = -INFINITY; int have = 0;
+      for (int64_t r = r0; r < r1; ++r) {
+        const row_red* q = &rows[r].red;
+        if (q->status & ORA_ROW_BAD) continue;
+        double key = A->fallback_mode == ORA_FB_MAX_CONF ? row_conf(q, sampled)
+                   : A->fallback_mode == ORA_FB_MIN_CONF ? -row_conf(q, sampled) : row_entropy(q);
+        if (!have || key > best) { if (have) second = best; best = key; pick = r; have = 1; }   /* strict: ties keep the lower position */
+        else if (key > second) second = key;
+      }
+      if (have) margin = best - second;
+    }
+    if (A->fallback_margin) A->fallback_margin[b] = fb ? margin : INFINITY;
     int32_t count = 0;
     for (int64_t r = r0; r < r1; ++r) {
       const row_red* q = &rows[r].red; int64_t at = (int64_t)b * Lt + rows[r].k;
-      int bad = (q->status & ORA_ROW_BAD) != 0;
-      double c = bad ? 0.0 : 1.0 / q->s;
-      int commit = fb ? (r == r0) : (c > lambda);                /* leftmost(M_t) or the threshold set */
+      int commit = fb ? (r == pick) : (row_conf(q, sampled) > lambda);   /* the fallback position, or the threshold set */
       if (!commit) continue;
-      A->tokens[at] = q->a; A->mask[at] = 0; ++count;
+      A->tokens[at] = row_cand(q, sampled); A->mask[at] = 0; ++count;
       if (A->commit_step) A->commit_step[at] = A->step;
       if (A->commit_fallback) A->commit_fallback[at] = (uint8_t)fb;
-      if (A->commit_logp) A->commit_logp[at] = bad ? NAN : -log(q->s);
+      if (A->commit_logp) A->commit_logp[at] = row_logp(q, sampled);
     }
     if (A->n_unmasked) A->n_unmasked[b] = count;
     if (A->is_fallback) A->is_fallback[b] = (uint8_t)fb;
-    if (A->fallback_pos) A->fallback_pos[b] = fb ? rows[r0].k : -1;
+    if (A->fallback_pos) A->fallback_pos[b] = fb ? rows[pick].k : -1;
     if (A->nfe) A->nfe[b] += 1;
     if (A->n_fallback) A->n_fallback[b] += fb;
   }
@@ -352,4 +465,104 @@ int fork_oracle_decode_loop(fork_oracle_step_args* A, int32_t block_len, int32_t
   if (steps_taken) *steps_taken = n;
   free(lo); free(hi);
   return rc;
+}
+
+/* ------------------------------------------------------------------------------------------ */
+/* JustGRPO-Fast position selection (Section 3.2, last paragraph; Section 4.2 Setup): of the   */
+/* eligible positions of each rollout keep the fraction `ratio` with the highest token entropy. */
+/* Reading: the count is floor(ratio * n) with n the number of eligible positions (at least 1   */
+/* when n > 0 and ratio > 0), equal entropies go to the lower position, NaN entropies rank last. */
+int fork_oracle_select_top_entropy(const float* entropy, const uint8_t* eligible, int32_t B, int32_t Lt,
+                                   float ratio, uint8_t* select, int32_t* n_selected) {
+  if (!entropy || !eligible || !select || B < 0 || Lt <= 0 || !(ratio >= 0.0f) || ratio > 1.0f) return ORA_ERR_ARG;
+  for (int32_t b = 0; b < B; ++b) {
+    const float* H = entropy + (int64_t)b * Lt; const uint8_t* E = eligible + (int64_t)b * Lt;
+    uint8_t* S = select + (int64_t)b * Lt;
+    int32_t n = 0;
+    for (int32_t k = 0; k < Lt; ++k) { S[k] = 0; if (E[k]) ++n; }
+    int32_t want = (int32_t)floor((double)ratio * (double)n);
+    if (want < 1 && n > 0 && ratio > 0.0f) want = 1;
+    for (int32_t pick = 0; pick < want; ++pick) {           /* selection by repeated maximum */
+      int32_t arg = -1;
+      for (int32_t k = 0; k < Lt; ++k) {
+        if (!E[k] || S[k]) continue;
+        if (arg < 0) { arg = k; continue; }
+        int k_nan = isnan(H[k]), a_nan = isnan(H[arg]);
+        if ((a_nan && !k_nan) || (!a_nan && !k_nan && H[k] > H[arg])) arg = k;
+      }
+      S[arg] = 1;
+    }
+    if (n_selected) n_selected[b] = want;
+  }
+  return ORA_OK;
+}
+
+/* ------------------------------------------------------------------------------------------ */
+/* The ForkGRPO objective (Eq. 2) on a batch of B = P * G rollouts, rollout i = p * G + j.       */
+/*   rho_{i,t}  = exp(logp_new - logp_old) at the selected (fallback) positions,                 */
+/*   A_i        = (r_i - mean_group) / std_group   (group-standardised; population std; a group  */
+/*                with std 0 is skipped: its rollouts contribute nothing),                       */
+/*   obj_i      = 1/|F_i| * sum_t min(rho A_i, clip(rho, 1-eps_lo, 1+eps_hi) A_i),               */
+/*   J          = 1/B * sum_i obj_i      (1/G sum_i inside the expectation over prompts).        */
+/* dlogp = dJ/dlogp_new: rho A_i / (B |F_i|) where the unclipped term is the minimum, else 0.    */
+int fork_oracle_grpo_loss(int32_t B, int32_t Lt, int32_t group, const float* logp_new, const float* logp_old,
+                          const uint8_t* select, const float* reward, float eps_lo, float eps_hi,
+                          double* adv /*[B]*/, double* ratio /*[B,Lt]*/, double* seq_obj /*[B]*/,
+                          double* objective /*[1]*/, double* dlogp /*[B,Lt]*/, uint8_t* skipped /*[B/group]*/) {
+  if (B < 0 || Lt <= 0 || group <= 0 || B % group != 0 || !logp_new || !logp_old || !select || !reward) return ORA_ERR_ARG;
+  double J = 0.0;
+  for (int32_t p = 0; p < B / group; ++p) {
+    double mean = 0.0, var = 0.0;
+    for (int32_t j = 0; j < group; ++j) mean += (double)reward[p * group + j];
+    mean /= group;
+    for (int32_t j = 0; j < group; ++j) { double d = (double)reward[p * group + j] - mean; var += d * d; }
+    double sd = sqrt(var / group);
+    int skip = !(sd > 0.0);
+    if (skipped) skipped[p] = (uint8_t)skip;
+    for (int32_t j = 0; j < group; ++j) {
+      int32_t i = p * group + j;
+      double A = skip ? 0.0 : ((double)reward[i] - mean) / sd;
+      if (adv) adv[i] = A;
+      int32_t nf = 0;
+      for (int32_t k = 0; k < Lt; ++k) if (select[(int64_t)i * Lt + k]) ++nf;
+      double acc = 0.0;
+      for (int32_t k = 0; k < Lt; ++k) {
+        int64_t at = (int64_t)i * Lt + k;
+        if (ratio) ratio[at] = 0.0;
+        if (dlogp) dlogp[at] = 0.0;
+        if (!select[at]) continue;
+        double rho = exp((double)logp_new[at] - (double)logp_old[at]);
+        double clipped = rho < 1.0 - (double)eps_lo ? 1.0 - (double)eps_lo : (rho > 1.0 + (double)eps_hi ? 1.0 + (double)eps_hi : rho);
+        double u = rho * A, c = clipped * A;
+        acc += (u <= c) ? u : c;
+        if (ratio) ratio[at] = rho;
+        if (dlogp && !skip && u <= c) dlogp[at] = rho * A / ((double)B * (double)nf);
+      }
+      double obj = nf > 0 ? acc / nf : 0.0;
+      if (seq_obj) seq_obj[i] = obj;
+      J += obj;
+    }
+  }
+  if (objective) *objective = B > 0 ? J / B : 0.0;
+  return ORA_OK;
+}
+
+/* Derivative of w * log q(tok) with respect to the logits of one row:                          */
+/*   d/dx_v [x_tok - m - ln s] = 1[v = tok] - p_v,   p_v = exp(x_v - m)/s.                       */
+int fork_oracle_row_logp_grad(const void* row, int32_t V, int32_t dtype, int32_t tok, double w, double* grad /*[V]*/) {
+  if (!row || !grad || V <= 0 || tok < 0 || tok >= V) return ORA_ERR_ARG;
+  row_red r; reduce_row(row, V, dtype, &r);
+  if (r.status & ORA_ROW_BAD) { for (int32_t v = 0; v < V; ++v) grad[v] = NAN; return ORA_OK; }
+  for (int32_t v = 0; v < V; ++v) {
+    double x = load_logit(row, v, dtype);
+    double p = isinf(x) ? 0.0 : exp(x - r.m) / r.s;
+    grad[v] = w * ((v == tok ? 1.0 : 0.0) - p);
+  }
+  return ORA_OK;
+}
+
+/* Log-sum-exp m + ln s of one row (what the scoring pass hands to the backward pass). */
+double fork_oracle_row_lse(const void* row, int32_t V, int32_t dtype) {
+  row_red r; reduce_row(row, V, dtype, &r);
+  return (r.status & ORA_ROW_BAD) ? NAN : r.m + log(r.s);
 }
