@@ -66,6 +66,24 @@ typedef enum fork_dtype { FORK_BF16 = 0, FORK_F32 = 1 } fork_dtype;
  * Arguments of one sampling step (Algorithm 2; inputs x_t, q_theta, lambda -> x_{t-1}).
  * Output pointers marked "optional" may be NULL.
  */
+/*
+ * Which position a fallback step (no confidence above lambda) commits.
+ *   LEFTMOST    Fork-dLLM: the leftmost masked position of the block (Algorithm 2, highlighted line)
+ *   MAX_CONF    Fast-dLLM: arg-max_k c_t^k (Algorithm 1)
+ *   MIN_CONF, MAX_ENTROPY, RANDOM   the fallback ablations of Section 4.1 (lowest confidence,
+ *               highest token entropy, a random masked position)
+ * Equal keys go to the lower position.  Rows flagged FORK_ROW_NONFINITE are passed over unless every
+ * live row of the block is flagged, in which case the leftmost is taken.  A step with a non-empty
+ * threshold set is the same under every mode.
+ */
+typedef enum fork_fallback_mode {
+  FORK_FALLBACK_LEFTMOST = 0,
+  FORK_FALLBACK_MAX_CONF = 1,
+  FORK_FALLBACK_MIN_CONF = 2,
+  FORK_FALLBACK_MAX_ENTROPY = 3,
+  FORK_FALLBACK_RANDOM = 4
+} fork_fallback_mode;
+
 typedef struct fork_step_args {
   const void* logits;        /* model output q_theta(.|x_t) as logits; see the layout rule above */
   int64_t stride_b, stride_l;/* in elements; stride_l >= V */
@@ -88,14 +106,21 @@ typedef struct fork_step_args {
      (conf/entropy/logp are last written at the step that commits the position, so after a
      decode loop they hold the values at commit time.) */
   int32_t* commit_step;      /* [B,Lt] */
-  uint8_t* commit_fallback;  /* [B,Lt] 1 if committed by the leftmost fallback (a step in F_i) */
+  uint8_t* commit_fallback;  /* [B,Lt] 1 if committed by a fallback step (a step in F_i) */
   float* commit_logp;        /* [B,Lt] log-probability of the committed token (old-policy term of the ForkGRPO ratio) */
   /* per sequence; all optional */
   int32_t* n_unmasked;       /* [B] |U_t| (0 if the sequence had no live position) */
-  uint8_t* is_fallback;      /* [B] 1 if U_t was empty and the leftmost position was taken */
+  uint8_t* is_fallback;      /* [B] 1 if U_t was empty and the fallback position was taken */
   int32_t* fallback_pos;     /* [B] that position, else -1 */
   int32_t* nfe;              /* [B] += 1 if the sequence had a live position (model evaluations used) */
   int32_t* n_fallback;       /* [B] += is_fallback */
+  /* variants the paper compares with; all zero = Algorithm 2 with arg-max candidates */
+  int32_t fallback_mode;     /* fork_fallback_mode: which position a fallback step commits */
+  const uint32_t* fallback_rand; /* [B] FORK_FALLBACK_RANDOM only: the step takes live position number
+                                (fallback_rand[b] mod live count) of the block, counted from the left;
+                                read at every step, so a loop's provider may refresh it */
+  float temperature;         /* tau >= 0 of Algorithm 2 line 4; 0 = arg-max candidates */
+  uint64_t sample_seed;      /* noise stream of the candidates when tau > 0 */
 } fork_step_args;
 
 /*

@@ -303,6 +303,7 @@ int fork_oracle_step(const fork_oracle_step_args* A) {
       if (A->n_unmasked) A->n_unmasked[b] = 0;
       if (A->is_fallback) A->is_fallback[b] = 0;
       if (A->fallback_pos) A->fallback_pos[b] = -1;
+      if (A->fallback_margin) A->fallback_margin[b] = INFINITY;
       continue;
     }
     int any_above = 0;

@@ -19,6 +19,8 @@ FORK_OK, FORK_ERR_INVALID_ARG, FORK_ERR_CUDA, FORK_ERR_WORKSPACE, FORK_ERR_MAX_S
 FORK_BF16, FORK_F32 = 0, 1
 FORK_ROW_NONFINITE, FORK_ROW_BAD_TOKEN = 1, 2
 FORK_DEV_WINDOW_CLAMPED, FORK_DEV_TIMEOUT = 1, 2
+FORK_FALLBACK_LEFTMOST, FORK_FALLBACK_MAX_CONF, FORK_FALLBACK_MIN_CONF, FORK_FALLBACK_MAX_ENTROPY, \
+    FORK_FALLBACK_RANDOM = 0, 1, 2, 3, 4
 FORK_TUNE_VARIANT, FORK_TUNE_CTAS_PER_SM, FORK_TUNE_PDL, FORK_TUNE_STAGES = 0, 1, 2, 3
 
 
@@ -33,6 +35,8 @@ class fork_step_args(C.Structure):
         ("commit_step", C.c_void_p), ("commit_fallback", C.c_void_p), ("commit_logp", C.c_void_p),
         ("n_unmasked", C.c_void_p), ("is_fallback", C.c_void_p), ("fallback_pos", C.c_void_p),
         ("nfe", C.c_void_p), ("n_fallback", C.c_void_p),
+        ("fallback_mode", C.c_int32), ("fallback_rand", C.c_void_p),
+        ("temperature", C.c_float), ("sample_seed", C.c_uint64),
     ]
 
 
@@ -170,7 +174,8 @@ class ForkState:
 
 
 def make_step_args(st: ForkState, logits: torch.Tensor, blk_lo, blk_hi, threshold: float, step: int = 0,
-                   pos0: int = 0) -> fork_step_args:
+                   pos0: int = 0, fallback_mode: int = FORK_FALLBACK_LEFTMOST, fallback_rand=None,
+                   temperature: float = 0.0, sample_seed: int = 0) -> fork_step_args:
     assert logits.dim() == 3 and logits.stride(2) == 1, "logits must be [B, Ll, V] with V contiguous"
     B, Ll, V = logits.shape
     assert B == st.B
@@ -183,13 +188,16 @@ def make_step_args(st: ForkState, logits: torch.Tensor, blk_lo, blk_hi, threshol
     a.threshold, a.step = float(threshold), int(step)
     for name, _, _ in ForkState.PER_POS + ForkState.PER_SEQ:
         setattr(a, name, getattr(st, name).data_ptr())
+    a.fallback_mode, a.fallback_rand = int(fallback_mode), _p(fallback_rand)
+    a.temperature, a.sample_seed = float(temperature), int(sample_seed)
     return a
 
 
 def fork_step(st: ForkState, logits: torch.Tensor, blk_lo: torch.Tensor, blk_hi: torch.Tensor, threshold: float,
-              step: int = 0, pos0: int = 0, stream=None) -> None:
-    """One Fork-dLLM sampling step on device buffers (asynchronous on the stream)."""
-    a = make_step_args(st, logits, blk_lo, blk_hi, threshold, step, pos0)
+              step: int = 0, pos0: int = 0, stream=None, **variant) -> None:
+    """One sampling step on device buffers (asynchronous on the stream).  `variant` takes the
+    fallback_mode / fallback_rand / temperature / sample_seed fields of fork_step_args."""
+    a = make_step_args(st, logits, blk_lo, blk_hi, threshold, step, pos0, **variant)
     rc = lib().fork_step(C.byref(a), C.c_void_p(st.ws_ptr), st.ws_bytes, _stream_ptr(stream))
     if rc != FORK_OK:
         raise ForkError(rc, "fork_step")
@@ -236,12 +244,12 @@ def fork_logprob(logits: torch.Tensor, tokens: torch.Tensor, select: torch.Tenso
 
 def fork_decode_loop(st: ForkState, logits: torch.Tensor, block_len: int, gen_lo: int, gen_hi: int, provider,
                      ctx, threshold: float, max_steps: int, step0: int = 0, pos0: int = 0, stream=None,
-                     raise_on_error: bool = True):
+                     raise_on_error: bool = True, **variant):
     """Semi-autoregressive decoding.  `provider` is either a C function pointer (int address or
     ctypes function) with the fork_logits_fn signature plus its `ctx` pointer, or a Python callable
     ``provider(step, lo_ptr, hi_ptr, stream_ptr) -> int`` that enqueues the work filling `logits`.
     Returns (status, steps_taken)."""
-    a = make_step_args(st, logits, None, None, threshold, step0, pos0)
+    a = make_step_args(st, logits, None, None, threshold, step0, pos0, **variant)
     keep = None
     if callable(provider) and not isinstance(provider, (int, C._CFuncPtr)):
         def _tramp(_ctx, step, _tok, _mask, lo, hi, _out, stream_p):

@@ -94,6 +94,7 @@ struct ReduceParams {
   float* conf; int32_t* cand; float* entropy; float* logp; uint32_t* row_status;
   int32_t* commit_step; uint8_t* commit_fallback; float* commit_logp;
   int32_t* n_unmasked; uint8_t* is_fallback; int32_t* fallback_pos; int32_t* nfe; int32_t* n_fallback;
+  int fallback_mode; const uint32_t* fallback_rand;
   /* log-probability mode */
   const int32_t* lp_tokens; float* lp_out; float* seq_sum; int32_t* seq_cnt;
 };
@@ -385,17 +386,29 @@ __device__ __forceinline__ SeqHint load_seq_hint(const ReduceParams& p, int b) {
   return h;
 }
 
+/* Key by which a fallback step ranks a row under the orders other than "leftmost" (the largest key
+   wins, equal keys go to the lower row): the confidence (Algorithm 1), its negative, or the token
+   entropy (the ablations of Section 4.1).  Flagged rows rank below every other row. */
+__device__ __forceinline__ float fallback_key(int mode, float conf, float entropy, bool bad) {
+  if (bad) return -INFINITY;
+  return mode == FORK_FALLBACK_MAX_CONF ? conf : (mode == FORK_FALLBACK_MIN_CONF ? -conf : entropy);
+}
+
 /* The unmask rule for one sequence, run by one warp once every part of the sequence has arrived
-   (Algorithm 2 lines 6-9): commit every live position whose confidence exceeds lambda, or the
-   leftmost live position when none does; write tokens, mask and the per-token records. */
+   (Algorithm 2 lines 6-9): commit every live position whose confidence exceeds lambda, or one
+   position when none does -- the leftmost live one (Fork-dLLM), or the one the requested
+   comparison order picks; write tokens, mask and the per-token records. */
 template <typename T>
 __device__ void finalize_step_sequence(const ReduceParams& p, const PartitionCtx& c, int b, const SeqHint& h) {
   const int lane = threadIdx.x & 31;
   const int r0 = h.r0, r1 = h.r1;
   const bool one_batch = (r1 - r0) <= 32;                    /* the usual case: results stay in registers */
+  const bool ranked = p.fallback_mode >= FORK_FALLBACK_MAX_CONF && p.fallback_mode <= FORK_FALLBACK_MAX_ENTROPY;
   int any = 0;
   float4 keep = make_float4(0.f, 0.f, 0.f, 0.f);
   int keep_k = 0;
+  float best_key = -INFINITY;                                /* this lane's best row under a ranked order */
+  int best_r = 0x7fffffff;
   for (int base = r0; base < r1; base += 32) {
     Part merged; int k;
     const RowOut o = finalize_rows_warp<T, true>(p, c, b, base, r1, merged, k, base == r0 ? h.k : -1);
@@ -411,19 +424,37 @@ __device__ void finalize_step_sequence(const ReduceParams& p, const PartitionCtx
       keep_k = k;
       if (!one_batch) p.final_rec[r] = keep;
       any |= (o.conf > p.threshold) ? 1 : 0;                 /* U_t non-empty (Algorithm 2, line 6) */
+      if (ranked) {
+        const float key = fallback_key(p.fallback_mode, o.conf, o.entropy, o.status != 0u);
+        if (key > best_key) { best_key = key; best_r = r; }  /* rows ascend within a lane: strict > keeps the lower */
+      }
     }
   }
   any = __any_sync(0xffffffffu, any);
   const int fb = any ? 0 : 1;                                /* fallback step: max_k c <= lambda */
-  int count = 0;
+  int pick = r0;                                             /* leftmost(M_t) inside the block */
+  if (fb && ranked) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ok = __shfl_xor_sync(0xffffffffu, best_key, o);
+      const int orow = __shfl_xor_sync(0xffffffffu, best_r, o);
+      if (ok > best_key || (ok == best_key && orow < best_r)) { best_key = ok; best_r = orow; }
+    }
+    if (best_key > -INFINITY) pick = best_r;                 /* every row flagged: stay with the leftmost */
+  } else if (fb && p.fallback_mode == FORK_FALLBACK_RANDOM) {
+    pick = r0 + (int)(p.fallback_rand[b] % (uint32_t)(r1 - r0));
+  }
+  int count = 0, pick_k = -1;
   for (int base = r0; base < r1; base += 32) {
     const int r = base + lane;
     bool commit = false;
     if (r < r1) {
       const float4 f = one_batch ? keep : p.final_rec[r];    /* written by this same lane above */
-      commit = fb ? (r == r0) : (f.x > p.threshold);         /* leftmost(M_t), or the threshold set */
+      commit = fb ? (r == pick) : (f.x > p.threshold);       /* the fallback position, or the threshold set */
       if (commit) {
-        const size_t at = (size_t)b * p.Lt + (one_batch ? keep_k : p.rows[r].y);
+        const int k = one_batch ? keep_k : p.rows[r].y;
+        const size_t at = (size_t)b * p.Lt + k;
+        if (fb) pick_k = k;
         p.tokens[at] = __float_as_int(f.z);
         p.mask[at] = 0;
         if (p.commit_step) p.commit_step[at] = p.step;
@@ -433,10 +464,14 @@ __device__ void finalize_step_sequence(const ReduceParams& p, const PartitionCtx
     }
     count += __popc(__ballot_sync(0xffffffffu, commit));
   }
+  if (fb) {                                                  /* exactly one lane committed: tell lane 0 where */
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) pick_k = max(pick_k, __shfl_xor_sync(0xffffffffu, pick_k, o));
+  }
   if (lane == 0) {
     if (p.n_unmasked) p.n_unmasked[b] = count;
     if (p.is_fallback) p.is_fallback[b] = (uint8_t)fb;
-    if (p.fallback_pos) p.fallback_pos[b] = fb ? (one_batch ? keep_k : p.rows[r0].y) : -1;
+    if (p.fallback_pos) p.fallback_pos[b] = pick_k;
     if (p.nfe) p.nfe[b] += 1;
     if (p.n_fallback) p.n_fallback[b] += fb;
   }
@@ -1021,6 +1056,7 @@ static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const i
   rp.commit_step = a->commit_step; rp.commit_fallback = a->commit_fallback; rp.commit_logp = a->commit_logp;
   rp.n_unmasked = a->n_unmasked; rp.is_fallback = a->is_fallback; rp.fallback_pos = a->fallback_pos;
   rp.nfe = a->nfe; rp.n_fallback = a->n_fallback;
+  rp.fallback_mode = a->fallback_mode; rp.fallback_rand = a->fallback_rand;
   if (launch_reduce(rp, a->dtype, mode, G, st) != cudaSuccess) return FORK_ERR_CUDA;
   return FORK_OK;
 }
@@ -1032,6 +1068,10 @@ static fork_status check_step_args(const fork_step_args* a, bool need_bounds) {
   if (!a->tokens || !a->mask) return FORK_ERR_INVALID_ARG;
   if (need_bounds && (!a->blk_lo || !a->blk_hi)) return FORK_ERR_INVALID_ARG;
   if (a->threshold != a->threshold) return FORK_ERR_INVALID_ARG;      /* NaN threshold */
+  if (a->fallback_mode < FORK_FALLBACK_LEFTMOST || a->fallback_mode > FORK_FALLBACK_RANDOM) return FORK_ERR_INVALID_ARG;
+  if (a->fallback_mode == FORK_FALLBACK_RANDOM && !a->fallback_rand) return FORK_ERR_INVALID_ARG;
+  if (!(a->temperature >= 0.f) || a->temperature > 3.0e38f) return FORK_ERR_INVALID_ARG;
+  if (a->temperature != 0.f) return FORK_ERR_INVALID_ARG;             /* stochastic candidates: not in this build yet */
   return FORK_OK;
 }
 
@@ -1172,6 +1212,7 @@ struct StagingView {
   float* conf; int32_t* cand; float* entropy; float* logp; uint32_t* row_status;
   int32_t* commit_step; uint8_t* commit_fallback; float* commit_logp;
   int32_t* n_unmasked; uint8_t* is_fallback; int32_t* fallback_pos; int32_t* nfe; int32_t* n_fallback;
+  uint32_t* fallback_rand;
   size_t logits_bytes, bytes;
 };
 
@@ -1192,6 +1233,7 @@ static StagingView staging_view(void* base, const fork_step_args* a) {
   v.commit_step = (int32_t*)take(n * 4); v.commit_fallback = (uint8_t*)take(n); v.commit_logp = (float*)take(n * 4);
   v.n_unmasked = (int32_t*)take(nb * 4); v.is_fallback = (uint8_t*)take(nb); v.fallback_pos = (int32_t*)take(nb * 4);
   v.nfe = (int32_t*)take(nb * 4); v.n_fallback = (int32_t*)take(nb * 4);
+  v.fallback_rand = (uint32_t*)take(nb * 4);
   v.bytes = off;
   return v;
 }
@@ -1221,6 +1263,7 @@ extern "C" fork_status fork_step_host(const fork_step_args* h, void* staging, si
   FORK_H2D(v.tokens, h->tokens, n * 4); FORK_H2D(v.mask, h->mask, n);
   FORK_H2D(v.lo, h->blk_lo, nb * 4); FORK_H2D(v.hi, h->blk_hi, nb * 4);
   FORK_H2D(v.nfe, h->nfe, nb * 4); FORK_H2D(v.n_fallback, h->n_fallback, nb * 4);
+  FORK_H2D(v.fallback_rand, h->fallback_rand, nb * 4);
   fork_step_args d = *h;
   d.logits = v.logits; d.tokens = v.tokens; d.mask = v.mask; d.blk_lo = v.lo; d.blk_hi = v.hi;
   d.conf = h->conf ? v.conf : nullptr; d.cand = h->cand ? v.cand : nullptr;
@@ -1232,6 +1275,7 @@ extern "C" fork_status fork_step_host(const fork_step_args* h, void* staging, si
   d.n_unmasked = h->n_unmasked ? v.n_unmasked : nullptr; d.is_fallback = h->is_fallback ? v.is_fallback : nullptr;
   d.fallback_pos = h->fallback_pos ? v.fallback_pos : nullptr;
   d.nfe = h->nfe ? v.nfe : nullptr; d.n_fallback = h->n_fallback ? v.n_fallback : nullptr;
+  d.fallback_rand = h->fallback_rand ? v.fallback_rand : nullptr;
   /* per-position outputs are written only on the live / committed set: start from the host's values */
   FORK_H2D(v.conf, h->conf, n * 4); FORK_H2D(v.cand, h->cand, n * 4); FORK_H2D(v.entropy, h->entropy, n * 4);
   FORK_H2D(v.logp, h->logp, n * 4); FORK_H2D(v.row_status, h->row_status, n * 4);

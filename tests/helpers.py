@@ -56,11 +56,30 @@ def live_mask(mask, lo, hi):
     return (mask != 0) & (k >= np.asarray(lo)[:, None]) & (k < np.asarray(hi)[:, None])
 
 
+FALLBACK_MARGIN = {0: 0.0, 1: 5e-4, 2: 5e-4, 3: 5e-3, 4: 0.0}   # per fallback order: keys are confidences (<=1) or entropies (<=12 nats)
+SAMPLE_MARGIN = 1e-3                                             # gap between the two largest perturbed keys (nats)
+
+
+def decisions_are_clear(st, live, threshold, margin, fallback_mode=0, temperature=0.0):
+    """True when no decision of the step just taken sits within rounding distance of flipping:
+    confidences against the threshold, the fallback order's best against its runner-up, and (with
+    stochastic candidates) the winning perturbed key against the second."""
+    if not (np.abs(st.conf[live] - np.float64(np.float32(threshold))) >= margin).all():
+        return False
+    if not (st.fallback_margin >= FALLBACK_MARGIN[fallback_mode]).all():
+        return False
+    if temperature > 0 and not (st.sample_margin[live] >= SAMPLE_MARGIN).all():
+        return False
+    return True
+
+
 def oracle_reference_loop(w: "fs.Workload", nseq: int, threshold: float, margin: float = 1e-4,
-                          max_steps: int = 100000, nthreads: int = 0):
+                          max_steps: int = 100000, nthreads: int = 0, fallback_mode: int = 0,
+                          fallback_rand=None, temperature: float = 0.0, sample_seed: int = 0):
     """The oracle's semi-autoregressive loop on the first `nseq` sequences of workload `w`, with
-    host-generated logits.  At every step the nonce is bumped until no live confidence lies within
-    `margin` of the threshold, so fp32 and fp64 cannot disagree on the unmask decision.
+    host-generated logits.  At every step the nonce is bumped until no decision of the step lies
+    within rounding distance of flipping (see decisions_are_clear), so fp32 and fp64 cannot
+    disagree on it.
     Returns (final StepState, per-step nonces, steps taken, per-step live-row counts)."""
     cfg = w.cfg(B=nseq)
     st = oracle.StepState(nseq, w.Lt)
@@ -76,8 +95,10 @@ def oracle_reference_loop(w: "fs.Workload", nseq: int, threshold: float, margin:
         while True:
             fs.fill_host(cfg, step, st.mask, lo, hi, logits, nonce=nonce, nthreads=nthreads)
             trial = copy.deepcopy(st)
-            assert oracle.step(trial, logits, lo, hi, threshold, step_id=step, nthreads=nthreads) == 0
-            if (np.abs(trial.conf[live] - np.float64(np.float32(threshold))) >= margin).all():
+            assert oracle.step(trial, logits, lo, hi, threshold, step_id=step, nthreads=nthreads,
+                               fallback_mode=fallback_mode, fallback_rand=fallback_rand, temperature=temperature,
+                               sample_seed=sample_seed) == 0
+            if decisions_are_clear(trial, live, threshold, margin, fallback_mode, temperature):
                 break
             nonce += 1
             assert nonce < 64
