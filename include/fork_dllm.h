@@ -207,6 +207,18 @@ size_t fork_staging_bytes(const fork_step_args* host_args);
 fork_status fork_step_host(const fork_step_args* host_args, void* staging, size_t staging_bytes,
                            void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * Position selection of JustGRPO-Fast (Section 3.2, last paragraph; Section 4.2 Setup): of the
+ * eligible positions of each rollout, mark the fraction `ratio` with the highest token entropy, as
+ * the `select` input of fork_logprob.  The count is floor(ratio * n), n = eligible positions of the
+ * rollout, and at least 1 when n > 0 and ratio > 0; equal entropies go to the lower position; NaN
+ * entropies rank last.  All pointers are device memory: entropy [B,Lt] (e.g. the `entropy` output of
+ * the decode loop), eligible [B,Lt] (non-zero = may be selected), select [B,Lt] out (0/1 at every
+ * position), n_selected [B] out, optional.  0 <= ratio <= 1, Lt <= 32768.  Asynchronous on `stream`.
+ */
+fork_status fork_select_top_entropy(const float* entropy, const uint8_t* eligible, int32_t B, int32_t Lt,
+                                    float ratio, uint8_t* select, int32_t* n_selected, void* stream);
+
 /* Copies the device status word of the last call that used `workspace` to *host_out
    (FORK_DEV_* bits) and synchronises `stream`. */
 fork_status fork_device_status(const void* workspace, uint32_t* host_out, void* stream);

@@ -53,6 +53,7 @@ fork_logits_fn = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32, C.c_void_p, C.c_voi
                              C.c_void_p, C.c_void_p)
 
 EXPORTS = ("fork_workspace_bytes", "fork_step", "fork_step_static", "fork_logprob", "fork_decode_loop", "fork_staging_bytes",
+           "fork_select_top_entropy",
            "fork_step_host", "fork_device_status", "fork_status_string", "fork_set_tuning",
            "fork_kernel_launches", "fork_set_timing_events")
 
@@ -95,6 +96,9 @@ def lib():
     L.fork_set_tuning.argtypes = [C.c_int32, C.c_int32]
     L.fork_kernel_launches.restype = C.c_int64
     L.fork_kernel_launches.argtypes = []
+    L.fork_select_top_entropy.restype = C.c_int
+    L.fork_select_top_entropy.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float, C.c_void_p,
+                                          C.c_void_p, C.c_void_p]
     L.fork_set_timing_events.restype = None
     L.fork_set_timing_events.argtypes = [C.c_void_p, C.c_void_p]
     _lib = L
@@ -280,3 +284,18 @@ def fork_device_status(st: ForkState, stream=None) -> int:
     if rc != FORK_OK:
         raise ForkError(rc, "fork_device_status")
     return int(out.value)
+
+
+def fork_select_top_entropy(entropy: torch.Tensor, eligible: torch.Tensor, ratio: float, stream=None):
+    """JustGRPO-Fast's selection: returns (select [B,Lt] uint8, n_selected [B] int32) device tensors."""
+    assert entropy.dtype == torch.float32 and eligible.dtype == torch.uint8
+    assert entropy.is_contiguous() and eligible.is_contiguous() and entropy.shape == eligible.shape
+    B, Lt = entropy.shape
+    select = torch.empty((B, Lt), dtype=torch.uint8, device=entropy.device)
+    cnt = torch.empty((B,), dtype=torch.int32, device=entropy.device)
+    rc = lib().fork_select_top_entropy(C.c_void_p(entropy.data_ptr()), C.c_void_p(eligible.data_ptr()), B, Lt,
+                                       C.c_float(ratio), C.c_void_p(select.data_ptr()), C.c_void_p(cnt.data_ptr()),
+                                       _stream_ptr(stream))
+    if rc != FORK_OK:
+        raise ForkError(rc, "fork_select_top_entropy")
+    return select, cnt

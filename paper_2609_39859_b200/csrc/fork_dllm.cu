@@ -1206,6 +1206,71 @@ extern "C" fork_status fork_step_static(const fork_step_args* a, void* stream) {
   return step_impl(a, a->blk_lo, a->blk_hi, ws, (cudaStream_t)stream);
 }
 
+/* ---- top-entropy position selection (JustGRPO-Fast; Section 3.2, last paragraph) ------------ */
+/* One CTA per rollout.  Keys sit in shared memory: the entropy of an eligible position (-inf when it
+   is NaN, so that it ranks last), NaN for a position that is not eligible.  Position i is selected
+   when fewer than `want` eligible positions rank before it (higher entropy, or equal entropy and a
+   lower position). */
+constexpr int kSelectNT = 256;
+constexpr int kSelectMaxLt = 32768;
+
+__global__ void __launch_bounds__(kSelectNT) select_top_entropy_kernel(const float* __restrict__ entropy,
+                                                                      const uint8_t* __restrict__ eligible, int Lt,
+                                                                      float ratio, uint8_t* __restrict__ select,
+                                                                      int32_t* __restrict__ n_selected) {
+  extern __shared__ float sel_key[];
+  __shared__ int sh_n;
+  const int b = blockIdx.x, tid = threadIdx.x;
+  if (tid == 0) sh_n = 0;
+  __syncthreads();
+  int mine = 0;
+  for (int k = tid; k < Lt; k += kSelectNT) {
+    const size_t at = (size_t)b * Lt + k;
+    float key = __int_as_float(0x7fc00000);
+    if (eligible[at]) { const float h = entropy[at]; key = (h != h) ? -INFINITY : h; ++mine; }
+    sel_key[k] = key;
+  }
+  if (mine) atomicAdd(&sh_n, mine);
+  __syncthreads();
+  const int n = sh_n;
+  int want = (int)floor((double)ratio * (double)n);
+  if (want < 1 && n > 0 && ratio > 0.f) want = 1;
+  for (int i = tid; i < Lt; i += kSelectNT) {
+    const float ki = sel_key[i];
+    uint8_t out = 0;
+    if (ki == ki && want > 0) {
+      int before = 0;
+      for (int j = 0; j < Lt; ++j) {
+        const float kj = sel_key[j];                          /* a comparison with NaN is false: not eligible */
+        before += (kj > ki || (kj == ki && j < i)) ? 1 : 0;
+      }
+      out = before < want ? 1 : 0;
+    }
+    select[(size_t)b * Lt + i] = out;
+  }
+  if (tid == 0 && n_selected) n_selected[b] = want;
+}
+
+extern "C" fork_status fork_select_top_entropy(const float* entropy, const uint8_t* eligible, int32_t B, int32_t Lt,
+                                               float ratio, uint8_t* select, int32_t* n_selected, void* stream) {
+  if (!entropy || !eligible || !select || B < 0 || Lt <= 0 || Lt > kSelectMaxLt) return FORK_ERR_INVALID_ARG;
+  if (!(ratio >= 0.f) || ratio > 1.f) return FORK_ERR_INVALID_ARG;
+  if (B == 0) return FORK_OK;
+  const size_t smem = (size_t)Lt * sizeof(float);
+  static std::atomic<int> raised[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FORK_ERR_CUDA;
+  if (smem > 48 * 1024 && (dev >= 64 || !raised[dev].load())) {
+    if (cudaFuncSetAttribute(select_top_entropy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kSelectMaxLt * (int)sizeof(float)) != cudaSuccess) return FORK_ERR_CUDA;
+    if (dev < 64) raised[dev].store(1);
+  }
+  select_top_entropy_kernel<<<B, kSelectNT, smem, (cudaStream_t)stream>>>(entropy, eligible, Lt, ratio, select, n_selected);
+  if (cudaGetLastError() != cudaSuccess) return FORK_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return FORK_OK;
+}
+
 /* ---- host-buffer entry point --------------------------------------------------------------- */
 struct StagingView {
   char* logits; int32_t* tokens; uint8_t* mask; int32_t* lo; int32_t* hi;

@@ -136,3 +136,49 @@ def test_bad_variant_arguments_are_rejected():
         with pytest.raises(pkg.ForkError) as e:
             pkg.fork_step(st, lg, lo, hi, 0.9, **kw)
         assert e.value.status == pkg.FORK_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("Lt,ratio", [(256, 0.2), (1024, 0.25), (37, 0.5), (20000, 0.01), (64, 0.0), (64, 1.0)])
+def test_top_entropy_selection_matches_the_oracle(Lt, ratio):
+    """JustGRPO-Fast's selection: both sides rank the same fp32 entropies, so the result is exact."""
+    pkg = F()
+    rng = np.random.default_rng(Lt)
+    B = 5
+    H = rng.gamma(2.0, 1.0, (B, Lt)).astype(np.float32)
+    H[1, : Lt // 2] = H[1, 0]                                   # many ties
+    H[2, ::5] = np.nan
+    elig = (rng.random((B, Lt)) < 0.7).astype(np.uint8)
+    elig[3] = 1
+    elig[4] = 0
+    rc, want_sel, want_cnt = oracle.select_top_entropy(H, elig, ratio)
+    assert rc == 0
+    sel, cnt = pkg.fork_select_top_entropy(torch.from_numpy(H).cuda(), torch.from_numpy(elig).cuda(), ratio)
+    torch.cuda.synchronize()
+    assert np.array_equal(cnt.cpu().numpy(), want_cnt)
+    assert np.array_equal(sel.cpu().numpy(), want_sel)
+
+
+def test_top_entropy_selection_feeds_the_scoring_pass():
+    """Entropies of a decode loop -> selection -> fork_logprob on the selected positions."""
+    pkg = F()
+    w = fs.workload("tiny")
+    B = 4
+    ost, nonces, osteps, _ = oracle_reference_loop(w, B, w.threshold)
+    rc, steps, calls, h = gpu_loop(w, w.threshold, nonces, B=B)
+    assert rc == 0
+    ent = torch.from_numpy(h["entropy"]).cuda()
+    elig = torch.ones((B, w.Lt), dtype=torch.uint8, device="cuda")
+    sel, cnt = pkg.fork_select_top_entropy(ent, elig, 0.2)
+    rc, osel, ocnt = oracle.select_top_entropy(h["entropy"], np.ones((B, w.Lt), np.uint8), 0.2)
+    assert np.array_equal(sel.cpu().numpy(), osel) and (ocnt == 6).all()        # floor(0.2 * 32)
+    rng = np.random.default_rng(1)
+    x = (rng.standard_normal((B, w.Lt, w.V)) * 2).astype(np.float32)
+    st = pkg.ForkState(B, w.Lt)
+    tokens = torch.from_numpy(h["tokens"]).cuda()
+    lp, ssum, scnt, status = pkg.fork_logprob(torch.from_numpy(x).cuda(), tokens, sel, st)
+    torch.cuda.synchronize()
+    rc, olp, osum, ocnt2, _ = oracle.logprob(x, h["tokens"], osel)
+    from helpers import assert_close
+    assert_close("logp", lp.cpu().numpy(), olp)
+    assert_close("seq_sum", ssum.cpu().numpy(), osum)
+    assert np.array_equal(scnt.cpu().numpy(), ocnt2)
