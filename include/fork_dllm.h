@@ -138,7 +138,52 @@ typedef struct fork_logprob_args {
   int32_t* seq_cnt;          /* [B] out, optional: number of selected positions (|F_i|) */
   uint32_t* row_status;      /* [B,Lt] out, optional: FORK_ROW_* bits at selected positions.
                                 A token outside [0,V) sets FORK_ROW_BAD_TOKEN and scores 0. */
+  float* lse;                /* [B,Lt] out, optional: log-sum-exp (max + ln sum exp) of every selected row,
+                                which fork_logprob_backward takes back; untouched elsewhere */
 } fork_logprob_args;
+
+/*
+ * The ForkGRPO objective (Eq. 2) on B = prompts * group rollouts, rollout i = prompt * group + j:
+ *     rho_{i,t} = exp(logp_new - logp_old) at the selected positions (the fallback steps F_i),
+ *     A_i       = (r_i - mean of its group) / (population standard deviation of its group);
+ *                 a group whose rewards are all equal is skipped (A_i = 0 for its rollouts),
+ *     obj_i     = 1/|F_i| * sum_t min(rho A_i, clip(rho, 1 - eps_lo, 1 + eps_hi) A_i), 0 if F_i is empty,
+ *     J         = 1/B * sum_i obj_i,
+ *     dlogp     = dJ/dlogp_new = rho A_i / (B |F_i|) where the unclipped term is the minimum, else 0.
+ * All pointers are device memory.
+ */
+typedef struct fork_grpo_args {
+  int32_t B, Lt, group;      /* B must be a multiple of group */
+  const float* logp_new;     /* [B,Lt] log q_theta(token) at the selected positions (fork_logprob) */
+  const float* logp_old;     /* [B,Lt] log q_theta_old(token) there (commit_logp of the rollout) */
+  const uint8_t* select;     /* [B,Lt] non-zero at the positions of F_i */
+  const float* reward;       /* [B] */
+  float eps_lo, eps_hi;      /* clip range [1 - eps_lo, 1 + eps_hi] */
+  float* seq_obj;            /* [B] out: obj_i */
+  float* objective;          /* [1] out, optional: J */
+  float* adv;                /* [B] out, optional: A_i */
+  float* ratio;              /* [B,Lt] out, optional: rho at selected positions, 0 elsewhere */
+  float* dlogp;              /* [B,Lt] out, optional: dJ/dlogp_new, 0 where not selected */
+  uint8_t* skipped;          /* [B/group] out, optional: 1 for a group with equal rewards */
+} fork_grpo_args;
+
+/*
+ * Derivative of the scored log-likelihoods with respect to the logits (the log-softmax backward
+ * of Section 3.2's likelihood terms): for every selected position with a token inside [0,V),
+ *     grad[b,k,v] = dlogp[b,k] * (1[v == token] - exp(logits[b,k,v] - lse[b,k])),
+ * written over the whole row in the logits' dtype (bf16: round to nearest even).  Rows of
+ * positions that are not selected, or whose token is outside [0,V), are not touched.
+ */
+typedef struct fork_logprob_bwd_args {
+  const void* logits; int64_t stride_b, stride_l; int32_t pos0;
+  int32_t B, Lt, Ll, V; int32_t dtype;
+  const int32_t* tokens;     /* [B,Lt] */
+  const uint8_t* select;     /* [B,Lt] */
+  const float* lse;          /* [B,Lt] from fork_logprob on the same logits */
+  const float* dlogp;        /* [B,Lt] upstream derivative (fork_grpo_loss) */
+  void* grad;                /* out: same dtype and row addressing as logits, with its own strides */
+  int64_t grad_stride_b, grad_stride_l;   /* in elements; grad_stride_l >= V */
+} fork_logprob_bwd_args;
 
 /* Device scratch needed by any entry point for a batch of B sequences of buffer length Lt. */
 size_t fork_workspace_bytes(int32_t B, int32_t Lt);
@@ -148,6 +193,12 @@ fork_status fork_step(const fork_step_args* args, void* workspace, size_t worksp
 
 /* Log-likelihood of given tokens at selected positions (Section 3.2).  Asynchronous on `stream`. */
 fork_status fork_logprob(const fork_logprob_args* args, void* workspace, size_t workspace_bytes, void* stream);
+
+/* The ForkGRPO objective and its derivative with respect to the new log-likelihoods.  Asynchronous. */
+fork_status fork_grpo_loss(const fork_grpo_args* args, void* stream);
+
+/* Log-softmax backward at the selected rows.  Asynchronous; uses the workspace like fork_logprob. */
+fork_status fork_logprob_backward(const fork_logprob_bwd_args* args, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * fork_step without a workspace argument, for callers that have no device memory to give and
@@ -161,7 +212,7 @@ fork_status fork_logprob(const fork_logprob_args* args, void* workspace, size_t 
  *
  *   - Same arguments, results and asynchrony as fork_step.
  *   - Batches whose scratch need, fork_workspace_bytes(B, Lt), exceeds FORK_STATIC_SCRATCH_BYTES are
- *     rejected with FORK_ERR_WORKSPACE before anything is launched (B*Lt up to about 50,000
+ *     rejected with FORK_ERR_WORKSPACE before anything is launched (B*Lt up to about 42,000
  *     positions fits).
  *   - The first call on each device looks up the array's device address (one cudaGetSymbolAddress,
  *     with that device current) and caches it; make that first call outside any stream capture.

@@ -45,7 +45,26 @@ class fork_logprob_args(C.Structure):
         ("logits", C.c_void_p), ("stride_b", C.c_int64), ("stride_l", C.c_int64), ("pos0", C.c_int32),
         ("B", C.c_int32), ("Lt", C.c_int32), ("Ll", C.c_int32), ("V", C.c_int32), ("dtype", C.c_int32),
         ("tokens", C.c_void_p), ("select", C.c_void_p), ("logp", C.c_void_p), ("seq_sum", C.c_void_p),
-        ("seq_cnt", C.c_void_p), ("row_status", C.c_void_p),
+        ("seq_cnt", C.c_void_p), ("row_status", C.c_void_p), ("lse", C.c_void_p),
+    ]
+
+
+class fork_grpo_args(C.Structure):
+    _fields_ = [
+        ("B", C.c_int32), ("Lt", C.c_int32), ("group", C.c_int32),
+        ("logp_new", C.c_void_p), ("logp_old", C.c_void_p), ("select", C.c_void_p), ("reward", C.c_void_p),
+        ("eps_lo", C.c_float), ("eps_hi", C.c_float),
+        ("seq_obj", C.c_void_p), ("objective", C.c_void_p), ("adv", C.c_void_p), ("ratio", C.c_void_p),
+        ("dlogp", C.c_void_p), ("skipped", C.c_void_p),
+    ]
+
+
+class fork_logprob_bwd_args(C.Structure):
+    _fields_ = [
+        ("logits", C.c_void_p), ("stride_b", C.c_int64), ("stride_l", C.c_int64), ("pos0", C.c_int32),
+        ("B", C.c_int32), ("Lt", C.c_int32), ("Ll", C.c_int32), ("V", C.c_int32), ("dtype", C.c_int32),
+        ("tokens", C.c_void_p), ("select", C.c_void_p), ("lse", C.c_void_p), ("dlogp", C.c_void_p),
+        ("grad", C.c_void_p), ("grad_stride_b", C.c_int64), ("grad_stride_l", C.c_int64),
     ]
 
 
@@ -53,7 +72,7 @@ fork_logits_fn = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32, C.c_void_p, C.c_voi
                              C.c_void_p, C.c_void_p)
 
 EXPORTS = ("fork_workspace_bytes", "fork_step", "fork_step_static", "fork_logprob", "fork_decode_loop", "fork_staging_bytes",
-           "fork_select_top_entropy",
+           "fork_select_top_entropy", "fork_grpo_loss", "fork_logprob_backward",
            "fork_step_host", "fork_device_status", "fork_status_string", "fork_set_tuning",
            "fork_kernel_launches", "fork_set_timing_events")
 
@@ -99,6 +118,10 @@ def lib():
     L.fork_select_top_entropy.restype = C.c_int
     L.fork_select_top_entropy.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float, C.c_void_p,
                                           C.c_void_p, C.c_void_p]
+    L.fork_grpo_loss.restype = C.c_int
+    L.fork_grpo_loss.argtypes = [C.POINTER(fork_grpo_args), C.c_void_p]
+    L.fork_logprob_backward.restype = C.c_int
+    L.fork_logprob_backward.argtypes = [C.POINTER(fork_logprob_bwd_args), C.c_void_p, C.c_size_t, C.c_void_p]
     L.fork_set_timing_events.restype = None
     L.fork_set_timing_events.argtypes = [C.c_void_p, C.c_void_p]
     _lib = L
@@ -222,9 +245,10 @@ def fork_step_static(st: ForkState, logits: torch.Tensor, blk_lo: torch.Tensor, 
 
 
 def fork_logprob(logits: torch.Tensor, tokens: torch.Tensor, select: torch.Tensor, st: ForkState, pos0: int = 0,
-                 stream=None):
+                 stream=None, want_lse: bool = False):
     """Log-likelihood of `tokens` at the selected positions; returns (logp [B,Lt], seq_sum [B],
-    seq_cnt [B], row_status [B,Lt]) as device tensors (asynchronous on the stream)."""
+    seq_cnt [B], row_status [B,Lt]) as device tensors (asynchronous on the stream), plus the
+    rows' log-sum-exp [B,Lt] (for fork_logprob_backward) when `want_lse`."""
     assert logits.dim() == 3 and logits.stride(2) == 1
     B, Ll, V = logits.shape
     Lt = tokens.shape[1]
@@ -240,10 +264,12 @@ def fork_logprob(logits: torch.Tensor, tokens: torch.Tensor, select: torch.Tenso
     assert tokens.dtype == torch.int32 and select.dtype == torch.uint8 and tokens.is_contiguous() and select.is_contiguous()
     a.tokens, a.select = tokens.data_ptr(), select.data_ptr()
     a.logp, a.seq_sum, a.seq_cnt, a.row_status = logp.data_ptr(), seq_sum.data_ptr(), seq_cnt.data_ptr(), status.data_ptr()
+    lse = torch.zeros((B, Lt), dtype=torch.float32, device=dev) if want_lse else None
+    a.lse = _p(lse)
     rc = lib().fork_logprob(C.byref(a), C.c_void_p(st.ws_ptr), st.ws_bytes, _stream_ptr(stream))
     if rc != FORK_OK:
         raise ForkError(rc, "fork_logprob")
-    return logp, seq_sum, seq_cnt, status
+    return (logp, seq_sum, seq_cnt, status, lse) if want_lse else (logp, seq_sum, seq_cnt, status)
 
 
 def fork_decode_loop(st: ForkState, logits: torch.Tensor, block_len: int, gen_lo: int, gen_hi: int, provider,
@@ -299,3 +325,46 @@ def fork_select_top_entropy(entropy: torch.Tensor, eligible: torch.Tensor, ratio
     if rc != FORK_OK:
         raise ForkError(rc, "fork_select_top_entropy")
     return select, cnt
+
+
+def fork_grpo_loss(logp_new: torch.Tensor, logp_old: torch.Tensor, select: torch.Tensor, reward: torch.Tensor,
+                   group: int, eps_lo: float, eps_hi: float, stream=None) -> dict:
+    """The ForkGRPO objective (Eq. 2) and its derivative with respect to logp_new; device tensors."""
+    for t, dt in ((logp_new, torch.float32), (logp_old, torch.float32), (select, torch.uint8), (reward, torch.float32)):
+        assert t.dtype == dt and t.is_contiguous()
+    B, Lt = logp_new.shape
+    dev = logp_new.device
+    out = dict(seq_obj=torch.empty(B, dtype=torch.float32, device=dev),
+               objective=torch.empty(1, dtype=torch.float32, device=dev),
+               adv=torch.empty(B, dtype=torch.float32, device=dev),
+               ratio=torch.empty((B, Lt), dtype=torch.float32, device=dev),
+               dlogp=torch.empty((B, Lt), dtype=torch.float32, device=dev),
+               skipped=torch.empty(max(B // max(group, 1), 1), dtype=torch.uint8, device=dev))
+    a = fork_grpo_args()
+    a.B, a.Lt, a.group = B, Lt, group
+    a.logp_new, a.logp_old, a.select, a.reward = (t.data_ptr() for t in (logp_new, logp_old, select, reward))
+    a.eps_lo, a.eps_hi = float(eps_lo), float(eps_hi)
+    for name, t in out.items():
+        setattr(a, name, t.data_ptr())
+    rc = lib().fork_grpo_loss(C.byref(a), _stream_ptr(stream))
+    if rc != FORK_OK:
+        raise ForkError(rc, "fork_grpo_loss")
+    return out
+
+
+def fork_logprob_backward(logits: torch.Tensor, tokens: torch.Tensor, select: torch.Tensor, lse: torch.Tensor,
+                          dlogp: torch.Tensor, grad: torch.Tensor, st: ForkState, pos0: int = 0, stream=None) -> None:
+    """Writes d(sum dlogp * logp)/d logits into the rows of `grad` ([B,Ll,V] like `logits`) that belong
+    to selected positions; other rows are left as they are."""
+    assert logits.dim() == 3 and logits.stride(2) == 1 and grad.dim() == 3 and grad.stride(2) == 1
+    assert grad.dtype == logits.dtype and grad.shape == logits.shape
+    B, Ll, V = logits.shape
+    a = fork_logprob_bwd_args()
+    a.logits = logits.data_ptr()
+    a.stride_b, a.stride_l, a.pos0 = logits.stride(0), logits.stride(1), pos0
+    a.B, a.Lt, a.Ll, a.V, a.dtype = B, tokens.shape[1], Ll, V, _dtype_code(logits)
+    a.tokens, a.select, a.lse, a.dlogp = tokens.data_ptr(), select.data_ptr(), lse.data_ptr(), dlogp.data_ptr()
+    a.grad, a.grad_stride_b, a.grad_stride_l = grad.data_ptr(), grad.stride(0), grad.stride(1)
+    rc = lib().fork_logprob_backward(C.byref(a), C.c_void_p(st.ws_ptr), st.ws_bytes, _stream_ptr(stream))
+    if rc != FORK_OK:
+        raise ForkError(rc, "fork_logprob_backward")

@@ -30,7 +30,8 @@ constexpr int kNT = 256;             /* threads per CTA of the streaming kernel 
 constexpr int kUnroll = 4;           /* 128-bit loads in flight per thread */
 constexpr int kSetupNT = 1024;       /* threads of the one-CTA set-up kernels */
 
-enum Mode { kModeStep = 0, kModeLogprob = 1 };
+enum Mode { kModeStep = 0, kModeLogprob = 1, kModeSample = 2 };   /* kModeSample: a step with stochastic candidates (tau > 0) */
+__host__ __device__ constexpr bool mode_is_step(int mode) { return mode != kModeLogprob; }
 
 /* ---- workspace ---------------------------------------------------------------------------- */
 struct WsHeader {                    /* 256 bytes at the start of the workspace */
@@ -53,6 +54,7 @@ struct WsView {
   int2* rows;                        /* [B*Lt] (b, k) of each live row, ascending */
   float4* final_rec;                 /* [B*Lt] per-row results kept between the finaliser's passes */
   float4* parts;                     /* [B*Lt + FORK_MAX_GRID] partial results, slot r+g */
+  float2* kparts;                    /* [B*Lt + FORK_MAX_GRID] best perturbed key of each part (stochastic candidates) */
   size_t bytes;
 };
 
@@ -72,6 +74,7 @@ static WsView ws_view(void* base, int32_t B, int32_t Lt) {
   v.rows = (int2*)(p + off); off = align_up(off + rows * sizeof(int2), 256);
   v.final_rec = (float4*)(p + off); off = align_up(off + rows * sizeof(float4), 256);
   v.parts = (float4*)(p + off); off = align_up(off + (rows + FORK_MAX_GRID) * sizeof(float4), 256);
+  v.kparts = (float2*)(p + off); off = align_up(off + (rows + FORK_MAX_GRID) * sizeof(float2), 256);
   v.bytes = off;
   return v;
 }
@@ -88,15 +91,16 @@ struct ReduceParams {
   int B, Lt, C, fast;
   /* workspace */
   const WsHeader* hdr; const int32_t* seq_off; const int32_t* expected; int32_t* ticket;
-  const int2* rows; float4* final_rec; float4* parts;
+  const int2* rows; float4* final_rec; float4* parts; float2* kparts;
   /* step mode */
   int32_t* tokens; uint8_t* mask; float threshold; int32_t step;
   float* conf; int32_t* cand; float* entropy; float* logp; uint32_t* row_status;
   int32_t* commit_step; uint8_t* commit_fallback; float* commit_logp;
   int32_t* n_unmasked; uint8_t* is_fallback; int32_t* fallback_pos; int32_t* nfe; int32_t* n_fallback;
   int fallback_mode; const uint32_t* fallback_rand;
+  float noise_c; unsigned long long sample_seed;      /* stochastic candidates: log2(e)/tau and the noise stream */
   /* log-probability mode */
-  const int32_t* lp_tokens; float* lp_out; float* seq_sum; int32_t* seq_cnt;
+  const int32_t* lp_tokens; float* lp_out; float* seq_sum; int32_t* seq_cnt; float* lse_out;
 };
 
 template <typename T>
@@ -340,9 +344,22 @@ __device__ Part careful_row_warp(const T* row, int V, bool& bad) {
   return Part{m, s, t, idx};
 }
 
+__device__ __forceinline__ KeyPart key_from(const float2& v) { return KeyPart{v.x, __float_as_int(v.y)}; }
+
+/* Largest perturbed key of row r over its n parts (slots r+g0 ...), by one lane. */
+__device__ __forceinline__ KeyPart merge_row_keys(const ReduceParams& p, int r, int g0, int n) {
+  const float2* q = p.kparts + (r + g0);
+  KeyPart acc = key_empty();
+#pragma unroll 4
+  for (int j = 0; j < n; ++j) acc = key_merge(acc, key_from(__ldcg(q + j)));
+  return acc;
+}
+
 /* Final statistics of up to 32 rows (one per lane) of sequence b starting at row `base`.
-   Rows whose streamed result is not finite are re-read by the whole warp with the guarded routine. */
-template <typename T, bool WANT_INDEX>
+   Rows whose streamed result is not finite are re-read by the whole warp with the guarded routine.
+   With SAMPLE the candidate is the drawn token (the element holding the row's largest perturbed
+   key) and confidence / log-probability are those of that token; flagged rows keep the arg-max. */
+template <typename T, bool WANT_INDEX, bool SAMPLE>
 __device__ __forceinline__ RowOut finalize_rows_warp(const ReduceParams& p, const PartitionCtx& c, int b, int base,
                                                      int r1, Part& merged, int& k, int k_hint) {
   const int lane = threadIdx.x & 31;
@@ -371,6 +388,15 @@ __device__ __forceinline__ RowOut finalize_rows_warp(const ReduceParams& p, cons
     const Part cp = careful_row_warp<T>(row_ptr<T>(p.src, b, kk), p.src.V, bd);
     if (lane == src) { merged = cp; bad = bd; }
   }
+  if (SAMPLE) {
+    float xs = 0.f;
+    if (valid && !bad) {
+      const KeyPart kp = merge_row_keys(p, r, g0, nparts);
+      const NoiseRow nz = noise_row(p.sample_seed, p.step, b, k, p.noise_c);
+      merged.idx = resolve_sample<T>(row_ptr<T>(p.src, b, k), nz, kp.vec, p.src.V, kp.key, xs);
+    }
+    return row_out_sampled(merged, bad, xs);
+  }
   if (valid && WANT_INDEX && !bad) merged.idx = resolve_index<T>(row_ptr<T>(p.src, b, k), merged.idx, p.src.V, merged.m);
   return row_out_from(merged, bad);
 }
@@ -398,7 +424,7 @@ __device__ __forceinline__ float fallback_key(int mode, float conf, float entrop
    (Algorithm 2 lines 6-9): commit every live position whose confidence exceeds lambda, or one
    position when none does -- the leftmost live one (Fork-dLLM), or the one the requested
    comparison order picks; write tokens, mask and the per-token records. */
-template <typename T>
+template <typename T, bool SAMPLE>
 __device__ void finalize_step_sequence(const ReduceParams& p, const PartitionCtx& c, int b, const SeqHint& h) {
   const int lane = threadIdx.x & 31;
   const int r0 = h.r0, r1 = h.r1;
@@ -411,7 +437,7 @@ __device__ void finalize_step_sequence(const ReduceParams& p, const PartitionCtx
   int best_r = 0x7fffffff;
   for (int base = r0; base < r1; base += 32) {
     Part merged; int k;
-    const RowOut o = finalize_rows_warp<T, true>(p, c, b, base, r1, merged, k, base == r0 ? h.k : -1);
+    const RowOut o = finalize_rows_warp<T, true, SAMPLE>(p, c, b, base, r1, merged, k, base == r0 ? h.k : -1);
     const int r = base + lane;
     if (r < r1) {
       const size_t at = (size_t)b * p.Lt + k;
@@ -486,7 +512,7 @@ __device__ void finalize_logprob_sequence(const ReduceParams& p, const Partition
   float local = 0.f;
   for (int base = r0; base < r1; base += 32) {
     Part merged; int k;
-    const RowOut o = finalize_rows_warp<T, false>(p, c, b, base, r1, merged, k, base == r0 ? h.k : -1);
+    const RowOut o = finalize_rows_warp<T, false, false>(p, c, b, base, r1, merged, k, base == r0 ? h.k : -1);
     const int r = base + lane;
     if (r < r1) {
       const size_t at = (size_t)b * p.Lt + k;
@@ -497,6 +523,7 @@ __device__ void finalize_logprob_sequence(const ReduceParams& p, const Partition
       else if (o.status) lp = o.logp;                        /* NaN for a non-finite row */
       else lp = (to_f32(row_ptr<T>(p.src, b, k)[tok]) - merged.m) + o.logp;   /* x_tok - m - ln s */
       p.lp_out[at] = lp;
+      if (p.lse_out) p.lse_out[at] = o.status ? o.logp : merged.m - o.logp;   /* m + ln s; NaN for a flagged row */
       if (p.row_status) p.row_status[at] = st;
       local += lp;
     }
@@ -511,10 +538,12 @@ __device__ void finalize_logprob_sequence(const ReduceParams& p, const Partition
 
 /* Lane 0 of the calling warp publishes one part of row r (sequence b) and takes a ticket; returns
    (to every lane) whether this was the last part the sequence was waiting for. */
-__device__ __forceinline__ bool publish_part(const ReduceParams& p, const Part& part, int r, int g, int b, int want) {
+__device__ __forceinline__ bool publish_part(const ReduceParams& p, const Part& part, int r, int g, int b, int want,
+                                             const KeyPart* kp = nullptr) {
   int last = 0;
   if ((threadIdx.x & 31) == 0) {
     p.parts[r + g] = make_float4(part.m, part.s, part.t, __int_as_float(part.idx));
+    if (kp) p.kparts[r + g] = make_float2(kp->key, __int_as_float(kp->vec));
     int old;                                 /* release our part, acquire everybody else's */
     asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(p.ticket + b) : "memory");
     last = (old + 1 == want) ? 1 : 0;
@@ -547,15 +576,18 @@ struct SegmentIter {
 /* ---- kernel 2a: direct 128-bit loads (also the path for buffers that are not 16-byte aligned) -- */
 struct Smem {
   Part parts[kNT / 32];
+  KeyPart keys[kNT / 32];
   float fl[kNT / 32];
   int flag;
 };
 
 template <typename T, int MODE>
 __global__ void __launch_bounds__(kNT, 4) reduce_select_kernel(ReduceParams p) {
-  constexpr bool WITH_T = (MODE == kModeStep);
+  constexpr bool WITH_T = mode_is_step(MODE);
+  constexpr bool SAMPLE = (MODE == kModeSample);
   __shared__ Smem sm;
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;");
   const int R = p.hdr->R;
   if (R <= 0) return;
   const PartitionCtx c = make_partition(R, p.C, (int)gridDim.x);
@@ -569,19 +601,28 @@ __global__ void __launch_bounds__(kNT, 4) reduce_select_kernel(ReduceParams p) {
     const int2 bk = p.rows[sg.r];
     const T* row = row_ptr<T>(p.src, bk.x, bk.y);
     Part part;
+    KeyTrack kt;
+    kt.init();
+    NoiseRow nz = NoiseRow{0u, 0u, 0.f};
+    if (SAMPLE) nz = noise_row(p.sample_seed, p.step, bk.x, bk.y, p.noise_c);
     if (p.fast) {
       part = part_block_reduce<kNT>(
-          stream_thread<T, WITH_T, kNT, kUnroll>(row, sg.e0, sg.e1, threadIdx.x, threadIdx.x == 0, sticky), sm.parts);
+          stream_thread<T, WITH_T, kNT, kUnroll, SAMPLE>(row, sg.e0, sg.e1, threadIdx.x, threadIdx.x == 0, sticky, &kt, &nz),
+          sm.parts);
     } else {
       bool bad;
       part = careful_segment<T, kNT>(row, sg.e0, sg.e1, sm.parts, sm.fl, bad);
+      if (SAMPLE)
+        for (int i = sg.e0 + (int)threadIdx.x; i < sg.e1; i += kNT) kt.one(nz, to_f32(row[i]), i);
     }
+    KeyPart kp = key_empty();
+    if (SAMPLE) kp = key_block_reduce<kNT>(kt.best, sm.keys);
     if (threadIdx.x < 32) {
-      const bool last = publish_part(p, part, sg.r, g, bk.x, p.expected[bk.x]);
+      const bool last = publish_part(p, part, sg.r, g, bk.x, p.expected[bk.x], SAMPLE ? &kp : nullptr);
       if (last) {                                           /* every part of sequence b has been delivered */
         const SeqHint h = load_seq_hint(p, bk.x);
-        if (MODE == kModeStep) finalize_step_sequence<T>(p, c, bk.x, h);
-        else finalize_logprob_sequence<T>(p, c, bk.x, h);
+        if (MODE == kModeLogprob) finalize_logprob_sequence<T>(p, c, bk.x, h);
+        else finalize_step_sequence<T, SAMPLE>(p, c, bk.x, h);
       }
     }
   }
@@ -610,6 +651,7 @@ constexpr int ring_stage_bytes(int cw) { return cw * 32 * kUnroll * 16; }   /* 1
 struct RingSmem {
   unsigned long long full[kMaxStages], empty[kMaxStages], mfull[kMail], mempty[kMail];
   Part mail[kMail][kMaxCW];
+  KeyPart kmail[kMail][kMaxCW];
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -643,7 +685,8 @@ __device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32
 
 template <typename T, int MODE, int kCW>
 __global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_select_ring_kernel(ReduceParams p, int n_stages) {
-  constexpr bool WITH_T = (MODE == kModeStep);
+  constexpr bool WITH_T = mode_is_step(MODE);
+  constexpr bool SAMPLE = (MODE == kModeSample);
   constexpr int VEC = 16 / (int)sizeof(T);
   constexpr int kCT = kCW * 32;                              /* consumer threads */
   constexpr int kStageVecs = kCT * kUnroll;                  /* 128-bit vectors per stage */
@@ -704,6 +747,10 @@ __global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_sel
     while (it.next(sg)) {
       Acc<T, WITH_T, false> a;
       a.init();
+      KeyTrack kt;                                            /* stochastic candidates: largest perturbed key */
+      kt.init();
+      NoiseRow nz = NoiseRow{0u, 0u, 0.f};
+      if (SAMPLE) { const int2 bk = p.rows[sg.r]; nz = noise_row(p.sample_seed, p.step, bk.x, bk.y, p.noise_c); }
       const int nvec = (sg.e1 - sg.e0) / VEC;
       for (int voff = 0; voff < nvec; voff += kStageVecs) {
         if (!mbar_wait(&rs.full[s], ph, p)) return;
@@ -719,6 +766,7 @@ __global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_sel
           __syncwarp();
           if (lane == 0) mbar_arrive(&rs.empty[s]);
           if (!sticky) a.template accumulate<kUnroll>(v);
+          if (SAMPLE) kt.template update<kUnroll>(T{}, nz, v, sg.e0 + (voff + ctid) * VEC, kCT * VEC);
         } else {
           /* the last, partly filled stage of a segment: same unrolled code, vectors past the end
              replaced by the clamp value (contributes 2^-huge = 0 and never wins the maximum
@@ -731,17 +779,29 @@ __global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_sel
           __syncwarp();
           if (lane == 0) mbar_arrive(&rs.empty[s]);
           if (!sticky) a.template accumulate<kUnroll>(v);
+          if (SAMPLE) {                                       /* only the vectors that exist draw noise */
+#pragma unroll
+            for (int j = 0; j < kUnroll; ++j)
+              if (ctid + j * kCT < nv) {
+                const uint4 one[1] = {v[j]};
+                kt.template update<1>(T{}, nz, one, sg.e0 + (voff + ctid + j * kCT) * VEC, kCT * VEC);
+              }
+          }
         }
         if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1u; }
       }
       const bool tail = (ctid == 0) && (sg.e0 + nvec * VEC < sg.e1);   /* fewer than VEC trailing elements */
       Part pt;
-      if (!sticky) {
-        if (tail) {
-          const int2 bk = p.rows[sg.r];
-          const T* row = row_ptr<T>(p.src, bk.x, bk.y);
-          for (int e = sg.e0 + nvec * VEC; e < sg.e1; ++e) a.one(to_f32(row[e]), e);
+      if (tail && (SAMPLE || !sticky)) {
+        const int2 bk = p.rows[sg.r];
+        const T* row = row_ptr<T>(p.src, bk.x, bk.y);
+        for (int e = sg.e0 + nvec * VEC; e < sg.e1; ++e) {
+          const float x = to_f32(row[e]);
+          if (!sticky) a.one(x, e);
+          if (SAMPLE) kt.one(nz, x, e);
         }
+      }
+      if (!sticky) {
         pt = a.part();
         if (!part_is_finite(pt)) sticky = true;
       }
@@ -752,10 +812,13 @@ __global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_sel
       }
       __syncwarp();
       pt = part_warp_reduce(pt);
+      KeyPart kp = key_empty();
+      if (SAMPLE) kp = key_warp_reduce(kt.best);
       if (lane == 0) {
         const uint32_t d = nseg % kMail, mph = (nseg / kMail) & 1u;
         if (mbar_wait(&rs.mempty[d], mph ^ 1u, p)) {
           rs.mail[d][warp] = pt;
+          if (SAMPLE) rs.kmail[d][warp] = kp;
           mbar_arrive(&rs.mfull[d]);
         }
       }
@@ -774,12 +837,15 @@ __global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_sel
     const uint32_t d = nseg % kMail, ph = (nseg / kMail) & 1u;
     if (!mbar_wait(&rs.mfull[d], ph, p)) return;
     Part pt = (lane < kCW) ? rs.mail[d][lane] : part_empty();
+    KeyPart kp = key_empty();
+    if (SAMPLE && lane < kCW) kp = rs.kmail[d][lane];
     __syncwarp();
     if (lane == 0) mbar_arrive(&rs.mempty[d]);
     pt = part_warp_reduce(pt);
-    if (publish_part(p, pt, sg.r, g, b, want)) {
-      if (MODE == kModeStep) finalize_step_sequence<T>(p, c, b, h);
-      else finalize_logprob_sequence<T>(p, c, b, h);
+    if (SAMPLE) kp = key_warp_reduce(kp);
+    if (publish_part(p, pt, sg.r, g, b, want, SAMPLE ? &kp : nullptr)) {
+      if (MODE == kModeLogprob) finalize_logprob_sequence<T>(p, c, b, h);
+      else finalize_step_sequence<T, SAMPLE>(p, c, b, h);
     }
     ++nseg;
   }
@@ -833,9 +899,9 @@ static std::atomic<int> g_tune[FORK_TUNE_COUNT_];
 static size_t ring_smem_bytes(int n_stages, int cw) { return (size_t)n_stages * ring_stage_bytes(cw) + sizeof(RingSmem); }
 
 /* two CTAs per SM with 8 consumer warps each (default), or one with 16 */
-static void ring_config(int* ctas_per_sm, int* n_stages, int* cw) {
+static void ring_config(int mode, int* ctas_per_sm, int* n_stages, int* cw) {
   int per_sm = g_tune[FORK_TUNE_CTAS_PER_SM].load();
-  if (per_sm != 1) per_sm = 2;
+  if (per_sm != 1 || mode == kModeSample) per_sm = 2;        /* the sampling kernel exists in the 8-warp form only */
   const int warps = (per_sm == 1) ? 16 : 8;
   int st = g_tune[FORK_TUNE_STAGES].load();
   const int max_st = (int)((220 * 1024 / per_sm - sizeof(RingSmem) - 1024) / ring_stage_bytes(warps));
@@ -845,7 +911,7 @@ static void ring_config(int* ctas_per_sm, int* n_stages, int* cw) {
   *ctas_per_sm = per_sm; *n_stages = st; *cw = warps;
 }
 
-struct DeviceInfo { int sms = 0; int occ[2][2] = {{0, 0}, {0, 0}}; bool ring_ready = false; };
+struct DeviceInfo { int sms = 0; int occ[2][3] = {{0, 0, 0}, {0, 0, 0}}; bool ring_ready = false; };
 static DeviceInfo g_dev[64];
 
 template <typename T, int MODE>
@@ -866,13 +932,16 @@ static bool device_info(DeviceInfo** out) {
     d.occ[0][1] = occupancy_of<bf16_t, kModeLogprob>();
     d.occ[1][0] = occupancy_of<float, kModeStep>();
     d.occ[1][1] = occupancy_of<float, kModeLogprob>();
+    d.occ[0][2] = occupancy_of<bf16_t, kModeSample>();
+    d.occ[1][2] = occupancy_of<float, kModeSample>();
     const int max_dyn = 220 * 1024;
     auto allow = [&](const void* fn) { return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn) == cudaSuccess; };
     d.ring_ready =
         allow((const void*)reduce_select_ring_kernel<bf16_t, kModeStep, 8>) && allow((const void*)reduce_select_ring_kernel<bf16_t, kModeLogprob, 8>) &&
         allow((const void*)reduce_select_ring_kernel<float, kModeStep, 8>) && allow((const void*)reduce_select_ring_kernel<float, kModeLogprob, 8>) &&
         allow((const void*)reduce_select_ring_kernel<bf16_t, kModeStep, 16>) && allow((const void*)reduce_select_ring_kernel<bf16_t, kModeLogprob, 16>) &&
-        allow((const void*)reduce_select_ring_kernel<float, kModeStep, 16>) && allow((const void*)reduce_select_ring_kernel<float, kModeLogprob, 16>);
+        allow((const void*)reduce_select_ring_kernel<float, kModeStep, 16>) && allow((const void*)reduce_select_ring_kernel<float, kModeLogprob, 16>) &&
+        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeSample, 8>) && allow((const void*)reduce_select_ring_kernel<float, kModeSample, 8>);
     if (!d.ring_ready) return false;
     d.sms = sms;
   }
@@ -884,7 +953,7 @@ static int grid_size(const DeviceInfo& d, int dtype, int mode, bool fast) {
   const int variant = g_tune[FORK_TUNE_VARIANT].load();
   if (fast && (variant == 0 || variant == 2)) {
     int per, stages, cw;
-    ring_config(&per, &stages, &cw);
+    ring_config(mode, &per, &stages, &cw);
     return d.sms * per;
   }
   int per_sm = g_tune[FORK_TUNE_CTAS_PER_SM].load();
@@ -967,7 +1036,11 @@ static cudaError_t launch_reduce_inner(const ReduceParams& rp, int dtype, int mo
   const bool pdl = g_tune[FORK_TUNE_PDL].load() >= 0;
   if (use_ring(rp)) {
     int per_sm, n_stages, cw;
-    ring_config(&per_sm, &n_stages, &cw);
+    ring_config(mode, &per_sm, &n_stages, &cw);
+    if (mode == kModeSample) {
+      if (dtype == FORK_BF16) return launch_ring<bf16_t, kModeSample, 8>(rp, G, n_stages, pdl, st);
+      return launch_ring<float, kModeSample, 8>(rp, G, n_stages, pdl, st);
+    }
     if (cw == 16) {
       if (dtype == FORK_BF16) {
         if (mode == kModeStep) return launch_ring<bf16_t, kModeStep, 16>(rp, G, n_stages, pdl, st);
@@ -982,6 +1055,10 @@ static cudaError_t launch_reduce_inner(const ReduceParams& rp, int dtype, int mo
     }
     if (mode == kModeStep) return launch_ring<float, kModeStep, 8>(rp, G, n_stages, pdl, st);
     return launch_ring<float, kModeLogprob, 8>(rp, G, n_stages, pdl, st);
+  }
+  if (mode == kModeSample) {
+    if (dtype == FORK_BF16) return launch(reduce_select_kernel<bf16_t, kModeSample>, dim3(G), dim3(kNT), st, pdl, rp);
+    return launch(reduce_select_kernel<float, kModeSample>, dim3(G), dim3(kNT), st, pdl, rp);
   }
   if (dtype == FORK_BF16) {
     if (mode == kModeStep) return launch(reduce_select_kernel<bf16_t, kModeStep>, dim3(G), dim3(kNT), st, pdl, rp);
@@ -1031,7 +1108,7 @@ static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const i
   DeviceInfo* dev;
   if (!device_info(&dev)) return FORK_ERR_CUDA;
   WsView w = ws_view(ws, a->B, a->Lt);
-  const int mode = kModeStep;
+  const int mode = a->temperature > 0.f ? kModeSample : kModeStep;
   const bool fast = source_is_vector_aligned(a->logits, a->stride_b, a->stride_l, a->dtype);
   const int G = grid_size(*dev, a->dtype, mode, fast);
   const int C = (a->V + FORK_CHUNK - 1) / FORK_CHUNK;
@@ -1050,7 +1127,9 @@ static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const i
   rp.B = a->B; rp.Lt = a->Lt; rp.C = C;
   rp.fast = fast ? 1 : 0;
   rp.hdr = w.hdr; rp.seq_off = w.seq_off; rp.expected = w.expected; rp.ticket = w.ticket;
-  rp.rows = w.rows; rp.final_rec = w.final_rec; rp.parts = w.parts;
+  rp.rows = w.rows; rp.final_rec = w.final_rec; rp.parts = w.parts; rp.kparts = w.kparts;
+  rp.noise_c = mode == kModeSample ? (float)(1.4426950408889634 / (double)a->temperature) : 0.f;
+  rp.sample_seed = a->sample_seed;
   rp.tokens = a->tokens; rp.mask = a->mask; rp.threshold = a->threshold; rp.step = a->step;
   rp.conf = a->conf; rp.cand = a->cand; rp.entropy = a->entropy; rp.logp = a->logp; rp.row_status = a->row_status;
   rp.commit_step = a->commit_step; rp.commit_fallback = a->commit_fallback; rp.commit_logp = a->commit_logp;
@@ -1071,7 +1150,6 @@ static fork_status check_step_args(const fork_step_args* a, bool need_bounds) {
   if (a->fallback_mode < FORK_FALLBACK_LEFTMOST || a->fallback_mode > FORK_FALLBACK_RANDOM) return FORK_ERR_INVALID_ARG;
   if (a->fallback_mode == FORK_FALLBACK_RANDOM && !a->fallback_rand) return FORK_ERR_INVALID_ARG;
   if (!(a->temperature >= 0.f) || a->temperature > 3.0e38f) return FORK_ERR_INVALID_ARG;
-  if (a->temperature != 0.f) return FORK_ERR_INVALID_ARG;             /* stochastic candidates: not in this build yet */
   return FORK_OK;
 }
 
@@ -1118,6 +1196,7 @@ extern "C" fork_status fork_logprob(const fork_logprob_args* a, void* ws, size_t
   rp.hdr = w.hdr; rp.seq_off = w.seq_off; rp.expected = w.expected; rp.ticket = w.ticket;
   rp.rows = w.rows; rp.final_rec = w.final_rec; rp.parts = w.parts;
   rp.lp_tokens = a->tokens; rp.lp_out = a->logp; rp.seq_sum = a->seq_sum; rp.seq_cnt = a->seq_cnt;
+  rp.lse_out = a->lse;
   rp.row_status = a->row_status;
   if (launch_reduce(rp, a->dtype, mode, G, st) != cudaSuccess) return FORK_ERR_CUDA;
   return FORK_OK;
@@ -1269,6 +1348,214 @@ extern "C" fork_status fork_select_top_entropy(const float* entropy, const uint8
   if (cudaGetLastError() != cudaSuccess) return FORK_ERR_CUDA;
   g_launches.fetch_add(1);
   return FORK_OK;
+}
+
+/* ---- ForkGRPO objective (Eq. 2) ------------------------------------------------------------- */
+/* One CTA per prompt group.  Group statistics in fp64 (a handful of values), the per-position terms
+   in fp32; one warp per rollout walks its positions twice (count of fallback steps, then the
+   terms).  A second one-CTA kernel sums the per-rollout objectives in a fixed order. */
+constexpr int kGrpoNT = 256;
+
+__global__ void __launch_bounds__(kGrpoNT) grpo_group_kernel(fork_grpo_args a) {
+  __shared__ double sh_mean, sh_sd;
+  const int p = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = kGrpoNT / 32;
+  const int G = a.group, B = a.B, Lt = a.Lt;
+  if (tid == 0) {
+    double mean = 0.0, var = 0.0;
+    for (int j = 0; j < G; ++j) mean += (double)a.reward[p * G + j];
+    mean /= G;
+    for (int j = 0; j < G; ++j) { const double d = (double)a.reward[p * G + j] - mean; var += d * d; }
+    sh_mean = mean; sh_sd = sqrt(var / G);
+    if (a.skipped) a.skipped[p] = (uint8_t)(!(sh_sd > 0.0));
+  }
+  __syncthreads();
+  const bool skip = !(sh_sd > 0.0);
+  for (int j = warp; j < G; j += nwarp) {
+    const int i = p * G + j;
+    const float A = skip ? 0.f : (float)(((double)a.reward[i] - sh_mean) / sh_sd);
+    int nf = 0;
+    for (int k0 = 0; k0 < Lt; k0 += 32) {
+      const int k = k0 + lane;
+      nf += __popc(__ballot_sync(0xffffffffu, k < Lt && a.select[(size_t)i * Lt + k] != 0));
+    }
+    const float scale = nf > 0 ? 1.f / ((float)B * (float)nf) : 0.f;
+    float acc = 0.f;
+    for (int k = lane; k < Lt; k += 32) {
+      const size_t at = (size_t)i * Lt + k;
+      float rho = 0.f, d = 0.f;
+      if (a.select[at]) {
+        rho = expf(a.logp_new[at] - a.logp_old[at]);
+        const float clipped = fminf(fmaxf(rho, 1.f - a.eps_lo), 1.f + a.eps_hi);
+        const float u = rho * A, c = clipped * A;
+        acc += (u <= c) ? u : c;                             /* the clipped minimum of Eq. 2 */
+        if (!skip && u <= c) d = rho * A * scale;            /* the unclipped term is active */
+      }
+      if (a.ratio) a.ratio[at] = rho;
+      if (a.dlogp) a.dlogp[at] = d;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) {
+      if (a.adv) a.adv[i] = A;
+      a.seq_obj[i] = nf > 0 ? acc / (float)nf : 0.f;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kGrpoNT) grpo_sum_kernel(const float* seq_obj, int B, float* objective) {
+  __shared__ double sh[kGrpoNT];
+  double acc = 0.0;
+  for (int i = threadIdx.x; i < B; i += kGrpoNT) acc += (double)seq_obj[i];
+  sh[threadIdx.x] = acc;
+  __syncthreads();
+  for (int o = kGrpoNT / 2; o > 0; o >>= 1) {
+    if ((int)threadIdx.x < o) sh[threadIdx.x] += sh[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *objective = B > 0 ? (float)(sh[0] / B) : 0.f;
+}
+
+extern "C" fork_status fork_grpo_loss(const fork_grpo_args* a, void* stream) {
+  if (!a || a->B < 0 || a->Lt <= 0 || a->group <= 0 || a->B % a->group != 0) return FORK_ERR_INVALID_ARG;
+  if (!a->logp_new || !a->logp_old || !a->select || !a->reward || !a->seq_obj) return FORK_ERR_INVALID_ARG;
+  if (!(a->eps_lo >= 0.f) || !(a->eps_hi >= 0.f)) return FORK_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (a->B > 0) {
+    grpo_group_kernel<<<a->B / a->group, kGrpoNT, 0, st>>>(*a);
+    if (cudaGetLastError() != cudaSuccess) return FORK_ERR_CUDA;
+    g_launches.fetch_add(1);
+  }
+  if (a->objective) {
+    grpo_sum_kernel<<<1, kGrpoNT, 0, st>>>(a->seq_obj, a->B, a->objective);
+    if (cudaGetLastError() != cudaSuccess) return FORK_ERR_CUDA;
+    g_launches.fetch_add(1);
+  }
+  return FORK_OK;
+}
+
+/* ---- derivative of the scored log-likelihoods with respect to the logits -------------------- */
+/* d/dx_v [w (x_tok - lse)] = w (1[v = tok] - p_v), p_v = exp(x_v - lse): one read of the row, one
+   write of the same size.  Work is cut into units of kBwdNT * kBwdVecs 128-bit vectors of one row;
+   the rows are those of the row list the active-set kernel built from `select`. */
+constexpr int kBwdNT = 256;
+constexpr int kBwdVecs = 2;
+
+struct BwdParams {
+  RowSource src; void* grad; long long gstride_b, gstride_l;
+  const WsHeader* hdr; const int2* rows;
+  const int32_t* tokens; const float* lse; const float* dlogp; int Lt, vector_ok;
+};
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ void store_grad(bf16_t* p, float g) {
+  p->bits = (uint16_t)(pack_bf16x2(g, 0.f) & 0xffffu);
+}
+__device__ __forceinline__ void store_grad(float* p, float g) { *p = g; }
+
+template <typename T>
+__global__ void __launch_bounds__(kBwdNT) logprob_backward_kernel(BwdParams p) {
+  constexpr int VEC = 16 / (int)sizeof(T);
+  constexpr int kUnitElems = kBwdNT * kBwdVecs * VEC;
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int R = p.hdr->R;
+  const int V = p.src.V;
+  const int units_per_row = (V + kUnitElems - 1) / kUnitElems;
+  const long long U = (long long)R * units_per_row;
+  for (long long u = blockIdx.x; u < U; u += gridDim.x) {
+    const int r = (int)(u / units_per_row);
+    const int e0 = (int)(u - (long long)r * units_per_row) * kUnitElems;
+    const int2 bk = p.rows[r];
+    const size_t at = (size_t)bk.x * p.Lt + bk.y;
+    const int tok = p.tokens[at];
+    if (tok < 0 || tok >= V) continue;                       /* scored as FORK_ROW_BAD_TOKEN: no gradient */
+    const float w = p.dlogp[at];
+    const float nl = -p.lse[at] * kLog2e;
+    const T* row = row_ptr<T>(p.src, bk.x, bk.y);
+    T* grow = reinterpret_cast<T*>(p.grad) + ((long long)bk.x * p.gstride_b + (long long)(bk.y - p.src.pos0) * p.gstride_l);
+    if (p.vector_ok) {
+      uint4 v[kBwdVecs];
+      int e[kBwdVecs];
+#pragma unroll
+      for (int j = 0; j < kBwdVecs; ++j) {
+        e[j] = e0 + ((int)threadIdx.x + j * kBwdNT) * VEC;
+        if (e[j] + VEC <= V) v[j] = ld_stream(reinterpret_cast<const uint4*>(row + e[j]));
+      }
+#pragma unroll
+      for (int j = 0; j < kBwdVecs; ++j) {
+        if (e[j] + VEC <= V) {
+          float x[VEC];
+          if (sizeof(T) == 2) {
+            x[0] = bf16_lo(v[j].x); x[1] = bf16_hi(v[j].x); x[2 % VEC] = bf16_lo(v[j].y); x[3 % VEC] = bf16_hi(v[j].y);
+            x[4 % VEC] = bf16_lo(v[j].z); x[5 % VEC] = bf16_hi(v[j].z); x[6 % VEC] = bf16_lo(v[j].w); x[7 % VEC] = bf16_hi(v[j].w);
+          } else {
+            x[0] = __uint_as_float(v[j].x); x[1] = __uint_as_float(v[j].y); x[2] = __uint_as_float(v[j].z); x[3] = __uint_as_float(v[j].w);
+          }
+          float gr[VEC];
+#pragma unroll
+          for (int q = 0; q < VEC; ++q) {
+            const float pr = ex2_approx(fmaf(x[q], kLog2e, nl));
+            gr[q] = w * ((e[j] + q == tok ? 1.f : 0.f) - pr);
+          }
+          uint4 o;
+          if (sizeof(T) == 2) {
+            o.x = pack_bf16x2(gr[0], gr[1]); o.y = pack_bf16x2(gr[2 % VEC], gr[3 % VEC]);
+            o.z = pack_bf16x2(gr[4 % VEC], gr[5 % VEC]); o.w = pack_bf16x2(gr[6 % VEC], gr[7 % VEC]);
+          } else {
+            o.x = __float_as_uint(gr[0]); o.y = __float_as_uint(gr[1]); o.z = __float_as_uint(gr[2]); o.w = __float_as_uint(gr[3]);
+          }
+          __stcs(reinterpret_cast<uint4*>(grow + e[j]), o);
+        } else {
+          for (int q = e[j]; q < V && q < e[j] + VEC; ++q) {  /* the ragged end of the row */
+            const float pr = exp2f(fmaf(to_f32(row[q]), kLog2e, nl));
+            store_grad(grow + q, w * ((q == tok ? 1.f : 0.f) - pr));
+          }
+        }
+      }
+    } else {
+      const int e1 = min(e0 + kUnitElems, V);
+      for (int q = e0 + (int)threadIdx.x; q < e1; q += kBwdNT) {
+        const float pr = exp2f(fmaf(to_f32(row[q]), kLog2e, nl));
+        store_grad(grow + q, w * ((q == tok ? 1.f : 0.f) - pr));
+      }
+    }
+  }
+}
+
+extern "C" fork_status fork_logprob_backward(const fork_logprob_bwd_args* a, void* ws, size_t ws_bytes, void* stream) {
+  if (!a) return FORK_ERR_INVALID_ARG;
+  if (bad_source(a->logits, a->stride_b, a->stride_l, a->pos0, a->B, a->Lt, a->Ll, a->V, a->dtype))
+    return FORK_ERR_INVALID_ARG;
+  if (!a->tokens || !a->select || !a->lse || !a->dlogp || !a->grad) return FORK_ERR_INVALID_ARG;
+  if (a->grad_stride_l < a->V || a->grad_stride_b < 0) return FORK_ERR_INVALID_ARG;
+  fork_status s = check_workspace(ws, ws_bytes, a->B, a->Lt);
+  if (s != FORK_OK) return s;
+  if (a->B == 0) return FORK_OK;
+  cudaStream_t st = (cudaStream_t)stream;
+  DeviceInfo* dev;
+  if (!device_info(&dev)) return FORK_ERR_CUDA;
+  WsView w = ws_view(ws, a->B, a->Lt);
+  SetupParams sp;
+  memset(&sp, 0, sizeof(sp));
+  sp.flags = a->select; sp.lo = nullptr; sp.hi = nullptr;
+  sp.B = a->B; sp.Lt = a->Lt; sp.pos0 = a->pos0; sp.Ll = a->Ll; sp.C = 1; sp.G = 1;
+  sp.hdr = w.hdr; sp.seq_off = w.seq_off; sp.expected = w.expected; sp.ticket = w.ticket; sp.rows = w.rows;
+  const bool pdl = g_tune[FORK_TUNE_PDL].load() >= 0;
+  if (launch(active_set_kernel, dim3(1), dim3(kSetupNT), st, pdl, sp) != cudaSuccess) return FORK_ERR_CUDA;
+  BwdParams bp;
+  memset(&bp, 0, sizeof(bp));
+  bp.src = RowSource{a->logits, (long long)a->stride_b, (long long)a->stride_l, a->pos0, a->Ll, a->V};
+  bp.grad = a->grad; bp.gstride_b = a->grad_stride_b; bp.gstride_l = a->grad_stride_l;
+  bp.hdr = w.hdr; bp.rows = w.rows; bp.tokens = a->tokens; bp.lse = a->lse; bp.dlogp = a->dlogp; bp.Lt = a->Lt;
+  bp.vector_ok = (source_is_vector_aligned(a->logits, a->stride_b, a->stride_l, a->dtype) &&
+                  source_is_vector_aligned(a->grad, a->grad_stride_b, a->grad_stride_l, a->dtype)) ? 1 : 0;
+  const int grid = dev->sms * 8;
+  cudaError_t e = a->dtype == FORK_BF16 ? launch(logprob_backward_kernel<bf16_t>, dim3(grid), dim3(kBwdNT), st, pdl, bp)
+                                        : launch(logprob_backward_kernel<float>, dim3(grid), dim3(kBwdNT), st, pdl, bp);
+  return e == cudaSuccess ? FORK_OK : FORK_ERR_CUDA;
 }
 
 /* ---- host-buffer entry point --------------------------------------------------------------- */

@@ -368,6 +368,127 @@ struct Acc<float, WITH_T, CLAMP> : AccCore<WITH_T> {
 
 __device__ __forceinline__ bool part_is_finite(const Part& p) { return isfinite(p.s) && isfinite(p.t); }
 
+/* ------------------------------------------------------------------------------------------ */
+/* Stochastic candidates (Algorithm 2 line 4 with tau > 0): x_0 ~ softmax(x / tau) drawn as
+ * arg-max_v (x_v / tau + g_v), g_v standard Gumbel noise (Gumbel-max).  The noise stream is a
+ * counter-based generator: a 64-bit key per (seed, step, sequence, position), a 32-bit hash per
+ * vocabulary entry, the uniform u = ((h >> 9) + 1/2) 2^-23, g = -ln E with E = -ln u.
+ * Keys are compared in log2 units with constants dropped:  key = x * (log2 e / tau) - log2 E.
+ * log2 E takes two special-function evaluations, except close to u = 1, where lg2.approx has only
+ * an absolute error bound and E = w + w^2/2 + ... (w = 1 - u, exact) is used instead:
+ *     log2 E = log2 w + w / (2 ln 2)            for w < 2^-8,
+ *     log2 E = log2(-log2 u) + log2(ln 2)       otherwise.                                       */
+struct NoiseRow {
+  uint32_t lo, hi;             /* the row's key */
+  float c;                     /* log2(e) / tau */
+};
+
+__device__ __forceinline__ uint64_t noise_mix64(uint64_t z) {
+  z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ull; z ^= z >> 27; z *= 0x94D049BB133111EBull; z ^= z >> 31;
+  return z;
+}
+__device__ __forceinline__ NoiseRow noise_row(uint64_t seed, int step, int b, int k, float c) {
+  uint64_t z = noise_mix64(seed + 0x9E3779B97F4A7C15ull * (uint64_t)((uint32_t)step + 1u));
+  z = noise_mix64(z ^ (((uint64_t)(uint32_t)b << 32) | (uint64_t)(uint32_t)k));
+  return NoiseRow{(uint32_t)z, (uint32_t)(z >> 32), c};
+}
+__device__ __forceinline__ float lg2_approx(float x) {
+  float y;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+/* perturbed key of logit x at vocabulary index v */
+__device__ __forceinline__ float noise_key(const NoiseRow& nz, float x, uint32_t v) {
+  uint32_t h = (v ^ nz.hi) * 0x9E3779B1u + nz.lo;
+  h ^= h >> 16; h *= 0x21F0AAADu; h ^= h >> 15; h *= 0x735A2D97u; h ^= h >> 15;
+  const float f = __uint_as_float((h >> 9) | 0x3f800000u);   /* 1 + n 2^-23 */
+  const float u = f - 0.99999994f;                           /* (2n+1) 2^-24, exact */
+  const float w = 1.0f - u;                                  /* (2^24 - 2n - 1) 2^-24, exact */
+  const bool near_one = w < 0.00390625f;
+  const float l1 = lg2_approx(u);
+  const float l2 = lg2_approx(near_one ? w : -l1);
+  const float corr = near_one ? w * 0.72134752f : -0.52876637f;
+  return __fmaf_rn(x, nz.c, -(l2 + corr));
+}
+
+/* The largest perturbed key a thread / warp / CTA / row has seen, and where: `vec` is the start of
+   the 128-bit vector holding it (or the exact index for elements handled one at a time); equal keys
+   go to the lower position.  resolve_sample() recomputes the keys of that vector to find the
+   element. */
+struct KeyPart {
+  float key; int vec;
+};
+__device__ __forceinline__ KeyPart key_empty() { return KeyPart{-INFINITY, kIdxNone}; }
+__device__ __forceinline__ KeyPart key_merge(const KeyPart& a, const KeyPart& b) {
+  const bool bwins = (b.key > a.key) || (b.key == a.key && b.vec < a.vec);
+  return bwins ? b : a;
+}
+__device__ __forceinline__ KeyPart key_warp_reduce(KeyPart p) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    KeyPart q;
+    q.key = __shfl_xor_sync(0xffffffffu, p.key, o);
+    q.vec = __shfl_xor_sync(0xffffffffu, p.vec, o);
+    p = key_merge(p, q);
+  }
+  return p;
+}
+
+struct KeyTrack {
+  KeyPart best;
+  __device__ __forceinline__ void init() { best = key_empty(); }
+  /* N vectors; vector j starts at vocabulary index base + j*stride (ascending within a thread, so a
+     strict comparison keeps the lowest position among equal keys) */
+  template <int N>
+  __device__ __forceinline__ void update(bf16_t, const NoiseRow& nz, const uint4 (&v)[N], int base, int stride) {
+#pragma unroll
+    for (int j = 0; j < N; ++j) {
+      const uint32_t e = (uint32_t)(base + j * stride);
+      float k0 = noise_key(nz, bf16_lo(v[j].x), e), k1 = noise_key(nz, bf16_hi(v[j].x), e + 1);
+      float k2 = noise_key(nz, bf16_lo(v[j].y), e + 2), k3 = noise_key(nz, bf16_hi(v[j].y), e + 3);
+      float k4 = noise_key(nz, bf16_lo(v[j].z), e + 4), k5 = noise_key(nz, bf16_hi(v[j].z), e + 5);
+      float k6 = noise_key(nz, bf16_lo(v[j].w), e + 6), k7 = noise_key(nz, bf16_hi(v[j].w), e + 7);
+      const float vm = fmaxf(fmaxf(fmaxf(k0, k1), fmaxf(k2, k3)), fmaxf(fmaxf(k4, k5), fmaxf(k6, k7)));
+      if (vm > best.key) { best.key = vm; best.vec = (int)e; }
+    }
+  }
+  template <int N>
+  __device__ __forceinline__ void update(float, const NoiseRow& nz, const uint4 (&v)[N], int base, int stride) {
+#pragma unroll
+    for (int j = 0; j < N; ++j) {
+      const uint32_t e = (uint32_t)(base + j * stride);
+      float k0 = noise_key(nz, __uint_as_float(v[j].x), e), k1 = noise_key(nz, __uint_as_float(v[j].y), e + 1);
+      float k2 = noise_key(nz, __uint_as_float(v[j].z), e + 2), k3 = noise_key(nz, __uint_as_float(v[j].w), e + 3);
+      const float vm = fmaxf(fmaxf(k0, k1), fmaxf(k2, k3));
+      if (vm > best.key) { best.key = vm; best.vec = (int)e; }
+    }
+  }
+  /* one element at its exact index */
+  __device__ __forceinline__ void one(const NoiseRow& nz, float x, int idx) {
+    const float k = noise_key(nz, x, (uint32_t)idx);
+    if (k > best.key || (k == best.key && idx < best.vec)) { best.key = k; best.vec = idx; }
+  }
+};
+
+/* The element that holds the row's largest perturbed key: the first of the (up to) one vector's
+   worth of elements from `vec` on whose recomputed key equals `key`; also returns its logit. */
+template <typename T>
+__device__ __forceinline__ int resolve_sample(const T* row, const NoiseRow& nz, int vec, int V, float key, float& x_out) {
+  constexpr int VEC = 16 / (int)sizeof(T);
+  int best = -1;
+  x_out = 0.f;
+  if (vec < 0 || vec >= V) return 0;
+#pragma unroll
+  for (int j = VEC - 1; j >= 0; --j) {
+    if (vec + j < V) {
+      const float x = to_f32(row[vec + j]);
+      if (noise_key(nz, x, (uint32_t)(vec + j)) == key) { best = vec + j; x_out = x; }
+    }
+  }
+  if (best < 0) { best = vec; x_out = to_f32(row[vec]); }
+  return best;
+}
+
 /* The exact position of the row maximum M, given the start `idx` of the vector that holds its
    first occurrence (or the exact position): look at one vector's worth of elements.  All loads are
    issued before any comparison (one 128-bit load when the window is aligned), because this sits
@@ -399,9 +520,11 @@ __device__ __forceinline__ int resolve_index(const T* row, int idx, int V, float
 /* One thread's share of elements [e0,e1) of a row, read with 128-bit loads straight from global
    memory: vectors tid, tid+NT, tid+2NT, ... (ascending indices), in groups of UNROLL; the thread
    with `tail` also takes the fewer-than-a-vector trailing elements.  e0 is a multiple of the vector
-   width and the row base is 16-byte aligned. */
-template <typename T, bool WITH_T, bool CLAMP, int NT, int UNROLL>
-__device__ __forceinline__ Part stream_thread_once(const T* row, int e0, int e1, int tid, bool tail) {
+   width and the row base is 16-byte aligned.  With SAMPLE the perturbed keys of the same elements
+   go through `kt`. */
+template <typename T, bool WITH_T, bool CLAMP, int NT, int UNROLL, bool SAMPLE>
+__device__ __forceinline__ Part stream_thread_once(const T* row, int e0, int e1, int tid, bool tail, KeyTrack* kt,
+                                                   const NoiseRow* nz) {
   Acc<T, WITH_T, CLAMP> a;
   a.init();
   constexpr int VEC = 16 / (int)sizeof(T);
@@ -412,15 +535,21 @@ __device__ __forceinline__ Part stream_thread_once(const T* row, int e0, int e1,
     uint4 v[UNROLL];
 #pragma unroll
     for (int j = 0; j < UNROLL; ++j) v[j] = ld_stream(p + i + j * NT);
+    if (SAMPLE) kt->template update<UNROLL>(T{}, *nz, v, e0 + i * VEC, NT * VEC);
     a.template group<UNROLL>(v, e0 + i * VEC, NT * VEC);
   }
   for (; i < nvec; i += NT) {
     uint4 v[1];
     v[0] = ld_stream(p + i);
+    if (SAMPLE) kt->template update<1>(T{}, *nz, v, e0 + i * VEC, NT * VEC);
     a.template group<1>(v, e0 + i * VEC, NT * VEC);
   }
   if (tail) {
-    for (int e = e0 + nvec * VEC; e < e1; ++e) a.one(to_f32(row[e]), e);
+    for (int e = e0 + nvec * VEC; e < e1; ++e) {
+      const float x = to_f32(row[e]);
+      if (SAMPLE) kt->one(*nz, x, e);
+      a.one(x, e);
+    }
   }
   return a.part();
 }
@@ -429,16 +558,35 @@ __device__ __forceinline__ Part stream_thread_once(const T* row, int e0, int e1,
    (it met a -inf logit, or the row really holds NaN / +inf and will be flagged by the finaliser). */
 template <typename T, bool WITH_T, int NT>
 __device__ __noinline__ Part stream_thread_clamped(const T* row, int e0, int e1, int tid, bool tail) {
-  return stream_thread_once<T, WITH_T, true, NT, 1>(row, e0, e1, tid, tail);
+  return stream_thread_once<T, WITH_T, true, NT, 1, false>(row, e0, e1, tid, tail, nullptr, nullptr);
+}
+
+/* The perturbed keys of one thread's share, on their own (for a thread that starts clamped). */
+template <typename T, int NT>
+__device__ __noinline__ void stream_thread_keys(const T* row, int e0, int e1, int tid, bool tail, KeyTrack* kt,
+                                                const NoiseRow* nz) {
+  constexpr int VEC = 16 / (int)sizeof(T);
+  const uint4* p = reinterpret_cast<const uint4*>(row + e0);
+  const int nvec = (e1 - e0) / VEC;
+  for (int i = tid; i < nvec; i += NT) {
+    uint4 v[1];
+    v[0] = ld_stream(p + i);
+    kt->template update<1>(T{}, *nz, v, e0 + i * VEC, NT * VEC);
+  }
+  if (tail)
+    for (int e = e0 + nvec * VEC; e < e1; ++e) kt->one(*nz, to_f32(row[e]), e);
 }
 
 /* `sticky` remembers that this thread has met a -inf before and starts clamped from then on. */
-template <typename T, bool WITH_T, int NT, int UNROLL>
-__device__ __forceinline__ Part stream_thread(const T* row, int e0, int e1, int tid, bool tail, bool& sticky) {
+template <typename T, bool WITH_T, int NT, int UNROLL, bool SAMPLE>
+__device__ __forceinline__ Part stream_thread(const T* row, int e0, int e1, int tid, bool tail, bool& sticky,
+                                              KeyTrack* kt, const NoiseRow* nz) {
   if (!sticky) {
-    const Part pt = stream_thread_once<T, WITH_T, false, NT, UNROLL>(row, e0, e1, tid, tail);
+    const Part pt = stream_thread_once<T, WITH_T, false, NT, UNROLL, SAMPLE>(row, e0, e1, tid, tail, kt, nz);
     if (part_is_finite(pt)) return pt;
     sticky = true;
+  } else if (SAMPLE) {
+    stream_thread_keys<T, NT>(row, e0, e1, tid, tail, kt, nz);
   }
   return stream_thread_clamped<T, WITH_T, NT>(row, e0, e1, tid, tail);
 }
@@ -464,6 +612,19 @@ __device__ __forceinline__ float block_sum_f32(float v, float* sh /*[NT/32]*/) {
   __syncthreads();
   r = sh[0];
   return r;                                                /* same value in every thread */
+}
+
+/* Largest key over the CTA; valid in thread 0.  `sh` holds NT/32 entries. */
+template <int NT>
+__device__ __forceinline__ KeyPart key_block_reduce(KeyPart k, KeyPart* sh) {
+  constexpr int NW = NT / 32;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  k = key_warp_reduce(k);
+  __syncthreads();
+  if (lane == 0) sh[warp] = k;
+  __syncthreads();
+  if (warp == 0) k = key_warp_reduce((lane < NW) ? sh[lane] : key_empty());
+  return k;
 }
 
 /* Guarded scalar reduction of elements [e0,e1) of one row by the whole CTA: two passes, every
@@ -529,6 +690,20 @@ __device__ __forceinline__ RowOut row_out_from(const Part& p, bool bad) {
   o.conf = 1.0f / p.s;
   o.entropy = fmaxf(lns - (p.t * kLn2) / p.s, 0.f);
   o.logp = -lns;
+  o.status = 0u;
+  return o;
+}
+
+/* The same with a drawn candidate whose logit is xs: its probability under the untempered softmax
+   is the confidence (Algorithm 2 line 5 has no temperature), p.idx is the drawn token. */
+__device__ __forceinline__ RowOut row_out_sampled(const Part& p, bool bad, float xs) {
+  if (bad) return row_out_from(p, true);
+  RowOut o;
+  o.cand = (p.idx == kIdxNone) ? 0 : p.idx;
+  const float lns = logf(p.s), d = xs - p.m;
+  o.conf = exp2f(d * kLog2e) / p.s;
+  o.entropy = fmaxf(lns - (p.t * kLn2) / p.s, 0.f);
+  o.logp = d - lns;
   o.status = 0u;
   return o;
 }

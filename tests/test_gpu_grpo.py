@@ -1,0 +1,147 @@
+"""ForkGRPO objective (Eq. 2) and the log-softmax backward on the GPU against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import fork_synth as fs
+import oracle
+from helpers import assert_close, to_torch_logits
+from test_gpu_step import make_rows
+
+pytestmark = pytest.mark.gpu
+
+
+def F():
+    import paper_2609_39859_b200 as pkg
+    return pkg
+
+
+def close(name, got, want, rtol, atol):
+    got = np.asarray(got, np.float64)
+    want = np.asarray(want, np.float64)
+    ok = (np.isnan(got) & np.isnan(want)) | (np.abs(got - want) <= atol + rtol * np.abs(want))
+    assert ok.all(), "%s: %d outside tolerance, e.g. got %s want %s" % (
+        name, (~ok).sum(), got.ravel()[np.flatnonzero(~ok.ravel())[:4]], want.ravel()[np.flatnonzero(~ok.ravel())[:4]])
+
+
+@pytest.mark.parametrize("B,Lt,G", [(32, 64, 8), (128, 256, 8), (6, 5, 3), (16, 33, 16)])
+def test_grpo_loss_matches_the_oracle(B, Lt, G):
+    pkg = F()
+    eps_lo, eps_hi = 0.2, 0.28
+    for seed in range(6):
+        rng = np.random.default_rng(seed * 31 + B)
+        old = rng.normal(-1.5, 0.7, (B, Lt)).astype(np.float32)
+        new = (old + rng.normal(0, 0.2, (B, Lt))).astype(np.float32)
+        sel = (rng.random((B, Lt)) < 0.2).astype(np.uint8)
+        sel[1] = 0                                             # a rollout without fallback steps
+        reward = (rng.random(B) < 0.5).astype(np.float32)
+        reward[:G] = 1.0                                       # a group with equal rewards: skipped
+        o = oracle.grpo_loss(new, old, sel, reward, G, eps_lo, eps_hi)
+        rho = o["ratio"][sel != 0]
+        if (np.abs(rho - (1 - np.float32(eps_lo))) < 1e-4).any() or (np.abs(rho - (1 + np.float32(eps_hi))) < 1e-4).any():
+            continue                                           # a ratio on a clip boundary: fp32 may pick the other branch
+        g = pkg.fork_grpo_loss(*(torch.from_numpy(x).cuda() for x in (new, old, sel, reward)), G, eps_lo, eps_hi)
+        torch.cuda.synchronize()
+        h = {k: v.cpu().numpy() for k, v in g.items()}
+        assert np.array_equal(h["skipped"][: B // G], o["skipped"][: B // G]) and o["skipped"][0] == 1
+        close("adv", h["adv"], o["adv"], 1e-5, 1e-6)
+        close("ratio", h["ratio"], o["ratio"], 1e-5, 1e-7)
+        close("seq_obj", h["seq_obj"], o["seq_obj"], 1e-4, 1e-6)
+        close("objective", h["objective"][0], o["objective"], 1e-4, 1e-6)
+        close("dlogp", h["dlogp"], o["dlogp"], 1e-4, 1e-9)
+        assert (h["dlogp"][sel == 0] == 0).all() and (h["dlogp"][:G] == 0).all()
+        return
+    raise AssertionError("no input away from the clip boundaries")
+
+
+def test_grpo_loss_rejects_bad_arguments():
+    pkg = F()
+    z = torch.zeros((4, 8), dtype=torch.float32, device="cuda")
+    sel = torch.zeros((4, 8), dtype=torch.uint8, device="cuda")
+    r = torch.zeros(4, dtype=torch.float32, device="cuda")
+    for group, lo, hi in ((3, 0.2, 0.2), (0, 0.2, 0.2), (2, -0.1, 0.2), (2, 0.2, float("nan"))):
+        with pytest.raises(pkg.ForkError) as e:
+            pkg.fork_grpo_loss(z, z, sel, r, group, lo, hi)
+        assert e.value.status == pkg.FORK_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("V", [5, 8, 1000, 4096, 5003, 40000])
+def test_logprob_backward_matches_the_oracle(V, dtype):
+    """Score, then differentiate: rows of selected positions hold dlogp * (onehot - softmax), every
+    other row keeps its canary.  Unaligned V takes the scalar path, the rest the 128-bit path with
+    a ragged end."""
+    pkg = F()
+    rng = np.random.default_rng(V + (dtype == "f32"))
+    B, Lt = 3, 12
+    x = make_rows(rng, (B, Lt), V, dtype, peak=5.0)
+    if V > 100:
+        xf = x if dtype == "f32" else None
+        if xf is not None:
+            xf[0, 1, 10:50] = -np.inf                          # banned tokens get no probability
+    tokens = rng.integers(0, V, (B, Lt)).astype(np.int32)
+    sel = (rng.random((B, Lt)) < 0.5).astype(np.uint8)
+    sel[0, 1] = 1
+    tokens[2, 3] = V + 5                                       # out of range: flagged when scored, no gradient
+    sel[2, 3] = 1
+    dlogp = rng.normal(0, 0.01, (B, Lt)).astype(np.float32)
+    st = pkg.ForkState(B, Lt)
+    xt = to_torch_logits(x)
+    tok_d, sel_d = torch.from_numpy(tokens).cuda(), torch.from_numpy(sel).cuda()
+    lp, ssum, scnt, status, lse = pkg.fork_logprob(xt, tok_d, sel_d, st, want_lse=True)
+    grad = torch.full_like(xt, 7.0)
+    pkg.fork_logprob_backward(xt, tok_d, sel_d, lse, torch.from_numpy(dlogp).cuda(), grad, st)
+    torch.cuda.synchronize()
+    g = grad.float().cpu().numpy()
+    lse_h = lse.cpu().numpy()
+    for b in range(B):
+        for k in range(Lt):
+            if not sel[b, k] or tokens[b, k] >= V:
+                assert (g[b, k] == 7.0).all(), (b, k)
+                continue
+            assert abs(lse_h[b, k] - oracle.row_lse(x[b, k])) <= 1e-5 + 1e-5 * abs(lse_h[b, k])
+            want = oracle.row_logp_grad(x[b, k], int(tokens[b, k]), float(dlogp[b, k]))
+            w = abs(float(dlogp[b, k]))
+            if dtype == "f32":
+                close("grad", g[b, k], want, 1e-4, 2e-6 * w)
+            else:
+                close("grad", g[b, k], want, 2.0 ** -8, 2e-6 * w)
+            assert abs(g[b, k].sum()) <= (1e-4 if dtype == "f32" else 2e-2) * w * max(1.0, np.abs(want).sum() / w)
+
+
+def test_scoring_loss_backward_chain_at_the_training_shape_of_a_few_rows():
+    """V = 126464 fp32 rows through fork_logprob -> fork_grpo_loss -> fork_logprob_backward."""
+    pkg = F()
+    w = fs.workload("grpo")
+    B, Lt, V, G = 8, 4, w.V, 4
+    cfg = w.cfg(B=B)
+    x = np.empty((B, Lt, V), np.float32)
+    for b in range(B):
+        for l in range(Lt):
+            x[b, l] = fs.row_host(cfg, 0, b, l)
+    rng = np.random.default_rng(0)
+    tokens = x.argmax(-1).astype(np.int32)
+    tokens[:, 1] = rng.integers(0, V, B)
+    sel = np.ones((B, Lt), np.uint8)
+    sel[:, 3] = 0
+    reward = rng.random(B).astype(np.float32)
+    st = pkg.ForkState(B, Lt)
+    xt = torch.from_numpy(x).cuda()
+    tok_d, sel_d = torch.from_numpy(tokens).cuda(), torch.from_numpy(sel).cuda()
+    lp, ssum, scnt, status, lse = pkg.fork_logprob(xt, tok_d, sel_d, st, want_lse=True)
+    old = (lp + 0.05 * torch.randn_like(lp)) * (sel_d != 0)
+    out = pkg.fork_grpo_loss(lp, old.contiguous(), sel_d, torch.from_numpy(reward).cuda(), G, 0.2, 0.2)
+    grad = torch.zeros_like(xt)
+    pkg.fork_logprob_backward(xt, tok_d, sel_d, lse, out["dlogp"], grad, st)
+    torch.cuda.synchronize()
+    rc, olp, osum, ocnt, _ = oracle.logprob(x, tokens, sel)
+    assert_close("logp", lp.cpu().numpy(), olp)
+    o = oracle.grpo_loss(lp.cpu().numpy(), old.cpu().numpy(), sel, reward, G, 0.2, 0.2)
+    close("objective", out["objective"].cpu().numpy()[0], o["objective"], 1e-4, 1e-6)
+    close("dlogp", out["dlogp"].cpu().numpy(), o["dlogp"], 1e-4, 1e-9)
+    g = grad.cpu().numpy()
+    d = out["dlogp"].cpu().numpy()
+    for b, k in ((0, 0), (3, 1), (7, 2)):
+        want = oracle.row_logp_grad(x[b, k], int(tokens[b, k]), float(d[b, k]))
+        close("grad", g[b, k], want, 1e-4, 2e-6 * abs(float(d[b, k])))
+    assert (g[:, 3] == 0).all()

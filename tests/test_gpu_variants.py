@@ -182,3 +182,136 @@ def test_top_entropy_selection_feeds_the_scoring_pass():
     assert_close("logp", lp.cpu().numpy(), olp)
     assert_close("seq_sum", ssum.cpu().numpy(), osum)
     assert np.array_equal(scnt.cpu().numpy(), ocnt2)
+
+
+# ---- stochastic candidates (temperature > 0) -----------------------------------------------------
+def sample_both(x, mask, lo, hi, lam, tau, seed, step=3, pos0=0, logits_t=None):
+    """One step with drawn candidates on both sides; None for the GPU side when some decision of
+    the oracle (threshold, winning perturbed key) has no clear margin."""
+    pkg = F()
+    B, Ll, V = x.shape
+    Lt = mask.shape[1]
+    o = oracle.StepState(B, Lt, mask=mask)
+    assert oracle.step(o, x, lo, hi, lam, step_id=step, pos0=pos0, temperature=tau, sample_seed=seed) == 0
+    if not decisions_are_clear(o, live_mask(mask, lo, hi), lam, 1e-4, 0, tau):
+        return None, o
+    g = pkg.ForkState(B, Lt, mask=mask)
+    keep = [torch.from_numpy(np.asarray(a)).cuda() for a in (lo, hi)]
+    lg = to_torch_logits(x) if logits_t is None else logits_t
+    pkg.fork_step(g, lg, keep[0], keep[1], lam, step=step, pos0=pos0, temperature=tau, sample_seed=seed)
+    torch.cuda.synchronize()
+    return g.host(), o
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("V", [2, 7, 8, 1023, 1024, 2049, 4104, 6151, 40000])
+def test_sampled_step_small_vocabularies(V, dtype):
+    """Aligned V takes the bulk-copy ring, unaligned V the scalar path; several chunks, ragged tails."""
+    done = 0
+    for seed in range(20):
+        rng = np.random.default_rng(V * 7 + seed)
+        B, Lt = 4, 24
+        mask = (rng.random((B, Lt)) < 0.7).astype(np.uint8)
+        lo = rng.integers(0, 10, size=B).astype(np.int32)
+        hi = (lo + rng.integers(0, 14, size=B)).astype(np.int32)
+        x = make_rows(rng, (B, Lt), V, dtype, peak=6.0)
+        g, o = sample_both(x, mask, lo, hi, 0.9 if V > 8 else 0.45, tau=[0.8, 1.3][seed % 2], seed=1000 + seed)
+        if g is None:
+            continue
+        compare_step_state(g, o)
+        done += 1
+        if done == 3:
+            return
+    raise AssertionError("too few inputs with clear margins")
+
+
+def test_sampled_step_full_vocabulary_rows_span_many_ctas():
+    """V = 126464 bf16: every row is cut into parts over several CTAs; the drawn token must come out
+    of the merge of their best keys."""
+    w = fs.workload("b8")
+    B, Lt, V = 2, 8, w.V
+    cfg = w.cfg(B=B)
+    mask = np.ones((B, Lt), np.uint8)
+    lo, hi = np.zeros(B, np.int32), np.full(B, Lt, np.int32)
+    for nonce in range(8):
+        x = np.empty((B, Lt, V), np.uint16)
+        for b in range(B):
+            for l in range(Lt):
+                x[b, l] = fs.row_host(cfg, 0, b, l, nonce=nonce)
+        g, o = sample_both(x, mask, lo, hi, w.threshold, tau=0.8, seed=77)
+        if g is None:
+            continue
+        compare_step_state(g, o)
+        return
+    raise AssertionError("no input with clear margins found")
+
+
+def test_sampled_step_with_banned_token_ranges():
+    """-inf logits (banned tokens) can never be drawn; threads that meet them take their clamped path."""
+    for seed in range(10):
+        rng = np.random.default_rng(50 + seed)
+        B, Lt, V = 2, 6, 8200
+        mask = np.ones((B, Lt), np.uint8)
+        lo, hi = np.zeros(B, np.int32), np.full(B, Lt, np.int32)
+        x = make_rows(rng, (B, Lt), V, "f32", peak=3.0)
+        x[:, :, 100:3000] = -np.inf
+        x[0, 2, :] = -np.inf
+        x[0, 2, 4097] = 1.0                                     # a single allowed token
+        g, o = sample_both(x, mask, lo, hi, 0.9, tau=1.5, seed=seed)
+        if g is None:
+            continue
+        compare_step_state(g, o)
+        assert g["cand"][0, 2] == 4097 and not ((g["cand"] >= 100) & (g["cand"] < 3000)).any()
+        return
+    raise AssertionError("no input with clear margins found")
+
+
+@pytest.mark.parametrize("V,dtype", [(6, "f32"), (8, "f32"), (16, "bf16")])
+def test_sampled_candidates_follow_tempered_softmax_on_the_gpu(V, dtype):
+    """Distribution pin of the CUDA sampler on its own: frequencies against scipy's softmax(x/tau)."""
+    from scipy.special import softmax
+    pkg = F()
+    rng = np.random.default_rng(V)
+    xrow = rng.normal(0, 1.5, V).astype(np.float32)
+    if dtype == "bf16":
+        xrow = fs.bf16_bits_to_f32(fs.f32_to_bf16_bits(xrow))
+    B, Lt, tau = 64, 128, 0.9
+    x = np.ascontiguousarray(np.broadcast_to(xrow, (B, Lt, V))).copy()
+    xt = to_torch_logits(x if dtype == "f32" else fs.f32_to_bf16_bits(x))
+    lo = torch.zeros(B, dtype=torch.int32, device="cuda")
+    hi = torch.full((B,), Lt, dtype=torch.int32, device="cuda")
+    counts = np.zeros(V)
+    for step in range(3):
+        st = pkg.ForkState(B, Lt)
+        pkg.fork_step(st, xt, lo, hi, -1.0, step=step, temperature=tau, sample_seed=4242)
+        torch.cuda.synchronize()
+        h = st.host()
+        assert (h["mask"] == 0).all()
+        counts += np.bincount(h["tokens"].ravel(), minlength=V)
+        p_plain = softmax(xrow.astype(np.float64))
+        assert np.allclose(h["conf"], p_plain[h["tokens"]], rtol=1e-4, atol=1e-6)
+    n = counts.sum()
+    expect = softmax(xrow.astype(np.float64) / tau) * n
+    chi2 = float(((counts - expect) ** 2 / expect).sum())
+    assert chi2 < 3.0 * V + 25.0, (chi2, counts, expect)
+
+
+def test_tiny_decode_loop_with_sampled_candidates():
+    w = fs.workload("tiny")
+    B, tau, seed = 4, 0.8, 2024
+    ost, nonces, osteps, _ = oracle_reference_loop(w, B, w.threshold, temperature=tau, sample_seed=seed)
+    pkg = F()
+    cfg = w.cfg(B=B)
+    logits = torch.empty((B, w.Lt, w.V), dtype=torch.float32, device="cuda")
+    st = pkg.ForkState(B, w.Lt)
+    prov = fs.Provider(cfg, w.Lt * w.V, w.V, 0, w.Lt, nonce=nonces)
+    rc, steps = pkg.fork_decode_loop(st, logits, w.block_len, 0, w.Lt, prov.address, prov.ctx, w.threshold, 10000,
+                                     temperature=tau, sample_seed=seed)
+    torch.cuda.synchronize()
+    prov.close()
+    assert rc == 0 and steps == osteps
+    h = st.host()
+    compare_step_state(h, ost)
+    assert (h["tokens"] == h["cand"]).all()
+    greedy, _, _, _ = oracle_reference_loop(w, B, w.threshold)
+    assert (greedy.tokens != ost.tokens).any()                 # the draws are not the arg-max everywhere
