@@ -159,7 +159,7 @@ def reset_states(states):
     states[0].pool_mask[:len(states)].fill_(1)
 
 
-def time_full_block(w, seed, steps, warmup, device, use_graph=True):
+def time_full_block(w, seed, steps, warmup, device, use_graph=True, variant=None):
     """Times `steps` fork_step calls (after `warmup`), each on B*block_len live rows.  The timed
     steps are replayed from one CUDA graph when `use_graph` (host launch cost would otherwise bound
     a ~10 us step); a second, un-graphed pass brackets each step's streaming kernel with events."""
@@ -177,7 +177,7 @@ def time_full_block(w, seed, steps, warmup, device, use_graph=True):
         s, b = i % n_state, i % n_buf
         a = cache.get((s, b))
         if a is None:
-            a = cache[(s, b)] = pkg.make_step_args(states[s], bufs[b], lo, hi, w.threshold, step=0)
+            a = cache[(s, b)] = pkg.make_step_args(states[s], bufs[b], lo, hi, w.threshold, step=0, **(variant or {}))
         rc = L.fork_step(C.byref(a), C.c_void_p(states[s].ws_ptr), states[s].ws_bytes, sp)
         if rc != 0:
             raise RuntimeError("fork_step: " + pkg.fork_status_string(rc))
@@ -324,10 +324,57 @@ def time_logprob(device, peak):
     ms = e0.elapsed_time(e1) / n
     rows = int(select.sum())
     gbs = rows * w.V * 4 / (ms * 1e-3) / 1e9
-    del t
+    out = [{"workload": "grpo: fork_logprob B=128 Lt=256 V=126464 f32, %d selected rows (3.3 GB >> L2)" % rows,
+            "positions_per_s": rows / (ms * 1e-3), "ms": ms, "hbm_gbs": gbs, "frac_of_measured_peak": gbs / peak}]
+    # the training half of the same shape: objective (Eq. 2) and the log-softmax backward at the selected rows
+    lp, ssum, scnt, status, lse = pkg.fork_logprob(t, tok_d, sel_d, st, want_lse=True)
+    old = (lp + 0.05 * torch.randn_like(lp)) * (sel_d != 0)
+    reward = (torch.rand(w.B, device=device) < 0.5).float()
+    for _ in range(3):
+        loss = pkg.fork_grpo_loss(lp, old, sel_d, reward, 8, 0.2, 0.2)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(20):
+        loss = pkg.fork_grpo_loss(lp, old, sel_d, reward, 8, 0.2, 0.2)
+    e1.record()
+    torch.cuda.synchronize()
+    out.append({"workload": "grpo: fork_grpo_loss B=128 (16 groups of 8) Lt=256", "ms": e0.elapsed_time(e1) / 20,
+                "kernels_per_call": 2})
+    grad = torch.empty_like(t)
+    for _ in range(2):
+        pkg.fork_logprob_backward(t, tok_d, sel_d, lse, loss["dlogp"], grad, st)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(n):
+        pkg.fork_logprob_backward(t, tok_d, sel_d, lse, loss["dlogp"], grad, st)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / n
+    gbs = 2 * rows * w.V * 4 / (ms * 1e-3) / 1e9
+    out.append({"workload": "grpo: fork_logprob_backward, same %d rows: one read + one write of each row (6.6 GB)" % rows,
+                "positions_per_s": rows / (ms * 1e-3), "ms": ms, "hbm_gbs_read_plus_write": gbs,
+                "frac_of_measured_peak": gbs / peak})
+    del t, grad
     torch.cuda.empty_cache()
-    return {"workload": "grpo: fork_logprob B=128 Lt=256 V=126464 f32, %d selected rows (3.3 GB >> L2)" % rows,
-            "positions_per_s": rows / (ms * 1e-3), "ms": ms, "hbm_gbs": gbs, "frac_of_measured_peak": gbs / peak}
+    return out
+
+
+def time_select(device):
+    """JustGRPO-Fast's top-entropy selection at the scoring shape."""
+    import torch
+    import paper_2609_39859_b200 as pkg
+    B, Lt = 128, 256
+    ent = torch.rand((B, Lt), device=device) * 5
+    elig = torch.ones((B, Lt), dtype=torch.uint8, device=device)
+    for _ in range(3):
+        pkg.fork_select_top_entropy(ent, elig, 0.2)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(20):
+        pkg.fork_select_top_entropy(ent, elig, 0.2)
+    e1.record()
+    torch.cuda.synchronize()
+    return {"workload": "fork_select_top_entropy B=128 Lt=256 ratio 0.2", "ms": e0.elapsed_time(e1) / 20}
 
 
 def loop_stats(device):
@@ -452,6 +499,8 @@ def main():
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--pdl", type=int, default=0, help="0 = programmatic dependent launch (default), -1 = off")
+    ap.add_argument("--temperature", type=float, default=0.0,
+                    help="time the step with stochastic candidates at this temperature (default 0: arg-max candidates)")
     args = ap.parse_args()
     if args.impl == "reference":
         return reference_arm(args)
@@ -481,7 +530,8 @@ def main():
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
-    r = time_full_block(w, seed, steps, warmup, device, use_graph=args.graph and not args.no_graph)
+    variant = dict(temperature=args.temperature, sample_seed=12345) if args.temperature > 0 else None
+    r = time_full_block(w, seed, steps, warmup, device, use_graph=args.graph and not args.no_graph, variant=variant)
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
@@ -507,7 +557,9 @@ def main():
         "dtype": "f32", "data": "synthetic",
         "config": dict(workload_config(w, rows),
                        l2="inputs rotate over %d logits buffers (%.0f MB in total, > 2x the 126 MB L2)" %
-                          (r["n_buf"], r["n_buf"] * rows * row_bytes / 1e6)),
+                          (r["n_buf"], r["n_buf"] * rows * row_bytes / 1e6),
+                       **({"candidates": "drawn at temperature %g (Gumbel-max in the same pass)" % args.temperature}
+                          if args.temperature > 0 else {})),
         "launch": ("one CUDA graph of the K steps" if r["graph"] else "plain stream launches, programmatic dependent launch"),
         "host_submit_ms_per_step": r["host_submit_ms"] / steps,
         "hbm_gbs_per_gpu": step_gbs, "frac_of_8TBs_nominal": step_gbs / NOMINAL_HBM_GBS,
@@ -531,22 +583,30 @@ def main():
     torch.cuda.empty_cache()
     if rank == 0 and not args.no_extras and world == 1:
         also = []
-        for name in ("b8", "passk", "sweep"):
-            if name == args.workload:
-                continue
-            w2 = fs.workload(name)
-            r2 = time_full_block(w2, w2.seed, min(steps, 50), 5, device)
+
+        def shape_line(w2, variant=None, label=""):
+            r2 = time_full_block(w2, w2.seed, min(steps, 50), 5, device, use_graph=False, variant=variant)
             r2.pop("setup", None)
             r2.pop("keep", None)
             torch.cuda.empty_cache()
             g2 = r2["rows"] * r2["row_bytes"] / (min(r2["kernel_ms"], r2["ms_per_step"]) * 1e-3) / 1e9
             s2 = r2["rows"] * r2["row_bytes"] / (r2["ms_per_step"] * 1e-3) / 1e9
-            also.append({"workload": workload_config(w2, r2["rows"])["workload"],
-                         "positions_per_s": r2["rows"] / (r2["ms_per_step"] * 1e-3), "ms_per_step": r2["ms_per_step"],
-                         "whole_step_gbs": s2, "whole_step_frac_of_measured_peak": s2 / peak,
-                         "kernel_gbs": g2, "kernel_frac_of_measured_peak": g2 / peak,
-                         "kernel_frac_of_8TBs_nominal": g2 / NOMINAL_HBM_GBS})
-        also.append(time_logprob(device, peak))
+            return {"workload": workload_config(w2, r2["rows"])["workload"] + label,
+                    "positions_per_s": r2["rows"] / (r2["ms_per_step"] * 1e-3), "ms_per_step": r2["ms_per_step"],
+                    "whole_step_gbs": s2, "whole_step_frac_of_measured_peak": s2 / peak,
+                    "kernel_gbs": g2, "kernel_frac_of_measured_peak": g2 / peak,
+                    "kernel_frac_of_8TBs_nominal": g2 / NOMINAL_HBM_GBS,
+                    "logits_per_s": r2["rows"] * w2.V / (min(r2["kernel_ms"], r2["ms_per_step"]) * 1e-3)}
+
+        for name in ("b8", "passk", "sweep"):
+            if name != args.workload:
+                also.append(shape_line(fs.workload(name)))
+        # the paper's rollout setting: candidates drawn at temperature 0.8 inside the same pass (ALU-bound)
+        for name in ("b8", "passk"):
+            also.append(shape_line(fs.workload(name), dict(temperature=0.8, sample_seed=12345),
+                                   " -- stochastic candidates, tau=0.8"))
+        also.extend(time_logprob(device, peak))
+        also.append(time_select(device))
         out["also"] = also
         out["cpu_baseline"] = cpu_baseline(w, seed)
         if args.loops:

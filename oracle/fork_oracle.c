@@ -92,7 +92,7 @@ typedef struct {
 
 /* ---- the noise stream of stochastic candidates -------------------------------------------------
  * One 64-bit key per (seed, step, b, k); one 32-bit hash per vocabulary entry; a uniform on the
- * 2^-23 grid of midpoints, u = ((h >> 9) + 1/2) 2^-23 in (0,1); standard Gumbel g = -ln(-ln u).
+ * 2^-23 grid of midpoints, u = ((h mod 2^23) + 1/2) 2^-23 in (0,1); standard Gumbel g = -ln(-ln u).
  * The draw arg-max_v (x_v/tau + g_v) is then a sample of softmax(x/tau) (Gumbel-max), up to the
  * grid of u (largest g = 16.6).  The CUDA path implements the same integer recipe on its own. */
 static uint64_t mix64(uint64_t z) {
@@ -104,11 +104,12 @@ static uint64_t noise_row_key(uint64_t seed, int32_t step, int32_t b, int32_t k)
   return mix64(z ^ (((uint64_t)(uint32_t)b << 32) | (uint64_t)(uint32_t)k));
 }
 static uint32_t noise_hash(uint64_t row_key, uint32_t v) {
-  uint32_t x = (v ^ (uint32_t)(row_key >> 32)) * 0x9E3779B1u + (uint32_t)row_key;
-  x ^= x >> 16; x *= 0x21F0AAADu; x ^= x >> 15; x *= 0x735A2D97u; x ^= x >> 15;
-  return x;
+  uint64_t p = (uint64_t)(v ^ (uint32_t)(row_key >> 32)) * 0x9E3779B1ULL;      /* two multiply-and-fold rounds */
+  uint32_t h = (uint32_t)(p >> 32) ^ (uint32_t)p ^ (uint32_t)row_key;
+  p = (uint64_t)h * 0x85EBCA77ULL;
+  return (uint32_t)(p >> 32) ^ (uint32_t)p;
 }
-static double noise_uniform(uint32_t h) { return ((double)(h >> 9) + 0.5) * (1.0 / 8388608.0); }
+static double noise_uniform(uint32_t h) { return ((double)(h & 0x7FFFFFu) + 0.5) * (1.0 / 8388608.0); }
 static double noise_gumbel(uint32_t h) { return -log(-log(noise_uniform(h))); }
 
 /* Exported for the pins: the uniform and the Gumbel variate of entry v of row (seed, step, b, k). */

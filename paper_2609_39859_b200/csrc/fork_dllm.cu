@@ -1435,10 +1435,11 @@ extern "C" fork_status fork_grpo_loss(const fork_grpo_args* a, void* stream) {
 
 /* ---- derivative of the scored log-likelihoods with respect to the logits -------------------- */
 /* d/dx_v [w (x_tok - lse)] = w (1[v = tok] - p_v), p_v = exp(x_v - lse): one read of the row, one
-   write of the same size.  Work is cut into units of kBwdNT * kBwdVecs 128-bit vectors of one row;
+   write of the same size.  Work is cut into units of kBwdNT * kBwdVecs * kBwdIters 128-bit vectors of one row;
    the rows are those of the row list the active-set kernel built from `select`. */
 constexpr int kBwdNT = 256;
 constexpr int kBwdVecs = 2;
+constexpr int kBwdIters = 8;          /* a unit = kBwdIters inner iterations of one row (64 KB): per-row values are fetched once per unit */
 
 struct BwdParams {
   RowSource src; void* grad; long long gstride_b, gstride_l;
@@ -1459,7 +1460,8 @@ __device__ __forceinline__ void store_grad(float* p, float g) { *p = g; }
 template <typename T>
 __global__ void __launch_bounds__(kBwdNT) logprob_backward_kernel(BwdParams p) {
   constexpr int VEC = 16 / (int)sizeof(T);
-  constexpr int kUnitElems = kBwdNT * kBwdVecs * VEC;
+  constexpr int kStepElems = kBwdNT * kBwdVecs * VEC;          /* elements per inner iteration */
+  constexpr int kUnitElems = kStepElems * kBwdIters;           /* elements of one row per unit */
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const int R = p.hdr->R;
   const int V = p.src.V;
@@ -1467,7 +1469,8 @@ __global__ void __launch_bounds__(kBwdNT) logprob_backward_kernel(BwdParams p) {
   const long long U = (long long)R * units_per_row;
   for (long long u = blockIdx.x; u < U; u += gridDim.x) {
     const int r = (int)(u / units_per_row);
-    const int e0 = (int)(u - (long long)r * units_per_row) * kUnitElems;
+    const int u0 = (int)(u - (long long)r * units_per_row) * kUnitElems;
+    const int u1 = min(u0 + kUnitElems, V);
     const int2 bk = p.rows[r];
     const size_t at = (size_t)bk.x * p.Lt + bk.y;
     const int tok = p.tokens[at];
@@ -1476,7 +1479,14 @@ __global__ void __launch_bounds__(kBwdNT) logprob_backward_kernel(BwdParams p) {
     const float nl = -p.lse[at] * kLog2e;
     const T* row = row_ptr<T>(p.src, bk.x, bk.y);
     T* grow = reinterpret_cast<T*>(p.grad) + ((long long)bk.x * p.gstride_b + (long long)(bk.y - p.src.pos0) * p.gstride_l);
-    if (p.vector_ok) {
+    if (!p.vector_ok) {
+      for (int q = u0 + (int)threadIdx.x; q < u1; q += kBwdNT) {
+        const float pr = exp2f(fmaf(to_f32(row[q]), kLog2e, nl));
+        store_grad(grow + q, w * ((q == tok ? 1.f : 0.f) - pr));
+      }
+      continue;
+    }
+    for (int e0 = u0; e0 < u1; e0 += kStepElems) {
       uint4 v[kBwdVecs];
       int e[kBwdVecs];
 #pragma unroll
@@ -1514,12 +1524,6 @@ __global__ void __launch_bounds__(kBwdNT) logprob_backward_kernel(BwdParams p) {
             store_grad(grow + q, w * ((q == tok ? 1.f : 0.f) - pr));
           }
         }
-      }
-    } else {
-      const int e1 = min(e0 + kUnitElems, V);
-      for (int q = e0 + (int)threadIdx.x; q < e1; q += kBwdNT) {
-        const float pr = exp2f(fmaf(to_f32(row[q]), kLog2e, nl));
-        store_grad(grow + q, w * ((q == tok ? 1.f : 0.f) - pr));
       }
     }
   }

@@ -372,12 +372,11 @@ __device__ __forceinline__ bool part_is_finite(const Part& p) { return isfinite(
 /* Stochastic candidates (Algorithm 2 line 4 with tau > 0): x_0 ~ softmax(x / tau) drawn as
  * arg-max_v (x_v / tau + g_v), g_v standard Gumbel noise (Gumbel-max).  The noise stream is a
  * counter-based generator: a 64-bit key per (seed, step, sequence, position), a 32-bit hash per
- * vocabulary entry, the uniform u = ((h >> 9) + 1/2) 2^-23, g = -ln E with E = -ln u.
- * Keys are compared in log2 units with constants dropped:  key = x * (log2 e / tau) - log2 E.
- * log2 E takes two special-function evaluations, except close to u = 1, where lg2.approx has only
- * an absolute error bound and E = w + w^2/2 + ... (w = 1 - u, exact) is used instead:
- *     log2 E = log2 w + w / (2 ln 2)            for w < 2^-8,
- *     log2 E = log2(-log2 u) + log2(ln 2)       otherwise.                                       */
+ * vocabulary entry, the uniform u = ((h mod 2^23) + 1/2) 2^-23, g = -ln E with E = -ln u.
+ * Keys are compared in log2 units with constants dropped:  key = x * (log2 e / tau) - log2(E / ln 2).
+ * E / ln 2 = -log2 u comes from lg2.approx, except close to u = 1, where that instruction has only
+ * an absolute error bound and the series -log2(1 - w) = (w + w^2/2 + ...) / ln 2 in w = 1 - u (exact)
+ * is used instead (w < 2^-8: the dropped terms are below 2e-6 relative).                          */
 struct NoiseRow {
   uint32_t lo, hi;             /* the row's key */
   float c;                     /* log2(e) / tau */
@@ -399,16 +398,17 @@ __device__ __forceinline__ float lg2_approx(float x) {
 }
 /* perturbed key of logit x at vocabulary index v */
 __device__ __forceinline__ float noise_key(const NoiseRow& nz, float x, uint32_t v) {
-  uint32_t h = (v ^ nz.hi) * 0x9E3779B1u + nz.lo;
-  h ^= h >> 16; h *= 0x21F0AAADu; h ^= h >> 15; h *= 0x735A2D97u; h ^= h >> 15;
-  const float f = __uint_as_float((h >> 9) | 0x3f800000u);   /* 1 + n 2^-23 */
+  uint64_t p = (uint64_t)(v ^ nz.hi) * 0x9E3779B1ull;          /* two multiply-and-fold rounds */
+  uint32_t h = (uint32_t)(p >> 32) ^ (uint32_t)p ^ nz.lo;
+  p = (uint64_t)h * 0x85EBCA77ull;
+  h = (uint32_t)(p >> 32) ^ (uint32_t)p;
+  const float f = __uint_as_float((h & 0x007fffffu) | 0x3f800000u);   /* 1 + n 2^-23 */
   const float u = f - 0.99999994f;                           /* (2n+1) 2^-24, exact */
   const float w = 1.0f - u;                                  /* (2^24 - 2n - 1) 2^-24, exact */
-  const bool near_one = w < 0.00390625f;
-  const float l1 = lg2_approx(u);
-  const float l2 = lg2_approx(near_one ? w : -l1);
-  const float corr = near_one ? w * 0.72134752f : -0.52876637f;
-  return __fmaf_rn(x, nz.c, -(l2 + corr));
+  /* E / ln 2 = -log2 u, from the series in w where lg2.approx is not accurate enough */
+  const float series = w * __fmaf_rn(0.72134752f, w, 1.44269504f);
+  const float e2 = (w < 0.00390625f) ? series : -lg2_approx(u);
+  return __fmaf_rn(x, nz.c, -lg2_approx(e2));                /* log2(ln 2) is the same for every entry: dropped */
 }
 
 /* The largest perturbed key a thread / warp / CTA / row has seen, and where: `vec` is the start of
