@@ -359,6 +359,46 @@ def time_logprob(device, peak):
     return out
 
 
+def time_vocab_parallel(device, peak, n_ranks=8):
+    """Per-rank work of the vocabulary-parallel step at the passk shape: fork_vp_reduce on one
+    rank's slice (V/n_ranks entries of every live row) and fork_vp_select on n_ranks gathered
+    buffers.  The all-gather between them (16 bytes per position and rank) is not run here."""
+    import torch
+    import fork_synth as fs
+    import paper_2609_39859_b200 as pkg
+    w = fs.workload("passk")
+    cfg, bufs, states, lo, hi = full_block_setup(w, w.seed, 2, 1, device)
+    st = states[0]
+    off, n = pkg.vocab_shards(w.V, n_ranks, w.es)[1]
+    shard = bufs[0][:, :, off:off + n]
+    parts = []
+    for r, (o, m) in enumerate(pkg.vocab_shards(w.V, n_ranks, w.es)):
+        parts.append(pkg.fork_vp_reduce(st, bufs[0][:, :, o:o + m], lo, hi, w.threshold, o)[0])
+    gathered = torch.stack(parts, 0)
+    e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+    t_red = t_sel = 0.0
+    reps = 20
+    for i in range(reps + 3):
+        reset_states([st])
+        flush = bufs[1].view(torch.int16)[:, :8].sum()          # touch another buffer: the slice is 65 MB, within L2
+        e0.record()
+        pkg.fork_vp_reduce(st, shard, lo, hi, w.threshold, off)
+        e1.record()
+        pkg.fork_vp_select(st, gathered, None, lo, hi, w.threshold, Ll=w.block_len)
+        e2.record()
+        torch.cuda.synchronize()
+        if i >= 3:
+            t_red += e0.elapsed_time(e1)
+            t_sel += e1.elapsed_time(e2)
+    rows = w.B * w.block_len
+    ms_red, ms_sel = t_red / reps, t_sel / reps
+    return {"workload": "passk sharded over %d ranks along V (one rank's share, emulated on one GPU): "
+                        "fork_vp_reduce on a [%d,%d,%d] slice + fork_vp_select on %d gathered buffers" %
+                        (n_ranks, w.B, w.block_len, n, n_ranks),
+            "reduce_ms": ms_red, "select_ms": ms_sel, "slice_gbs": rows * n * w.es / (ms_red * 1e-3) / 1e9,
+            "exchange_bytes_per_rank": rows * 16, "note": "slice (%.0f MB) may be L2-resident between repetitions" % (rows * n * w.es / 1e6)}
+
+
 def time_select(device):
     """JustGRPO-Fast's top-entropy selection at the scoring shape."""
     import torch
@@ -607,6 +647,7 @@ def main():
                                    " -- stochastic candidates, tau=0.8"))
         also.extend(time_logprob(device, peak))
         also.append(time_select(device))
+        also.append(time_vocab_parallel(device, peak))
         out["also"] = also
         out["cpu_baseline"] = cpu_baseline(w, seed)
         if args.loops:

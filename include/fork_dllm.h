@@ -201,6 +201,31 @@ fork_status fork_grpo_loss(const fork_grpo_args* args, void* stream);
 fork_status fork_logprob_backward(const fork_logprob_bwd_args* args, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The step with the vocabulary sharded over N ranks (a vocabulary-parallel LM head): rank j holds
+ * logits [B, Ll, V_j], the entries [offset_j, offset_j + V_j) of every row, offsets ascending with
+ * the rank.  tokens / mask / block bounds are replicated.  The paper runs on one GPU and has no
+ * counterpart; the merge is the associative one the single-GPU kernels already use between CTAs.
+ *
+ *   1. fork_vp_reduce on every rank: args as for fork_step with logits = the slice and V = V_j; nothing
+ *      is committed.  For every live position it writes part_out[b,k] = (m, s, t2, index) as four
+ *      32-bit words (float, float, float, int32: slice maximum, sum 2^((x-m) log2 e), sum of
+ *      (x-m) log2 e * 2^(...), GLOBAL index of the lowest arg-max; s = NaN if the slice holds NaN or
+ *      +inf; m = -inf, s = t2 = 0 if it holds nothing but -inf), and with temperature > 0 also
+ *      key_out[b,k] = (largest perturbed key, global index of that entry, its logit, 0).  The noise
+ *      of an entry depends on its global index, so the draw does not depend on the sharding.
+ *      part_out / key_out: device, [B,Lt] x 16 bytes, 16-byte aligned; other positions untouched.
+ *   2. the caller gathers the N buffers (e.g. one all-gather) into [N][B,Lt] in rank order.
+ *   3. fork_vp_select on every rank: merges the N parts of each live row in rank order, derives
+ *      confidence, candidate, entropy, log-probability, and applies the unmask rule exactly as
+ *      fork_step does (all of its outputs, all fallback orders).  args->logits is not read; Ll and
+ *      pos0 must be those given to fork_vp_reduce (Ll = 0 means the whole sequence).
+ */
+fork_status fork_vp_reduce(const fork_step_args* args, int32_t vocab_offset, void* part_out, void* key_out,
+                           void* workspace, size_t workspace_bytes, void* stream);
+fork_status fork_vp_select(const fork_step_args* args, const void* parts, const void* keys, int32_t n_ranks,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * fork_step without a workspace argument, for callers that have no device memory to give and
  * cannot allocate any.  (The paper has no counterpart of this entry point; it exists for
  * deployment.)  Typical callers: an inference server whose memory pool already owns the whole

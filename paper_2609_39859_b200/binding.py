@@ -72,7 +72,7 @@ fork_logits_fn = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32, C.c_void_p, C.c_voi
                              C.c_void_p, C.c_void_p)
 
 EXPORTS = ("fork_workspace_bytes", "fork_step", "fork_step_static", "fork_logprob", "fork_decode_loop", "fork_staging_bytes",
-           "fork_select_top_entropy", "fork_grpo_loss", "fork_logprob_backward",
+           "fork_select_top_entropy", "fork_grpo_loss", "fork_logprob_backward", "fork_vp_reduce", "fork_vp_select",
            "fork_step_host", "fork_device_status", "fork_status_string", "fork_set_tuning",
            "fork_kernel_launches", "fork_set_timing_events")
 
@@ -122,6 +122,12 @@ def lib():
     L.fork_grpo_loss.argtypes = [C.POINTER(fork_grpo_args), C.c_void_p]
     L.fork_logprob_backward.restype = C.c_int
     L.fork_logprob_backward.argtypes = [C.POINTER(fork_logprob_bwd_args), C.c_void_p, C.c_size_t, C.c_void_p]
+    L.fork_vp_reduce.restype = C.c_int
+    L.fork_vp_reduce.argtypes = [C.POINTER(fork_step_args), C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                                 C.c_void_p]
+    L.fork_vp_select.restype = C.c_int
+    L.fork_vp_select.argtypes = [C.POINTER(fork_step_args), C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_size_t,
+                                 C.c_void_p]
     L.fork_set_timing_events.restype = None
     L.fork_set_timing_events.argtypes = [C.c_void_p, C.c_void_p]
     _lib = L
@@ -203,13 +209,16 @@ class ForkState:
 def make_step_args(st: ForkState, logits: torch.Tensor, blk_lo, blk_hi, threshold: float, step: int = 0,
                    pos0: int = 0, fallback_mode: int = FORK_FALLBACK_LEFTMOST, fallback_rand=None,
                    temperature: float = 0.0, sample_seed: int = 0) -> fork_step_args:
-    assert logits.dim() == 3 and logits.stride(2) == 1, "logits must be [B, Ll, V] with V contiguous"
-    B, Ll, V = logits.shape
-    assert B == st.B
     a = fork_step_args()
-    a.logits = logits.data_ptr()
-    a.stride_b, a.stride_l, a.pos0 = logits.stride(0), logits.stride(1), pos0
-    a.B, a.Lt, a.Ll, a.V, a.dtype = B, st.Lt, Ll, V, _dtype_code(logits)
+    if logits is None:                   # fork_vp_select: the logits are not read
+        a.B, a.Lt, a.pos0 = st.B, st.Lt, pos0
+    else:
+        assert logits.dim() == 3 and logits.stride(2) == 1, "logits must be [B, Ll, V] with V contiguous"
+        B, Ll, V = logits.shape
+        assert B == st.B
+        a.logits = logits.data_ptr()
+        a.stride_b, a.stride_l, a.pos0 = logits.stride(0), logits.stride(1), pos0
+        a.B, a.Lt, a.Ll, a.V, a.dtype = B, st.Lt, Ll, V, _dtype_code(logits)
     a.tokens, a.mask = st.tokens.data_ptr(), st.mask.data_ptr()
     a.blk_lo, a.blk_hi = _p(blk_lo), _p(blk_hi)
     a.threshold, a.step = float(threshold), int(step)
@@ -368,3 +377,64 @@ def fork_logprob_backward(logits: torch.Tensor, tokens: torch.Tensor, select: to
     rc = lib().fork_logprob_backward(C.byref(a), C.c_void_p(st.ws_ptr), st.ws_bytes, _stream_ptr(stream))
     if rc != FORK_OK:
         raise ForkError(rc, "fork_logprob_backward")
+
+
+# ---- vocabulary-parallel step -------------------------------------------------------------------
+def vocab_shards(V: int, n_ranks: int, elem_size: int):
+    """(offset, length) of every rank's slice of the vocabulary: equal sizes rounded so that each
+    slice starts on a 16-byte boundary (the last rank takes the remainder)."""
+    per = 16 // elem_size
+    base = -(-V // n_ranks)
+    base = -(-base // per) * per
+    out = []
+    for r in range(n_ranks):
+        lo = min(r * base, V)
+        out.append((lo, max(0, min(V, lo + base) - lo)))
+    return out
+
+
+def fork_vp_reduce(st: ForkState, logits_slice: torch.Tensor, blk_lo, blk_hi, threshold: float, vocab_offset: int,
+                   step: int = 0, pos0: int = 0, stream=None, **variant):
+    """Local phase on this rank's slice [B, Ll, V_local]: returns (parts [B,Lt,4] float32, keys
+    [B,Lt,4] float32 or None) for the exchange; nothing is committed."""
+    a = make_step_args(st, logits_slice, blk_lo, blk_hi, threshold, step, pos0, **variant)
+    dev = logits_slice.device
+    parts = torch.zeros((st.B, st.Lt, 4), dtype=torch.float32, device=dev)
+    keys = torch.zeros((st.B, st.Lt, 4), dtype=torch.float32, device=dev) if a.temperature > 0 else None
+    rc = lib().fork_vp_reduce(C.byref(a), int(vocab_offset), C.c_void_p(parts.data_ptr()), C.c_void_p(_p(keys) or 0),
+                              C.c_void_p(st.ws_ptr), st.ws_bytes, _stream_ptr(stream))
+    if rc != FORK_OK:
+        raise ForkError(rc, "fork_vp_reduce")
+    return parts, keys
+
+
+def fork_vp_select(st: ForkState, parts: torch.Tensor, keys, blk_lo, blk_hi, threshold: float, step: int = 0,
+                   pos0: int = 0, Ll: int = 0, stream=None, **variant) -> None:
+    """Select phase on the gathered slices: parts (and keys) are [N, B, Lt, 4] in rank order."""
+    assert parts.dim() == 4 and parts.is_contiguous() and parts.dtype == torch.float32
+    a = make_step_args(st, None, blk_lo, blk_hi, threshold, step, pos0, **variant)
+    a.Ll = Ll
+    rc = lib().fork_vp_select(C.byref(a), C.c_void_p(parts.data_ptr()), C.c_void_p(_p(keys) or 0), parts.shape[0],
+                              C.c_void_p(st.ws_ptr), st.ws_bytes, _stream_ptr(stream))
+    if rc != FORK_OK:
+        raise ForkError(rc, "fork_vp_select")
+
+
+def gather_rank_major(t: torch.Tensor, group=None) -> torch.Tensor:
+    """All-gather of one tensor per rank into [world, ...] in rank order (torch.distributed)."""
+    import torch.distributed as dist
+    world = dist.get_world_size(group)
+    out = [torch.empty_like(t) for _ in range(world)]
+    dist.all_gather(out, t.contiguous(), group=group)
+    return torch.stack(out, 0)
+
+
+def fork_step_vocab_parallel(st: ForkState, logits_slice: torch.Tensor, blk_lo, blk_hi, threshold: float,
+                             vocab_offset: int, step: int = 0, pos0: int = 0, group=None, stream=None, **variant) -> None:
+    """One sampling step with the vocabulary sharded over the ranks of `group`: local reduction, one
+    all-gather of 16 (32 with drawn candidates) bytes per position, selection on every rank.  Slices
+    must ascend with the rank (vocab_shards)."""
+    parts, keys = fork_vp_reduce(st, logits_slice, blk_lo, blk_hi, threshold, vocab_offset, step, pos0, stream, **variant)
+    g_parts = gather_rank_major(parts, group)
+    g_keys = gather_rank_major(keys, group) if keys is not None else None
+    fork_vp_select(st, g_parts, g_keys, blk_lo, blk_hi, threshold, step, pos0, logits_slice.shape[1], stream, **variant)

@@ -99,6 +99,10 @@ struct ReduceParams {
   int32_t* n_unmasked; uint8_t* is_fallback; int32_t* fallback_pos; int32_t* nfe; int32_t* n_fallback;
   int fallback_mode; const uint32_t* fallback_rand;
   float noise_c; unsigned long long sample_seed;      /* stochastic candidates: log2(e)/tau and the noise stream */
+  /* vocabulary-parallel slices */
+  int vocab_offset;                  /* global index of entry 0 of this buffer */
+  float4* vp_part; float4* vp_key;   /* [B,Lt] local phase: per-position results for the exchange instead of the unmask rule */
+  const float4* vp_parts_in; const float4* vp_keys_in; int vp_ranks;   /* select phase: gathered [ranks][B,Lt] */
   /* log-probability mode */
   const int32_t* lp_tokens; float* lp_out; float* seq_sum; int32_t* seq_cnt; float* lse_out;
 };
@@ -306,7 +310,7 @@ __device__ __forceinline__ Part merge_row_parts_warp(const ReduceParams& p, int 
 
 /* Guarded scalar reduction of a whole row by ONE warp (every lane returns the same Part). */
 template <typename T>
-__device__ Part careful_row_warp(const T* row, int V, bool& bad) {
+__device__ Part careful_row_warp(const T* row, int V, bool& bad, bool* nonfinite = nullptr) {
   const int lane = threadIdx.x & 31;
   float m = -INFINITY;
   int idx = -1, isbad = 0;
@@ -325,6 +329,7 @@ __device__ Part careful_row_warp(const T* row, int V, bool& bad) {
     if (take) { m = om; idx = oi; }
   }
   isbad = __any_sync(0xffffffffu, isbad);
+  if (nonfinite) *nonfinite = isbad != 0;                    /* NaN or +inf seen (as opposed to nothing but -inf) */
   if (isbad || idx == kIdxNone || m == -INFINITY) {
     bad = true;
     return Part{m, __int_as_float(0x7fc00000), __int_as_float(0x7fc00000), idx == kIdxNone ? 0 : idx};
@@ -359,46 +364,63 @@ __device__ __forceinline__ KeyPart merge_row_keys(const ReduceParams& p, int r, 
    Rows whose streamed result is not finite are re-read by the whole warp with the guarded routine.
    With SAMPLE the candidate is the drawn token (the element holding the row's largest perturbed
    key) and confidence / log-probability are those of that token; flagged rows keep the arg-max. */
+/* Rows base .. base+31 of sequence b, one per lane: the row's parts merged, rows whose streamed
+   result is not finite re-read by the whole warp with the guarded routine. */
+struct MergedRow {
+  Part merged; int k, g0, nparts; bool valid, bad, nonfinite;
+};
+template <typename T>
+__device__ __forceinline__ MergedRow merge_rows_warp(const ReduceParams& p, const PartitionCtx& c, int b, int base, int r1,
+                                                     int k_hint) {
+  const int lane = threadIdx.x & 31;
+  const int r = base + lane;
+  MergedRow m;
+  m.valid = r < r1; m.bad = false; m.nonfinite = false;
+  m.merged = part_empty();
+  m.k = 0; m.g0 = 0; m.nparts = 0;
+  bool redo = false;
+  if (m.valid) { m.k = (k_hint >= 0) ? k_hint : p.rows[r].y; m.merged = merge_row_parts(p, c, r, m.g0, m.nparts); }
+  unsigned many = __ballot_sync(0xffffffffu, m.valid && m.nparts > kLaneMergeMax);
+  while (many) {                                             /* rows cut into very many parts: all lanes help */
+    const int src = __ffs(many) - 1;
+    many &= many - 1;
+    const Part w = merge_row_parts_warp(p, __shfl_sync(0xffffffffu, r, src), __shfl_sync(0xffffffffu, m.g0, src),
+                                        __shfl_sync(0xffffffffu, m.nparts, src));
+    if (lane == src) m.merged = w;
+  }
+  if (m.valid) redo = part_needs_careful(m.merged);
+  unsigned todo = __ballot_sync(0xffffffffu, m.valid && redo);
+  while (todo) {
+    const int src = __ffs(todo) - 1;
+    todo &= todo - 1;
+    const int kk = __shfl_sync(0xffffffffu, m.k, src);
+    bool bd, nf;
+    const Part cp = careful_row_warp<T>(row_ptr<T>(p.src, b, kk), p.src.V, bd, &nf);
+    if (lane == src) { m.merged = cp; m.bad = bd; m.nonfinite = nf; }
+  }
+  return m;
+}
+
 template <typename T, bool WANT_INDEX, bool SAMPLE>
 __device__ __forceinline__ RowOut finalize_rows_warp(const ReduceParams& p, const PartitionCtx& c, int b, int base,
                                                      int r1, Part& merged, int& k, int k_hint) {
   const int lane = threadIdx.x & 31;
   const int r = base + lane;
-  const bool valid = r < r1;
-  bool redo = false, bad = false;
-  merged = part_empty();
-  k = 0;
-  int g0 = 0, nparts = 0;
-  if (valid) { k = (k_hint >= 0) ? k_hint : p.rows[r].y; merged = merge_row_parts(p, c, r, g0, nparts); }
-  unsigned many = __ballot_sync(0xffffffffu, valid && nparts > kLaneMergeMax);
-  while (many) {                                             /* rows cut into very many parts: all lanes help */
-    const int src = __ffs(many) - 1;
-    many &= many - 1;
-    const Part m = merge_row_parts_warp(p, __shfl_sync(0xffffffffu, r, src), __shfl_sync(0xffffffffu, g0, src),
-                                        __shfl_sync(0xffffffffu, nparts, src));
-    if (lane == src) merged = m;
-  }
-  if (valid) redo = part_needs_careful(merged);
-  unsigned todo = __ballot_sync(0xffffffffu, valid && redo);
-  while (todo) {
-    const int src = __ffs(todo) - 1;
-    todo &= todo - 1;
-    const int kk = __shfl_sync(0xffffffffu, k, src);
-    bool bd;
-    const Part cp = careful_row_warp<T>(row_ptr<T>(p.src, b, kk), p.src.V, bd);
-    if (lane == src) { merged = cp; bad = bd; }
-  }
+  MergedRow m = merge_rows_warp<T>(p, c, b, base, r1, k_hint);
+  k = m.k;
   if (SAMPLE) {
     float xs = 0.f;
-    if (valid && !bad) {
-      const KeyPart kp = merge_row_keys(p, r, g0, nparts);
-      const NoiseRow nz = noise_row(p.sample_seed, p.step, b, k, p.noise_c);
-      merged.idx = resolve_sample<T>(row_ptr<T>(p.src, b, k), nz, kp.vec, p.src.V, kp.key, xs);
+    if (m.valid && !m.bad) {
+      const KeyPart kp = merge_row_keys(p, r, m.g0, m.nparts);
+      const NoiseRow nz = noise_row(p.sample_seed, p.step, b, k, p.noise_c, (uint32_t)p.vocab_offset);
+      m.merged.idx = resolve_sample<T>(row_ptr<T>(p.src, b, k), nz, kp.vec, p.src.V, kp.key, xs);
     }
-    return row_out_sampled(merged, bad, xs);
+    merged = m.merged;
+    return row_out_sampled(merged, m.bad, xs);
   }
-  if (valid && WANT_INDEX && !bad) merged.idx = resolve_index<T>(row_ptr<T>(p.src, b, k), merged.idx, p.src.V, merged.m);
-  return row_out_from(merged, bad);
+  if (m.valid && WANT_INDEX && !m.bad) m.merged.idx = resolve_index<T>(row_ptr<T>(p.src, b, k), m.merged.idx, p.src.V, m.merged.m);
+  merged = m.merged;
+  return row_out_from(merged, m.bad);
 }
 
 /* What a finaliser can load about a sequence BEFORE its last part arrives (it idles until then):
@@ -410,6 +432,67 @@ __device__ __forceinline__ SeqHint load_seq_hint(const ReduceParams& p, int b) {
   const int r = h.r0 + (int)(threadIdx.x & 31);
   h.k = (r < h.r1) ? p.rows[r].y : -1;
   return h;
+}
+
+/* ---- vocabulary-parallel slices ------------------------------------------------------------- */
+/* Local phase: what this slice contributes to every live row of sequence b, written per position
+   for the exchange: (m, s, t2, global index of the lowest arg-max), s = NaN when the slice holds
+   NaN or +inf, the neutral element (m = -inf, s = t2 = 0) when it holds nothing but -inf; with
+   stochastic candidates also (largest perturbed key, global index of its entry, that logit). */
+template <typename T, bool SAMPLE>
+__device__ void finalize_vp_local(const ReduceParams& p, const PartitionCtx& c, int b, const SeqHint& h) {
+  const int lane = threadIdx.x & 31;
+  const float qnan = __int_as_float(0x7fc00000);
+  for (int base = h.r0; base < h.r1; base += 32) {
+    const int r = base + lane;
+    MergedRow m = merge_rows_warp<T>(p, c, b, base, h.r1, base == h.r0 ? h.k : -1);
+    if (!m.valid) continue;
+    const size_t at = (size_t)b * p.Lt + m.k;
+    const T* row = row_ptr<T>(p.src, b, m.k);
+    float4 out, kout = make_float4(-INFINITY, __int_as_float(kIdxNone), 0.f, 0.f);
+    if (m.bad && !m.nonfinite) {
+      out = make_float4(-INFINITY, 0.f, 0.f, __int_as_float(p.vocab_offset));
+    } else if (m.bad) {
+      out = make_float4(m.merged.m, qnan, qnan, __int_as_float(p.vocab_offset + m.merged.idx));
+    } else {
+      const int idx = resolve_index<T>(row, m.merged.idx, p.src.V, m.merged.m);
+      out = make_float4(m.merged.m, m.merged.s, m.merged.t, __int_as_float(p.vocab_offset + idx));
+      if (SAMPLE) {
+        const KeyPart kp = merge_row_keys(p, r, m.g0, m.nparts);
+        const NoiseRow nz = noise_row(p.sample_seed, p.step, b, m.k, p.noise_c, (uint32_t)p.vocab_offset);
+        float xs;
+        const int si = resolve_sample<T>(row, nz, kp.vec, p.src.V, kp.key, xs);
+        kout = make_float4(kp.key, __int_as_float(p.vocab_offset + si), xs, 0.f);
+      }
+    }
+    p.vp_part[at] = out;
+    if (SAMPLE) p.vp_key[at] = kout;
+  }
+}
+
+/* Select phase: the statistics of rows base .. base+31 of sequence b from the gathered slices,
+   merged in rank order (ascending vocabulary offset; ties keep the lowest global index). */
+template <bool SAMPLE>
+__device__ __forceinline__ RowOut gathered_rows_warp(const ReduceParams& p, int b, int base, int r1, int& k, int k_hint) {
+  const int lane = threadIdx.x & 31;
+  const int r = base + lane;
+  k = 0;
+  if (r >= r1) return row_out_from(part_empty(), true);
+  k = (k_hint >= 0) ? k_hint : p.rows[r].y;
+  const size_t at = (size_t)b * p.Lt + k, n = (size_t)p.B * p.Lt;
+  Part acc = part_empty();
+  for (int j = 0; j < p.vp_ranks; ++j) acc = part_merge(acc, part_from(__ldg(p.vp_parts_in + j * n + at)));
+  const bool bad = !(isfinite(acc.s) && isfinite(acc.t)) || !(acc.m > -INFINITY) || acc.m == INFINITY;
+  if (!SAMPLE || bad) return row_out_from(acc, bad);
+  float best = -INFINITY, xs = 0.f;
+  int bidx = kIdxNone;
+  for (int j = 0; j < p.vp_ranks; ++j) {
+    const float4 q = __ldg(p.vp_keys_in + j * n + at);
+    const int qi = __float_as_int(q.y);
+    if (q.x > best || (q.x == best && qi < bidx)) { best = q.x; bidx = qi; xs = q.z; }
+  }
+  acc.idx = bidx;
+  return row_out_sampled(acc, false, xs);
 }
 
 /* Key by which a fallback step ranks a row under the orders other than "leftmost" (the largest key
@@ -424,7 +507,7 @@ __device__ __forceinline__ float fallback_key(int mode, float conf, float entrop
    (Algorithm 2 lines 6-9): commit every live position whose confidence exceeds lambda, or one
    position when none does -- the leftmost live one (Fork-dLLM), or the one the requested
    comparison order picks; write tokens, mask and the per-token records. */
-template <typename T, bool SAMPLE>
+template <typename T, bool SAMPLE, bool GATHERED = false>
 __device__ void finalize_step_sequence(const ReduceParams& p, const PartitionCtx& c, int b, const SeqHint& h) {
   const int lane = threadIdx.x & 31;
   const int r0 = h.r0, r1 = h.r1;
@@ -437,7 +520,8 @@ __device__ void finalize_step_sequence(const ReduceParams& p, const PartitionCtx
   int best_r = 0x7fffffff;
   for (int base = r0; base < r1; base += 32) {
     Part merged; int k;
-    const RowOut o = finalize_rows_warp<T, true, SAMPLE>(p, c, b, base, r1, merged, k, base == r0 ? h.k : -1);
+    const RowOut o = GATHERED ? gathered_rows_warp<SAMPLE>(p, b, base, r1, k, base == r0 ? h.k : -1)
+                              : finalize_rows_warp<T, true, SAMPLE>(p, c, b, base, r1, merged, k, base == r0 ? h.k : -1);
     const int r = base + lane;
     if (r < r1) {
       const size_t at = (size_t)b * p.Lt + k;
@@ -603,8 +687,8 @@ __global__ void __launch_bounds__(kNT, 4) reduce_select_kernel(ReduceParams p) {
     Part part;
     KeyTrack kt;
     kt.init();
-    NoiseRow nz = NoiseRow{0u, 0u, 0.f};
-    if (SAMPLE) nz = noise_row(p.sample_seed, p.step, bk.x, bk.y, p.noise_c);
+    NoiseRow nz = NoiseRow{0u, 0u, 0.f, 0u};
+    if (SAMPLE) nz = noise_row(p.sample_seed, p.step, bk.x, bk.y, p.noise_c, (uint32_t)p.vocab_offset);
     if (p.fast) {
       part = part_block_reduce<kNT>(
           stream_thread<T, WITH_T, kNT, kUnroll, SAMPLE>(row, sg.e0, sg.e1, threadIdx.x, threadIdx.x == 0, sticky, &kt, &nz),
@@ -622,6 +706,7 @@ __global__ void __launch_bounds__(kNT, 4) reduce_select_kernel(ReduceParams p) {
       if (last) {                                           /* every part of sequence b has been delivered */
         const SeqHint h = load_seq_hint(p, bk.x);
         if (MODE == kModeLogprob) finalize_logprob_sequence<T>(p, c, bk.x, h);
+        else if (p.vp_part) finalize_vp_local<T, SAMPLE>(p, c, bk.x, h);
         else finalize_step_sequence<T, SAMPLE>(p, c, bk.x, h);
       }
     }
@@ -749,8 +834,8 @@ __global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_sel
       a.init();
       KeyTrack kt;                                            /* stochastic candidates: largest perturbed key */
       kt.init();
-      NoiseRow nz = NoiseRow{0u, 0u, 0.f};
-      if (SAMPLE) { const int2 bk = p.rows[sg.r]; nz = noise_row(p.sample_seed, p.step, bk.x, bk.y, p.noise_c); }
+      NoiseRow nz = NoiseRow{0u, 0u, 0.f, 0u};
+      if (SAMPLE) { const int2 bk = p.rows[sg.r]; nz = noise_row(p.sample_seed, p.step, bk.x, bk.y, p.noise_c, (uint32_t)p.vocab_offset); }
       const int nvec = (sg.e1 - sg.e0) / VEC;
       for (int voff = 0; voff < nvec; voff += kStageVecs) {
         if (!mbar_wait(&rs.full[s], ph, p)) return;
@@ -845,10 +930,25 @@ __global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_sel
     if (SAMPLE) kp = key_warp_reduce(kp);
     if (publish_part(p, pt, sg.r, g, b, want, SAMPLE ? &kp : nullptr)) {
       if (MODE == kModeLogprob) finalize_logprob_sequence<T>(p, c, b, h);
+      else if (p.vp_part) finalize_vp_local<T, SAMPLE>(p, c, b, h);
       else finalize_step_sequence<T, SAMPLE>(p, c, b, h);
     }
     ++nseg;
   }
+}
+
+/* ---- vocabulary-parallel select phase: one warp per sequence on the gathered slices ---------- */
+constexpr int kVpNT = 256;
+template <bool SAMPLE>
+__global__ void __launch_bounds__(kVpNT) vp_select_kernel(ReduceParams p) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int b = (int)blockIdx.x * (kVpNT / 32) + (int)(threadIdx.x >> 5);
+  if (b >= p.B) return;
+  const SeqHint h = load_seq_hint(p, b);
+  if (h.r1 <= h.r0) return;                                  /* no live row: the active-set kernel wrote its outputs */
+  PartitionCtx c;
+  c.U = 0; c.G = 1; c.C = 1; c.small = true;
+  finalize_step_sequence<float, SAMPLE, true>(p, c, b, h);
 }
 
 /* ---- decode-loop helpers ------------------------------------------------------------------- */
@@ -1103,8 +1203,10 @@ static fork_status check_workspace(void* ws, size_t bytes, int32_t B, int32_t Lt
   return FORK_OK;
 }
 
+struct VpLocal { int32_t vocab_offset; float4* part; float4* key; };
+
 static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const int32_t* hi, void* ws,
-                             cudaStream_t st) {
+                             cudaStream_t st, const VpLocal* vp = nullptr) {
   DeviceInfo* dev;
   if (!device_info(&dev)) return FORK_ERR_CUDA;
   WsView w = ws_view(ws, a->B, a->Lt);
@@ -1118,7 +1220,7 @@ static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const i
   sp.flags = a->mask; sp.lo = lo; sp.hi = hi;
   sp.B = a->B; sp.Lt = a->Lt; sp.pos0 = a->pos0; sp.Ll = a->Ll; sp.C = C; sp.G = G;
   sp.hdr = w.hdr; sp.seq_off = w.seq_off; sp.expected = w.expected; sp.ticket = w.ticket; sp.rows = w.rows;
-  sp.n_unmasked = a->n_unmasked; sp.is_fallback = a->is_fallback; sp.fallback_pos = a->fallback_pos;
+  if (!vp) { sp.n_unmasked = a->n_unmasked; sp.is_fallback = a->is_fallback; sp.fallback_pos = a->fallback_pos; }
   if (launch(active_set_kernel, dim3(1), dim3(kSetupNT), st, g_tune[FORK_TUNE_PDL].load() >= 0, sp) != cudaSuccess) return FORK_ERR_CUDA;
 
   ReduceParams rp;
@@ -1136,6 +1238,7 @@ static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const i
   rp.n_unmasked = a->n_unmasked; rp.is_fallback = a->is_fallback; rp.fallback_pos = a->fallback_pos;
   rp.nfe = a->nfe; rp.n_fallback = a->n_fallback;
   rp.fallback_mode = a->fallback_mode; rp.fallback_rand = a->fallback_rand;
+  if (vp) { rp.vocab_offset = vp->vocab_offset; rp.vp_part = vp->part; rp.vp_key = vp->key; }
   if (launch_reduce(rp, a->dtype, mode, G, st) != cudaSuccess) return FORK_ERR_CUDA;
   return FORK_OK;
 }
@@ -1559,6 +1662,63 @@ extern "C" fork_status fork_logprob_backward(const fork_logprob_bwd_args* a, voi
   const int grid = dev->sms * 8;
   cudaError_t e = a->dtype == FORK_BF16 ? launch(logprob_backward_kernel<bf16_t>, dim3(grid), dim3(kBwdNT), st, pdl, bp)
                                         : launch(logprob_backward_kernel<float>, dim3(grid), dim3(kBwdNT), st, pdl, bp);
+  return e == cudaSuccess ? FORK_OK : FORK_ERR_CUDA;
+}
+
+/* ---- vocabulary-parallel entry points ------------------------------------------------------- */
+extern "C" fork_status fork_vp_reduce(const fork_step_args* a, int32_t vocab_offset, void* part_out, void* key_out,
+                                      void* ws, size_t ws_bytes, void* stream) {
+  fork_status s = check_step_args(a, true);
+  if (s != FORK_OK) return s;
+  if (!part_out || vocab_offset < 0 || (int64_t)vocab_offset + a->V > 0x7fffffffLL) return FORK_ERR_INVALID_ARG;
+  if (a->temperature > 0.f && !key_out) return FORK_ERR_INVALID_ARG;
+  if (((uintptr_t)part_out % 16) != 0 || ((uintptr_t)key_out % 16) != 0) return FORK_ERR_INVALID_ARG;
+  s = check_workspace(ws, ws_bytes, a->B, a->Lt);
+  if (s != FORK_OK) return s;
+  if (a->B == 0) return FORK_OK;
+  VpLocal vp{vocab_offset, (float4*)part_out, (float4*)key_out};
+  return step_impl(a, a->blk_lo, a->blk_hi, ws, (cudaStream_t)stream, &vp);
+}
+
+extern "C" fork_status fork_vp_select(const fork_step_args* a, const void* parts, const void* keys, int32_t n_ranks,
+                                      void* ws, size_t ws_bytes, void* stream) {
+  if (!a || a->B < 0 || a->Lt <= 0 || !a->tokens || !a->mask || !a->blk_lo || !a->blk_hi) return FORK_ERR_INVALID_ARG;
+  if ((int64_t)a->B * a->Lt > (int64_t)1 << 30) return FORK_ERR_INVALID_ARG;
+  if (a->threshold != a->threshold) return FORK_ERR_INVALID_ARG;
+  if (a->fallback_mode < FORK_FALLBACK_LEFTMOST || a->fallback_mode > FORK_FALLBACK_RANDOM) return FORK_ERR_INVALID_ARG;
+  if (a->fallback_mode == FORK_FALLBACK_RANDOM && !a->fallback_rand) return FORK_ERR_INVALID_ARG;
+  if (!(a->temperature >= 0.f) || a->temperature > 3.0e38f) return FORK_ERR_INVALID_ARG;
+  if (!parts || n_ranks <= 0 || (a->temperature > 0.f && !keys)) return FORK_ERR_INVALID_ARG;
+  if (((uintptr_t)parts % 16) != 0 || ((uintptr_t)keys % 16) != 0) return FORK_ERR_INVALID_ARG;
+  fork_status s = check_workspace(ws, ws_bytes, a->B, a->Lt);
+  if (s != FORK_OK) return s;
+  if (a->B == 0) return FORK_OK;
+  cudaStream_t st = (cudaStream_t)stream;
+  WsView w = ws_view(ws, a->B, a->Lt);
+  const bool pdl = g_tune[FORK_TUNE_PDL].load() >= 0;
+  SetupParams sp;
+  memset(&sp, 0, sizeof(sp));
+  sp.flags = a->mask; sp.lo = a->blk_lo; sp.hi = a->blk_hi;
+  sp.B = a->B; sp.Lt = a->Lt; sp.pos0 = 0; sp.Ll = a->Lt; sp.C = 1; sp.G = 1;
+  if (a->Ll > 0) { sp.pos0 = a->pos0; sp.Ll = a->Ll; }      /* the window the slices covered */
+  sp.hdr = w.hdr; sp.seq_off = w.seq_off; sp.expected = w.expected; sp.ticket = w.ticket; sp.rows = w.rows;
+  sp.n_unmasked = a->n_unmasked; sp.is_fallback = a->is_fallback; sp.fallback_pos = a->fallback_pos;
+  if (launch(active_set_kernel, dim3(1), dim3(kSetupNT), st, pdl, sp) != cudaSuccess) return FORK_ERR_CUDA;
+  ReduceParams rp;
+  memset(&rp, 0, sizeof(rp));
+  rp.B = a->B; rp.Lt = a->Lt; rp.C = 1;
+  rp.hdr = w.hdr; rp.seq_off = w.seq_off; rp.expected = w.expected; rp.ticket = w.ticket;
+  rp.rows = w.rows; rp.final_rec = w.final_rec; rp.parts = w.parts; rp.kparts = w.kparts;
+  rp.tokens = a->tokens; rp.mask = a->mask; rp.threshold = a->threshold; rp.step = a->step;
+  rp.conf = a->conf; rp.cand = a->cand; rp.entropy = a->entropy; rp.logp = a->logp; rp.row_status = a->row_status;
+  rp.commit_step = a->commit_step; rp.commit_fallback = a->commit_fallback; rp.commit_logp = a->commit_logp;
+  rp.n_unmasked = a->n_unmasked; rp.is_fallback = a->is_fallback; rp.fallback_pos = a->fallback_pos;
+  rp.nfe = a->nfe; rp.n_fallback = a->n_fallback;
+  rp.fallback_mode = a->fallback_mode; rp.fallback_rand = a->fallback_rand;
+  rp.vp_parts_in = (const float4*)parts; rp.vp_keys_in = (const float4*)keys; rp.vp_ranks = n_ranks;
+  const dim3 grid((unsigned)((a->B + kVpNT / 32 - 1) / (kVpNT / 32)));
+  cudaError_t e = a->temperature > 0.f ? launch(vp_select_kernel<true>, grid, dim3(kVpNT), st, pdl, rp)
+                                       : launch(vp_select_kernel<false>, grid, dim3(kVpNT), st, pdl, rp);
   return e == cudaSuccess ? FORK_OK : FORK_ERR_CUDA;
 }
 

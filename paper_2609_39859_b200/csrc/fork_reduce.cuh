@@ -380,16 +380,17 @@ __device__ __forceinline__ bool part_is_finite(const Part& p) { return isfinite(
 struct NoiseRow {
   uint32_t lo, hi;             /* the row's key */
   float c;                     /* log2(e) / tau */
+  uint32_t voff;               /* global vocabulary index of the buffer's entry 0 (a vocabulary-parallel slice) */
 };
 
 __device__ __forceinline__ uint64_t noise_mix64(uint64_t z) {
   z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ull; z ^= z >> 27; z *= 0x94D049BB133111EBull; z ^= z >> 31;
   return z;
 }
-__device__ __forceinline__ NoiseRow noise_row(uint64_t seed, int step, int b, int k, float c) {
+__device__ __forceinline__ NoiseRow noise_row(uint64_t seed, int step, int b, int k, float c, uint32_t voff) {
   uint64_t z = noise_mix64(seed + 0x9E3779B97F4A7C15ull * (uint64_t)((uint32_t)step + 1u));
   z = noise_mix64(z ^ (((uint64_t)(uint32_t)b << 32) | (uint64_t)(uint32_t)k));
-  return NoiseRow{(uint32_t)z, (uint32_t)(z >> 32), c};
+  return NoiseRow{(uint32_t)z, (uint32_t)(z >> 32), c, voff};
 }
 __device__ __forceinline__ float lg2_approx(float x) {
   float y;
@@ -398,7 +399,7 @@ __device__ __forceinline__ float lg2_approx(float x) {
 }
 /* perturbed key of logit x at vocabulary index v */
 __device__ __forceinline__ float noise_key(const NoiseRow& nz, float x, uint32_t v) {
-  uint64_t p = (uint64_t)(v ^ nz.hi) * 0x9E3779B1ull;          /* two multiply-and-fold rounds */
+  uint64_t p = (uint64_t)((v + nz.voff) ^ nz.hi) * 0x9E3779B1ull;   /* two multiply-and-fold rounds */
   uint32_t h = (uint32_t)(p >> 32) ^ (uint32_t)p ^ nz.lo;
   p = (uint64_t)h * 0x85EBCA77ull;
   h = (uint32_t)(p >> 32) ^ (uint32_t)p;

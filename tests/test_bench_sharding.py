@@ -66,3 +66,48 @@ def test_single_process_needs_no_process_group():
     import bench
     assert bench.max_over_ranks(3.5, torch.device("cpu")) == 3.5
     assert bench.shard_seed(5, 0) == 5
+
+
+def _vp_worker(rank, world, port, q):
+    import torch
+    import torch.distributed as dist
+    from paper_2609_39859_b200.binding import gather_rank_major, vocab_shards
+    dist.init_process_group("gloo", init_method="tcp://127.0.0.1:%d" % port, rank=rank, world_size=world)
+    try:
+        shards = vocab_shards(126464, world, 2)
+        off, n = shards[rank]
+        mine = torch.full((3, 5, 4), float(rank), dtype=torch.float32)
+        mine[0, 0, 3] = off
+        got = gather_rank_major(mine)
+        ok = got.shape == (world, 3, 5, 4) and all(float(got[r, 1, 1, 0]) == r and int(got[r, 0, 0, 3]) == shards[r][0]
+                                                    for r in range(world))
+        q.put((rank, bool(ok)))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_vocab_shards_and_rank_major_gather_with_two_gloo_ranks():
+    """Host side of the vocabulary-parallel step: slices cover the vocabulary, start on 16-byte
+    boundaries and ascend with the rank; the gather returns the ranks' buffers in rank order."""
+    import multiprocessing as mp
+    import socket
+    from paper_2609_39859_b200.binding import vocab_shards
+    for V, n, es in ((126464, 8, 2), (152064, 4, 2), (126464, 3, 4), (1000, 3, 2), (7, 4, 4)):
+        sh = vocab_shards(V, n, es)
+        assert sum(l for _, l in sh) == V and sh[0][0] == 0
+        for (o0, l0), (o1, _) in zip(sh, sh[1:]):
+            assert o1 == o0 + l0 or (l0 == 0 and o1 == V)
+        assert all((o * es) % 16 == 0 for o, l in sh if l > 0)
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_vp_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+    assert res == [(0, True), (1, True)]

@@ -315,3 +315,96 @@ def test_tiny_decode_loop_with_sampled_candidates():
     assert (h["tokens"] == h["cand"]).all()
     greedy, _, _, _ = oracle_reference_loop(w, B, w.threshold)
     assert (greedy.tokens != ost.tokens).any()                 # the draws are not the arg-max everywhere
+
+
+# ---- vocabulary-parallel slices (ranks emulated one after the other on one GPU) -------------------
+def vp_both(x, mask, lo, hi, lam, n_ranks, **variant):
+    """fork_vp_reduce on every slice in turn, then fork_vp_select, against the oracle on the whole
+    vocabulary."""
+    pkg = F()
+    B, Ll, V = x.shape
+    Lt = mask.shape[1]
+    o = oracle.StepState(B, Lt, mask=mask)
+    ov = dict(variant)
+    if "fallback_rand" in ov:
+        ov["fallback_rand"] = ov["fallback_rand"].cpu().numpy().view(np.uint32)
+    assert oracle.step(o, x, lo, hi, lam, step_id=4, **ov) == 0
+    if not decisions_are_clear(o, live_mask(mask, lo, hi), lam, 1e-4, variant.get("fallback_mode", 0),
+                               variant.get("temperature", 0.0)):
+        return None, o
+    g = pkg.ForkState(B, Lt, mask=mask)
+    xt = to_torch_logits(x)
+    lo_d, hi_d = torch.from_numpy(np.asarray(lo)).cuda(), torch.from_numpy(np.asarray(hi)).cuda()
+    parts, keys = [], []
+    for off, n in pkg.vocab_shards(V, n_ranks, xt.element_size()):
+        p_, k_ = pkg.fork_vp_reduce(g, xt[:, :, off:off + n], lo_d, hi_d, lam, off, step=4, **variant)
+        parts.append(p_)
+        keys.append(k_)
+    torch.cuda.synchronize()
+    assert (g.mask.cpu().numpy() == mask).all()                 # the local phase commits nothing
+    keys_t = torch.stack(keys, 0) if keys[0] is not None else None
+    pkg.fork_vp_select(g, torch.stack(parts, 0), keys_t, lo_d, hi_d, lam, step=4, Ll=Ll, **variant)
+    torch.cuda.synchronize()
+    return g.host(), o
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("V,n_ranks", [(4096, 2), (6151, 4), (40000, 8), (1000, 3)])
+def test_vocab_parallel_step_equals_the_full_vocabulary_oracle(V, n_ranks, dtype):
+    for seed in range(6):
+        rng = np.random.default_rng(V + n_ranks + seed)
+        B, Lt = 4, 40
+        mask = (rng.random((B, Lt)) < 0.7).astype(np.uint8)
+        lo = rng.integers(0, 10, size=B).astype(np.int32)
+        hi = (lo + rng.integers(0, 36, size=B)).astype(np.int32)
+        mask[2, lo[2]:hi[2]] = 0
+        x = make_rows(rng, (B, Lt), V, dtype, peak=6.0)
+        g, o = vp_both(x, mask, lo, hi, 0.9, n_ranks)
+        if g is None:
+            continue
+        compare_step_state(g, o)
+        return
+    raise AssertionError("no input with clear margins found")
+
+
+def test_vocab_parallel_special_rows():
+    """Slices holding nothing but -inf, NaN / +inf in one slice, a row that is -inf everywhere, ties
+    across slices (lowest global index), more than 32 live rows."""
+    rng = np.random.default_rng(9)
+    B, Lt, V, n_ranks = 2, 48, 4096, 4
+    mask = np.ones((B, Lt), np.uint8)
+    lo, hi = np.zeros(B, np.int32), np.full(B, Lt, np.int32)
+    x = make_rows(rng, (B, Lt), V, "f32", peak=6.0)
+    x[0, 0, :1024] = -np.inf                                  # first slice empty
+    x[0, 1, 1024:] = -np.inf                                  # only the first slice holds anything
+    x[0, 2, 2000] = np.nan
+    x[0, 3, 3000] = np.inf
+    x[0, 4, :] = -np.inf
+    x[0, 5, :] = 0.0                                          # ties everywhere: index 0 wins
+    top = x[0, 6].max() + 1.0
+    x[0, 6, 1500] = top
+    x[0, 6, 3500] = top                                       # tie across slices
+    g, o = vp_both(x, mask, lo, hi, 0.9, n_ranks)
+    assert g is not None
+    compare_step_state(g, o)
+    assert g["cand"][0, 5] == 0 and g["cand"][0, 6] == 1500 and g["row_status"][0, 4] == 1
+
+
+@pytest.mark.parametrize("n_ranks", [2, 4])
+def test_vocab_parallel_with_drawn_candidates_and_other_fallback_orders(n_ranks):
+    done = 0
+    for seed in range(12):
+        rng = np.random.default_rng(300 + seed)
+        B, Lt, V = 3, 20, 8192
+        mask = np.ones((B, Lt), np.uint8)
+        lo, hi = np.zeros(B, np.int32), np.full(B, Lt, np.int32)
+        x = make_rows(rng, (B, Lt), V, "bf16", peak=4.0, peak_frac=0.3)
+        rand = torch.from_numpy(rng.integers(0, 2 ** 31, B).astype(np.int32)).cuda()
+        variant = [dict(temperature=0.8, sample_seed=5 + seed), dict(fallback_mode=1),
+                   dict(temperature=1.2, sample_seed=seed, fallback_mode=3), dict(fallback_mode=4, fallback_rand=rand)][seed % 4]
+        g, o = vp_both(x, mask, lo, hi, 0.9, n_ranks, **variant)
+        if g is None:
+            continue
+        compare_step_state(g, o)
+        done += 1
+    assert done >= 6
