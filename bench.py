@@ -173,8 +173,9 @@ def time_full_block(w, seed, steps, warmup, device, use_graph=True, variant=None
     L = pkg.lib()
     cache = {}
 
-    def call(i, sp):
-        s, b = i % n_state, i % n_buf
+    def call(i, sp, s=None):
+        """step number i (selects the logits buffer) on state s (default i mod pool size)"""
+        s, b = (i % n_state if s is None else s), i % n_buf
         a = cache.get((s, b))
         if a is None:
             a = cache[(s, b)] = pkg.make_step_args(states[s], bufs[b], lo, hi, w.threshold, step=0, **(variant or {}))
@@ -189,7 +190,7 @@ def time_full_block(w, seed, steps, warmup, device, use_graph=True, variant=None
             chunk = min(n_state, n - done)
             reset_states(states[:chunk])
             for j in range(chunk):
-                call(first + done + j, sp)
+                call(first + done + j, sp, s=j)          # exactly the states that were just re-armed
             done += chunk
 
     stream = torch.cuda.current_stream()
@@ -235,7 +236,7 @@ def time_full_block(w, seed, steps, warmup, device, use_graph=True, variant=None
     torch.cuda.synchronize()
     for j in range(n):
         L.fork_set_timing_events(C.c_void_p(evs[j][0].cuda_event), C.c_void_p(evs[j][1].cuda_event))
-        call(warmup + j, sp)
+        call(warmup + j, sp, s=j)
     torch.cuda.synchronize()
     kernel_ms = sum(a.elapsed_time(b) for a, b in evs) / n
     return dict(rows=rows, row_bytes=row_bytes, total_ms=total_ms, ms_per_step=total_ms / steps,

@@ -727,11 +727,12 @@ __global__ void __launch_bounds__(kNT, 4) reduce_select_kernel(ReduceParams p) {
  *              ticket and, if it was the last, applies the unmask rule for that sequence.
  * Every mbarrier wait is bounded: after kSpinLimit failed polls the thread records
  * FORK_DEV_TIMEOUT in the workspace header and leaves its loop.                                   */
-constexpr int kMaxCW = 16;                                 /* consumer warps: 8 (two CTAs per SM) or 16 (one CTA per SM) */
+constexpr int kCW = 8;                                     /* consumer warps per CTA */
+constexpr int kMaxCW = kCW;
 constexpr int kMail = 4;                                   /* mailbox depth (row segments in flight to the finaliser) */
 constexpr int kMaxStages = 13;
 constexpr uint32_t kSpinLimit = 1u << 22;
-constexpr int ring_stage_bytes(int cw) { return cw * 32 * kUnroll * 16; }   /* 16 KB (8 warps) or 32 KB (16 warps) */
+constexpr int ring_stage_bytes() { return kCW * 32 * kUnroll * 16; }     /* 16 KB */
 
 struct RingSmem {
   unsigned long long full[kMaxStages], empty[kMaxStages], mfull[kMail], mempty[kMail];
@@ -768,8 +769,8 @@ __device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32
 }
 
 
-template <typename T, int MODE, int kCW>
-__global__ void __launch_bounds__((kCW + 2) * 32, (kCW == 8) ? 2 : 1) reduce_select_ring_kernel(ReduceParams p, int n_stages) {
+template <typename T, int MODE, int kPerSM>
+__global__ void __launch_bounds__((kCW + 2) * 32, kPerSM) reduce_select_ring_kernel(ReduceParams p, int n_stages) {
   constexpr bool WITH_T = mode_is_step(MODE);
   constexpr bool SAMPLE = (MODE == kModeSample);
   constexpr int VEC = 16 / (int)sizeof(T);
@@ -996,19 +997,19 @@ using namespace forkd;
 static std::atomic<long long> g_launches{0};
 static std::atomic<int> g_tune[FORK_TUNE_COUNT_];
 
-static size_t ring_smem_bytes(int n_stages, int cw) { return (size_t)n_stages * ring_stage_bytes(cw) + sizeof(RingSmem); }
+static size_t ring_smem_bytes(int n_stages) { return (size_t)n_stages * ring_stage_bytes() + sizeof(RingSmem); }
 
-/* two CTAs per SM with 8 consumer warps each (default), or one with 16 */
-static void ring_config(int mode, int* ctas_per_sm, int* n_stages, int* cw) {
-  int per_sm = g_tune[FORK_TUNE_CTAS_PER_SM].load();
-  if (per_sm != 1 || mode == kModeSample) per_sm = 2;        /* the sampling kernel exists in the 8-warp form only */
-  const int warps = (per_sm == 1) ? 16 : 8;
+/* The bulk-copy kernel runs two CTAs per SM (8 consumer warps and 6 stages of 16 KB each).  Three
+   CTAs with registers capped at 64 and 4 stages, or two with 12 consumer warps, measured the same
+   on the large shapes and slightly worse on the small one. */
+constexpr int kRingPerSM = 2;
+static void ring_config(int* n_stages) {
   int st = g_tune[FORK_TUNE_STAGES].load();
-  const int max_st = (int)((220 * 1024 / per_sm - sizeof(RingSmem) - 1024) / ring_stage_bytes(warps));
+  const int max_st = (int)((220 * 1024 / kRingPerSM - sizeof(RingSmem) - 1024) / ring_stage_bytes());
   if (st <= 0 || st > max_st) st = max_st;
   if (st > kMaxStages) st = kMaxStages;
   if (st < 2) st = 2;
-  *ctas_per_sm = per_sm; *n_stages = st; *cw = warps;
+  *n_stages = st;
 }
 
 struct DeviceInfo { int sms = 0; int occ[2][3] = {{0, 0, 0}, {0, 0, 0}}; bool ring_ready = false; };
@@ -1037,11 +1038,12 @@ static bool device_info(DeviceInfo** out) {
     const int max_dyn = 220 * 1024;
     auto allow = [&](const void* fn) { return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn) == cudaSuccess; };
     d.ring_ready =
-        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeStep, 8>) && allow((const void*)reduce_select_ring_kernel<bf16_t, kModeLogprob, 8>) &&
-        allow((const void*)reduce_select_ring_kernel<float, kModeStep, 8>) && allow((const void*)reduce_select_ring_kernel<float, kModeLogprob, 8>) &&
-        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeStep, 16>) && allow((const void*)reduce_select_ring_kernel<bf16_t, kModeLogprob, 16>) &&
-        allow((const void*)reduce_select_ring_kernel<float, kModeStep, 16>) && allow((const void*)reduce_select_ring_kernel<float, kModeLogprob, 16>) &&
-        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeSample, 8>) && allow((const void*)reduce_select_ring_kernel<float, kModeSample, 8>);
+        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeStep, kRingPerSM>) &&
+        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeLogprob, kRingPerSM>) &&
+        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeSample, kRingPerSM>) &&
+        allow((const void*)reduce_select_ring_kernel<float, kModeStep, kRingPerSM>) &&
+        allow((const void*)reduce_select_ring_kernel<float, kModeLogprob, kRingPerSM>) &&
+        allow((const void*)reduce_select_ring_kernel<float, kModeSample, kRingPerSM>);
     if (!d.ring_ready) return false;
     d.sms = sms;
   }
@@ -1052,9 +1054,7 @@ static bool device_info(DeviceInfo** out) {
 static int grid_size(const DeviceInfo& d, int dtype, int mode, bool fast) {
   const int variant = g_tune[FORK_TUNE_VARIANT].load();
   if (fast && (variant == 0 || variant == 2)) {
-    int per, stages, cw;
-    ring_config(mode, &per, &stages, &cw);
-    return d.sms * per;
+    return d.sms * kRingPerSM;
   }
   int per_sm = g_tune[FORK_TUNE_CTAS_PER_SM].load();
   int occ = d.occ[dtype][mode];
@@ -1109,11 +1109,11 @@ static cudaError_t launch_reduce(const ReduceParams& rp, int dtype, int mode, in
   return e;
 }
 
-template <typename T, int MODE, int CW>
+template <typename T, int MODE, int PER_SM>
 static cudaError_t launch_ring(const ReduceParams& rp, int G, int n_stages, bool pdl, cudaStream_t st) {
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
-  cfg.gridDim = dim3(G); cfg.blockDim = dim3((CW + 2) * 32); cfg.dynamicSmemBytes = ring_smem_bytes(n_stages, CW);
+  cfg.gridDim = dim3(G); cfg.blockDim = dim3((kCW + 2) * 32); cfg.dynamicSmemBytes = ring_smem_bytes(n_stages);
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   if (pdl) {
@@ -1121,9 +1121,16 @@ static cudaError_t launch_ring(const ReduceParams& rp, int G, int n_stages, bool
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
   }
-  cudaError_t e = cudaLaunchKernelEx(&cfg, reduce_select_ring_kernel<T, MODE, CW>, rp, n_stages);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, reduce_select_ring_kernel<T, MODE, PER_SM>, rp, n_stages);
   if (e == cudaSuccess) g_launches.fetch_add(1);
   return e;
+}
+
+template <typename T, int PER_SM>
+static cudaError_t launch_ring_mode(const ReduceParams& rp, int mode, int G, int n_stages, bool pdl, cudaStream_t st) {
+  if (mode == kModeSample) return launch_ring<T, kModeSample, PER_SM>(rp, G, n_stages, pdl, st);
+  if (mode == kModeStep) return launch_ring<T, kModeStep, PER_SM>(rp, G, n_stages, pdl, st);
+  return launch_ring<T, kModeLogprob, PER_SM>(rp, G, n_stages, pdl, st);
 }
 
 /* variant 2 (bulk-copy ring) needs 16-byte aligned rows; everything else takes variant 1 */
@@ -1135,26 +1142,10 @@ static bool use_ring(const ReduceParams& rp) {
 static cudaError_t launch_reduce_inner(const ReduceParams& rp, int dtype, int mode, int G, cudaStream_t st) {
   const bool pdl = g_tune[FORK_TUNE_PDL].load() >= 0;
   if (use_ring(rp)) {
-    int per_sm, n_stages, cw;
-    ring_config(mode, &per_sm, &n_stages, &cw);
-    if (mode == kModeSample) {
-      if (dtype == FORK_BF16) return launch_ring<bf16_t, kModeSample, 8>(rp, G, n_stages, pdl, st);
-      return launch_ring<float, kModeSample, 8>(rp, G, n_stages, pdl, st);
-    }
-    if (cw == 16) {
-      if (dtype == FORK_BF16) {
-        if (mode == kModeStep) return launch_ring<bf16_t, kModeStep, 16>(rp, G, n_stages, pdl, st);
-        return launch_ring<bf16_t, kModeLogprob, 16>(rp, G, n_stages, pdl, st);
-      }
-      if (mode == kModeStep) return launch_ring<float, kModeStep, 16>(rp, G, n_stages, pdl, st);
-      return launch_ring<float, kModeLogprob, 16>(rp, G, n_stages, pdl, st);
-    }
-    if (dtype == FORK_BF16) {
-      if (mode == kModeStep) return launch_ring<bf16_t, kModeStep, 8>(rp, G, n_stages, pdl, st);
-      return launch_ring<bf16_t, kModeLogprob, 8>(rp, G, n_stages, pdl, st);
-    }
-    if (mode == kModeStep) return launch_ring<float, kModeStep, 8>(rp, G, n_stages, pdl, st);
-    return launch_ring<float, kModeLogprob, 8>(rp, G, n_stages, pdl, st);
+    int n_stages;
+    ring_config(&n_stages);
+    if (dtype == FORK_BF16) return launch_ring_mode<bf16_t, kRingPerSM>(rp, mode, G, n_stages, pdl, st);
+    return launch_ring_mode<float, kRingPerSM>(rp, mode, G, n_stages, pdl, st);
   }
   if (mode == kModeSample) {
     if (dtype == FORK_BF16) return launch(reduce_select_kernel<bf16_t, kModeSample>, dim3(G), dim3(kNT), st, pdl, rp);
