@@ -283,3 +283,93 @@ def test_loop_resumes_from_its_buffers():
     h = st.host()
     for name in h:
         assert h[name].tobytes() == h_full[name].tobytes(), name
+
+
+def test_sampled_full_block_step_at_the_pass_at_k_shape():
+    """The launch the benchmark times with --temperature 0.8 (B=64, every position of a block live):
+    the first two sequences exactly against the oracle (inputs re-drawn until its decisions are
+    clear), every sequence through invariants of the drawn candidates."""
+    from helpers import decisions_are_clear
+    pkg = F()
+    w = fs.workload("passk")
+    BL, tau, seed, nseq = w.block_len, 0.8, 4711, 2
+    cfg_small = w.cfg(B=nseq)
+    lo_h, hi_h = np.zeros(nseq, np.int32), np.full(nseq, BL, np.int32)
+    for nonce in range(16):
+        x = np.empty((nseq, BL, w.V), np.uint16)
+        for b in range(nseq):
+            for l in range(BL):
+                x[b, l] = fs.row_host(cfg_small, 0, b, l, nonce=nonce)
+        o = oracle.StepState(nseq, w.Lt)
+        assert oracle.step(o, x, lo_h, hi_h, w.threshold, step_id=0, temperature=tau, sample_seed=seed) == 0
+        if decisions_are_clear(o, live_mask(np.ones((nseq, w.Lt), np.uint8), lo_h, hi_h), w.threshold, 1e-4, 0, tau):
+            break
+    else:
+        raise AssertionError("no nonce with clear margins")
+    cfg = w.cfg()
+    t = device_logits(w, w.B, Ll=BL)
+    st = pkg.ForkState(w.B, w.Lt)
+    lo = torch.zeros(w.B, dtype=torch.int32, device="cuda")
+    hi = torch.full((w.B,), BL, dtype=torch.int32, device="cuda")
+    fs.cuda_fill(cfg, 0, st.mask.data_ptr(), lo.data_ptr(), hi.data_ptr(), t.data_ptr(), BL * w.V, w.V, 0, BL, nonce=nonce)
+    pkg.fork_step(st, t, lo, hi, w.threshold, step=0, temperature=tau, sample_seed=seed)
+    torch.cuda.synchronize()
+    h = st.host()
+    compare_step_state(h, o, nseq=nseq)
+    conf, logp = h["conf"][:, :BL], h["logp"][:, :BL]
+    assert ((conf > 0) & (conf <= 1.0 + 1e-6)).all()
+    assert (np.abs(np.log(conf) - logp) <= 1e-5 + 1e-4 * np.abs(logp)).all()       # both describe the drawn token
+    committed = h["mask"][:, :BL] == 0
+    assert (h["tokens"][:, :BL][committed] == h["cand"][:, :BL][committed]).all()
+    for b in range(w.B):
+        above = conf[b] > np.float32(w.threshold)
+        want = above if above.any() else (np.arange(BL) == 0)
+        assert (committed[b] == want).all()
+    # a drawn token is not always the arg-max: some candidates differ from the greedy step's
+    st2 = pkg.ForkState(w.B, w.Lt)
+    pkg.fork_step(st2, t, lo, hi, w.threshold, step=0)
+    torch.cuda.synchronize()
+    assert (st2.host()["cand"][:, :BL] != h["cand"][:, :BL]).any()
+
+
+def test_grpo_training_chain_full_size_sampled_rows():
+    """Scoring -> Eq. 2 -> log-softmax backward at B=128, Lt=256, V=126464 fp32 (16.6 GB of logits and
+    as much gradient): the objective on the whole batch, gradients on sampled rows."""
+    pkg = F()
+    w = fs.workload("grpo")
+    cfg = w.cfg()
+    tokens, select = fs.scoring_inputs(w, cfg)
+    t = device_logits(w, w.B)
+    sel_d, tok_d = torch.from_numpy(select).cuda(), torch.from_numpy(tokens).cuda()
+    fs.cuda_fill(cfg, 0, sel_d.data_ptr(), None, None, t.data_ptr(), w.Lt * w.V, w.V, 0, w.Lt)
+    st = pkg.ForkState(w.B, w.Lt)
+    lp, ssum, scnt, status, lse = pkg.fork_logprob(t, tok_d, sel_d, st, want_lse=True)
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    old = ((lp + 0.1 * torch.randn(lp.shape, device="cuda", generator=gen)) * (sel_d != 0)).contiguous()
+    reward = (torch.rand(w.B, device="cuda", generator=gen) < 0.4).float()
+    reward[:8] = 1.0                                              # one prompt group with equal rewards
+    out = pkg.fork_grpo_loss(lp, old, sel_d, reward, 8, 0.2, 0.2)
+    grad = torch.empty_like(t)
+    fs.cuda_canary(grad.data_ptr(), grad.numel(), w.dtype, torch.cuda.current_stream().cuda_stream)
+    pkg.fork_logprob_backward(t, tok_d, sel_d, lse, out["dlogp"], grad, st)
+    torch.cuda.synchronize()
+    o = oracle.grpo_loss(lp.cpu().numpy(), old.cpu().numpy(), select, reward.cpu().numpy(), 8, 0.2, 0.2)
+    rho = o["ratio"][select != 0]
+    near = (np.abs(rho - 0.8) < 1e-4) | (np.abs(rho - 1.2) < 1e-4)
+    d = out["dlogp"].cpu().numpy()
+    ok = np.abs(d - o["dlogp"]) <= 1e-9 + 1e-4 * np.abs(o["dlogp"])
+    assert ok[select != 0][~near].all() and (d[select == 0] == 0).all() and (d[:8] == 0).all()
+    assert abs(float(out["objective"].cpu()[0]) - o["objective"]) <= 1e-6 + 1e-4 * abs(o["objective"])
+    assert o["skipped"][0] == 1 and out["skipped"].cpu().numpy()[0] == 1
+    rng = np.random.default_rng(4)
+    bs, ks = np.nonzero(select[8:])                               # rollouts with a non-zero advantage
+    lse_h = lse.cpu().numpy()
+    for i in rng.choice(len(bs), size=4, replace=False):
+        b, k = int(bs[i]) + 8, int(ks[i])
+        row = fs.row_host(cfg, 0, b, k)
+        assert abs(lse_h[b, k] - oracle.row_lse(row)) <= 1e-5 + 1e-5 * abs(lse_h[b, k])
+        want = oracle.row_logp_grad(row, int(tokens[b, k]), float(d[b, k]))
+        got = grad[b, k].cpu().numpy().astype(np.float64)
+        assert (np.abs(got - want) <= 2e-6 * abs(float(d[b, k])) + 1e-4 * np.abs(want)).all()
+    b, k = map(int, np.argwhere(select == 0)[123])
+    assert torch.isnan(grad[b, k]).all()                          # rows of unselected positions keep the canary
