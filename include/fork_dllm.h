@@ -4,13 +4,21 @@
  * One sampling step of a masked diffusion language model, as Fork-dLLM defines it
  * (Algorithm 2 of the paper; Section 2, "Sampling in masked dLLMs"):
  *   M_t   = still-masked positions (here: mask[b,k] != 0 inside the sequence's active block),
- *   x_0^k = candidate token at temperature 0 = arg-max of the position's distribution,
- *   c_t^k = q_theta^k(x_0^k | x_t) = largest softmax probability of the position's logits,
+ *   x_0^k = candidate token; at temperature 0 the arg-max of the position's distribution,
+ *   c_t^k = q_theta^k(x_0^k | x_t) = its softmax probability (the largest one at temperature 0),
  *   U_t   = {k in M_t : c_t^k > lambda}; if U_t is empty, U_t = {leftmost(M_t)}   (the Fork fallback),
  *   x_{t-1}^k = x_0^k for k in U_t.
  * Besides the commit, the step emits per position the confidence, candidate, token entropy
  * (Section 3.1) and log-probability, and per sequence whether the step was a fallback step
  * (the set F_i of Section 3.2), which is what ForkGRPO scores.
+ *
+ * Entry points: fork_step (one step), fork_decode_loop (steps until nothing is masked),
+ * fork_logprob (log-likelihood scoring of Section 3.2), fork_step_host (host buffers),
+ * fork_step_static (no workspace argument); the variants the paper compares with or trains with:
+ * candidates drawn at temperature tau > 0 and the other fallback orders (fields of fork_step_args),
+ * fork_select_top_entropy (JustGRPO-Fast's position selection), fork_grpo_loss (Eq. 2) and
+ * fork_logprob_backward (its log-softmax backward); fork_vp_reduce / fork_vp_select (the step with
+ * the vocabulary sharded over ranks).
  *
  * Conventions for every entry point
  *   - All data pointers are DEVICE pointers owned by the caller unless a comment says "host".

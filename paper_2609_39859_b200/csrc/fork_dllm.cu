@@ -12,6 +12,13 @@
  *      the leftmost masked position when that set is empty) and writes tokens, mask and records.
  * Cross-CTA hand-over uses "last one to arrive" ticket counters (fence + atomic): nothing in
  * here ever waits for another CTA.
+ *
+ * The same two kernels serve the log-likelihood scoring (Section 3.2), the step with candidates
+ * drawn at a temperature (a third instance of the streaming kernels that also tracks the largest
+ * Gumbel-perturbed key) and the local phase of the vocabulary-parallel step (the finaliser writes
+ * per-position parts instead of applying the rule).  Small kernels of their own: block cursors of the
+ * decode loop, the select phase on gathered parts, top-entropy position selection, the ForkGRPO
+ * objective (Eq. 2) and the log-softmax backward at the scored rows.
  */
 #include <cuda_runtime.h>
 

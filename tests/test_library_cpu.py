@@ -131,3 +131,55 @@ def test_partition_is_a_partition():
     # sizes of the real workloads: no overflow in the 64-bit arithmetic
     U = 32768 * 75
     assert L.fork_debug_part_begin(U, 2048, 2048) == U and L.fork_debug_part_owner(U, 2048, U - 1) == 2047
+
+
+def test_invalid_arguments_of_the_variant_entry_points():
+    """Fallback order / temperature fields, selection, objective, backward and the vocabulary-parallel
+    pair: every bad argument is refused before any CUDA call."""
+    L = pkg.lib()
+    ws, nbytes = C.c_void_p(0x100000), pkg.fork_workspace_bytes(2, 32)
+    INV = pkg.FORK_ERR_INVALID_ARG
+    for field, value in (("fallback_mode", 5), ("fallback_mode", -1), ("fallback_mode", pkg.FORK_FALLBACK_RANDOM),
+                         ("temperature", -0.5), ("temperature", float("nan")), ("temperature", float("inf"))):
+        a = good_step_args()
+        setattr(a, field, value)
+        assert L.fork_step(C.byref(a), ws, nbytes, None) == INV, field
+        assert L.fork_vp_reduce(C.byref(a), 0, C.c_void_p(0x9000), C.c_void_p(0xA000), ws, nbytes, None) == INV, field
+    a = good_step_args()
+    assert L.fork_vp_reduce(C.byref(a), 0, None, None, ws, nbytes, None) == INV              # no output buffer
+    assert L.fork_vp_reduce(C.byref(a), -1, C.c_void_p(0x9000), None, ws, nbytes, None) == INV
+    assert L.fork_vp_reduce(C.byref(a), 0, C.c_void_p(0x9004), None, ws, nbytes, None) == INV  # not 16-byte aligned
+    a.temperature = 0.8
+    assert L.fork_vp_reduce(C.byref(a), 0, C.c_void_p(0x9000), None, ws, nbytes, None) == INV  # keys needed
+    assert L.fork_vp_select(C.byref(a), C.c_void_p(0x9000), None, 2, ws, nbytes, None) == INV
+    a.temperature = 0.0
+    assert L.fork_vp_select(C.byref(a), None, None, 2, ws, nbytes, None) == INV
+    assert L.fork_vp_select(C.byref(a), C.c_void_p(0x9000), None, 0, ws, nbytes, None) == INV
+    assert L.fork_vp_select(C.byref(a), C.c_void_p(0x9000), None, 2, ws, 16, None) == pkg.FORK_ERR_WORKSPACE
+    p = C.c_void_p(0x9000)
+    assert L.fork_select_top_entropy(None, p, 2, 8, 0.2, p, None, None) == INV
+    assert L.fork_select_top_entropy(p, p, 2, 8, 1.5, p, None, None) == INV
+    assert L.fork_select_top_entropy(p, p, 2, 8, -0.1, p, None, None) == INV
+    assert L.fork_select_top_entropy(p, p, 2, 40000, 0.2, p, None, None) == INV
+    assert L.fork_select_top_entropy(p, p, 0, 8, 0.2, p, None, None) == pkg.FORK_OK          # empty batch
+    g = pkg.fork_grpo_args()
+    g.B, g.Lt, g.group = 4, 8, 2
+    g.logp_new = g.logp_old = g.select = g.reward = g.seq_obj = 0x9000
+    g.eps_lo = g.eps_hi = 0.2
+    for field, value in (("group", 3), ("group", 0), ("Lt", 0), ("logp_new", None), ("reward", None), ("seq_obj", None),
+                         ("eps_lo", -1.0), ("eps_hi", float("nan"))):
+        bad = pkg.fork_grpo_args.from_buffer_copy(g)
+        setattr(bad, field, value)
+        assert L.fork_grpo_loss(C.byref(bad), None) == INV, field
+    assert L.fork_grpo_loss(None, None) == INV
+    b = pkg.fork_logprob_bwd_args()
+    b.logits = 0x1000
+    b.stride_b, b.stride_l, b.pos0 = 32 * 1024, 1024, 0
+    b.B, b.Lt, b.Ll, b.V, b.dtype = 2, 32, 32, 1024, pkg.FORK_BF16
+    b.tokens = b.select = b.lse = b.dlogp = b.grad = 0x9000
+    b.grad_stride_b, b.grad_stride_l = 32 * 1024, 1024
+    for field, value in (("grad", None), ("lse", None), ("dlogp", None), ("grad_stride_l", 100), ("V", 0)):
+        bad = pkg.fork_logprob_bwd_args.from_buffer_copy(b)
+        setattr(bad, field, value)
+        assert L.fork_logprob_backward(C.byref(bad), ws, nbytes, None) == INV, field
+    assert L.fork_logprob_backward(C.byref(b), ws, 16, None) == pkg.FORK_ERR_WORKSPACE
