@@ -589,8 +589,9 @@ __device__ void finalize_step_sequence(const ReduceParams& p, const PartitionCtx
     if (p.n_unmasked) p.n_unmasked[b] = count;
     if (p.is_fallback) p.is_fallback[b] = (uint8_t)fb;
     if (p.fallback_pos) p.fallback_pos[b] = pick_k;
-    if (p.nfe) p.nfe[b] += 1;
-    if (p.n_fallback) p.n_fallback[b] += fb;
+    /* reductions without a return value: no load at the very end of the step to wait for */
+    if (p.nfe) atomicAdd(p.nfe + b, 1);
+    if (p.n_fallback && fb) atomicAdd(p.n_fallback + b, 1);
   }
 }
 
