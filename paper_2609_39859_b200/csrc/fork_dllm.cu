@@ -4,8 +4,8 @@
  * A step is two launches on the caller's stream:
  *   1. active_set_kernel (one CTA): M_t restricted to each sequence's block (Algorithm 2, line 3)
  *      compacted into a row list, per-sequence row offsets, and the number of partial results each
- *      sequence will receive.  It snapshots the mask, so the second kernel never reads `mask`
- *      (which it modifies).
+ *      sequence will receive.  The row list is the step's snapshot of the mask: the second kernel
+ *      never reads `mask` (which it modifies).
  *   2. reduce_select_kernel (persistent grid): streams every live row once (lines 4-5: arg-max
  *      candidate and its softmax probability, plus entropy), and the CTA that delivers the last
  *      partial result of a sequence applies the unmask rule for it (lines 6-9: threshold set, or
