@@ -400,6 +400,32 @@ def time_vocab_parallel(device, peak, n_ranks=8):
             "exchange_bytes_per_rank": rows * 16, "note": "slice (%.0f MB) may be L2-resident between repetitions" % (rows * n * w.es / 1e6)}
 
 
+def read_only_ceiling(device):
+    """GB/s of the library's read-only streaming probe on 2 GiB (>> L2), median of 3 runs of 5 launches."""
+    import torch
+    import paper_2609_39859_b200 as pkg
+    buf = torch.empty(2 << 30, dtype=torch.uint8, device=device)
+    buf.zero_()
+    sink = torch.zeros(1, dtype=torch.int32, device=device)
+    L = pkg.lib()
+    st = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    rates = []
+    for i in range(4):                                   # back-to-back launches: no host gap inside the timed region
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n = 5
+        e0.record()
+        for _ in range(n):
+            rc = L.fork_read_probe(C.c_void_p(buf.data_ptr()), buf.numel(), C.c_void_p(sink.data_ptr()), st)
+            assert rc == 0
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= 1:
+            rates.append(n * buf.numel() / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+    del buf
+    torch.cuda.empty_cache()
+    return statistics.median(rates)
+
+
 def time_select(device):
     """JustGRPO-Fast's top-entropy selection at the scoring shape."""
     import torch
@@ -650,6 +676,9 @@ def main():
         also.append(time_select(device))
         also.append(time_vocab_parallel(device, peak))
         out["also"] = also
+        ro = read_only_ceiling(device)
+        out["roofline"]["read_only_ceiling_gbs"] = ro          # the library's own read-only streaming probe, same run
+        out["roofline"]["frac_of_read_only_ceiling"] = kern_gbs / ro
         out["cpu_baseline"] = cpu_baseline(w, seed)
         if args.loops:
             out["loops"] = loop_stats(device)

@@ -303,6 +303,11 @@ fork_status fork_step_host(const fork_step_args* host_args, void* staging, size_
 fork_status fork_select_top_entropy(const float* entropy, const uint8_t* eligible, int32_t B, int32_t Lt,
                                     float ratio, uint8_t* select, int32_t* n_selected, void* stream);
 
+/* Benchmark aid: reads `bytes` of device memory once with the kernels' own streaming loads and does
+   nothing else (buffer 16-byte aligned; sink4 = 4 bytes of device memory).  Its rate is the
+   read-only ceiling that bench.py reports beside the measured copy rate.  Asynchronous. */
+fork_status fork_read_probe(const void* buffer, size_t bytes, void* sink4, void* stream);
+
 /* Copies the device status word of the last call that used `workspace` to *host_out
    (FORK_DEV_* bits) and synchronises `stream`. */
 fork_status fork_device_status(const void* workspace, uint32_t* host_out, void* stream);

@@ -72,7 +72,7 @@ fork_logits_fn = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32, C.c_void_p, C.c_voi
                              C.c_void_p, C.c_void_p)
 
 EXPORTS = ("fork_workspace_bytes", "fork_step", "fork_step_static", "fork_logprob", "fork_decode_loop", "fork_staging_bytes",
-           "fork_select_top_entropy", "fork_grpo_loss", "fork_logprob_backward", "fork_vp_reduce", "fork_vp_select",
+           "fork_select_top_entropy", "fork_grpo_loss", "fork_logprob_backward", "fork_vp_reduce", "fork_vp_select", "fork_read_probe",
            "fork_step_host", "fork_device_status", "fork_status_string", "fork_set_tuning",
            "fork_kernel_launches", "fork_set_timing_events")
 
@@ -128,6 +128,8 @@ def lib():
     L.fork_vp_select.restype = C.c_int
     L.fork_vp_select.argtypes = [C.POINTER(fork_step_args), C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_size_t,
                                  C.c_void_p]
+    L.fork_read_probe.restype = C.c_int
+    L.fork_read_probe.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
     L.fork_set_timing_events.restype = None
     L.fork_set_timing_events.argtypes = [C.c_void_p, C.c_void_p]
     _lib = L

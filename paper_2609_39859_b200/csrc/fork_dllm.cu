@@ -1812,6 +1812,38 @@ extern "C" fork_status fork_step_host(const fork_step_args* h, void* staging, si
   return FORK_OK;
 }
 
+/* ---- read-only streaming probe ---------------------------------------------------------------- */
+/* The rate at which this GPU delivers a buffer that is only read (128-bit streaming loads, a
+   persistent grid, nothing computed but an XOR): the practical ceiling for the reduction kernels,
+   which never write more than a few bytes per row.  The benchmark reports it beside the measured
+   copy rate. */
+__global__ void __launch_bounds__(256, 4) read_probe_kernel(const uint4* __restrict__ p, long long nvec, uint32_t* sink) {
+  /* every CTA reads one contiguous share, like the reduction kernels */
+  const long long per = (nvec + gridDim.x - 1) / gridDim.x;
+  const long long lo = (long long)blockIdx.x * per, hi = (lo + per < nvec) ? lo + per : nvec;
+  uint32_t x = 0;
+  long long i = lo + threadIdx.x;
+  for (; i + 3 * 256 < hi; i += 256 * 4) {
+    uint4 v[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) v[j] = ld_stream(p + i + j * 256);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) x ^= v[j].x ^ v[j].y ^ v[j].z ^ v[j].w;
+  }
+  for (; i < hi; i += 256) { const uint4 v = ld_stream(p + i); x ^= v.x ^ v.y ^ v.z ^ v.w; }
+  if (x == 0x9e3779b9u) *sink = x;                           /* practically never: keeps the loads alive */
+}
+
+extern "C" fork_status fork_read_probe(const void* buffer, size_t bytes, void* sink4, void* stream) {
+  if (!buffer || !sink4 || (reinterpret_cast<uintptr_t>(buffer) & 15u) != 0) return FORK_ERR_INVALID_ARG;
+  DeviceInfo* dev;
+  if (!device_info(&dev)) return FORK_ERR_CUDA;
+  read_probe_kernel<<<dev->sms * 4, 256, 0, (cudaStream_t)stream>>>((const uint4*)buffer, (long long)(bytes / 16), (uint32_t*)sink4);
+  if (cudaGetLastError() != cudaSuccess) return FORK_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return FORK_OK;
+}
+
 /* ---- host-side view of the partition, for tests ------------------------------------------- */
 extern "C" int64_t fork_debug_part_begin(int64_t U, int32_t G, int32_t g) { return fork_part_begin(U, G, g); }
 extern "C" int32_t fork_debug_part_owner(int64_t U, int32_t G, int64_t x) { return fork_part_owner(U, G, x); }

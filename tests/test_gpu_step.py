@@ -312,3 +312,17 @@ def test_step_host_entry_point_matches_device_entry_point():
                nfe=h.nfe, n_fallback=h.n_fallback, conf=conf32, entropy=ent32, logp=lp32, commit_logp=clp32)
     for name in got:
         assert got[name].tobytes() == g[name].tobytes(), name
+
+
+def test_read_probe_runs_and_rejects_bad_arguments():
+    import ctypes as C
+    pkg = F()
+    L = pkg.lib()
+    buf = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    sink = torch.zeros(1, dtype=torch.int32, device="cuda")
+    assert L.fork_read_probe(C.c_void_p(buf.data_ptr()), buf.numel(), C.c_void_p(sink.data_ptr()), None) == 0
+    assert L.fork_read_probe(C.c_void_p(buf.data_ptr()), 1000, C.c_void_p(sink.data_ptr()), None) == 0      # ragged size
+    torch.cuda.synchronize()
+    assert int(sink.cpu()[0]) == 0
+    assert L.fork_read_probe(None, 16, C.c_void_p(sink.data_ptr()), None) == pkg.FORK_ERR_INVALID_ARG
+    assert L.fork_read_probe(C.c_void_p(buf.data_ptr() + 4), 16, C.c_void_p(sink.data_ptr()), None) == pkg.FORK_ERR_INVALID_ARG
