@@ -19,6 +19,11 @@
  * per-position parts instead of applying the rule).  Small kernels of their own: block cursors of the
  * decode loop, the select phase on gathered parts, top-entropy position selection, the ForkGRPO
  * objective (Eq. 2) and the log-softmax backward at the scored rows.
+ *
+ * Files: fork_reduce.cuh (per-thread accumulators, parts, noise stream), fork_partition.h (work
+ * partition), fork_params.cuh (workspace and kernel parameters), fork_setup.cuh (active set, block
+ * cursors), fork_finalize.cuh (merging parts, the unmask rule, scoring, vocabulary-parallel phases),
+ * fork_stream.cuh (the two streaming kernels), this file (host side, the C ABI, the small kernels).
  */
 #include <cuda_runtime.h>
 
@@ -30,972 +35,10 @@
 #include "../../include/fork_dllm.h"
 #include "fork_partition.h"
 #include "fork_reduce.cuh"
-
-namespace forkd {
-
-constexpr int kNT = 256;             /* threads per CTA of the streaming kernel */
-constexpr int kUnroll = 4;           /* 128-bit loads in flight per thread */
-constexpr int kSetupNT = 1024;       /* threads of the one-CTA set-up kernels */
-
-enum Mode { kModeStep = 0, kModeLogprob = 1, kModeSample = 2 };   /* kModeSample: a step with stochastic candidates (tau > 0) */
-__host__ __device__ constexpr bool mode_is_step(int mode) { return mode != kModeLogprob; }
-
-/* ---- workspace ---------------------------------------------------------------------------- */
-struct WsHeader {                    /* 256 bytes at the start of the workspace */
-  int32_t R;                         /* live rows of the current call */
-  int32_t C;                         /* units per row */
-  int32_t G;                         /* grid size the partition was computed for */
-  uint32_t dev_status;               /* FORK_DEV_* bits */
-  int32_t remaining;                 /* decode loop: sequences that still hold a masked position */
-  int32_t pad[59];
-};
-static_assert(sizeof(WsHeader) == 256, "header size");
-
-struct WsView {
-  WsHeader* hdr;
-  int32_t* seq_off;                  /* [B+1] first row of each sequence */
-  int32_t* expected;                 /* [B] parts the sequence will receive */
-  int32_t* ticket;                   /* [B] parts received so far */
-  int32_t* loop_lo;                  /* [B] decode-loop block cursors */
-  int32_t* loop_hi;                  /* [B] */
-  int2* rows;                        /* [B*Lt] (b, k) of each live row, ascending */
-  float4* final_rec;                 /* [B*Lt] per-row results kept between the finaliser's passes */
-  float4* parts;                     /* [B*Lt + FORK_MAX_GRID] partial results, slot r+g */
-  float2* kparts;                    /* [B*Lt + FORK_MAX_GRID] best perturbed key of each part (stochastic candidates) */
-  size_t bytes;
-};
-
-static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
-
-static WsView ws_view(void* base, int32_t B, int32_t Lt) {
-  WsView v;
-  char* p = (char*)base;
-  size_t off = 0;
-  const size_t nb = (size_t)(B > 0 ? B : 1), rows = nb * (size_t)(Lt > 0 ? Lt : 1);
-  v.hdr = (WsHeader*)(p + off); off += sizeof(WsHeader);
-  v.seq_off = (int32_t*)(p + off); off = align_up(off + (nb + 1) * 4, 256);
-  v.expected = (int32_t*)(p + off); off = align_up(off + nb * 4, 256);
-  v.ticket = (int32_t*)(p + off); off = align_up(off + nb * 4, 256);
-  v.loop_lo = (int32_t*)(p + off); off = align_up(off + nb * 4, 256);
-  v.loop_hi = (int32_t*)(p + off); off = align_up(off + nb * 4, 256);
-  v.rows = (int2*)(p + off); off = align_up(off + rows * sizeof(int2), 256);
-  v.final_rec = (float4*)(p + off); off = align_up(off + rows * sizeof(float4), 256);
-  v.parts = (float4*)(p + off); off = align_up(off + (rows + FORK_MAX_GRID) * sizeof(float4), 256);
-  v.kparts = (float2*)(p + off); off = align_up(off + (rows + FORK_MAX_GRID) * sizeof(float2), 256);
-  v.bytes = off;
-  return v;
-}
-
-/* ---- kernel parameters -------------------------------------------------------------------- */
-struct RowSource {                   /* where the logits rows are */
-  const void* logits;
-  long long stride_b, stride_l;
-  int pos0, Ll, V;
-};
-
-struct ReduceParams {
-  RowSource src;
-  int B, Lt, C, fast;
-  /* workspace */
-  const WsHeader* hdr; const int32_t* seq_off; const int32_t* expected; int32_t* ticket;
-  const int2* rows; float4* final_rec; float4* parts; float2* kparts;
-  /* step mode */
-  int32_t* tokens; uint8_t* mask; float threshold; int32_t step;
-  float* conf; int32_t* cand; float* entropy; float* logp; uint32_t* row_status;
-  int32_t* commit_step; uint8_t* commit_fallback; float* commit_logp;
-  int32_t* n_unmasked; uint8_t* is_fallback; int32_t* fallback_pos; int32_t* nfe; int32_t* n_fallback;
-  int fallback_mode; const uint32_t* fallback_rand;
-  float noise_c; unsigned long long sample_seed;      /* stochastic candidates: log2(e)/tau and the noise stream */
-  /* vocabulary-parallel slices */
-  int vocab_offset;                  /* global index of entry 0 of this buffer */
-  float4* vp_part; float4* vp_key;   /* [B,Lt] local phase: per-position results for the exchange instead of the unmask rule */
-  const float4* vp_parts_in; const float4* vp_keys_in; int vp_ranks;   /* select phase: gathered [ranks][B,Lt] */
-  /* log-probability mode */
-  const int32_t* lp_tokens; float* lp_out; float* seq_sum; int32_t* seq_cnt; float* lse_out;
-};
-
-template <typename T>
-__device__ __forceinline__ const T* row_ptr(const RowSource& s, int b, int k) {
-  return reinterpret_cast<const T*>(s.logits) + ((long long)b * s.stride_b + (long long)(k - s.pos0) * s.stride_l);
-}
-
-__device__ __forceinline__ float4 ld_cg_f4(const float4* p) { return __ldcg(p); }
-
-/* ---- the partition as the kernels see it ---------------------------------------------------- */
-struct PartitionCtx {
-  long long U; int G; int C;
-  bool small;                                    /* (U+1)*G < 2^32: 32-bit division is exact */
-  __device__ __forceinline__ int owner(long long x) const {
-    if (small) return (int)((((uint32_t)x + 1u) * (uint32_t)G - 1u) / (uint32_t)U);
-    return fork_part_owner(U, G, x);
-  }
-};
-
-__device__ __forceinline__ PartitionCtx make_partition(int R, int C, int grid) {
-  PartitionCtx c;
-  c.U = (long long)R * C;
-  c.G = fork_effective_grid(c.U, grid);
-  c.C = C;
-  c.small = (unsigned long long)(c.U + 1) * (unsigned long long)c.G < 0xffffffffull;
-  return c;
-}
-
-/* ---- kernel 1: the active set -------------------------------------------------------------- */
-/* One CTA.  live(b,k) = flags[b,k] != 0 and k inside the sequence's window (block bounds clipped
-   to the sequence buffer and to the positions the logits buffer covers). */
-struct SetupParams {
-  const uint8_t* flags;              /* mask (step) or select (log-probability) */
-  const int32_t* lo; const int32_t* hi;   /* NULL: the whole sequence */
-  int B, Lt, pos0, Ll, C, G;
-  WsHeader* hdr; int32_t* seq_off; int32_t* expected; int32_t* ticket; int2* rows;
-  /* outputs for sequences without a live row */
-  int32_t* n_unmasked; uint8_t* is_fallback; int32_t* fallback_pos;   /* step mode */
-  float* seq_sum; int32_t* seq_cnt;                                   /* log-probability mode */
-};
-
-__device__ __forceinline__ void seq_window(const SetupParams& p, int b, int& lo, int& hi, bool& clipped) {
-  int l0 = p.lo ? p.lo[b] : 0, h0 = p.hi ? p.hi[b] : p.Lt;
-  lo = l0; hi = h0;
-  if (lo < 0) lo = 0;
-  if (hi > p.Lt) hi = p.Lt;
-  if (lo < p.pos0) lo = p.pos0;
-  if (hi > p.pos0 + p.Ll) hi = p.pos0 + p.Ll;
-  clipped = (h0 > l0) && (lo != l0 || hi != h0);
-  if (hi < lo) hi = lo;
-}
-
-constexpr int kSetupMaxB = 4096;     /* sequences whose counts fit in shared memory (more: counts go through global memory) */
-
-__global__ void __launch_bounds__(kSetupNT, 1) active_set_kernel(SetupParams p) {
-  /* with programmatic dependent launch this grid may already be resident while the kernel before
-     it in the stream (normally the previous step) is still running: nothing is read or written
-     before that kernel has completed; the streaming kernel of this step may be made resident now */
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  asm volatile("griddepcontrol.launch_dependents;");
-  __shared__ int sh_cnt[kSetupMaxB + 1];          /* sh_cnt[b+1] = live rows of b, then their inclusive scan */
-  __shared__ int sh_warp[kSetupNT / 32];
-  __shared__ int sh_carry;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = kSetupNT / 32;
-  int* cnt = (p.B <= kSetupMaxB) ? sh_cnt : p.seq_off;       /* cnt[0..B] */
-  unsigned clipped_any = 0;
-
-  /* pass 1: live rows per sequence */
-  for (int b = warp; b < p.B; b += nwarp) {
-    int lo, hi; bool clipped;
-    seq_window(p, b, lo, hi, clipped);
-    clipped_any |= clipped ? 1u : 0u;
-    int n = 0;
-    for (int k0 = lo; k0 < hi; k0 += 32) {
-      int k = k0 + lane;
-      bool live = (k < hi) && p.flags[(size_t)b * p.Lt + k] != 0;
-      n += __popc(__ballot_sync(0xffffffffu, live));
-    }
-    if (lane == 0) { cnt[b + 1] = n; p.ticket[b] = 0; }
-  }
-  if (tid == 0) { cnt[0] = 0; sh_carry = 0; }
-  __syncthreads();
-
-  /* pass 2: inclusive scan of the counts, kSetupNT sequences at a time */
-  for (int base = 0; base < p.B; base += kSetupNT) {
-    int b = base + tid;
-    int x = (b < p.B) ? cnt[b + 1] : 0;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) { int y = __shfl_up_sync(0xffffffffu, x, o); if (lane >= o) x += y; }
-    if (lane == 31) sh_warp[warp] = x;
-    __syncthreads();
-    if (warp == 0) {
-      int w = sh_warp[lane];
-      int xs = w;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) { int y = __shfl_up_sync(0xffffffffu, xs, o); if (lane >= o) xs += y; }
-      sh_warp[lane] = xs - w;                       /* exclusive prefix of the warp totals */
-    }
-    __syncthreads();
-    int incl = sh_carry + sh_warp[warp] + x;
-    if (b < p.B) cnt[b + 1] = incl;
-    __syncthreads();
-    if (tid == kSetupNT - 1) sh_carry = incl;
-    __syncthreads();
-  }
-  const int R = sh_carry;
-  const PartitionCtx c = make_partition(R, p.C, p.G);
-  if (tid == 0) {
-    p.hdr->R = R; p.hdr->C = p.C; p.hdr->G = c.G;
-  }
-
-  /* pass 3: row list, expected part counts, outputs of idle sequences */
-  for (int b = warp; b < p.B; b += nwarp) {
-    int lo, hi; bool clipped;
-    seq_window(p, b, lo, hi, clipped);
-    const int r0 = cnt[b], r1 = cnt[b + 1];
-    int run = r0;
-    for (int k0 = lo; k0 < hi; k0 += 32) {
-      int k = k0 + lane;
-      bool live = (k < hi) && p.flags[(size_t)b * p.Lt + k] != 0;
-      unsigned bal = __ballot_sync(0xffffffffu, live);
-      if (live) p.rows[run + __popc(bal & ((1u << lane) - 1u))] = make_int2(b, k);
-      run += __popc(bal);
-    }
-    int parts = 0;
-    for (int r = r0 + lane; r < r1; r += 32)
-      parts += c.owner((long long)(r + 1) * c.C - 1) - c.owner((long long)r * c.C) + 1;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) parts += __shfl_down_sync(0xffffffffu, parts, o);
-    if (lane == 0) {
-      p.expected[b] = parts;
-      if (cnt == sh_cnt) { p.seq_off[b + 1] = r1; if (b == 0) p.seq_off[0] = 0; }
-      if (r0 == r1) {
-        if (p.n_unmasked) p.n_unmasked[b] = 0;
-        if (p.is_fallback) p.is_fallback[b] = 0;
-        if (p.fallback_pos) p.fallback_pos[b] = -1;
-        if (p.seq_sum) p.seq_sum[b] = 0.f;
-        if (p.seq_cnt) p.seq_cnt[b] = 0;
-      }
-    }
-  }
-  clipped_any = __syncthreads_or((int)clipped_any);
-  if (tid == 0) p.hdr->dev_status = clipped_any ? FORK_DEV_WINDOW_CLAMPED : 0u;
-}
-
-/* ---- shared by both streaming kernels: merging parts, the unmask rule, scoring ------------- */
-__device__ __forceinline__ Part part_from(const float4& v) { return Part{v.x, v.y, v.z, __float_as_int(v.w)}; }
-
-constexpr int kLaneMergeMax = 24;
-/* Parts of row r, by one lane, loaded four at a time and merged in ascending CTA order.  `n`
-   returns how many parts the row has; rows with more than kLaneMergeMax (very few live rows, the
-   whole grid on them) are merged by merge_row_parts_warp instead. */
-__device__ __forceinline__ Part merge_row_parts(const ReduceParams& p, const PartitionCtx& c, int r, int& g0, int& n) {
-  g0 = c.owner((long long)r * c.C);
-  const int g1 = c.owner((long long)(r + 1) * c.C - 1);
-  n = g1 - g0 + 1;
-  const float4* q = p.parts + (r + g0);
-  const float4 v0 = ld_cg_f4(q);
-  float4 v1 = v0, v2 = v0, v3 = v0;
-  if (n > 1) v1 = ld_cg_f4(q + 1);
-  if (n > 2) v2 = ld_cg_f4(q + 2);
-  if (n > 3) v3 = ld_cg_f4(q + 3);
-  Part acc = part_from(v0);
-  if (n > 1) acc = part_merge(acc, part_from(v1));
-  if (n > 2) acc = part_merge(acc, part_from(v2));
-  if (n > 3) acc = part_merge(acc, part_from(v3));
-  if (n <= kLaneMergeMax) {                                  /* a moderate number: this lane goes on, four loads at a time */
-    for (int j = 4; j < n; j += 4) {
-      const float4 w0 = ld_cg_f4(q + j);
-      float4 w1 = w0, w2 = w0, w3 = w0;
-      if (j + 1 < n) w1 = ld_cg_f4(q + j + 1);
-      if (j + 2 < n) w2 = ld_cg_f4(q + j + 2);
-      if (j + 3 < n) w3 = ld_cg_f4(q + j + 3);
-      acc = part_merge(acc, part_from(w0));
-      if (j + 1 < n) acc = part_merge(acc, part_from(w1));
-      if (j + 2 < n) acc = part_merge(acc, part_from(w2));
-      if (j + 3 < n) acc = part_merge(acc, part_from(w3));
-    }
-  }
-  return acc;
-}
-
-/* A row cut into many parts (few live rows, many CTAs): the whole warp loads 32 parts at a time
-   and tree-merges them; every lane returns the same Part. */
-__device__ __forceinline__ Part merge_row_parts_warp(const ReduceParams& p, int r, int g0, int n) {
-  const int lane = threadIdx.x & 31;
-  const float4* q = p.parts + (r + g0);
-  Part acc = part_empty();
-  for (int j0 = 0; j0 < n; j0 += 32) {
-    Part x = (j0 + lane < n) ? part_from(ld_cg_f4(q + j0 + lane)) : part_empty();
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      Part y;
-      y.m = __shfl_xor_sync(0xffffffffu, x.m, o); y.s = __shfl_xor_sync(0xffffffffu, x.s, o);
-      y.t = __shfl_xor_sync(0xffffffffu, x.t, o); y.idx = __shfl_xor_sync(0xffffffffu, x.idx, o);
-      const bool low = (lane & o) == 0;                      /* both partners compute merge(lower, upper) */
-      x = low ? part_merge(x, y) : part_merge(y, x);
-    }
-    acc = part_merge(acc, x);
-  }
-  return acc;
-}
-
-/* Guarded scalar reduction of a whole row by ONE warp (every lane returns the same Part). */
-template <typename T>
-__device__ Part careful_row_warp(const T* row, int V, bool& bad, bool* nonfinite = nullptr) {
-  const int lane = threadIdx.x & 31;
-  float m = -INFINITY;
-  int idx = -1, isbad = 0;
-  for (int i = lane; i < V; i += 32) {
-    const float x = to_f32(row[i]);
-    if (x != x) { isbad = 1; continue; }
-    if (x == INFINITY) isbad = 1;
-    if (idx < 0 || x > m) { m = x; idx = i; }
-  }
-  if (idx < 0) idx = kIdxNone;
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const float om = __shfl_xor_sync(0xffffffffu, m, o);
-    const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
-    const bool take = (oi != kIdxNone) && (idx == kIdxNone || om > m || (om == m && oi < idx));
-    if (take) { m = om; idx = oi; }
-  }
-  isbad = __any_sync(0xffffffffu, isbad);
-  if (nonfinite) *nonfinite = isbad != 0;                    /* NaN or +inf seen (as opposed to nothing but -inf) */
-  if (isbad || idx == kIdxNone || m == -INFINITY) {
-    bad = true;
-    return Part{m, __int_as_float(0x7fc00000), __int_as_float(0x7fc00000), idx == kIdxNone ? 0 : idx};
-  }
-  bad = false;
-  float s = 0.f, t = 0.f;
-  for (int i = lane; i < V; i += 32) {
-    const float x = to_f32(row[i]);
-    if (x == -INFINITY) continue;
-    const float y = (x - m) * kLog2e;
-    const float e = exp2f(y);
-    s += e;
-    if (e > 0.f) t = fmaf(y, e, t);
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) { s += __shfl_xor_sync(0xffffffffu, s, o); t += __shfl_xor_sync(0xffffffffu, t, o); }
-  return Part{m, s, t, idx};
-}
-
-__device__ __forceinline__ KeyPart key_from(const float2& v) { return KeyPart{v.x, __float_as_int(v.y)}; }
-
-/* Largest perturbed key of row r over its n parts (slots r+g0 ...), by one lane. */
-__device__ __forceinline__ KeyPart merge_row_keys(const ReduceParams& p, int r, int g0, int n) {
-  const float2* q = p.kparts + (r + g0);
-  KeyPart acc = key_empty();
-#pragma unroll 4
-  for (int j = 0; j < n; ++j) acc = key_merge(acc, key_from(__ldcg(q + j)));
-  return acc;
-}
-
-/* Final statistics of up to 32 rows (one per lane) of sequence b starting at row `base`.
-   Rows whose streamed result is not finite are re-read by the whole warp with the guarded routine.
-   With SAMPLE the candidate is the drawn token (the element holding the row's largest perturbed
-   key) and confidence / log-probability are those of that token; flagged rows keep the arg-max. */
-/* Rows base .. base+31 of sequence b, one per lane: the row's parts merged, rows whose streamed
-   result is not finite re-read by the whole warp with the guarded routine. */
-struct MergedRow {
-  Part merged; int k, g0, nparts; bool valid, bad, nonfinite;
-};
-template <typename T>
-__device__ __forceinline__ MergedRow merge_rows_warp(const ReduceParams& p, const PartitionCtx& c, int b, int base, int r1,
-                                                     int k_hint) {
-  const int lane = threadIdx.x & 31;
-  const int r = base + lane;
-  MergedRow m;
-  m.valid = r < r1; m.bad = false; m.nonfinite = false;
-  m.merged = part_empty();
-  m.k = 0; m.g0 = 0; m.nparts = 0;
-  bool redo = false;
-  if (m.valid) { m.k = (k_hint >= 0) ? k_hint : p.rows[r].y; m.merged = merge_row_parts(p, c, r, m.g0, m.nparts); }
-  unsigned many = __ballot_sync(0xffffffffu, m.valid && m.nparts > kLaneMergeMax);
-  while (many) {                                             /* rows cut into very many parts: all lanes help */
-    const int src = __ffs(many) - 1;
-    many &= many - 1;
-    const Part w = merge_row_parts_warp(p, __shfl_sync(0xffffffffu, r, src), __shfl_sync(0xffffffffu, m.g0, src),
-                                        __shfl_sync(0xffffffffu, m.nparts, src));
-    if (lane == src) m.merged = w;
-  }
-  if (m.valid) redo = part_needs_careful(m.merged);
-  unsigned todo = __ballot_sync(0xffffffffu, m.valid && redo);
-  while (todo) {
-    const int src = __ffs(todo) - 1;
-    todo &= todo - 1;
-    const int kk = __shfl_sync(0xffffffffu, m.k, src);
-    bool bd, nf;
-    const Part cp = careful_row_warp<T>(row_ptr<T>(p.src, b, kk), p.src.V, bd, &nf);
-    if (lane == src) { m.merged = cp; m.bad = bd; m.nonfinite = nf; }
-  }
-  return m;
-}
-
-template <typename T, bool WANT_INDEX, bool SAMPLE>
-__device__ __forceinline__ RowOut finalize_rows_warp(const ReduceParams& p, const PartitionCtx& c, int b, int base,
-                                                     int r1, Part& merged, int& k, int k_hint) {
-  const int lane = threadIdx.x & 31;
-  const int r = base + lane;
-  MergedRow m = merge_rows_warp<T>(p, c, b, base, r1, k_hint);
-  k = m.k;
-  if (SAMPLE) {
-    float xs = 0.f;
-    if (m.valid && !m.bad) {
-      const KeyPart kp = merge_row_keys(p, r, m.g0, m.nparts);
-      const NoiseRow nz = noise_row(p.sample_seed, p.step, b, k, p.noise_c, (uint32_t)p.vocab_offset);
-      m.merged.idx = resolve_sample<T>(row_ptr<T>(p.src, b, k), nz, kp.vec, p.src.V, kp.key, xs);
-    }
-    merged = m.merged;
-    return row_out_sampled(merged, m.bad, xs);
-  }
-  if (m.valid && WANT_INDEX && !m.bad) m.merged.idx = resolve_index<T>(row_ptr<T>(p.src, b, k), m.merged.idx, p.src.V, m.merged.m);
-  merged = m.merged;
-  return row_out_from(merged, m.bad);
-}
-
-/* What a finaliser can load about a sequence BEFORE its last part arrives (it idles until then):
-   the sequence's row range and this lane's position among its first 32 rows. */
-struct SeqHint { int r0, r1, k; };
-__device__ __forceinline__ SeqHint load_seq_hint(const ReduceParams& p, int b) {
-  SeqHint h;
-  h.r0 = p.seq_off[b]; h.r1 = p.seq_off[b + 1];
-  const int r = h.r0 + (int)(threadIdx.x & 31);
-  h.k = (r < h.r1) ? p.rows[r].y : -1;
-  return h;
-}
-
-/* ---- vocabulary-parallel slices ------------------------------------------------------------- */
-/* Local phase: what this slice contributes to every live row of sequence b, written per position
-   for the exchange: (m, s, t2, global index of the lowest arg-max), s = NaN when the slice holds
-   NaN or +inf, the neutral element (m = -inf, s = t2 = 0) when it holds nothing but -inf; with
-   stochastic candidates also (largest perturbed key, global index of its entry, that logit). */
-template <typename T, bool SAMPLE>
-__device__ void finalize_vp_local(const ReduceParams& p, const PartitionCtx& c, int b, const SeqHint& h) {
-  const int lane = threadIdx.x & 31;
-  const float qnan = __int_as_float(0x7fc00000);
-  for (int base = h.r0; base < h.r1; base += 32) {
-    const int r = base + lane;
-    MergedRow m = merge_rows_warp<T>(p, c, b, base, h.r1, base == h.r0 ? h.k : -1);
-    if (!m.valid) continue;
-    const size_t at = (size_t)b * p.Lt + m.k;
-    const T* row = row_ptr<T>(p.src, b, m.k);
-    float4 out, kout = make_float4(-INFINITY, __int_as_float(kIdxNone), 0.f, 0.f);
-    if (m.bad && !m.nonfinite) {
-      out = make_float4(-INFINITY, 0.f, 0.f, __int_as_float(p.vocab_offset));
-    } else if (m.bad) {
-      out = make_float4(m.merged.m, qnan, qnan, __int_as_float(p.vocab_offset + m.merged.idx));
-    } else {
-      const int idx = resolve_index<T>(row, m.merged.idx, p.src.V, m.merged.m);
-      out = make_float4(m.merged.m, m.merged.s, m.merged.t, __int_as_float(p.vocab_offset + idx));
-      if (SAMPLE) {
-        const KeyPart kp = merge_row_keys(p, r, m.g0, m.nparts);
-        const NoiseRow nz = noise_row(p.sample_seed, p.step, b, m.k, p.noise_c, (uint32_t)p.vocab_offset);
-        float xs;
-        const int si = resolve_sample<T>(row, nz, kp.vec, p.src.V, kp.key, xs);
-        kout = make_float4(kp.key, __int_as_float(p.vocab_offset + si), xs, 0.f);
-      }
-    }
-    p.vp_part[at] = out;
-    if (SAMPLE) p.vp_key[at] = kout;
-  }
-}
-
-/* Select phase: the statistics of rows base .. base+31 of sequence b from the gathered slices,
-   merged in rank order (ascending vocabulary offset; ties keep the lowest global index). */
-template <bool SAMPLE>
-__device__ __forceinline__ RowOut gathered_rows_warp(const ReduceParams& p, int b, int base, int r1, int& k, int k_hint) {
-  const int lane = threadIdx.x & 31;
-  const int r = base + lane;
-  k = 0;
-  if (r >= r1) return row_out_from(part_empty(), true);
-  k = (k_hint >= 0) ? k_hint : p.rows[r].y;
-  const size_t at = (size_t)b * p.Lt + k, n = (size_t)p.B * p.Lt;
-  Part acc = part_empty();
-  for (int j = 0; j < p.vp_ranks; ++j) acc = part_merge(acc, part_from(__ldg(p.vp_parts_in + j * n + at)));
-  const bool bad = !(isfinite(acc.s) && isfinite(acc.t)) || !(acc.m > -INFINITY) || acc.m == INFINITY;
-  if (!SAMPLE || bad) return row_out_from(acc, bad);
-  float best = -INFINITY, xs = 0.f;
-  int bidx = kIdxNone;
-  for (int j = 0; j < p.vp_ranks; ++j) {
-    const float4 q = __ldg(p.vp_keys_in + j * n + at);
-    const int qi = __float_as_int(q.y);
-    if (q.x > best || (q.x == best && qi < bidx)) { best = q.x; bidx = qi; xs = q.z; }
-  }
-  acc.idx = bidx;
-  return row_out_sampled(acc, false, xs);
-}
-
-/* Key by which a fallback step ranks a row under the orders other than "leftmost" (the largest key
-   wins, equal keys go to the lower row): the confidence (Algorithm 1), its negative, or the token
-   entropy (the ablations of Section 4.1).  Flagged rows rank below every other row. */
-__device__ __forceinline__ float fallback_key(int mode, float conf, float entropy, bool bad) {
-  if (bad) return -INFINITY;
-  return mode == FORK_FALLBACK_MAX_CONF ? conf : (mode == FORK_FALLBACK_MIN_CONF ? -conf : entropy);
-}
-
-/* The unmask rule for one sequence, run by one warp once every part of the sequence has arrived
-   (Algorithm 2 lines 6-9): commit every live position whose confidence exceeds lambda, or one
-   position when none does -- the leftmost live one (Fork-dLLM), or the one the requested
-   comparison order picks; write tokens, mask and the per-token records. */
-template <typename T, bool SAMPLE, bool GATHERED = false>
-__device__ void finalize_step_sequence(const ReduceParams& p, const PartitionCtx& c, int b, const SeqHint& h) {
-  const int lane = threadIdx.x & 31;
-  const int r0 = h.r0, r1 = h.r1;
-  const bool one_batch = (r1 - r0) <= 32;                    /* the usual case: results stay in registers */
-  const bool ranked = p.fallback_mode >= FORK_FALLBACK_MAX_CONF && p.fallback_mode <= FORK_FALLBACK_MAX_ENTROPY;
-  int any = 0;
-  float4 keep = make_float4(0.f, 0.f, 0.f, 0.f);
-  int keep_k = 0;
-  float best_key = -INFINITY;                                /* this lane's best row under a ranked order */
-  int best_r = 0x7fffffff;
-  for (int base = r0; base < r1; base += 32) {
-    Part merged; int k;
-    const RowOut o = GATHERED ? gathered_rows_warp<SAMPLE>(p, b, base, r1, k, base == r0 ? h.k : -1)
-                              : finalize_rows_warp<T, true, SAMPLE>(p, c, b, base, r1, merged, k, base == r0 ? h.k : -1);
-    const int r = base + lane;
-    if (r < r1) {
-      const size_t at = (size_t)b * p.Lt + k;
-      if (p.conf) p.conf[at] = o.conf;
-      if (p.cand) p.cand[at] = o.cand;
-      if (p.entropy) p.entropy[at] = o.entropy;
-      if (p.logp) p.logp[at] = o.logp;
-      if (p.row_status) p.row_status[at] = o.status;
-      keep = make_float4(o.conf, o.logp, __int_as_float(o.cand), 0.f);
-      keep_k = k;
-      if (!one_batch) p.final_rec[r] = keep;
-      any |= (o.conf > p.threshold) ? 1 : 0;                 /* U_t non-empty (Algorithm 2, line 6) */
-      if (ranked) {
-        const float key = fallback_key(p.fallback_mode, o.conf, o.entropy, o.status != 0u);
-        if (key > best_key) { best_key = key; best_r = r; }  /* rows ascend within a lane: strict > keeps the lower */
-      }
-    }
-  }
-  any = __any_sync(0xffffffffu, any);
-  const int fb = any ? 0 : 1;                                /* fallback step: max_k c <= lambda */
-  int pick = r0;                                             /* leftmost(M_t) inside the block */
-  if (fb && ranked) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float ok = __shfl_xor_sync(0xffffffffu, best_key, o);
-      const int orow = __shfl_xor_sync(0xffffffffu, best_r, o);
-      if (ok > best_key || (ok == best_key && orow < best_r)) { best_key = ok; best_r = orow; }
-    }
-    if (best_key > -INFINITY) pick = best_r;                 /* every row flagged: stay with the leftmost */
-  } else if (fb && p.fallback_mode == FORK_FALLBACK_RANDOM) {
-    pick = r0 + (int)(p.fallback_rand[b] % (uint32_t)(r1 - r0));
-  }
-  int count = 0, pick_k = -1;
-  for (int base = r0; base < r1; base += 32) {
-    const int r = base + lane;
-    bool commit = false;
-    if (r < r1) {
-      const float4 f = one_batch ? keep : p.final_rec[r];    /* written by this same lane above */
-      commit = fb ? (r == pick) : (f.x > p.threshold);       /* the fallback position, or the threshold set */
-      if (commit) {
-        const int k = one_batch ? keep_k : p.rows[r].y;
-        const size_t at = (size_t)b * p.Lt + k;
-        if (fb) pick_k = k;
-        p.tokens[at] = __float_as_int(f.z);
-        p.mask[at] = 0;
-        if (p.commit_step) p.commit_step[at] = p.step;
-        if (p.commit_fallback) p.commit_fallback[at] = (uint8_t)fb;
-        if (p.commit_logp) p.commit_logp[at] = f.y;
-      }
-    }
-    count += __popc(__ballot_sync(0xffffffffu, commit));
-  }
-  if (fb) {                                                  /* exactly one lane committed: tell lane 0 where */
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) pick_k = max(pick_k, __shfl_xor_sync(0xffffffffu, pick_k, o));
-  }
-  if (lane == 0) {
-    if (p.n_unmasked) p.n_unmasked[b] = count;
-    if (p.is_fallback) p.is_fallback[b] = (uint8_t)fb;
-    if (p.fallback_pos) p.fallback_pos[b] = pick_k;
-    /* reductions without a return value: no load at the very end of the step to wait for */
-    if (p.nfe) atomicAdd(p.nfe + b, 1);
-    if (p.n_fallback && fb) atomicAdd(p.n_fallback + b, 1);
-  }
-}
-
-/* Scoring for one sequence by one warp: log q(token) = x_tok - m - ln s at every selected position
-   and their sum (Section 3.2 of the paper: the likelihood terms of the ForkGRPO ratio). */
-template <typename T>
-__device__ void finalize_logprob_sequence(const ReduceParams& p, const PartitionCtx& c, int b, const SeqHint& h) {
-  const int lane = threadIdx.x & 31;
-  const int r0 = h.r0, r1 = h.r1;
-  float local = 0.f;
-  for (int base = r0; base < r1; base += 32) {
-    Part merged; int k;
-    const RowOut o = finalize_rows_warp<T, false, false>(p, c, b, base, r1, merged, k, base == r0 ? h.k : -1);
-    const int r = base + lane;
-    if (r < r1) {
-      const size_t at = (size_t)b * p.Lt + k;
-      const int tok = p.lp_tokens[at];
-      uint32_t st = o.status;
-      float lp;
-      if (tok < 0 || tok >= p.src.V) { st |= FORK_ROW_BAD_TOKEN; lp = 0.f; }
-      else if (o.status) lp = o.logp;                        /* NaN for a non-finite row */
-      else lp = (to_f32(row_ptr<T>(p.src, b, k)[tok]) - merged.m) + o.logp;   /* x_tok - m - ln s */
-      p.lp_out[at] = lp;
-      if (p.lse_out) p.lse_out[at] = o.status ? o.logp : merged.m - o.logp;   /* m + ln s; NaN for a flagged row */
-      if (p.row_status) p.row_status[at] = st;
-      local += lp;
-    }
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) local += __shfl_xor_sync(0xffffffffu, local, o);
-  if (lane == 0) {
-    if (p.seq_sum) p.seq_sum[b] = local;
-    if (p.seq_cnt) p.seq_cnt[b] = r1 - r0;
-  }
-}
-
-/* Lane 0 of the calling warp publishes one part of row r (sequence b) and takes a ticket; returns
-   (to every lane) whether this was the last part the sequence was waiting for. */
-__device__ __forceinline__ bool publish_part(const ReduceParams& p, const Part& part, int r, int g, int b, int want,
-                                             const KeyPart* kp = nullptr) {
-  int last = 0;
-  if ((threadIdx.x & 31) == 0) {
-    p.parts[r + g] = make_float4(part.m, part.s, part.t, __int_as_float(part.idx));
-    if (kp) p.kparts[r + g] = make_float2(kp->key, __int_as_float(kp->vec));
-    int old;                                 /* release our part, acquire everybody else's */
-    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(p.ticket + b) : "memory");
-    last = (old + 1 == want) ? 1 : 0;
-  }
-  return __shfl_sync(0xffffffffu, last, 0) != 0;
-}
-
-/* The rows a CTA works on: its contiguous unit range cut at row boundaries. */
-struct Segment { int r, e0, e1; };
-struct SegmentIter {
-  long long u, u1; int C, V;
-  __device__ __forceinline__ void init(const PartitionCtx& c, int g, int V_) {
-    u = fork_part_begin(c.U, c.G, g); u1 = fork_part_begin(c.U, c.G, g + 1); C = c.C; V = V_;
-  }
-  __device__ __forceinline__ bool next(Segment& s) {
-    if (u >= u1) return false;
-    s.r = (u < 0x7fffffffLL) ? (int)((uint32_t)u / (uint32_t)C) : (int)(u / C);
-    const int c0 = (int)(u - (long long)s.r * C);
-    long long uend = (long long)(s.r + 1) * C;
-    if (uend > u1) uend = u1;
-    const int c1 = (int)(uend - (long long)s.r * C);
-    s.e0 = c0 * FORK_CHUNK;
-    s.e1 = c1 * FORK_CHUNK;
-    if (s.e1 > V) s.e1 = V;
-    u = uend;
-    return true;
-  }
-};
-
-/* ---- kernel 2a: direct 128-bit loads (also the path for buffers that are not 16-byte aligned) -- */
-struct Smem {
-  Part parts[kNT / 32];
-  KeyPart keys[kNT / 32];
-  float fl[kNT / 32];
-  int flag;
-};
-
-template <typename T, int MODE>
-__global__ void __launch_bounds__(kNT, 4) reduce_select_kernel(ReduceParams p) {
-  constexpr bool WITH_T = mode_is_step(MODE);
-  constexpr bool SAMPLE = (MODE == kModeSample);
-  __shared__ Smem sm;
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  asm volatile("griddepcontrol.launch_dependents;");
-  const int R = p.hdr->R;
-  if (R <= 0) return;
-  const PartitionCtx c = make_partition(R, p.C, (int)gridDim.x);
-  const int g = blockIdx.x;
-  if (g >= c.G) return;                                     /* CTAs beyond the number of units have no work */
-  SegmentIter it;
-  it.init(c, g, p.src.V);
-  Segment sg;
-  bool sticky = false;
-  while (it.next(sg)) {
-    const int2 bk = p.rows[sg.r];
-    const T* row = row_ptr<T>(p.src, bk.x, bk.y);
-    Part part;
-    KeyTrack kt;
-    kt.init();
-    NoiseRow nz = NoiseRow{0u, 0u, 0.f, 0u};
-    if (SAMPLE) nz = noise_row(p.sample_seed, p.step, bk.x, bk.y, p.noise_c, (uint32_t)p.vocab_offset);
-    if (p.fast) {
-      part = part_block_reduce<kNT>(
-          stream_thread<T, WITH_T, kNT, kUnroll, SAMPLE>(row, sg.e0, sg.e1, threadIdx.x, threadIdx.x == 0, sticky, &kt, &nz),
-          sm.parts);
-    } else {
-      bool bad;
-      part = careful_segment<T, kNT>(row, sg.e0, sg.e1, sm.parts, sm.fl, bad);
-      if (SAMPLE)
-        for (int i = sg.e0 + (int)threadIdx.x; i < sg.e1; i += kNT) kt.one(nz, to_f32(row[i]), i);
-    }
-    KeyPart kp = key_empty();
-    if (SAMPLE) kp = key_block_reduce<kNT>(kt.best, sm.keys);
-    if (threadIdx.x < 32) {
-      const bool last = publish_part(p, part, sg.r, g, bk.x, p.expected[bk.x], SAMPLE ? &kp : nullptr);
-      if (last) {                                           /* every part of sequence b has been delivered */
-        const SeqHint h = load_seq_hint(p, bk.x);
-        if (MODE == kModeLogprob) finalize_logprob_sequence<T>(p, c, bk.x, h);
-        else if (p.vp_part) finalize_vp_local<T, SAMPLE>(p, c, bk.x, h);
-        else finalize_step_sequence<T, SAMPLE>(p, c, bk.x, h);
-      }
-    }
-  }
-}
-
-/* ---- kernel 2b: bulk-copy (TMA) shared-memory ring, warp-specialised --------------------------
- * Warps 0..kCW-1 consume, warp kCW produces, warp kCW+1 finalises.
- *   producer : one lane walks the CTA's segments and issues cp.async.bulk copies of up to one stage
- *              (kStageBytes) into a ring of shared-memory stages, each guarded by a full/empty
- *              mbarrier pair; it runs ahead of the consumers by the depth of the ring, across row
- *              boundaries, so HBM requests never drain while rows are being wrapped up.
- *   consumers: wait for a stage, read their 128-bit vectors from shared memory, accumulate, release
- *              the stage; at the end of a row segment each warp shuffle-reduces its threads' Parts
- *              and hands ONE Part to the finaliser through a small mbarrier-guarded mailbox, then
- *              goes straight on to the next segment.
- *   finaliser: merges the kCW warp Parts, publishes the CTA's part of the row, takes the sequence's
- *              ticket and, if it was the last, applies the unmask rule for that sequence.
- * Every mbarrier wait is bounded: after kSpinLimit failed polls the thread records
- * FORK_DEV_TIMEOUT in the workspace header and leaves its loop.                                   */
-constexpr int kCW = 8;                                     /* consumer warps per CTA */
-constexpr int kMaxCW = kCW;
-constexpr int kMail = 4;                                   /* mailbox depth (row segments in flight to the finaliser) */
-constexpr int kMaxStages = 13;
-constexpr uint32_t kSpinLimit = 1u << 22;
-constexpr int ring_stage_bytes() { return kCW * 32 * kUnroll * 16; }     /* 16 KB */
-
-struct RingSmem {
-  unsigned long long full[kMaxStages], empty[kMaxStages], mfull[kMail], mempty[kMail];
-  Part mail[kMail][kMaxCW];
-  KeyPart kmail[kMail][kMaxCW];
-};
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-               : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
-}
-/* bounded wait; false (and a status bit in the workspace header) if the phase never completed */
-__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity, const ReduceParams& p) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
-  atomicOr(const_cast<uint32_t*>(&p.hdr->dev_status), FORK_DEV_TIMEOUT);
-  return false;
-}
-__device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               :: "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
-}
-
-
-template <typename T, int MODE, int kPerSM>
-__global__ void __launch_bounds__((kCW + 2) * 32, kPerSM) reduce_select_ring_kernel(ReduceParams p, int n_stages) {
-  constexpr bool WITH_T = mode_is_step(MODE);
-  constexpr bool SAMPLE = (MODE == kModeSample);
-  constexpr int VEC = 16 / (int)sizeof(T);
-  constexpr int kCT = kCW * 32;                              /* consumer threads */
-  constexpr int kStageVecs = kCT * kUnroll;                  /* 128-bit vectors per stage */
-  constexpr int kStageBytes = kStageVecs * 16;
-  extern __shared__ __align__(1024) unsigned char dyn_smem[];
-  unsigned char* ring = dyn_smem;
-  RingSmem& rs = *reinterpret_cast<RingSmem*>(dyn_smem + (size_t)n_stages * kStageBytes);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < n_stages; ++s) { mbar_init(&rs.full[s], 1); mbar_init(&rs.empty[s], kCW); }
-    for (int d = 0; d < kMail; ++d) { mbar_init(&rs.mfull[d], kCW); mbar_init(&rs.mempty[d], 1); }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  }
-  __syncthreads();
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  asm volatile("griddepcontrol.launch_dependents;");          /* the next kernel in the stream may take free SM slots */
-  const int R = p.hdr->R;
-  if (R <= 0) return;
-  const PartitionCtx c = make_partition(R, p.C, (int)gridDim.x);
-  const int g = blockIdx.x;
-  if (g >= c.G) return;
-  SegmentIter it;
-  it.init(c, g, p.src.V);
-  Segment sg;
-
-  if (warp == kCW) {
-    /* ---------------- producer ---------------- */
-    if (lane != 0) return;
-    uint32_t n = 0, s = 0, ph = 0;                           /* stages issued, ring slot, its phase */
-    bool ok = true;
-    while (ok && it.next(sg)) {
-      const int2 bk = p.rows[sg.r];
-      const char* src = reinterpret_cast<const char*>(row_ptr<T>(p.src, bk.x, bk.y) + sg.e0);
-      const uint32_t total = (uint32_t)((sg.e1 - sg.e0) / VEC) * 16u;
-      for (uint32_t off = 0; off < total; off += kStageBytes, ++n) {
-        const uint32_t bytes = (total - off < (uint32_t)kStageBytes) ? (total - off) : (uint32_t)kStageBytes;
-        if (!mbar_wait(&rs.empty[s], ph ^ 1u, p)) { ok = false; break; }
-        mbar_arrive_expect_tx(&rs.full[s], bytes);
-        bulk_copy_g2s(ring + (size_t)s * kStageBytes, src + off, bytes, &rs.full[s]);
-        if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1u; }
-      }
-    }
-    if (!ok) {                                               /* do not leave with copies still landing */
-      const uint32_t first = n > (uint32_t)n_stages ? n - (uint32_t)n_stages : 0u;
-      for (uint32_t q = first; q < n; ++q)
-        mbar_wait(&rs.full[q % (uint32_t)n_stages], (q / (uint32_t)n_stages) & 1u, p);
-    }
-    return;
-  }
-
-  if (warp < kCW) {
-    /* ---------------- consumers ---------------- */
-    const int ctid = threadIdx.x;                           /* 0 .. kCT-1 */
-    uint32_t s = 0, ph = 0, nseg = 0;                       /* ring slot, its phase, segments done */
-    bool sticky = false;                                    /* this thread has met a -inf logit before */
-    while (it.next(sg)) {
-      Acc<T, WITH_T, false> a;
-      a.init();
-      KeyTrack kt;                                            /* stochastic candidates: largest perturbed key */
-      kt.init();
-      NoiseRow nz = NoiseRow{0u, 0u, 0.f, 0u};
-      if (SAMPLE) { const int2 bk = p.rows[sg.r]; nz = noise_row(p.sample_seed, p.step, bk.x, bk.y, p.noise_c, (uint32_t)p.vocab_offset); }
-      const int nvec = (sg.e1 - sg.e0) / VEC;
-      for (int voff = 0; voff < nvec; voff += kStageVecs) {
-        if (!mbar_wait(&rs.full[s], ph, p)) return;
-        const uint4* sp = reinterpret_cast<const uint4*>(ring + (size_t)s * kStageBytes);
-        const int nv = nvec - voff;
-        if (nv >= kStageVecs) {
-          /* a full stage: kUnroll vectors per thread; the stage is handed back to the producer as
-             soon as the values sit in registers (track() has consumed every loaded word) */
-          uint4 v[kUnroll];
-#pragma unroll
-          for (int j = 0; j < kUnroll; ++j) v[j] = sp[ctid + j * kCT];
-          if (!sticky) a.template track<kUnroll>(v, sg.e0 + (voff + ctid) * VEC, kCT * VEC);
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&rs.empty[s]);
-          if (!sticky) a.template accumulate<kUnroll>(v);
-          if (SAMPLE) kt.template update<kUnroll>(T{}, nz, v, sg.e0 + (voff + ctid) * VEC, kCT * VEC);
-        } else {
-          /* the last, partly filled stage of a segment: same unrolled code, vectors past the end
-             replaced by the clamp value (contributes 2^-huge = 0 and never wins the maximum
-             against a finite logit; an all -inf row is re-read by the finaliser anyway) */
-          uint4 v[kUnroll];
-#pragma unroll
-          for (int j = 0; j < kUnroll; ++j)
-            v[j] = (ctid + j * kCT < nv) ? sp[ctid + j * kCT] : neutral_vector(T{});
-          if (!sticky) a.template track<kUnroll>(v, sg.e0 + (voff + ctid) * VEC, kCT * VEC);
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&rs.empty[s]);
-          if (!sticky) a.template accumulate<kUnroll>(v);
-          if (SAMPLE) {                                       /* only the vectors that exist draw noise */
-#pragma unroll
-            for (int j = 0; j < kUnroll; ++j)
-              if (ctid + j * kCT < nv) {
-                const uint4 one[1] = {v[j]};
-                kt.template update<1>(T{}, nz, one, sg.e0 + (voff + ctid + j * kCT) * VEC, kCT * VEC);
-              }
-          }
-        }
-        if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1u; }
-      }
-      const bool tail = (ctid == 0) && (sg.e0 + nvec * VEC < sg.e1);   /* fewer than VEC trailing elements */
-      Part pt;
-      if (tail && (SAMPLE || !sticky)) {
-        const int2 bk = p.rows[sg.r];
-        const T* row = row_ptr<T>(p.src, bk.x, bk.y);
-        for (int e = sg.e0 + nvec * VEC; e < sg.e1; ++e) {
-          const float x = to_f32(row[e]);
-          if (!sticky) a.one(x, e);
-          if (SAMPLE) kt.one(nz, x, e);
-        }
-      }
-      if (!sticky) {
-        pt = a.part();
-        if (!part_is_finite(pt)) sticky = true;
-      }
-      /* a thread that met -inf (now or earlier) takes its own vectors again from global memory, clamped */
-      if (sticky) {
-        const int2 bk = p.rows[sg.r];
-        pt = stream_thread_clamped<T, WITH_T, kCT>(row_ptr<T>(p.src, bk.x, bk.y), sg.e0, sg.e1, ctid, ctid == 0);
-      }
-      __syncwarp();
-      pt = part_warp_reduce(pt);
-      KeyPart kp = key_empty();
-      if (SAMPLE) kp = key_warp_reduce(kt.best);
-      if (lane == 0) {
-        const uint32_t d = nseg % kMail, mph = (nseg / kMail) & 1u;
-        if (mbar_wait(&rs.mempty[d], mph ^ 1u, p)) {
-          rs.mail[d][warp] = pt;
-          if (SAMPLE) rs.kmail[d][warp] = kp;
-          mbar_arrive(&rs.mfull[d]);
-        }
-      }
-      ++nseg;
-    }
-    return;
-  }
-
-  /* ---------------- finaliser ---------------- */
-  uint32_t nseg = 0;
-  while (it.next(sg)) {
-    /* everything that does not depend on the parts is fetched while the consumers still stream */
-    const int b = p.rows[sg.r].x;
-    const int want = p.expected[b];
-    const SeqHint h = load_seq_hint(p, b);
-    const uint32_t d = nseg % kMail, ph = (nseg / kMail) & 1u;
-    if (!mbar_wait(&rs.mfull[d], ph, p)) return;
-    Part pt = (lane < kCW) ? rs.mail[d][lane] : part_empty();
-    KeyPart kp = key_empty();
-    if (SAMPLE && lane < kCW) kp = rs.kmail[d][lane];
-    __syncwarp();
-    if (lane == 0) mbar_arrive(&rs.mempty[d]);
-    pt = part_warp_reduce(pt);
-    if (SAMPLE) kp = key_warp_reduce(kp);
-    if (publish_part(p, pt, sg.r, g, b, want, SAMPLE ? &kp : nullptr)) {
-      if (MODE == kModeLogprob) finalize_logprob_sequence<T>(p, c, b, h);
-      else if (p.vp_part) finalize_vp_local<T, SAMPLE>(p, c, b, h);
-      else finalize_step_sequence<T, SAMPLE>(p, c, b, h);
-    }
-    ++nseg;
-  }
-}
-
-/* ---- vocabulary-parallel select phase: one warp per sequence on the gathered slices ---------- */
-constexpr int kVpNT = 256;
-template <bool SAMPLE>
-__global__ void __launch_bounds__(kVpNT) vp_select_kernel(ReduceParams p) {
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  const int b = (int)blockIdx.x * (kVpNT / 32) + (int)(threadIdx.x >> 5);
-  if (b >= p.B) return;
-  const SeqHint h = load_seq_hint(p, b);
-  if (h.r1 <= h.r0) return;                                  /* no live row: the active-set kernel wrote its outputs */
-  PartitionCtx c;
-  c.U = 0; c.G = 1; c.C = 1; c.small = true;
-  finalize_step_sequence<float, SAMPLE, true>(p, c, b, h);
-}
-
-/* ---- decode-loop helpers ------------------------------------------------------------------- */
-struct CursorParams {
-  const uint8_t* mask; int B, Lt, gen_lo, gen_hi, block_len;
-  int32_t* lo; int32_t* hi; WsHeader* hdr; int init;
-};
-
-/* One warp per sequence: the first block at or after the current one that holds a masked
-   position; lo = hi = gen_hi when there is none.  hdr->remaining counts unfinished sequences. */
-__global__ void __launch_bounds__(kSetupNT, 1) block_cursor_kernel(CursorParams p) {
-  __shared__ int sh_remaining;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = kSetupNT / 32;
-  if (tid == 0) sh_remaining = 0;
-  __syncthreads();
-  for (int b = warp; b < p.B; b += nwarp) {
-    int from = p.gen_lo;
-    if (!p.init) { int cur = p.lo[b]; if (cur >= p.gen_lo && cur < p.gen_hi) from = cur; }
-    int found_lo = p.gen_hi, found_hi = p.gen_hi;
-    for (int s = from; s < p.gen_hi; s += p.block_len) {
-      int e = s + p.block_len; if (e > p.gen_hi) e = p.gen_hi;
-      unsigned any = 0;
-      for (int k0 = s; k0 < e; k0 += 32) {
-        int k = k0 + lane;
-        any |= __ballot_sync(0xffffffffu, (k < e) && p.mask[(size_t)b * p.Lt + k] != 0);
-      }
-      if (any) { found_lo = s; found_hi = e; break; }
-    }
-    if (lane == 0) {
-      p.lo[b] = found_lo; p.hi[b] = found_hi;
-      if (found_lo < found_hi) atomicAdd(&sh_remaining, 1);
-    }
-  }
-  __syncthreads();
-  if (tid == 0) p.hdr->remaining = sh_remaining;
-}
-
-}  // namespace forkd
+#include "fork_params.cuh"
+#include "fork_setup.cuh"
+#include "fork_finalize.cuh"
+#include "fork_stream.cuh"
 
 /* =============================================================================================
  *  Host side: argument checks, launch configuration, the C ABI
