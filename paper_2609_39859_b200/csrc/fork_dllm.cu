@@ -48,15 +48,15 @@ using namespace forkd;
 static std::atomic<long long> g_launches{0};
 static std::atomic<int> g_tune[FORK_TUNE_COUNT_];
 
-static size_t ring_smem_bytes(int n_stages) { return (size_t)n_stages * ring_stage_bytes() + sizeof(RingSmem); }
+static size_t ring_smem_bytes(int n_stages) { return kHalves * ring_half_bytes(n_stages); }
 
-/* The bulk-copy kernel runs two CTAs per SM (8 consumer warps and 6 stages of 16 KB each).  Three
-   CTAs with registers capped at 64 and 4 stages, or two with 12 consumer warps, measured the same
-   on the large shapes and slightly worse on the small one. */
-constexpr int kRingPerSM = 2;
+/* The bulk-copy kernel runs one CTA per SM made of two independent halves (8 consumer warps and 6
+   stages of 16 KB each per half); the work partition counts halves ("virtual CTAs").  Two separate
+   CTAs per SM, three with registers capped at 64, or 12 consumer warps per group measured worse. */
+constexpr int kRingPerSM = kHalves;                        /* virtual CTAs per SM */
 static void ring_config(int* n_stages) {
   int st = g_tune[FORK_TUNE_STAGES].load();
-  const int max_st = (int)((220 * 1024 / kRingPerSM - sizeof(RingSmem) - 1024) / ring_stage_bytes());
+  const int max_st = (int)((220 * 1024 / kHalves - sizeof(RingSmem) - 1024) / ring_stage_bytes());
   if (st <= 0 || st > max_st) st = max_st;
   if (st > kMaxStages) st = kMaxStages;
   if (st < 2) st = 2;
@@ -89,12 +89,12 @@ static bool device_info(DeviceInfo** out) {
     const int max_dyn = 220 * 1024;
     auto allow = [&](const void* fn) { return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn) == cudaSuccess; };
     d.ring_ready =
-        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeStep, kRingPerSM>) &&
-        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeLogprob, kRingPerSM>) &&
-        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeSample, kRingPerSM>) &&
-        allow((const void*)reduce_select_ring_kernel<float, kModeStep, kRingPerSM>) &&
-        allow((const void*)reduce_select_ring_kernel<float, kModeLogprob, kRingPerSM>) &&
-        allow((const void*)reduce_select_ring_kernel<float, kModeSample, kRingPerSM>);
+        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeStep>) &&
+        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeLogprob>) &&
+        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeSample>) &&
+        allow((const void*)reduce_select_ring_kernel<float, kModeStep>) &&
+        allow((const void*)reduce_select_ring_kernel<float, kModeLogprob>) &&
+        allow((const void*)reduce_select_ring_kernel<float, kModeSample>);
     if (!d.ring_ready) return false;
     d.sms = sms;
   }
@@ -160,11 +160,12 @@ static cudaError_t launch_reduce(const ReduceParams& rp, int dtype, int mode, in
   return e;
 }
 
-template <typename T, int MODE, int PER_SM>
+/* G counts virtual CTAs: the launch has G / kHalves CTAs of kHalves * kHalfThreads threads */
+template <typename T, int MODE>
 static cudaError_t launch_ring(const ReduceParams& rp, int G, int n_stages, bool pdl, cudaStream_t st) {
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
-  cfg.gridDim = dim3(G); cfg.blockDim = dim3((kCW + 2) * 32); cfg.dynamicSmemBytes = ring_smem_bytes(n_stages);
+  cfg.gridDim = dim3(G / kHalves); cfg.blockDim = dim3(kHalfThreads * kHalves); cfg.dynamicSmemBytes = ring_smem_bytes(n_stages);
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   if (pdl) {
@@ -172,16 +173,16 @@ static cudaError_t launch_ring(const ReduceParams& rp, int G, int n_stages, bool
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
   }
-  cudaError_t e = cudaLaunchKernelEx(&cfg, reduce_select_ring_kernel<T, MODE, PER_SM>, rp, n_stages);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, reduce_select_ring_kernel<T, MODE>, rp, n_stages);
   if (e == cudaSuccess) g_launches.fetch_add(1);
   return e;
 }
 
-template <typename T, int PER_SM>
+template <typename T>
 static cudaError_t launch_ring_mode(const ReduceParams& rp, int mode, int G, int n_stages, bool pdl, cudaStream_t st) {
-  if (mode == kModeSample) return launch_ring<T, kModeSample, PER_SM>(rp, G, n_stages, pdl, st);
-  if (mode == kModeStep) return launch_ring<T, kModeStep, PER_SM>(rp, G, n_stages, pdl, st);
-  return launch_ring<T, kModeLogprob, PER_SM>(rp, G, n_stages, pdl, st);
+  if (mode == kModeSample) return launch_ring<T, kModeSample>(rp, G, n_stages, pdl, st);
+  if (mode == kModeStep) return launch_ring<T, kModeStep>(rp, G, n_stages, pdl, st);
+  return launch_ring<T, kModeLogprob>(rp, G, n_stages, pdl, st);
 }
 
 /* variant 2 (bulk-copy ring) needs 16-byte aligned rows; everything else takes variant 1 */
@@ -195,8 +196,8 @@ static cudaError_t launch_reduce_inner(const ReduceParams& rp, int dtype, int mo
   if (use_ring(rp)) {
     int n_stages;
     ring_config(&n_stages);
-    if (dtype == FORK_BF16) return launch_ring_mode<bf16_t, kRingPerSM>(rp, mode, G, n_stages, pdl, st);
-    return launch_ring_mode<float, kRingPerSM>(rp, mode, G, n_stages, pdl, st);
+    if (dtype == FORK_BF16) return launch_ring_mode<bf16_t>(rp, mode, G, n_stages, pdl, st);
+    return launch_ring_mode<float>(rp, mode, G, n_stages, pdl, st);
   }
   if (mode == kModeSample) {
     if (dtype == FORK_BF16) return launch(reduce_select_kernel<bf16_t, kModeSample>, dim3(G), dim3(kNT), st, pdl, rp);

@@ -64,7 +64,8 @@ __global__ void __launch_bounds__(kNT, 4) reduce_select_kernel(ReduceParams p) {
 }
 
 /* ---- kernel 2b: bulk-copy (TMA) shared-memory ring, warp-specialised --------------------------
- * Warps 0..kCW-1 consume, warp kCW produces, warp kCW+1 finalises.
+ * One CTA per SM holds two such groups ("halves").  In each half warps 0..kCW-1 consume, warp kCW
+ * produces, warp kCW+1 finalises.
  *   producer : one lane walks the CTA's segments and issues cp.async.bulk copies of up to one stage
  *              (kStageBytes) into a ring of shared-memory stages, each guarded by a full/empty
  *              mbarrier pair; it runs ahead of the consumers by the depth of the ring, across row
@@ -81,6 +82,8 @@ constexpr int kCW = 8;                                     /* consumer warps per
 constexpr int kMaxCW = kCW;
 constexpr int kMail = 4;                                   /* mailbox depth (row segments in flight to the finaliser) */
 constexpr int kMaxStages = 13;
+constexpr int kHalves = 2;                                 /* independent producer/consumer groups per CTA */
+constexpr int kHalfThreads = (kCW + 2) * 32;
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr int ring_stage_bytes() { return kCW * 32 * kUnroll * 16; }     /* 16 KB */
 
@@ -89,6 +92,11 @@ struct RingSmem {
   Part mail[kMail][kMaxCW];
   KeyPart kmail[kMail][kMaxCW];
 };
+
+/* shared memory of one half: its stages and its barriers, rounded to 1 KB */
+__host__ __device__ constexpr size_t ring_half_bytes(int n_stages) {
+  return ((size_t)n_stages * ring_stage_bytes() + sizeof(RingSmem) + 1023) / 1024 * 1024;
+}
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t count) {
@@ -119,20 +127,28 @@ __device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32
 }
 
 
-template <typename T, int MODE, int kPerSM>
-__global__ void __launch_bounds__((kCW + 2) * 32, kPerSM) reduce_select_ring_kernel(ReduceParams p, int n_stages) {
+template <typename T, int MODE>
+__global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_kernel(ReduceParams p, int n_stages) {
   constexpr bool WITH_T = mode_is_step(MODE);
   constexpr bool SAMPLE = (MODE == kModeSample);
   constexpr int VEC = 16 / (int)sizeof(T);
   constexpr int kCT = kCW * 32;                              /* consumer threads */
   constexpr int kStageVecs = kCT * kUnroll;                  /* 128-bit vectors per stage */
   constexpr int kStageBytes = kStageVecs * 16;
-  extern __shared__ __align__(1024) unsigned char dyn_smem[];
+  extern __shared__ __align__(1024) unsigned char dyn_smem_all[];
+  /* One CTA per SM made of kHalves independent halves, each a complete producer / consumers /
+     finaliser group with its own ring, barriers and share of the work ("virtual CTA" g).  As two
+     separate CTAs on one SM the group launched first was favoured by the warp schedulers and finished
+     some 15% ahead of its neighbour, which then ran the rest alone; warps of one CTA are treated
+     alike. */
+  const int half = (int)threadIdx.x / kHalfThreads;
+  const int htid = (int)threadIdx.x % kHalfThreads;          /* thread within the half */
+  unsigned char* dyn_smem = dyn_smem_all + (size_t)half * ring_half_bytes(n_stages);
   unsigned char* ring = dyn_smem;
   RingSmem& rs = *reinterpret_cast<RingSmem*>(dyn_smem + (size_t)n_stages * kStageBytes);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warp = htid >> 5, lane = htid & 31;
 
-  if (threadIdx.x == 0) {
+  if (htid == 0) {
     for (int s = 0; s < n_stages; ++s) { mbar_init(&rs.full[s], 1); mbar_init(&rs.empty[s], kCW); }
     for (int d = 0; d < kMail; ++d) { mbar_init(&rs.mfull[d], kCW); mbar_init(&rs.mempty[d], 1); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -143,8 +159,8 @@ __global__ void __launch_bounds__((kCW + 2) * 32, kPerSM) reduce_select_ring_ker
   asm volatile("griddepcontrol.launch_dependents;");          /* the next kernel in the stream may take free SM slots */
   const int R = p.hdr->R;
   if (R <= 0) return;
-  const PartitionCtx c = make_partition(R, p.C, (int)gridDim.x);
-  const int g = blockIdx.x;
+  const PartitionCtx c = make_partition(R, p.C, (int)gridDim.x * kHalves);
+  const int g = (int)blockIdx.x * kHalves + half;             /* the virtual CTA this half plays */
   if (g >= c.G) return;
   SegmentIter it;
   it.init(c, g, p.src.V);
@@ -177,7 +193,7 @@ __global__ void __launch_bounds__((kCW + 2) * 32, kPerSM) reduce_select_ring_ker
 
   if (warp < kCW) {
     /* ---------------- consumers ---------------- */
-    const int ctid = threadIdx.x;                           /* 0 .. kCT-1 */
+    const int ctid = htid;                                  /* 0 .. kCT-1 */
     uint32_t s = 0, ph = 0, nseg = 0;                       /* ring slot, its phase, segments done */
     bool sticky = false;                                    /* this thread has met a -inf logit before */
     while (it.next(sg)) {
