@@ -566,6 +566,7 @@ def main():
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--pdl", type=int, default=0, help="0 = programmatic dependent launch (default), -1 = off")
+    ap.add_argument("--one-kernel", type=int, default=0, help="0 = small batches run the step as one kernel (default), -1 = always the set-up kernel first")
     ap.add_argument("--temperature", type=float, default=0.0,
                     help="time the step with stochastic candidates at this temperature (default 0: arg-max candidates)")
     args = ap.parse_args()
@@ -592,6 +593,7 @@ def main():
     pkg.fork_set_tuning(pkg.FORK_TUNE_CTAS_PER_SM, args.ctas_per_sm)
     pkg.fork_set_tuning(pkg.FORK_TUNE_STAGES, args.stages)
     pkg.fork_set_tuning(pkg.FORK_TUNE_PDL, args.pdl)
+    pkg.fork_set_tuning(pkg.FORK_TUNE_ONE_KERNEL, args.one_kernel)
 
     sampler = ClockSampler(local_rank) if rank == 0 else None
     if world > 1:
@@ -628,6 +630,7 @@ def main():
                        **({"candidates": "drawn at temperature %g (Gumbel-max in the same pass)" % args.temperature}
                           if args.temperature > 0 else {})),
         "launch": ("one CUDA graph of the K steps" if r["graph"] else "plain stream launches, programmatic dependent launch"),
+        "kernels_per_step": int(r["launches"]) // max(1, steps),
         "host_submit_ms_per_step": r["host_submit_ms"] / steps,
         "hbm_gbs_per_gpu": step_gbs, "frac_of_8TBs_nominal": step_gbs / NOMINAL_HBM_GBS,
         "gpu_launches": int(r["launches"]),
@@ -652,7 +655,7 @@ def main():
         also = []
 
         def shape_line(w2, variant=None, label=""):
-            r2 = time_full_block(w2, w2.seed, min(steps, 50), 5, device, use_graph=False, variant=variant)
+            r2 = time_full_block(w2, w2.seed, steps, max(warmup, 5), device, use_graph=False, variant=variant)
             r2.pop("setup", None)
             r2.pop("keep", None)
             torch.cuda.empty_cache()
@@ -668,6 +671,10 @@ def main():
         for name in ("b8", "passk", "sweep"):
             if name != args.workload:
                 also.append(shape_line(fs.workload(name)))
+        # not one of the five configurations: the pass@k recipe at twice the batch, where the fixed cost
+        # of a launch weighs half as much (how far the streaming rate itself is from the HBM ceiling)
+        import dataclasses
+        also.append(shape_line(dataclasses.replace(fs.workload("passk"), name="passk recipe at B=128", B=128)))
         # the paper's rollout setting: candidates drawn at temperature 0.8 inside the same pass (ALU-bound)
         for name in ("b8", "passk"):
             also.append(shape_line(fs.workload(name), dict(temperature=0.8, sample_seed=12345),

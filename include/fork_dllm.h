@@ -27,7 +27,10 @@
  *     stream reaches that point.  They never synchronise, allocate or free.
  *   - `workspace` is device scratch of at least fork_workspace_bytes(B, Lt) bytes, 256-byte
  *     aligned, private to one call at a time on one stream; its contents need not be kept
- *     between calls (fork_decode_loop keeps its block cursors there while it runs).
+ *     between calls (fork_decode_loop keeps its block cursors there while it runs) and need
+ *     not be initialised.  State that must be clean when a kernel starts (the one-kernel step,
+ *     see FORK_TUNE_ONE_KERNEL) lives in control blocks inside the library, one per workspace
+ *     address and device, up to 1024; workspace addresses beyond that run the two-kernel step.
  *   - Argument errors are found on the host before anything is launched and return
  *     FORK_ERR_INVALID_ARG / FORK_ERR_WORKSPACE; a failed launch returns FORK_ERR_CUDA.
  *   - Logits rows are contiguous in V.  Row (b,k) starts at element
@@ -68,7 +71,9 @@ typedef enum fork_dtype { FORK_BF16 = 0, FORK_F32 = 1 } fork_dtype;
 
 /* bits of the device status word (fork_device_status) */
 #define FORK_DEV_WINDOW_CLAMPED 1u /* a block [lo,hi) reached outside [pos0,pos0+Ll) or [0,Lt) and was clipped */
-#define FORK_DEV_TIMEOUT 2u        /* a bounded in-kernel wait gave up; the results of that call are not valid */
+#define FORK_DEV_TIMEOUT 2u        /* a bounded in-kernel wait gave up; the results of that call are not valid.  Reading
+                                      this bit with fork_device_status also puts the library's control block of that
+                                      workspace back to its initial state; do that before the next step on it. */
 
 /*
  * Arguments of one sampling step (Algorithm 2; inputs x_t, q_theta, lambda -> x_{t-1}).
@@ -323,9 +328,15 @@ const char* fork_status_string(int status);
  *   FORK_TUNE_PDL           0 = launch both kernels of a step with programmatic dependent launch (each
  *                           waits on-device for its predecessor before touching memory), -1 = plain launches
  *   FORK_TUNE_STAGES        0 = automatic, else shared-memory stages (16 KB each) per CTA of variant 2
+ *   FORK_TUNE_ONE_KERNEL    0 = a step of at most 256 sequences whose logits cover at most 1024 words of
+ *                           32 positions over all sequences runs as ONE kernel on variant 2 (every CTA
+ *                           derives the active set itself), -1 = always the set-up kernel first
+ *   FORK_TUNE_LATE_CTA      testing only: g + 1 makes virtual CTA g of a one-kernel step start about
+ *                           0.1 ms late (exercises the hand-over of mask updates), 0 = off
  * Returns the previous value, or -1 for an unknown key.
  */
-enum { FORK_TUNE_VARIANT = 0, FORK_TUNE_CTAS_PER_SM = 1, FORK_TUNE_PDL = 2, FORK_TUNE_STAGES = 3, FORK_TUNE_COUNT_ = 4 };
+enum { FORK_TUNE_VARIANT = 0, FORK_TUNE_CTAS_PER_SM = 1, FORK_TUNE_PDL = 2, FORK_TUNE_STAGES = 3,
+       FORK_TUNE_ONE_KERNEL = 4, FORK_TUNE_LATE_CTA = 5, FORK_TUNE_COUNT_ = 6 };
 int32_t fork_set_tuning(int32_t key, int32_t value);
 
 /* Profiling hook: the next fork_step / fork_logprob call made by this host thread records the two
@@ -335,6 +346,11 @@ void fork_set_timing_events(void* start, void* stop);
 
 /* Number of kernels this library has launched since it was loaded (all entry points). */
 int64_t fork_kernel_launches(void);
+
+/* One-kernel steps: how many times, since the library was loaded on the current device, a sequence's
+   mask update was handed on because a CTA of the launch had not yet read the mask (see
+   FORK_TUNE_LATE_CTA).  Synchronises the device; -1 on a CUDA error.  For tests. */
+int64_t fork_mask_handovers(void);
 
 #ifdef __cplusplus
 }

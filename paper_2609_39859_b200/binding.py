@@ -21,7 +21,7 @@ FORK_ROW_NONFINITE, FORK_ROW_BAD_TOKEN = 1, 2
 FORK_DEV_WINDOW_CLAMPED, FORK_DEV_TIMEOUT = 1, 2
 FORK_FALLBACK_LEFTMOST, FORK_FALLBACK_MAX_CONF, FORK_FALLBACK_MIN_CONF, FORK_FALLBACK_MAX_ENTROPY, \
     FORK_FALLBACK_RANDOM = 0, 1, 2, 3, 4
-FORK_TUNE_VARIANT, FORK_TUNE_CTAS_PER_SM, FORK_TUNE_PDL, FORK_TUNE_STAGES = 0, 1, 2, 3
+FORK_TUNE_VARIANT, FORK_TUNE_CTAS_PER_SM, FORK_TUNE_PDL, FORK_TUNE_STAGES, FORK_TUNE_ONE_KERNEL, FORK_TUNE_LATE_CTA = 0, 1, 2, 3, 4, 5
 
 
 class fork_step_args(C.Structure):
@@ -74,7 +74,7 @@ fork_logits_fn = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32, C.c_void_p, C.c_voi
 EXPORTS = ("fork_workspace_bytes", "fork_step", "fork_step_static", "fork_logprob", "fork_decode_loop", "fork_staging_bytes",
            "fork_select_top_entropy", "fork_grpo_loss", "fork_logprob_backward", "fork_vp_reduce", "fork_vp_select", "fork_read_probe",
            "fork_step_host", "fork_device_status", "fork_status_string", "fork_set_tuning",
-           "fork_kernel_launches", "fork_set_timing_events")
+           "fork_kernel_launches", "fork_mask_handovers", "fork_set_timing_events")
 
 _lib = None
 
@@ -115,6 +115,8 @@ def lib():
     L.fork_set_tuning.argtypes = [C.c_int32, C.c_int32]
     L.fork_kernel_launches.restype = C.c_int64
     L.fork_kernel_launches.argtypes = []
+    L.fork_mask_handovers.restype = C.c_int64
+    L.fork_mask_handovers.argtypes = []
     L.fork_select_top_entropy.restype = C.c_int
     L.fork_select_top_entropy.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float, C.c_void_p,
                                           C.c_void_p, C.c_void_p]
@@ -156,6 +158,10 @@ def fork_set_tuning(key: int, value: int) -> int:
 
 def fork_kernel_launches() -> int:
     return int(lib().fork_kernel_launches())
+
+
+def fork_mask_handovers() -> int:
+    return int(lib().fork_mask_handovers())
 
 
 def _p(t):

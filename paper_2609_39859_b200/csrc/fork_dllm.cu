@@ -1,7 +1,7 @@
 /*
  * Kernels and C ABI of the Fork-dLLM confidence pass (see include/fork_dllm.h for the contract).
  *
- * A step is two launches on the caller's stream:
+ * A step is one or two launches on the caller's stream:
  *   1. active_set_kernel (one CTA): M_t restricted to each sequence's block (Algorithm 2, line 3)
  *      compacted into a row list, per-sequence row offsets, and the number of partial results each
  *      sequence will receive.  The row list is the step's snapshot of the mask: the second kernel
@@ -10,6 +10,9 @@
  *      candidate and its softmax probability, plus entropy), and the CTA that delivers the last
  *      partial result of a sequence applies the unmask rule for it (lines 6-9: threshold set, or
  *      the leftmost masked position when that set is empty) and writes tokens, mask and records.
+ *   Small batches on the bulk-copy kernel skip launch 1: every CTA takes the snapshot for itself
+ *   (bitmaps of the block windows in shared memory), and no sequence's mask is modified before
+ *   every CTA of the launch has done so (FusedCtl in fork_params.cuh).
  * Cross-CTA hand-over uses "last one to arrive" ticket counters (fence + atomic): nothing in
  * here ever waits for another CTA.
  *
@@ -28,6 +31,8 @@
 #include <cuda_runtime.h>
 
 #include <atomic>
+#include <mutex>
+#include <unordered_map>
 #include <cstdint>
 #include <cstdio>
 #include <cstring>
@@ -56,7 +61,7 @@ static size_t ring_smem_bytes(int n_stages) { return kHalves * ring_half_bytes(n
 constexpr int kRingPerSM = kHalves;                        /* virtual CTAs per SM */
 static void ring_config(int* n_stages) {
   int st = g_tune[FORK_TUNE_STAGES].load();
-  const int max_st = (int)((220 * 1024 / kHalves - sizeof(RingSmem) - 1024) / ring_stage_bytes());
+  const int max_st = (int)((220 * 1024 / kHalves - sizeof(RingSmem) - sizeof(SnapSmem) - 1024) / ring_stage_bytes());
   if (st <= 0 || st > max_st) st = max_st;
   if (st > kMaxStages) st = kMaxStages;
   if (st < 2) st = 2;
@@ -235,6 +240,12 @@ extern "C" int32_t fork_set_tuning(int32_t key, int32_t value) {
 
 extern "C" int64_t fork_kernel_launches(void) { return g_launches.load(); }
 
+extern "C" int64_t fork_mask_handovers(void) {
+  unsigned long long n = 0;
+  if (cudaMemcpyFromSymbol(&n, g_mask_handovers, sizeof(n)) != cudaSuccess) return -1;
+  return (int64_t)n;
+}
+
 extern "C" void fork_set_timing_events(void* start, void* stop) {
   t_ev_start = (cudaEvent_t)start;
   t_ev_stop = (cudaEvent_t)stop;
@@ -248,6 +259,53 @@ static fork_status check_workspace(void* ws, size_t bytes, int32_t B, int32_t Lt
 
 struct VpLocal { int32_t vocab_offset; float4* part; float4* key; };
 
+/* ---- one-kernel steps: the control blocks ---------------------------------------------------
+ * Part of the library's device image (zero when loaded), one per workspace address seen on a
+ * device, handed out on first sight and kept for the life of the process; every launch leaves its
+ * block clean, so it does not matter what the caller does with the workspace memory in between,
+ * or whether the address later belongs to a new allocation.  Blocks are never taken back (a CUDA
+ * graph may hold one); when all are taken, further workspace addresses run the two-kernel step. */
+constexpr int kFusedSlots = 1024;
+static __device__ FusedCtl g_fused_ctl[kFusedSlots];
+struct FusedTable {
+  FusedCtl* base = nullptr;
+  std::unordered_map<const void*, int> slot_of;
+  int Gv[kFusedSlots] = {};
+};
+static FusedTable g_fused[64];
+static std::mutex g_fused_mu;
+
+/* The control block of workspace `ws` for launches of Gv virtual CTAs; NULL if none is left.
+   `started` is only meaningful modulo the launch size: when that changes it is put back to zero,
+   in stream order. */
+static FusedCtl* fused_ctl_for(const void* ws, int Gv, cudaStream_t st, bool* cuda_ok) {
+  *cuda_ok = true;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { *cuda_ok = false; return nullptr; }
+  std::lock_guard<std::mutex> lock(g_fused_mu);
+  FusedTable& t = g_fused[dev];
+  if (!t.base) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_fused_ctl) != cudaSuccess || !p) { *cuda_ok = false; return nullptr; }
+    t.base = (FusedCtl*)p;
+  }
+  int i;
+  auto it = t.slot_of.find(ws);
+  if (it != t.slot_of.end()) {
+    i = it->second;
+  } else {
+    if ((int)t.slot_of.size() == kFusedSlots) return nullptr;
+    i = (int)t.slot_of.size();
+    t.slot_of.emplace(ws, i);
+    t.Gv[i] = Gv;
+  }
+  if (t.Gv[i] != Gv) {
+    if (cudaMemsetAsync(&t.base[i].started, 0, sizeof(unsigned long long), st) != cudaSuccess) { *cuda_ok = false; return nullptr; }
+    t.Gv[i] = Gv;
+  }
+  return t.base + i;
+}
+
 static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const int32_t* hi, void* ws,
                              cudaStream_t st, const VpLocal* vp = nullptr) {
   DeviceInfo* dev;
@@ -258,13 +316,27 @@ static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const i
   const int G = grid_size(*dev, a->dtype, mode, fast);
   const int C = (a->V + FORK_CHUNK - 1) / FORK_CHUNK;
 
-  SetupParams sp;
-  memset(&sp, 0, sizeof(sp));
-  sp.flags = a->mask; sp.lo = lo; sp.hi = hi;
-  sp.B = a->B; sp.Lt = a->Lt; sp.pos0 = a->pos0; sp.Ll = a->Ll; sp.C = C; sp.G = G;
-  sp.hdr = w.hdr; sp.seq_off = w.seq_off; sp.expected = w.expected; sp.ticket = w.ticket; sp.rows = w.rows;
-  if (!vp) { sp.n_unmasked = a->n_unmasked; sp.is_fallback = a->is_fallback; sp.fallback_pos = a->fallback_pos; }
-  if (launch(active_set_kernel, dim3(1), dim3(kSetupNT), st, g_tune[FORK_TUNE_PDL].load() >= 0, sp) != cudaSuccess) return FORK_ERR_CUDA;
+  /* a small batch on the bulk-copy kernel runs as one kernel: each virtual CTA takes its own
+     snapshot of the active set, there is no set-up kernel */
+  const int W = (a->Ll + 31) / 32;
+  FusedCtl* ctl = nullptr;
+  const int v = g_tune[FORK_TUNE_VARIANT].load();
+  if (!vp && lo && hi && fast && (v == 0 || v == 2) && g_tune[FORK_TUNE_ONE_KERNEL].load() >= 0 &&
+      a->B <= kFuseMaxB && (long long)a->B * W <= kFuseMaxWords) {
+    bool cuda_ok;
+    ctl = fused_ctl_for(ws, G, st, &cuda_ok);
+    if (!cuda_ok) return FORK_ERR_CUDA;
+  }
+
+  if (!ctl) {
+    SetupParams sp;
+    memset(&sp, 0, sizeof(sp));
+    sp.flags = a->mask; sp.lo = lo; sp.hi = hi;
+    sp.B = a->B; sp.Lt = a->Lt; sp.pos0 = a->pos0; sp.Ll = a->Ll; sp.C = C; sp.G = G;
+    sp.hdr = w.hdr; sp.seq_off = w.seq_off; sp.expected = w.expected; sp.ticket = w.ticket; sp.rows = w.rows;
+    if (!vp) { sp.n_unmasked = a->n_unmasked; sp.is_fallback = a->is_fallback; sp.fallback_pos = a->fallback_pos; }
+    if (launch(active_set_kernel, dim3(1), dim3(kSetupNT), st, g_tune[FORK_TUNE_PDL].load() >= 0, sp) != cudaSuccess) return FORK_ERR_CUDA;
+  }
 
   ReduceParams rp;
   memset(&rp, 0, sizeof(rp));
@@ -282,6 +354,10 @@ static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const i
   rp.nfe = a->nfe; rp.n_fallback = a->n_fallback;
   rp.fallback_mode = a->fallback_mode; rp.fallback_rand = a->fallback_rand;
   if (vp) { rp.vocab_offset = vp->vocab_offset; rp.vp_part = vp->part; rp.vp_key = vp->key; }
+  if (ctl) {
+    rp.ctl = ctl; rp.ticket = ctl->ticket; rp.blk_lo = lo; rp.blk_hi = hi; rp.commit_bits = w.commit_bits;
+    rp.W = W; rp.Gv = G; rp.late_g = g_tune[FORK_TUNE_LATE_CTA].load();
+  }
   if (launch_reduce(rp, a->dtype, mode, G, st) != cudaSuccess) return FORK_ERR_CUDA;
   return FORK_OK;
 }
@@ -392,6 +468,19 @@ extern "C" fork_status fork_device_status(const void* ws, uint32_t* host_out, vo
   cudaStream_t st = (cudaStream_t)stream;
   if (cudaMemcpyAsync(host_out, &h->dev_status, sizeof(uint32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
       cudaStreamSynchronize(st) != cudaSuccess) return FORK_ERR_CUDA;
+  if (*host_out & FORK_DEV_TIMEOUT) {
+    /* a launch that gave up may have left the workspace's control block with tickets or its
+       snapshot count in the middle of a step: put it back to its initial state */
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FORK_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_fused_mu);
+    FusedTable& t = g_fused[dev];
+    auto it = t.slot_of.find(ws);
+    if (it != t.slot_of.end() && t.base) {
+      if (cudaMemsetAsync(t.base + it->second, 0, sizeof(FusedCtl), st) != cudaSuccess ||
+          cudaStreamSynchronize(st) != cudaSuccess) return FORK_ERR_CUDA;
+    }
+  }
   return FORK_OK;
 }
 

@@ -128,8 +128,8 @@ struct MergedRow {
   Part merged; int k, g0, nparts; bool valid, bad, nonfinite;
 };
 template <typename T>
-__device__ __forceinline__ MergedRow merge_rows_warp(const ReduceParams& p, const PartitionCtx& c, int b, int base, int r1,
-                                                     int k_hint) {
+__device__ __forceinline__ MergedRow merge_rows_warp(const ReduceParams& p, const RowMap& rm, const PartitionCtx& c, int b,
+                                                     int base, int r1, int k_hint) {
   const int lane = threadIdx.x & 31;
   const int r = base + lane;
   MergedRow m;
@@ -137,7 +137,7 @@ __device__ __forceinline__ MergedRow merge_rows_warp(const ReduceParams& p, cons
   m.merged = part_empty();
   m.k = 0; m.g0 = 0; m.nparts = 0;
   bool redo = false;
-  if (m.valid) { m.k = (k_hint >= 0) ? k_hint : p.rows[r].y; m.merged = merge_row_parts(p, c, r, m.g0, m.nparts); }
+  if (m.valid) { m.k = (k_hint >= 0) ? k_hint : rm.k_of(b, r); m.merged = merge_row_parts(p, c, r, m.g0, m.nparts); }
   unsigned many = __ballot_sync(0xffffffffu, m.valid && m.nparts > kLaneMergeMax);
   while (many) {                                             /* rows cut into very many parts: all lanes help */
     const int src = __ffs(many) - 1;
@@ -160,11 +160,11 @@ __device__ __forceinline__ MergedRow merge_rows_warp(const ReduceParams& p, cons
 }
 
 template <typename T, bool WANT_INDEX, bool SAMPLE>
-__device__ __forceinline__ RowOut finalize_rows_warp(const ReduceParams& p, const PartitionCtx& c, int b, int base,
-                                                     int r1, Part& merged, int& k, int k_hint) {
+__device__ __forceinline__ RowOut finalize_rows_warp(const ReduceParams& p, const RowMap& rm, const PartitionCtx& c, int b,
+                                                     int base, int r1, Part& merged, int& k, int k_hint) {
   const int lane = threadIdx.x & 31;
   const int r = base + lane;
-  MergedRow m = merge_rows_warp<T>(p, c, b, base, r1, k_hint);
+  MergedRow m = merge_rows_warp<T>(p, rm, c, b, base, r1, k_hint);
   k = m.k;
   if (SAMPLE) {
     float xs = 0.f;
@@ -184,12 +184,43 @@ __device__ __forceinline__ RowOut finalize_rows_warp(const ReduceParams& p, cons
 /* What a finaliser can load about a sequence BEFORE its last part arrives (it idles until then):
    the sequence's row range and this lane's position among its first 32 rows. */
 struct SeqHint { int r0, r1, k; };
-__device__ __forceinline__ SeqHint load_seq_hint(const ReduceParams& p, int b) {
+__device__ __forceinline__ SeqHint load_seq_hint(const RowMap& rm, int b) {
   SeqHint h;
-  h.r0 = p.seq_off[b]; h.r1 = p.seq_off[b + 1];
+  rm.seq_range(b, h.r0, h.r1);
   const int r = h.r0 + (int)(threadIdx.x & 31);
-  h.k = (r < h.r1) ? p.rows[r].y : -1;
+  h.k = (r < h.r1) ? rm.k_of(b, r) : -1;
   return h;
+}
+
+/* Parts sequence b will receive (rows r0 .. r1-1 under partition c), by the whole warp: what the
+   set-up kernel stores in `expected` when there is one. */
+__device__ __forceinline__ int seq_expected_warp(const PartitionCtx& c, int r0, int r1) {
+  int parts = 0;
+  for (int r = r0 + (int)(threadIdx.x & 31); r < r1; r += 32)
+    parts += c.owner((long long)(r + 1) * c.C - 1) - c.owner((long long)r * c.C) + 1;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) parts += __shfl_xor_sync(0xffffffffu, parts, o);
+  return parts;
+}
+
+/* ---- one-kernel step: when may `mask` be modified ------------------------------------------- */
+__device__ unsigned long long g_mask_handovers;               /* mask updates handed on since the library was loaded (all workspaces) */
+__device__ __forceinline__ bool snapshots_complete(const ReduceParams& p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(&p.ctl->started) : "memory");
+  return v % (unsigned long long)p.Gv == 0ull;
+}
+/* One thread: clear the mask at the positions sequence b's finaliser recorded, then drop the flag. */
+__device__ __forceinline__ void apply_deferred(const ReduceParams& p, int b) {
+  for (int i = 0; i < p.W; ++i) {
+    uint32_t x = __ldcg(p.commit_bits + (size_t)b * p.W + i);
+    while (x) {
+      const int bit = __ffs(x) - 1;
+      x &= x - 1;
+      p.mask[(size_t)b * p.Lt + p.src.pos0 + 32 * i + bit] = 0;
+    }
+  }
+  atomicExch(p.ctl->deferred + b, 0u);
 }
 
 /* ---- vocabulary-parallel slices ------------------------------------------------------------- */
@@ -198,12 +229,12 @@ __device__ __forceinline__ SeqHint load_seq_hint(const ReduceParams& p, int b) {
    NaN or +inf, the neutral element (m = -inf, s = t2 = 0) when it holds nothing but -inf; with
    stochastic candidates also (largest perturbed key, global index of its entry, that logit). */
 template <typename T, bool SAMPLE>
-__device__ void finalize_vp_local(const ReduceParams& p, const PartitionCtx& c, int b, const SeqHint& h) {
+__device__ void finalize_vp_local(const ReduceParams& p, const RowMap& rm, const PartitionCtx& c, int b, const SeqHint& h) {
   const int lane = threadIdx.x & 31;
   const float qnan = __int_as_float(0x7fc00000);
   for (int base = h.r0; base < h.r1; base += 32) {
     const int r = base + lane;
-    MergedRow m = merge_rows_warp<T>(p, c, b, base, h.r1, base == h.r0 ? h.k : -1);
+    MergedRow m = merge_rows_warp<T>(p, rm, c, b, base, h.r1, base == h.r0 ? h.k : -1);
     if (!m.valid) continue;
     const size_t at = (size_t)b * p.Lt + m.k;
     const T* row = row_ptr<T>(p.src, b, m.k);
@@ -231,12 +262,13 @@ __device__ void finalize_vp_local(const ReduceParams& p, const PartitionCtx& c, 
 /* Select phase: the statistics of rows base .. base+31 of sequence b from the gathered slices,
    merged in rank order (ascending vocabulary offset; ties keep the lowest global index). */
 template <bool SAMPLE>
-__device__ __forceinline__ RowOut gathered_rows_warp(const ReduceParams& p, int b, int base, int r1, int& k, int k_hint) {
+__device__ __forceinline__ RowOut gathered_rows_warp(const ReduceParams& p, const RowMap& rm, int b, int base, int r1, int& k,
+                                                     int k_hint) {
   const int lane = threadIdx.x & 31;
   const int r = base + lane;
   k = 0;
   if (r >= r1) return row_out_from(part_empty(), true);
-  k = (k_hint >= 0) ? k_hint : p.rows[r].y;
+  k = (k_hint >= 0) ? k_hint : rm.k_of(b, r);
   const size_t at = (size_t)b * p.Lt + k, n = (size_t)p.B * p.Lt;
   Part acc = part_empty();
   for (int j = 0; j < p.vp_ranks; ++j) acc = part_merge(acc, part_from(__ldg(p.vp_parts_in + j * n + at)));
@@ -264,9 +296,12 @@ __device__ __forceinline__ float fallback_key(int mode, float conf, float entrop
 /* The unmask rule for one sequence, run by one warp once every part of the sequence has arrived
    (Algorithm 2 lines 6-9): commit every live position whose confidence exceeds lambda, or one
    position when none does -- the leftmost live one (Fork-dLLM), or the one the requested
-   comparison order picks; write tokens, mask and the per-token records. */
+   comparison order picks; write tokens, mask and the per-token records.  `snapshots_done`: the
+   caller already knows that `mask` may be modified (always so when a set-up kernel took the
+   snapshot). */
 template <typename T, bool SAMPLE, bool GATHERED = false>
-__device__ void finalize_step_sequence(const ReduceParams& p, const PartitionCtx& c, int b, const SeqHint& h) {
+__device__ void finalize_step_sequence(const ReduceParams& p, const RowMap& rm, const PartitionCtx& c, int b, const SeqHint& h,
+                                       bool snapshots_done = true) {
   const int lane = threadIdx.x & 31;
   const int r0 = h.r0, r1 = h.r1;
   const bool one_batch = (r1 - r0) <= 32;                    /* the usual case: results stay in registers */
@@ -278,8 +313,8 @@ __device__ void finalize_step_sequence(const ReduceParams& p, const PartitionCtx
   int best_r = 0x7fffffff;
   for (int base = r0; base < r1; base += 32) {
     Part merged; int k;
-    const RowOut o = GATHERED ? gathered_rows_warp<SAMPLE>(p, b, base, r1, k, base == r0 ? h.k : -1)
-                              : finalize_rows_warp<T, true, SAMPLE>(p, c, b, base, r1, merged, k, base == r0 ? h.k : -1);
+    const RowOut o = GATHERED ? gathered_rows_warp<SAMPLE>(p, rm, b, base, r1, k, base == r0 ? h.k : -1)
+                              : finalize_rows_warp<T, true, SAMPLE>(p, rm, c, b, base, r1, merged, k, base == r0 ? h.k : -1);
     const int r = base + lane;
     if (r < r1) {
       const size_t at = (size_t)b * p.Lt + k;
@@ -312,6 +347,12 @@ __device__ void finalize_step_sequence(const ReduceParams& p, const PartitionCtx
   } else if (fb && p.fallback_mode == FORK_FALLBACK_RANDOM) {
     pick = r0 + (int)(p.fallback_rand[b] % (uint32_t)(r1 - r0));
   }
+  /* one-kernel step: a virtual CTA that has not started yet must still find M_t in `mask` */
+  const bool direct = !p.ctl || snapshots_done || snapshots_complete(p);
+  if (!direct) {
+    for (int i = lane; i < p.W; i += 32) p.commit_bits[(size_t)b * p.W + i] = 0u;
+    __syncwarp();
+  }
   int count = 0, pick_k = -1;
   for (int base = r0; base < r1; base += 32) {
     const int r = base + lane;
@@ -320,11 +361,12 @@ __device__ void finalize_step_sequence(const ReduceParams& p, const PartitionCtx
       const float4 f = one_batch ? keep : p.final_rec[r];    /* written by this same lane above */
       commit = fb ? (r == pick) : (f.x > p.threshold);       /* the fallback position, or the threshold set */
       if (commit) {
-        const int k = one_batch ? keep_k : p.rows[r].y;
+        const int k = one_batch ? keep_k : rm.k_of(b, r);
         const size_t at = (size_t)b * p.Lt + k;
         if (fb) pick_k = k;
         p.tokens[at] = __float_as_int(f.z);
-        p.mask[at] = 0;
+        if (direct) p.mask[at] = 0;
+        else atomicOr(p.commit_bits + (size_t)b * p.W + ((k - p.src.pos0) >> 5), 1u << ((k - p.src.pos0) & 31));
         if (p.commit_step) p.commit_step[at] = p.step;
         if (p.commit_fallback) p.commit_fallback[at] = (uint8_t)fb;
         if (p.commit_logp) p.commit_logp[at] = f.y;
@@ -344,18 +386,31 @@ __device__ void finalize_step_sequence(const ReduceParams& p, const PartitionCtx
     if (p.nfe) atomicAdd(p.nfe + b, 1);
     if (p.n_fallback && fb) atomicAdd(p.n_fallback + b, 1);
   }
+  if (!direct) {
+    /* hand the mask update on: record, raise the flag, look again.  The CTA that counts itself last
+       raises its count, then reads the flags; with a sequentially consistent fence on both sides
+       at least one of the two sees the other. */
+    __syncwarp();
+    if (lane == 0) {
+      atomicAdd(&g_mask_handovers, 1ull);
+      __threadfence();
+      atomicExch(p.ctl->deferred + b, 1u);
+      asm volatile("fence.sc.gpu;" ::: "memory");
+      if (snapshots_complete(p)) apply_deferred(p, b);
+    }
+  }
 }
 
 /* Scoring for one sequence by one warp: log q(token) = x_tok - m - ln s at every selected position
    and their sum (Section 3.2 of the paper: the likelihood terms of the ForkGRPO ratio). */
 template <typename T>
-__device__ void finalize_logprob_sequence(const ReduceParams& p, const PartitionCtx& c, int b, const SeqHint& h) {
+__device__ void finalize_logprob_sequence(const ReduceParams& p, const RowMap& rm, const PartitionCtx& c, int b, const SeqHint& h) {
   const int lane = threadIdx.x & 31;
   const int r0 = h.r0, r1 = h.r1;
   float local = 0.f;
   for (int base = r0; base < r1; base += 32) {
     Part merged; int k;
-    const RowOut o = finalize_rows_warp<T, false, false>(p, c, b, base, r1, merged, k, base == r0 ? h.k : -1);
+    const RowOut o = finalize_rows_warp<T, false, false>(p, rm, c, b, base, r1, merged, k, base == r0 ? h.k : -1);
     const int r = base + lane;
     if (r < r1) {
       const size_t at = (size_t)b * p.Lt + k;
@@ -390,6 +445,7 @@ __device__ __forceinline__ bool publish_part(const ReduceParams& p, const Part& 
     int old;                                 /* release our part, acquire everybody else's */
     asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(p.ticket + b) : "memory");
     last = (old + 1 == want) ? 1 : 0;
+    if (last) p.ticket[b] = 0;               /* nobody else touches it again in this launch: clean for the next one */
   }
   return __shfl_sync(0xffffffffu, last, 0) != 0;
 }
@@ -399,7 +455,13 @@ struct Segment { int r, e0, e1; };
 struct SegmentIter {
   long long u, u1; int C, V;
   __device__ __forceinline__ void init(const PartitionCtx& c, int g, int V_) {
-    u = fork_part_begin(c.U, c.G, g); u1 = fork_part_begin(c.U, c.G, g + 1); C = c.C; V = V_;
+    if (c.small) {                                           /* g*U < 2^32: two 32-bit divisions instead of two 64-bit ones */
+      u = (long long)((uint32_t)g * (uint32_t)c.U / (uint32_t)c.G);
+      u1 = (long long)((uint32_t)(g + 1) * (uint32_t)c.U / (uint32_t)c.G);
+    } else {
+      u = fork_part_begin(c.U, c.G, g); u1 = fork_part_begin(c.U, c.G, g + 1);
+    }
+    C = c.C; V = V_;
   }
   __device__ __forceinline__ bool next(Segment& s) {
     if (u >= u1) return false;

@@ -42,6 +42,7 @@ struct WsView {
   float4* final_rec;                 /* [B*Lt] per-row results kept between the finaliser's passes */
   float4* parts;                     /* [B*Lt + FORK_MAX_GRID] partial results, slot r+g */
   float2* kparts;                    /* [B*Lt + FORK_MAX_GRID] best perturbed key of each part (stochastic candidates) */
+  uint32_t* commit_bits;             /* [B * ceil(Lt/32)] positions committed by a step whose mask update was handed on */
   size_t bytes;
 };
 
@@ -62,9 +63,34 @@ static WsView ws_view(void* base, int32_t B, int32_t Lt) {
   v.final_rec = (float4*)(p + off); off = align_up(off + rows * sizeof(float4), 256);
   v.parts = (float4*)(p + off); off = align_up(off + (rows + FORK_MAX_GRID) * sizeof(float4), 256);
   v.kparts = (float2*)(p + off); off = align_up(off + (rows + FORK_MAX_GRID) * sizeof(float2), 256);
+  v.commit_bits = (uint32_t*)(p + off); off = align_up(off + nb * (size_t)(((Lt > 0 ? Lt : 1) + 31) / 32) * 4, 256);
   v.bytes = off;
   return v;
 }
+
+/* ---- one-kernel step: control block ------------------------------------------------------------
+ * A step whose batch is small enough runs as ONE kernel: every virtual CTA of the streaming kernel
+ * derives the active set itself from `mask` and the block bounds when it starts (its snapshot),
+ * instead of reading the lists a set-up kernel would have written.  That needs state that is clean
+ * when the kernel starts without a kernel before it to clean it: it lives in a control block that
+ * the library owns (zero when the library is loaded, left clean by every launch), never in the
+ * caller's workspace, whose bytes may be anything.
+ *   started  : virtual CTAs that have taken their snapshot, summed over all launches.  Every virtual
+ *              CTA of a launch adds one, so between launches it is a multiple of the launch size and
+ *              "all of this launch have their snapshot" reads started % size == 0.  No sequence's
+ *              mask is modified before that holds (a CTA that starts late must still see M_t).
+ *   ticket   : parts received per sequence; the last arriver puts it back to zero.
+ *   deferred : set by a finaliser that found snapshots still missing: its mask update (positions in
+ *              WsView::commit_bits) is applied by the CTA that counts itself last, or by itself if
+ *              that has happened in the meantime; applying twice is harmless. */
+constexpr int kFuseMaxB = 256;        /* sequences */
+constexpr int kFuseMaxWords = 1024;   /* 32-position words of block window over all sequences */
+struct FusedCtl {
+  unsigned long long started;
+  unsigned long long pad;
+  int32_t ticket[kFuseMaxB];
+  uint32_t deferred[kFuseMaxB];
+};
 
 /* ---- kernel parameters -------------------------------------------------------------------- */
 struct RowSource {                   /* where the logits rows are */
@@ -77,7 +103,7 @@ struct ReduceParams {
   RowSource src;
   int B, Lt, C, fast;
   /* workspace */
-  const WsHeader* hdr; const int32_t* seq_off; const int32_t* expected; int32_t* ticket;
+  WsHeader* hdr; const int32_t* seq_off; const int32_t* expected; int32_t* ticket;
   const int2* rows; float4* final_rec; float4* parts; float2* kparts;
   /* step mode */
   int32_t* tokens; uint8_t* mask; float threshold; int32_t step;
@@ -92,7 +118,49 @@ struct ReduceParams {
   const float4* vp_parts_in; const float4* vp_keys_in; int vp_ranks;   /* select phase: gathered [ranks][B,Lt] */
   /* log-probability mode */
   const int32_t* lp_tokens; float* lp_out; float* seq_sum; int32_t* seq_cnt; float* lse_out;
+  /* one-kernel step (ctl != NULL): the block bounds, the control block, words per sequence of the
+     window bitmaps, virtual CTAs of the launch; late_g - 1 = a virtual CTA that dawdles before its
+     snapshot (testing the handed-on mask update), 0 = none */
+  FusedCtl* ctl; const int32_t* blk_lo; const int32_t* blk_hi; uint32_t* commit_bits; int W, Gv, late_g;
 };
+
+/* Row r of the step -> (sequence, position).  Two-kernel step: the lists the set-up kernel wrote.
+   One-kernel step: this group's snapshot in shared memory -- off[b] = first row of sequence b,
+   bits[b*W + i] = live positions pos0 + 32 i .. pos0 + 32 i + 31 of sequence b. */
+/* the snapshot lookups are rare (once per row segment) and kept out of line: inlined at every use
+   they lengthen the streaming loops' code, which is what the instruction cache has to hold */
+__device__ __noinline__ int snap_seq_of(const int32_t* off, int B, int r) {       /* the last b with off[b] <= r */
+  int lo = 0, hi = B;
+  while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (off[mid] <= r) lo = mid; else hi = mid; }
+  return lo;
+}
+__device__ __noinline__ int snap_pos_of(const uint32_t* w, int W, int pos0, int j) {   /* position of live row j of a sequence */
+  for (int i = 0; i < W; ++i) {
+    const uint32_t x = w[i];
+    const int n = __popc(x);
+    if (j < n) return pos0 + 32 * i + (int)__fns(x, 0u, j + 1);
+    j -= n;
+  }
+  return pos0;
+}
+struct RowMap {
+  const int2* rows; const int32_t* seq_off;
+  const int32_t* off; const uint32_t* bits; int B, W, pos0;
+  __device__ __forceinline__ int seq_of(int r) const { return snap_seq_of(off, B, r); }
+  __device__ __forceinline__ int pos_of(int b, int j) const { return snap_pos_of(bits + b * W, W, pos0, j); }
+  __device__ __forceinline__ int2 bk(int r) const {
+    if (!off) return rows[r];
+    const int b = seq_of(r);
+    return make_int2(b, pos_of(b, r - off[b]));
+  }
+  __device__ __forceinline__ int k_of(int b, int r) const { return off ? pos_of(b, r - off[b]) : rows[r].y; }
+  __device__ __forceinline__ void seq_range(int b, int& r0, int& r1) const {
+    if (off) { r0 = off[b]; r1 = off[b + 1]; } else { r0 = seq_off[b]; r1 = seq_off[b + 1]; }
+  }
+};
+__device__ __forceinline__ RowMap row_map_lists(const ReduceParams& p) {
+  return RowMap{p.rows, p.seq_off, nullptr, nullptr, p.B, 0, p.src.pos0};
+}
 
 template <typename T>
 __device__ __forceinline__ const T* row_ptr(const RowSource& s, int b, int k) {

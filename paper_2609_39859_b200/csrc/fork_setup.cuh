@@ -31,7 +31,10 @@ __device__ __forceinline__ void seq_window(const SetupParams& p, int b, int& lo,
   if (hi < lo) hi = lo;
 }
 
-constexpr int kSetupMaxB = 4096;     /* sequences whose counts fit in shared memory (more: counts go through global memory) */
+/* sequences whose counts fit in shared memory (more: counts go through global memory); small enough
+   that this CTA fits on an SM beside a CTA of the bulk-copy kernel, so that with programmatic
+   dependent launch it is already resident when the step before it ends */
+constexpr int kSetupMaxB = 2048;
 
 __global__ void __launch_bounds__(kSetupNT, 1) active_set_kernel(SetupParams p) {
   /* with programmatic dependent launch this grid may already be resident while the kernel before

@@ -16,7 +16,7 @@ struct Smem {
 };
 
 template <typename T, int MODE>
-__global__ void __launch_bounds__(kNT, 4) reduce_select_kernel(ReduceParams p) {
+__global__ void __launch_bounds__(kNT, 4) reduce_select_kernel(const __grid_constant__ ReduceParams p) {
   constexpr bool WITH_T = mode_is_step(MODE);
   constexpr bool SAMPLE = (MODE == kModeSample);
   __shared__ Smem sm;
@@ -27,12 +27,13 @@ __global__ void __launch_bounds__(kNT, 4) reduce_select_kernel(ReduceParams p) {
   const PartitionCtx c = make_partition(R, p.C, (int)gridDim.x);
   const int g = blockIdx.x;
   if (g >= c.G) return;                                     /* CTAs beyond the number of units have no work */
+  const RowMap rm = row_map_lists(p);
   SegmentIter it;
   it.init(c, g, p.src.V);
   Segment sg;
   bool sticky = false;
   while (it.next(sg)) {
-    const int2 bk = p.rows[sg.r];
+    const int2 bk = rm.bk(sg.r);
     const T* row = row_ptr<T>(p.src, bk.x, bk.y);
     Part part;
     KeyTrack kt;
@@ -54,10 +55,10 @@ __global__ void __launch_bounds__(kNT, 4) reduce_select_kernel(ReduceParams p) {
     if (threadIdx.x < 32) {
       const bool last = publish_part(p, part, sg.r, g, bk.x, p.expected[bk.x], SAMPLE ? &kp : nullptr);
       if (last) {                                           /* every part of sequence b has been delivered */
-        const SeqHint h = load_seq_hint(p, bk.x);
-        if (MODE == kModeLogprob) finalize_logprob_sequence<T>(p, c, bk.x, h);
-        else if (p.vp_part) finalize_vp_local<T, SAMPLE>(p, c, bk.x, h);
-        else finalize_step_sequence<T, SAMPLE>(p, c, bk.x, h);
+        const SeqHint h = load_seq_hint(rm, bk.x);
+        if (MODE == kModeLogprob) finalize_logprob_sequence<T>(p, rm, c, bk.x, h);
+        else if (p.vp_part) finalize_vp_local<T, SAMPLE>(p, rm, c, bk.x, h);
+        else finalize_step_sequence<T, SAMPLE>(p, rm, c, bk.x, h);
       }
     }
   }
@@ -87,15 +88,26 @@ constexpr int kHalfThreads = (kCW + 2) * 32;
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr int ring_stage_bytes() { return kCW * 32 * kUnroll * 16; }     /* 16 KB */
 
+constexpr int kSegRing = 16;                               /* > stages: the producer is never that many segments ahead */
 struct RingSmem {
   unsigned long long full[kMaxStages], empty[kMaxStages], mfull[kMail], mempty[kMail];
   Part mail[kMail][kMaxCW];
   KeyPart kmail[kMail][kMaxCW];
+  int2 seg_bk[kSegRing];                                   /* (sequence, position) of the producer's recent segments, for the consumers */
+};
+static_assert(kSegRing > kMaxStages, "segment ring shorter than the stage ring");
+
+/* the snapshot of the active set a half takes for itself in a one-kernel step */
+struct SnapSmem {
+  int off[kFuseMaxB + 1];                                  /* first row of each sequence; off[B] = R */
+  int lo[kFuseMaxB], hi[kFuseMaxB];                        /* the clipped block window, absolute positions */
+  uint32_t bits[kFuseMaxWords];                            /* live positions, W words per sequence, bit 0 of word 0 = pos0 */
+  int clipped;
 };
 
-/* shared memory of one half: its stages and its barriers, rounded to 1 KB */
+/* shared memory of one half: its stages, its barriers and its snapshot, rounded to 1 KB */
 __host__ __device__ constexpr size_t ring_half_bytes(int n_stages) {
-  return ((size_t)n_stages * ring_stage_bytes() + sizeof(RingSmem) + 1023) / 1024 * 1024;
+  return ((size_t)n_stages * ring_stage_bytes() + sizeof(RingSmem) + sizeof(SnapSmem) + 1023) / 1024 * 1024;
 }
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -118,17 +130,128 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t 
 __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity, const ReduceParams& p) {
   for (uint32_t i = 0; i < kSpinLimit; ++i)
     if (mbar_try_wait(bar, parity)) return true;
-  atomicOr(const_cast<uint32_t*>(&p.hdr->dev_status), FORK_DEV_TIMEOUT);
+  atomicOr(&p.hdr->dev_status, FORK_DEV_TIMEOUT);
   return false;
 }
 __device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                :: "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
+/* barrier among the threads of one half (barrier 0 belongs to __syncthreads) */
+__device__ __forceinline__ void half_sync(int half) {
+  /* immediate barrier numbers: with a register operand the compiler reserves all sixteen */
+  if (half == 0) asm volatile("bar.sync 1, %0;" :: "n"(kHalfThreads) : "memory");
+  else asm volatile("bar.sync 2, %0;" :: "n"(kHalfThreads) : "memory");
+}
 
+__device__ __forceinline__ uint32_t low_bits(int n) { return n >= 32 ? 0xffffffffu : (n <= 0 ? 0u : ((1u << n) - 1u)); }
+
+/* One-kernel step: this half's own snapshot of the active set (Algorithm 2, line 3) -- M_t restricted
+   to each sequence's block window, as bitmaps, and the first row of each sequence.  Every thread of
+   the half calls it; on return the snapshot is complete and visible to all of them.  The same clipping
+   rules as the set-up kernel. */
+struct SnapArgs { const uint8_t* mask; const int32_t* blk_lo; const int32_t* blk_hi; int B, W, Lt; RowSource src; };
+__device__ __noinline__ void take_snapshot(const SnapArgs p, SnapSmem& sn, int half, int htid) {
+  const int warp = htid >> 5, lane = htid & 31;
+  constexpr int kWarps = kHalfThreads / 32;
+  constexpr int kBatch = 8;                                  /* (sequence, word) pairs a warp has in flight */
+  /* Every load below is independent of every other (the bounds and the mask bytes of the whole
+     range the logits cover), so the snapshot costs one trip to memory, not one per item: after a
+     step has streamed its logits through L2 these small arrays are usually back in HBM. */
+  int l0 = 0, h0 = 0;
+  if (htid < p.B) { l0 = p.blk_lo[htid]; h0 = p.blk_hi[htid]; }
+  const int n_items = p.B * p.W;                             /* one warp per pair, 32 positions each */
+  const int lim = min(p.Lt, p.src.pos0 + p.src.Ll);
+  for (int it0 = warp; it0 < n_items; it0 += kBatch * kWarps) {
+    unsigned live[kBatch];
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      const int it = min(it0 + u * kWarps, n_items - 1);
+      const int b = it / p.W, k = p.src.pos0 + 32 * (it - b * p.W) + lane;
+      live[u] = p.mask[(size_t)b * p.Lt + min(k, lim - 1)];  /* always a valid address; positions past the end are dropped below */
+      if (k >= lim) live[u] = 0u;
+    }
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      const int it = it0 + u * kWarps;
+      const unsigned word = __ballot_sync(0xffffffffu, live[u] != 0u);
+      if (it < n_items && lane == 0) sn.bits[it] = word;
+    }
+  }
+  for (int b = htid; b < p.B; b += kHalfThreads) {          /* the same clipping rules as the set-up kernel */
+    if (b != htid) { l0 = p.blk_lo[b]; h0 = p.blk_hi[b]; }
+    int lo = l0, hi = h0;
+    if (lo < 0) lo = 0;
+    if (hi > p.Lt) hi = p.Lt;
+    if (lo < p.src.pos0) lo = p.src.pos0;
+    if (hi > p.src.pos0 + p.src.Ll) hi = p.src.pos0 + p.src.Ll;
+    if (hi < lo) hi = lo;
+    sn.lo[b] = lo; sn.hi[b] = hi;
+    if ((h0 > l0) && (lo != l0 || hi != h0)) sn.clipped = 1;  /* zeroed before the CTA-wide barrier */
+  }
+  half_sync(half);
+  if (warp == 0) {                                           /* cut each sequence's words to its window; rows and their running sum */
+    int carry = 0;
+    for (int b0 = 0; b0 < p.B; b0 += 32) {
+      const int b = b0 + lane;
+      int n = 0;
+      if (b < p.B) {
+        const int lo = sn.lo[b], hi = sn.hi[b];
+        for (int i = 0; i < p.W; ++i) {
+          const int first = p.src.pos0 + 32 * i;
+          const uint32_t word = sn.bits[b * p.W + i] & low_bits(hi - first) & ~low_bits(lo - first);
+          sn.bits[b * p.W + i] = word;
+          n += __popc(word);
+        }
+      }
+      int x = n;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, x, o); if (lane >= o) x += y; }
+      if (b < p.B) sn.off[b + 1] = carry + x;
+      carry += __shfl_sync(0xffffffffu, x, 31);
+    }
+    if (lane == 0) sn.off[0] = 0;
+  }
+  half_sync(half);
+}
+
+/* One-kernel step, finaliser warp of every half, once the snapshot is taken: count this half (its
+   reads of `mask` are complete: the barrier that ended take_snapshot orders them before this); the
+   half that counts itself last applies the mask updates that finalisers had to hand on; virtual
+   CTA 0 reports what the set-up kernel would have.  Returns whether every virtual CTA of the launch
+   has its snapshot. */
+__device__ __noinline__ bool count_snapshot(const ReduceParams& p, const SnapSmem& sn, int g, int R, int G_eff) {
+  const int lane = threadIdx.x & 31;
+  unsigned long long old = 0ull;
+  if (lane == 0)
+    asm volatile("atom.acq_rel.gpu.global.add.u64 %0, [%1], 1;" : "=l"(old) : "l"(&p.ctl->started) : "memory");
+  old = __shfl_sync(0xffffffffu, old, 0);
+  const bool snap_done = (old + 1ull) % (unsigned long long)p.Gv == 0ull;
+  if (snap_done) {
+    asm volatile("fence.sc.gpu;" ::: "memory");
+    for (int b = lane; b < p.B; b += 32) {
+      uint32_t f;
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(f) : "l"(p.ctl->deferred + b) : "memory");
+      if (f) apply_deferred(p, b);
+    }
+  }
+  if (g == 0) {
+    if (lane == 0) {
+      p.hdr->R = R; p.hdr->C = p.C; p.hdr->G = G_eff;
+      p.hdr->dev_status = sn.clipped ? FORK_DEV_WINDOW_CLAMPED : 0u;
+    }
+    for (int b = lane; b < p.B; b += 32)
+      if (sn.off[b] == sn.off[b + 1]) {                       /* no live row: the sequence takes no part in the step */
+        if (p.n_unmasked) p.n_unmasked[b] = 0;
+        if (p.is_fallback) p.is_fallback[b] = 0;
+        if (p.fallback_pos) p.fallback_pos[b] = -1;
+      }
+  }
+  return snap_done;
+}
 
 template <typename T, int MODE>
-__global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_kernel(ReduceParams p, int n_stages) {
+__global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_kernel(const __grid_constant__ ReduceParams p, int n_stages) {
   constexpr bool WITH_T = mode_is_step(MODE);
   constexpr bool SAMPLE = (MODE == kModeSample);
   constexpr int VEC = 16 / (int)sizeof(T);
@@ -146,33 +269,53 @@ __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_
   unsigned char* dyn_smem = dyn_smem_all + (size_t)half * ring_half_bytes(n_stages);
   unsigned char* ring = dyn_smem;
   RingSmem& rs = *reinterpret_cast<RingSmem*>(dyn_smem + (size_t)n_stages * kStageBytes);
+  SnapSmem& sn = *reinterpret_cast<SnapSmem*>(dyn_smem + (size_t)n_stages * kStageBytes + sizeof(RingSmem));
   const int warp = htid >> 5, lane = htid & 31;
 
   if (htid == 0) {
+    sn.clipped = 0;
     for (int s = 0; s < n_stages; ++s) { mbar_init(&rs.full[s], 1); mbar_init(&rs.empty[s], kCW); }
     for (int d = 0; d < kMail; ++d) { mbar_init(&rs.mfull[d], kCW); mbar_init(&rs.mempty[d], 1); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
+  const int g = (int)blockIdx.x * kHalves + half;             /* the virtual CTA this half plays */
+  const bool fused = p.ctl != nullptr;                        /* one-kernel step: no set-up kernel ran */
+  RowMap rm = row_map_lists(p);
+  if (fused) { rm.off = sn.off; rm.bits = sn.bits; rm.W = p.W; }
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;");          /* the next kernel in the stream may take free SM slots */
-  const int R = p.hdr->R;
-  if (R <= 0) return;
+  int R;
+  if (fused) {
+    if (p.late_g == g + 1)                                    /* test hook: this virtual CTA takes its snapshot late */
+      for (int i = 0; i < 100; ++i) __nanosleep(1000);
+    take_snapshot(SnapArgs{p.mask, p.blk_lo, p.blk_hi, p.B, p.W, p.Lt, p.src}, sn, half, htid);
+    R = sn.off[p.B];
+  } else {
+    R = p.hdr->R;
+  }
   const PartitionCtx c = make_partition(R, p.C, (int)gridDim.x * kHalves);
-  const int g = (int)blockIdx.x * kHalves + half;             /* the virtual CTA this half plays */
-  if (g >= c.G) return;
   SegmentIter it;
-  it.init(c, g, p.src.V);
-  Segment sg;
+  Segment sg = Segment{0, 0, 0};
+  bool have = false;                                          /* this half has a first segment */
+  if (R > 0 && g < c.G) {
+    it.init(c, g, p.src.V);
+    have = it.next(sg);
+  }
+  bool snap_done = true;                                      /* every virtual CTA of the launch has its snapshot */
+  if (fused && warp == kCW + 1) snap_done = count_snapshot(p, sn, g, R, c.G);
+  if (!have) return;                                          /* no live row, or more virtual CTAs than units */
 
   if (warp == kCW) {
     /* ---------------- producer ---------------- */
     if (lane != 0) return;
     uint32_t n = 0, s = 0, ph = 0;                           /* stages issued, ring slot, its phase */
     bool ok = true;
-    while (ok && it.next(sg)) {
-      const int2 bk = p.rows[sg.r];
+    uint32_t pseg = 0;
+    for (; ok && have; have = it.next(sg), ++pseg) {
+      const int2 bk = rm.bk(sg.r);
+      rs.seg_bk[pseg % kSegRing] = bk;                       /* visible to the consumers through the stage's full barrier */
       const char* src = reinterpret_cast<const char*>(row_ptr<T>(p.src, bk.x, bk.y) + sg.e0);
       const uint32_t total = (uint32_t)((sg.e1 - sg.e0) / VEC) * 16u;
       for (uint32_t off = 0; off < total; off += kStageBytes, ++n) {
@@ -196,14 +339,21 @@ __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_
     const int ctid = htid;                                  /* 0 .. kCT-1 */
     uint32_t s = 0, ph = 0, nseg = 0;                       /* ring slot, its phase, segments done */
     bool sticky = false;                                    /* this thread has met a -inf logit before */
-    while (it.next(sg)) {
+    for (; have; have = it.next(sg)) {
       Acc<T, WITH_T, false> a;
       a.init();
       KeyTrack kt;                                            /* stochastic candidates: largest perturbed key */
       kt.init();
       NoiseRow nz = NoiseRow{0u, 0u, 0.f, 0u};
-      if (SAMPLE) { const int2 bk = p.rows[sg.r]; nz = noise_row(p.sample_seed, p.step, bk.x, bk.y, p.noise_c, (uint32_t)p.vocab_offset); }
       const int nvec = (sg.e1 - sg.e0) / VEC;
+      /* (sequence, position) of this segment: posted by the producer before the segment's first
+         copy, so readable once a stage of the segment has landed; a segment shorter than one vector
+         has no stage and looks its row up itself */
+      if (SAMPLE) {                                           /* the noise stream of the row is needed from the first element on */
+        if (nvec > 0 && !mbar_wait(&rs.full[s], ph, p)) return;   /* (the stage loop waits on the same phase again: it stays complete) */
+        const int2 bk = nvec > 0 ? rs.seg_bk[nseg % kSegRing] : rm.bk(sg.r);
+        nz = noise_row(p.sample_seed, p.step, bk.x, bk.y, p.noise_c, (uint32_t)p.vocab_offset);
+      }
       for (int voff = 0; voff < nvec; voff += kStageVecs) {
         if (!mbar_wait(&rs.full[s], ph, p)) return;
         const uint4* sp = reinterpret_cast<const uint4*>(ring + (size_t)s * kStageBytes);
@@ -245,7 +395,7 @@ __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_
       const bool tail = (ctid == 0) && (sg.e0 + nvec * VEC < sg.e1);   /* fewer than VEC trailing elements */
       Part pt;
       if (tail && (SAMPLE || !sticky)) {
-        const int2 bk = p.rows[sg.r];
+        const int2 bk = nvec > 0 ? rs.seg_bk[nseg % kSegRing] : rm.bk(sg.r);
         const T* row = row_ptr<T>(p.src, bk.x, bk.y);
         for (int e = sg.e0 + nvec * VEC; e < sg.e1; ++e) {
           const float x = to_f32(row[e]);
@@ -259,7 +409,7 @@ __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_
       }
       /* a thread that met -inf (now or earlier) takes its own vectors again from global memory, clamped */
       if (sticky) {
-        const int2 bk = p.rows[sg.r];
+        const int2 bk = nvec > 0 ? rs.seg_bk[nseg % kSegRing] : rm.bk(sg.r);
         pt = stream_thread_clamped<T, WITH_T, kCT>(row_ptr<T>(p.src, bk.x, bk.y), sg.e0, sg.e1, ctid, ctid == 0);
       }
       __syncwarp();
@@ -281,11 +431,17 @@ __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_
 
   /* ---------------- finaliser ---------------- */
   uint32_t nseg = 0;
-  while (it.next(sg)) {
+  int cur_b = -1, want = 0;
+  SeqHint h = SeqHint{0, 0, -1};
+  for (; have; have = it.next(sg)) {
     /* everything that does not depend on the parts is fetched while the consumers still stream */
-    const int b = p.rows[sg.r].x;
-    const int want = p.expected[b];
-    const SeqHint h = load_seq_hint(p, b);
+    const int b = fused ? rm.seq_of(sg.r) : p.rows[sg.r].x;
+    if (b != cur_b) {
+      cur_b = b;
+      h = load_seq_hint(rm, b);
+      want = fused ? seq_expected_warp(c, h.r0, h.r1) : p.expected[b];
+    }
+    if (fused && !snap_done) snap_done = snapshots_complete(p);
     const uint32_t d = nseg % kMail, ph = (nseg / kMail) & 1u;
     if (!mbar_wait(&rs.mfull[d], ph, p)) return;
     Part pt = (lane < kCW) ? rs.mail[d][lane] : part_empty();
@@ -296,9 +452,9 @@ __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_
     pt = part_warp_reduce(pt);
     if (SAMPLE) kp = key_warp_reduce(kp);
     if (publish_part(p, pt, sg.r, g, b, want, SAMPLE ? &kp : nullptr)) {
-      if (MODE == kModeLogprob) finalize_logprob_sequence<T>(p, c, b, h);
-      else if (p.vp_part) finalize_vp_local<T, SAMPLE>(p, c, b, h);
-      else finalize_step_sequence<T, SAMPLE>(p, c, b, h);
+      if (MODE == kModeLogprob) finalize_logprob_sequence<T>(p, rm, c, b, h);
+      else if (p.vp_part) finalize_vp_local<T, SAMPLE>(p, rm, c, b, h);
+      else finalize_step_sequence<T, SAMPLE>(p, rm, c, b, h, snap_done);
     }
     ++nseg;
   }
@@ -307,15 +463,16 @@ __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_
 /* ---- vocabulary-parallel select phase: one warp per sequence on the gathered slices ---------- */
 constexpr int kVpNT = 256;
 template <bool SAMPLE>
-__global__ void __launch_bounds__(kVpNT) vp_select_kernel(ReduceParams p) {
+__global__ void __launch_bounds__(kVpNT) vp_select_kernel(const __grid_constant__ ReduceParams p) {
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const int b = (int)blockIdx.x * (kVpNT / 32) + (int)(threadIdx.x >> 5);
   if (b >= p.B) return;
-  const SeqHint h = load_seq_hint(p, b);
+  const RowMap rm = row_map_lists(p);
+  const SeqHint h = load_seq_hint(rm, b);
   if (h.r1 <= h.r0) return;                                  /* no live row: the active-set kernel wrote its outputs */
   PartitionCtx c;
   c.U = 0; c.G = 1; c.C = 1; c.small = true;
-  finalize_step_sequence<float, SAMPLE, true>(p, c, b, h);
+  finalize_step_sequence<float, SAMPLE, true>(p, rm, c, b, h);
 }
 
 }  // namespace forkd

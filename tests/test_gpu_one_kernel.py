@@ -1,0 +1,151 @@
+"""The step as ONE kernel (every CTA derives the active set itself; small batches on the bulk-copy
+kernel) against the step with the set-up kernel first, and against the fp64 oracle: same bytes, the
+hand-over of mask updates when a CTA starts late, and the cases that must take the two-kernel path."""
+import numpy as np
+import pytest
+import torch
+
+import fork_synth as fs
+import oracle
+from helpers import compare_step_state, to_torch_logits
+from test_gpu_step import make_rows
+
+pytestmark = pytest.mark.gpu
+
+
+def F():
+    import paper_2609_39859_b200 as pkg
+    return pkg
+
+
+class tuning:
+    def __init__(self, key, value):
+        self.key, self.value = key, value
+
+    def __enter__(self):
+        self.old = F().fork_set_tuning(self.key, self.value)
+
+    def __exit__(self, *a):
+        F().fork_set_tuning(self.key, self.old)
+
+
+def decode(x_steps, mask0, lo, hi, lam, pos0=0, **kw):
+    """Steps on fixed windows with one logits array per step; returns (host dict, launches per step)."""
+    pkg = F()
+    B, Lt = mask0.shape
+    st = pkg.ForkState(B, Lt, mask=mask0)
+    lo_t, hi_t = torch.from_numpy(np.asarray(lo, np.int32)).cuda(), torch.from_numpy(np.asarray(hi, np.int32)).cuda()
+    per_step = []
+    for i, x in enumerate(x_steps):
+        n0 = pkg.fork_kernel_launches()
+        pkg.fork_step(st, to_torch_logits(x), lo_t, hi_t, lam, step=i, pos0=pos0, **kw)
+        per_step.append(pkg.fork_kernel_launches() - n0)
+    torch.cuda.synchronize()
+    assert pkg.fork_device_status(st) == 0
+    return st.host(), per_step
+
+
+def oracle_decode(x_steps, mask0, lo, hi, lam, pos0=0, **kw):
+    B, Lt = mask0.shape
+    o = oracle.StepState(B, Lt, mask=mask0)
+    for i, x in enumerate(x_steps):
+        assert oracle.step(o, x, lo, hi, lam, step_id=i, pos0=pos0, **kw) == 0
+    return o
+
+
+@pytest.mark.parametrize("dtype,V", [("bf16", 126464), ("f32", 4104), ("bf16", 1024)])
+def test_one_kernel_and_two_kernel_steps_give_the_same_bytes(dtype, V):
+    pkg = F()
+    rng = np.random.default_rng(41)
+    B, Lt, pos0, Ll = 5, 96, 32, 48
+    xs = [make_rows(rng, (B, Ll), V, dtype, peak_frac=0.4) for _ in range(4)]
+    mask = (rng.random((B, Lt)) < 0.85).astype(np.uint8)
+    mask[3] = 0                                                # a sequence that takes no part
+    lo, hi = np.array([32, 40, 32, 32, 70], np.int32), np.array([64, 72, 33, 80, 80], np.int32)
+    with tuning(pkg.FORK_TUNE_ONE_KERNEL, 0):
+        one, n_one = decode(xs, mask, lo, hi, 0.9, pos0=pos0)
+    with tuning(pkg.FORK_TUNE_ONE_KERNEL, -1):
+        two, n_two = decode(xs, mask, lo, hi, 0.9, pos0=pos0)
+    assert n_one == [1] * 4 and n_two == [2] * 4
+    for name in one:
+        assert one[name].tobytes() == two[name].tobytes(), name
+    compare_step_state(one, oracle_decode(xs, mask, lo, hi, 0.9, pos0=pos0))
+
+
+def test_one_kernel_step_with_drawn_candidates_and_ranked_fallback():
+    pkg = F()
+    rng = np.random.default_rng(42)
+    B, Lt, V = 6, 64, 20000
+    xs = [make_rows(rng, (B, Lt), V, "bf16", peak_frac=0.2) for _ in range(2)]
+    mask = (rng.random((B, Lt)) < 0.9).astype(np.uint8)
+    lo, hi = np.zeros(B, np.int32), np.full(B, 64, np.int32)
+    kw = dict(fallback_mode=pkg.FORK_FALLBACK_MAX_CONF, temperature=0.7, sample_seed=99)
+    with tuning(pkg.FORK_TUNE_ONE_KERNEL, 0):
+        one, n_one = decode(xs, mask, lo, hi, 0.9, **kw)
+    with tuning(pkg.FORK_TUNE_ONE_KERNEL, -1):
+        two, n_two = decode(xs, mask, lo, hi, 0.9, **kw)
+    assert n_one == [1, 1] and n_two == [2, 2]
+    for name in one:
+        assert one[name].tobytes() == two[name].tobytes(), name
+
+
+@pytest.mark.parametrize("late", ["first", "middle", "last"])
+def test_a_cta_that_starts_late_still_sees_the_mask_of_the_step(late):
+    """One virtual CTA takes its snapshot ~0.1 ms after the others: sequences it has no part in finish
+    long before, must not touch the mask until it has read it, and hand their updates on."""
+    pkg = F()
+    rng = np.random.default_rng(43)
+    B, Lt, V = 8, 32, 126464
+    xs = [make_rows(rng, (B, Lt), V, "bf16", peak_frac=0.6) for _ in range(3)]
+    mask = np.ones((B, Lt), np.uint8)
+    lo, hi = np.zeros(B, np.int32), np.full(B, Lt, np.int32)
+    want = oracle_decode(xs, mask, lo, hi, 0.9)
+    n_virtual = 2 * torch.cuda.get_device_properties(0).multi_processor_count
+    g = {"first": 0, "middle": n_virtual // 2, "last": n_virtual - 1}[late]
+    before = pkg.fork_mask_handovers()
+    with tuning(pkg.FORK_TUNE_ONE_KERNEL, 0), tuning(pkg.FORK_TUNE_LATE_CTA, g + 1):
+        got, n = decode(xs, mask, lo, hi, 0.9)
+    assert n == [1, 1, 1]
+    assert pkg.fork_mask_handovers() > before                  # the path under test did run
+    compare_step_state(got, want)
+    # the control block is clean again: further steps without the late CTA behave as always
+    again, _ = decode(xs, mask, lo, hi, 0.9)
+    compare_step_state(again, want)
+    assert pkg.fork_mask_handovers() >= before
+
+
+def test_batches_too_large_for_the_snapshot_take_the_set_up_kernel():
+    pkg = F()
+    rng = np.random.default_rng(44)
+    for B, Lt, V in ((300, 8, 600), (40, 1024, 130)):          # more than 256 sequences; more than 1024 window words
+        x = make_rows(rng, (B, Lt), V, "f32", peak_frac=0.3)
+        mask = (rng.random((B, Lt)) < 0.5).astype(np.uint8)
+        lo, hi = np.zeros(B, np.int32), np.full(B, Lt, np.int32)
+        got, n = decode([x], mask, lo, hi, 0.9)
+        assert n == [2]
+        compare_step_state(got, oracle_decode([x], mask, lo, hi, 0.9))
+
+
+def test_more_workspaces_than_control_blocks():
+    """Each workspace address gets a control block of its own until the library runs out; the rest
+    run the two-kernel step.  Results do not depend on which."""
+    pkg = F()
+    rng = np.random.default_rng(45)
+    B, Lt, V = 2, 16, 3000
+    x = make_rows(rng, (B, Lt), V, "bf16")
+    mask = np.ones((B, Lt), np.uint8)
+    lo, hi = np.zeros(B, np.int32), np.full(B, Lt, np.int32)
+    want = oracle_decode([x], mask, lo, hi, 0.9)
+    xt = to_torch_logits(x)
+    lo_t, hi_t = torch.from_numpy(lo).cuda(), torch.from_numpy(hi).cuda()
+    states, launches = [], []
+    for _ in range(1100):
+        st = pkg.ForkState(B, Lt, mask=mask)
+        states.append(st)                                      # keep every workspace alive: 1100 distinct addresses
+        n0 = pkg.fork_kernel_launches()
+        pkg.fork_step(st, xt, lo_t, hi_t, 0.9)
+        launches.append(pkg.fork_kernel_launches() - n0)
+    torch.cuda.synchronize()
+    assert set(launches) <= {1, 2} and launches[-1] == 2       # 1024 control blocks per device
+    for st in states[:8] + states[-8:] + states[500:1100:97]:
+        compare_step_state(st.host(), want)
