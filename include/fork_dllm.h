@@ -328,9 +328,9 @@ const char* fork_status_string(int status);
  *   FORK_TUNE_PDL           0 = launch both kernels of a step with programmatic dependent launch (each
  *                           waits on-device for its predecessor before touching memory), -1 = plain launches
  *   FORK_TUNE_STAGES        0 = automatic, else shared-memory stages (16 KB each) per CTA of variant 2
- *   FORK_TUNE_ONE_KERNEL    0 = a step of at most 256 sequences whose logits cover at most 1024 words of
- *                           32 positions over all sequences runs as ONE kernel on variant 2 (every CTA
- *                           derives the active set itself), -1 = always the set-up kernel first
+ *   FORK_TUNE_ONE_KERNEL    0 = a step of at most 256 sequences whose logits cover at most 2048 positions
+ *                           per sequence and 32768 over all sequences runs as ONE kernel on variant 2
+ *                           (every CTA derives the active set itself), -1 = always the set-up kernel first
  *   FORK_TUNE_LATE_CTA      testing only: g + 1 makes virtual CTA g of a one-kernel step start about
  *                           0.1 ms late (exercises the hand-over of mask updates), 0 = off
  * Returns the previous value, or -1 for an unknown key.

@@ -322,7 +322,7 @@ static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const i
   FusedCtl* ctl = nullptr;
   const int v = g_tune[FORK_TUNE_VARIANT].load();
   if (!vp && lo && hi && fast && (v == 0 || v == 2) && g_tune[FORK_TUNE_ONE_KERNEL].load() >= 0 &&
-      a->B <= kFuseMaxB && (long long)a->B * W <= kFuseMaxWords) {
+      a->B <= kFuseMaxB && W <= kFuseMaxSeqWords && (long long)a->B * W <= kFuseMaxWords) {
     bool cuda_ok;
     ctl = fused_ctl_for(ws, G, st, &cuda_ok);
     if (!cuda_ok) return FORK_ERR_CUDA;

@@ -85,6 +85,7 @@ static WsView ws_view(void* base, int32_t B, int32_t Lt) {
  *              that has happened in the meantime; applying twice is harmless. */
 constexpr int kFuseMaxB = 256;        /* sequences */
 constexpr int kFuseMaxWords = 1024;   /* 32-position words of block window over all sequences */
+constexpr int kFuseMaxSeqWords = 64;  /* ... and per sequence (a row look-up walks a sequence's words) */
 struct FusedCtl {
   unsigned long long started;
   unsigned long long pad;
