@@ -636,7 +636,13 @@ def main():
         "gpu_launches": int(r["launches"]),
         "roofline": {"bound": "hbm", "kernel": "reduce_select_ring_kernel<%s,step,8>" % ("bf16" if w.es == 2 else "f32"),
                      "achieved": kern_gbs, "peak": peak, "unit": "GB/s", "frac": kern_gbs / peak,
-                     "peak_source": peak_src, "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
+                     "peak_source": peak_src,
+                     # no capture of its own: the passk capture scaled by the bytes one launch streams
+                     # (traffic is the logits read once plus per-row results, both proportional to them)
+                     "traffic": NCU_TRAFFIC_BYTES.get(args.workload) or int(round(
+                         NCU_TRAFFIC_BYTES["passk"] / (2048 * 252928) * rows * row_bytes)),
+                     "traffic_source": ("ncu capture of this workload (profiles/)" if args.workload in NCU_TRAFFIC_BYTES
+                                        else "ncu capture of the passk workload scaled by algorithmic bytes"),
                      "algorithmic_bytes_per_launch": rows * row_bytes, "kernel_ms": kern_ms, "kernel_ms_source": kern_src,
                      "kernel_ms_event_bracketed": r["kernel_ms"],
                      "whole_step_gbs": step_gbs, "whole_step_frac": step_gbs / peak,
