@@ -68,7 +68,7 @@ static void ring_config(int* n_stages) {
   *n_stages = st;
 }
 
-struct DeviceInfo { int sms = 0; int occ[2][3] = {{0, 0, 0}, {0, 0, 0}}; bool ring_ready = false; };
+struct DeviceInfo { int sms = 0; int occ[2][kModeCount] = {}; bool ring_ready = false; };
 static DeviceInfo g_dev[64];
 
 template <typename T, int MODE>
@@ -91,6 +91,10 @@ static bool device_info(DeviceInfo** out) {
     d.occ[1][1] = occupancy_of<float, kModeLogprob>();
     d.occ[0][2] = occupancy_of<bf16_t, kModeSample>();
     d.occ[1][2] = occupancy_of<float, kModeSample>();
+    d.occ[0][3] = occupancy_of<bf16_t, kModeVp>();
+    d.occ[1][3] = occupancy_of<float, kModeVp>();
+    d.occ[0][4] = occupancy_of<bf16_t, kModeVpSample>();
+    d.occ[1][4] = occupancy_of<float, kModeVpSample>();
     const int max_dyn = 220 * 1024;
     auto allow = [&](const void* fn) { return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn) == cudaSuccess; };
     d.ring_ready =
@@ -99,7 +103,11 @@ static bool device_info(DeviceInfo** out) {
         allow((const void*)reduce_select_ring_kernel<bf16_t, kModeSample>) &&
         allow((const void*)reduce_select_ring_kernel<float, kModeStep>) &&
         allow((const void*)reduce_select_ring_kernel<float, kModeLogprob>) &&
-        allow((const void*)reduce_select_ring_kernel<float, kModeSample>);
+        allow((const void*)reduce_select_ring_kernel<float, kModeSample>) &&
+        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeVp>) &&
+        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeVpSample>) &&
+        allow((const void*)reduce_select_ring_kernel<float, kModeVp>) &&
+        allow((const void*)reduce_select_ring_kernel<float, kModeVpSample>);
     if (!d.ring_ready) return false;
     d.sms = sms;
   }
@@ -187,6 +195,8 @@ template <typename T>
 static cudaError_t launch_ring_mode(const ReduceParams& rp, int mode, int G, int n_stages, bool pdl, cudaStream_t st) {
   if (mode == kModeSample) return launch_ring<T, kModeSample>(rp, G, n_stages, pdl, st);
   if (mode == kModeStep) return launch_ring<T, kModeStep>(rp, G, n_stages, pdl, st);
+  if (mode == kModeVp) return launch_ring<T, kModeVp>(rp, G, n_stages, pdl, st);
+  if (mode == kModeVpSample) return launch_ring<T, kModeVpSample>(rp, G, n_stages, pdl, st);
   return launch_ring<T, kModeLogprob>(rp, G, n_stages, pdl, st);
 }
 
@@ -194,6 +204,19 @@ static cudaError_t launch_ring_mode(const ReduceParams& rp, int mode, int G, int
 static bool use_ring(const ReduceParams& rp) {
   const int v = g_tune[FORK_TUNE_VARIANT].load();
   return rp.fast && (v == 0 || v == 2);
+}
+
+template <typename T>
+static cudaError_t launch_direct(const ReduceParams& rp, int mode, int G, bool pdl, cudaStream_t st) {
+  if (mode == kModeSample) return launch(reduce_select_kernel<T, kModeSample>, dim3(G), dim3(kNT), st, pdl, rp);
+  if (mode == kModeStep) return launch(reduce_select_kernel<T, kModeStep>, dim3(G), dim3(kNT), st, pdl, rp);
+  if (mode == kModeVp) return launch(reduce_select_kernel<T, kModeVp>, dim3(G), dim3(kNT), st, pdl, rp);
+  if (mode == kModeVpSample) return launch(reduce_select_kernel<T, kModeVpSample>, dim3(G), dim3(kNT), st, pdl, rp);
+  return launch(reduce_select_kernel<T, kModeLogprob>, dim3(G), dim3(kNT), st, pdl, rp);
+}
+static cudaError_t launch_direct_dtype(const ReduceParams& rp, int dtype, int mode, int G, bool pdl, cudaStream_t st) {
+  if (dtype == FORK_BF16) return launch_direct<bf16_t>(rp, mode, G, pdl, st);
+  return launch_direct<float>(rp, mode, G, pdl, st);
 }
 
 static cudaError_t launch_reduce_inner(const ReduceParams& rp, int dtype, int mode, int G, cudaStream_t st) {
@@ -204,16 +227,7 @@ static cudaError_t launch_reduce_inner(const ReduceParams& rp, int dtype, int mo
     if (dtype == FORK_BF16) return launch_ring_mode<bf16_t>(rp, mode, G, n_stages, pdl, st);
     return launch_ring_mode<float>(rp, mode, G, n_stages, pdl, st);
   }
-  if (mode == kModeSample) {
-    if (dtype == FORK_BF16) return launch(reduce_select_kernel<bf16_t, kModeSample>, dim3(G), dim3(kNT), st, pdl, rp);
-    return launch(reduce_select_kernel<float, kModeSample>, dim3(G), dim3(kNT), st, pdl, rp);
-  }
-  if (dtype == FORK_BF16) {
-    if (mode == kModeStep) return launch(reduce_select_kernel<bf16_t, kModeStep>, dim3(G), dim3(kNT), st, pdl, rp);
-    return launch(reduce_select_kernel<bf16_t, kModeLogprob>, dim3(G), dim3(kNT), st, pdl, rp);
-  }
-  if (mode == kModeStep) return launch(reduce_select_kernel<float, kModeStep>, dim3(G), dim3(kNT), st, pdl, rp);
-  return launch(reduce_select_kernel<float, kModeLogprob>, dim3(G), dim3(kNT), st, pdl, rp);
+  return launch_direct_dtype(rp, dtype, mode, G, pdl, st);
 }
 
 extern "C" size_t fork_workspace_bytes(int32_t B, int32_t Lt) {
@@ -311,7 +325,8 @@ static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const i
   DeviceInfo* dev;
   if (!device_info(&dev)) return FORK_ERR_CUDA;
   WsView w = ws_view(ws, a->B, a->Lt);
-  const int mode = a->temperature > 0.f ? kModeSample : kModeStep;
+  const bool drawn = a->temperature > 0.f;
+  const int mode = vp ? (drawn ? kModeVpSample : kModeVp) : (drawn ? kModeSample : kModeStep);
   const bool fast = source_is_vector_aligned(a->logits, a->stride_b, a->stride_l, a->dtype);
   const int G = grid_size(*dev, a->dtype, mode, fast);
   const int C = (a->V + FORK_CHUNK - 1) / FORK_CHUNK;
@@ -345,7 +360,7 @@ static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const i
   rp.fast = fast ? 1 : 0;
   rp.hdr = w.hdr; rp.seq_off = w.seq_off; rp.expected = w.expected; rp.ticket = w.ticket;
   rp.rows = w.rows; rp.final_rec = w.final_rec; rp.parts = w.parts; rp.kparts = w.kparts;
-  rp.noise_c = mode == kModeSample ? (float)(1.4426950408889634 / (double)a->temperature) : 0.f;
+  rp.noise_c = drawn ? (float)(1.4426950408889634 / (double)a->temperature) : 0.f;
   rp.sample_seed = a->sample_seed;
   rp.tokens = a->tokens; rp.mask = a->mask; rp.threshold = a->threshold; rp.step = a->step;
   rp.conf = a->conf; rp.cand = a->cand; rp.entropy = a->entropy; rp.logp = a->logp; rp.row_status = a->row_status;

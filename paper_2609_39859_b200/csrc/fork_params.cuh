@@ -17,8 +17,14 @@ constexpr int kNT = 256;             /* threads per CTA of the streaming kernel 
 constexpr int kUnroll = 4;           /* 128-bit loads in flight per thread */
 constexpr int kSetupNT = 1024;       /* threads of the one-CTA set-up kernels */
 
-enum Mode { kModeStep = 0, kModeLogprob = 1, kModeSample = 2 };   /* kModeSample: a step with stochastic candidates (tau > 0) */
+/* kModeSample: a step with stochastic candidates (tau > 0); kModeVp / kModeVpSample: the local phase
+   of the vocabulary-parallel step (per-position parts for the exchange instead of the unmask rule).
+   Instances of their own, so that no kernel carries finalisation code it never runs: the
+   streaming loops share the SM's instruction cache with whatever else the kernel contains. */
+enum Mode { kModeStep = 0, kModeLogprob = 1, kModeSample = 2, kModeVp = 3, kModeVpSample = 4, kModeCount = 5 };
 __host__ __device__ constexpr bool mode_is_step(int mode) { return mode != kModeLogprob; }
+__host__ __device__ constexpr bool mode_is_sample(int mode) { return mode == kModeSample || mode == kModeVpSample; }
+__host__ __device__ constexpr bool mode_is_vp(int mode) { return mode == kModeVp || mode == kModeVpSample; }
 
 /* ---- workspace ---------------------------------------------------------------------------- */
 struct WsHeader {                    /* 256 bytes at the start of the workspace */

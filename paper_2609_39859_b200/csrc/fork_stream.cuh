@@ -18,7 +18,8 @@ struct Smem {
 template <typename T, int MODE>
 __global__ void __launch_bounds__(kNT, 4) reduce_select_kernel(const __grid_constant__ ReduceParams p) {
   constexpr bool WITH_T = mode_is_step(MODE);
-  constexpr bool SAMPLE = (MODE == kModeSample);
+  constexpr bool SAMPLE = mode_is_sample(MODE);
+  constexpr bool VP = mode_is_vp(MODE);
   __shared__ Smem sm;
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;");
@@ -57,7 +58,7 @@ __global__ void __launch_bounds__(kNT, 4) reduce_select_kernel(const __grid_cons
       if (last) {                                           /* every part of sequence b has been delivered */
         const SeqHint h = load_seq_hint(rm, bk.x);
         if (MODE == kModeLogprob) finalize_logprob_sequence<T>(p, rm, c, bk.x, h);
-        else if (p.vp_part) finalize_vp_local<T, SAMPLE>(p, rm, c, bk.x, h);
+        else if (VP) finalize_vp_local<T, SAMPLE>(p, rm, c, bk.x, h);
         else finalize_step_sequence<T, SAMPLE>(p, rm, c, bk.x, h);
       }
     }
@@ -153,30 +154,30 @@ __device__ __forceinline__ uint32_t low_bits(int n) { return n >= 32 ? 0xfffffff
 struct SnapArgs { const uint8_t* mask; const int32_t* blk_lo; const int32_t* blk_hi; int B, W, Lt; RowSource src; };
 __device__ __noinline__ void take_snapshot(const SnapArgs p, SnapSmem& sn, int half, int htid) {
   const int warp = htid >> 5, lane = htid & 31;
-  constexpr int kWarps = kHalfThreads / 32;
-  constexpr int kBatch = 8;                                  /* (sequence, word) pairs a warp has in flight */
-  /* Every load below is independent of every other (the bounds and the mask bytes of the whole
-     range the logits cover), so the snapshot costs one trip to memory, not one per item: after a
-     step has streamed its logits through L2 these small arrays are usually back in HBM. */
+  /* This runs cold at the start of every launch (instructions are fetched at a fraction of the
+     normal rate), and after a step has streamed its logits through L2 the small arrays it reads are
+     usually back in HBM.  So: few instructions, and every load independent of every other -- one
+     thread per (sequence, 32-position word), two 128-bit loads of mask bytes, the bytes squeezed
+     to bits with SIMD compares; one trip to memory for the whole snapshot. */
   int l0 = 0, h0 = 0;
   if (htid < p.B) { l0 = p.blk_lo[htid]; h0 = p.blk_hi[htid]; }
-  const int n_items = p.B * p.W;                             /* one warp per pair, 32 positions each */
-  const int lim = min(p.Lt, p.src.pos0 + p.src.Ll);
-  for (int it0 = warp; it0 < n_items; it0 += kBatch * kWarps) {
-    unsigned live[kBatch];
+  const int n_items = p.B * p.W;
+  const int lim = min(p.Lt, p.src.pos0 + p.src.Ll);         /* positions at or past it do not exist */
+  for (int it = htid; it < n_items; it += kHalfThreads) {
+    const int b = it / p.W, first = p.src.pos0 + 32 * (it - b * p.W);
+    const uint8_t* m = p.mask + (size_t)b * p.Lt + first;
+    uint32_t word = 0u;
+    if (first + 32 <= p.Lt && (reinterpret_cast<uintptr_t>(m) & 15u) == 0) {
+      const uint4 a = *reinterpret_cast<const uint4*>(m), c = *reinterpret_cast<const uint4*>(m + 16);
+      const uint32_t w8[8] = {a.x, a.y, a.z, a.w, c.x, c.y, c.z, c.w};
 #pragma unroll
-    for (int u = 0; u < kBatch; ++u) {
-      const int it = min(it0 + u * kWarps, n_items - 1);
-      const int b = it / p.W, k = p.src.pos0 + 32 * (it - b * p.W) + lane;
-      live[u] = p.mask[(size_t)b * p.Lt + min(k, lim - 1)];  /* always a valid address; positions past the end are dropped below */
-      if (k >= lim) live[u] = 0u;
+      for (int j = 0; j < 8; ++j)                            /* byte != 0 -> 0xff -> one bit each, four at a time */
+        word |= (((__vcmpne4(w8[j], 0u) & 0x01010101u) * 0x01020408u) >> 24) << (4 * j);
+    } else {
+      for (int j = 0; j < 32; ++j)
+        if (first + j < p.Lt && m[j] != 0) word |= 1u << j;
     }
-#pragma unroll
-    for (int u = 0; u < kBatch; ++u) {
-      const int it = it0 + u * kWarps;
-      const unsigned word = __ballot_sync(0xffffffffu, live[u] != 0u);
-      if (it < n_items && lane == 0) sn.bits[it] = word;
-    }
+    sn.bits[it] = word & low_bits(lim - first);
   }
   for (int b = htid; b < p.B; b += kHalfThreads) {          /* the same clipping rules as the set-up kernel */
     if (b != htid) { l0 = p.blk_lo[b]; h0 = p.blk_hi[b]; }
@@ -253,7 +254,8 @@ __device__ __noinline__ bool count_snapshot(const ReduceParams& p, const SnapSme
 template <typename T, int MODE>
 __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_kernel(const __grid_constant__ ReduceParams p, int n_stages) {
   constexpr bool WITH_T = mode_is_step(MODE);
-  constexpr bool SAMPLE = (MODE == kModeSample);
+  constexpr bool SAMPLE = mode_is_sample(MODE);
+  constexpr bool VP = mode_is_vp(MODE);
   constexpr int VEC = 16 / (int)sizeof(T);
   constexpr int kCT = kCW * 32;                              /* consumer threads */
   constexpr int kStageVecs = kCT * kUnroll;                  /* 128-bit vectors per stage */
@@ -453,7 +455,7 @@ __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_
     if (SAMPLE) kp = key_warp_reduce(kp);
     if (publish_part(p, pt, sg.r, g, b, want, SAMPLE ? &kp : nullptr)) {
       if (MODE == kModeLogprob) finalize_logprob_sequence<T>(p, rm, c, b, h);
-      else if (p.vp_part) finalize_vp_local<T, SAMPLE>(p, rm, c, b, h);
+      else if (VP) finalize_vp_local<T, SAMPLE>(p, rm, c, b, h);
       else finalize_step_sequence<T, SAMPLE>(p, rm, c, b, h, snap_done);
     }
     ++nseg;
