@@ -47,7 +47,7 @@ __device__ __forceinline__ Part merge_row_parts(const ReduceParams& p, const Par
 
 /* A row cut into many parts (few live rows, many CTAs): the whole warp loads 32 parts at a time
    and tree-merges them; every lane returns the same Part. */
-__device__ __noinline__ Part merge_row_parts_warp(const ReduceParams& p, int r, int g0, int n) {
+__device__ __forceinline__ Part merge_row_parts_warp(const ReduceParams& p, int r, int g0, int n) {
   const int lane = threadIdx.x & 31;
   const float4* q = p.parts + (r + g0);
   Part acc = part_empty();
@@ -68,7 +68,7 @@ __device__ __noinline__ Part merge_row_parts_warp(const ReduceParams& p, int r, 
 
 /* Guarded scalar reduction of a whole row by ONE warp (every lane returns the same Part). */
 template <typename T>
-__device__ __noinline__ Part careful_row_warp(const T* row, int V, bool& bad, bool* nonfinite = nullptr) {
+__device__ Part careful_row_warp(const T* row, int V, bool& bad, bool* nonfinite = nullptr) {
   const int lane = threadIdx.x & 31;
   float m = -INFINITY;
   int idx = -1, isbad = 0;
