@@ -298,12 +298,16 @@ def time_e2e(w, setup, steps, warmup, device):
     return dict(ms_per_step=dt * 1e3 / n, steps=n, h2d=int(h2d), d2h=int(d2h))
 
 
-def time_logprob(device, peak):
-    """ForkGRPO scoring shape: B=128 fp32, ~20% of positions selected (one call)."""
+def time_logprob(device, peak, B=None):
+    """ForkGRPO scoring shape: B=128 fp32, ~20% of positions selected (one call).  `B`: the same
+    recipe with fewer sequences (a multiple of the group size 8), for profiler captures."""
+    import dataclasses
     import torch
     import fork_synth as fs
     import paper_2609_39859_b200 as pkg
     w = fs.workload("grpo")
+    if B is not None:
+        w = dataclasses.replace(w, B=B)
     cfg = w.cfg()
     tokens, select = fs.scoring_inputs(w, cfg)
     t = torch.empty((w.B, w.Lt, w.V), dtype=torch.float32, device=device)
@@ -325,7 +329,7 @@ def time_logprob(device, peak):
     ms = e0.elapsed_time(e1) / n
     rows = int(select.sum())
     gbs = rows * w.V * 4 / (ms * 1e-3) / 1e9
-    out = [{"workload": "grpo: fork_logprob B=128 Lt=256 V=126464 f32, %d selected rows (3.3 GB >> L2)" % rows,
+    out = [{"workload": "grpo: fork_logprob B=%d Lt=256 V=126464 f32, %d selected rows (%.2f GB >> L2)" % (w.B, rows, rows * w.V * 4 / 1e9),
             "positions_per_s": rows / (ms * 1e-3), "ms": ms, "hbm_gbs": gbs, "frac_of_measured_peak": gbs / peak}]
     # the training half of the same shape: objective (Eq. 2) and the log-softmax backward at the selected rows
     lp, ssum, scnt, status, lse = pkg.fork_logprob(t, tok_d, sel_d, st, want_lse=True)
@@ -339,7 +343,7 @@ def time_logprob(device, peak):
         loss = pkg.fork_grpo_loss(lp, old, sel_d, reward, 8, 0.2, 0.2)
     e1.record()
     torch.cuda.synchronize()
-    out.append({"workload": "grpo: fork_grpo_loss B=128 (16 groups of 8) Lt=256", "ms": e0.elapsed_time(e1) / 20,
+    out.append({"workload": "grpo: fork_grpo_loss B=%d (%d groups of 8) Lt=256" % (w.B, w.B // 8), "ms": e0.elapsed_time(e1) / 20,
                 "kernels_per_call": 2})
     grad = torch.empty_like(t)
     for _ in range(2):
@@ -352,7 +356,7 @@ def time_logprob(device, peak):
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / n
     gbs = 2 * rows * w.V * 4 / (ms * 1e-3) / 1e9
-    out.append({"workload": "grpo: fork_logprob_backward, same %d rows: one read + one write of each row (6.6 GB)" % rows,
+    out.append({"workload": "grpo: fork_logprob_backward, same %d rows: one read + one write of each row (%.2f GB)" % (rows, 2 * rows * w.V * 4 / 1e9),
                 "positions_per_s": rows / (ms * 1e-3), "ms": ms, "hbm_gbs_read_plus_write": gbs,
                 "frac_of_measured_peak": gbs / peak})
     del t, grad
@@ -566,6 +570,8 @@ def main():
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--pdl", type=int, default=0, help="0 = programmatic dependent launch (default), -1 = off")
+    ap.add_argument("--scoring-only", type=int, default=0, metavar="B",
+                    help="run only the ForkGRPO scoring / objective / backward timings with B sequences (multiple of 8) and print them")
     ap.add_argument("--one-kernel", type=int, default=0, help="0 = small batches run the step as one kernel (default), -1 = always the set-up kernel first")
     ap.add_argument("--temperature", type=float, default=0.0,
                     help="time the step with stochastic candidates at this temperature (default 0: arg-max candidates)")
@@ -594,6 +600,11 @@ def main():
     pkg.fork_set_tuning(pkg.FORK_TUNE_STAGES, args.stages)
     pkg.fork_set_tuning(pkg.FORK_TUNE_PDL, args.pdl)
     pkg.fork_set_tuning(pkg.FORK_TUNE_ONE_KERNEL, args.one_kernel)
+
+    if args.scoring_only:                                      # a profiling aid, not the benchmark line
+        if rank == 0:
+            print(json.dumps({"scoring_only": time_logprob(device, peak, B=args.scoring_only)}))
+        return 0
 
     sampler = ClockSampler(local_rank) if rank == 0 else None
     if world > 1:
