@@ -325,7 +325,7 @@ const char* fork_status_string(int status);
  *   FORK_TUNE_VARIANT       0 = automatic, 1 = direct vector loads, 2 = bulk-copy shared-memory ring
  *   FORK_TUNE_CTAS_PER_SM   0 = automatic, else resident CTAs per SM used to size the grid of variant 1
  *                           (variant 2 always runs two per SM)
- *   FORK_TUNE_PDL           0 = launch both kernels of a step with programmatic dependent launch (each
+ *   FORK_TUNE_PDL           0 = launch the kernels of a step with programmatic dependent launch (each
  *                           waits on-device for its predecessor before touching memory), -1 = plain launches
  *   FORK_TUNE_STAGES        0 = automatic, else shared-memory stages (16 KB each) per CTA of variant 2
  *   FORK_TUNE_ONE_KERNEL    0 = a step of at most 256 sequences whose logits cover at most 2048 positions
