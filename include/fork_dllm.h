@@ -30,7 +30,8 @@
  *     between calls (fork_decode_loop keeps its block cursors there while it runs) and need
  *     not be initialised.  State that must be clean when a kernel starts (the one-kernel step,
  *     see FORK_TUNE_ONE_KERNEL) lives in control blocks inside the library, one per workspace
- *     address and device, up to 1024; workspace addresses beyond that run the two-kernel step.
+ *     address and device, up to 1024 at a time (fork_workspace_release gives one back); workspace
+ *     addresses beyond that run the two-kernel step.
  *   - Argument errors are found on the host before anything is launched and return
  *     FORK_ERR_INVALID_ARG / FORK_ERR_WORKSPACE; a failed launch returns FORK_ERR_CUDA.
  *   - Logits rows are contiguous in V.  Row (b,k) starts at element
@@ -312,6 +313,13 @@ fork_status fork_select_top_entropy(const float* entropy, const uint8_t* eligibl
    nothing else (buffer 16-byte aligned; sink4 = 4 bytes of device memory).  Its rate is the
    read-only ceiling that bench.py reports beside the measured copy rate.  Asynchronous. */
 fork_status fork_read_probe(const void* buffer, size_t bytes, void* sink4, void* stream);
+
+/* One-kernel steps keep a small control block inside the library for every workspace address they
+   have seen on the current device (see "Conventions").  Call this when a workspace is done with --
+   every call that used it has completed, and no CUDA graph that captured such a call will be
+   launched again -- to give its block back; addresses that are never released simply keep theirs.
+   Releasing an address the library has not seen is not an error. */
+fork_status fork_workspace_release(const void* workspace);
 
 /* Copies the device status word of the last call that used `workspace` to *host_out
    (FORK_DEV_* bits) and synchronises `stream`. */

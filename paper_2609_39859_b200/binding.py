@@ -74,7 +74,7 @@ fork_logits_fn = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32, C.c_void_p, C.c_voi
 EXPORTS = ("fork_workspace_bytes", "fork_step", "fork_step_static", "fork_logprob", "fork_decode_loop", "fork_staging_bytes",
            "fork_select_top_entropy", "fork_grpo_loss", "fork_logprob_backward", "fork_vp_reduce", "fork_vp_select", "fork_read_probe",
            "fork_step_host", "fork_device_status", "fork_status_string", "fork_set_tuning",
-           "fork_kernel_launches", "fork_mask_handovers", "fork_set_timing_events")
+           "fork_kernel_launches", "fork_mask_handovers", "fork_workspace_release", "fork_set_timing_events")
 
 _lib = None
 
@@ -117,6 +117,8 @@ def lib():
     L.fork_kernel_launches.argtypes = []
     L.fork_mask_handovers.restype = C.c_int64
     L.fork_mask_handovers.argtypes = []
+    L.fork_workspace_release.restype = C.c_int
+    L.fork_workspace_release.argtypes = [C.c_void_p]
     L.fork_select_top_entropy.restype = C.c_int
     L.fork_select_top_entropy.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float, C.c_void_p,
                                           C.c_void_p, C.c_void_p]
@@ -208,6 +210,22 @@ class ForkState:
         self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=dev)
         off = (-self.workspace.data_ptr()) % 256
         self.ws_ptr, self.ws_bytes = self.workspace.data_ptr() + off, nbytes
+
+    def close(self):
+        """Give the control block the library keeps for this workspace address back (one-kernel
+        steps).  Waits for the device first: the library's condition is that every call that used
+        the workspace has completed."""
+        ptr, self.ws_ptr = getattr(self, "ws_ptr", None), None
+        if ptr and _lib is not None:
+            with torch.cuda.device(self.device):
+                torch.cuda.synchronize()
+                _lib.fork_workspace_release(C.c_void_p(ptr))
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:                  # interpreter or CUDA context already going away
+            pass
 
     def host(self) -> dict:
         names = ["tokens", "mask"] + [n for n, _, _ in self.PER_POS] + [n for n, _, _ in self.PER_SEQ]

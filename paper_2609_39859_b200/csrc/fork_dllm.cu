@@ -277,14 +277,19 @@ struct VpLocal { int32_t vocab_offset; float4* part; float4* key; };
  * Part of the library's device image (zero when loaded), one per workspace address seen on a
  * device, handed out on first sight and kept for the life of the process; every launch leaves its
  * block clean, so it does not matter what the caller does with the workspace memory in between,
- * or whether the address later belongs to a new allocation.  Blocks are never taken back (a CUDA
- * graph may hold one); when all are taken, further workspace addresses run the two-kernel step. */
+ * or whether the address later belongs to a new allocation.  A block goes back to the pool only
+ * when the caller says the workspace is done with (fork_workspace_release: nothing in here can tell
+ * whether a launch or a CUDA graph still refers to it); when all are taken, further workspace
+ * addresses run the two-kernel step. */
 constexpr int kFusedSlots = 1024;
 static __device__ FusedCtl g_fused_ctl[kFusedSlots];
 struct FusedTable {
   FusedCtl* base = nullptr;
   std::unordered_map<const void*, int> slot_of;
   int Gv[kFusedSlots] = {};
+  int n_used = 0;                     /* blocks handed out at least once */
+  int free_list[kFusedSlots] = {};    /* ... and given back */
+  int n_free = 0;
 };
 static FusedTable g_fused[64];
 static std::mutex g_fused_mu;
@@ -308,10 +313,10 @@ static FusedCtl* fused_ctl_for(const void* ws, int Gv, cudaStream_t st, bool* cu
   if (it != t.slot_of.end()) {
     i = it->second;
   } else {
-    if ((int)t.slot_of.size() == kFusedSlots) return nullptr;
-    i = (int)t.slot_of.size();
+    if (t.n_free > 0) i = t.free_list[--t.n_free];
+    else if (t.n_used < kFusedSlots) { i = t.n_used++; t.Gv[i] = Gv; }
+    else return nullptr;
     t.slot_of.emplace(ws, i);
-    t.Gv[i] = Gv;
   }
   if (t.Gv[i] != Gv) {
     if (cudaMemsetAsync(&t.base[i].started, 0, sizeof(unsigned long long), st) != cudaSuccess) { *cuda_ok = false; return nullptr; }
@@ -475,6 +480,20 @@ extern "C" fork_status fork_decode_loop(const fork_step_args* proto, int32_t blo
   }
   if (steps_taken) *steps_taken = n;
   return rc;
+}
+
+extern "C" fork_status fork_workspace_release(const void* ws) {
+  if (!ws) return FORK_ERR_INVALID_ARG;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FORK_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_fused_mu);
+  FusedTable& t = g_fused[dev];
+  auto it = t.slot_of.find(ws);
+  if (it != t.slot_of.end()) {
+    t.free_list[t.n_free++] = it->second;
+    t.slot_of.erase(it);
+  }
+  return FORK_OK;
 }
 
 extern "C" fork_status fork_device_status(const void* ws, uint32_t* host_out, void* stream) {

@@ -127,8 +127,9 @@ def test_batches_too_large_for_the_snapshot_take_the_set_up_kernel():
 
 
 def test_more_workspaces_than_control_blocks():
-    """Each workspace address gets a control block of its own until the library runs out; the rest
-    run the two-kernel step.  Results do not depend on which."""
+    """Each workspace address gets a control block of its own until the library runs out (1024 per
+    device); the rest run the two-kernel step, and releasing a workspace gives its block to the next
+    one.  Results do not depend on which path ran."""
     pkg = F()
     rng = np.random.default_rng(45)
     B, Lt, V = 2, 16, 3000
@@ -138,16 +139,28 @@ def test_more_workspaces_than_control_blocks():
     want = oracle_decode([x], mask, lo, hi, 0.9)
     xt = to_torch_logits(x)
     lo_t, hi_t = torch.from_numpy(lo).cuda(), torch.from_numpy(hi).cuda()
-    states, launches = [], []
-    for _ in range(1100):
+
+    def step_on_new_state():
         st = pkg.ForkState(B, Lt, mask=mask)
-        states.append(st)                                      # keep every workspace alive: 1100 distinct addresses
         n0 = pkg.fork_kernel_launches()
         pkg.fork_step(st, xt, lo_t, hi_t, 0.9)
-        launches.append(pkg.fork_kernel_launches() - n0)
+        return st, pkg.fork_kernel_launches() - n0
+
+    states, launches = [], []
+    for _ in range(1100):                                      # every workspace stays alive: 1100 distinct addresses
+        st, n = step_on_new_state()
+        states.append(st)
+        launches.append(n)
     torch.cuda.synchronize()
-    assert set(launches) <= {1, 2} and launches[-1] == 2       # 1024 control blocks per device
+    assert set(launches) <= {1, 2} and launches[-1] == 2
     for st in states[:8] + states[-8:] + states[500:1100:97]:
+        compare_step_state(st.host(), want)
+    for st in states[:600]:                                    # hand 600 blocks back ...
+        st.close()
+    again = [step_on_new_state() for _ in range(100)]          # ... and new workspaces find one
+    torch.cuda.synchronize()
+    assert [n for _, n in again] == [1] * 100
+    for st, _ in again[::9]:
         compare_step_state(st.host(), want)
 
 
@@ -191,3 +204,25 @@ def test_random_windows_alignments_and_masks_match_the_oracle_on_both_paths():
                 assert not (pkg.fork_device_status(st) & pkg.FORK_DEV_TIMEOUT)
                 compare_step_state(st.host(), want)
     assert ran >= 30
+
+
+@pytest.mark.parametrize("B,Ll,kernels", [(256, 128, 1), (256, 129, 2), (257, 32, 2), (16, 2048, 1), (16, 2049, 2)])
+def test_the_limits_of_the_one_kernel_step(B, Ll, kernels):
+    """Exactly at the snapshot's capacity (256 sequences, 64 words per sequence, 1024 words in all) and
+    one past it: which path runs, and that either agrees with the oracle."""
+    rng = np.random.default_rng(47 + B + Ll)
+    Lt, V = Ll + 7, 40
+    x = make_rows(rng, (B, Ll), V, "f32", peak_frac=0.5)
+    mask = (rng.random((B, Lt)) < 0.3).astype(np.uint8)
+    lo = rng.integers(0, 8, B).astype(np.int32)
+    hi = np.full(B, Lt, np.int32)                              # reaches past the logits buffer: clipped to it
+    pkg = F()
+    st = pkg.ForkState(B, Lt, mask=mask)
+    n0 = pkg.fork_kernel_launches()
+    pkg.fork_step(st, to_torch_logits(x), torch.from_numpy(lo).cuda(), torch.from_numpy(hi).cuda(), 0.9, step=3)
+    assert pkg.fork_kernel_launches() - n0 == kernels
+    torch.cuda.synchronize()
+    assert pkg.fork_device_status(st) == pkg.FORK_DEV_WINDOW_CLAMPED
+    want = oracle.StepState(B, Lt, mask=mask)
+    assert oracle.step(want, x, lo, hi, 0.9, step_id=3) == 0
+    compare_step_state(st.host(), want)
