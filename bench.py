@@ -395,9 +395,23 @@ def time_vocab_parallel(device, peak, n_ranks=8):
         if i >= 3:
             t_red += e0.elapsed_time(e1)
             t_sel += e1.elapsed_time(e2)
+    # the same reduction with the exchange fused in: stores into n_ranks gather buffers (all on this GPU here)
+    Lt = st.Lt
+    peers = [torch.zeros((n_ranks, w.B, Lt, 4), dtype=torch.float32, device=device) for _ in range(n_ranks)]
+    t_fused = 0.0
+    for i in range(reps + 3):
+        reset_states([st])
+        flush = bufs[1].view(torch.int16)[:, :8].sum()
+        e0.record()
+        pkg.fork_vp_reduce_peers(st, shard, lo, hi, w.threshold, off, 1, peers)
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= 3:
+            t_fused += e0.elapsed_time(e1)
     rows = w.B * w.block_len
     ms_red, ms_sel = t_red / reps, t_sel / reps
-    return {"workload": "passk sharded over %d ranks along V (one rank's share, emulated on one GPU): "
+    return {"reduce_with_fused_exchange_ms": t_fused / reps,
+            "workload": "passk sharded over %d ranks along V (one rank's share, emulated on one GPU): "
                         "fork_vp_reduce on a [%d,%d,%d] slice + fork_vp_select on %d gathered buffers" %
                         (n_ranks, w.B, w.block_len, n, n_ranks),
             "reduce_ms": ms_red, "select_ms": ms_sel, "slice_gbs": rows * n * w.es / (ms_red * 1e-3) / 1e9,

@@ -17,8 +17,8 @@
  * fork_step_static (no workspace argument); the variants the paper compares with or trains with:
  * candidates drawn at temperature tau > 0 and the other fallback orders (fields of fork_step_args),
  * fork_select_top_entropy (JustGRPO-Fast's position selection), fork_grpo_loss (Eq. 2) and
- * fork_logprob_backward (its log-softmax backward); fork_vp_reduce / fork_vp_select (the step with
- * the vocabulary sharded over ranks).
+ * fork_logprob_backward (its log-softmax backward); fork_vp_reduce / fork_vp_reduce_peers /
+ * fork_vp_select (the step with the vocabulary sharded over ranks).
  *
  * Conventions for every entry point
  *   - All data pointers are DEVICE pointers owned by the caller unless a comment says "host".
@@ -238,6 +238,27 @@ fork_status fork_vp_reduce(const fork_step_args* args, int32_t vocab_offset, voi
                            void* workspace, size_t workspace_bytes, void* stream);
 fork_status fork_vp_select(const fork_step_args* args, const void* parts, const void* keys, int32_t n_ranks,
                            void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Steps 1 and 2 in one kernel: fork_vp_reduce with the exchange fused in.  Instead of filling one
+ * local [B,Lt] buffer for the caller to all-gather, the kernel stores each live position's 16 bytes,
+ * as soon as the slice's reduction of that sequence is complete, straight into the gather buffer of
+ * EVERY rank at [rank][b,k] -- plain 16-byte stores, the remote ones travelling over NVLink while
+ * the rest of the slice is still being reduced.  Nothing is ever loaded from another GPU's memory.
+ *   - peer_parts: HOST array of n_ranks device addresses, valid on THIS GPU: entry j is rank j's
+ *     gather buffer [n_ranks][B,Lt] x 16 bytes (this GPU's own buffer for j == rank; for the others
+ *     memory of GPU j mapped here: CUDA IPC, cuMem with peer access, or symmetric memory), 16-byte
+ *     aligned.  peer_keys: the same for the perturbed keys, needed when temperature > 0, else NULL.
+ *     n_ranks <= FORK_VP_MAX_RANKS.  The arrays are read during the call only.
+ *   - Ordering is the caller's: fork_vp_select on any rank must not start before the kernels of
+ *     this call have COMPLETED on all ranks (e.g. synchronise the stream, then a barrier among the
+ *     ranks; or a stream-ordered collective on one word).  Positions that are not live are not
+ *     written: fork_vp_select reads live positions only.
+ */
+#define FORK_VP_MAX_RANKS 16
+fork_status fork_vp_reduce_peers(const fork_step_args* args, int32_t vocab_offset, int32_t rank, int32_t n_ranks,
+                                 void* const* peer_parts, void* const* peer_keys,
+                                 void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * fork_step without a workspace argument, for callers that have no device memory to give and

@@ -72,7 +72,7 @@ fork_logits_fn = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32, C.c_void_p, C.c_voi
                              C.c_void_p, C.c_void_p)
 
 EXPORTS = ("fork_workspace_bytes", "fork_step", "fork_step_static", "fork_logprob", "fork_decode_loop", "fork_staging_bytes",
-           "fork_select_top_entropy", "fork_grpo_loss", "fork_logprob_backward", "fork_vp_reduce", "fork_vp_select", "fork_read_probe",
+           "fork_select_top_entropy", "fork_grpo_loss", "fork_logprob_backward", "fork_vp_reduce", "fork_vp_reduce_peers", "fork_vp_select", "fork_read_probe",
            "fork_step_host", "fork_device_status", "fork_status_string", "fork_set_tuning",
            "fork_kernel_launches", "fork_mask_handovers", "fork_workspace_release", "fork_set_timing_events")
 
@@ -119,6 +119,9 @@ def lib():
     L.fork_mask_handovers.argtypes = []
     L.fork_workspace_release.restype = C.c_int
     L.fork_workspace_release.argtypes = [C.c_void_p]
+    L.fork_vp_reduce_peers.restype = C.c_int
+    L.fork_vp_reduce_peers.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                                       C.c_void_p, C.c_size_t, C.c_void_p]
     L.fork_select_top_entropy.restype = C.c_int
     L.fork_select_top_entropy.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float, C.c_void_p,
                                           C.c_void_p, C.c_void_p]
@@ -434,6 +437,35 @@ def fork_vp_reduce(st: ForkState, logits_slice: torch.Tensor, blk_lo, blk_hi, th
     return parts, keys
 
 
+def fork_vp_reduce_peers(st: ForkState, logits_slice: torch.Tensor, blk_lo, blk_hi, threshold: float, vocab_offset: int,
+                         rank: int, gather_parts, gather_keys=None, step: int = 0, pos0: int = 0, stream=None,
+                         **variant) -> None:
+    """Local phase with the exchange fused in: this rank's slice results go straight into slot `rank`
+    of EVERY rank's gather buffer.  gather_parts[j] (and gather_keys[j] with drawn candidates) is rank
+    j's buffer [N, B, Lt, 4] float32 as addressable from this GPU: a tensor, or an integer device
+    address of peer-mapped memory.  The caller orders the select phase after the completion of this
+    call on all ranks."""
+    a = make_step_args(st, logits_slice, blk_lo, blk_hi, threshold, step, pos0, **variant)
+    n = len(gather_parts)
+
+    def addresses(bufs):
+        arr = (C.c_void_p * n)()
+        for j, t in enumerate(bufs):
+            if isinstance(t, torch.Tensor):
+                assert t.dtype == torch.float32 and t.is_contiguous() and tuple(t.shape) == (n, st.B, st.Lt, 4)
+                arr[j] = t.data_ptr()
+            else:
+                arr[j] = int(t)
+        return arr
+
+    parts_arr = addresses(gather_parts)
+    keys_arr = addresses(gather_keys) if (a.temperature > 0 and gather_keys is not None) else None
+    rc = lib().fork_vp_reduce_peers(C.byref(a), int(vocab_offset), int(rank), n, parts_arr, keys_arr,
+                                    C.c_void_p(st.ws_ptr), st.ws_bytes, _stream_ptr(stream))
+    if rc != FORK_OK:
+        raise ForkError(rc, "fork_vp_reduce_peers")
+
+
 def fork_vp_select(st: ForkState, parts: torch.Tensor, keys, blk_lo, blk_hi, threshold: float, step: int = 0,
                    pos0: int = 0, Ll: int = 0, stream=None, **variant) -> None:
     """Select phase on the gathered slices: parts (and keys) are [N, B, Lt, 4] in rank order."""
@@ -456,10 +488,26 @@ def gather_rank_major(t: torch.Tensor, group=None) -> torch.Tensor:
 
 
 def fork_step_vocab_parallel(st: ForkState, logits_slice: torch.Tensor, blk_lo, blk_hi, threshold: float,
-                             vocab_offset: int, step: int = 0, pos0: int = 0, group=None, stream=None, **variant) -> None:
-    """One sampling step with the vocabulary sharded over the ranks of `group`: local reduction, one
-    all-gather of 16 (32 with drawn candidates) bytes per position, selection on every rank.  Slices
-    must ascend with the rank (vocab_shards)."""
+                             vocab_offset: int, step: int = 0, pos0: int = 0, group=None, stream=None,
+                             peer_buffers=None, **variant) -> None:
+    """One sampling step with the vocabulary sharded over the ranks of `group`: local reduction, an
+    exchange of 16 (32 with drawn candidates) bytes per position, selection on every rank.  Slices
+    must ascend with the rank (vocab_shards).
+    The exchange is one all-gather (torch.distributed), or, with `peer_buffers` = (gather_parts,
+    gather_keys or None) as fork_vp_reduce_peers takes them (every rank's gather buffer mapped on
+    this GPU), stores issued by the reduction kernel itself followed by a barrier of the group."""
+    if peer_buffers is not None:
+        import torch.distributed as dist
+        rank = dist.get_rank(group)
+        g_parts_all, g_keys_all = peer_buffers
+        fork_vp_reduce_peers(st, logits_slice, blk_lo, blk_hi, threshold, vocab_offset, rank, g_parts_all, g_keys_all,
+                             step, pos0, stream, **variant)
+        (stream or torch.cuda.current_stream()).synchronize()      # this rank's stores are out ...
+        dist.barrier(group)                                        # ... and so are everybody else's
+        mine = g_parts_all[rank]
+        keys_mine = g_keys_all[rank] if (g_keys_all is not None and variant.get("temperature", 0.0) > 0) else None
+        fork_vp_select(st, mine, keys_mine, blk_lo, blk_hi, threshold, step, pos0, logits_slice.shape[1], stream, **variant)
+        return
     parts, keys = fork_vp_reduce(st, logits_slice, blk_lo, blk_hi, threshold, vocab_offset, step, pos0, stream, **variant)
     g_parts = gather_rank_major(parts, group)
     g_keys = gather_rank_major(keys, group) if keys is not None else None

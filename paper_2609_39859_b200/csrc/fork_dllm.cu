@@ -271,7 +271,10 @@ static fork_status check_workspace(void* ws, size_t bytes, int32_t B, int32_t Lt
   return FORK_OK;
 }
 
-struct VpLocal { int32_t vocab_offset; float4* part; float4* key; };
+struct VpLocal {
+  int32_t vocab_offset; float4* part; float4* key;
+  int32_t rank = 0, peers = 0; void* const* peer_parts = nullptr; void* const* peer_keys = nullptr;
+};
 
 /* ---- one-kernel steps: the control blocks ---------------------------------------------------
  * Part of the library's device image (zero when loaded), one per workspace address seen on a
@@ -373,7 +376,21 @@ static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const i
   rp.n_unmasked = a->n_unmasked; rp.is_fallback = a->is_fallback; rp.fallback_pos = a->fallback_pos;
   rp.nfe = a->nfe; rp.n_fallback = a->n_fallback;
   rp.fallback_mode = a->fallback_mode; rp.fallback_rand = a->fallback_rand;
-  if (vp) { rp.vocab_offset = vp->vocab_offset; rp.vp_part = vp->part; rp.vp_key = vp->key; }
+  if (vp) {
+    rp.vocab_offset = vp->vocab_offset; rp.vp_part = vp->part; rp.vp_key = vp->key;
+    rp.vp_rank = vp->rank; rp.vp_peers = vp->peers;
+    if (vp->peers > 0) {                                     /* the addresses go through the workspace (copied from a host
+                                                                temporary: staged by the runtime before the call returns) */
+      VpPeerTable tab;
+      memset(&tab, 0, sizeof(tab));
+      for (int j = 0; j < vp->peers; ++j) {
+        tab.part[j] = (float4*)vp->peer_parts[j];
+        tab.key[j] = vp->peer_keys ? (float4*)vp->peer_keys[j] : nullptr;
+      }
+      if (cudaMemcpyAsync(w.vp_peer_tab, &tab, sizeof(tab), cudaMemcpyHostToDevice, st) != cudaSuccess) return FORK_ERR_CUDA;
+      rp.vp_peer_tab = w.vp_peer_tab;
+    }
+  }
   if (ctl) {
     rp.ctl = ctl; rp.ticket = ctl->ticket; rp.blk_lo = lo; rp.blk_hi = hi; rp.commit_bits = w.commit_bits;
     rp.W = W; rp.Gv = G; rp.late_g = g_tune[FORK_TUNE_LATE_CTA].load();
@@ -843,6 +860,26 @@ extern "C" fork_status fork_vp_reduce(const fork_step_args* a, int32_t vocab_off
   if (s != FORK_OK) return s;
   if (a->B == 0) return FORK_OK;
   VpLocal vp{vocab_offset, (float4*)part_out, (float4*)key_out};
+  return step_impl(a, a->blk_lo, a->blk_hi, ws, (cudaStream_t)stream, &vp);
+}
+
+extern "C" fork_status fork_vp_reduce_peers(const fork_step_args* a, int32_t vocab_offset, int32_t rank, int32_t n_ranks,
+                                            void* const* peer_parts, void* const* peer_keys,
+                                            void* ws, size_t ws_bytes, void* stream) {
+  fork_status s = check_step_args(a, true);
+  if (s != FORK_OK) return s;
+  if (!peer_parts || n_ranks <= 0 || n_ranks > FORK_VP_MAX_RANKS || rank < 0 || rank >= n_ranks) return FORK_ERR_INVALID_ARG;
+  if (vocab_offset < 0 || (int64_t)vocab_offset + a->V > 0x7fffffffLL) return FORK_ERR_INVALID_ARG;
+  if (a->temperature > 0.f && !peer_keys) return FORK_ERR_INVALID_ARG;
+  for (int j = 0; j < n_ranks; ++j) {
+    if (!peer_parts[j] || ((uintptr_t)peer_parts[j] % 16) != 0) return FORK_ERR_INVALID_ARG;
+    if (a->temperature > 0.f && (!peer_keys[j] || ((uintptr_t)peer_keys[j] % 16) != 0)) return FORK_ERR_INVALID_ARG;
+  }
+  s = check_workspace(ws, ws_bytes, a->B, a->Lt);
+  if (s != FORK_OK) return s;
+  if (a->B == 0) return FORK_OK;
+  VpLocal vp{vocab_offset, nullptr, nullptr};
+  vp.rank = rank; vp.peers = n_ranks; vp.peer_parts = peer_parts; vp.peer_keys = a->temperature > 0.f ? peer_keys : nullptr;
   return step_impl(a, a->blk_lo, a->blk_hi, ws, (cudaStream_t)stream, &vp);
 }
 

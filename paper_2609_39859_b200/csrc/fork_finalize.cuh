@@ -254,8 +254,18 @@ __device__ void finalize_vp_local(const ReduceParams& p, const RowMap& rm, const
         kout = make_float4(kp.key, __int_as_float(p.vocab_offset + si), xs, 0.f);
       }
     }
-    p.vp_part[at] = out;
-    if (SAMPLE) p.vp_key[at] = kout;
+    if (p.vp_peers > 0) {
+      /* the exchange itself: plain 16-byte stores into every rank's gather buffer, the remote ones
+         over NVLink while the rest of the reduction goes on; nothing is ever loaded from a peer */
+      const size_t slot = (size_t)p.vp_rank * ((size_t)p.B * p.Lt) + at;
+      for (int j = 0; j < p.vp_peers; ++j) {
+        p.vp_peer_tab->part[j][slot] = out;
+        if (SAMPLE) p.vp_peer_tab->key[j][slot] = kout;
+      }
+    } else {
+      p.vp_part[at] = out;
+      if (SAMPLE) p.vp_key[at] = kout;
+    }
   }
 }
 

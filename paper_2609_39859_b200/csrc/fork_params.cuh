@@ -37,6 +37,8 @@ struct WsHeader {                    /* 256 bytes at the start of the workspace 
 };
 static_assert(sizeof(WsHeader) == 256, "header size");
 
+struct VpPeerTable { float4* part[FORK_VP_MAX_RANKS]; float4* key[FORK_VP_MAX_RANKS]; };
+
 struct WsView {
   WsHeader* hdr;
   int32_t* seq_off;                  /* [B+1] first row of each sequence */
@@ -49,6 +51,7 @@ struct WsView {
   float4* parts;                     /* [B*Lt + FORK_MAX_GRID] partial results, slot r+g */
   float2* kparts;                    /* [B*Lt + FORK_MAX_GRID] best perturbed key of each part (stochastic candidates) */
   uint32_t* commit_bits;             /* [B * ceil(Lt/32)] positions committed by a step whose mask update was handed on */
+  VpPeerTable* vp_peer_tab;          /* gather-buffer addresses of a vocabulary-parallel reduction with the exchange fused in */
   size_t bytes;
 };
 
@@ -70,6 +73,7 @@ static WsView ws_view(void* base, int32_t B, int32_t Lt) {
   v.parts = (float4*)(p + off); off = align_up(off + (rows + FORK_MAX_GRID) * sizeof(float4), 256);
   v.kparts = (float2*)(p + off); off = align_up(off + (rows + FORK_MAX_GRID) * sizeof(float2), 256);
   v.commit_bits = (uint32_t*)(p + off); off = align_up(off + nb * (size_t)(((Lt > 0 ? Lt : 1) + 31) / 32) * 4, 256);
+  v.vp_peer_tab = (VpPeerTable*)(p + off); off = align_up(off + sizeof(VpPeerTable), 256);
   v.bytes = off;
   return v;
 }
@@ -106,29 +110,36 @@ struct RowSource {                   /* where the logits rows are */
   int pos0, Ll, V;
 };
 
+/* Every kernel of the library takes this block, and at the start of a launch -- cold caches, the
+   critical path of every CTA -- each 64-byte line of it that is touched costs a trip to the constant
+   cache's backing store: what the start of the streaming kernels reads comes first and together;
+   what only the finalisation reads comes last. */
 struct ReduceParams {
+  /* read on the way to the first copy */
   RowSource src;
   int B, Lt, C, fast;
-  /* workspace */
-  WsHeader* hdr; const int32_t* seq_off; const int32_t* expected; int32_t* ticket;
-  const int2* rows; float4* final_rec; float4* parts; float2* kparts;
-  /* step mode */
-  int32_t* tokens; uint8_t* mask; float threshold; int32_t step;
+  FusedCtl* ctl; uint8_t* mask; const int32_t* blk_lo; const int32_t* blk_hi;   /* one-kernel step (ctl != NULL): control block, block bounds */
+  int W, Gv, late_g;                 /* ... words per sequence of the window bitmaps, virtual CTAs of the launch, and
+                                        late_g - 1 = a virtual CTA that dawdles before its snapshot (a test hook; 0 = none) */
+  int vocab_offset;                  /* vocabulary-parallel slices: global index of entry 0 of this buffer */
+  WsHeader* hdr; const int2* rows; const int32_t* seq_off; const int32_t* expected; int32_t* ticket;   /* workspace */
+  float noise_c; int32_t step; unsigned long long sample_seed;   /* stochastic candidates: log2(e)/tau and the noise stream */
+  /* read at segment ends and in the finalisation */
+  float4* parts; float2* kparts; float4* final_rec; uint32_t* commit_bits;
+  int32_t* tokens; float threshold; int fallback_mode; const uint32_t* fallback_rand;
   float* conf; int32_t* cand; float* entropy; float* logp; uint32_t* row_status;
   int32_t* commit_step; uint8_t* commit_fallback; float* commit_logp;
   int32_t* n_unmasked; uint8_t* is_fallback; int32_t* fallback_pos; int32_t* nfe; int32_t* n_fallback;
-  int fallback_mode; const uint32_t* fallback_rand;
-  float noise_c; unsigned long long sample_seed;      /* stochastic candidates: log2(e)/tau and the noise stream */
   /* vocabulary-parallel slices */
-  int vocab_offset;                  /* global index of entry 0 of this buffer */
   float4* vp_part; float4* vp_key;   /* [B,Lt] local phase: per-position results for the exchange instead of the unmask rule */
   const float4* vp_parts_in; const float4* vp_keys_in; int vp_ranks;   /* select phase: gathered [ranks][B,Lt] */
+  /* local phase with the exchange fused in (vp_peers > 0): the gather buffers [vp_peers][B,Lt] of all
+     ranks as this GPU addresses them (its own, and peer-mapped memory); slot vp_rank of each is
+     written.  The addresses sit in the workspace, not here: the size of this block is felt at
+     every launch. */
+  const VpPeerTable* vp_peer_tab; int vp_rank, vp_peers;
   /* log-probability mode */
   const int32_t* lp_tokens; float* lp_out; float* seq_sum; int32_t* seq_cnt; float* lse_out;
-  /* one-kernel step (ctl != NULL): the block bounds, the control block, words per sequence of the
-     window bitmaps, virtual CTAs of the launch; late_g - 1 = a virtual CTA that dawdles before its
-     snapshot (testing the handed-on mask update), 0 = none */
-  FusedCtl* ctl; const int32_t* blk_lo; const int32_t* blk_hi; uint32_t* commit_bits; int W, Gv, late_g;
 };
 
 /* Row r of the step -> (sequence, position).  Two-kernel step: the lists the set-up kernel wrote.

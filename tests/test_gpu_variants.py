@@ -408,3 +408,61 @@ def test_vocab_parallel_with_drawn_candidates_and_other_fallback_orders(n_ranks)
         compare_step_state(g, o)
         done += 1
     assert done >= 6
+
+
+@pytest.mark.parametrize("n_ranks,variant", [(2, {}), (4, dict(temperature=0.9, sample_seed=11)), (8, dict(fallback_mode=1))])
+def test_vocab_parallel_with_the_exchange_fused_into_the_reduction(n_ranks, variant):
+    """fork_vp_reduce_peers: every (emulated) rank's reduction kernel stores its slice results into
+    slot `rank` of every rank's gather buffer; afterwards all gather buffers are identical and the
+    select phase on each rank's own buffer reproduces the full-vocabulary oracle.  The ranks run one
+    after the other on one GPU, each with its own replica of the state; the "peer" buffers are
+    ordinary tensors of the same device."""
+    pkg = F()
+    done = 0
+    for seed in range(8):
+        rng = np.random.default_rng(500 + 10 * n_ranks + seed)
+        B, Lt, V = 3, 40, 6151
+        mask = (rng.random((B, Lt)) < 0.8).astype(np.uint8)
+        lo = rng.integers(0, 6, size=B).astype(np.int32)
+        hi = (lo + rng.integers(0, 34, size=B)).astype(np.int32)
+        x = make_rows(rng, (B, Lt), V, "bf16", peak=6.0)
+        o = oracle.StepState(B, Lt, mask=mask)
+        assert oracle.step(o, x, lo, hi, 0.9, step_id=4, **variant) == 0
+        if not decisions_are_clear(o, live_mask(mask, lo, hi), 0.9, 1e-4, variant.get("fallback_mode", 0),
+                                   variant.get("temperature", 0.0)):
+            continue
+        xt = to_torch_logits(x)
+        lo_d, hi_d = torch.from_numpy(lo).cuda(), torch.from_numpy(hi).cuda()
+        sampled = variant.get("temperature", 0.0) > 0
+        gp = [torch.full((n_ranks, B, Lt, 4), float("nan"), device="cuda") for _ in range(n_ranks)]
+        gk = [torch.full((n_ranks, B, Lt, 4), float("nan"), device="cuda") for _ in range(n_ranks)] if sampled else None
+        states = [pkg.ForkState(B, Lt, mask=mask) for _ in range(n_ranks)]
+        for r, (off, n) in enumerate(pkg.vocab_shards(V, n_ranks, xt.element_size())):
+            pkg.fork_vp_reduce_peers(states[r], xt[:, :, off:off + n], lo_d, hi_d, 0.9, off, r, gp, gk, step=4, **variant)
+        torch.cuda.synchronize()                                # stands for the barrier among real ranks
+        for j in range(1, n_ranks):
+            assert gp[j].cpu().numpy().tobytes() == gp[0].cpu().numpy().tobytes()
+        for j in range(n_ranks):
+            assert (states[j].mask.cpu().numpy() == mask).all()  # the local phase commits nothing
+            pkg.fork_vp_select(states[j], gp[j], gk[j] if sampled else None, lo_d, hi_d, 0.9, step=4, Ll=Lt, **variant)
+        torch.cuda.synchronize()
+        for j in range(n_ranks):
+            compare_step_state(states[j].host(), o)
+        done += 1
+        if done == 2:
+            return
+    raise AssertionError("no input with clear margins found")
+
+
+def test_fused_exchange_rejects_bad_arguments():
+    pkg = F()
+    st = pkg.ForkState(1, 8)
+    x = torch.zeros((1, 8, 64), dtype=torch.float32, device="cuda")
+    lo, hi = torch.zeros(1, dtype=torch.int32).cuda(), torch.full((1,), 8, dtype=torch.int32).cuda()
+    buf = [torch.zeros((2, 1, 8, 4), device="cuda") for _ in range(2)]
+    with pytest.raises(pkg.ForkError):                         # rank outside the group
+        pkg.fork_vp_reduce_peers(st, x, lo, hi, 0.9, 0, 2, buf)
+    with pytest.raises(pkg.ForkError):                         # drawn candidates need key buffers
+        pkg.fork_vp_reduce_peers(st, x, lo, hi, 0.9, 0, 0, buf, None, temperature=0.7, sample_seed=1)
+    with pytest.raises(pkg.ForkError):                         # a null peer address
+        pkg.fork_vp_reduce_peers(st, x, lo, hi, 0.9, 0, 0, [buf[0], 0])
