@@ -87,7 +87,7 @@ constexpr int kMaxStages = 13;
 constexpr int kHalves = 2;                                 /* independent producer/consumer groups per CTA */
 constexpr int kHalfThreads = (kCW + 2) * 32;
 constexpr uint32_t kSpinLimit = 1u << 22;
-constexpr int ring_stage_bytes() { return kCW * 32 * kUnroll * 16; }     /* 16 KB */
+__host__ __device__ constexpr int ring_stage_bytes() { return kCW * 32 * kUnroll * 16; }     /* 16 KB */
 
 constexpr int kSegRing = 16;                               /* > stages: the producer is never that many segments ahead */
 struct RingSmem {
