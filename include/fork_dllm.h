@@ -24,7 +24,8 @@
  *   - All data pointers are DEVICE pointers owned by the caller unless a comment says "host".
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  fork_step and
  *     fork_logprob only enqueue work on it and return; results are in device memory once the
- *     stream reaches that point.  They never synchronise, allocate or free.
+ *     stream reaches that point.  They never synchronise, and never allocate or free device
+ *     memory (the first call with a new workspace address adds an entry to a small host table).
  *   - `workspace` is device scratch of at least fork_workspace_bytes(B, Lt) bytes, 256-byte
  *     aligned, private to one call at a time on one stream; its contents need not be kept
  *     between calls (fork_decode_loop keeps its block cursors there while it runs) and need
@@ -276,10 +277,11 @@ fork_status fork_vp_reduce_peers(const fork_step_args* args, int32_t vocab_offse
  *     positions fits).
  *   - The first call on each device looks up the array's device address (one cudaGetSymbolAddress,
  *     with that device current) and caches it; make that first call outside any stream capture.
- *   - All calls on a device share the one array, which simply keeps what the previous call left:
- *     the step's first kernel re-initialises everything it reads (row list, offsets, ticket
- *     counters are cleared), so back-to-back calls on one stream are fine, but two calls that can
- *     overlap on the GPU (different streams, or different threads without ordering) race on it.
+ *   - All calls on a device share the one array (and one control block reserved for it), which
+ *     simply keep what the previous call left: a step reads nothing there that it has not written
+ *     itself, and leaves the counters of the control block as it found them, so back-to-back calls
+ *     on one stream are fine, but two calls that can overlap on the GPU (different streams, or
+ *     different threads without ordering) race on it.
  */
 #define FORK_STATIC_SCRATCH_BYTES (2u * 1024u * 1024u)
 fork_status fork_step_static(const fork_step_args* args, void* stream);

@@ -285,11 +285,11 @@ struct VpLocal {
  * whether a launch or a CUDA graph still refers to it); when all are taken, further workspace
  * addresses run the two-kernel step. */
 constexpr int kFusedSlots = 1024;
-static __device__ FusedCtl g_fused_ctl[kFusedSlots];
+static __device__ FusedCtl g_fused_ctl[kFusedSlots + 1];   /* the last one belongs to the library's own static scratch */
 struct FusedTable {
   FusedCtl* base = nullptr;
   std::unordered_map<const void*, int> slot_of;
-  int Gv[kFusedSlots] = {};
+  int Gv[kFusedSlots + 1] = {};
   int n_used = 0;                     /* blocks handed out at least once */
   int free_list[kFusedSlots] = {};    /* ... and given back */
   int n_free = 0;
@@ -300,7 +300,7 @@ static std::mutex g_fused_mu;
 /* The control block of workspace `ws` for launches of Gv virtual CTAs; NULL if none is left.
    `started` is only meaningful modulo the launch size: when that changes it is put back to zero,
    in stream order. */
-static FusedCtl* fused_ctl_for(const void* ws, int Gv, cudaStream_t st, bool* cuda_ok) {
+static FusedCtl* fused_ctl_for(const void* ws, int Gv, cudaStream_t st, bool* cuda_ok, bool own_scratch) {
   *cuda_ok = true;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { *cuda_ok = false; return nullptr; }
@@ -312,8 +312,11 @@ static FusedCtl* fused_ctl_for(const void* ws, int Gv, cudaStream_t st, bool* cu
     t.base = (FusedCtl*)p;
   }
   int i;
-  auto it = t.slot_of.find(ws);
-  if (it != t.slot_of.end()) {
+  auto it = own_scratch ? t.slot_of.end() : t.slot_of.find(ws);
+  if (own_scratch) {
+    i = kFusedSlots;                  /* no table entry, no host allocation: fork_step_static promises none */
+    if (t.Gv[i] == 0) t.Gv[i] = Gv;
+  } else if (it != t.slot_of.end()) {
     i = it->second;
   } else {
     if (t.n_free > 0) i = t.free_list[--t.n_free];
@@ -329,7 +332,7 @@ static FusedCtl* fused_ctl_for(const void* ws, int Gv, cudaStream_t st, bool* cu
 }
 
 static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const int32_t* hi, void* ws,
-                             cudaStream_t st, const VpLocal* vp = nullptr) {
+                             cudaStream_t st, const VpLocal* vp = nullptr, bool own_scratch = false) {
   DeviceInfo* dev;
   if (!device_info(&dev)) return FORK_ERR_CUDA;
   WsView w = ws_view(ws, a->B, a->Lt);
@@ -347,7 +350,7 @@ static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const i
   if (!vp && lo && hi && fast && (v == 0 || v == 2) && g_tune[FORK_TUNE_ONE_KERNEL].load() >= 0 &&
       a->B <= kFuseMaxB && W <= kFuseMaxSeqWords && (long long)a->B * W <= kFuseMaxWords) {
     bool cuda_ok;
-    ctl = fused_ctl_for(ws, G, st, &cuda_ok);
+    ctl = fused_ctl_for(ws, G, st, &cuda_ok, own_scratch);
     if (!cuda_ok) return FORK_ERR_CUDA;
   }
 
@@ -566,9 +569,9 @@ extern "C" fork_status fork_step_static(const fork_step_args* a, void* stream) {
   void* ws = nullptr;
   s = static_scratch(&ws);
   if (s != FORK_OK) return s;
-  /* nothing in the scratch has to survive from call to call: the active-set kernel rewrites the
-     row list and offsets and clears the per-sequence ticket counters at the start of every step */
-  return step_impl(a, a->blk_lo, a->blk_hi, ws, (cudaStream_t)stream);
+  /* nothing in the scratch has to survive from call to call: what a step reads there it has
+     written itself; the one-kernel step's control block is a reserved one of the library's */
+  return step_impl(a, a->blk_lo, a->blk_hi, ws, (cudaStream_t)stream, nullptr, true);
 }
 
 /* ---- top-entropy position selection (JustGRPO-Fast; Section 3.2, last paragraph) ------------ */
