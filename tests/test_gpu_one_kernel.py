@@ -226,3 +226,38 @@ def test_the_limits_of_the_one_kernel_step(B, Ll, kernels):
     want = oracle.StepState(B, Lt, mask=mask)
     assert oracle.step(want, x, lo, hi, 0.9, step_id=3) == 0
     compare_step_state(st.host(), want)
+
+
+def test_steps_of_different_states_overlapping_on_three_streams():
+    """Kernels of different steps share the SMs: the CTAs of one launch then start at very different
+    times without any test hook (in a ten-minute run of this pattern mask updates were handed on
+    dozens of times).  Each state has its own workspace, hence its own control block."""
+    pkg = F()
+    rng = np.random.default_rng(48)
+    streams = [torch.cuda.Stream() for _ in range(3)]
+    for _ in range(6):
+        cases = []
+        for s in streams:
+            B, Lt = int(rng.integers(1, 9)), int(rng.choice([16, 32]))
+            V = int(rng.choice([20000, 126464]))
+            xs = [make_rows(rng, (B, Lt), V, "bf16", peak_frac=0.5) for _ in range(3)]
+            mask = (rng.random((B, Lt)) < 0.8).astype(np.uint8)
+            lo = rng.integers(0, Lt // 2, B).astype(np.int32)
+            hi = (lo + rng.integers(1, 33, B)).astype(np.int32)
+            want = oracle.StepState(B, Lt, mask=mask)
+            clear = True
+            for i, x in enumerate(xs):
+                assert oracle.step(want, x, lo, hi, 0.9, step_id=i) == 0
+                live = np.isfinite(want.conf)
+                clear &= bool((np.abs(want.conf[live] - np.float64(np.float32(0.9))) >= 1e-4).all())
+            if clear:
+                cases.append((s, pkg.ForkState(B, Lt, mask=mask), [to_torch_logits(x) for x in xs],
+                              torch.from_numpy(lo).cuda(), torch.from_numpy(hi).cuda(), want))
+        torch.cuda.synchronize()
+        for i in range(3):
+            for s, st, xt, lo_t, hi_t, _ in cases:
+                pkg.fork_step(st, xt[i], lo_t, hi_t, 0.9, step=i, stream=s)
+        torch.cuda.synchronize()
+        for _, st, _, _, _, want in cases:
+            assert not (pkg.fork_device_status(st) & pkg.FORK_DEV_TIMEOUT)
+            compare_step_state(st.host(), want)
