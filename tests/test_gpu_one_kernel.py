@@ -230,7 +230,7 @@ def test_the_limits_of_the_one_kernel_step(B, Ll, kernels):
 
 def test_steps_of_different_states_overlapping_on_three_streams():
     """Kernels of different steps share the SMs: the CTAs of one launch then start at very different
-    times without any test hook (in a ten-minute run of this pattern mask updates were handed on
+    times without any test hook (in a five-minute run of this pattern mask updates were handed on
     dozens of times).  Each state has its own workspace, hence its own control block."""
     pkg = F()
     rng = np.random.default_rng(48)
