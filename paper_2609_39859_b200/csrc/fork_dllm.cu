@@ -347,7 +347,7 @@ static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const i
   const int W = (a->Ll + 31) / 32;
   FusedCtl* ctl = nullptr;
   const int v = g_tune[FORK_TUNE_VARIANT].load();
-  if (!vp && lo && hi && fast && (v == 0 || v == 2) && g_tune[FORK_TUNE_ONE_KERNEL].load() >= 0 &&
+  if (lo && hi && fast && (v == 0 || v == 2) && g_tune[FORK_TUNE_ONE_KERNEL].load() >= 0 &&
       a->B <= kFuseMaxB && W <= kFuseMaxSeqWords && (long long)a->B * W <= kFuseMaxWords) {
     bool cuda_ok;
     ctl = fused_ctl_for(ws, G, st, &cuda_ok, own_scratch);
@@ -376,7 +376,7 @@ static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const i
   rp.tokens = a->tokens; rp.mask = a->mask; rp.threshold = a->threshold; rp.step = a->step;
   rp.conf = a->conf; rp.cand = a->cand; rp.entropy = a->entropy; rp.logp = a->logp; rp.row_status = a->row_status;
   rp.commit_step = a->commit_step; rp.commit_fallback = a->commit_fallback; rp.commit_logp = a->commit_logp;
-  rp.n_unmasked = a->n_unmasked; rp.is_fallback = a->is_fallback; rp.fallback_pos = a->fallback_pos;
+  if (!vp) { rp.n_unmasked = a->n_unmasked; rp.is_fallback = a->is_fallback; rp.fallback_pos = a->fallback_pos; }   /* (the local phase of a vocabulary-parallel step decides nothing) */
   rp.nfe = a->nfe; rp.n_fallback = a->n_fallback;
   rp.fallback_mode = a->fallback_mode; rp.fallback_rand = a->fallback_rand;
   if (vp) {
