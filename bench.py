@@ -39,7 +39,7 @@ L2_BYTES = 126 * 1024 * 1024
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the streaming kernel, from the committed
 # ncu captures (profiles/reduce_select_ring_bf16_b8_and_passk.md)
-NCU_TRAFFIC_BYTES = {"b8": 65_057_792, "passk": 522_074_112}
+NCU_TRAFFIC_BYTES = {"b8": 65_025_536, "passk": 522_427_392}
 FALLBACK_HBM_GBS = 6650.0
 
 
