@@ -1,10 +1,14 @@
 #!/usr/bin/env python
 """Benchmark of the Fork-dLLM confidence pass (fork_step) on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload b8|passk|sweep]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload passk|b8|sweep]
 
-A "step" is one fork_step call (active-set kernel + streaming reduce/select/commit kernel) on a
-batch whose active block is fully masked: B*block_len live rows, each V logits read once.
+A "step" is one fork_step call (one kernel launch: the streaming reduce/select/commit kernel that
+also derives the active set) on a batch whose active block is fully masked: B*block_len live rows,
+each V logits read once.  The default workload is the pass@k rollout shape (B=64, V=126464 bf16:
+2048 live rows, 518 MB per launch).  The K steps are timed as one chunk between two CUDA events;
+chunks are repeated until at least half a second of GPU time has been measured, and the line
+reports the median chunk (with the spread over chunks).
 Prints ONE JSON line (rank 0).  `value` is masked positions per second with the logits already in
 HBM; `e2e` is the same metric through fork_step_host with pinned HOST buffers (H2D of the logits
 window and D2H of every output inside the timed region); `roofline` is the streaming kernel's
@@ -37,9 +41,13 @@ METRIC = "masked positions/s (fork_step; HBM GB/s and fraction of peak in `roofl
 UNIT = "positions/s"
 L2_BYTES = 126 * 1024 * 1024
 NOMINAL_HBM_GBS = 8000.0
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the streaming kernel, from the committed
-# ncu captures (profiles/reduce_select_ring_bf16_b8_and_passk.md)
-NCU_TRAFFIC_BYTES = {"b8": 65_025_536, "passk": 522_427_392}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the streaming kernel (arg-max candidates),
+# from one ncu capture of that workload; `source` names the summary that holds it.  A shape without a
+# capture of its own reports null.
+NCU_TRAFFIC = {
+    "b8": {"bytes": 65_025_536, "source": "ncu capture of this workload: profiles/reduce_select_ring_bf16_b8_and_passk.md"},
+    "passk": {"bytes": 522_427_392, "source": "ncu capture of this workload: profiles/reduce_select_ring_bf16_b8_and_passk.md"},
+}
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -159,10 +167,12 @@ def reset_states(states):
     states[0].pool_mask[:len(states)].fill_(1)
 
 
-def time_full_block(w, seed, steps, warmup, device, use_graph=True, variant=None):
-    """Times `steps` fork_step calls (after `warmup`), each on B*block_len live rows.  The timed
-    steps are replayed from one CUDA graph when `use_graph` (host launch cost would otherwise bound
-    a ~10 us step); a second, un-graphed pass brackets each step's streaming kernel with events."""
+def time_full_block(w, seed, steps, warmup, device, use_graph=False, variant=None, min_gpu_s=0.5, max_chunks=4000):
+    """Times chunks of `steps` fork_step calls (after `warmup`), each call on B*block_len live rows.
+    One chunk = exactly `steps` steps between two CUDA events on the launching stream (plain stream
+    launches with programmatic dependent launch, or one CUDA graph of the chunk when `use_graph`);
+    chunks repeat until `min_gpu_s` seconds of GPU time are on record.  The result carries the median
+    chunk and the spread; a last, separate pass brackets each step's streaming kernel with events."""
     import torch
     import paper_2609_39859_b200 as pkg
     rows = w.B * w.block_len
@@ -197,8 +207,8 @@ def time_full_block(w, seed, steps, warmup, device, use_graph=True, variant=None
     sp = C.c_void_p(stream.cuda_stream)
     run(warmup, 0, sp)
     torch.cuda.synchronize()
-    launches0 = pkg.fork_kernel_launches()
     graph = None
+    launches0 = pkg.fork_kernel_launches()
     if use_graph:
         try:
             graph = torch.cuda.CUDAGraph()
@@ -211,22 +221,48 @@ def time_full_block(w, seed, steps, warmup, device, use_graph=True, variant=None
     launches = pkg.fork_kernel_launches() - launches0 if graph is not None else None
     stream = torch.cuda.current_stream()
     sp = C.c_void_p(stream.cuda_stream)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def chunk(first):
+        """one timed chunk: exactly `steps` steps between two events; returns the event pair"""
+        nonlocal launches
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if graph is not None:
+            e0.record(stream)
+            graph.replay()
+            e1.record(stream)
+        else:
+            l0 = pkg.fork_kernel_launches()
+            if steps <= n_state:                   # the re-arm of the pool stays outside the events
+                reset_states(states[:steps])
+                e0.record(stream)
+                for j in range(steps):
+                    call(first + j, sp, s=j)
+                e1.record(stream)
+            else:
+                e0.record(stream)
+                run(steps, first, sp)
+                e1.record(stream)
+            launches = pkg.fork_kernel_launches() - l0
+        return e0, e1
+
     host_t0 = time.perf_counter()
-    if graph is not None:
-        e0.record(stream)
-        graph.replay()
-        e1.record(stream)
-    else:
-        launches0 = pkg.fork_kernel_launches()
-        e0.record(stream)
-        run(steps, warmup, sp)
-        e1.record(stream)
-        launches = pkg.fork_kernel_launches() - launches0
+    ev = chunk(warmup)
     host_submit_ms = (time.perf_counter() - host_t0) * 1e3
     torch.cuda.synchronize()
-    total_ms = e0.elapsed_time(e1)
-    # second pass: events around each step's streaming kernel (plain launches)
+    first_ms = ev[0].elapsed_time(ev[1])
+    times = [first_ms]
+    want = int(min(max_chunks, max(3, -(-min_gpu_s * 1e3 // max(first_ms, 1e-3)))))
+    pending = []
+    for c in range(1, want):
+        pending.append(chunk(warmup + c * steps))
+        if len(pending) >= 64:                     # bound the host's lead over the device
+            torch.cuda.synchronize()
+            times += [a.elapsed_time(b) for a, b in pending]
+            pending = []
+    torch.cuda.synchronize()
+    times += [a.elapsed_time(b) for a, b in pending]
+    total_ms = statistics.median(times)
+    # last pass: events around each step's streaming kernel (plain launches)
     n = min(steps, n_state)
     reset_states(states[:n])
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
@@ -238,8 +274,9 @@ def time_full_block(w, seed, steps, warmup, device, use_graph=True, variant=None
         L.fork_set_timing_events(C.c_void_p(evs[j][0].cuda_event), C.c_void_p(evs[j][1].cuda_event))
         call(warmup + j, sp, s=j)
     torch.cuda.synchronize()
-    kernel_ms = sum(a.elapsed_time(b) for a, b in evs) / n
+    kernel_ms = statistics.median(a.elapsed_time(b) for a, b in evs)
     return dict(rows=rows, row_bytes=row_bytes, total_ms=total_ms, ms_per_step=total_ms / steps,
+                chunks=len(times), chunk_ms_min=min(times), chunk_ms_max=max(times), gpu_s_timed=sum(times) * 1e-3,
                 kernel_ms=kernel_ms, launches=launches, n_buf=n_buf, graph=graph is not None,
                 host_submit_ms=host_submit_ms, setup=(cfg, bufs, states, lo, hi), keep=graph)
 
@@ -462,36 +499,119 @@ def time_select(device):
     return {"workload": "fork_select_top_entropy B=128 Lt=256 ratio 0.2", "ms": e0.elapsed_time(e1) / 20}
 
 
-def loop_stats(device):
-    """Full semi-autoregressive decode loops of the configurations (generator as the model): model
-    evaluations used versus tokens, share of tokens committed at fallback steps, live rows."""
+LOOP_BINS = ((1, 16), (17, 64), (65, 256), (257, 1024), (1025, 1 << 30))
+
+
+def live_rows_per_step(commit_step, block_len, steps):
+    """Live rows (masked positions inside the sequences' active blocks) at every step of a finished
+    decode loop, rebuilt from the per-position commit steps: a sequence works on its blocks in
+    order, each block from the step after the previous block's last commit to its own last commit,
+    and a position of the active block is live until the step that commits it."""
+    B, Lt = commit_step.shape
+    live = np.zeros(steps, np.int64)
+    for b in range(B):
+        start = 0
+        for s in range(0, Lt, block_len):
+            cs = commit_step[b, s:s + block_len]
+            cs = cs[cs >= 0]
+            if cs.size == 0:
+                continue
+            end = int(cs.max())
+            for n in range(start, end + 1):
+                live[n] += int((cs >= n).sum())
+            start = end + 1
+    return live
+
+
+def loop_stats(device, names=("b8", "passk")):
+    """Full semi-autoregressive decode loops (fork_decode_loop, the generator standing in for the
+    model) with CUDA events around every step's fork_step kernels and, separately, around the
+    generator: what the many short steps of a real decode cost."""
     import torch
     import fork_synth as fs
     import paper_2609_39859_b200 as pkg
+    L = pkg.lib()
     out = []
-    for name, lams in (("tiny", None), ("b8", None), ("passk", None), ("sweep", "all")):
+    for name in names:
         w = fs.workload(name)
-        for lam in (w.thresholds if lams == "all" else (w.threshold,)):
-            cfg = w.cfg()
-            tdt = torch.bfloat16 if w.dtype == fs.BF16 else torch.float32
-            logits = torch.empty((w.B, w.Lt, w.V), dtype=tdt, device=device)
-            fs.cuda_canary(logits.data_ptr(), logits.numel(), w.dtype, torch.cuda.current_stream().cuda_stream)
+        cfg = w.cfg()
+        tdt = torch.bfloat16 if w.dtype == fs.BF16 else torch.float32
+        logits = torch.empty((w.B, w.Lt, w.V), dtype=tdt, device=device)
+        stream = torch.cuda.current_stream()
+        fs.cuda_canary(logits.data_ptr(), logits.numel(), w.dtype, stream.cuda_stream)
+        row_bytes = w.V * w.es
+        cap = w.Lt + 16
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(cap)]
+        for q in ev:                                 # creates the CUDA events that are re-recorded below
+            for e in q:
+                e.record(stream)
+        torch.cuda.synchronize()
+        # pass 1: per-step CUDA events (the callback arms the library's timing hook and brackets the generator)
+        best = None
+        for rep in range(3):                         # the first repetition warms up; the fastest of the others is reported
             st = pkg.ForkState(w.B, w.Lt, device=device)
-            prov = fs.Provider(cfg, w.Lt * w.V, w.V, 0, w.Lt)
+            mask_ptr, logits_ptr = st.mask.data_ptr(), logits.data_ptr()
+
+            def provider(step, lo_ptr, hi_ptr, stream_p, ev=ev, mask_ptr=mask_ptr, logits_ptr=logits_ptr):
+                g0, g1, k0, k1 = ev[min(step, cap - 1)]
+                g0.record(stream)
+                fs.cuda_fill(cfg, step, mask_ptr, lo_ptr, hi_ptr, logits_ptr, w.Lt * w.V, w.V, 0, w.Lt, stream_ptr=stream_p)
+                g1.record(stream)
+                L.fork_set_timing_events(C.c_void_p(k0.cuda_event), C.c_void_p(k1.cuda_event))
+                return 0
+
+            rc, steps = pkg.fork_decode_loop(st, logits, w.block_len, 0, w.Lt, provider, None, w.threshold, cap - 8)
             torch.cuda.synchronize()
-            t0 = time.perf_counter()
-            rc, steps = pkg.fork_decode_loop(st, logits, w.block_len, 0, w.Lt, prov.address, prov.ctx, lam, 100000)
-            torch.cuda.synchronize()
-            dt = time.perf_counter() - t0
-            prov.close()
-            h = st.host()
-            out.append({"workload": name, "threshold": lam, "B": w.B, "tokens_per_sequence": w.Lt,
-                        "steps_taken": steps, "nfe_mean": float(h["nfe"].mean()),
-                        "fallback_token_share": float(h["commit_fallback"].mean()),
-                        "tokens_committed": int((h["commit_step"] >= 0).sum()),
-                        "wall_ms_incl_generator": dt * 1e3})
-            del logits
-            torch.cuda.empty_cache()
+            kern = np.array([ev[n][2].elapsed_time(ev[n][3]) for n in range(steps)])
+            gen = np.array([ev[n][0].elapsed_time(ev[n][1]) for n in range(steps)])
+            if rep > 0 and (best is None or kern.sum() < best[0].sum()):
+                best = (kern, gen, 0.0, steps, st.host())
+            st.close()
+        # pass 2: wall clock of the whole loop with the generator called from C (no events, no Python per step)
+        walls = {}
+        for ahead in (0, 4):                         # steps the host may enqueue beyond the last outcome it has read
+            pkg.fork_set_tuning(pkg.FORK_TUNE_LOOP_AHEAD, ahead)
+            for rep in range(4):
+                st = pkg.ForkState(w.B, w.Lt, device=device)
+                prov = fs.Provider(cfg, w.Lt * w.V, w.V, 0, w.Lt)
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                rc, steps2 = pkg.fork_decode_loop(st, logits, w.block_len, 0, w.Lt, prov.address, prov.ctx, w.threshold, cap - 8)
+                torch.cuda.synchronize()
+                wall_ms = (time.perf_counter() - t0) * 1e3
+                prov.close()
+                assert steps2 == best[3]
+                if rep > 0:
+                    walls[ahead] = min(walls.get(ahead, 1e30), wall_ms)
+                st.close()
+        pkg.fork_set_tuning(pkg.FORK_TUNE_LOOP_AHEAD, 0)
+        kern, gen, wall_ms, steps, h = best
+        live = live_rows_per_step(h["commit_step"], w.block_len, steps)
+        bins = []
+        for lo_r, hi_r in LOOP_BINS:
+            sel = (live >= lo_r) & (live <= hi_r)
+            if sel.any():
+                ms = float(kern[sel].sum())
+                bins.append({"live_rows": "%d-%s" % (lo_r, hi_r if hi_r < (1 << 30) else "up"), "steps": int(sel.sum()),
+                             "mean_us_per_step": ms * 1e3 / int(sel.sum()),
+                             "hbm_gbs": float(live[sel].sum()) * row_bytes / (ms * 1e-3) / 1e9})
+        total_rows, kern_ms = int(live.sum()), float(kern.sum())
+        out.append({"workload": "%s: full decode loop, B=%d, %d tokens per sequence in blocks of %d, threshold %.2f" %
+                                (name, w.B, w.Lt, w.block_len, w.threshold),
+                    "steps_taken": steps, "nfe_min_mean_max": [int(h["nfe"].min()), float(h["nfe"].mean()), int(h["nfe"].max())],
+                    "tokens_committed": int((h["commit_step"] >= 0).sum()),
+                    "fallback_token_share": float((h["commit_fallback"] == 1).mean()),
+                    "live_rows_total": total_rows, "fork_step_kernel_ms_total": kern_ms,
+                    "positions_per_s": total_rows / (kern_ms * 1e-3), "hbm_gbs": total_rows * row_bytes / (kern_ms * 1e-3) / 1e9,
+                    "mean_us_per_step": kern_ms * 1e3 / steps, "by_live_rows": bins,
+                    "generator_ms_total": float(gen.sum()),
+                    # whole loops by the host's clock, the generator called from C, no events: the host waits for every
+                    # step's outcome before the next model call (0), or enqueues up to 4 steps ahead of the outcomes
+                    "loop_wall_ms": walls[0], "loop_wall_ms_4_steps_ahead": walls[4],
+                    "wall_us_per_step": walls[0] * 1e3 / steps, "wall_us_per_step_4_steps_ahead": walls[4] * 1e3 / steps,
+                    "generator_us_per_step": float(gen.sum()) * 1e3 / steps})
+        del logits
+        torch.cuda.empty_cache()
     return out
 
 
@@ -524,36 +644,52 @@ def cpu_baseline(w, seed, target_cpu_seconds=12.0):
 
 
 def reference_arm(args):
-    """--impl reference: the fp64 oracle is the timed arm (host cores, rank 0 only)."""
+    """--impl reference: the fp64 oracle is the timed arm (host cores, rank 0 only).  A step is one
+    full-block step of the same workload; when K+W such steps would not end within a few minutes,
+    every step covers the first sequences of the batch only (`sample` says how many)."""
     rank, _, world = rank_info()
     if rank != 0:
         return 0
     import fork_synth as fs
     import oracle
     w = fs.workload(args.workload)
-    cfg = w.cfg()
     B, BL, V = w.B, w.block_len, w.V
-    logits = np.empty((B, BL, V), w.np_dtype)
-    mask = np.ones((B, w.Lt), np.uint8)
-    lo, hi = np.zeros(B, np.int32), np.full(B, BL, np.int32)
-    fs.fill_host(cfg, 0, mask, lo, hi, logits)
-    rows = B * BL
+    steps, warm = max(1, args.steps), max(0, args.warmup)
+
+    def inputs(nb):
+        cfg = w.cfg(B=nb)
+        logits = np.empty((nb, BL, V), w.np_dtype)
+        mask = np.ones((nb, w.Lt), np.uint8)
+        lo, hi = np.zeros(nb, np.int32), np.full(nb, BL, np.int32)
+        fs.fill_host(cfg, 0, mask, lo, hi, logits)
+        return logits, lo, hi
+
+    probe_b = min(B, 2)                                  # 2 sequences = 2*BL rows: enough to occupy the host cores
+    logits, lo, hi = inputs(probe_b)
+    t0 = time.perf_counter()
+    oracle.step(oracle.StepState(probe_b, w.Lt), logits, lo, hi, w.threshold)
+    per_row = (time.perf_counter() - t0) / (probe_b * BL)
+    budget_s = 150.0
+    nb = B
+    while nb > 1 and per_row * nb * BL * (steps + warm) > budget_s:
+        nb = max(1, nb // 2)
+    logits, lo, hi = inputs(nb)
+    rows = nb * BL
     cores = oracle.threads_used(0, rows)
-    steps = max(1, min(args.steps, 40))
-    warm = max(1, min(args.warmup, 3))
     for _ in range(warm):
-        oracle.step(oracle.StepState(B, w.Lt), logits, lo, hi, w.threshold)
+        oracle.step(oracle.StepState(nb, w.Lt), logits, lo, hi, w.threshold)
     t0 = time.perf_counter()
     for _ in range(steps):
-        oracle.step(oracle.StepState(B, w.Lt), logits, lo, hi, w.threshold)
+        oracle.step(oracle.StepState(nb, w.Lt), logits, lo, hi, w.threshold)
     dt = time.perf_counter() - t0
     value = rows * steps / dt
-    sample = "%d full-block steps (%d rows each) of workload %s on the host cores" % (steps, rows, w.name)
+    sample = ("%d full-block steps of workload %s on the host cores, each on %d of its %d sequences (%d rows)" %
+              (steps, w.name, nb, B, rows))
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
         "warmup": warm, "ms_per_step": dt * 1e3 / steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": workload_config(w, rows),
+        "config": workload_config(w, B * BL),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0}))
@@ -572,21 +708,23 @@ def workload_config(w, rows):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
-    ap.add_argument("--workload", default="b8", choices=["b8", "passk", "sweep"])
-    ap.add_argument("--no-extras", action="store_true", help="skip the other shapes, e2e and the CPU baseline")
-    ap.add_argument("--loops", action="store_true", help="also run the full decode loops of the configurations and report their statistics")
+    ap.add_argument("--workload", default="passk", choices=["b8", "passk", "sweep"])
+    ap.add_argument("--no-extras", action="store_true", help="skip the other shapes, the decode loops, e2e and the CPU baseline")
+    ap.add_argument("--min-gpu-seconds", type=float, default=0.5, help="repeat the K-step chunk until this much GPU time is on record")
     ap.add_argument("--graph", action="store_true", help="replay the K timed steps from one CUDA graph instead of plain stream launches")
-    ap.add_argument("--no-graph", action="store_true", help="(default) plain stream launches")
     ap.add_argument("--variant", type=int, default=0, help="0 auto, 1 direct loads, 2 bulk-copy shared-memory ring")
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--pdl", type=int, default=0, help="0 = programmatic dependent launch (default), -1 = off")
     ap.add_argument("--scoring-only", type=int, default=0, metavar="B",
                     help="run only the ForkGRPO scoring / objective / backward timings with B sequences (multiple of 8) and print them")
+    ap.add_argument("--loops-only", default="", metavar="NAMES", help="run only the decode loops of these workloads (comma separated) and print their statistics")
     ap.add_argument("--one-kernel", type=int, default=0, help="0 = small batches run the step as one kernel (default), -1 = always the set-up kernel first")
+    ap.add_argument("--min-units", type=int, default=0, help="0 = automatic; units of 2048 logits per participating CTA in small steps")
+    ap.add_argument("--l2-hint", type=int, default=0, help="0 = logits are copied with the L2 evict-first hint (default), -1 = no hint")
     ap.add_argument("--temperature", type=float, default=0.0,
                     help="time the step with stochastic candidates at this temperature (default 0: arg-max candidates)")
     args = ap.parse_args()
@@ -614,7 +752,13 @@ def main():
     pkg.fork_set_tuning(pkg.FORK_TUNE_STAGES, args.stages)
     pkg.fork_set_tuning(pkg.FORK_TUNE_PDL, args.pdl)
     pkg.fork_set_tuning(pkg.FORK_TUNE_ONE_KERNEL, args.one_kernel)
+    pkg.fork_set_tuning(pkg.FORK_TUNE_L2_EVICT_FIRST, args.l2_hint)
+    pkg.fork_set_tuning(pkg.FORK_TUNE_MIN_UNITS, args.min_units)
 
+    if args.loops_only:                                        # a profiling aid, not the benchmark line
+        if rank == 0:
+            print(json.dumps({"loops": loop_stats(device, tuple(args.loops_only.split(",")))}))
+        return 0
     if args.scoring_only:                                      # a profiling aid, not the benchmark line
         if rank == 0:
             print(json.dumps({"scoring_only": time_logprob(device, peak, B=args.scoring_only)}))
@@ -625,56 +769,64 @@ def main():
         dist.barrier()
     torch.cuda.synchronize()
     variant = dict(temperature=args.temperature, sample_seed=12345) if args.temperature > 0 else None
-    r = time_full_block(w, seed, steps, warmup, device, use_graph=args.graph and not args.no_graph, variant=variant)
+    r = time_full_block(w, seed, steps, warmup, device, use_graph=args.graph, variant=variant,
+                        min_gpu_s=args.min_gpu_seconds)
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
     max_ms = max_over_ranks(r["total_ms"], device)
-    # keep the same load running so that nvidia-smi (100 ms period) samples clocks under it
-    t_end = time.time() + 1.5
+    # nvidia-smi reports every 100 ms and its utilisation figure lags: keep the same load running a
+    # little longer so that samples under it exist
+    t_end = time.time() + 1.0
     while time.time() < t_end:
         time_full_block_again(r, w, pkg)
     torch.cuda.synchronize()
     clocks = sampler.stop() if sampler else None
 
     rows, row_bytes = r["rows"], r["row_bytes"]
+    ldt = "bf16" if w.es == 2 else "f32"
     value = aggregate(rows, steps, world, max_ms)
     step_gbs = rows * row_bytes / (r["ms_per_step"] * 1e-3) / 1e9
+    kernels_per_step = int(r["launches"]) // max(1, steps)
     # the event-bracketed duration includes the streaming kernel's launch latency (the events break the
     # dependent-launch chain); the kernel cannot take longer than the whole step that contains it
     kern_ms = min(r["kernel_ms"], r["ms_per_step"])
-    kern_src = "events around the kernel" if kern_ms == r["kernel_ms"] else "whole step (upper bound on the kernel; bracketing events add launch latency)"
+    kern_src = ("events around the kernel (median over the steps of one chunk)" if kern_ms == r["kernel_ms"] else
+                "whole step: the step is %d kernel launch(es), and the events that bracket a kernel break the "
+                "dependent-launch chain and add its launch latency (bracketed figure in kernel_ms_event_bracketed)" % kernels_per_step)
     kern_gbs = rows * row_bytes / (kern_ms * 1e-3) / 1e9
+    cap = NCU_TRAFFIC.get(args.workload) if not variant else None
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": max_ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic",
+        "dtype": ldt, "accumulate_dtype": "f32", "data": "synthetic",
         "config": dict(workload_config(w, rows),
-                       l2="inputs rotate over %d logits buffers (%.0f MB in total, > 2x the 126 MB L2)" %
-                          (r["n_buf"], r["n_buf"] * rows * row_bytes / 1e6),
-                       **({"candidates": "drawn at temperature %g (Gumbel-max in the same pass)" % args.temperature}
+                       **({"candidates": "drawn at temperature %g in the same pass" % args.temperature}
                           if args.temperature > 0 else {})),
+        "l2": "inputs rotate over %d logits buffers (%.0f MB in total, > 2x the 126 MB L2)" %
+              (r["n_buf"], r["n_buf"] * rows * row_bytes / 1e6),
+        "timing": {"chunk": "%d steps between two CUDA events" % steps, "chunks": r["chunks"],
+                   "gpu_seconds_timed": r["gpu_s_timed"], "reported": "median chunk",
+                   "ms_per_step_min": r["chunk_ms_min"] / steps, "ms_per_step_max": r["chunk_ms_max"] / steps},
         "launch": ("one CUDA graph of the K steps" if r["graph"] else "plain stream launches, programmatic dependent launch"),
-        "kernels_per_step": int(r["launches"]) // max(1, steps),
+        "kernels_per_step": kernels_per_step,
         "host_submit_ms_per_step": r["host_submit_ms"] / steps,
         "hbm_gbs_per_gpu": step_gbs, "frac_of_8TBs_nominal": step_gbs / NOMINAL_HBM_GBS,
         "gpu_launches": int(r["launches"]),
-        "roofline": {"bound": "hbm", "kernel": "reduce_select_ring_kernel<%s,step,8>" % ("bf16" if w.es == 2 else "f32"),
+        "roofline": {"bound": "hbm", "kernel": "reduce_select_ring_kernel<%s,%s>" % (ldt, "sample" if variant else "step"),
                      "achieved": kern_gbs, "peak": peak, "unit": "GB/s", "frac": kern_gbs / peak,
                      "peak_source": peak_src,
-                     # no capture of its own: the passk capture scaled by the bytes one launch streams
-                     # (traffic is the logits read once plus per-row results, both proportional to them)
-                     "traffic": NCU_TRAFFIC_BYTES.get(args.workload) or int(round(
-                         NCU_TRAFFIC_BYTES["passk"] / (2048 * 252928) * rows * row_bytes)),
-                     "traffic_source": ("ncu capture of this workload (profiles/)" if args.workload in NCU_TRAFFIC_BYTES
-                                        else "ncu capture of the passk workload scaled by algorithmic bytes"),
+                     "traffic": cap["bytes"] if cap else None,
+                     "traffic_source": (cap["source"] if cap else
+                                        "no ncu capture of this shape (the captured shapes: %s)" % ", ".join(sorted(NCU_TRAFFIC))),
                      "algorithmic_bytes_per_launch": rows * row_bytes, "kernel_ms": kern_ms, "kernel_ms_source": kern_src,
-                     "kernel_ms_event_bracketed": r["kernel_ms"],
+                     "kernel_ms_event_bracketed": r["kernel_ms"], "kernels_per_step": kernels_per_step,
                      "whole_step_gbs": step_gbs, "whole_step_frac": step_gbs / peak,
                      "frac_of_8TBs_nominal": kern_gbs / NOMINAL_HBM_GBS},
         "clocks": clocks,
     }
-    if rank == 0 and not args.no_extras:
+    extras = rank == 0 and not args.no_extras
+    if extras:
         e = time_e2e(w, r["setup"], steps, warmup, device)
         out["e2e"] = {"value": rows * world / (e["ms_per_step"] * 1e-3), "unit": UNIT,
                       "h2d_bytes_per_step": e["h2d"], "d2h_bytes_per_step": e["d2h"], "ms_per_step": e["ms_per_step"],
@@ -682,44 +834,65 @@ def main():
     r.pop("setup", None)
     r.pop("keep", None)
     torch.cuda.empty_cache()
-    if rank == 0 and not args.no_extras and world == 1:
-        also = []
+    if extras and world == 1:
+        also, summary = [], {}
 
-        def shape_line(w2, variant=None, label=""):
-            r2 = time_full_block(w2, w2.seed, steps, max(warmup, 5), device, use_graph=False, variant=variant)
+        def shape_line(key, w2, variant=None, label=""):
+            r2 = time_full_block(w2, w2.seed, steps, max(warmup, 5), device, use_graph=False, variant=variant, min_gpu_s=0.2)
             r2.pop("setup", None)
             r2.pop("keep", None)
             torch.cuda.empty_cache()
-            g2 = r2["rows"] * r2["row_bytes"] / (min(r2["kernel_ms"], r2["ms_per_step"]) * 1e-3) / 1e9
+            k2 = min(r2["kernel_ms"], r2["ms_per_step"])
+            g2 = r2["rows"] * r2["row_bytes"] / (k2 * 1e-3) / 1e9
             s2 = r2["rows"] * r2["row_bytes"] / (r2["ms_per_step"] * 1e-3) / 1e9
+            summary[key] = {"us_per_step": round(r2["ms_per_step"] * 1e3, 2), "frac": round(g2 / peak, 4)}
             return {"workload": workload_config(w2, r2["rows"])["workload"] + label,
                     "positions_per_s": r2["rows"] / (r2["ms_per_step"] * 1e-3), "ms_per_step": r2["ms_per_step"],
+                    "ms_per_step_min_max": [r2["chunk_ms_min"] / steps, r2["chunk_ms_max"] / steps], "chunks": r2["chunks"],
                     "whole_step_gbs": s2, "whole_step_frac_of_measured_peak": s2 / peak,
                     "kernel_gbs": g2, "kernel_frac_of_measured_peak": g2 / peak,
                     "kernel_frac_of_8TBs_nominal": g2 / NOMINAL_HBM_GBS,
-                    "logits_per_s": r2["rows"] * w2.V / (min(r2["kernel_ms"], r2["ms_per_step"]) * 1e-3)}
+                    "logits_per_s": r2["rows"] * w2.V / (k2 * 1e-3)}
 
-        for name in ("b8", "passk", "sweep"):
+        summary[args.workload] = {"us_per_step": round(r["ms_per_step"] * 1e3, 2), "frac": round(kern_gbs / peak, 4)}
+        for name in ("passk", "b8", "sweep"):
             if name != args.workload:
-                also.append(shape_line(fs.workload(name)))
+                also.append(shape_line(name, fs.workload(name)))
         # not one of the five configurations: the pass@k recipe at twice the batch, where the fixed cost
         # of a launch weighs half as much (how far the streaming rate itself is from the HBM ceiling)
         import dataclasses
-        also.append(shape_line(dataclasses.replace(fs.workload("passk"), name="passk recipe at B=128", B=128)))
-        # the paper's rollout setting: candidates drawn at temperature 0.8 inside the same pass (ALU-bound)
+        also.append(shape_line("passk_B128", dataclasses.replace(fs.workload("passk"), name="passk recipe at B=128", B=128)))
+        # the paper's rollout setting: candidates drawn at temperature 0.8 inside the same pass
         for name in ("b8", "passk"):
-            also.append(shape_line(fs.workload(name), dict(temperature=0.8, sample_seed=12345),
+            also.append(shape_line(name + "_tau0.8", fs.workload(name), dict(temperature=0.8, sample_seed=12345),
                                    " -- stochastic candidates, tau=0.8"))
-        also.extend(time_logprob(device, peak))
+        lp = time_logprob(device, peak)
+        summary["grpo_logprob"] = {"us_per_call": round(lp[0]["ms"] * 1e3, 1), "frac": round(lp[0]["frac_of_measured_peak"], 4)}
+        summary["grpo_backward"] = {"us_per_call": round(lp[2]["ms"] * 1e3, 1), "frac": round(lp[2]["frac_of_measured_peak"], 4)}
+        also.extend(lp)
         also.append(time_select(device))
-        also.append(time_vocab_parallel(device, peak))
-        out["also"] = also
+        vp = time_vocab_parallel(device, peak)
+        summary["vp_reduce_slice"] = {"us_per_call": round(vp["reduce_ms"] * 1e3, 1), "frac": round(vp["slice_gbs"] / peak, 4)}
+        also.append(vp)
         ro = read_only_ceiling(device)
         out["roofline"]["read_only_ceiling_gbs"] = ro          # the library's own read-only streaming probe, same run
         out["roofline"]["frac_of_read_only_ceiling"] = kern_gbs / ro
+        loops = loop_stats(device)
+        for q in loops:
+            summary["loop_" + q["workload"].split(":")[0]] = {"steps": q["steps_taken"], "kernel_us_per_step": round(q["mean_us_per_step"], 2),
+                                                              "hbm_gbs": round(q["hbm_gbs"], 1),
+                                                              "wall_us_per_step_incl_generator": round(q["wall_us_per_step"], 1)}
         out["cpu_baseline"] = cpu_baseline(w, seed)
-        if args.loops:
-            out["loops"] = loop_stats(device)
+        # what a truncated copy of this line must still carry comes first: every shape as (time, fraction of the peak)
+        head = {k: out[k] for k in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better",
+                                    "scaling", "vs_baseline", "dtype", "accumulate_dtype", "data", "config")}
+        head["also_summary"] = summary
+        for k, v in out.items():
+            if k not in head:
+                head[k] = v
+        head["loops"] = loops
+        head["also"] = also
+        out = head
     if rank == 0:
         print(json.dumps(out))
     if world > 1:

@@ -299,12 +299,23 @@ typedef int (*fork_logits_fn)(void* ctx, int32_t step, const int32_t* tokens, co
  * Semi-autoregressive decoding (Section 2: repeat sampling steps until nothing is masked;
  * Section 4.1: blocks of block_len inside the generation window [gen_lo,gen_hi)).
  * Every sequence keeps its own block cursor: the first block that still holds a masked
- * position.  Each iteration calls provider once, runs fork_step on every unfinished sequence's
- * block (step ids proto->step, proto->step+1, ...), advances the cursors and reads one int back
- * to the host to test for termination (one stream synchronisation per step).
- * proto->blk_lo / blk_hi are ignored.  *steps_taken (host) receives the number of provider
- * calls.  Returns FORK_ERR_MAX_STEPS if masked positions remain after max_steps steps, and
- * FORK_ERR_PROVIDER if the callback fails; device state then reflects the steps completed.
+ * position.  Each iteration calls provider once and runs fork_step on every unfinished sequence's
+ * block (step ids proto->step, proto->step+1, ...); the step itself moves the cursors on (the
+ * finaliser of a sequence whose block is complete looks for the next block that holds a masked
+ * position) and its last finaliser reports how many sequences are unfinished in eight bytes of
+ * pinned host memory, which the host polls: no kernel besides the step's own, no stream
+ * synchronisation.  (The first call in a process allocates 2 KB of pinned host memory for these
+ * reports; up to 32 loops may run at the same time.)
+ * By default the host waits for the report of a step before it calls the provider for the next
+ * one.  With FORK_TUNE_LOOP_AHEAD = d > 0 it runs up to d steps ahead of the reports, so the GPU
+ * never waits for the host; the price is up to d provider calls (and steps, which then find nothing
+ * to do: they change neither sequences nor records nor evaluation counts, only n_unmasked /
+ * is_fallback / fallback_pos, which describe the last step enqueued, an empty one) after the batch
+ * is in fact complete.
+ * proto->blk_lo / blk_hi are ignored.  *steps_taken (host) receives the number of steps after
+ * which nothing was masked (= provider calls when d = 0).  Returns FORK_ERR_MAX_STEPS if masked
+ * positions remain after max_steps steps, and FORK_ERR_PROVIDER if the callback fails; device state
+ * then reflects the steps completed and *steps_taken the steps enqueued.
  */
 fork_status fork_decode_loop(const fork_step_args* proto, int32_t block_len, int32_t gen_lo, int32_t gen_hi,
                              fork_logits_fn provider, void* ctx, int32_t max_steps, int32_t* steps_taken,
@@ -363,11 +374,21 @@ const char* fork_status_string(int status);
  *                           per sequence and 32768 over all sequences runs as ONE kernel on variant 2
  *                           (every CTA derives the active set itself), -1 = always the set-up kernel first
  *   FORK_TUNE_LATE_CTA      testing only: g + 1 makes virtual CTA g of a one-kernel step start about
- *                           0.1 ms late (exercises the hand-over of mask updates), 0 = off
+ *                           0.1 ms late (exercises the hand-over of mask updates), 0 = off.  A non-zero
+ *                           value selects an instance of the kernel compiled with that hook; the
+ *                           instances that run otherwise do not contain it.
+ *   FORK_TUNE_L2_EVICT_FIRST 0 = the bulk copies of logits carry the L2 "evict first" hint (a row is read
+ *                           once; what a step re-reads stays cached), -1 = no hint
+ *   FORK_TUNE_LOOP_AHEAD    fork_decode_loop: how many steps the host may enqueue beyond the last step whose
+ *                           outcome it has read (0..6, default 0); see fork_decode_loop
+ *   FORK_TUNE_MIN_UNITS     0 = automatic (8), else how many units of 2048 logits a participating CTA gets at
+ *                           least, on average: a step with few live rows then runs on fewer CTAs, which
+ *                           leaves fewer partial results to hand over and merge
  * Returns the previous value, or -1 for an unknown key.
  */
 enum { FORK_TUNE_VARIANT = 0, FORK_TUNE_CTAS_PER_SM = 1, FORK_TUNE_PDL = 2, FORK_TUNE_STAGES = 3,
-       FORK_TUNE_ONE_KERNEL = 4, FORK_TUNE_LATE_CTA = 5, FORK_TUNE_COUNT_ = 6 };
+       FORK_TUNE_ONE_KERNEL = 4, FORK_TUNE_LATE_CTA = 5, FORK_TUNE_L2_EVICT_FIRST = 6, FORK_TUNE_MIN_UNITS = 7,
+       FORK_TUNE_LOOP_AHEAD = 8, FORK_TUNE_COUNT_ = 9 };
 int32_t fork_set_tuning(int32_t key, int32_t value);
 
 /* Profiling hook: the next fork_step / fork_logprob call made by this host thread records the two

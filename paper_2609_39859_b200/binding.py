@@ -21,7 +21,8 @@ FORK_ROW_NONFINITE, FORK_ROW_BAD_TOKEN = 1, 2
 FORK_DEV_WINDOW_CLAMPED, FORK_DEV_TIMEOUT = 1, 2
 FORK_FALLBACK_LEFTMOST, FORK_FALLBACK_MAX_CONF, FORK_FALLBACK_MIN_CONF, FORK_FALLBACK_MAX_ENTROPY, \
     FORK_FALLBACK_RANDOM = 0, 1, 2, 3, 4
-FORK_TUNE_VARIANT, FORK_TUNE_CTAS_PER_SM, FORK_TUNE_PDL, FORK_TUNE_STAGES, FORK_TUNE_ONE_KERNEL, FORK_TUNE_LATE_CTA = 0, 1, 2, 3, 4, 5
+FORK_TUNE_VARIANT, FORK_TUNE_CTAS_PER_SM, FORK_TUNE_PDL, FORK_TUNE_STAGES, FORK_TUNE_ONE_KERNEL, FORK_TUNE_LATE_CTA, \
+    FORK_TUNE_L2_EVICT_FIRST, FORK_TUNE_MIN_UNITS, FORK_TUNE_LOOP_AHEAD = 0, 1, 2, 3, 4, 5, 6, 7, 8
 
 
 class fork_step_args(C.Structure):

@@ -107,7 +107,9 @@ static bool device_info(DeviceInfo** out) {
         allow((const void*)reduce_select_ring_kernel<bf16_t, kModeVp>) &&
         allow((const void*)reduce_select_ring_kernel<bf16_t, kModeVpSample>) &&
         allow((const void*)reduce_select_ring_kernel<float, kModeVp>) &&
-        allow((const void*)reduce_select_ring_kernel<float, kModeVpSample>);
+        allow((const void*)reduce_select_ring_kernel<float, kModeVpSample>) &&
+        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeStep, true>) &&
+        allow((const void*)reduce_select_ring_kernel<float, kModeStep, true>);
     if (!d.ring_ready) return false;
     d.sms = sms;
   }
@@ -127,6 +129,13 @@ static int grid_size(const DeviceInfo& d, int dtype, int mode, bool fast) {
   long long G = (long long)d.sms * per_sm;
   if (G > FORK_MAX_GRID) G = FORK_MAX_GRID;
   return (int)G;
+}
+
+/* units (of FORK_CHUNK logits) a participating CTA gets at least, on average, in a small step */
+constexpr int kDefaultMinUnits = 8;
+static int min_units_setting() {
+  const int v = g_tune[FORK_TUNE_MIN_UNITS].load();
+  return v > 0 ? v : kDefaultMinUnits;
 }
 
 static bool bad_source(const void* logits, int64_t sb, int64_t sl, int32_t pos0, int32_t B, int32_t Lt,
@@ -186,7 +195,9 @@ static cudaError_t launch_ring(const ReduceParams& rp, int G, int n_stages, bool
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
   }
-  cudaError_t e = cudaLaunchKernelEx(&cfg, reduce_select_ring_kernel<T, MODE>, rp, n_stages);
+  cudaError_t e;
+  if (MODE == kModeStep && rp.late_g != 0) e = cudaLaunchKernelEx(&cfg, reduce_select_ring_kernel<T, kModeStep, true>, rp, n_stages);
+  else e = cudaLaunchKernelEx(&cfg, reduce_select_ring_kernel<T, MODE>, rp, n_stages);
   if (e == cudaSuccess) g_launches.fetch_add(1);
   return e;
 }
@@ -332,7 +343,8 @@ static FusedCtl* fused_ctl_for(const void* ws, int Gv, cudaStream_t st, bool* cu
 }
 
 static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const int32_t* hi, void* ws,
-                             cudaStream_t st, const VpLocal* vp = nullptr, bool own_scratch = false) {
+                             cudaStream_t st, const VpLocal* vp = nullptr, bool own_scratch = false,
+                             LoopCtl* loop = nullptr) {
   DeviceInfo* dev;
   if (!device_info(&dev)) return FORK_ERR_CUDA;
   WsView w = ws_view(ws, a->B, a->Lt);
@@ -358,9 +370,10 @@ static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const i
     SetupParams sp;
     memset(&sp, 0, sizeof(sp));
     sp.flags = a->mask; sp.lo = lo; sp.hi = hi;
-    sp.B = a->B; sp.Lt = a->Lt; sp.pos0 = a->pos0; sp.Ll = a->Ll; sp.C = C; sp.G = G;
+    sp.B = a->B; sp.Lt = a->Lt; sp.pos0 = a->pos0; sp.Ll = a->Ll; sp.C = C; sp.G = G; sp.min_units = min_units_setting();
     sp.hdr = w.hdr; sp.seq_off = w.seq_off; sp.expected = w.expected; sp.ticket = w.ticket; sp.rows = w.rows;
     if (!vp) { sp.n_unmasked = a->n_unmasked; sp.is_fallback = a->is_fallback; sp.fallback_pos = a->fallback_pos; }
+    sp.loop = loop; sp.step = a->step;
     if (launch(active_set_kernel, dim3(1), dim3(kSetupNT), st, g_tune[FORK_TUNE_PDL].load() >= 0, sp) != cudaSuccess) return FORK_ERR_CUDA;
   }
 
@@ -369,6 +382,8 @@ static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const i
   rp.src = RowSource{a->logits, (long long)a->stride_b, (long long)a->stride_l, a->pos0, a->Ll, a->V};
   rp.B = a->B; rp.Lt = a->Lt; rp.C = C;
   rp.fast = fast ? 1 : 0;
+  rp.l2_evict_first = g_tune[FORK_TUNE_L2_EVICT_FIRST].load() >= 0 ? 1 : 0;
+  rp.min_units = min_units_setting();
   rp.hdr = w.hdr; rp.seq_off = w.seq_off; rp.expected = w.expected; rp.ticket = w.ticket;
   rp.rows = w.rows; rp.final_rec = w.final_rec; rp.parts = w.parts; rp.kparts = w.kparts;
   rp.noise_c = drawn ? (float)(1.4426950408889634 / (double)a->temperature) : 0.f;
@@ -394,8 +409,9 @@ static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const i
       rp.vp_peer_tab = w.vp_peer_tab;
     }
   }
+  rp.loop = loop; rp.blk_lo = lo; rp.blk_hi = hi;
   if (ctl) {
-    rp.ctl = ctl; rp.ticket = ctl->ticket; rp.blk_lo = lo; rp.blk_hi = hi; rp.commit_bits = w.commit_bits;
+    rp.ctl = ctl; rp.ticket = ctl->ticket; rp.commit_bits = w.commit_bits;
     rp.W = W; rp.Gv = G; rp.late_g = g_tune[FORK_TUNE_LATE_CTA].load();
   }
   if (launch_reduce(rp, a->dtype, mode, G, st) != cudaSuccess) return FORK_ERR_CUDA;
@@ -445,7 +461,7 @@ extern "C" fork_status fork_logprob(const fork_logprob_args* a, void* ws, size_t
   SetupParams sp;
   memset(&sp, 0, sizeof(sp));
   sp.flags = a->select; sp.lo = nullptr; sp.hi = nullptr;
-  sp.B = a->B; sp.Lt = a->Lt; sp.pos0 = a->pos0; sp.Ll = a->Ll; sp.C = C; sp.G = G;
+  sp.B = a->B; sp.Lt = a->Lt; sp.pos0 = a->pos0; sp.Ll = a->Ll; sp.C = C; sp.G = G; sp.min_units = min_units_setting();
   sp.hdr = w.hdr; sp.seq_off = w.seq_off; sp.expected = w.expected; sp.ticket = w.ticket; sp.rows = w.rows;
   sp.seq_sum = a->seq_sum; sp.seq_cnt = a->seq_cnt;
   if (launch(active_set_kernel, dim3(1), dim3(kSetupNT), st, g_tune[FORK_TUNE_PDL].load() >= 0, sp) != cudaSuccess) return FORK_ERR_CUDA;
@@ -455,6 +471,8 @@ extern "C" fork_status fork_logprob(const fork_logprob_args* a, void* ws, size_t
   rp.src = RowSource{a->logits, (long long)a->stride_b, (long long)a->stride_l, a->pos0, a->Ll, a->V};
   rp.B = a->B; rp.Lt = a->Lt; rp.C = C;
   rp.fast = fast ? 1 : 0;
+  rp.l2_evict_first = g_tune[FORK_TUNE_L2_EVICT_FIRST].load() >= 0 ? 1 : 0;
+  rp.min_units = min_units_setting();
   rp.hdr = w.hdr; rp.seq_off = w.seq_off; rp.expected = w.expected; rp.ticket = w.ticket;
   rp.rows = w.rows; rp.final_rec = w.final_rec; rp.parts = w.parts;
   rp.lp_tokens = a->tokens; rp.lp_out = a->logp; rp.seq_sum = a->seq_sum; rp.seq_cnt = a->seq_cnt;
@@ -462,6 +480,53 @@ extern "C" fork_status fork_logprob(const fork_logprob_args* a, void* ws, size_t
   rp.row_status = a->row_status;
   if (launch_reduce(rp, a->dtype, mode, G, st) != cudaSuccess) return FORK_ERR_CUDA;
   return FORK_OK;
+}
+
+/* ---- the decode loop ------------------------------------------------------------------------
+ * The host's part is to call the provider and enqueue the step; whether anything is still masked
+ * it learns from eight bytes of pinned host memory that the last finaliser of every step writes
+ * (ticket, remaining), not from a stream synchronisation.  A call takes a ring of kLoopFlags such
+ * words from a small pool that is allocated once per process. */
+constexpr int kLoopCalls = 32;                              /* loops that may run at the same time in one process */
+static unsigned long long* g_loop_flags = nullptr;          /* pinned, mapped: [kLoopCalls][kLoopFlags] */
+static bool g_loop_used[kLoopCalls];
+static std::mutex g_loop_mu;
+static std::atomic<uint32_t> g_loop_ticket{1};
+
+static int loop_ring_acquire() {
+  std::lock_guard<std::mutex> lock(g_loop_mu);
+  if (!g_loop_flags) {
+    void* p = nullptr;
+    if (cudaHostAlloc(&p, sizeof(unsigned long long) * kLoopCalls * kLoopFlags, cudaHostAllocPortable | cudaHostAllocMapped) != cudaSuccess)
+      return -1;
+    memset(p, 0, sizeof(unsigned long long) * kLoopCalls * kLoopFlags);
+    g_loop_flags = (unsigned long long*)p;
+  }
+  for (int i = 0; i < kLoopCalls; ++i)
+    if (!g_loop_used[i]) { g_loop_used[i] = true; return i; }
+  return -1;
+}
+static void loop_ring_release(int i) {
+  std::lock_guard<std::mutex> lock(g_loop_mu);
+  g_loop_used[i] = false;
+}
+
+/* Waits until the word carries `ticket`; returns the count that came with it, or -1 if the stream
+   ran dry (or failed) without the word arriving.  The wait is a host-side poll; every few thousand
+   polls it asks the stream whether it still has work, so a failed launch cannot hold it for ever. */
+static int loop_wait_flag(const volatile unsigned long long* word, uint32_t ticket, cudaStream_t st) {
+  for (unsigned long long it = 0;; ++it) {
+    const unsigned long long v = *word;
+    if ((uint32_t)v == ticket) return (int)(uint32_t)(v >> 32);
+    if ((it & 4095ull) == 4095ull) {
+      const cudaError_t q = cudaStreamQuery(st);
+      if (q == cudaSuccess) {                               /* everything enqueued has run: the word is there now or never */
+        const unsigned long long v2 = *word;
+        return ((uint32_t)v2 == ticket) ? (int)(uint32_t)(v2 >> 32) : -1;
+      }
+      if (q != cudaErrorNotReady) return -1;
+    }
+  }
 }
 
 extern "C" fork_status fork_decode_loop(const fork_step_args* proto, int32_t block_len, int32_t gen_lo,
@@ -477,28 +542,72 @@ extern "C" fork_status fork_decode_loop(const fork_step_args* proto, int32_t blo
   if (proto->B == 0) return FORK_OK;
   cudaStream_t st = (cudaStream_t)stream;
   WsView w = ws_view(ws, proto->B, proto->Lt);
+  int ahead = g_tune[FORK_TUNE_LOOP_AHEAD].load();
+  if (ahead < 0) ahead = 0;
+  if (ahead > kLoopFlags - 2) ahead = kLoopFlags - 2;
 
-  CursorParams cp{proto->mask, proto->B, proto->Lt, gen_lo, gen_hi, block_len, w.loop_lo, w.loop_hi, w.hdr, 1};
-  if (launch(block_cursor_kernel, dim3(1), dim3(kSetupNT), st, false, cp) != cudaSuccess) return FORK_ERR_CUDA;
-  cp.init = 0;
-  int32_t n = 0;
+  const int ring = loop_ring_acquire();
+  if (ring < 0) return FORK_ERR_CUDA;
+  unsigned long long* flags = g_loop_flags + (size_t)ring * kLoopFlags;
+  void* flags_dev = nullptr;
+  if (cudaHostGetDevicePointer(&flags_dev, flags, 0) != cudaSuccess) { loop_ring_release(ring); return FORK_ERR_CUDA; }
+  const uint32_t ticket0 = g_loop_ticket.fetch_add((uint32_t)max_steps + 2u) + 1u;
+
+  LoopCtl lc;
+  memset(&lc, 0, sizeof(lc));
+  lc.gen_lo = gen_lo; lc.gen_hi = gen_hi; lc.block_len = block_len; lc.step0 = proto->step;
+  lc.ticket0 = ticket0; lc.flags = (unsigned long long*)flags_dev;
+  for (int i = 0; i < 2; ++i) { lc.lo[i] = w.loop_lo[i]; lc.hi[i] = w.loop_hi[i]; }
   fork_status rc = FORK_OK;
-  for (;;) {
-    int32_t remaining = 0;
-    if (cudaMemcpyAsync(&remaining, &w.hdr->remaining, sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
-        cudaStreamSynchronize(st) != cudaSuccess) { rc = FORK_ERR_CUDA; break; }
-    if (remaining == 0) break;
-    if (n >= max_steps) { rc = FORK_ERR_MAX_STEPS; break; }
-    if (provider(ctx, proto->step + n, proto->tokens, proto->mask, w.loop_lo, w.loop_hi,
-                 const_cast<void*>(proto->logits), stream) != 0) { rc = FORK_ERR_PROVIDER; break; }
-    fork_step_args a = *proto;
-    a.step = proto->step + n;
-    rc = step_impl(&a, w.loop_lo, w.loop_hi, ws, st);
-    if (rc != FORK_OK) break;
-    ++n;
-    if (launch(block_cursor_kernel, dim3(1), dim3(kSetupNT), st, false, cp) != cudaSuccess) { rc = FORK_ERR_CUDA; break; }
+  int32_t issued = 0, confirmed = 0, done_at = -1;         /* steps enqueued; steps whose report has been read; the step after which nothing was masked */
+  int remaining = -1;
+  /* (the struct is copied from this host temporary: staged by the runtime before the call returns) */
+  CursorParams cp{proto->mask, proto->B, proto->Lt, gen_lo, gen_hi, block_len, w.loop_lo[0], w.loop_hi[0], w.loop, 1};
+  if (cudaMemcpyAsync(w.loop, &lc, sizeof(lc), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      launch(block_cursor_kernel, dim3(1), dim3(kSetupNT), st, false, cp) != cudaSuccess) rc = FORK_ERR_CUDA;
+  if (rc == FORK_OK) {
+    remaining = loop_wait_flag(flags + (kLoopFlags - 1), ticket0 - 1u, st);
+    if (remaining < 0) rc = FORK_ERR_CUDA;
+    else if (remaining == 0) done_at = 0;
   }
-  if (steps_taken) *steps_taken = n;
+  while (rc == FORK_OK && done_at < 0) {
+    /* read the reports that are due: all that have arrived, and those without which the loop would
+       run more than `ahead` steps past what it knows */
+    while (confirmed < issued && done_at < 0) {
+      const volatile unsigned long long* word = flags + (confirmed % kLoopFlags);
+      const uint32_t ticket = ticket0 + (uint32_t)confirmed;
+      const bool must = issued - confirmed > ahead || issued >= max_steps;
+      if (!must && (uint32_t)*word != ticket) break;
+      remaining = loop_wait_flag(word, ticket, st);
+      if (remaining < 0) { rc = FORK_ERR_CUDA; break; }
+      ++confirmed;
+      if (remaining == 0) done_at = confirmed;
+    }
+    if (rc != FORK_OK || done_at >= 0) break;
+    if (issued >= max_steps) { rc = FORK_ERR_MAX_STEPS; break; }      /* every report is in: something is still masked */
+    const int32_t* lo = w.loop_lo[issued & 1];
+    const int32_t* hi = w.loop_hi[issued & 1];
+    if (provider(ctx, proto->step + issued, proto->tokens, proto->mask, lo, hi, const_cast<void*>(proto->logits), stream) != 0) {
+      rc = FORK_ERR_PROVIDER;
+      break;
+    }
+    fork_step_args a = *proto;
+    a.step = proto->step + issued;
+    rc = step_impl(&a, lo, hi, ws, st, nullptr, false, w.loop);
+    if (rc != FORK_OK) break;
+    ++issued;
+  }
+  /* steps still in flight (enqueued ahead of the reports) find nothing to do once the batch is
+     complete; their reports are taken in before the ring of words goes back to the pool */
+  while (confirmed < issued) {
+    const int r = loop_wait_flag(flags + (confirmed % kLoopFlags), ticket0 + (uint32_t)confirmed, st);
+    if (r < 0) { if (rc == FORK_OK) rc = FORK_ERR_CUDA; break; }
+    ++confirmed;
+    if (r == 0 && done_at < 0) done_at = confirmed;
+  }
+  if (rc == FORK_ERR_PROVIDER && done_at >= 0) rc = FORK_OK;      /* the failed call was one made ahead, for a step that had nothing left to do */
+  loop_ring_release(ring);
+  if (steps_taken) *steps_taken = done_at >= 0 ? done_at : issued;
   return rc;
 }
 
@@ -834,7 +943,7 @@ extern "C" fork_status fork_logprob_backward(const fork_logprob_bwd_args* a, voi
   SetupParams sp;
   memset(&sp, 0, sizeof(sp));
   sp.flags = a->select; sp.lo = nullptr; sp.hi = nullptr;
-  sp.B = a->B; sp.Lt = a->Lt; sp.pos0 = a->pos0; sp.Ll = a->Ll; sp.C = 1; sp.G = 1;
+  sp.B = a->B; sp.Lt = a->Lt; sp.pos0 = a->pos0; sp.Ll = a->Ll; sp.C = 1; sp.G = 1; sp.min_units = 1;
   sp.hdr = w.hdr; sp.seq_off = w.seq_off; sp.expected = w.expected; sp.ticket = w.ticket; sp.rows = w.rows;
   const bool pdl = g_tune[FORK_TUNE_PDL].load() >= 0;
   if (launch(active_set_kernel, dim3(1), dim3(kSetupNT), st, pdl, sp) != cudaSuccess) return FORK_ERR_CUDA;
@@ -905,14 +1014,14 @@ extern "C" fork_status fork_vp_select(const fork_step_args* a, const void* parts
   SetupParams sp;
   memset(&sp, 0, sizeof(sp));
   sp.flags = a->mask; sp.lo = a->blk_lo; sp.hi = a->blk_hi;
-  sp.B = a->B; sp.Lt = a->Lt; sp.pos0 = 0; sp.Ll = a->Lt; sp.C = 1; sp.G = 1;
+  sp.B = a->B; sp.Lt = a->Lt; sp.pos0 = 0; sp.Ll = a->Lt; sp.C = 1; sp.G = 1; sp.min_units = 1;
   if (a->Ll > 0) { sp.pos0 = a->pos0; sp.Ll = a->Ll; }      /* the window the slices covered */
   sp.hdr = w.hdr; sp.seq_off = w.seq_off; sp.expected = w.expected; sp.ticket = w.ticket; sp.rows = w.rows;
   sp.n_unmasked = a->n_unmasked; sp.is_fallback = a->is_fallback; sp.fallback_pos = a->fallback_pos;
   if (launch(active_set_kernel, dim3(1), dim3(kSetupNT), st, pdl, sp) != cudaSuccess) return FORK_ERR_CUDA;
   ReduceParams rp;
   memset(&rp, 0, sizeof(rp));
-  rp.B = a->B; rp.Lt = a->Lt; rp.C = 1;
+  rp.B = a->B; rp.Lt = a->Lt; rp.C = 1; rp.min_units = 1;
   rp.hdr = w.hdr; rp.seq_off = w.seq_off; rp.expected = w.expected; rp.ticket = w.ticket;
   rp.rows = w.rows; rp.final_rec = w.final_rec; rp.parts = w.parts; rp.kparts = w.kparts;
   rp.tokens = a->tokens; rp.mask = a->mask; rp.threshold = a->threshold; rp.step = a->step;
@@ -1056,4 +1165,4 @@ extern "C" int64_t fork_debug_part_begin(int64_t U, int32_t G, int32_t g) { retu
 extern "C" int32_t fork_debug_part_owner(int64_t U, int32_t G, int64_t x) { return fork_part_owner(U, G, x); }
 extern "C" int32_t fork_debug_row_parts(int64_t U, int32_t G, int32_t C, int64_t r) { return fork_row_parts(U, G, C, r); }
 extern "C" int32_t fork_debug_chunk(void) { return FORK_CHUNK; }
-extern "C" int32_t fork_debug_effective_grid(int64_t U, int32_t G) { return fork_effective_grid(U, G); }
+extern "C" int32_t fork_debug_effective_grid(int64_t U, int32_t G, int32_t min_units) { return fork_effective_grid(U, G, min_units); }

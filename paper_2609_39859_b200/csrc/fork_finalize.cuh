@@ -183,13 +183,56 @@ __device__ __forceinline__ RowOut finalize_rows_warp(const ReduceParams& p, cons
 
 /* What a finaliser can load about a sequence BEFORE its last part arrives (it idles until then):
    the sequence's row range and this lane's position among its first 32 rows. */
-struct SeqHint { int r0, r1, k; };
-__device__ __forceinline__ SeqHint load_seq_hint(const RowMap& rm, int b) {
+struct SeqHint {
+  int r0, r1, k;
+  int cur_lo, cur_hi;        /* decode loop: the sequence's cursor if its block still holds a masked position after the step ... */
+  int nxt_lo, nxt_hi;        /* ... and if it does not: the next block that holds one (gen_hi, gen_hi when there is none) */
+};
+__device__ __forceinline__ SeqHint load_seq_hint(const ReduceParams& p, const RowMap& rm, int b) {
   SeqHint h;
   rm.seq_range(b, h.r0, h.r1);
-  const int r = h.r0 + (int)(threadIdx.x & 31);
+  const int lane = (int)(threadIdx.x & 31);
+  const int r = h.r0 + lane;
   h.k = (r < h.r1) ? rm.k_of(b, r) : -1;
+  h.cur_lo = h.cur_hi = h.nxt_lo = h.nxt_hi = 0;
+  if (p.loop) {
+    /* Section 4.1: blocks are decoded in order, and a block is left when it holds no masked position
+       any more.  Which block comes next does not depend on this step (it touches the current block
+       only), so it is looked up now, while the row's parts are still on their way. */
+    const LoopCtl* L = p.loop;
+    const int lo = rm.win_lo ? rm.win_lo[b] : p.blk_lo[b], hi = rm.win_hi ? rm.win_hi[b] : p.blk_hi[b];
+    const int gen_hi = L->gen_hi, bl = L->block_len;
+    h.cur_lo = lo; h.cur_hi = hi;
+    /* a window that reaches outside the logits buffer keeps masked positions the steps cannot see:
+       its cursor never moves on (the loop then ends at its step limit) */
+    const bool whole = lo >= 0 && hi <= p.Lt && lo >= p.src.pos0 && hi <= p.src.pos0 + p.src.Ll;
+    h.nxt_lo = h.nxt_hi = whole ? gen_hi : -1;
+    if (whole) {
+      for (int s = lo + bl; s < gen_hi; s += bl) {
+        const int e = min(s + bl, gen_hi);
+        unsigned any = 0u;
+        for (int k0 = s; k0 < e; k0 += 32) {
+          const int k = k0 + lane;
+          any |= __ballot_sync(0xffffffffu, k < e && p.mask[(size_t)b * p.Lt + k] != 0);
+        }
+        if (any) { h.nxt_lo = s; h.nxt_hi = e; break; }
+      }
+    }
+  }
   return h;
+}
+
+/* Decode loop, sequence b after its step committed `committed` of its `live` positions: the cursor
+   for the next step goes into the other buffer, a finished sequence leaves the count of unfinished
+   ones, and the sequence is counted as dealt with.  One thread. */
+__device__ __forceinline__ void loop_advance_cursor(const ReduceParams& p, int b, const SeqHint& h, int live, int committed) {
+  LoopCtl* L = p.loop;
+  const bool leaves = committed == live && h.nxt_lo >= 0;
+  const int nlo = leaves ? h.nxt_lo : h.cur_lo, nhi = leaves ? h.nxt_hi : h.cur_hi;
+  const int nxt = ((p.step - L->step0) + 1) & 1;
+  L->lo[nxt][b] = nlo; L->hi[nxt][b] = nhi;
+  if (nlo >= nhi) atomicSub(&L->remaining, 1);
+  loop_sequences_done(L, p.step, p.B, 1);
 }
 
 /* Parts sequence b will receive (rows r0 .. r1-1 under partition c), by the whole warp: what the
@@ -396,6 +439,7 @@ __device__ void finalize_step_sequence(const ReduceParams& p, const RowMap& rm, 
     if (p.nfe) atomicAdd(p.nfe + b, 1);
     if (p.n_fallback && fb) atomicAdd(p.n_fallback + b, 1);
   }
+  if (p.loop && lane == 0) loop_advance_cursor(p, b, h, r1 - r0, count);
   if (!direct) {
     /* hand the mask update on: record, raise the flag, look again.  The CTA that counts itself last
        raises its count, then reads the flags; with a sequentially consistent fence on both sides

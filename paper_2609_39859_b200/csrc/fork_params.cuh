@@ -37,6 +37,24 @@ struct WsHeader {                    /* 256 bytes at the start of the workspace 
 };
 static_assert(sizeof(WsHeader) == 256, "header size");
 
+/* ---- decode loop: state the steps of a loop hand on to one another on the device -------------
+ * The block cursors are double buffered: step i of a loop reads lo/hi[i & 1] (they are the step's
+ * block bounds) and writes lo/hi[(i + 1) & 1] -- every sequence's finaliser its own cursor, after
+ * its commits (the same block, or the next block that still holds a masked position), and whoever
+ * handles the sequences without a live row copies theirs -- so nothing a CTA of the step still has
+ * to read is ever modified.  `remaining` counts the sequences that still hold a masked position;
+ * `seq_done` counts the sequences dealt with in the current step, and whoever brings it to B puts
+ * it back to zero and reports (ticket0 + i, remaining) to the host through flags[i % kLoopFlags],
+ * eight bytes of pinned host memory that the host polls instead of synchronising the stream. */
+constexpr int kLoopFlags = 8;
+struct LoopCtl {
+  int32_t remaining, seq_done;
+  int32_t gen_lo, gen_hi, block_len, step0;
+  uint32_t ticket0; int32_t pad;
+  unsigned long long* flags;
+  int32_t* lo[2]; int32_t* hi[2];
+};
+
 struct VpPeerTable { float4* part[FORK_VP_MAX_RANKS]; float4* key[FORK_VP_MAX_RANKS]; };
 
 struct WsView {
@@ -44,8 +62,9 @@ struct WsView {
   int32_t* seq_off;                  /* [B+1] first row of each sequence */
   int32_t* expected;                 /* [B] parts the sequence will receive */
   int32_t* ticket;                   /* [B] parts received so far */
-  int32_t* loop_lo;                  /* [B] decode-loop block cursors */
-  int32_t* loop_hi;                  /* [B] */
+  int32_t* loop_lo[2];               /* [B] decode-loop block cursors, double buffered */
+  int32_t* loop_hi[2];               /* [B] */
+  LoopCtl* loop;                     /* decode-loop state */
   int2* rows;                        /* [B*Lt] (b, k) of each live row, ascending */
   float4* final_rec;                 /* [B*Lt] per-row results kept between the finaliser's passes */
   float4* parts;                     /* [B*Lt + FORK_MAX_GRID] partial results, slot r+g */
@@ -66,8 +85,11 @@ static WsView ws_view(void* base, int32_t B, int32_t Lt) {
   v.seq_off = (int32_t*)(p + off); off = align_up(off + (nb + 1) * 4, 256);
   v.expected = (int32_t*)(p + off); off = align_up(off + nb * 4, 256);
   v.ticket = (int32_t*)(p + off); off = align_up(off + nb * 4, 256);
-  v.loop_lo = (int32_t*)(p + off); off = align_up(off + nb * 4, 256);
-  v.loop_hi = (int32_t*)(p + off); off = align_up(off + nb * 4, 256);
+  for (int i = 0; i < 2; ++i) {
+    v.loop_lo[i] = (int32_t*)(p + off); off = align_up(off + nb * 4, 256);
+    v.loop_hi[i] = (int32_t*)(p + off); off = align_up(off + nb * 4, 256);
+  }
+  v.loop = (LoopCtl*)(p + off); off = align_up(off + sizeof(LoopCtl), 256);
   v.rows = (int2*)(p + off); off = align_up(off + rows * sizeof(int2), 256);
   v.final_rec = (float4*)(p + off); off = align_up(off + rows * sizeof(float4), 256);
   v.parts = (float4*)(p + off); off = align_up(off + (rows + FORK_MAX_GRID) * sizeof(float4), 256);
@@ -120,7 +142,11 @@ struct ReduceParams {
   int B, Lt, C, fast;
   FusedCtl* ctl; uint8_t* mask; const int32_t* blk_lo; const int32_t* blk_hi;   /* one-kernel step (ctl != NULL): control block, block bounds */
   int W, Gv, late_g;                 /* ... words per sequence of the window bitmaps, virtual CTAs of the launch, and
-                                        late_g - 1 = a virtual CTA that dawdles before its snapshot (a test hook; 0 = none) */
+                                        late_g - 1 = a virtual CTA that dawdles before its snapshot (read by the test-only
+                                        instance of the kernel alone; 0 = none) */
+  int l2_evict_first;                /* bulk copies of logits carry the L2 "evict first" hint */
+  int min_units;                     /* small steps: units per participating CTA (fork_effective_grid) */
+  LoopCtl* loop;                     /* a step of fork_decode_loop: where the cursors of the next step go (else NULL) */
   int vocab_offset;                  /* vocabulary-parallel slices: global index of entry 0 of this buffer */
   WsHeader* hdr; const int2* rows; const int32_t* seq_off; const int32_t* expected; int32_t* ticket;   /* workspace */
   float noise_c; int32_t step; unsigned long long sample_seed;   /* stochastic candidates: log2(e)/tau and the noise stream */
@@ -164,6 +190,7 @@ __device__ __noinline__ int snap_pos_of(const uint32_t* w, int W, int pos0, int 
 struct RowMap {
   const int2* rows; const int32_t* seq_off;
   const int32_t* off; const uint32_t* bits; int B, W, pos0;
+  const int* win_lo; const int* win_hi;   /* one-kernel step: the block windows as the snapshot holds them, or NULL when one of them had to be clipped */
   __device__ __forceinline__ int seq_of(int r) const { return snap_seq_of(off, B, r); }
   __device__ __forceinline__ int pos_of(int b, int j) const { return snap_pos_of(bits + b * W, W, pos0, j); }
   __device__ __forceinline__ int2 bk(int r) const {
@@ -177,7 +204,7 @@ struct RowMap {
   }
 };
 __device__ __forceinline__ RowMap row_map_lists(const ReduceParams& p) {
-  return RowMap{p.rows, p.seq_off, nullptr, nullptr, p.B, 0, p.src.pos0};
+  return RowMap{p.rows, p.seq_off, nullptr, nullptr, p.B, 0, p.src.pos0, nullptr, nullptr};
 }
 
 template <typename T>
@@ -186,6 +213,30 @@ __device__ __forceinline__ const T* row_ptr(const RowSource& s, int b, int k) {
 }
 
 __device__ __forceinline__ float4 ld_cg_f4(const float4* p) { return __ldcg(p); }
+
+/* ---- decode loop: cursors of the next step, termination ------------------------------------- */
+/* `n` more sequences of step p.step have been dealt with (by one thread).  The one that completes
+   the batch leaves the counter clean and tells the host how many sequences still hold a masked
+   position: one 8-byte store (ticket, remaining) into pinned host memory. */
+__device__ __forceinline__ void loop_sequences_done(LoopCtl* L, int step, int B, int n) {
+  int old;
+  asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(&L->seq_done), "r"(n) : "memory");
+  if (old + n == B) {
+    L->seq_done = 0;
+    int rem;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(rem) : "l"(&L->remaining) : "memory");
+    const uint32_t i = (uint32_t)(step - L->step0);
+    const unsigned long long v = ((unsigned long long)(uint32_t)rem << 32) | (unsigned long long)(L->ticket0 + i);
+    *reinterpret_cast<volatile unsigned long long*>(L->flags + (i % kLoopFlags)) = v;   /* posted; nothing else for the host depends on it */
+  }
+}
+
+/* The sequences without a live row in this step keep their cursors; `idle` of them, handled by
+   the calling warp (lanes stride over b). */
+__device__ __forceinline__ void loop_copy_idle_cursor(LoopCtl* L, int step, const int32_t* lo, const int32_t* hi, int b) {
+  const int nxt = ((step - L->step0) + 1) & 1;
+  L->lo[nxt][b] = lo[b]; L->hi[nxt][b] = hi[b];
+}
 
 /* ---- the partition as the kernels see it ---------------------------------------------------- */
 struct PartitionCtx {
@@ -197,10 +248,10 @@ struct PartitionCtx {
   }
 };
 
-__device__ __forceinline__ PartitionCtx make_partition(int R, int C, int grid) {
+__device__ __forceinline__ PartitionCtx make_partition(int R, int C, int grid, int min_units) {
   PartitionCtx c;
   c.U = (long long)R * C;
-  c.G = fork_effective_grid(c.U, grid);
+  c.G = fork_effective_grid(c.U, grid, min_units);
   c.C = C;
   c.small = (unsigned long long)(c.U + 1) * (unsigned long long)c.G < 0xffffffffull;
   return c;

@@ -24,9 +24,16 @@
 #define FORK_CHUNK 2048          /* vocabulary entries per unit */
 #define FORK_MAX_GRID 2048       /* upper bound on the persistent grid, sizes the part array */
 
-/* Only min(G, U) CTAs take part, so that every participating CTA owns at least one unit: the
-   range starts are then strictly increasing and the CTAs overlapping a row are consecutive. */
-FORK_HD int32_t fork_effective_grid(int64_t U, int32_t G) { return (U < (int64_t)G) ? (int32_t)U : G; }
+/* Only min(G, ceil(U / min_units)) CTAs take part, so that every participating CTA owns at least
+   one unit (the range starts are then strictly increasing and the CTAs overlapping a row are
+   consecutive) and, when the step is small, at least min_units of them on average: a step of a few
+   rows is latency-bound whatever the number of CTAs, and every CTA less is a part less to publish,
+   count and merge at the end. */
+FORK_HD int32_t fork_effective_grid(int64_t U, int32_t G, int32_t min_units) {
+  if (min_units < 1) min_units = 1;
+  const int64_t cap = (U + min_units - 1) / min_units;
+  return (cap < (int64_t)G) ? (int32_t)(cap < 1 ? 1 : cap) : G;
+}
 
 FORK_HD int64_t fork_part_begin(int64_t U, int32_t G, int32_t g) {
   return (int64_t)(((uint64_t)g * (uint64_t)U) / (uint64_t)G);

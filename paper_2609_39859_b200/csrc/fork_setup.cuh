@@ -13,11 +13,12 @@ namespace forkd {
 struct SetupParams {
   const uint8_t* flags;              /* mask (step) or select (log-probability) */
   const int32_t* lo; const int32_t* hi;   /* NULL: the whole sequence */
-  int B, Lt, pos0, Ll, C, G;
+  int B, Lt, pos0, Ll, C, G, min_units;
   WsHeader* hdr; int32_t* seq_off; int32_t* expected; int32_t* ticket; int2* rows;
   /* outputs for sequences without a live row */
   int32_t* n_unmasked; uint8_t* is_fallback; int32_t* fallback_pos;   /* step mode */
   float* seq_sum; int32_t* seq_cnt;                                   /* log-probability mode */
+  LoopCtl* loop; int step;                                            /* a step of fork_decode_loop (else NULL) */
 };
 
 __device__ __forceinline__ void seq_window(const SetupParams& p, int b, int& lo, int& hi, bool& clipped) {
@@ -44,8 +45,9 @@ __global__ void __launch_bounds__(kSetupNT, 1) active_set_kernel(SetupParams p) 
   asm volatile("griddepcontrol.launch_dependents;");
   __shared__ int sh_cnt[kSetupMaxB + 1];          /* sh_cnt[b+1] = live rows of b, then their inclusive scan */
   __shared__ int sh_warp[kSetupNT / 32];
-  __shared__ int sh_carry;
+  __shared__ int sh_carry, sh_idle;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = kSetupNT / 32;
+  if (tid == 0) sh_idle = 0;
   int* cnt = (p.B <= kSetupMaxB) ? sh_cnt : p.seq_off;       /* cnt[0..B] */
   unsigned clipped_any = 0;
 
@@ -88,7 +90,7 @@ __global__ void __launch_bounds__(kSetupNT, 1) active_set_kernel(SetupParams p) 
     __syncthreads();
   }
   const int R = sh_carry;
-  const PartitionCtx c = make_partition(R, p.C, p.G);
+  const PartitionCtx c = make_partition(R, p.C, p.G, p.min_units);
   if (tid == 0) {
     p.hdr->R = R; p.hdr->C = p.C; p.hdr->G = c.G;
   }
@@ -120,21 +122,26 @@ __global__ void __launch_bounds__(kSetupNT, 1) active_set_kernel(SetupParams p) 
         if (p.fallback_pos) p.fallback_pos[b] = -1;
         if (p.seq_sum) p.seq_sum[b] = 0.f;
         if (p.seq_cnt) p.seq_cnt[b] = 0;
+        if (p.loop) { loop_copy_idle_cursor(p.loop, p.step, p.lo, p.hi, b); atomicAdd(&sh_idle, 1); }
       }
     }
   }
   clipped_any = __syncthreads_or((int)clipped_any);
-  if (tid == 0) p.hdr->dev_status = clipped_any ? FORK_DEV_WINDOW_CLAMPED : 0u;
+  if (tid == 0) {
+    p.hdr->dev_status = clipped_any ? FORK_DEV_WINDOW_CLAMPED : 0u;
+    if (p.loop && sh_idle > 0) { __threadfence(); loop_sequences_done(p.loop, p.step, p.B, sh_idle); }
+  }
 }
 
 /* ---- decode-loop helpers ------------------------------------------------------------------- */
 struct CursorParams {
   const uint8_t* mask; int B, Lt, gen_lo, gen_hi, block_len;
-  int32_t* lo; int32_t* hi; WsHeader* hdr; int init;
+  int32_t* lo; int32_t* hi; LoopCtl* loop; int init;
 };
 
-/* One warp per sequence: the first block at or after the current one that holds a masked
-   position; lo = hi = gen_hi when there is none.  hdr->remaining counts unfinished sequences. */
+/* Start of a decode loop.  One warp per sequence: the first block that holds a masked position;
+   lo = hi = gen_hi when there is none.  Sets up the loop state and reports the number of
+   unfinished sequences to the host under the ticket before the first step's. */
 __global__ void __launch_bounds__(kSetupNT, 1) block_cursor_kernel(CursorParams p) {
   __shared__ int sh_remaining;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = kSetupNT / 32;
@@ -159,7 +166,13 @@ __global__ void __launch_bounds__(kSetupNT, 1) block_cursor_kernel(CursorParams 
     }
   }
   __syncthreads();
-  if (tid == 0) p.hdr->remaining = sh_remaining;
+  if (tid == 0) {
+    LoopCtl* L = p.loop;
+    L->remaining = sh_remaining; L->seq_done = 0;
+    const unsigned long long v = ((unsigned long long)(uint32_t)sh_remaining << 32) | (unsigned long long)(L->ticket0 - 1u);
+    *reinterpret_cast<volatile unsigned long long*>(L->flags + (kLoopFlags - 1)) = v;
+    __threadfence_system();
+  }
 }
 
 }  // namespace forkd

@@ -25,7 +25,7 @@ __global__ void __launch_bounds__(kNT, 4) reduce_select_kernel(const __grid_cons
   asm volatile("griddepcontrol.launch_dependents;");
   const int R = p.hdr->R;
   if (R <= 0) return;
-  const PartitionCtx c = make_partition(R, p.C, (int)gridDim.x);
+  const PartitionCtx c = make_partition(R, p.C, (int)gridDim.x, p.min_units);
   const int g = blockIdx.x;
   if (g >= c.G) return;                                     /* CTAs beyond the number of units have no work */
   const RowMap rm = row_map_lists(p);
@@ -56,7 +56,7 @@ __global__ void __launch_bounds__(kNT, 4) reduce_select_kernel(const __grid_cons
     if (threadIdx.x < 32) {
       const bool last = publish_part(p, part, sg.r, g, bk.x, p.expected[bk.x], SAMPLE ? &kp : nullptr);
       if (last) {                                           /* every part of sequence b has been delivered */
-        const SeqHint h = load_seq_hint(rm, bk.x);
+        const SeqHint h = load_seq_hint(p, rm, bk.x);
         if (MODE == kModeLogprob) finalize_logprob_sequence<T>(p, rm, c, bk.x, h);
         else if (VP) finalize_vp_local<T, SAMPLE>(p, rm, c, bk.x, h);
         else finalize_step_sequence<T, SAMPLE>(p, rm, c, bk.x, h);
@@ -137,6 +137,20 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t pari
 __device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                :: "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+/* The same copy with an L2 eviction-priority hint.  A row is read exactly once, so its lines are
+   marked "evict first": what the step needs again -- the kernel's own code, mask and bounds, parts,
+   tickets, the per-position outputs -- then survives in L2 while hundreds of MB of logits stream
+   through it, instead of being fetched from HBM at the start and the end of every launch. */
+__device__ __forceinline__ unsigned long long l2_policy_evict_first() {
+  unsigned long long pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void bulk_copy_g2s_hint(void* dst, const void* src, uint32_t bytes, unsigned long long* bar,
+                                                   unsigned long long pol) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+               :: "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(pol) : "memory");
 }
 /* barrier among the threads of one half (barrier 0 belongs to __syncthreads) */
 __device__ __forceinline__ void half_sync(int half) {
@@ -241,17 +255,24 @@ __device__ __noinline__ bool count_snapshot(const ReduceParams& p, const SnapSme
       p.hdr->R = R; p.hdr->C = p.C; p.hdr->G = G_eff;
       p.hdr->dev_status = sn.clipped ? FORK_DEV_WINDOW_CLAMPED : 0u;
     }
+    int idle = 0;
     for (int b = lane; b < p.B; b += 32)
       if (sn.off[b] == sn.off[b + 1]) {                       /* no live row: the sequence takes no part in the step */
         if (p.n_unmasked) p.n_unmasked[b] = 0;
         if (p.is_fallback) p.is_fallback[b] = 0;
         if (p.fallback_pos) p.fallback_pos[b] = -1;
+        if (p.loop) { loop_copy_idle_cursor(p.loop, p.step, p.blk_lo, p.blk_hi, b); ++idle; }
       }
+    if (p.loop) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) idle += __shfl_xor_sync(0xffffffffu, idle, o);
+      if (lane == 0 && idle > 0) loop_sequences_done(p.loop, p.step, p.B, idle);
+    }
   }
   return snap_done;
 }
 
-template <typename T, int MODE>
+template <typename T, int MODE, bool LATE_HOOK = false>
 __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_kernel(const __grid_constant__ ReduceParams p, int n_stages) {
   constexpr bool WITH_T = mode_is_step(MODE);
   constexpr bool SAMPLE = mode_is_sample(MODE);
@@ -290,14 +311,15 @@ __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_
   asm volatile("griddepcontrol.launch_dependents;");          /* the next kernel in the stream may take free SM slots */
   int R;
   if (fused) {
-    if (p.late_g == g + 1)                                    /* test hook: this virtual CTA takes its snapshot late */
+    if (LATE_HOOK && p.late_g == g + 1)                       /* test-only instance: this virtual CTA takes its snapshot late */
       for (int i = 0; i < 100; ++i) __nanosleep(1000);
     take_snapshot(SnapArgs{p.mask, p.blk_lo, p.blk_hi, p.B, p.W, p.Lt, p.src}, sn, half, htid);
     R = sn.off[p.B];
+    if (!sn.clipped) { rm.win_lo = sn.lo; rm.win_hi = sn.hi; }
   } else {
     R = p.hdr->R;
   }
-  const PartitionCtx c = make_partition(R, p.C, (int)gridDim.x * kHalves);
+  const PartitionCtx c = make_partition(R, p.C, (int)gridDim.x * kHalves, p.min_units);
   SegmentIter it;
   Segment sg = Segment{0, 0, 0};
   bool have = false;                                          /* this half has a first segment */
@@ -314,6 +336,8 @@ __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_
     if (lane != 0) return;
     uint32_t n = 0, s = 0, ph = 0;                           /* stages issued, ring slot, its phase */
     bool ok = true;
+    const bool hint = p.l2_evict_first != 0;
+    const unsigned long long pol = l2_policy_evict_first();
     uint32_t pseg = 0;
     for (; ok && have; have = it.next(sg), ++pseg) {
       const int2 bk = rm.bk(sg.r);
@@ -324,7 +348,8 @@ __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_
         const uint32_t bytes = (total - off < (uint32_t)kStageBytes) ? (total - off) : (uint32_t)kStageBytes;
         if (!mbar_wait(&rs.empty[s], ph ^ 1u, p)) { ok = false; break; }
         mbar_arrive_expect_tx(&rs.full[s], bytes);
-        bulk_copy_g2s(ring + (size_t)s * kStageBytes, src + off, bytes, &rs.full[s]);
+        if (hint) bulk_copy_g2s_hint(ring + (size_t)s * kStageBytes, src + off, bytes, &rs.full[s], pol);
+        else bulk_copy_g2s(ring + (size_t)s * kStageBytes, src + off, bytes, &rs.full[s]);
         if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1u; }
       }
     }
@@ -434,13 +459,13 @@ __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_
   /* ---------------- finaliser ---------------- */
   uint32_t nseg = 0;
   int cur_b = -1, want = 0;
-  SeqHint h = SeqHint{0, 0, -1};
+  SeqHint h = SeqHint{0, 0, -1, 0, 0, 0, 0};
   for (; have; have = it.next(sg)) {
     /* everything that does not depend on the parts is fetched while the consumers still stream */
     const int b = fused ? rm.seq_of(sg.r) : p.rows[sg.r].x;
     if (b != cur_b) {
       cur_b = b;
-      h = load_seq_hint(rm, b);
+      h = load_seq_hint(p, rm, b);
       want = fused ? seq_expected_warp(c, h.r0, h.r1) : p.expected[b];
     }
     if (fused && !snap_done) snap_done = snapshots_complete(p);
@@ -470,7 +495,7 @@ __global__ void __launch_bounds__(kVpNT) vp_select_kernel(const __grid_constant_
   const int b = (int)blockIdx.x * (kVpNT / 32) + (int)(threadIdx.x >> 5);
   if (b >= p.B) return;
   const RowMap rm = row_map_lists(p);
-  const SeqHint h = load_seq_hint(rm, b);
+  const SeqHint h = load_seq_hint(p, rm, b);
   if (h.r1 <= h.r0) return;                                  /* no live row: the active-set kernel wrote its outputs */
   PartitionCtx c;
   c.U = 0; c.G = 1; c.C = 1; c.small = true;

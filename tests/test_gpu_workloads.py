@@ -137,9 +137,9 @@ def test_b8_full_decode_loop(variant):
         assert 0.15 < frac < 0.45, frac
 
 
-def test_passk_decode_loop_prefix_exact_rest_by_invariants():
+def test_passk_decode_loop_every_sequence_exact():
     w = fs.workload("passk")
-    nseq = 4
+    nseq = w.B                               # all 64 sequences against the oracle (about 16,000 rows of fp64 work)
     ost, nonces, osteps, _ = oracle_reference_loop(w, nseq, w.threshold)
     rc, steps, calls, h = gpu_loop(w, w.threshold, nonces)
     assert rc == 0 and steps == calls
@@ -150,7 +150,7 @@ def test_passk_decode_loop_prefix_exact_rest_by_invariants():
     # fork rows (exact or one-ulp ties in bf16) resolved to the lowest index of the maximum
     cfg = w.cfg()
     checked = 0
-    for b in range(nseq, w.B, 7):
+    for b in range(0, w.B, 7):
         for l in range(0, w.Lt, 5):
             p = fs.plan_host(cfg, b, l)
             if p["is_fork"]:
@@ -167,7 +167,7 @@ def test_passk_decode_loop_prefix_exact_rest_by_invariants():
 @pytest.mark.parametrize("lam", [0.5, 0.7, 0.9, 0.95, 0.99])
 def test_sweep_decode_loop(lam):
     w = fs.workload("sweep")
-    nseq = 1
+    nseq = 8 if lam in (0.7, 0.95) else 1    # eight sequences exactly at two thresholds, one at the others, the rest by invariants
     ost, nonces, osteps, _ = oracle_reference_loop(w, nseq, lam)
     rc, steps, calls, h = gpu_loop(w, lam, nonces)
     assert rc == 0 and steps == calls
@@ -264,6 +264,37 @@ def test_decode_loop_error_paths_and_python_provider():
     h1 = st.host()
     for name in h1:
         assert h1[name].tobytes() == h2[name].tobytes(), name
+
+
+def test_loop_that_runs_ahead_of_the_outcomes_gives_the_same_bytes():
+    """With FORK_TUNE_LOOP_AHEAD the host enqueues model calls and steps before it has read the
+    outcome of the earlier ones; the steps enqueued after the batch was complete must find nothing
+    to do and change nothing (not even the per-sequence evaluation counts)."""
+    pkg = F()
+    for name, B in (("tiny", None), ("b8", 3)):
+        w = fs.workload(name)
+        rc0, steps0, calls0, h0 = gpu_loop(w, w.threshold, B=B)
+        assert rc0 == 0 and calls0 == steps0
+        for ahead in (1, 4, 6):
+            old = pkg.fork_set_tuning(pkg.FORK_TUNE_LOOP_AHEAD, ahead)
+            try:
+                rc, steps, calls, h = gpu_loop(w, w.threshold, B=B)
+            finally:
+                pkg.fork_set_tuning(pkg.FORK_TUNE_LOOP_AHEAD, old)
+            assert rc == 0 and steps == steps0 and steps0 <= calls <= steps0 + ahead
+            for key in h:                    # (the three per-sequence outputs that describe the LAST step enqueued are those of an empty step)
+                if calls == steps0 or key not in ("n_unmasked", "is_fallback", "fallback_pos"):
+                    assert h[key].tobytes() == h0[key].tobytes(), (name, ahead, key)
+        # the step limit and a failing model call behave as without look-ahead
+        old = pkg.fork_set_tuning(pkg.FORK_TUNE_LOOP_AHEAD, 4)
+        try:
+            rc, steps, calls, h = gpu_loop(w, 1.0, max_steps=5, B=B, raise_on_error=False)
+            assert rc == pkg.FORK_ERR_MAX_STEPS and steps == 5 and calls == 5
+            assert int((h["commit_step"] >= 0).sum()) == 5 * h["mask"].shape[0]
+            rc, steps, calls, h = gpu_loop(w, 1.0, B=B, raise_on_error=False, fail_at=3)
+            assert rc == pkg.FORK_ERR_PROVIDER and steps == 3
+        finally:
+            pkg.fork_set_tuning(pkg.FORK_TUNE_LOOP_AHEAD, old)
 
 
 def test_loop_resumes_from_its_buffers():

@@ -107,13 +107,13 @@ def test_partition_is_a_partition():
     L.fork_debug_row_parts.argtypes = [C.c_int64, C.c_int32, C.c_int32, C.c_int64]
     assert L.fork_debug_chunk() == 2048
     L.fork_debug_effective_grid.restype = C.c_int32
-    L.fork_debug_effective_grid.argtypes = [C.c_int64, C.c_int32]
+    L.fork_debug_effective_grid.argtypes = [C.c_int64, C.c_int32, C.c_int32]
     for R in (1, 2, 3, 8, 31, 32, 33, 256, 700):
         for Cc in (1, 2, 5, 62, 75):
-            for G0 in (1, 3, 148, 592, 2048):
+            for G0, mu in ((1, 1), (3, 1), (148, 1), (592, 1), (2048, 1), (296, 8), (296, 3), (592, 64)):
                 U = R * Cc
-                G = L.fork_debug_effective_grid(U, G0)
-                assert G == min(G0, U)
+                G = L.fork_debug_effective_grid(U, G0, mu)
+                assert G == min(G0, -(-U // mu)) and 1 <= G <= U        # every CTA owns a unit; small steps use fewer CTAs
                 begins = [L.fork_debug_part_begin(U, G, g) for g in range(G + 1)]
                 assert begins[0] == 0 and begins[-1] == U and all(x <= y for x, y in zip(begins, begins[1:]))
                 assert max(y - x for x, y in zip(begins, begins[1:])) - min(y - x for x, y in zip(begins, begins[1:])) <= 1
