@@ -282,6 +282,7 @@ fork_status fork_vp_reduce_peers(const fork_step_args* args, int32_t vocab_offse
  *     itself, and leaves the counters of the control block as it found them, so back-to-back calls
  *     on one stream are fine, but two calls that can overlap on the GPU (different streams, or
  *     different threads without ordering) race on it.
+ *   - fork_device_status(NULL, ...) reads the device status word of the last call.
  */
 #define FORK_STATIC_SCRATCH_BYTES (2u * 1024u * 1024u)
 fork_status fork_step_static(const fork_step_args* args, void* stream);
@@ -356,7 +357,10 @@ fork_status fork_read_probe(const void* buffer, size_t bytes, void* sink4, void*
 fork_status fork_workspace_release(const void* workspace);
 
 /* Copies the device status word of the last call that used `workspace` to *host_out
-   (FORK_DEV_* bits) and synchronises `stream`. */
+   (FORK_DEV_* bits) and synchronises `stream`.  workspace = NULL asks about the scratch inside the
+   library, i.e. about the last fork_step_static call on the current device (and, like for any
+   workspace, a reported FORK_DEV_TIMEOUT puts the control block reserved for it back to its
+   initial state). */
 fork_status fork_device_status(const void* workspace, uint32_t* host_out, void* stream);
 
 /* Human-readable name of a status code. */

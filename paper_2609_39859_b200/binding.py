@@ -343,9 +343,11 @@ def fork_decode_loop(st: ForkState, logits: torch.Tensor, block_len: int, gen_lo
     return int(rc), int(steps.value)
 
 
-def fork_device_status(st: ForkState, stream=None) -> int:
+def fork_device_status(st, stream=None) -> int:
+    """Device status word (FORK_DEV_* bits) of the last call on `st`'s workspace; `st` = None asks
+    about the library's built-in scratch (fork_step_static)."""
     out = C.c_uint32(0)
-    rc = lib().fork_device_status(C.c_void_p(st.ws_ptr), C.byref(out), _stream_ptr(stream))
+    rc = lib().fork_device_status(C.c_void_p(st.ws_ptr) if st is not None else None, C.byref(out), _stream_ptr(stream))
     if rc != FORK_OK:
         raise ForkError(rc, "fork_device_status")
     return int(out.value)

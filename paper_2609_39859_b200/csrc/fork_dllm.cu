@@ -70,6 +70,7 @@ static void ring_config(int* n_stages) {
 
 struct DeviceInfo { int sms = 0; int occ[2][kModeCount] = {}; bool ring_ready = false; };
 static DeviceInfo g_dev[64];
+static std::once_flag g_dev_once[64];                      /* first call on a device: one thread fills its entry, the others wait */
 
 template <typename T, int MODE>
 static int occupancy_of() {
@@ -78,42 +79,44 @@ static int occupancy_of() {
   return n;
 }
 
+static void device_info_init(int dev) {
+  DeviceInfo& d = g_dev[dev];
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return;
+  d.occ[0][0] = occupancy_of<bf16_t, kModeStep>();
+  d.occ[0][1] = occupancy_of<bf16_t, kModeLogprob>();
+  d.occ[1][0] = occupancy_of<float, kModeStep>();
+  d.occ[1][1] = occupancy_of<float, kModeLogprob>();
+  d.occ[0][2] = occupancy_of<bf16_t, kModeSample>();
+  d.occ[1][2] = occupancy_of<float, kModeSample>();
+  d.occ[0][3] = occupancy_of<bf16_t, kModeVp>();
+  d.occ[1][3] = occupancy_of<float, kModeVp>();
+  d.occ[0][4] = occupancy_of<bf16_t, kModeVpSample>();
+  d.occ[1][4] = occupancy_of<float, kModeVpSample>();
+  const int max_dyn = 220 * 1024;
+  auto allow = [&](const void* fn) { return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn) == cudaSuccess; };
+  d.ring_ready =
+      allow((const void*)reduce_select_ring_kernel<bf16_t, kModeStep>) &&
+      allow((const void*)reduce_select_ring_kernel<bf16_t, kModeLogprob>) &&
+      allow((const void*)reduce_select_ring_kernel<bf16_t, kModeSample>) &&
+      allow((const void*)reduce_select_ring_kernel<float, kModeStep>) &&
+      allow((const void*)reduce_select_ring_kernel<float, kModeLogprob>) &&
+      allow((const void*)reduce_select_ring_kernel<float, kModeSample>) &&
+      allow((const void*)reduce_select_ring_kernel<bf16_t, kModeVp>) &&
+      allow((const void*)reduce_select_ring_kernel<bf16_t, kModeVpSample>) &&
+      allow((const void*)reduce_select_ring_kernel<float, kModeVp>) &&
+      allow((const void*)reduce_select_ring_kernel<float, kModeVpSample>) &&
+      allow((const void*)reduce_select_ring_kernel<bf16_t, kModeStep, true>) &&
+      allow((const void*)reduce_select_ring_kernel<float, kModeStep, true>);
+  if (d.ring_ready) d.sms = sms;                           /* written last: sms != 0 means the entry is complete */
+}
+
 static bool device_info(DeviceInfo** out) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
-  DeviceInfo& d = g_dev[dev];
-  if (d.sms == 0) {
-    int sms = 0;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return false;
-    d.occ[0][0] = occupancy_of<bf16_t, kModeStep>();
-    d.occ[0][1] = occupancy_of<bf16_t, kModeLogprob>();
-    d.occ[1][0] = occupancy_of<float, kModeStep>();
-    d.occ[1][1] = occupancy_of<float, kModeLogprob>();
-    d.occ[0][2] = occupancy_of<bf16_t, kModeSample>();
-    d.occ[1][2] = occupancy_of<float, kModeSample>();
-    d.occ[0][3] = occupancy_of<bf16_t, kModeVp>();
-    d.occ[1][3] = occupancy_of<float, kModeVp>();
-    d.occ[0][4] = occupancy_of<bf16_t, kModeVpSample>();
-    d.occ[1][4] = occupancy_of<float, kModeVpSample>();
-    const int max_dyn = 220 * 1024;
-    auto allow = [&](const void* fn) { return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn) == cudaSuccess; };
-    d.ring_ready =
-        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeStep>) &&
-        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeLogprob>) &&
-        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeSample>) &&
-        allow((const void*)reduce_select_ring_kernel<float, kModeStep>) &&
-        allow((const void*)reduce_select_ring_kernel<float, kModeLogprob>) &&
-        allow((const void*)reduce_select_ring_kernel<float, kModeSample>) &&
-        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeVp>) &&
-        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeVpSample>) &&
-        allow((const void*)reduce_select_ring_kernel<float, kModeVp>) &&
-        allow((const void*)reduce_select_ring_kernel<float, kModeVpSample>) &&
-        allow((const void*)reduce_select_ring_kernel<bf16_t, kModeStep, true>) &&
-        allow((const void*)reduce_select_ring_kernel<float, kModeStep, true>);
-    if (!d.ring_ready) return false;
-    d.sms = sms;
-  }
-  *out = &d;
+  std::call_once(g_dev_once[dev], device_info_init, dev);
+  if (g_dev[dev].sms == 0) return false;
+  *out = &g_dev[dev];
   return true;
 }
 
@@ -625,8 +628,17 @@ extern "C" fork_status fork_workspace_release(const void* ws) {
   return FORK_OK;
 }
 
+static fork_status static_scratch(void** out);
+
 extern "C" fork_status fork_device_status(const void* ws, uint32_t* host_out, void* stream) {
-  if (!ws || !host_out) return FORK_ERR_INVALID_ARG;
+  if (!host_out) return FORK_ERR_INVALID_ARG;
+  const bool own = ws == nullptr;              /* NULL: the scratch inside the library that fork_step_static runs on */
+  if (own) {
+    void* p = nullptr;
+    const fork_status s = static_scratch(&p);
+    if (s != FORK_OK) return s;
+    ws = p;
+  }
   const WsHeader* h = (const WsHeader*)ws;
   cudaStream_t st = (cudaStream_t)stream;
   if (cudaMemcpyAsync(host_out, &h->dev_status, sizeof(uint32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
@@ -638,9 +650,11 @@ extern "C" fork_status fork_device_status(const void* ws, uint32_t* host_out, vo
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FORK_ERR_CUDA;
     std::lock_guard<std::mutex> lock(g_fused_mu);
     FusedTable& t = g_fused[dev];
-    auto it = t.slot_of.find(ws);
-    if (it != t.slot_of.end() && t.base) {
-      if (cudaMemsetAsync(t.base + it->second, 0, sizeof(FusedCtl), st) != cudaSuccess ||
+    int slot = -1;
+    if (own) slot = kFusedSlots;
+    else { auto it = t.slot_of.find(ws); if (it != t.slot_of.end()) slot = it->second; }
+    if (slot >= 0 && t.base) {
+      if (cudaMemsetAsync(t.base + slot, 0, sizeof(FusedCtl), st) != cudaSuccess ||
           cudaStreamSynchronize(st) != cudaSuccess) return FORK_ERR_CUDA;
     }
   }
@@ -655,17 +669,18 @@ extern "C" fork_status fork_device_status(const void* ws, uint32_t* host_out, vo
    cudaGetSymbolAddress and cached. */
 static __device__ __align__(256) unsigned char g_static_scratch[FORK_STATIC_SCRATCH_BYTES];
 static void* g_static_scratch_ptr[64];
-static std::atomic<int> g_static_scratch_ready[64];
+static std::once_flag g_static_scratch_once[64];
+
+static void static_scratch_init(int dev) {
+  void* ptr = nullptr;                         /* set-up, once per device, with that device current */
+  if (cudaGetSymbolAddress(&ptr, g_static_scratch) == cudaSuccess) g_static_scratch_ptr[dev] = ptr;
+}
 
 static fork_status static_scratch(void** out) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FORK_ERR_CUDA;
-  if (!g_static_scratch_ready[dev].load(std::memory_order_acquire)) {
-    void* ptr = nullptr;                       /* set-up, once per device, with that device current */
-    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) return FORK_ERR_CUDA;
-    g_static_scratch_ptr[dev] = ptr;           /* every thread that gets here stores the same address */
-    g_static_scratch_ready[dev].store(1, std::memory_order_release);
-  }
+  std::call_once(g_static_scratch_once[dev], static_scratch_init, dev);
+  if (g_static_scratch_ptr[dev] == nullptr) return FORK_ERR_CUDA;
   *out = g_static_scratch_ptr[dev];
   return FORK_OK;
 }

@@ -87,6 +87,7 @@ constexpr int kMaxStages = 13;
 constexpr int kHalves = 2;                                 /* independent producer/consumer groups per CTA */
 constexpr int kHalfThreads = (kCW + 2) * 32;
 constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr uint32_t kSpinLimitTest = 1u << 13;              /* the test-only instance gives up after a fraction of a millisecond */
 __host__ __device__ constexpr int ring_stage_bytes() { return kCW * 32 * kUnroll * 16; }     /* 16 KB */
 
 constexpr int kSegRing = 16;                               /* > stages: the producer is never that many segments ahead */
@@ -128,8 +129,9 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t 
   return ok != 0;
 }
 /* bounded wait; false (and a status bit in the workspace header) if the phase never completed */
+template <uint32_t LIMIT = kSpinLimit>
 __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity, const ReduceParams& p) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i)
+  for (uint32_t i = 0; i < LIMIT; ++i)
     if (mbar_try_wait(bar, parity)) return true;
   atomicOr(&p.hdr->dev_status, FORK_DEV_TIMEOUT);
   return false;
@@ -281,6 +283,12 @@ __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_
   constexpr int kCT = kCW * 32;                              /* consumer threads */
   constexpr int kStageVecs = kCT * kUnroll;                  /* 128-bit vectors per stage */
   constexpr int kStageBytes = kStageVecs * 16;
+  /* The test-only instance has two hooks (p.late_g): g + 1 > 0 makes virtual CTA g take its snapshot
+     late; -(g + 1) < 0 makes the producer of virtual CTA g leave out the copy of its second stage, so
+     that the bounded waits of that half run out -- with a limit short enough for a test -- and the
+     give-up path can be checked: every thread of the half returns, FORK_DEV_TIMEOUT is reported,
+     nothing is left in flight. */
+  constexpr uint32_t kLimit = LATE_HOOK ? kSpinLimitTest : kSpinLimit;
   extern __shared__ __align__(1024) unsigned char dyn_smem_all[];
   /* One CTA per SM made of kHalves independent halves, each a complete producer / consumers /
      finaliser group with its own ring, barriers and share of the work ("virtual CTA" g).  As two
@@ -338,7 +346,7 @@ __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_
     bool ok = true;
     const bool hint = p.l2_evict_first != 0;
     const unsigned long long pol = l2_policy_evict_first();
-    uint32_t pseg = 0;
+    uint32_t pseg = 0, withheld = 0xffffffffu;
     for (; ok && have; have = it.next(sg), ++pseg) {
       const int2 bk = rm.bk(sg.r);
       rs.seg_bk[pseg % kSegRing] = bk;                       /* visible to the consumers through the stage's full barrier */
@@ -346,17 +354,21 @@ __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_
       const uint32_t total = (uint32_t)((sg.e1 - sg.e0) / VEC) * 16u;
       for (uint32_t off = 0; off < total; off += kStageBytes, ++n) {
         const uint32_t bytes = (total - off < (uint32_t)kStageBytes) ? (total - off) : (uint32_t)kStageBytes;
-        if (!mbar_wait(&rs.empty[s], ph ^ 1u, p)) { ok = false; break; }
-        mbar_arrive_expect_tx(&rs.full[s], bytes);
-        if (hint) bulk_copy_g2s_hint(ring + (size_t)s * kStageBytes, src + off, bytes, &rs.full[s], pol);
-        else bulk_copy_g2s(ring + (size_t)s * kStageBytes, src + off, bytes, &rs.full[s]);
+        if (!mbar_wait<kLimit>(&rs.empty[s], ph ^ 1u, p)) { ok = false; break; }
+        if (LATE_HOOK && p.late_g == -(g + 1) && n == 1) {
+          withheld = n;                                      /* never armed, never copied: its consumers wait in vain */
+        } else {
+          mbar_arrive_expect_tx(&rs.full[s], bytes);
+          if (hint) bulk_copy_g2s_hint(ring + (size_t)s * kStageBytes, src + off, bytes, &rs.full[s], pol);
+          else bulk_copy_g2s(ring + (size_t)s * kStageBytes, src + off, bytes, &rs.full[s]);
+        }
         if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1u; }
       }
     }
     if (!ok) {                                               /* do not leave with copies still landing */
       const uint32_t first = n > (uint32_t)n_stages ? n - (uint32_t)n_stages : 0u;
-      for (uint32_t q = first; q < n; ++q)
-        mbar_wait(&rs.full[q % (uint32_t)n_stages], (q / (uint32_t)n_stages) & 1u, p);
+      for (uint32_t q = first; q < n; ++q)                   /* (with the full limit: a copy that is in flight does land) */
+        if (q != withheld) mbar_wait(&rs.full[q % (uint32_t)n_stages], (q / (uint32_t)n_stages) & 1u, p);
     }
     return;
   }
@@ -377,12 +389,12 @@ __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_
          copy, so readable once a stage of the segment has landed; a segment shorter than one vector
          has no stage and looks its row up itself */
       if (SAMPLE) {                                           /* the noise stream of the row is needed from the first element on */
-        if (nvec > 0 && !mbar_wait(&rs.full[s], ph, p)) return;   /* (the stage loop waits on the same phase again: it stays complete) */
+        if (nvec > 0 && !mbar_wait<kLimit>(&rs.full[s], ph, p)) return;   /* (the stage loop waits on the same phase again: it stays complete) */
         const int2 bk = nvec > 0 ? rs.seg_bk[nseg % kSegRing] : rm.bk(sg.r);
         nz = noise_row(p.sample_seed, p.step, bk.x, bk.y, p.noise_c, (uint32_t)p.vocab_offset);
       }
       for (int voff = 0; voff < nvec; voff += kStageVecs) {
-        if (!mbar_wait(&rs.full[s], ph, p)) return;
+        if (!mbar_wait<kLimit>(&rs.full[s], ph, p)) return;
         const uint4* sp = reinterpret_cast<const uint4*>(ring + (size_t)s * kStageBytes);
         const int nv = nvec - voff;
         if (nv >= kStageVecs) {
@@ -445,7 +457,7 @@ __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_
       if (SAMPLE) kp = key_warp_reduce(kt.best);
       if (lane == 0) {
         const uint32_t d = nseg % kMail, mph = (nseg / kMail) & 1u;
-        if (mbar_wait(&rs.mempty[d], mph ^ 1u, p)) {
+        if (mbar_wait<kLimit>(&rs.mempty[d], mph ^ 1u, p)) {
           rs.mail[d][warp] = pt;
           if (SAMPLE) rs.kmail[d][warp] = kp;
           mbar_arrive(&rs.mfull[d]);
@@ -470,7 +482,7 @@ __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_
     }
     if (fused && !snap_done) snap_done = snapshots_complete(p);
     const uint32_t d = nseg % kMail, ph = (nseg / kMail) & 1u;
-    if (!mbar_wait(&rs.mfull[d], ph, p)) return;
+    if (!mbar_wait<kLimit>(&rs.mfull[d], ph, p)) return;
     Part pt = (lane < kCW) ? rs.mail[d][lane] : part_empty();
     KeyPart kp = key_empty();
     if (SAMPLE && lane < kCW) kp = rs.kmail[d][lane];

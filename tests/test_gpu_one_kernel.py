@@ -114,6 +114,40 @@ def test_a_cta_that_starts_late_still_sees_the_mask_of_the_step(late):
     assert pkg.fork_mask_handovers() >= before
 
 
+def test_a_wait_that_runs_out_returns_with_a_status_and_the_workspace_recovers():
+    """The give-up path of the bounded in-kernel waits, without faulting or hanging anything: in the
+    test-only instance of the kernel one producer leaves out the copy of its second stage, so the
+    consumers and the finaliser of that half wait for data that never comes, run out of their
+    (shortened) limit and return.  The call must come back, report FORK_DEV_TIMEOUT, reading that
+    status must put the workspace's control block back, and the next step on the same workspace
+    must be exact again."""
+    pkg = F()
+    rng = np.random.default_rng(45)
+    B, Lt, V = 8, 32, 126464
+    xs = [make_rows(rng, (B, Lt), V, "bf16", peak_frac=0.6) for _ in range(2)]
+    mask = np.ones((B, Lt), np.uint8)
+    lo, hi = np.zeros(B, np.int32), np.full(B, Lt, np.int32)
+    lo_t, hi_t = torch.from_numpy(lo).cuda(), torch.from_numpy(hi).cuda()
+    n_virtual = 2 * torch.cuda.get_device_properties(0).multi_processor_count
+    st = pkg.ForkState(B, Lt, mask=mask)
+    with tuning(pkg.FORK_TUNE_ONE_KERNEL, 0), tuning(pkg.FORK_TUNE_LATE_CTA, -(n_virtual // 3 + 1)):
+        pkg.fork_step(st, to_torch_logits(xs[0]), lo_t, hi_t, 0.9, step=0)
+        torch.cuda.synchronize()                               # the launch ends by itself
+    assert pkg.fork_device_status(st) & pkg.FORK_DEV_TIMEOUT   # ... says what happened, and resets the control block
+    h = st.host()
+    assert (h["mask"] != 0).any()                              # the sequence that half had a part in was not finalised
+    # the same workspace, from a fresh state: two exact steps
+    st.mask.copy_(torch.from_numpy(mask).cuda())
+    for name, dt, fill in pkg.ForkState.PER_POS + pkg.ForkState.PER_SEQ:
+        getattr(st, name).fill_(fill)
+    st.tokens.zero_()
+    for i, x in enumerate(xs):
+        pkg.fork_step(st, to_torch_logits(x), lo_t, hi_t, 0.9, step=i)
+    torch.cuda.synchronize()
+    assert pkg.fork_device_status(st) == 0
+    compare_step_state(st.host(), oracle_decode(xs, mask, lo, hi, 0.9))
+
+
 def test_batches_too_large_for_the_snapshot_take_the_set_up_kernel():
     pkg = F()
     rng = np.random.default_rng(44)
