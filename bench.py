@@ -455,6 +455,71 @@ def time_vocab_parallel(device, peak, n_ranks=8):
             "exchange_bytes_per_rank": rows * 16, "note": "slice (%.0f MB) may be L2-resident between repetitions" % (rows * n * w.es / 1e6)}
 
 
+def time_fused_head(device, hbm_peak, shapes=((64, 32), (8, 32), (1, 8))):
+    """fork_step_fused_head (hidden states x LM-head weight -> step, logits never stored) at the LLaDA-8B
+    head shape (d = 4096, V = 126464, bf16) against the unfused pair timed beside it as a stated baseline:
+    the library GEMM (torch.matmul, bf16 logits written to HBM) followed by fork_step on those logits."""
+    import torch
+    import paper_2609_39859_b200 as pkg
+    d, V = 4096, 126464
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            mp = json.load(f)
+        tf_peak, tf_src = float(mp["bf16_tflops"]), "measured (MEASURED_PEAKS.json, cuBLAS bf16 burst)"
+    except Exception:
+        tf_peak, tf_src = 1590.0, "fallback (earlier measurement on this pool)"
+    gen = torch.Generator(device=device).manual_seed(1234)
+    W = torch.randn((V, d), device=device, generator=gen, dtype=torch.float32).to(torch.bfloat16)
+    out = []
+    for B, Ll in shapes:
+        R = B * Ll
+        Lt = 256
+        hid = (torch.randn((B, Ll, d), device=device, generator=gen, dtype=torch.float32) * (3.0 / d ** 0.5))
+        tok = torch.randint(0, V, (B, Ll), device=device, generator=gen)
+        hid = (hid + (24.0 / d) * W[tok].float()).to(torch.bfloat16)      # a clear peak per row, N(0, 3^2) background
+        lo = torch.zeros(B, dtype=torch.int32, device=device)
+        hi = torch.full((B,), Ll, dtype=torch.int32, device=device)
+        st = pkg.ForkState(B, Lt, device=device)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+        def timed(fn, reps):
+            for _ in range(3):
+                st.mask.fill_(1)
+                fn()
+            torch.cuda.synchronize()
+            ts = []
+            for _ in range(reps):
+                st.mask.fill_(1)
+                e0.record()
+                fn()
+                e1.record()
+                torch.cuda.synchronize()
+                ts.append(e0.elapsed_time(e1))
+            return statistics.median(ts)
+
+        def fused():
+            pkg.fork_step_fused_head(st, hid, W, lo, hi, 0.9)
+
+        def unfused():
+            logits = torch.matmul(hid.view(R, d), W.t()).view(B, Ll, V)
+            pkg.fork_step(st, logits, lo, hi, 0.9)
+
+        reps = 10 if R >= 1024 else 20
+        ms_f, ms_u = timed(fused, reps), timed(unfused, reps)
+        flops = 2.0 * R * V * d
+        out.append({"workload": "fused LM-head step: %d window rows (B=%d, block %d), d=%d, V=%d, bf16 x bf16 -> fp32" % (R, B, Ll, d, V),
+                    "fused_ms": ms_f, "unfused_gemm_plus_fork_step_ms": ms_u, "speedup_vs_unfused": ms_u / ms_f,
+                    "tflops": flops / (ms_f * 1e-3) / 1e12, "frac_of_bf16_peak": flops / (ms_f * 1e-3) / 1e12 / tf_peak,
+                    "bf16_peak_tflops": tf_peak, "peak_source": tf_src,
+                    "weight_read_gbs": V * d * 2 / (ms_f * 1e-3) / 1e9, "weight_read_frac_of_hbm_peak": V * d * 2 / (ms_f * 1e-3) / 1e9 / hbm_peak,
+                    "hbm_bytes_not_moved": 2 * R * V * 2,
+                    "bound": "tensor" if flops / (tf_peak * 1e12) > V * d * 2 / (hbm_peak * 1e9) else "hbm (one read of the weight)"})
+        del st, hid
+    del W
+    torch.cuda.empty_cache()
+    return out
+
+
 def read_only_ceiling(device):
     """GB/s of the library's read-only streaming probe on 2 GiB (>> L2), median of 3 runs of 5 launches."""
     import torch
@@ -722,6 +787,7 @@ def main():
     ap.add_argument("--scoring-only", type=int, default=0, metavar="B",
                     help="run only the ForkGRPO scoring / objective / backward timings with B sequences (multiple of 8) and print them")
     ap.add_argument("--loops-only", default="", metavar="NAMES", help="run only the decode loops of these workloads (comma separated) and print their statistics")
+    ap.add_argument("--head-only", default="", metavar="BxL[,BxL]", help="run only the fused LM-head step timings at these window shapes and print them")
     ap.add_argument("--one-kernel", type=int, default=0, help="0 = small batches run the step as one kernel (default), -1 = always the set-up kernel first")
     ap.add_argument("--min-units", type=int, default=0, help="0 = automatic; units of 2048 logits per participating CTA in small steps")
     ap.add_argument("--l2-hint", type=int, default=0, help="0 = logits are copied with the L2 evict-first hint (default), -1 = no hint")
@@ -758,6 +824,10 @@ def main():
     if args.loops_only:                                        # a profiling aid, not the benchmark line
         if rank == 0:
             print(json.dumps({"loops": loop_stats(device, tuple(args.loops_only.split(",")))}))
+        return 0
+    if args.head_only:                                         # a profiling aid, not the benchmark line
+        if rank == 0:
+            print(json.dumps({"fused_head": time_fused_head(device, peak, tuple((int(x.split("x")[0]), int(x.split("x")[1])) for x in args.head_only.split(",")))}))
         return 0
     if args.scoring_only:                                      # a profiling aid, not the benchmark line
         if rank == 0:
@@ -874,6 +944,13 @@ def main():
         vp = time_vocab_parallel(device, peak)
         summary["vp_reduce_slice"] = {"us_per_call": round(vp["reduce_ms"] * 1e3, 1), "frac": round(vp["slice_gbs"] / peak, 4)}
         also.append(vp)
+        fh = time_fused_head(device, peak)
+        summary["fused_head_R2048"] = {"us_per_step": round(fh[0]["fused_ms"] * 1e3, 1), "frac_of_bf16_peak": round(fh[0]["frac_of_bf16_peak"], 4),
+                                       "vs_unfused": round(fh[0]["speedup_vs_unfused"], 3)}
+        summary["fused_head_R256"] = {"us_per_step": round(fh[1]["fused_ms"] * 1e3, 1),
+                                      "weight_read_frac_of_hbm_peak": round(fh[1]["weight_read_frac_of_hbm_peak"], 4),
+                                      "vs_unfused": round(fh[1]["speedup_vs_unfused"], 3)}
+        also.extend(fh)
         ro = read_only_ceiling(device)
         out["roofline"]["read_only_ceiling_gbs"] = ro          # the library's own read-only streaming probe, same run
         out["roofline"]["frac_of_read_only_ceiling"] = kern_gbs / ro

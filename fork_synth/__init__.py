@@ -317,3 +317,28 @@ def scoring_inputs(w: Workload, cfg: Cfg):
             p = plan_host(cfg, b, l)
             tokens[b, l] = uni[b, l] if (off[b, l] or p["n_planted"] == 0) else p["tok"][0]
     return tokens, select
+
+
+def head_weight(V: int, d: int, seed: int) -> np.ndarray:
+    """A seeded stand-in for an LM-head weight [V, d] (bf16 bit patterns): independent N(0,1) entries."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    out = np.empty((V, d), np.uint16)
+    step = 8192
+    for v0 in range(0, V, step):
+        out[v0:v0 + step] = f32_to_bf16_bits(rng.standard_normal((min(step, V - v0), d), dtype=np.float32))
+    return out
+
+
+def head_hidden(weight_bits: np.ndarray, n_rows: int, seed: int, sigma: float = 3.0, h_lo: float = 0.0, h_hi: float = 12.0):
+    """Seeded hidden states [n_rows, d] (bf16 bit patterns) whose logits under `weight_bits` look like
+    the calibrated workloads: a N(0, sigma^2) background (hidden = sigma / sqrt(d) * noise), plus, on
+    a random token per row, a peak of height ln V + sigma^2/2 - 1.4 + h, h ~ U(h_lo, h_hi) (hidden +=
+    height / d * weight[token]: the token's own logit rises by about `height`, the others hardly).
+    Returns (hidden_bits, tokens)."""
+    V, d = weight_bits.shape
+    rng = np.random.Generator(np.random.PCG64(seed))
+    hid = rng.standard_normal((n_rows, d), dtype=np.float32) * np.float32(sigma / math.sqrt(d))
+    tok = rng.integers(0, V, size=n_rows)
+    height = (math.log(V) + 0.5 * sigma * sigma - 1.4 + rng.uniform(h_lo, h_hi, size=n_rows)).astype(np.float32)
+    hid += (height / np.float32(d))[:, None] * bf16_bits_to_f32(weight_bits[tok])
+    return f32_to_bf16_bits(hid), tok.astype(np.int64)

@@ -14,7 +14,8 @@
  *
  * Entry points: fork_step (one step), fork_decode_loop (steps until nothing is masked),
  * fork_logprob (log-likelihood scoring of Section 3.2), fork_step_host (host buffers),
- * fork_step_static (no workspace argument); the variants the paper compares with or trains with:
+ * fork_step_static (no workspace argument), fork_step_fused_head (the step fused into the LM-head
+ * product: hidden states and weight in, no logits in memory); the variants the paper compares with or trains with:
  * candidates drawn at temperature tau > 0 and the other fallback orders (fields of fork_step_args),
  * fork_select_top_entropy (JustGRPO-Fast's position selection), fork_grpo_loss (Eq. 2) and
  * fork_logprob_backward (its log-softmax backward); fork_vp_reduce / fork_vp_reduce_peers /
@@ -260,6 +261,34 @@ fork_status fork_vp_select(const fork_step_args* args, const void* parts, const 
 fork_status fork_vp_reduce_peers(const fork_step_args* args, int32_t vocab_offset, int32_t rank, int32_t n_ranks,
                                  void* const* peer_parts, void* const* peer_keys,
                                  void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The step fused into the LM-head product (the paper's model "predicts a distribution
+ * q_theta^k(.|x_t) for every k in M_t", Section 2: the logits of a step are hidden states times the
+ * output embedding).  Instead of reading logits from memory, this entry point takes the hidden
+ * states of the logits window and the LM-head weight, forms logits = hidden x weight^T tile by tile
+ * on the tensor cores (bf16 inputs, fp32 accumulation) and reduces every tile to the step's per-row
+ * statistics while it is still in tensor memory; the logits are never written anywhere.  Then the
+ * unmask rule runs exactly as in fork_step (all outputs, all fallback orders).
+ *   - hidden: device, bf16, [B * Ll, d]: row b * Ll + (k - pos0) is the final hidden state of position
+ *     k of sequence b (every position of the window, masked or not), rows hidden_stride elements apart.
+ *   - weight: device, bf16, [V, d], rows weight_stride elements apart: logit v = <hidden row, weight row v>.
+ *   - d a multiple of 64; both base addresses 16-byte aligned and both strides multiples of 8 elements.
+ *   - args->logits, stride_b, stride_l and dtype are ignored; temperature must be 0.
+ *   - The logits are the fp32-accumulated products themselves (not rounded to bf16 on the way), so
+ *     results agree with fork_step on materialised bf16 logits only up to that rounding.  A row whose
+ *     logits hold NaN or an infinity is flagged FORK_ROW_NONFINITE.
+ * Asynchronous on `stream`; three kernels (active set, product + reduction, merge + unmask rule).
+ */
+typedef struct fork_head_args {
+  const void* hidden;        /* [B*Ll, d] bf16 */
+  int64_t hidden_stride;     /* elements between rows, >= d */
+  const void* weight;        /* [V, d] bf16 */
+  int64_t weight_stride;     /* elements between rows, >= d */
+  int32_t d;                 /* hidden size */
+} fork_head_args;
+fork_status fork_step_fused_head(const fork_step_args* args, const fork_head_args* head, void* workspace,
+                                 size_t workspace_bytes, void* stream);
 
 /*
  * fork_step without a workspace argument, for callers that have no device memory to give and

@@ -311,3 +311,18 @@ def row_logp_grad(row: np.ndarray, tok: int, w: float = 1.0) -> np.ndarray:
 def row_lse(row: np.ndarray) -> float:
     row = np.ascontiguousarray(row)
     return float(lib().fork_oracle_row_lse(row.ctypes.data, row.shape[0], _dtype_of(row)))
+
+
+def head_logits(hidden_bits: np.ndarray, weight_bits: np.ndarray) -> np.ndarray:
+    """Logits of the LM head for the fused step (Section 2: the model's distribution at a position
+    is the soft-max of hidden state times output embedding): ``logits[i, v] = <hidden[i], weight[v]>``
+    with the bf16 inputs (``uint16`` bit patterns, [n, d] and [V, d]) widened exactly to fp64, the
+    products summed in fp64 (a library matrix product), and the result rounded ONCE to fp32 -- the
+    fused path's logits are its fp32 accumulators, never rounded to bf16."""
+    h = (np.ascontiguousarray(hidden_bits, np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    out = np.empty((h.shape[0], weight_bits.shape[0]), np.float32)
+    step = 8192                                    # weight rows per slab: bounds the fp64 copy of the weight
+    for v0 in range(0, weight_bits.shape[0], step):
+        w = (np.ascontiguousarray(weight_bits[v0:v0 + step], np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+        out[:, v0:v0 + step] = (h @ w.T).astype(np.float32)
+    return out

@@ -9,7 +9,7 @@ _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libfork_dllm.so")
 SOURCES = ["fork_dllm.cu"]
-HEADERS = ["fork_partition.h", "fork_reduce.cuh", "fork_params.cuh", "fork_setup.cuh", "fork_finalize.cuh", "fork_stream.cuh"]
+HEADERS = ["fork_partition.h", "fork_reduce.cuh", "fork_params.cuh", "fork_setup.cuh", "fork_finalize.cuh", "fork_stream.cuh", "fork_head.cuh"]
 
 
 def sources():

@@ -69,10 +69,15 @@ class fork_logprob_bwd_args(C.Structure):
     ]
 
 
+class fork_head_args(C.Structure):
+    _fields_ = [("hidden", C.c_void_p), ("hidden_stride", C.c_int64), ("weight", C.c_void_p), ("weight_stride", C.c_int64),
+                ("d", C.c_int32)]
+
+
 fork_logits_fn = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                              C.c_void_p, C.c_void_p)
 
-EXPORTS = ("fork_workspace_bytes", "fork_step", "fork_step_static", "fork_logprob", "fork_decode_loop", "fork_staging_bytes",
+EXPORTS = ("fork_workspace_bytes", "fork_step", "fork_step_static", "fork_step_fused_head", "fork_logprob", "fork_decode_loop", "fork_staging_bytes",
            "fork_select_top_entropy", "fork_grpo_loss", "fork_logprob_backward", "fork_vp_reduce", "fork_vp_reduce_peers", "fork_vp_select", "fork_read_probe",
            "fork_step_host", "fork_device_status", "fork_status_string", "fork_set_tuning",
            "fork_kernel_launches", "fork_mask_handovers", "fork_workspace_release", "fork_set_timing_events")
@@ -99,6 +104,8 @@ def lib():
     L.fork_step.argtypes = [C.POINTER(fork_step_args), C.c_void_p, C.c_size_t, C.c_void_p]
     L.fork_step_static.restype = C.c_int
     L.fork_step_static.argtypes = [C.POINTER(fork_step_args), C.c_void_p]
+    L.fork_step_fused_head.restype = C.c_int
+    L.fork_step_fused_head.argtypes = [C.POINTER(fork_step_args), C.POINTER(fork_head_args), C.c_void_p, C.c_size_t, C.c_void_p]
     L.fork_logprob.restype = C.c_int
     L.fork_logprob.argtypes = [C.POINTER(fork_logprob_args), C.c_void_p, C.c_size_t, C.c_void_p]
     L.fork_decode_loop.restype = C.c_int
@@ -281,6 +288,24 @@ def fork_step_static(st: ForkState, logits: torch.Tensor, blk_lo: torch.Tensor, 
     rc = lib().fork_step_static(C.byref(a), _stream_ptr(stream))
     if rc != FORK_OK:
         raise ForkError(rc, "fork_step_static")
+
+
+def fork_step_fused_head(st: ForkState, hidden: torch.Tensor, weight: torch.Tensor, blk_lo: torch.Tensor, blk_hi: torch.Tensor,
+                         threshold: float, step: int = 0, pos0: int = 0, stream=None, **variant) -> None:
+    """One sampling step from hidden states [B, Ll, d] (bf16) and the LM-head weight [V, d] (bf16): the
+    logits are formed and reduced on the fly, never stored.  Asynchronous on the stream."""
+    assert hidden.dtype == torch.bfloat16 and weight.dtype == torch.bfloat16
+    assert hidden.dim() == 3 and hidden.stride(2) == 1 and hidden.stride(0) == hidden.shape[1] * hidden.stride(1)
+    assert weight.dim() == 2 and weight.stride(1) == 1 and weight.shape[1] == hidden.shape[2]
+    B, Ll, d = hidden.shape
+    assert B == st.B
+    a = make_step_args(st, None, blk_lo, blk_hi, threshold, step, pos0, **variant)
+    a.Ll, a.V = Ll, weight.shape[0]
+    h = fork_head_args()
+    h.hidden, h.hidden_stride, h.weight, h.weight_stride, h.d = hidden.data_ptr(), hidden.stride(1), weight.data_ptr(), weight.stride(0), d
+    rc = lib().fork_step_fused_head(C.byref(a), C.byref(h), C.c_void_p(st.ws_ptr), st.ws_bytes, _stream_ptr(stream))
+    if rc != FORK_OK:
+        raise ForkError(rc, "fork_step_fused_head")
 
 
 def fork_logprob(logits: torch.Tensor, tokens: torch.Tensor, select: torch.Tensor, st: ForkState, pos0: int = 0,

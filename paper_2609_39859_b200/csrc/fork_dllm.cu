@@ -44,6 +44,7 @@
 #include "fork_setup.cuh"
 #include "fork_finalize.cuh"
 #include "fork_stream.cuh"
+#include "fork_head.cuh"
 
 /* =============================================================================================
  *  Host side: argument checks, launch configuration, the C ABI
@@ -1050,6 +1051,117 @@ extern "C" fork_status fork_vp_select(const fork_step_args* a, const void* parts
   cudaError_t e = a->temperature > 0.f ? launch(vp_select_kernel<true>, grid, dim3(kVpNT), st, pdl, rp)
                                        : launch(vp_select_kernel<false>, grid, dim3(kVpNT), st, pdl, rp);
   return e == cudaSuccess ? FORK_OK : FORK_ERR_CUDA;
+}
+
+/* ---- the step fused into the LM-head GEMM -------------------------------------------------- */
+typedef CUresult (*tensor_map_encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                         const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                         CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static tensor_map_encode_fn g_tensor_map_encode = nullptr;
+static std::once_flag g_head_once;
+static bool g_head_ready = false;
+
+static void head_init() {
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || !fn) return;
+  g_tensor_map_encode = (tensor_map_encode_fn)fn;
+  g_head_ready = true;
+}
+
+/* a [rows, d] bf16 matrix, d contiguous, row stride `ld` elements, cut into boxes of box_rows x 64 with the 128-byte swizzle */
+static bool head_tensor_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t d, uint64_t ld, uint32_t box_rows) {
+  const cuuint64_t dims[2] = {d, rows};
+  const cuuint64_t strides[1] = {ld * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)kHeadK, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return g_tensor_map_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+extern "C" fork_status fork_step_fused_head(const fork_step_args* a, const fork_head_args* h, void* ws, size_t ws_bytes,
+                                            void* stream) {
+  if (!a || !h) return FORK_ERR_INVALID_ARG;
+  if (a->B < 0 || a->Lt <= 0 || a->Ll <= 0 || a->V <= 0 || a->pos0 < 0 || !a->tokens || !a->mask || !a->blk_lo || !a->blk_hi)
+    return FORK_ERR_INVALID_ARG;
+  if ((int64_t)a->B * a->Lt > (int64_t)1 << 30 || a->pos0 + (int64_t)a->Ll > a->Lt) return FORK_ERR_INVALID_ARG;
+  if (a->threshold != a->threshold) return FORK_ERR_INVALID_ARG;
+  if (a->fallback_mode < FORK_FALLBACK_LEFTMOST || a->fallback_mode > FORK_FALLBACK_RANDOM) return FORK_ERR_INVALID_ARG;
+  if (a->fallback_mode == FORK_FALLBACK_RANDOM && !a->fallback_rand) return FORK_ERR_INVALID_ARG;
+  if (a->temperature != 0.f) return FORK_ERR_INVALID_ARG;              /* arg-max candidates only */
+  if (!h->hidden || !h->weight || h->d <= 0 || h->d % kHeadK != 0) return FORK_ERR_INVALID_ARG;
+  if (h->hidden_stride < h->d || h->weight_stride < h->d) return FORK_ERR_INVALID_ARG;
+  if (((uintptr_t)h->hidden % 16) != 0 || ((uintptr_t)h->weight % 16) != 0 || (h->hidden_stride % 8) != 0 ||
+      (h->weight_stride % 8) != 0) return FORK_ERR_INVALID_ARG;        /* tensor copies need 16-byte aligned rows */
+  fork_status s = check_workspace(ws, ws_bytes, a->B, a->Lt);
+  if (s != FORK_OK) return s;
+  if (a->B == 0) return FORK_OK;
+  DeviceInfo* dev;
+  if (!device_info(&dev)) return FORK_ERR_CUDA;
+  std::call_once(g_head_once, head_init);
+  if (!g_head_ready) return FORK_ERR_CUDA;
+  {
+    static std::once_flag smem_once[64];
+    int di = 0;
+    if (cudaGetDevice(&di) != cudaSuccess || di < 0 || di >= 64) return FORK_ERR_CUDA;
+    std::call_once(smem_once[di], [] {
+      cudaFuncSetAttribute(head_gemm_reduce_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHeadSmemBytes);
+    });
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  WsView w = ws_view(ws, a->B, a->Lt);
+  const bool pdl = g_tune[FORK_TUNE_PDL].load() >= 0;
+
+  HeadParams hp;
+  memset(&hp, 0, sizeof(hp));
+  hp.rows = a->B * a->Ll; hp.V = a->V; hp.d = h->d;
+  hp.n_tiles = (a->V + kHeadN - 1) / kHeadN;
+  hp.m_blocks = (hp.rows + kHeadM - 1) / kHeadM;
+  int splits = dev->sms / hp.m_blocks;
+  if (splits < 1) splits = 1;
+  if (splits > hp.n_tiles) splits = hp.n_tiles;
+  hp.tiles_per_split = (hp.n_tiles + splits - 1) / splits;
+  hp.n_splits = (hp.n_tiles + hp.tiles_per_split - 1) / hp.tiles_per_split;
+  if ((size_t)hp.n_splits * hp.m_blocks * kHeadM > (size_t)a->B * a->Lt + kHeadPartsExtra) return FORK_ERR_WORKSPACE;
+  hp.parts = w.head_parts; hp.hdr = w.hdr;
+  CUtensorMap map_h, map_w;
+  if (!head_tensor_map(&map_h, h->hidden, (uint64_t)hp.rows, (uint64_t)h->d, (uint64_t)h->hidden_stride, kHeadM) ||
+      !head_tensor_map(&map_w, h->weight, (uint64_t)a->V, (uint64_t)h->d, (uint64_t)h->weight_stride, kHeadN))
+    return FORK_ERR_INVALID_ARG;
+
+  /* the active set (Algorithm 2, line 3): row list and per-sequence ranges for the select phase */
+  SetupParams sp;
+  memset(&sp, 0, sizeof(sp));
+  sp.flags = a->mask; sp.lo = a->blk_lo; sp.hi = a->blk_hi;
+  sp.B = a->B; sp.Lt = a->Lt; sp.pos0 = a->pos0; sp.Ll = a->Ll; sp.C = 1; sp.G = 1; sp.min_units = 1;
+  sp.hdr = w.hdr; sp.seq_off = w.seq_off; sp.expected = w.expected; sp.ticket = w.ticket; sp.rows = w.rows;
+  sp.n_unmasked = a->n_unmasked; sp.is_fallback = a->is_fallback; sp.fallback_pos = a->fallback_pos;
+  if (launch(active_set_kernel, dim3(1), dim3(kSetupNT), st, pdl, sp) != cudaSuccess) return FORK_ERR_CUDA;
+
+  /* logits tile by tile in tensor memory, reduced to one part per row and vocabulary split */
+  head_gemm_reduce_kernel<<<dim3((unsigned)(hp.m_blocks * hp.n_splits)), dim3(kHeadThreads), kHeadSmemBytes, st>>>(map_h, map_w, hp);
+  if (cudaGetLastError() != cudaSuccess) return FORK_ERR_CUDA;
+  g_launches.fetch_add(1);
+
+  /* the splits of a row merged like the slices of a vocabulary-parallel step, then the unmask rule */
+  ReduceParams rp;
+  memset(&rp, 0, sizeof(rp));
+  rp.src.pos0 = a->pos0; rp.src.Ll = a->Ll; rp.src.V = a->V;
+  rp.B = a->B; rp.Lt = a->Lt; rp.C = 1; rp.min_units = 1;
+  rp.hdr = w.hdr; rp.seq_off = w.seq_off; rp.expected = w.expected; rp.ticket = w.ticket;
+  rp.rows = w.rows; rp.final_rec = w.final_rec; rp.parts = w.parts; rp.kparts = w.kparts;
+  rp.tokens = a->tokens; rp.mask = a->mask; rp.threshold = a->threshold; rp.step = a->step;
+  rp.conf = a->conf; rp.cand = a->cand; rp.entropy = a->entropy; rp.logp = a->logp; rp.row_status = a->row_status;
+  rp.commit_step = a->commit_step; rp.commit_fallback = a->commit_fallback; rp.commit_logp = a->commit_logp;
+  rp.n_unmasked = a->n_unmasked; rp.is_fallback = a->is_fallback; rp.fallback_pos = a->fallback_pos;
+  rp.nfe = a->nfe; rp.n_fallback = a->n_fallback;
+  rp.fallback_mode = a->fallback_mode; rp.fallback_rand = a->fallback_rand;
+  rp.vp_parts_in = w.head_parts; rp.vp_ranks = hp.n_splits; rp.vp_row_stride = hp.m_blocks * kHeadM;
+  const dim3 grid((unsigned)((a->B + kVpNT / 32 - 1) / (kVpNT / 32)));
+  if (launch(vp_select_kernel<false>, grid, dim3(kVpNT), st, false, rp) != cudaSuccess) return FORK_ERR_CUDA;
+  return FORK_OK;
 }
 
 /* ---- host-buffer entry point --------------------------------------------------------------- */

@@ -322,7 +322,8 @@ __device__ __forceinline__ RowOut gathered_rows_warp(const ReduceParams& p, cons
   k = 0;
   if (r >= r1) return row_out_from(part_empty(), true);
   k = (k_hint >= 0) ? k_hint : rm.k_of(b, r);
-  const size_t at = (size_t)b * p.Lt + k, n = (size_t)p.B * p.Lt;
+  const size_t at = p.vp_row_stride > 0 ? (size_t)b * p.src.Ll + (size_t)(k - p.src.pos0) : (size_t)b * p.Lt + k;
+  const size_t n = p.vp_row_stride > 0 ? (size_t)p.vp_row_stride : (size_t)p.B * p.Lt;
   Part acc = part_empty();
   for (int j = 0; j < p.vp_ranks; ++j) acc = part_merge(acc, part_from(__ldg(p.vp_parts_in + j * n + at)));
   const bool bad = !(isfinite(acc.s) && isfinite(acc.t)) || !(acc.m > -INFINITY) || acc.m == INFINITY;

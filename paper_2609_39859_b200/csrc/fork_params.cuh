@@ -57,6 +57,9 @@ struct LoopCtl {
 
 struct VpPeerTable { float4* part[FORK_VP_MAX_RANKS]; float4* key[FORK_VP_MAX_RANKS]; };
 
+/* splits x row blocks of the fused LM-head step never exceed max(SMs, row blocks): room for 160 SMs */
+constexpr size_t kHeadPartsExtra = 128 * 161;
+
 struct WsView {
   WsHeader* hdr;
   int32_t* seq_off;                  /* [B+1] first row of each sequence */
@@ -71,6 +74,7 @@ struct WsView {
   float2* kparts;                    /* [B*Lt + FORK_MAX_GRID] best perturbed key of each part (stochastic candidates) */
   uint32_t* commit_bits;             /* [B * ceil(Lt/32)] positions committed by a step whose mask update was handed on */
   VpPeerTable* vp_peer_tab;          /* gather-buffer addresses of a vocabulary-parallel reduction with the exchange fused in */
+  float4* head_parts;                /* [splits][row blocks * 128] per-row results of the fused LM-head step, one per vocabulary split */
   size_t bytes;
 };
 
@@ -96,6 +100,7 @@ static WsView ws_view(void* base, int32_t B, int32_t Lt) {
   v.kparts = (float2*)(p + off); off = align_up(off + (rows + FORK_MAX_GRID) * sizeof(float2), 256);
   v.commit_bits = (uint32_t*)(p + off); off = align_up(off + nb * (size_t)(((Lt > 0 ? Lt : 1) + 31) / 32) * 4, 256);
   v.vp_peer_tab = (VpPeerTable*)(p + off); off = align_up(off + sizeof(VpPeerTable), 256);
+  v.head_parts = (float4*)(p + off); off = align_up(off + (rows + kHeadPartsExtra) * sizeof(float4), 256);
   v.bytes = off;
   return v;
 }
@@ -159,6 +164,8 @@ struct ReduceParams {
   /* vocabulary-parallel slices */
   float4* vp_part; float4* vp_key;   /* [B,Lt] local phase: per-position results for the exchange instead of the unmask rule */
   const float4* vp_parts_in; const float4* vp_keys_in; int vp_ranks;   /* select phase: gathered [ranks][B,Lt] */
+  int vp_row_stride;                 /* > 0: the gathered parts are indexed [rank][b * Ll + (k - pos0)] with this many rows
+                                        per rank (the fused LM-head step), not [rank][b * Lt + k] */
   /* local phase with the exchange fused in (vp_peers > 0): the gather buffers [vp_peers][B,Lt] of all
      ranks as this GPU addresses them (its own, and peer-mapped memory); slot vp_rank of each is
      written.  The addresses sit in the workspace, not here: the size of this block is felt at

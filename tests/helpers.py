@@ -10,7 +10,8 @@ import oracle
 RTOL, ATOL = 1e-4, 1e-5          # |gpu - oracle| <= ATOL + RTOL * |oracle| for conf, entropy, log-prob
 
 
-def assert_close(name, got, want, where=None):
+def assert_close(name, got, want, where=None, rtol=None, atol=None):
+    RTOL, ATOL = (globals()["RTOL"] if rtol is None else rtol), (globals()["ATOL"] if atol is None else atol)
     got = np.asarray(got, np.float64)
     want = np.asarray(want, np.float64)
     if where is not None:
@@ -34,7 +35,7 @@ def assert_equal(name, got, want, where=None):
         raise AssertionError("%s differs at %s: got=%s want=%s" % (name, bad, got.ravel()[bad], want.ravel()[bad]))
 
 
-def compare_step_state(g: dict, o: "oracle.StepState", nseq=None, last_step_outputs=True):
+def compare_step_state(g: dict, o: "oracle.StepState", nseq=None, last_step_outputs=True, rtol=None, atol=None):
     """Bit-exact integers, floats within tolerance.  `g` is ForkState.host(); compares the first
     `nseq` sequences (all by default).  Positions never written keep their initial fill on both
     sides (-1 / 255 / NaN), so whole arrays can be compared."""
@@ -47,7 +48,7 @@ def compare_step_state(g: dict, o: "oracle.StepState", nseq=None, last_step_outp
     for name in per_seq:
         assert_equal(name, g[name][:n], getattr(o, name)[:n])
     for name in ("conf", "entropy", "logp", "commit_logp"):
-        assert_close(name, g[name][:n], getattr(o, name)[:n])
+        assert_close(name, g[name][:n], getattr(o, name)[:n], rtol=rtol, atol=atol)
 
 
 def live_mask(mask, lo, hi):

@@ -1,0 +1,95 @@
+"""The step fused into the LM-head product (hidden states and weight in, logits never stored) against
+the oracle: fp64 product of the same bf16 inputs, rounded once to fp32, then Algorithm 2 as always.
+Shapes: the LLaDA-8B head the paper names (d = 4096, V = 126464) at 8, 256 and 2048 window rows, and
+small ragged ones.  Inputs are re-drawn until no decision of the checked rows sits within rounding
+distance of flipping (confidence against the threshold, the two largest logits against each other).
+
+Tolerance.  The logits of this path are the tensor cores' fp32 accumulators.  A tcgen05.mma adds 16
+products to the running sum with a rounding of at most one unit in the last place of that sum, and
+a row's logit takes d / 16 = 256 of them; with |logit| <= 32 that bounds the error of a logit by
+256 * 2^-23 * 32 = 1e-3 (observed: a few 1e-4 on the largest logits, where the partial sums are
+largest).  Confidence and log-probability move by at most that much relatively / absolutely, the
+entropy by that much times its own size plus the same absolute amount, so the floats are compared at
+|gpu - oracle| <= 1e-4 + 1e-3 |oracle| (the step on stored logits: 1e-5 + 1e-4 |oracle|), and the
+margins of the decisions are widened accordingly (2e-3 on confidences, 5e-3 on the top-two gap)."""
+HEAD_RTOL, HEAD_ATOL = 1e-3, 1e-4
+import numpy as np
+import pytest
+import torch
+
+import fork_synth as fs
+import oracle
+from helpers import compare_step_state
+
+pytestmark = pytest.mark.gpu
+
+_W = {}
+
+
+def weight(V, d):
+    if (V, d) not in _W:
+        bits = fs.head_weight(V, d, seed=0x39859_00A0 + V + d)
+        _W.clear()                                    # one large weight at a time
+        _W[(V, d)] = (bits, torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16))
+    return _W[(V, d)]
+
+
+def run_case(B, Ll, Lt, pos0, V, d, lam, n_check, mask_density=1.0, seed=1):
+    import paper_2609_39859_b200 as pkg
+    w_bits, w_dev = weight(V, d)
+    rng = np.random.default_rng(seed)
+    mask = (rng.random((B, Lt)) < mask_density).astype(np.uint8)
+    lo = np.full(B, pos0, np.int32)
+    hi = np.full(B, pos0 + Ll, np.int32)
+    if B > 2:
+        hi[-1] = lo[-1]                               # a sequence that sits out
+        hi[1] = pos0 + max(1, Ll // 2)                # a shorter block
+    for nonce in range(8):
+        h_bits, _ = fs.head_hidden(w_bits, B * Ll, seed=seed * 100 + nonce)
+        chk = n_check * Ll
+        logits = oracle.head_logits(h_bits[:chk], w_bits).reshape(n_check, Ll, V)
+        o = oracle.StepState(n_check, Lt, mask=mask[:n_check])
+        assert oracle.step(o, logits, lo[:n_check], hi[:n_check], lam, step_id=3, pos0=pos0) == 0
+        k = np.arange(Lt)[None, :]
+        live = (mask[:n_check] != 0) & (k >= lo[:n_check, None]) & (k < hi[:n_check, None])
+        top2 = np.partition(logits, V - 2, axis=2)[:, :, V - 2:]
+        gap = (top2[:, :, 1] - top2[:, :, 0])
+        gap_full = np.full((n_check, Lt), np.inf)
+        gap_full[:, pos0:pos0 + Ll] = gap
+        if (np.abs(o.conf[live] - np.float64(np.float32(lam))) >= 2e-3).all() and (gap_full[live] >= 5e-3).all():
+            break
+    else:
+        raise AssertionError("no draw with clear margins")
+    st = pkg.ForkState(B, Lt, mask=mask)
+    hid = torch.from_numpy(h_bits.view(np.int16)).cuda().view(torch.bfloat16).view(B, Ll, d)
+    n0 = pkg.fork_kernel_launches()
+    pkg.fork_step_fused_head(st, hid, w_dev, torch.from_numpy(lo).cuda(), torch.from_numpy(hi).cuda(), lam, step=3, pos0=pos0)
+    torch.cuda.synchronize()
+    assert pkg.fork_kernel_launches() - n0 == 3
+    assert pkg.fork_device_status(st) == 0
+    g = st.host()
+    compare_step_state(g, o, nseq=n_check, rtol=HEAD_RTOL, atol=HEAD_ATOL)
+    # every sequence: the unmask rule on the step's own confidences
+    for b in range(B):
+        k = np.arange(Lt)
+        live_b = (mask[b] != 0) & (k >= lo[b]) & (k < hi[b])
+        if not live_b.any():
+            assert g["n_unmasked"][b] == 0 and (g["mask"][b] == mask[b]).all()
+            continue
+        above = live_b & (g["conf"][b] > np.float32(lam))
+        want = above if above.any() else (k == k[live_b][0])
+        assert ((g["mask"][b] == 0) & (mask[b] != 0) == want).all()
+        assert g["is_fallback"][b] == (0 if above.any() else 1)
+        assert (g["mask"][b][~live_b] == mask[b][~live_b]).all()
+    return g
+
+
+def test_small_ragged_shapes():
+    # V not a multiple of the 256-column tile, rows not a multiple of 128, a window inside a longer buffer
+    run_case(B=3, Ll=5, Lt=16, pos0=4, V=1000, d=128, lam=0.9, n_check=3, mask_density=0.8, seed=2)
+    run_case(B=5, Ll=40, Lt=40, pos0=0, V=5000, d=256, lam=0.5, n_check=5, mask_density=0.7, seed=3)
+
+
+@pytest.mark.parametrize("B,Ll,n_check", [(1, 8, 1), (8, 32, 8), (64, 32, 6)])
+def test_llada_head_shapes(B, Ll, n_check):
+    run_case(B=B, Ll=Ll, Lt=256, pos0=32, V=126464, d=4096, lam=0.9, n_check=n_check, seed=10 + B)

@@ -417,3 +417,23 @@ def test_logprob_matches_step_and_sums_in_order():
     toks[1, 4] = V
     rc, lp, ssum, scnt, status = oracle.logprob(x, toks, np.ones((B, Lt), np.uint8))
     assert status[1, 4] & oracle.ROW_BAD_TOKEN and lp[1, 4] == 0.0 and scnt[1] == Lt
+
+
+def test_head_logits_is_the_plain_product():
+    """oracle.head_logits against what fixes it: an identity-like weight returns the hidden states,
+    and a small case equals the triple loop in exact rational arithmetic rounded once to fp32."""
+    from fractions import Fraction
+    rng = np.random.default_rng(5)
+    d, V, n = 8, 11, 3
+    eye = np.zeros((d, d), np.float32)
+    np.fill_diagonal(eye, 1.0)
+    h = fs.f32_to_bf16_bits(rng.standard_normal((n, d)).astype(np.float32))
+    assert (oracle.head_logits(h, fs.f32_to_bf16_bits(eye)) == fs.bf16_bits_to_f32(h)).all()
+    w = fs.f32_to_bf16_bits(rng.standard_normal((V, d)).astype(np.float32))
+    got = oracle.head_logits(h, w)
+    hf, wf = fs.bf16_bits_to_f32(h), fs.bf16_bits_to_f32(w)
+    for i in range(n):
+        for v in range(V):
+            exact = sum(Fraction(float(hf[i, j])) * Fraction(float(wf[v, j])) for j in range(d))
+            assert got[i, v] == np.float32(float(exact))
+    assert got.dtype == np.float32 and got.shape == (n, V)
