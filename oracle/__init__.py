@@ -52,6 +52,7 @@ class _StepArgs(C.Structure):
         ("fallback_mode", C.c_int32), ("fallback_rand", C.c_void_p),
         ("temperature", C.c_float), ("sample_seed", C.c_uint64),
         ("fallback_margin", C.c_void_p), ("sample_margin", C.c_void_p),
+        ("slice_off", C.c_void_p), ("n_slices", C.c_int32),
     ]
 
 
@@ -84,7 +85,7 @@ def lib():
         L.fork_oracle_threads_used.restype = C.c_int
         L.fork_oracle_threads_used.argtypes = [C.c_int32, C.c_int64]
         L.fork_oracle_noise.restype = None
-        L.fork_oracle_noise.argtypes = [C.c_uint64, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+        L.fork_oracle_noise.argtypes = [C.c_uint64, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
         L.fork_oracle_select_top_entropy.restype = C.c_int
         L.fork_oracle_select_top_entropy.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float,
                                                      C.c_void_p, C.c_void_p]
@@ -159,7 +160,7 @@ class StepState:
 
 
 def _fill_args(st: StepState, logits: np.ndarray, lo, hi, threshold, step, pos0, nthreads,
-               fallback_mode=FB_LEFTMOST, fallback_rand=None, temperature=0.0, sample_seed=0) -> _StepArgs:
+               fallback_mode=FB_LEFTMOST, fallback_rand=None, temperature=0.0, sample_seed=0, slices=None) -> _StepArgs:
     assert logits.ndim == 3 and logits.flags.c_contiguous
     B, Ll, V = logits.shape
     assert B == st.B
@@ -184,21 +185,27 @@ def _fill_args(st: StepState, logits: np.ndarray, lo, hi, threshold, step, pos0,
     a.sample_seed = int(sample_seed)
     a.fallback_margin = st.fallback_margin.ctypes.data
     a.sample_margin = st.sample_margin.ctypes.data
+    if slices is not None:                           # vocabulary cut into slices [off[r], off[r+1]): kept alive by the caller
+        a.slice_off, a.n_slices = slices.ctypes.data, len(slices) - 1
     return a
 
 
 def step(st: StepState, logits: np.ndarray, lo: np.ndarray, hi: np.ndarray, threshold: float,
          step_id: int = 0, pos0: int = 0, nthreads: int = 0, fallback_mode: int = FB_LEFTMOST,
-         fallback_rand=None, temperature: float = 0.0, sample_seed: int = 0) -> int:
+         fallback_rand=None, temperature: float = 0.0, sample_seed: int = 0, slices=None) -> int:
     """One sampling step on host buffers; ``st`` is updated in place.  The defaults give Fork-dLLM
     (Algorithm 2) with arg-max candidates; ``fallback_mode`` selects Fast-dLLM's order (Algorithm 1)
-    or an ablation order, ``temperature`` > 0 draws the candidates (noise stream ``sample_seed``)."""
+    or an ablation order, ``temperature`` > 0 draws the candidates (uniform stream ``sample_seed``;
+    ``slices`` = ascending offsets [0, ..., V] when the vocabulary is sharded, which fixes the order
+    in which the draw visits it)."""
+    if slices is not None:
+        slices = np.ascontiguousarray(slices, np.int32)
     lo = np.ascontiguousarray(lo, np.int32)
     hi = np.ascontiguousarray(hi, np.int32)
     if fallback_rand is not None:
         fallback_rand = np.ascontiguousarray(fallback_rand, np.uint32)
     a = _fill_args(st, logits, lo, hi, threshold, step_id, pos0, nthreads, fallback_mode, fallback_rand,
-                   temperature, sample_seed)
+                   temperature, sample_seed, slices)
     return int(lib().fork_oracle_step(C.byref(a)))
 
 
@@ -256,10 +263,10 @@ def decode_loop(st: StepState, logits: np.ndarray, block_len: int, gen_lo: int, 
     return int(rc), int(steps.value)
 
 
-def noise(seed: int, step_id: int, b: int, k: int, v: int):
-    """(u, g): the uniform and the standard Gumbel variate of vocabulary entry v of row (step, b, k)."""
+def noise(seed: int, step_id: int, b: int, k: int):
+    """(u_token, u_slice): the two uniform variates of row (step, b, k) that draw its candidate."""
     u, g = C.c_double(), C.c_double()
-    lib().fork_oracle_noise(int(seed), step_id, b, k, v, C.addressof(u), C.addressof(g))
+    lib().fork_oracle_noise(int(seed), step_id, b, k, C.addressof(u), C.addressof(g))
     return u.value, g.value
 
 

@@ -19,9 +19,12 @@
  *   - token entropy of q_theta^k (Section 3.1 / Figure 2), in nats, of the untempered softmax.
  *
  *   - candidates at temperature tau > 0: x_0^k ~ q_theta^k(. | x_t; tau)  (Section 2; Algorithm 2
- *       line 4), drawn as arg-max_v (x_v/tau + g_v) with g_v standard Gumbel noise from a stated
- *       counter-based generator; the confidence stays the UNtempered probability of the drawn token
- *       (Algorithm 2 line 5 has no tau).
+ *       line 4), drawn by inversion: the vocabulary is laid out in a stated order, the weights
+ *       exp((x_v - m)/tau) are summed along it, and the token is the first one at which the running
+ *       sum reaches U times the total, U a uniform variate from a stated counter-based generator
+ *       (one per position and step).  The paper fixes the distribution, not the method of drawing;
+ *       the order and the generator are this build's.  The confidence stays the UNtempered
+ *       probability of the drawn token (Algorithm 2 line 5 has no tau).
  *   - the fallback orders the paper compares with: highest confidence (Algorithm 1, Fast-dLLM) and
  *       the lowest-confidence / highest-entropy / random ablations (Section 4.1, ablations).
  *   - top-entropy position selection of JustGRPO-Fast (Section 3.2, last paragraph).
@@ -45,7 +48,7 @@
  * Parity pins (tests, CPU only): brute force without the max shift on tiny V, the one-peak /
  * k-way-tie closed forms, hand-worked rows and steps, library log-sum-exp/entropy, invariants,
  * AR and whole-block special cases of the loop; for the variants: moments and a chi-square of
- * the noise stream, scipy's softmax(x/tau) for the drawn candidates, hand-worked fallback choices
+ * the uniform stream, scipy's softmax(x/tau) for the drawn candidates, hand-worked fallback choices
  * of Algorithm 1 against Algorithm 2, numpy sorting for both selections, hand-worked advantages
  * and clipping cases of Eq. 2, finite differences for both derivatives.
  *
@@ -87,14 +90,15 @@ typedef struct {
   /* temperature > 0 only */
   int32_t a_s;         /* drawn token */
   double x_s;          /* its logit */
-  double key_margin;   /* best perturbed key minus the best strictly smaller one (+inf if none) */
+  double key_margin;   /* how far U * total is from the nearer end of the drawn token's stretch of the running sum,
+                          as a fraction of the total (with slices: the smaller of that and the same for the slice) */
 } row_red;
 
-/* ---- the noise stream of stochastic candidates -------------------------------------------------
- * One 64-bit key per (seed, step, b, k); one 32-bit hash per vocabulary entry; a uniform on the
- * 2^-23 grid of midpoints, u = ((h mod 2^23) + 1/2) 2^-23 in (0,1); standard Gumbel g = -ln(-ln u).
- * The draw arg-max_v (x_v/tau + g_v) is then a sample of softmax(x/tau) (Gumbel-max), up to the
- * grid of u (largest g = 16.6).  The CUDA path implements the same integer recipe on its own. */
+/* ---- the uniform variates of stochastic candidates ---------------------------------------------
+ * One 64-bit key per (seed, step, b, k) from two splitmix finalisers; two uniforms on the 2^-23
+ * grid of midpoints taken from disjoint bit fields of the key: U2 = ((key >> 41) + 1/2) 2^-23 draws
+ * the token inside a slice of the vocabulary, U1 = (((key >> 18) mod 2^23) + 1/2) 2^-23 picks the slice
+ * when the vocabulary is cut into several.  The CUDA path implements the same integer recipe on its own. */
 static uint64_t mix64(uint64_t z) {
   z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ULL; z ^= z >> 27; z *= 0x94D049BB133111EBULL; z ^= z >> 31;
   return z;
@@ -103,20 +107,14 @@ static uint64_t noise_row_key(uint64_t seed, int32_t step, int32_t b, int32_t k)
   uint64_t z = mix64(seed + 0x9E3779B97F4A7C15ULL * (uint64_t)((uint32_t)step + 1u));
   return mix64(z ^ (((uint64_t)(uint32_t)b << 32) | (uint64_t)(uint32_t)k));
 }
-static uint32_t noise_hash(uint64_t row_key, uint32_t v) {
-  uint64_t p = (uint64_t)(v ^ (uint32_t)(row_key >> 32)) * 0x9E3779B1ULL;      /* two multiply-and-fold rounds */
-  uint32_t h = (uint32_t)(p >> 32) ^ (uint32_t)p ^ (uint32_t)row_key;
-  p = (uint64_t)h * 0x85EBCA77ULL;
-  return (uint32_t)(p >> 32) ^ (uint32_t)p;
-}
-static double noise_uniform(uint32_t h) { return ((double)(h & 0x7FFFFFu) + 0.5) * (1.0 / 8388608.0); }
-static double noise_gumbel(uint32_t h) { return -log(-log(noise_uniform(h))); }
+static double uniform_token(uint64_t key) { return ((double)(key >> 41) + 0.5) * (1.0 / 8388608.0); }
+static double uniform_slice(uint64_t key) { return ((double)((key >> 18) & 0x7FFFFFu) + 0.5) * (1.0 / 8388608.0); }
 
-/* Exported for the pins: the uniform and the Gumbel variate of entry v of row (seed, step, b, k). */
-void fork_oracle_noise(uint64_t seed, int32_t step, int32_t b, int32_t k, int32_t v, double* u, double* g) {
-  uint32_t h = noise_hash(noise_row_key(seed, step, b, k), (uint32_t)v);
-  if (u) *u = noise_uniform(h);
-  if (g) *g = noise_gumbel(h);
+/* Exported for the pins: the two uniforms of row (seed, step, b, k). */
+void fork_oracle_noise(uint64_t seed, int32_t step, int32_t b, int32_t k, double* u_token, double* u_slice) {
+  const uint64_t key = noise_row_key(seed, step, b, k);
+  if (u_token) *u_token = uniform_token(key);
+  if (u_slice) *u_slice = uniform_slice(key);
 }
 
 /* m, a, s, t of one row, straight from the definitions */
@@ -141,21 +139,91 @@ static void reduce_row(const void* row, int32_t V, int dtype, row_red* out) {
   out->s = nsum_get(&s); out->t = nsum_get(&t);
 }
 
-/* x_0 ~ q(. ; tau) for tau > 0 (Algorithm 2 line 4) by Gumbel-max over the row; ties in the
-   perturbed key go to the lowest index.  Rows flagged bad keep the greedy candidate. */
-static void sample_row(const void* row, int32_t V, int dtype, double tau, uint64_t row_key, row_red* out) {
+/* ---- x_0 ~ q(. ; tau) for tau > 0 (Algorithm 2 line 4), by inversion -----------------------------
+ * The order in which the vocabulary is laid out.  A slice of the vocabulary (the whole of it unless
+ * the caller says otherwise) is cut into groups of G consecutive entries, G = 16 bytes' worth of
+ * logits (8 bf16, 4 fp32); group number j belongs to lane j mod 256.  The order is: lane 0's groups
+ * in ascending order, entries ascending inside a group; then lane 1's; ... ; then lane 255's; last the
+ * fewer-than-G entries left over at the end of the slice.  Slices follow one another in ascending
+ * order.  (Any fixed order gives a sample of the same distribution; this one is the order in which
+ * the kernels' threads meet the entries.)
+ *
+ * One slice: with weights w_v = exp((x_v - m)/tau) (0 for -inf), total W, the token is the first v
+ * in the order whose running sum reaches U2 * W.  Several slices: slice r is taken with probability
+ * W_r / sum W, by inversion with U1 over the slices in ascending order, and the token inside it as
+ * above with U2 and the slice's own total -- a two-stage draw of the same distribution.
+ * Rows flagged bad keep the greedy candidate. */
+enum { ORA_LANES = 256 };
+
+typedef struct { double total; int32_t tok; double margin; } slice_draw;
+
+static double tempered_weight(double x, double m, double tau) { return isinf(x) ? 0.0 : exp((x - m) / tau); }
+
+/* visit the entries [v0, v1) of the row in the stated order; calls fn(ctx, v) */
+static void visit_slice(int32_t v0, int32_t v1, int32_t G, void (*fn)(void*, int32_t), void* ctx) {
+  const int32_t n = v1 - v0, ngroups = n / G;
+  for (int32_t lane = 0; lane < ORA_LANES; ++lane)
+    for (int32_t j = lane; j < ngroups; j += ORA_LANES)
+      for (int32_t e = 0; e < G; ++e) fn(ctx, v0 + j * G + e);
+  for (int32_t v = v0 + ngroups * G; v < v1; ++v) fn(ctx, v);
+}
+
+typedef struct { const void* row; int dtype; double m, tau; nsum acc; double target, before, after; int32_t tok; int found; } draw_ctx;
+static void total_fn(void* c, int32_t v) {
+  draw_ctx* d = (draw_ctx*)c;
+  nsum_add(&d->acc, tempered_weight(load_logit(d->row, v, d->dtype), d->m, d->tau));
+}
+static void draw_fn(void* c, int32_t v) {
+  draw_ctx* d = (draw_ctx*)c;
+  if (d->found) return;
+  const double w = tempered_weight(load_logit(d->row, v, d->dtype), d->m, d->tau);
+  if (w <= 0.0) return;                                /* probability 0: never drawn */
+  const double before = nsum_get(&d->acc);
+  nsum_add(&d->acc, w);
+  d->tok = v; d->before = before; d->after = nsum_get(&d->acc);   /* (the last entry with weight stands if rounding leaves the sum short) */
+  if (d->after >= d->target) d->found = 1;
+}
+
+static slice_draw draw_in_slice(const void* row, int32_t v0, int32_t v1, int dtype, double m, double tau, double u) {
+  const int32_t G = dtype == ORA_BF16 ? 8 : 4;
+  draw_ctx d; memset(&d, 0, sizeof(d));
+  d.row = row; d.dtype = dtype; d.m = m; d.tau = tau;
+  visit_slice(v0, v1, G, total_fn, &d);
+  slice_draw out; out.total = nsum_get(&d.acc); out.tok = -1; out.margin = INFINITY;
+  if (!(out.total > 0.0)) return out;
+  d.acc.sum = d.acc.comp = 0.0; d.target = u * out.total; d.tok = -1;
+  visit_slice(v0, v1, G, draw_fn, &d);
+  out.tok = d.tok;
+  const double lo = d.target - d.before, hi = d.after - d.target;
+  out.margin = (lo < hi ? lo : hi) / out.total;
+  return out;
+}
+
+/* `slice_off`: n_slices + 1 ascending offsets into the row (NULL: the row is one slice) */
+static void sample_row(const void* row, int32_t V, int dtype, double tau, uint64_t row_key, const int32_t* slice_off,
+                       int32_t n_slices, row_red* out) {
   out->a_s = out->a; out->x_s = out->m; out->key_margin = INFINITY;
   if (out->status & ORA_ROW_BAD) return;
-  double best = -INFINITY, second = -INFINITY; int32_t arg = -1;
-  for (int32_t v = 0; v < V; ++v) {
-    double x = load_logit(row, v, dtype);
-    if (isinf(x)) continue;                          /* probability 0 */
-    double key = x / tau + noise_gumbel(noise_hash(row_key, (uint32_t)v));
-    if (arg < 0 || key > best) { if (arg >= 0 && best > second) second = best; best = key; arg = v; }
-    else if (key < best && key > second) second = key;
+  const int32_t one[2] = {0, V};
+  if (!slice_off || n_slices <= 0) { slice_off = one; n_slices = 1; }
+  double grand = 0.0;
+  slice_draw* d = (slice_draw*)malloc(sizeof(slice_draw) * (size_t)n_slices);
+  for (int32_t r = 0; r < n_slices; ++r) {
+    d[r] = draw_in_slice(row, slice_off[r], slice_off[r + 1], dtype, out->m, tau, uniform_token(row_key));
+    grand += d[r].total;
   }
-  out->a_s = arg; out->x_s = load_logit(row, arg, dtype);
-  out->key_margin = best - second;
+  const double target = uniform_slice(row_key) * grand;
+  double run = 0.0, margin = INFINITY; int32_t pick = -1;
+  for (int32_t r = 0; r < n_slices; ++r) {
+    if (!(d[r].total > 0.0)) continue;
+    const double before = run; run += d[r].total; pick = r;
+    if (run >= target) { const double lo = target - before, hi = run - target; margin = (lo < hi ? lo : hi) / grand; break; }
+  }
+  if (pick >= 0) {
+    out->a_s = d[pick].tok; out->x_s = load_logit(row, d[pick].tok, dtype);
+    out->key_margin = n_slices > 1 && margin < d[pick].margin ? margin : d[pick].margin;
+  }
+  free(d);
 }
 
 /* Exported: statistics of a single row. Any output pointer may be NULL. */
@@ -203,7 +271,9 @@ typedef struct fork_oracle_step_args {
   float temperature;                                                   /* tau; 0 = arg-max candidates */
   uint64_t sample_seed;                                                /* noise stream of tau > 0 */
   double* fallback_margin;   /* [B] test aid: gap between the chosen fallback position's key and the runner-up */
-  double* sample_margin;     /* [B,Lt] test aid: gap between the winning perturbed key and the runner-up */
+  double* sample_margin;     /* [B,Lt] test aid: distance of the draw from the nearest boundary of the running sum, over the total */
+  const int32_t* slice_off;  /* tau > 0: n_slices + 1 ascending offsets cutting the vocabulary into slices (NULL: one slice) */
+  int32_t n_slices;
 } fork_oracle_step_args;
 
 /* Which position a fallback step commits.  LEFTMOST is Fork-dLLM (Algorithm 2); MAX_CONF is
@@ -217,7 +287,7 @@ typedef struct { int32_t b, k; row_red red; } live_row;
 typedef struct {
   const void* logits; int64_t stride_b, stride_l; int32_t pos0; int32_t V, dtype; size_t es;
   live_row* rows; int64_t n; int64_t next; pthread_mutex_t mu;
-  double tau; uint64_t seed; int32_t step;
+  double tau; uint64_t seed; int32_t step; const int32_t* slice_off; int32_t n_slices;
 } reduce_job;
 
 static void* reduce_worker(void* p) {
@@ -230,7 +300,7 @@ static void* reduce_worker(void* p) {
         ((int64_t)lr->b * J->stride_b + (int64_t)(lr->k - J->pos0) * J->stride_l) * (int64_t)J->es;
     reduce_row(row, J->V, J->dtype, &lr->red);
     if (J->tau > 0.0)
-      sample_row(row, J->V, J->dtype, J->tau, noise_row_key(J->seed, J->step, lr->b, lr->k), &lr->red);
+      sample_row(row, J->V, J->dtype, J->tau, noise_row_key(J->seed, J->step, lr->b, lr->k), J->slice_off, J->n_slices, &lr->red);
   }
   return NULL;
 }
@@ -294,6 +364,7 @@ int fork_oracle_step(const fork_oracle_step_args* A) {
   reduce_job J; J.logits = A->logits; J.stride_b = A->stride_b; J.stride_l = A->stride_l; J.pos0 = A->pos0;
   J.V = A->V; J.dtype = A->dtype; J.es = (A->dtype == ORA_BF16) ? 2 : 4; J.rows = rows; J.n = n;
   J.tau = (double)A->temperature; J.seed = A->sample_seed; J.step = A->step;
+  J.slice_off = A->slice_off; J.n_slices = A->n_slices;
   reduce_rows_parallel(&J, A->nthreads);
   const int sampled = A->temperature > 0.0f;
 

@@ -1,7 +1,8 @@
 """Pins for the oracle's variants of the sampling step and for the ForkGRPO objective (CPU only).
 
-Each part is checked against something other than itself: moments and a chi-square of the noise
-stream, softmax(x/tau) from scipy for the drawn candidates, hand-worked fallback choices
+Each part is checked against something other than itself: the grid and a chi-square of the uniform
+stream, softmax(x/tau) from scipy for the drawn candidates (one slice and several), the draw
+recomputed here by a numpy cumulative sum along the stated order, hand-worked fallback choices
 (Algorithm 1 versus Algorithm 2), numpy sorting for the selections, hand-worked advantages and
 clipping cases of Eq. 2, and finite differences for both derivatives.
 """
@@ -30,30 +31,49 @@ def one_block_state(rows, masked):
     return st, logits, np.zeros(1, np.int32), np.full(1, n, np.int32)
 
 
-# ---- noise stream ---------------------------------------------------------------------------
-def test_noise_uniform_grid_and_gumbel_moments():
-    n = 200000
-    u = np.empty(n)
-    g = np.empty(n)
-    for v in range(n):
-        u[v], g[v] = oracle.noise(1234, 3, 1, 7, v)
-    assert u.min() > 0.0 and u.max() < 1.0
-    grid = u * 2.0 ** 23 - 0.5
-    assert np.all(grid == np.round(grid))                      # midpoints of the 2^-23 grid
-    counts, _ = np.histogram(u, bins=64, range=(0.0, 1.0))
-    chi2 = float(((counts - n / 64) ** 2 / (n / 64)).sum())
-    assert chi2 < 130.0                                        # 63 degrees of freedom, p ~ 1e-6
-    assert np.allclose(g, -np.log(-np.log(u)), rtol=0, atol=1e-12)
-    assert abs(g.mean() - 0.5772156649) < 0.01                 # Euler-Mascheroni
-    assert abs(g.var() - math.pi ** 2 / 6) < 0.03
-    # neighbouring entries, rows, steps and seeds are uncorrelated
-    assert abs(np.corrcoef(u[:-1], u[1:])[0, 1]) < 0.01
-    other = np.array([oracle.noise(1234, 3, 1, 8, v)[0] for v in range(20000)])
-    assert abs(np.corrcoef(u[:20000], other)[0, 1]) < 0.03
-    other = np.array([oracle.noise(1234, 4, 1, 7, v)[0] for v in range(20000)])
-    assert abs(np.corrcoef(u[:20000], other)[0, 1]) < 0.03
-    other = np.array([oracle.noise(1235, 3, 1, 7, v)[0] for v in range(20000)])
-    assert abs(np.corrcoef(u[:20000], other)[0, 1]) < 0.03
+# ---- uniform stream -------------------------------------------------------------------------
+def test_uniform_stream_grid_uniformity_independence():
+    n = 60000
+    u = np.array([oracle.noise(1234, 3, k // 256, k % 256) for k in range(n)])     # rows (b, k) of one step
+    for col in (0, 1):
+        assert u[:, col].min() > 0.0 and u[:, col].max() < 1.0
+        grid = u[:, col] * 2.0 ** 23 - 0.5
+        assert np.all(grid == np.round(grid))                  # midpoints of the 2^-23 grid
+        counts, _ = np.histogram(u[:, col], bins=64, range=(0.0, 1.0))
+        chi2 = float(((counts - n / 64) ** 2 / (n / 64)).sum())
+        assert chi2 < 130.0                                    # 63 degrees of freedom, p ~ 1e-6
+        assert abs(u[:, col].mean() - 0.5) < 0.01 and abs(u[:, col].var() - 1.0 / 12.0) < 0.005
+        assert abs(np.corrcoef(u[:-1, col], u[1:, col])[0, 1]) < 0.02      # neighbouring positions
+    assert abs(np.corrcoef(u[:, 0], u[:, 1])[0, 1]) < 0.02                # the token's and the slice's uniform
+    joint, _, _ = np.histogram2d(u[:, 0], u[:, 1], bins=8, range=((0, 1), (0, 1)))
+    assert float(((joint - n / 64) ** 2 / (n / 64)).sum()) < 130.0
+    # other steps and seeds are uncorrelated
+    base = u[:20000, 0]
+    other = np.array([oracle.noise(1234, 4, k // 256, k % 256)[0] for k in range(20000)])
+    assert abs(np.corrcoef(base, other)[0, 1]) < 0.03
+    other = np.array([oracle.noise(1235, 3, k // 256, k % 256)[0] for k in range(20000)])
+    assert abs(np.corrcoef(base, other)[0, 1]) < 0.03
+
+
+def visiting_order(v0, v1, group):
+    """The order in which a slice [v0, v1) is laid out: groups of `group` entries dealt to 256 lanes
+    round robin, lane after lane, the left-over entries last (written here independently of the oracle)."""
+    n = v1 - v0
+    ngroups = n // group
+    order = []
+    for lane in range(256):
+        for j in range(lane, ngroups, 256):
+            order.extend(range(v0 + j * group, v0 + (j + 1) * group))
+    order.extend(range(v0 + ngroups * group, v1))
+    return np.array(order, np.int64)
+
+
+def draw_by_cumsum(x, tau, u, order):
+    w = np.exp((x[order].astype(np.float64) - x.astype(np.float64).max()) / tau)
+    c = np.cumsum(w)
+    i = int(np.searchsorted(c, u * c[-1], side="left"))
+    lo = c[i - 1] if i > 0 else 0.0
+    return int(order[i]), min(u * c[-1] - lo, c[i] - u * c[-1]) / c[-1], float(c[-1])
 
 
 # ---- stochastic candidates --------------------------------------------------------------------
@@ -84,31 +104,71 @@ def test_sampled_candidates_follow_tempered_softmax(tau):
     assert float(((counts - greedy) ** 2).sum()) > 1e5          # and it is not the arg-max sampler
 
 
-def test_sampling_limits_and_margin():
+def test_sampling_limits_and_the_draw_recomputed():
     rng = np.random.default_rng(5)
-    B, Lt, V = 2, 16, 50
-    logits = rng.normal(0, 2, (B, Lt, V)).astype(np.float32)
-    lo, hi = np.zeros(B, np.int32), np.full(B, Lt, np.int32)
-    cold = oracle.StepState(B, Lt)
-    oracle.step(cold, logits, lo, hi, -1.0, temperature=1e-3, sample_seed=1)
-    assert np.array_equal(cold.tokens, logits.argmax(-1))       # tau -> 0 is the arg-max
-    zero = oracle.StepState(B, Lt)
-    oracle.step(zero, logits, lo, hi, -1.0, temperature=0.0, sample_seed=1)
-    assert np.array_equal(zero.tokens, logits.argmax(-1)) and np.all(np.isinf(zero.sample_margin))
-    warm = oracle.StepState(B, Lt)
-    oracle.step(warm, logits, lo, hi, -1.0, temperature=1.0, sample_seed=1)
-    # the reported margin is the gap between the two largest perturbed keys, recomputed here
-    for b in range(B):
-        for k in range(Lt):
-            keys = np.array([logits[b, k, v] / np.float64(np.float32(1.0)) + oracle.noise(1, 0, b, k, v)[1]
-                             for v in range(V)])
-            order = np.argsort(-keys, kind="stable")
-            assert warm.tokens[b, k] == order[0]
-            assert math.isclose(warm.sample_margin[b, k], keys[order[0]] - keys[order[1]], rel_tol=0, abs_tol=1e-12)
-    # a different seed or step gives different draws
-    other = oracle.StepState(B, Lt)
-    oracle.step(other, logits, lo, hi, -1.0, temperature=1.0, sample_seed=2)
-    assert not np.array_equal(other.tokens, warm.tokens)
+    B, Lt, V = 2, 16, 5003                                     # 625 groups of 8: more than one round of the 256 lanes, 3 left over
+    for dtype, group in ((np.float32, 4), (np.uint16, 8)):
+        xf = rng.normal(0, 2, (B, Lt, V)).astype(np.float32)
+        if dtype is np.uint16:
+            u32 = xf.view(np.uint32).astype(np.uint64)
+            logits = ((u32 + 0x7FFF + ((u32 >> 16) & 1)) >> 16).astype(np.uint16)
+            xf = (logits.astype(np.uint32) << 16).view(np.float32)
+        else:
+            logits = xf
+        lo, hi = np.zeros(B, np.int32), np.full(B, Lt, np.int32)
+        cold = oracle.StepState(B, Lt)
+        oracle.step(cold, logits, lo, hi, -1.0, temperature=1e-3, sample_seed=1)
+        picked = np.take_along_axis(xf, cold.tokens[..., None].astype(np.int64), -1)[..., 0]
+        assert np.array_equal(picked, xf.max(-1))                # tau -> 0 draws a maximum (any of them when bf16 values tie)
+        zero = oracle.StepState(B, Lt)
+        oracle.step(zero, logits, lo, hi, -1.0, temperature=0.0, sample_seed=1)
+        assert np.array_equal(zero.tokens, xf.argmax(-1)) and np.all(np.isinf(zero.sample_margin))
+        warm = oracle.StepState(B, Lt)
+        oracle.step(warm, logits, lo, hi, -1.0, temperature=1.0, sample_seed=1)
+        order = visiting_order(0, V, group)
+        assert sorted(order.tolist()) == list(range(V))
+        for b in range(B):
+            for k in range(Lt):
+                tok, margin, _ = draw_by_cumsum(xf[b, k], 1.0, oracle.noise(1, 0, b, k)[0], order)
+                assert warm.tokens[b, k] == tok
+                assert math.isclose(warm.sample_margin[b, k], margin, rel_tol=1e-6, abs_tol=1e-12)
+        # a different seed gives different draws
+        other = oracle.StepState(B, Lt)
+        oracle.step(other, logits, lo, hi, -1.0, temperature=1.0, sample_seed=2)
+        assert not np.array_equal(other.tokens, warm.tokens)
+        # the vocabulary in three slices: the slice by its own uniform, the token inside it by the other
+        cuts = np.array([0, 1672, 3344, V], np.int32)
+        cut = oracle.StepState(B, Lt)
+        oracle.step(cut, logits, lo, hi, -1.0, temperature=1.0, sample_seed=1, slices=cuts)
+        for b in range(B):
+            for k in range(Lt):
+                u_tok, u_slice = oracle.noise(1, 0, b, k)
+                draws = [draw_by_cumsum_slice(xf[b, k], 1.0, u_tok, int(cuts[r]), int(cuts[r + 1]), group) for r in range(3)]
+                totals = np.cumsum([d[2] for d in draws])
+                r = int(np.searchsorted(totals, u_slice * totals[-1], side="left"))
+                assert cut.tokens[b, k] == draws[r][0]
+
+
+def draw_by_cumsum_slice(x, tau, u, v0, v1, group):
+    order = visiting_order(v0, v1, group)
+    w = np.exp((x[order].astype(np.float64) - x.astype(np.float64).max()) / tau)
+    c = np.cumsum(w)
+    i = int(np.searchsorted(c, u * c[-1], side="left"))
+    return int(order[i]), 0.0, float(c[-1])
+
+
+def test_sampled_candidates_in_slices_follow_tempered_softmax():
+    x = np.array([2.0, 1.0, 0.5, 0.0, -1.0, 1.5, 0.3, -0.4, 1.1, 0.9, -2.0], np.float32)
+    B, Lt, V = 32, 64, x.shape[0]
+    logits = np.ascontiguousarray(np.broadcast_to(x, (B, Lt, V))).copy()
+    counts = np.zeros(V)
+    for step_id in range(4):
+        st = oracle.StepState(B, Lt)
+        assert oracle.step(st, logits, np.zeros(B, np.int32), np.full(B, Lt, np.int32), threshold=-1.0, step_id=step_id,
+                           temperature=0.9, sample_seed=7, slices=np.array([0, 4, 8, V], np.int32)) == 0
+        counts += np.bincount(st.tokens.ravel(), minlength=V)
+    expect = softmax(x.astype(np.float64) / 0.9) * counts.sum()
+    assert float(((counts - expect) ** 2 / expect).sum()) < 40.0   # 10 degrees of freedom, p ~ 1e-5
 
 
 def test_sampling_skips_minus_inf_and_flags_bad_rows():
