@@ -136,7 +136,13 @@ typedef struct fork_step_args {
                                 (fallback_rand[b] mod live count) of the block, counted from the left;
                                 read at every step, so a loop's provider may refresh it */
   float temperature;         /* tau >= 0 of Algorithm 2 line 4; 0 = arg-max candidates */
-  uint64_t sample_seed;      /* noise stream of the candidates when tau > 0 */
+  uint64_t sample_seed;      /* stream of uniform variates that draws the candidates when tau > 0 */
+  void* sample_scratch;      /* tau > 0 only: DEVICE scratch of at least fork_sample_scratch_bytes(B, Lt) bytes, 256-byte
+                                aligned, private to one call at a time like the workspace (FORK_ERR_WORKSPACE if missing).
+                                Unlike the workspace it must be ZERO-FILLED before its first use (its first 4*B*Lt
+                                bytes hold per-row arrival counters that every call leaves at zero again; after a call
+                                that reported FORK_DEV_TIMEOUT, zero them once more). */
+  size_t sample_scratch_bytes;
 } fork_step_args;
 
 /*
@@ -204,6 +210,18 @@ typedef struct fork_logprob_bwd_args {
 /* Device scratch needed by any entry point for a batch of B sequences of buffer length Lt. */
 size_t fork_workspace_bytes(int32_t B, int32_t Lt);
 
+/* Additional device scratch of a step that draws its candidates (temperature > 0): 1060 bytes per
+   position plus 2 MB; zero-filled once by the caller (see fork_step_args.sample_scratch).  How the draw works (Algorithm 2 line 4 fixes its distribution, softmax(x / tau),
+   not the method): by inversion.  The vocabulary is laid out in a fixed order -- 16-byte vectors of
+   logits dealt round robin to 256 lanes, lane after lane, the fewer-than-a-vector trailing entries last
+   --, the weights exp((x - max) / tau) are summed along it in the same pass that computes the soft-max
+   statistics (one more exponential per logit), and the candidate is the first entry at which the
+   running sum reaches U times the total, U one uniform variate per position and step from a
+   counter-based generator keyed by sample_seed.  The scratch holds the per-lane sums of every partial
+   result of a row; the warp that delivers a row's last partial result locates the entry from them and
+   re-reads the few dozen vectors of the row it can be in. */
+size_t fork_sample_scratch_bytes(int32_t B, int32_t Lt);
+
 /* One sampling step (Algorithm 2) for all B sequences.  Asynchronous on `stream`. */
 fork_status fork_step(const fork_step_args* args, void* workspace, size_t workspace_bytes, void* stream);
 
@@ -227,8 +245,12 @@ fork_status fork_logprob_backward(const fork_logprob_bwd_args* args, void* works
  *      32-bit words (float, float, float, int32: slice maximum, sum 2^((x-m) log2 e), sum of
  *      (x-m) log2 e * 2^(...), GLOBAL index of the lowest arg-max; s = NaN if the slice holds NaN or
  *      +inf; m = -inf, s = t2 = 0 if it holds nothing but -inf), and with temperature > 0 also
- *      key_out[b,k] = (largest perturbed key, global index of that entry, its logit, 0).  The noise
- *      of an entry depends on its global index, so the draw does not depend on the sharding.
+ *      key_out[b,k] = (sum of the slice's tempered weights against its own maximum, global index of
+ *      the entry the slice would contribute, its logit, 0).  The draw is two-stage: every rank draws
+ *      inside its slice with one uniform variate (the same on all ranks), the select phase picks
+ *      the slice, with probability proportional to its tempered total, with a second one; the
+ *      result is a sample of softmax(x / tau) over the whole vocabulary, and which sample depends
+ *      on how the vocabulary is cut.
  *      part_out / key_out: device, [B,Lt] x 16 bytes, 16-byte aligned; other positions untouched.
  *   2. the caller gathers the N buffers (e.g. one all-gather) into [N][B,Lt] in rank order.
  *   3. fork_vp_select on every rank: merges the N parts of each live row in rank order, derives

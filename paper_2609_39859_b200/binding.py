@@ -38,6 +38,7 @@ class fork_step_args(C.Structure):
         ("nfe", C.c_void_p), ("n_fallback", C.c_void_p),
         ("fallback_mode", C.c_int32), ("fallback_rand", C.c_void_p),
         ("temperature", C.c_float), ("sample_seed", C.c_uint64),
+        ("sample_scratch", C.c_void_p), ("sample_scratch_bytes", C.c_size_t),
     ]
 
 
@@ -77,7 +78,7 @@ class fork_head_args(C.Structure):
 fork_logits_fn = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                              C.c_void_p, C.c_void_p)
 
-EXPORTS = ("fork_workspace_bytes", "fork_step", "fork_step_static", "fork_step_fused_head", "fork_logprob", "fork_decode_loop", "fork_staging_bytes",
+EXPORTS = ("fork_workspace_bytes", "fork_sample_scratch_bytes", "fork_step", "fork_step_static", "fork_step_fused_head", "fork_logprob", "fork_decode_loop", "fork_staging_bytes",
            "fork_select_top_entropy", "fork_grpo_loss", "fork_logprob_backward", "fork_vp_reduce", "fork_vp_reduce_peers", "fork_vp_select", "fork_read_probe",
            "fork_step_host", "fork_device_status", "fork_status_string", "fork_set_tuning",
            "fork_kernel_launches", "fork_mask_handovers", "fork_workspace_release", "fork_set_timing_events")
@@ -100,6 +101,8 @@ def lib():
     L = C.CDLL(path)
     L.fork_workspace_bytes.restype = C.c_size_t
     L.fork_workspace_bytes.argtypes = [C.c_int32, C.c_int32]
+    L.fork_sample_scratch_bytes.restype = C.c_size_t
+    L.fork_sample_scratch_bytes.argtypes = [C.c_int32, C.c_int32]
     L.fork_step.restype = C.c_int
     L.fork_step.argtypes = [C.POINTER(fork_step_args), C.c_void_p, C.c_size_t, C.c_void_p]
     L.fork_step_static.restype = C.c_int
@@ -222,6 +225,15 @@ class ForkState:
         off = (-self.workspace.data_ptr()) % 256
         self.ws_ptr, self.ws_bytes = self.workspace.data_ptr() + off, nbytes
 
+    def sample_scratch_ptr(self):
+        """Device scratch of a step that draws its candidates, allocated when first asked for."""
+        if getattr(self, "_sample_scratch", None) is None:
+            n = int(lib().fork_sample_scratch_bytes(self.B, self.Lt))
+            self._sample_scratch = torch.zeros(n + 256, dtype=torch.uint8, device=self.device)   # (the library wants it zero-filled once)
+            self._sample_bytes = n
+        p = self._sample_scratch.data_ptr()
+        return p + (-p) % 256, self._sample_bytes
+
     def close(self):
         """Give the control block the library keeps for this workspace address back (one-kernel
         steps).  Waits for the device first: the library's condition is that every call that used
@@ -263,6 +275,8 @@ def make_step_args(st: ForkState, logits: torch.Tensor, blk_lo, blk_hi, threshol
         setattr(a, name, getattr(st, name).data_ptr())
     a.fallback_mode, a.fallback_rand = int(fallback_mode), _p(fallback_rand)
     a.temperature, a.sample_seed = float(temperature), int(sample_seed)
+    if temperature > 0:
+        a.sample_scratch, a.sample_scratch_bytes = st.sample_scratch_ptr()
     return a
 
 

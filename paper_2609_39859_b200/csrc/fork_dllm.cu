@@ -245,6 +245,13 @@ static cudaError_t launch_reduce_inner(const ReduceParams& rp, int dtype, int mo
   return launch_direct_dtype(rp, dtype, mode, G, pdl, st);
 }
 
+extern "C" size_t fork_sample_scratch_bytes(int32_t B, int32_t Lt) {
+  if (B < 0 || Lt <= 0) return 0;
+  const size_t rows = (size_t)(B > 0 ? B : 1) * (size_t)Lt;
+  return align_up(rows * sizeof(int32_t), 256) + align_up(rows * sizeof(float4), 256) +
+         (rows + FORK_MAX_GRID) * kSlotStride * sizeof(float);
+}
+
 extern "C" size_t fork_workspace_bytes(int32_t B, int32_t Lt) {
   if (B < 0 || Lt <= 0) return 0;
   return ws_view(nullptr, B, Lt).bytes;
@@ -389,8 +396,22 @@ static fork_status step_impl(const fork_step_args* a, const int32_t* lo, const i
   rp.l2_evict_first = g_tune[FORK_TUNE_L2_EVICT_FIRST].load() >= 0 ? 1 : 0;
   rp.min_units = min_units_setting();
   rp.hdr = w.hdr; rp.seq_off = w.seq_off; rp.expected = w.expected; rp.ticket = w.ticket;
-  rp.rows = w.rows; rp.final_rec = w.final_rec; rp.parts = w.parts; rp.kparts = w.kparts;
-  rp.noise_c = drawn ? (float)(1.4426950408889634 / (double)a->temperature) : 0.f;
+  rp.rows = w.rows; rp.final_rec = w.final_rec; rp.parts = w.parts;
+  if (drawn) {
+    /* lane sums of the tempered weights of every part go to the caller's sample scratch */
+    if (!a->sample_scratch || ((uintptr_t)a->sample_scratch % 256) != 0 ||
+        a->sample_scratch_bytes < fork_sample_scratch_bytes(a->B, a->Lt)) return FORK_ERR_WORKSPACE;
+    {                                                          /* tickets, draws, lane sums: in that order */
+      const size_t rows = (size_t)a->B * (size_t)a->Lt;
+      char* base = (char*)a->sample_scratch;
+      rp.row_ticket = (int32_t*)base;
+      rp.row_draw = (float4*)(base + align_up(rows * sizeof(int32_t), 256));
+      rp.sslots = (float*)(base + align_up(rows * sizeof(int32_t), 256) + align_up(rows * sizeof(float4), 256));
+    }
+    rp.noise_c = (float)(1.4426950408889634 / (double)a->temperature);
+    rp.inv_tau = 1.0f / a->temperature;
+    rp.raise_nats = fminf(32.f, 60.f * a->temperature);      /* tempered exponents stay below 60 * log2(e) < 127 */
+  }
   rp.sample_seed = a->sample_seed;
   rp.tokens = a->tokens; rp.mask = a->mask; rp.threshold = a->threshold; rp.step = a->step;
   rp.conf = a->conf; rp.cand = a->cand; rp.entropy = a->entropy; rp.logp = a->logp; rp.row_status = a->row_status;
@@ -1039,7 +1060,7 @@ extern "C" fork_status fork_vp_select(const fork_step_args* a, const void* parts
   memset(&rp, 0, sizeof(rp));
   rp.B = a->B; rp.Lt = a->Lt; rp.C = 1; rp.min_units = 1;
   rp.hdr = w.hdr; rp.seq_off = w.seq_off; rp.expected = w.expected; rp.ticket = w.ticket;
-  rp.rows = w.rows; rp.final_rec = w.final_rec; rp.parts = w.parts; rp.kparts = w.kparts;
+  rp.rows = w.rows; rp.final_rec = w.final_rec; rp.parts = w.parts;
   rp.tokens = a->tokens; rp.mask = a->mask; rp.threshold = a->threshold; rp.step = a->step;
   rp.conf = a->conf; rp.cand = a->cand; rp.entropy = a->entropy; rp.logp = a->logp; rp.row_status = a->row_status;
   rp.commit_step = a->commit_step; rp.commit_fallback = a->commit_fallback; rp.commit_logp = a->commit_logp;
@@ -1047,6 +1068,8 @@ extern "C" fork_status fork_vp_select(const fork_step_args* a, const void* parts
   rp.nfe = a->nfe; rp.n_fallback = a->n_fallback;
   rp.fallback_mode = a->fallback_mode; rp.fallback_rand = a->fallback_rand;
   rp.vp_parts_in = (const float4*)parts; rp.vp_keys_in = (const float4*)keys; rp.vp_ranks = n_ranks;
+  if (a->temperature > 0.f) rp.noise_c = (float)(1.4426950408889634 / (double)a->temperature);
+  rp.sample_seed = a->sample_seed;
   const dim3 grid((unsigned)((a->B + kVpNT / 32 - 1) / (kVpNT / 32)));
   cudaError_t e = a->temperature > 0.f ? launch(vp_select_kernel<true>, grid, dim3(kVpNT), st, pdl, rp)
                                        : launch(vp_select_kernel<false>, grid, dim3(kVpNT), st, pdl, rp);
@@ -1151,7 +1174,7 @@ extern "C" fork_status fork_step_fused_head(const fork_step_args* a, const fork_
   rp.src.pos0 = a->pos0; rp.src.Ll = a->Ll; rp.src.V = a->V;
   rp.B = a->B; rp.Lt = a->Lt; rp.C = 1; rp.min_units = 1;
   rp.hdr = w.hdr; rp.seq_off = w.seq_off; rp.expected = w.expected; rp.ticket = w.ticket;
-  rp.rows = w.rows; rp.final_rec = w.final_rec; rp.parts = w.parts; rp.kparts = w.kparts;
+  rp.rows = w.rows; rp.final_rec = w.final_rec; rp.parts = w.parts;
   rp.tokens = a->tokens; rp.mask = a->mask; rp.threshold = a->threshold; rp.step = a->step;
   rp.conf = a->conf; rp.cand = a->cand; rp.entropy = a->entropy; rp.logp = a->logp; rp.row_status = a->row_status;
   rp.commit_step = a->commit_step; rp.commit_fallback = a->commit_fallback; rp.commit_logp = a->commit_logp;

@@ -107,15 +107,259 @@ __device__ Part careful_row_warp(const T* row, int V, bool& bad, bool* nonfinite
   return Part{m, s, t, idx};
 }
 
-__device__ __forceinline__ KeyPart key_from(const float2& v) { return KeyPart{v.x, __float_as_int(v.y)}; }
+/* ---- candidates drawn at a temperature (Algorithm 2 line 4, tau > 0): the draw itself ----------
+ * By ONE lane for its row.  The parts of the row carry the sums of the tempered weights per lane of
+ * the draw's order (sslots); U2 times their total is located first among the 256 lanes (then the
+ * trailing elements), then among the parts of that lane (they follow one another in index order),
+ * and last among that lane's vectors inside the part, which are read again (a few dozen 16-byte
+ * loads) and summed element by element.  Returns the token (an index into this buffer) and its logit;
+ * `total` receives the sum of all tempered weights against M. */
+template <typename T>
+__device__ __forceinline__ float tempered_weight(T v, float M, float ct) {
+  const float x = to_f32(v);
+  return (x > -INFINITY) ? ex2_approx((x - M) * ct) : 0.f;
+}
 
-/* Largest perturbed key of row r over its n parts (slots r+g0 ...), by one lane. */
-__device__ __forceinline__ KeyPart merge_row_keys(const ReduceParams& p, int r, int g0, int n) {
-  const float2* q = p.kparts + (r + g0);
-  KeyPart acc = key_empty();
-#pragma unroll 4
-  for (int j = 0; j < n; ++j) acc = key_merge(acc, key_from(__ldcg(q + j)));
-  return acc;
+/* the slow way, for a row whose parts cannot be trusted (it was re-read by the guarded routine):
+   both passes over the whole row in the draw's order */
+template <typename T>
+__device__ __noinline__ int draw_token_scalar(const T* row, int V, float M, float ct, float u, float& xs, float& total) {
+  constexpr int VEC = 16 / (int)sizeof(T);
+  const int nvec = V / VEC;
+  float S = 0.f;
+  for (int e = 0; e < V; ++e) S += tempered_weight(row[e], M, ct);
+  total = S;
+  const float target = u * S;
+  float run = 0.f;
+  int last = -1;
+  for (int lane = 0; lane <= kLanes; ++lane) {
+    const int v0 = lane < kLanes ? lane : nvec, dv = lane < kLanes ? kLanes : 1, v1 = lane < kLanes ? nvec : nvec + 1;
+    for (int vec = v0; vec < v1; vec += dv)
+      for (int e = vec * VEC; e < min(vec * VEC + VEC, V); ++e) {
+        const float w = tempered_weight(row[e], M, ct);
+        if (w > 0.f) { last = e; run += w; if (run >= target) { xs = to_f32(row[e]); return e; } }
+      }
+  }
+  if (last < 0) last = 0;
+  xs = to_f32(row[last]);
+  return last;
+}
+
+/* The draw for row r (sequence b, position k), by a whole WARP, once every part of the row has stored
+   its lane sums: every lane returns the token (-1: nothing in the row has weight), its logit in `xs`,
+   the total of the tempered weights against the row's maximum in `total`.  Three short stretches of
+   loads, each followed by a warp scan: all 256 lane sums of all parts (lane l of the warp holds lanes
+   8l .. 8l+7 of the order, so a scan over the warp follows the order); the chosen lane's share of
+   every part (they follow one another in index order); that lane's vectors inside the chosen part,
+   at most two per lane of the warp, read again and summed element by element. */
+__device__ __forceinline__ float warp_scan_incl(float v) {
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) { const float y = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += y; }
+  return v;
+}
+
+/* Rounding left the running sum a hair short of the target: the last entry of the stretch that has
+   weight stands (one lane, scalar loads; practically never reached). */
+template <typename T>
+__device__ __noinline__ int draw_last_with_weight(const T* row, bool fast, bool in_tail, int first, int nv, int t0, int t1, float M,
+                                                  float ct, float& xs) {
+  constexpr int VEC = 16 / (int)sizeof(T);
+  int tok = -1;
+  if (in_tail) {
+    for (int e = t0; e < t1; ++e) if (tempered_weight(row[e], M, ct) > 0.f) { tok = e; xs = to_f32(row[e]); }
+  } else {
+    for (int i = 0; i < nv; ++i)
+      for (int j = 0; j < VEC; ++j) {
+        const int e = (first + i * kLanes) * VEC + j;
+        if (tempered_weight(row[e], M, ct) > 0.f) { tok = e; xs = to_f32(row[e]); }
+      }
+  }
+  return tok;
+}
+
+template <typename T>
+__device__ __noinline__ int row_draw_warp(const ReduceParams& p, const PartitionCtx& c, int r, int b, int k, float& xs, float& total) {
+  constexpr int VEC = 16 / (int)sizeof(T);
+  const int lane = threadIdx.x & 31;
+  const float ct = p.noise_c;
+  const int g0 = c.owner((long long)r * c.C), n = c.owner((long long)(r + 1) * c.C - 1) - g0 + 1;
+  const float4* pq = p.parts + (r + g0);
+  const float* sq = p.sslots + (size_t)(r + g0) * kSlotStride;
+  const T* row = row_ptr<T>(p.src, b, k);
+  /* The parts' maxima (lane j holds part j's; the rare row with more than 32 parts reads them again
+     as it goes) and, in the same trip to memory, stretch 1: lane sums 8*lane .. 8*lane+7 of the order
+     from every part, and the trailing elements'.  The weights need the row's maximum, the loads do not. */
+  const float m_lane = lane < n ? __ldcg(pq + lane).x : -INFINITY;
+  float M = (m_lane == m_lane) ? m_lane : -INFINITY;
+  for (int j = lane + 32; j < n; j += 32) { const float mj = __ldcg(pq + j).x; if (mj == mj) M = fmaxf(M, mj); }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+  xs = M; total = 0.f;
+  if (!(M > kClamp) || M == INFINITY) return -1;            /* nothing finite: the row is flagged elsewhere */
+  const float w_lane = (m_lane > kClamp && m_lane < INFINITY) ? ex2_approx((m_lane - M) * ct) : 0.f;
+  auto weight = [&](int j) -> float {                        /* weight of part j against the row's maximum */
+    if (j < 32) return __shfl_sync(0xffffffffu, w_lane, j);
+    const float mj = __ldcg(pq + j).x;
+    return (mj > kClamp && mj < INFINITY) ? ex2_approx((mj - M) * ct) : 0.f;
+  };
+  float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  float tail = 0.f;
+  for (int j = 0; j < n; ++j) {
+    const float4* q4 = reinterpret_cast<const float4*>(sq + (size_t)j * kSlotStride) + 2 * lane;
+    const float4 a0 = __ldcg(q4), a1 = __ldcg(q4 + 1);
+    const float tl = __ldcg(sq + (size_t)j * kSlotStride + kSlotTail);
+    const float w = weight(j);
+    v[0] = fmaf(w, a0.x, v[0]); v[1] = fmaf(w, a0.y, v[1]); v[2] = fmaf(w, a0.z, v[2]); v[3] = fmaf(w, a0.w, v[3]);
+    v[4] = fmaf(w, a1.x, v[4]); v[5] = fmaf(w, a1.y, v[5]); v[6] = fmaf(w, a1.z, v[6]); v[7] = fmaf(w, a1.w, v[7]);
+    tail = fmaf(w, tl, tail);
+  }
+  const float mine = ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
+  const float incl = warp_scan_incl(mine);
+  const float S = __shfl_sync(0xffffffffu, incl, 31) + tail;
+  total = S;
+  const float u = sample_uniform_token(sample_row_key(p.sample_seed, p.step, b, k));
+  const float target = u * S;
+  /* the first lane of the warp whose running sum reaches the target, then the lane of the order inside it */
+  const unsigned hit = __ballot_sync(0xffffffffu, incl >= target);
+  int slot = kLanes;                                         /* the trailing elements unless a lane takes it */
+  float rest = target - __shfl_sync(0xffffffffu, incl, 31);  /* ... what is left to cover there */
+  if (hit) {
+    const int wl = __ffs(hit) - 1;
+    float run = incl - mine;                                 /* sum of the lanes before this one's eight */
+    int sl = 8 * lane + 7;                                   /* (the last of the eight if rounding leaves the sum short) */
+    bool found = false;
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      if (!found) { if (run + v[i] >= target || i == 7) { sl = 8 * lane + i; found = true; } else run += v[i]; }
+    slot = __shfl_sync(0xffffffffu, sl, wl);
+    rest = target - __shfl_sync(0xffffffffu, run, wl);
+  }
+  /* stretch 2: which part of the row (a lane's vectors of part j come before those of part j + 1) */
+  int js = 0;
+  if (n > 1) {
+    js = n - 1;
+    float before = 0.f;
+    bool done = false;
+    for (int j0 = 0; j0 < n && !done; j0 += 32) {
+      const int j = j0 + lane;
+      const float wj = (j0 == 0) ? w_lane : (j < n ? weight(j) : 0.f);   /* round one: lane j holds part j's weight; later rounds (j >= 32) read it again */
+      const float pj = j < n ? wj * __ldcg(sq + (size_t)j * kSlotStride + slot) : 0.f;
+      const float inc = warp_scan_incl(pj);
+      const unsigned h2 = __ballot_sync(0xffffffffu, j < n && before + inc >= rest);
+      if (h2) {
+        const int wl = __ffs(h2) - 1;
+        js = j0 + wl;
+        rest -= before + __shfl_sync(0xffffffffu, inc - pj, wl);
+        done = true;
+      } else {
+        before += __shfl_sync(0xffffffffu, inc, 31);
+      }
+    }
+    if (!done) rest -= before - weight(n - 1) * __ldcg(sq + (size_t)(n - 1) * kSlotStride + slot);   /* rounding left the sum short: the last part */
+  }
+  /* stretch 3: the part's stretch of the row; the lane's vectors (or the trailing elements) inside it */
+  const int g = g0 + js;
+  int ub, ue;                                                /* the part's units, relative to the row's first */
+  if (c.small) {
+    ub = (int)((uint32_t)g * (uint32_t)c.U / (uint32_t)c.G) - r * c.C;
+    ue = (int)((uint32_t)(g + 1) * (uint32_t)c.U / (uint32_t)c.G) - r * c.C;
+  } else {
+    ub = (int)(fork_part_begin(c.U, c.G, g) - (long long)r * c.C);
+    ue = (int)(fork_part_begin(c.U, c.G, g + 1) - (long long)r * c.C);
+  }
+  ub = max(ub, 0); ue = min(ue, c.C);
+  const int e0 = ub * FORK_CHUNK, e1 = min(ue * FORK_CHUNK, p.src.V);
+  const int Vf = (p.src.V / VEC) * VEC;
+  const bool in_tail = slot >= kLanes;
+  /* entries are visited 64 vectors a round, two consecutive ones per lane of the warp, so that a scan
+     over the warp follows the order; the trailing elements (fewer than a vector) are one "vector" of
+     lane 0.  The running sum carries over from round to round. */
+  const int first = in_tail ? 0 : e0 / VEC + slot;
+  const int end_v = min(e1, Vf) / VEC;
+  const int nv = in_tail ? 1 : (end_v > first ? (end_v - first + kLanes - 1) / kLanes : 0);
+  float before = 0.f;
+  int tok = -1;
+  float x_tok = M;
+  for (int base = 0; base < nv && tok < 0; base += 64) {
+    float x[2 * VEC];
+    float both = 0.f;
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      const int i = base + 2 * lane + q;
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) x[q * VEC + j] = -INFINITY;
+      if (i < nv) {
+        if (in_tail) {
+          for (int j = 0; j < VEC; ++j) { const int e = max(e0, Vf) + j; if (e < e1) x[j] = to_f32(row[e]); }
+        } else {
+          const size_t at = (size_t)(first + i * kLanes) * VEC;
+          T raw[VEC];
+          if (p.fast) *reinterpret_cast<uint4*>(raw) = __ldg(reinterpret_cast<const uint4*>(row + at));
+          else
+            for (int j = 0; j < VEC; ++j) raw[j] = row[at + j];
+#pragma unroll
+          for (int j = 0; j < VEC; ++j) x[q * VEC + j] = to_f32(raw[j]);
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 2 * VEC; ++j) both += (x[j] > -INFINITY) ? ex2_approx((x[j] - M) * ct) : 0.f;
+    const float inc = warp_scan_incl(both);
+    const unsigned hit3 = __ballot_sync(0xffffffffu, both > 0.f && before + inc >= rest);
+    if (hit3) {
+      const int wl = __ffs(hit3) - 1;
+      int te = -1; float tx = M;
+      if (lane == wl) {
+        float acc = before + inc - both;
+        bool got = false;
+        for (int j = 0; j < 2 * VEC; ++j) {
+          const float w = (x[j] > -INFINITY) ? ex2_approx((x[j] - M) * ct) : 0.f;
+          if (w > 0.f && !got) {                             /* (the lane's last entry with weight stands if rounding leaves it short) */
+            acc += w;
+            const int q = j / VEC;
+            te = in_tail ? max(e0, Vf) + j : (first + (base + 2 * lane + q) * kLanes) * VEC + (j - q * VEC);
+            tx = x[j];
+            got = acc >= rest;
+          }
+        }
+      }
+      tok = __shfl_sync(0xffffffffu, te, wl); x_tok = __shfl_sync(0xffffffffu, tx, wl);
+    } else {
+      before += __shfl_sync(0xffffffffu, inc, 31);
+    }
+  }
+  if (tok < 0 && nv > 0) tok = draw_last_with_weight<T>(row, p.fast != 0, in_tail, first, nv, max(e0, Vf), e1, M, ct, x_tok);
+  xs = x_tok;
+  return tok;
+}
+
+/* After the calling warp has stored the lane sums of part (r, g): count the part in, and if it was
+   the row's last, draw the row's candidate and leave it in row_draw[r] for whoever finalises the
+   sequence.  Must run before the warp takes the sequence's ticket. */
+template <typename T>
+__device__ __forceinline__ void row_part_arrived(const ReduceParams& p, const PartitionCtx& c, int r, int b, int k) {
+  const int lane = threadIdx.x & 31;
+  const int n = c.owner((long long)(r + 1) * c.C - 1) - c.owner((long long)r * c.C) + 1;
+  int last = 1;
+  if (n > 1) {
+    __threadfence();
+    __syncwarp();
+    if (lane == 0) {
+      int old;
+      asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(p.row_ticket + r) : "memory");
+      last = (old + 1 == n) ? 1 : 0;
+      if (last) p.row_ticket[r] = 0;                         /* zero again for the next launch */
+    }
+    last = __shfl_sync(0xffffffffu, last, 0);
+  }
+  if (last) {
+    float xs, total;
+    const int tok = row_draw_warp<T>(p, c, r, b, k, xs, total);
+    if (lane == 0) p.row_draw[r] = make_float4(__int_as_float(tok), xs, total, 0.f);
+    __threadfence();
+    __syncwarp();
+  }
 }
 
 /* Final statistics of up to 32 rows (one per lane) of sequence b starting at row `base`.
@@ -125,7 +369,7 @@ __device__ __forceinline__ KeyPart merge_row_keys(const ReduceParams& p, int r, 
 /* Rows base .. base+31 of sequence b, one per lane: the row's parts merged, rows whose streamed
    result is not finite re-read by the whole warp with the guarded routine. */
 struct MergedRow {
-  Part merged; int k, g0, nparts; bool valid, bad, nonfinite;
+  Part merged; int k, g0, nparts; bool valid, bad, nonfinite, reread;
 };
 template <typename T>
 __device__ __forceinline__ MergedRow merge_rows_warp(const ReduceParams& p, const RowMap& rm, const PartitionCtx& c, int b,
@@ -133,7 +377,7 @@ __device__ __forceinline__ MergedRow merge_rows_warp(const ReduceParams& p, cons
   const int lane = threadIdx.x & 31;
   const int r = base + lane;
   MergedRow m;
-  m.valid = r < r1; m.bad = false; m.nonfinite = false;
+  m.valid = r < r1; m.bad = false; m.nonfinite = false; m.reread = false;
   m.merged = part_empty();
   m.k = 0; m.g0 = 0; m.nparts = 0;
   bool redo = false;
@@ -154,7 +398,7 @@ __device__ __forceinline__ MergedRow merge_rows_warp(const ReduceParams& p, cons
     const int kk = __shfl_sync(0xffffffffu, m.k, src);
     bool bd, nf;
     const Part cp = careful_row_warp<T>(row_ptr<T>(p.src, b, kk), p.src.V, bd, &nf);
-    if (lane == src) { m.merged = cp; m.bad = bd; m.nonfinite = nf; }
+    if (lane == src) { m.merged = cp; m.bad = bd; m.nonfinite = nf; m.reread = true; }
   }
   return m;
 }
@@ -169,9 +413,19 @@ __device__ __forceinline__ RowOut finalize_rows_warp(const ReduceParams& p, cons
   if (SAMPLE) {
     float xs = 0.f;
     if (m.valid && !m.bad) {
-      const KeyPart kp = merge_row_keys(p, r, m.g0, m.nparts);
-      const NoiseRow nz = noise_row(p.sample_seed, p.step, b, k, p.noise_c, (uint32_t)p.vocab_offset);
-      m.merged.idx = resolve_sample<T>(row_ptr<T>(p.src, b, k), nz, kp.vec, p.src.V, kp.key, xs);
+      const T* row = row_ptr<T>(p.src, b, k);
+      const int greedy = resolve_index<T>(row, m.merged.idx, p.src.V, m.merged.m);
+      float total;
+      int tok;
+      if (m.reread) {
+        const float u = sample_uniform_token(sample_row_key(p.sample_seed, p.step, b, k));
+        tok = draw_token_scalar<T>(row, p.src.V, m.merged.m, p.noise_c, u, xs, total);
+      } else {
+        const float4 d = __ldcg(p.row_draw + r);             /* left there by the warp that delivered the row's last part */
+        tok = __float_as_int(d.x); xs = d.y;
+      }
+      if (tok < 0) { tok = greedy; xs = m.merged.m; }
+      m.merged.idx = tok;
     }
     merged = m.merged;
     return row_out_sampled(merged, m.bad, xs);
@@ -281,7 +535,7 @@ __device__ void finalize_vp_local(const ReduceParams& p, const RowMap& rm, const
     if (!m.valid) continue;
     const size_t at = (size_t)b * p.Lt + m.k;
     const T* row = row_ptr<T>(p.src, b, m.k);
-    float4 out, kout = make_float4(-INFINITY, __int_as_float(kIdxNone), 0.f, 0.f);
+    float4 out, kout = make_float4(0.f, __int_as_float(kIdxNone), 0.f, 0.f);
     if (m.bad && !m.nonfinite) {
       out = make_float4(-INFINITY, 0.f, 0.f, __int_as_float(p.vocab_offset));
     } else if (m.bad) {
@@ -290,11 +544,19 @@ __device__ void finalize_vp_local(const ReduceParams& p, const RowMap& rm, const
       const int idx = resolve_index<T>(row, m.merged.idx, p.src.V, m.merged.m);
       out = make_float4(m.merged.m, m.merged.s, m.merged.t, __int_as_float(p.vocab_offset + idx));
       if (SAMPLE) {
-        const KeyPart kp = merge_row_keys(p, r, m.g0, m.nparts);
-        const NoiseRow nz = noise_row(p.sample_seed, p.step, b, m.k, p.noise_c, (uint32_t)p.vocab_offset);
-        float xs;
-        const int si = resolve_sample<T>(row, nz, kp.vec, p.src.V, kp.key, xs);
-        kout = make_float4(kp.key, __int_as_float(p.vocab_offset + si), xs, 0.f);
+        /* the slice's own draw (with U2), and the sum of its tempered weights against its maximum:
+           the select phase picks the slice with U1 and takes that slice's token */
+        float xs = m.merged.m, total = 0.f;
+        int si;
+        if (m.reread) {
+          const float u = sample_uniform_token(sample_row_key(p.sample_seed, p.step, b, m.k));
+          si = draw_token_scalar<T>(row, p.src.V, m.merged.m, p.noise_c, u, xs, total);
+        } else {
+          const float4 d = __ldcg(p.row_draw + r);
+          si = __float_as_int(d.x); xs = d.y; total = d.z;
+        }
+        if (si < 0) { si = idx; xs = m.merged.m; }
+        kout = make_float4(total, __int_as_float(p.vocab_offset + si), xs, 0.f);
       }
     }
     if (p.vp_peers > 0) {
@@ -328,12 +590,26 @@ __device__ __forceinline__ RowOut gathered_rows_warp(const ReduceParams& p, cons
   for (int j = 0; j < p.vp_ranks; ++j) acc = part_merge(acc, part_from(__ldg(p.vp_parts_in + j * n + at)));
   const bool bad = !(isfinite(acc.s) && isfinite(acc.t)) || !(acc.m > -INFINITY) || acc.m == INFINITY;
   if (!SAMPLE || bad) return row_out_from(acc, bad);
-  float best = -INFINITY, xs = 0.f;
-  int bidx = kIdxNone;
+  /* the slice by inversion with U1 over the slices' tempered totals (each against its own maximum,
+     re-weighted to the row's), in rank order; the token is that slice's own draw */
+  const float u1 = sample_uniform_slice(sample_row_key(p.sample_seed, p.step, b, k));
+  float grand = 0.f;
   for (int j = 0; j < p.vp_ranks; ++j) {
+    const float mj = __ldg(p.vp_parts_in + j * n + at).x;
+    if (mj > -INFINITY && mj < INFINITY) grand += __ldg(p.vp_keys_in + j * n + at).x * ex2_approx((mj - acc.m) * p.noise_c);
+  }
+  const float target = u1 * grand;
+  float run = 0.f, xs = acc.m;
+  int bidx = acc.idx;
+  for (int j = 0; j < p.vp_ranks; ++j) {
+    const float mj = __ldg(p.vp_parts_in + j * n + at).x;
+    if (!(mj > -INFINITY && mj < INFINITY)) continue;
     const float4 q = __ldg(p.vp_keys_in + j * n + at);
-    const int qi = __float_as_int(q.y);
-    if (q.x > best || (q.x == best && qi < bidx)) { best = q.x; bidx = qi; xs = q.z; }
+    const float wj = q.x * ex2_approx((mj - acc.m) * p.noise_c);
+    if (!(wj > 0.f)) continue;
+    run += wj;
+    bidx = __float_as_int(q.y); xs = q.z;                     /* (the last slice with weight stands if rounding leaves the sum short) */
+    if (run >= target) break;
   }
   acc.idx = bidx;
   return row_out_sampled(acc, false, xs);
@@ -491,12 +767,13 @@ __device__ void finalize_logprob_sequence(const ReduceParams& p, const RowMap& r
 
 /* Lane 0 of the calling warp publishes one part of row r (sequence b) and takes a ticket; returns
    (to every lane) whether this was the last part the sequence was waiting for. */
-__device__ __forceinline__ bool publish_part(const ReduceParams& p, const Part& part, int r, int g, int b, int want,
-                                             const KeyPart* kp = nullptr) {
+__device__ __forceinline__ void store_part(const ReduceParams& p, const Part& part, int r, int g) {
+  if ((threadIdx.x & 31) == 0) p.parts[r + g] = make_float4(part.m, part.s, part.t, __int_as_float(part.idx));
+}
+__device__ __forceinline__ bool publish_part(const ReduceParams& p, const Part& part, int r, int g, int b, int want) {
   int last = 0;
   if ((threadIdx.x & 31) == 0) {
     p.parts[r + g] = make_float4(part.m, part.s, part.t, __int_as_float(part.idx));
-    if (kp) p.kparts[r + g] = make_float2(kp->key, __int_as_float(kp->vec));
     int old;                                 /* release our part, acquire everybody else's */
     asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(p.ticket + b) : "memory");
     last = (old + 1 == want) ? 1 : 0;

@@ -71,7 +71,6 @@ struct WsView {
   int2* rows;                        /* [B*Lt] (b, k) of each live row, ascending */
   float4* final_rec;                 /* [B*Lt] per-row results kept between the finaliser's passes */
   float4* parts;                     /* [B*Lt + FORK_MAX_GRID] partial results, slot r+g */
-  float2* kparts;                    /* [B*Lt + FORK_MAX_GRID] best perturbed key of each part (stochastic candidates) */
   uint32_t* commit_bits;             /* [B * ceil(Lt/32)] positions committed by a step whose mask update was handed on */
   VpPeerTable* vp_peer_tab;          /* gather-buffer addresses of a vocabulary-parallel reduction with the exchange fused in */
   float4* head_parts;                /* [splits][row blocks * 128] per-row results of the fused LM-head step, one per vocabulary split */
@@ -97,7 +96,6 @@ static WsView ws_view(void* base, int32_t B, int32_t Lt) {
   v.rows = (int2*)(p + off); off = align_up(off + rows * sizeof(int2), 256);
   v.final_rec = (float4*)(p + off); off = align_up(off + rows * sizeof(float4), 256);
   v.parts = (float4*)(p + off); off = align_up(off + (rows + FORK_MAX_GRID) * sizeof(float4), 256);
-  v.kparts = (float2*)(p + off); off = align_up(off + (rows + FORK_MAX_GRID) * sizeof(float2), 256);
   v.commit_bits = (uint32_t*)(p + off); off = align_up(off + nb * (size_t)(((Lt > 0 ? Lt : 1) + 31) / 32) * 4, 256);
   v.vp_peer_tab = (VpPeerTable*)(p + off); off = align_up(off + sizeof(VpPeerTable), 256);
   v.head_parts = (float4*)(p + off); off = align_up(off + (rows + kHeadPartsExtra) * sizeof(float4), 256);
@@ -154,9 +152,15 @@ struct ReduceParams {
   LoopCtl* loop;                     /* a step of fork_decode_loop: where the cursors of the next step go (else NULL) */
   int vocab_offset;                  /* vocabulary-parallel slices: global index of entry 0 of this buffer */
   WsHeader* hdr; const int2* rows; const int32_t* seq_off; const int32_t* expected; int32_t* ticket;   /* workspace */
-  float noise_c; int32_t step; unsigned long long sample_seed;   /* stochastic candidates: log2(e)/tau and the noise stream */
+  float noise_c; int32_t step; unsigned long long sample_seed;   /* stochastic candidates: log2(e)/tau and the stream of uniforms */
+  float inv_tau, raise_nats;         /* ... 1/tau, and how far above a thread's reference the running maximum may rise
+                                        before the reference follows (keeps the tempered exponents in range) */
   /* read at segment ends and in the finalisation */
-  float4* parts; float2* kparts; float4* final_rec; uint32_t* commit_bits;
+  float4* parts; float4* final_rec; uint32_t* commit_bits;
+  /* candidates drawn at a temperature; all three in the caller's sample scratch */
+  float* sslots;                     /* [B*Lt + FORK_MAX_GRID][kSlotStride] lane sums of the tempered weights of every part */
+  int32_t* row_ticket;               /* [B*Lt] parts of a row that have arrived; zero between launches */
+  float4* row_draw;                  /* [B*Lt] per live row: (drawn token, its logit, total of the tempered weights, -) */
   int32_t* tokens; float threshold; int fallback_mode; const uint32_t* fallback_rand;
   float* conf; int32_t* cand; float* entropy; float* logp; uint32_t* row_status;
   int32_t* commit_step; uint8_t* commit_fallback; float* commit_logp;

@@ -165,29 +165,42 @@ __device__ __forceinline__ bool any_gt_bf16x2(uint32_t a, uint32_t b) {
   return r != 0;
 }
 
-template <typename T, bool WITH_T, bool CLAMP>
+template <typename T, bool WITH_T, bool CLAMP, bool TEMP = false>
 struct Acc;
 
 /* Shared arithmetic: four accumulator lanes held as two f32x2 pairs, so that y = x*L - ref*L,
    s += e and t += y*e each take ONE packed instruction (fma.rn.f32x2 / add.rn.f32x2, sm_100)
-   per pair of logits; the two exp2 of a pair stay scalar (MUFU has no packed form). */
-template <bool WITH_T>
+   per pair of logits; the two exp2 of a pair stay scalar (MUFU has no packed form).
+   TEMP (candidates drawn at a temperature): a third sum, the tempered weights 2^{y / tau}, costs
+   one packed multiply, two more exp2 and one packed add per pair; `tail_st` collects the tempered
+   weights of the fewer-than-a-vector trailing elements, which the draw visits last. */
+template <bool WITH_T, bool TEMP>
 struct AccCore {
   float ref;                   /* reference, -inf before the first group */
   float2 nrefL2;               /* (-ref*L, -ref*L) */
   float2 s2[2], t2[2];
+  float2 st2[2];               /* TEMP: sum 2^{(x-ref) L / tau} */
+  float inv_tau, tail_st;      /* TEMP */
+  float raise_nats;            /* the reference is raised when the running maximum exceeds it by this much */
 
   __device__ __forceinline__ void init_core() {
     ref = -INFINITY; nrefL2 = make_float2(INFINITY, INFINITY);
     s2[0] = s2[1] = t2[0] = t2[1] = make_float2(0.f, 0.f);
+    st2[0] = st2[1] = make_float2(0.f, 0.f);
+    inv_tau = 1.f; tail_st = 0.f; raise_nats = 32.f;
   }
+  __device__ __forceinline__ float raise_margin() const { return TEMP ? raise_nats : kRaiseNats; }
+  /* temperature of the draw; exponents up to raise_nats * L / tau must stay below the range of exp2 */
+  __device__ __forceinline__ void set_temperature(float inv_tau_, float raise_nats_) { inv_tau = inv_tau_; raise_nats = raise_nats_; }
   __device__ __forceinline__ void rescale(float newref) {
     if (ref <= kClamp) {                     /* nothing but -inf so far: weight 0 (NaN is kept) */
 #pragma unroll
       for (int j = 0; j < 2; ++j) {
         s2[j].x *= 0.f; s2[j].y *= 0.f;
         if (WITH_T) { t2[j].x *= 0.f; t2[j].y *= 0.f; }
+        if (TEMP) { st2[j].x = 0.f; st2[j].y = 0.f; }
       }
+      if (TEMP) tail_st = 0.f;
     } else {
       const float d = (ref - newref) * kLog2e;
       const float w = ex2_approx(d);
@@ -195,6 +208,12 @@ struct AccCore {
       for (int j = 0; j < 2; ++j) {
         if (WITH_T) { t2[j].x = w * fmaf(d, s2[j].x, t2[j].x); t2[j].y = w * fmaf(d, s2[j].y, t2[j].y); }
         s2[j].x *= w; s2[j].y *= w;
+      }
+      if (TEMP) {
+        const float wt = ex2_approx(d * inv_tau);
+#pragma unroll
+        for (int j = 0; j < 2; ++j) { st2[j].x *= wt; st2[j].y *= wt; }
+        tail_st *= wt;
       }
     }
     ref = newref;
@@ -207,12 +226,18 @@ struct AccCore {
     const float2 e = make_float2(ex2_approx(y.x), ex2_approx(y.y));
     s2[k] = __fadd2_rn(s2[k], e);
     if (WITH_T) t2[k] = __ffma2_rn(y, e, t2[k]);
+    if (TEMP) {
+      const float2 yt = __fmul2_rn(y, make_float2(inv_tau, inv_tau));
+      st2[k] = __fadd2_rn(st2[k], make_float2(ex2_approx(yt.x), ex2_approx(yt.y)));
+    }
   }
+  /* one trailing element (after all of the thread's vectors) */
   __device__ __forceinline__ void add1(float x) {
     const float y = fmaf(x, kLog2e, nrefL2.x);
     const float e = ex2_approx(y);
     s2[0].x += e;
     if (WITH_T) t2[0].x = fmaf(y, e, t2[0].x);
+    if (TEMP) tail_st += ex2_approx(y * inv_tau);
   }
   /* (s, t) re-expressed against the true maximum m >= ref */
   __device__ __forceinline__ void totals(float m, float& ss, float& tt) const {
@@ -225,13 +250,23 @@ struct AccCore {
       ss *= w;
     }
   }
+  /* TEMP: the tempered weights of the thread's vectors, and of its trailing elements, against m >= ref */
+  __device__ __forceinline__ void tempered(float m, float& vec_sum, float& tail_sum) const {
+    vec_sum = (st2[0].x + st2[0].y) + (st2[1].x + st2[1].y);
+    tail_sum = tail_st;
+    if (!(ref > kClamp)) { vec_sum = 0.f; tail_sum = 0.f; return; }
+    if (ref != m) {
+      const float w = ex2_approx((ref - m) * kLog2e * inv_tau);
+      vec_sum *= w; tail_sum *= w;
+    }
+  }
 };
 
 /* ---- bf16: 8 logits per 128-bit vector --------------------------------------------------------
  * CLAMP = false is the normal path: -inf logits are NOT clamped, so a thread that meets one ends
  * with a NaN in t (0 * -inf) and redoes its own vectors with CLAMP = true (see stream_thread). */
-template <bool WITH_T, bool CLAMP>
-struct Acc<bf16_t, WITH_T, CLAMP> : AccCore<WITH_T> {
+template <bool WITH_T, bool CLAMP, bool TEMP>
+struct Acc<bf16_t, WITH_T, CLAMP, TEMP> : AccCore<WITH_T, TEMP> {
   static constexpr int VEC = 8;
   uint32_t thr2;               /* packed bf16x2 (ref + kRaiseNats): a running max above it raises the reference */
   uint32_t pm;                 /* running packed maximum of the logits */
@@ -245,7 +280,7 @@ struct Acc<bf16_t, WITH_T, CLAMP> : AccCore<WITH_T> {
   }
   __device__ __forceinline__ void raise(float newref) {
     this->rescale(newref);
-    const uint32_t tb = __float_as_uint(newref + kRaiseNats) >> 16;
+    const uint32_t tb = __float_as_uint(newref + this->raise_margin()) >> 16;
     thr2 = tb | (tb << 16);
   }
   /* N vectors; vector j starts at vocabulary index base + j*stride.  track() touches every loaded
@@ -284,7 +319,7 @@ struct Acc<bf16_t, WITH_T, CLAMP> : AccCore<WITH_T> {
   __device__ __forceinline__ void one(float x, int idx) {
     if (CLAMP) x = max_nan_f32(x, kClamp);
     if (x > tail_m) { tail_m = x; tail_idx = idx; }
-    if (x > this->ref + kRaiseNats || this->ref == -INFINITY) raise(fmaxf(x, this->ref));
+    if (x > this->ref + this->raise_margin() || this->ref == -INFINITY) raise(fmaxf(x, this->ref));
     this->add1(x);
   }
   __device__ __forceinline__ Part part() const {
@@ -302,8 +337,8 @@ struct Acc<bf16_t, WITH_T, CLAMP> : AccCore<WITH_T> {
 };
 
 /* ---- fp32: 4 logits per 128-bit vector -------------------------------------------------------- */
-template <bool WITH_T, bool CLAMP>
-struct Acc<float, WITH_T, CLAMP> : AccCore<WITH_T> {
+template <bool WITH_T, bool CLAMP, bool TEMP>
+struct Acc<float, WITH_T, CLAMP, TEMP> : AccCore<WITH_T, TEMP> {
   static constexpr int VEC = 4;
   float thr;
   float fm;                    /* running maximum of the logits */
@@ -317,7 +352,7 @@ struct Acc<float, WITH_T, CLAMP> : AccCore<WITH_T> {
   }
   __device__ __forceinline__ void raise(float newref) {
     this->rescale(newref);
-    thr = newref + kRaiseNats;
+    thr = newref + this->raise_margin();
   }
   template <int N>
   __device__ __forceinline__ void track(uint4 (&v)[N], int base, int stride) {
@@ -352,7 +387,7 @@ struct Acc<float, WITH_T, CLAMP> : AccCore<WITH_T> {
   __device__ __forceinline__ void one(float x, int idx) {
     if (CLAMP) x = max_nan_f32(x, kClamp);
     if (x > tail_m) { tail_m = x; tail_idx = idx; }
-    if (x > this->ref + kRaiseNats || this->ref == -INFINITY) raise(fmaxf(x, this->ref));
+    if (x > this->ref + this->raise_margin() || this->ref == -INFINITY) raise(fmaxf(x, this->ref));
     this->add1(x);
   }
   __device__ __forceinline__ Part part() const {
@@ -369,126 +404,34 @@ struct Acc<float, WITH_T, CLAMP> : AccCore<WITH_T> {
 __device__ __forceinline__ bool part_is_finite(const Part& p) { return isfinite(p.s) && isfinite(p.t); }
 
 /* ------------------------------------------------------------------------------------------ */
-/* Stochastic candidates (Algorithm 2 line 4 with tau > 0): x_0 ~ softmax(x / tau) drawn as
- * arg-max_v (x_v / tau + g_v), g_v standard Gumbel noise (Gumbel-max).  The noise stream is a
- * counter-based generator: a 64-bit key per (seed, step, sequence, position), a 32-bit hash per
- * vocabulary entry, the uniform u = ((h mod 2^23) + 1/2) 2^-23, g = -ln E with E = -ln u.
- * Keys are compared in log2 units with constants dropped:  key = x * (log2 e / tau) - log2(E / ln 2).
- * E / ln 2 = -log2 u comes from lg2.approx, except close to u = 1, where that instruction has only
- * an absolute error bound and the series -log2(1 - w) = (w + w^2/2 + ...) / ln 2 in w = 1 - u (exact)
- * is used instead (w < 2^-8: the dropped terms are below 2e-6 relative).                          */
-struct NoiseRow {
-  uint32_t lo, hi;             /* the row's key */
-  float c;                     /* log2(e) / tau */
-  uint32_t voff;               /* global vocabulary index of the buffer's entry 0 (a vocabulary-parallel slice) */
-};
+/* Stochastic candidates (Algorithm 2 line 4 with tau > 0): x_0 ~ softmax(x / tau), drawn by inversion.
+ * The vocabulary (of a buffer: the whole of it, or one rank's slice) is laid out in a fixed order --
+ * 128-bit vectors dealt round robin to 256 lanes, lane after lane, the fewer-than-a-vector trailing
+ * elements last: the order in which a CTA's 256 streaming threads meet them -- the tempered weights
+ * 2^{(x - m) L / tau} are summed along it, and the token is the first at which the running sum reaches
+ * U2 times the total.  With the vocabulary in slices the slice is drawn first, with U1.  The two
+ * uniforms come from disjoint bit fields of one 64-bit key per (seed, step, sequence, position). */
+constexpr int kLanes = 256;                /* lanes of the draw's order = streaming threads of a CTA / consumer threads of a half */
+/* floats per part in the lane-sum storage: 256 lane sums, the trailing elements, the total, 2 spare
+   (a multiple of 4) */
+constexpr int kSlotTail = kLanes, kSlotTotal = kLanes + 1;
+constexpr int kSlotStride = kLanes + 4;
 
 __device__ __forceinline__ uint64_t noise_mix64(uint64_t z) {
   z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ull; z ^= z >> 27; z *= 0x94D049BB133111EBull; z ^= z >> 31;
   return z;
 }
-__device__ __forceinline__ NoiseRow noise_row(uint64_t seed, int step, int b, int k, float c, uint32_t voff) {
+__device__ __forceinline__ uint64_t sample_row_key(uint64_t seed, int step, int b, int k) {
   uint64_t z = noise_mix64(seed + 0x9E3779B97F4A7C15ull * (uint64_t)((uint32_t)step + 1u));
-  z = noise_mix64(z ^ (((uint64_t)(uint32_t)b << 32) | (uint64_t)(uint32_t)k));
-  return NoiseRow{(uint32_t)z, (uint32_t)(z >> 32), c, voff};
+  return noise_mix64(z ^ (((uint64_t)(uint32_t)b << 32) | (uint64_t)(uint32_t)k));
 }
-__device__ __forceinline__ float lg2_approx(float x) {
-  float y;
-  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-/* perturbed key of logit x at vocabulary index v */
-__device__ __forceinline__ float noise_key(const NoiseRow& nz, float x, uint32_t v) {
-  uint64_t p = (uint64_t)((v + nz.voff) ^ nz.hi) * 0x9E3779B1ull;   /* two multiply-and-fold rounds */
-  uint32_t h = (uint32_t)(p >> 32) ^ (uint32_t)p ^ nz.lo;
-  p = (uint64_t)h * 0x85EBCA77ull;
-  h = (uint32_t)(p >> 32) ^ (uint32_t)p;
-  const float f = __uint_as_float((h & 0x007fffffu) | 0x3f800000u);   /* 1 + n 2^-23 */
-  const float u = f - 0.99999994f;                           /* (2n+1) 2^-24, exact */
-  const float w = 1.0f - u;                                  /* (2^24 - 2n - 1) 2^-24, exact */
-  /* E / ln 2 = -log2 u, from the series in w where lg2.approx is not accurate enough */
-  const float series = w * __fmaf_rn(0.72134752f, w, 1.44269504f);
-  const float e2 = (w < 0.00390625f) ? series : -lg2_approx(u);
-  return __fmaf_rn(x, nz.c, -lg2_approx(e2));                /* log2(ln 2) is the same for every entry: dropped */
-}
+/* ((n + 1/2) 2^-23: exact in fp32) */
+__device__ __forceinline__ float sample_uniform_token(uint64_t key) { return ((float)(uint32_t)(key >> 41) + 0.5f) * (1.0f / 8388608.0f); }
+__device__ __forceinline__ float sample_uniform_slice(uint64_t key) { return ((float)(uint32_t)((key >> 18) & 0x7FFFFFu) + 0.5f) * (1.0f / 8388608.0f); }
 
-/* The largest perturbed key a thread / warp / CTA / row has seen, and where: `vec` is the start of
-   the 128-bit vector holding it (or the exact index for elements handled one at a time); equal keys
-   go to the lower position.  resolve_sample() recomputes the keys of that vector to find the
-   element. */
-struct KeyPart {
-  float key; int vec;
-};
-__device__ __forceinline__ KeyPart key_empty() { return KeyPart{-INFINITY, kIdxNone}; }
-__device__ __forceinline__ KeyPart key_merge(const KeyPart& a, const KeyPart& b) {
-  const bool bwins = (b.key > a.key) || (b.key == a.key && b.vec < a.vec);
-  return bwins ? b : a;
-}
-__device__ __forceinline__ KeyPart key_warp_reduce(KeyPart p) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    KeyPart q;
-    q.key = __shfl_xor_sync(0xffffffffu, p.key, o);
-    q.vec = __shfl_xor_sync(0xffffffffu, p.vec, o);
-    p = key_merge(p, q);
-  }
-  return p;
-}
-
-struct KeyTrack {
-  KeyPart best;
-  __device__ __forceinline__ void init() { best = key_empty(); }
-  /* N vectors; vector j starts at vocabulary index base + j*stride (ascending within a thread, so a
-     strict comparison keeps the lowest position among equal keys) */
-  template <int N>
-  __device__ __forceinline__ void update(bf16_t, const NoiseRow& nz, const uint4 (&v)[N], int base, int stride) {
-#pragma unroll
-    for (int j = 0; j < N; ++j) {
-      const uint32_t e = (uint32_t)(base + j * stride);
-      float k0 = noise_key(nz, bf16_lo(v[j].x), e), k1 = noise_key(nz, bf16_hi(v[j].x), e + 1);
-      float k2 = noise_key(nz, bf16_lo(v[j].y), e + 2), k3 = noise_key(nz, bf16_hi(v[j].y), e + 3);
-      float k4 = noise_key(nz, bf16_lo(v[j].z), e + 4), k5 = noise_key(nz, bf16_hi(v[j].z), e + 5);
-      float k6 = noise_key(nz, bf16_lo(v[j].w), e + 6), k7 = noise_key(nz, bf16_hi(v[j].w), e + 7);
-      const float vm = fmaxf(fmaxf(fmaxf(k0, k1), fmaxf(k2, k3)), fmaxf(fmaxf(k4, k5), fmaxf(k6, k7)));
-      if (vm > best.key) { best.key = vm; best.vec = (int)e; }
-    }
-  }
-  template <int N>
-  __device__ __forceinline__ void update(float, const NoiseRow& nz, const uint4 (&v)[N], int base, int stride) {
-#pragma unroll
-    for (int j = 0; j < N; ++j) {
-      const uint32_t e = (uint32_t)(base + j * stride);
-      float k0 = noise_key(nz, __uint_as_float(v[j].x), e), k1 = noise_key(nz, __uint_as_float(v[j].y), e + 1);
-      float k2 = noise_key(nz, __uint_as_float(v[j].z), e + 2), k3 = noise_key(nz, __uint_as_float(v[j].w), e + 3);
-      const float vm = fmaxf(fmaxf(k0, k1), fmaxf(k2, k3));
-      if (vm > best.key) { best.key = vm; best.vec = (int)e; }
-    }
-  }
-  /* one element at its exact index */
-  __device__ __forceinline__ void one(const NoiseRow& nz, float x, int idx) {
-    const float k = noise_key(nz, x, (uint32_t)idx);
-    if (k > best.key || (k == best.key && idx < best.vec)) { best.key = k; best.vec = idx; }
-  }
-};
-
-/* The element that holds the row's largest perturbed key: the first of the (up to) one vector's
-   worth of elements from `vec` on whose recomputed key equals `key`; also returns its logit. */
-template <typename T>
-__device__ __forceinline__ int resolve_sample(const T* row, const NoiseRow& nz, int vec, int V, float key, float& x_out) {
-  constexpr int VEC = 16 / (int)sizeof(T);
-  int best = -1;
-  x_out = 0.f;
-  if (vec < 0 || vec >= V) return 0;
-#pragma unroll
-  for (int j = VEC - 1; j >= 0; --j) {
-    if (vec + j < V) {
-      const float x = to_f32(row[vec + j]);
-      if (noise_key(nz, x, (uint32_t)(vec + j)) == key) { best = vec + j; x_out = x; }
-    }
-  }
-  if (best < 0) { best = vec; x_out = to_f32(row[vec]); }
-  return best;
-}
+/* what a thread hands on about its share of a row segment besides the Part: the tempered weights of
+   its vectors and of the trailing elements, against its own maximum (the Part's m) */
+struct TauPart { float vec, tail; };
 
 /* The exact position of the row maximum M, given the start `idx` of the vector that holds its
    first occurrence (or the exact position): look at one vector's worth of elements.  All loads are
@@ -521,13 +464,14 @@ __device__ __forceinline__ int resolve_index(const T* row, int idx, int V, float
 /* One thread's share of elements [e0,e1) of a row, read with 128-bit loads straight from global
    memory: vectors tid, tid+NT, tid+2NT, ... (ascending indices), in groups of UNROLL; the thread
    with `tail` also takes the fewer-than-a-vector trailing elements.  e0 is a multiple of the vector
-   width and the row base is 16-byte aligned.  With SAMPLE the perturbed keys of the same elements
-   go through `kt`. */
+   width and the row base is 16-byte aligned.  With SAMPLE the tempered weights of the same elements
+   come back in `tp` (against the returned Part's maximum). */
 template <typename T, bool WITH_T, bool CLAMP, int NT, int UNROLL, bool SAMPLE>
-__device__ __forceinline__ Part stream_thread_once(const T* row, int e0, int e1, int tid, bool tail, KeyTrack* kt,
-                                                   const NoiseRow* nz) {
-  Acc<T, WITH_T, CLAMP> a;
+__device__ __forceinline__ Part stream_thread_once(const T* row, int e0, int e1, int tid, bool tail, float inv_tau, float raise_nats,
+                                                   TauPart* tp) {
+  Acc<T, WITH_T, CLAMP, SAMPLE> a;
   a.init();
+  if (SAMPLE) a.set_temperature(inv_tau, raise_nats);
   constexpr int VEC = 16 / (int)sizeof(T);
   const uint4* p = reinterpret_cast<const uint4*>(row + e0);
   const int nvec = (e1 - e0) / VEC;
@@ -536,60 +480,39 @@ __device__ __forceinline__ Part stream_thread_once(const T* row, int e0, int e1,
     uint4 v[UNROLL];
 #pragma unroll
     for (int j = 0; j < UNROLL; ++j) v[j] = ld_stream(p + i + j * NT);
-    if (SAMPLE) kt->template update<UNROLL>(T{}, *nz, v, e0 + i * VEC, NT * VEC);
     a.template group<UNROLL>(v, e0 + i * VEC, NT * VEC);
   }
   for (; i < nvec; i += NT) {
     uint4 v[1];
     v[0] = ld_stream(p + i);
-    if (SAMPLE) kt->template update<1>(T{}, *nz, v, e0 + i * VEC, NT * VEC);
     a.template group<1>(v, e0 + i * VEC, NT * VEC);
   }
   if (tail) {
-    for (int e = e0 + nvec * VEC; e < e1; ++e) {
-      const float x = to_f32(row[e]);
-      if (SAMPLE) kt->one(*nz, x, e);
-      a.one(x, e);
-    }
+    for (int e = e0 + nvec * VEC; e < e1; ++e) a.one(to_f32(row[e]), e);
   }
-  return a.part();
+  const Part pt = a.part();
+  if (SAMPLE) a.tempered(pt.m, tp->vec, tp->tail);
+  return pt;
 }
 
 /* The same share again with -inf clamped, for a thread whose unclamped pass came out non-finite
    (it met a -inf logit, or the row really holds NaN / +inf and will be flagged by the finaliser). */
-template <typename T, bool WITH_T, int NT>
-__device__ __noinline__ Part stream_thread_clamped(const T* row, int e0, int e1, int tid, bool tail) {
-  return stream_thread_once<T, WITH_T, true, NT, 1, false>(row, e0, e1, tid, tail, nullptr, nullptr);
-}
-
-/* The perturbed keys of one thread's share, on their own (for a thread that starts clamped). */
-template <typename T, int NT>
-__device__ __noinline__ void stream_thread_keys(const T* row, int e0, int e1, int tid, bool tail, KeyTrack* kt,
-                                                const NoiseRow* nz) {
-  constexpr int VEC = 16 / (int)sizeof(T);
-  const uint4* p = reinterpret_cast<const uint4*>(row + e0);
-  const int nvec = (e1 - e0) / VEC;
-  for (int i = tid; i < nvec; i += NT) {
-    uint4 v[1];
-    v[0] = ld_stream(p + i);
-    kt->template update<1>(T{}, *nz, v, e0 + i * VEC, NT * VEC);
-  }
-  if (tail)
-    for (int e = e0 + nvec * VEC; e < e1; ++e) kt->one(*nz, to_f32(row[e]), e);
+template <typename T, bool WITH_T, int NT, bool SAMPLE>
+__device__ __noinline__ Part stream_thread_clamped(const T* row, int e0, int e1, int tid, bool tail, float inv_tau, float raise_nats,
+                                                   TauPart* tp) {
+  return stream_thread_once<T, WITH_T, true, NT, 1, SAMPLE>(row, e0, e1, tid, tail, inv_tau, raise_nats, tp);
 }
 
 /* `sticky` remembers that this thread has met a -inf before and starts clamped from then on. */
 template <typename T, bool WITH_T, int NT, int UNROLL, bool SAMPLE>
-__device__ __forceinline__ Part stream_thread(const T* row, int e0, int e1, int tid, bool tail, bool& sticky,
-                                              KeyTrack* kt, const NoiseRow* nz) {
+__device__ __forceinline__ Part stream_thread(const T* row, int e0, int e1, int tid, bool tail, bool& sticky, float inv_tau,
+                                              float raise_nats, TauPart* tp) {
   if (!sticky) {
-    const Part pt = stream_thread_once<T, WITH_T, false, NT, UNROLL, SAMPLE>(row, e0, e1, tid, tail, kt, nz);
+    const Part pt = stream_thread_once<T, WITH_T, false, NT, UNROLL, SAMPLE>(row, e0, e1, tid, tail, inv_tau, raise_nats, tp);
     if (part_is_finite(pt)) return pt;
     sticky = true;
-  } else if (SAMPLE) {
-    stream_thread_keys<T, NT>(row, e0, e1, tid, tail, kt, nz);
   }
-  return stream_thread_clamped<T, WITH_T, NT>(row, e0, e1, tid, tail);
+  return stream_thread_clamped<T, WITH_T, NT, SAMPLE>(row, e0, e1, tid, tail, inv_tau, raise_nats, tp);
 }
 
 /* ------------------------------------------------------------------------------------------ */
@@ -613,19 +536,6 @@ __device__ __forceinline__ float block_sum_f32(float v, float* sh /*[NT/32]*/) {
   __syncthreads();
   r = sh[0];
   return r;                                                /* same value in every thread */
-}
-
-/* Largest key over the CTA; valid in thread 0.  `sh` holds NT/32 entries. */
-template <int NT>
-__device__ __forceinline__ KeyPart key_block_reduce(KeyPart k, KeyPart* sh) {
-  constexpr int NW = NT / 32;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  k = key_warp_reduce(k);
-  __syncthreads();
-  if (lane == 0) sh[warp] = k;
-  __syncthreads();
-  if (warp == 0) k = key_warp_reduce((lane < NW) ? sh[lane] : key_empty());
-  return k;
 }
 
 /* Guarded scalar reduction of elements [e0,e1) of one row by the whole CTA: two passes, every

@@ -10,16 +10,38 @@ namespace forkd {
 /* ---- kernel 2a: direct 128-bit loads (also the path for buffers that are not 16-byte aligned) -- */
 struct Smem {
   Part parts[kNT / 32];
-  KeyPart keys[kNT / 32];
   float fl[kNT / 32];
+  float bmax;
   int flag;
 };
+
+/* Candidates drawn at a temperature, guarded scalar path (buffers that are not 16-byte aligned, rows
+   re-read after a non-finite result are flagged anyway): the tempered weights of segment [e0,e1) of
+   `row` against M, thread t taking the vectors that belong to lane t of the draw's order. */
+template <typename T>
+__device__ __forceinline__ TauPart tempered_scalar(const T* row, int e0, int e1, int V, float M, float ct, int tid) {
+  constexpr int VEC = 16 / (int)sizeof(T);
+  const int Vf = (V / VEC) * VEC, end = min(e1, Vf);
+  TauPart tp{0.f, 0.f};
+  for (int vec = e0 / VEC + tid; (vec + 1) * VEC <= end; vec += kLanes)
+    for (int j = 0; j < VEC; ++j) {
+      const float x = to_f32(row[vec * VEC + j]);
+      if (x > -INFINITY) tp.vec += exp2f((x - M) * ct);
+    }
+  if (tid == 0)
+    for (int e = max(e0, Vf); e < e1; ++e) {
+      const float x = to_f32(row[e]);
+      if (x > -INFINITY) tp.tail += exp2f((x - M) * ct);
+    }
+  return tp;
+}
 
 template <typename T, int MODE>
 __global__ void __launch_bounds__(kNT, 4) reduce_select_kernel(const __grid_constant__ ReduceParams p) {
   constexpr bool WITH_T = mode_is_step(MODE);
   constexpr bool SAMPLE = mode_is_sample(MODE);
   constexpr bool VP = mode_is_vp(MODE);
+  static_assert(kNT == kLanes, "the lanes of the draw's order are the streaming threads of a CTA");
   __shared__ Smem sm;
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;");
@@ -36,25 +58,43 @@ __global__ void __launch_bounds__(kNT, 4) reduce_select_kernel(const __grid_cons
   while (it.next(sg)) {
     const int2 bk = rm.bk(sg.r);
     const T* row = row_ptr<T>(p.src, bk.x, bk.y);
-    Part part;
-    KeyTrack kt;
-    kt.init();
-    NoiseRow nz = NoiseRow{0u, 0u, 0.f, 0u};
-    if (SAMPLE) nz = noise_row(p.sample_seed, p.step, bk.x, bk.y, p.noise_c, (uint32_t)p.vocab_offset);
+    Part part, mine = part_empty();
+    TauPart tp{0.f, 0.f};
+    bool bad = false;
     if (p.fast) {
-      part = part_block_reduce<kNT>(
-          stream_thread<T, WITH_T, kNT, kUnroll, SAMPLE>(row, sg.e0, sg.e1, threadIdx.x, threadIdx.x == 0, sticky, &kt, &nz),
-          sm.parts);
+      mine = stream_thread<T, WITH_T, kNT, kUnroll, SAMPLE>(row, sg.e0, sg.e1, threadIdx.x, threadIdx.x == 0, sticky, p.inv_tau,
+                                                            p.raise_nats, &tp);
+      part = part_block_reduce<kNT>(mine, sm.parts);
     } else {
-      bool bad;
       part = careful_segment<T, kNT>(row, sg.e0, sg.e1, sm.parts, sm.fl, bad);
-      if (SAMPLE)
-        for (int i = sg.e0 + (int)threadIdx.x; i < sg.e1; i += kNT) kt.one(nz, to_f32(row[i]), i);
     }
-    KeyPart kp = key_empty();
-    if (SAMPLE) kp = key_block_reduce<kNT>(kt.best, sm.keys);
+    if (SAMPLE) {
+      /* every thread's tempered weights against the CTA's maximum: the part's lane sums, its trailing
+         elements and its total, for whoever draws the row's candidate */
+      if (threadIdx.x == 0) sm.bmax = part.m;
+      __syncthreads();
+      const float M = sm.bmax;
+      float vec = 0.f, tl = 0.f;
+      if (p.fast) {
+        if (mine.m > kClamp && mine.m < INFINITY && M < INFINITY) {
+          const float w = ex2_approx((mine.m - M) * p.noise_c);
+          vec = tp.vec * w; tl = tp.tail * w;
+        }
+      } else if (!bad && M > kClamp && M < INFINITY) {
+        const TauPart q = tempered_scalar<T>(row, sg.e0, sg.e1, p.src.V, M, p.noise_c, (int)threadIdx.x);
+        vec = q.vec; tl = q.tail;
+      }
+      float* slot = p.sslots + (size_t)(sg.r + g) * kSlotStride;
+      slot[threadIdx.x] = vec;
+      const float total = block_sum_f32<kNT>(vec + tl, sm.fl);
+      if (threadIdx.x == 0) { slot[kSlotTail] = tl; slot[kSlotTotal] = total; }
+      if (threadIdx.x < 32) store_part(p, part, sg.r, g);      /* the row's maximum is taken from the parts' records */
+      __threadfence();
+      __syncthreads();
+      if (threadIdx.x < 32) row_part_arrived<T>(p, c, sg.r, bk.x, bk.y);
+    }
     if (threadIdx.x < 32) {
-      const bool last = publish_part(p, part, sg.r, g, bk.x, p.expected[bk.x], SAMPLE ? &kp : nullptr);
+      const bool last = publish_part(p, part, sg.r, g, bk.x, p.expected[bk.x]);
       if (last) {                                           /* every part of sequence b has been delivered */
         const SeqHint h = load_seq_hint(p, rm, bk.x);
         if (MODE == kModeLogprob) finalize_logprob_sequence<T>(p, rm, c, bk.x, h);
@@ -94,7 +134,8 @@ constexpr int kSegRing = 16;                               /* > stages: the prod
 struct RingSmem {
   unsigned long long full[kMaxStages], empty[kMaxStages], mfull[kMail], mempty[kMail];
   Part mail[kMail][kMaxCW];
-  KeyPart kmail[kMail][kMaxCW];
+  float slot[kMail][kLanes];                               /* candidates at a temperature: every consumer thread's tempered weights ... */
+  float tailw[kMail];                                      /* ... and those of the trailing elements, against the thread's warp's maximum */
   int2 seg_bk[kSegRing];                                   /* (sequence, position) of the producer's recent segments, for the consumers */
 };
 static_assert(kSegRing > kMaxStages, "segment ring shorter than the stage ring");
@@ -379,20 +420,13 @@ __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_
     uint32_t s = 0, ph = 0, nseg = 0;                       /* ring slot, its phase, segments done */
     bool sticky = false;                                    /* this thread has met a -inf logit before */
     for (; have; have = it.next(sg)) {
-      Acc<T, WITH_T, false> a;
+      Acc<T, WITH_T, false, SAMPLE> a;
       a.init();
-      KeyTrack kt;                                            /* stochastic candidates: largest perturbed key */
-      kt.init();
-      NoiseRow nz = NoiseRow{0u, 0u, 0.f, 0u};
+      if (SAMPLE) a.set_temperature(p.inv_tau, p.raise_nats);
       const int nvec = (sg.e1 - sg.e0) / VEC;
       /* (sequence, position) of this segment: posted by the producer before the segment's first
          copy, so readable once a stage of the segment has landed; a segment shorter than one vector
          has no stage and looks its row up itself */
-      if (SAMPLE) {                                           /* the noise stream of the row is needed from the first element on */
-        if (nvec > 0 && !mbar_wait<kLimit>(&rs.full[s], ph, p)) return;   /* (the stage loop waits on the same phase again: it stays complete) */
-        const int2 bk = nvec > 0 ? rs.seg_bk[nseg % kSegRing] : rm.bk(sg.r);
-        nz = noise_row(p.sample_seed, p.step, bk.x, bk.y, p.noise_c, (uint32_t)p.vocab_offset);
-      }
       for (int voff = 0; voff < nvec; voff += kStageVecs) {
         if (!mbar_wait<kLimit>(&rs.full[s], ph, p)) return;
         const uint4* sp = reinterpret_cast<const uint4*>(ring + (size_t)s * kStageBytes);
@@ -407,11 +441,10 @@ __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_
           __syncwarp();
           if (lane == 0) mbar_arrive(&rs.empty[s]);
           if (!sticky) a.template accumulate<kUnroll>(v);
-          if (SAMPLE) kt.template update<kUnroll>(T{}, nz, v, sg.e0 + (voff + ctid) * VEC, kCT * VEC);
         } else {
           /* the last, partly filled stage of a segment: same unrolled code, vectors past the end
-             replaced by the clamp value (contributes 2^-huge = 0 and never wins the maximum
-             against a finite logit; an all -inf row is re-read by the finaliser anyway) */
+             replaced by the clamp value (contributes 2^-huge = 0 to every sum and never wins the
+             maximum against a finite logit; an all -inf row is re-read by the finaliser anyway) */
           uint4 v[kUnroll];
 #pragma unroll
           for (int j = 0; j < kUnroll; ++j)
@@ -420,46 +453,49 @@ __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_
           __syncwarp();
           if (lane == 0) mbar_arrive(&rs.empty[s]);
           if (!sticky) a.template accumulate<kUnroll>(v);
-          if (SAMPLE) {                                       /* only the vectors that exist draw noise */
-#pragma unroll
-            for (int j = 0; j < kUnroll; ++j)
-              if (ctid + j * kCT < nv) {
-                const uint4 one[1] = {v[j]};
-                kt.template update<1>(T{}, nz, one, sg.e0 + (voff + ctid + j * kCT) * VEC, kCT * VEC);
-              }
-          }
         }
         if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1u; }
       }
       const bool tail = (ctid == 0) && (sg.e0 + nvec * VEC < sg.e1);   /* fewer than VEC trailing elements */
       Part pt;
-      if (tail && (SAMPLE || !sticky)) {
+      TauPart tp{0.f, 0.f};
+      if (tail && !sticky) {
         const int2 bk = nvec > 0 ? rs.seg_bk[nseg % kSegRing] : rm.bk(sg.r);
         const T* row = row_ptr<T>(p.src, bk.x, bk.y);
-        for (int e = sg.e0 + nvec * VEC; e < sg.e1; ++e) {
-          const float x = to_f32(row[e]);
-          if (!sticky) a.one(x, e);
-          if (SAMPLE) kt.one(nz, x, e);
-        }
+        for (int e = sg.e0 + nvec * VEC; e < sg.e1; ++e) a.one(to_f32(row[e]), e);
       }
       if (!sticky) {
         pt = a.part();
+        if (SAMPLE) a.tempered(pt.m, tp.vec, tp.tail);
         if (!part_is_finite(pt)) sticky = true;
       }
       /* a thread that met -inf (now or earlier) takes its own vectors again from global memory, clamped */
       if (sticky) {
         const int2 bk = nvec > 0 ? rs.seg_bk[nseg % kSegRing] : rm.bk(sg.r);
-        pt = stream_thread_clamped<T, WITH_T, kCT>(row_ptr<T>(p.src, bk.x, bk.y), sg.e0, sg.e1, ctid, ctid == 0);
+        pt = stream_thread_clamped<T, WITH_T, kCT, SAMPLE>(row_ptr<T>(p.src, bk.x, bk.y), sg.e0, sg.e1, ctid, ctid == 0, p.inv_tau,
+                                                           p.raise_nats, &tp);
       }
       __syncwarp();
+      const float m_own = pt.m;
       pt = part_warp_reduce(pt);
-      KeyPart kp = key_empty();
-      if (SAMPLE) kp = key_warp_reduce(kt.best);
-      if (lane == 0) {
-        const uint32_t d = nseg % kMail, mph = (nseg / kMail) & 1u;
+      const uint32_t d = nseg % kMail, mph = (nseg / kMail) & 1u;
+      if (SAMPLE) {
+        /* this thread's tempered weights against its warp's maximum: the finaliser turns the 256 of
+           them into the part's lane sums */
+        float w = 0.f;
+        if (m_own > kClamp && m_own < INFINITY && pt.m < INFINITY) w = ex2_approx((m_own - pt.m) * p.noise_c);
+        int ok = 1;
+        if (lane == 0) ok = mbar_wait<kLimit>(&rs.mempty[d], mph ^ 1u, p) ? 1 : 0;
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (ok) {
+          rs.slot[d][ctid] = tp.vec * w;
+          if (ctid == 0) rs.tailw[d] = tp.tail * w;
+          __syncwarp();
+          if (lane == 0) { rs.mail[d][warp] = pt; mbar_arrive(&rs.mfull[d]); }
+        }
+      } else if (lane == 0) {
         if (mbar_wait<kLimit>(&rs.mempty[d], mph ^ 1u, p)) {
           rs.mail[d][warp] = pt;
-          if (SAMPLE) rs.kmail[d][warp] = kp;
           mbar_arrive(&rs.mfull[d]);
         }
       }
@@ -484,13 +520,36 @@ __global__ void __launch_bounds__(kHalfThreads * kHalves, 1) reduce_select_ring_
     const uint32_t d = nseg % kMail, ph = (nseg / kMail) & 1u;
     if (!mbar_wait<kLimit>(&rs.mfull[d], ph, p)) return;
     Part pt = (lane < kCW) ? rs.mail[d][lane] : part_empty();
-    KeyPart kp = key_empty();
-    if (SAMPLE && lane < kCW) kp = rs.kmail[d][lane];
+    const float m_warp = pt.m;                                /* lane i: the maximum of consumer warp i */
+    float sv[kCW], tl = 0.f;
+    if (SAMPLE) {
+#pragma unroll
+      for (int i = 0; i < kCW; ++i) sv[i] = rs.slot[d][i * 32 + lane];
+      tl = rs.tailw[d];
+    }
     __syncwarp();
     if (lane == 0) mbar_arrive(&rs.mempty[d]);
     pt = part_warp_reduce(pt);
-    if (SAMPLE) kp = key_warp_reduce(kp);
-    if (publish_part(p, pt, sg.r, g, b, want, SAMPLE ? &kp : nullptr)) {
+    if (SAMPLE) {
+      /* the part's lane sums of the tempered weights, against the part's maximum */
+      float wq = 0.f;
+      if (lane < kCW && m_warp > kClamp && m_warp < INFINITY && pt.m < INFINITY) wq = ex2_approx((m_warp - pt.m) * p.noise_c);
+      float* slot = p.sslots + (size_t)(sg.r + g) * kSlotStride;
+      float tot = 0.f;
+#pragma unroll
+      for (int i = 0; i < kCW; ++i) {
+        const float v = sv[i] * __shfl_sync(0xffffffffu, wq, i);
+        slot[i * 32 + lane] = v;
+        tot += v;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+      const float tlv = tl * __shfl_sync(0xffffffffu, wq, 0);
+      if (lane == 0) { slot[kSlotTail] = tlv; slot[kSlotTotal] = tot + tlv; }
+      store_part(p, pt, sg.r, g);                             /* the row's maximum is taken from the parts' records */
+      row_part_arrived<T>(p, c, sg.r, b, rm.k_of(b, sg.r));
+    }
+    if (publish_part(p, pt, sg.r, g, b, want)) {
       if (MODE == kModeLogprob) finalize_logprob_sequence<T>(p, rm, c, b, h);
       else if (VP) finalize_vp_local<T, SAMPLE>(p, rm, c, b, h);
       else finalize_step_sequence<T, SAMPLE>(p, rm, c, b, h, snap_done);

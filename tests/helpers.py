@@ -58,13 +58,14 @@ def live_mask(mask, lo, hi):
 
 
 FALLBACK_MARGIN = {0: 0.0, 1: 5e-4, 2: 5e-4, 3: 5e-3, 4: 0.0}   # per fallback order: keys are confidences (<=1) or entropies (<=12 nats)
-SAMPLE_MARGIN = 1e-3                                             # gap between the two largest perturbed keys (nats)
+SAMPLE_MARGIN = 2e-6                                             # drawn candidates: distance of U * total from the nearest boundary of the running sum, over the total
 
 
 def decisions_are_clear(st, live, threshold, margin, fallback_mode=0, temperature=0.0):
     """True when no decision of the step just taken sits within rounding distance of flipping:
     confidences against the threshold, the fallback order's best against its runner-up, and (with
-    stochastic candidates) the winning perturbed key against the second."""
+    stochastic candidates) the point of the running sum that the draw hits against the boundaries of the
+    drawn token's stretch (fp32 sums in another order could otherwise land on a neighbour)."""
     if not (np.abs(st.conf[live] - np.float64(np.float32(threshold))) >= margin).all():
         return False
     if not (st.fallback_margin >= FALLBACK_MARGIN[fallback_mode]).all():

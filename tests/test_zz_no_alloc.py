@@ -8,6 +8,7 @@ amount of free device memory exactly where it was; and the device status word of
 be read although the caller has no workspace pointer to ask with.  Kept in a file that pytest
 collects last."""
 import ctypes as C
+import gc
 
 import numpy as np
 import pytest
