@@ -1130,7 +1130,7 @@ extern "C" fork_status fork_step_fused_head(const fork_step_args* a, const fork_
     int di = 0;
     if (cudaGetDevice(&di) != cudaSuccess || di < 0 || di >= 64) return FORK_ERR_CUDA;
     std::call_once(smem_once[di], [] {
-      cudaFuncSetAttribute(head_gemm_reduce_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHeadSmemBytes);
+      cudaFuncSetAttribute(head_gemm_reduce_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHeadSmemLimit);
     });
   }
   cudaStream_t st = (cudaStream_t)stream;
@@ -1140,19 +1140,34 @@ extern "C" fork_status fork_step_fused_head(const fork_step_args* a, const fork_
   HeadParams hp;
   memset(&hp, 0, sizeof(hp));
   hp.rows = a->B * a->Ll; hp.V = a->V; hp.d = h->d;
-  hp.n_tiles = (a->V + kHeadN - 1) / kHeadN;
+  hp.n_groups = (a->V + kHeadGroup - 1) / kHeadGroup;
   hp.m_blocks = (hp.rows + kHeadM - 1) / kHeadM;
+  hp.unit = hp.m_blocks == 1 ? 1 : kHeadN / kHeadGroup;
+  const int n_units = (hp.n_groups + hp.unit - 1) / hp.unit;
   int splits = dev->sms / hp.m_blocks;
   if (splits < 1) splits = 1;
-  if (splits > hp.n_tiles) splits = hp.n_tiles;
-  hp.tiles_per_split = (hp.n_tiles + splits - 1) / splits;
-  hp.n_splits = (hp.n_tiles + hp.tiles_per_split - 1) / hp.tiles_per_split;
+  if (splits > n_units) splits = n_units;
+  hp.n_splits = splits;
+  hp.u_base = n_units / splits; hp.u_rem = n_units % splits;
+  hp.a_box_rows = head_a_box_rows(hp.rows);
+  hp.stages = head_stages(hp.a_box_rows);
+  const size_t head_smem = (size_t)hp.stages * head_stage_bytes(hp.a_box_rows) + kHeadSmemExtra;
   if ((size_t)hp.n_splits * hp.m_blocks * kHeadM > (size_t)a->B * a->Lt + kHeadPartsExtra) return FORK_ERR_WORKSPACE;
   hp.parts = w.head_parts; hp.hdr = w.hdr;
-  CUtensorMap map_h, map_w;
-  if (!head_tensor_map(&map_h, h->hidden, (uint64_t)hp.rows, (uint64_t)h->d, (uint64_t)h->hidden_stride, kHeadM) ||
-      !head_tensor_map(&map_w, h->weight, (uint64_t)a->V, (uint64_t)h->d, (uint64_t)h->weight_stride, kHeadN))
+  HeadMaps maps;
+  memset(&maps, 0, sizeof(maps));
+  if (!head_tensor_map(&maps.h, h->hidden, (uint64_t)hp.rows, (uint64_t)h->d, (uint64_t)h->hidden_stride, (uint32_t)hp.a_box_rows))
     return FORK_ERR_INVALID_ARG;
+  bool have[kHeadN / kHeadGroup] = {};
+  for (int ns = 0; ns < splits; ++ns) {                                    /* the tile widths this launch uses (see the kernel) */
+    const int g = head_split_groups(hp, ns), per = kHeadN / kHeadGroup, tiles = (g + per - 1) / per;
+    for (int wg = g / tiles; wg <= g / tiles + (g % tiles ? 1 : 0); ++wg) {
+      if (have[wg - 1]) continue;
+      if (!head_tensor_map(&maps.w[wg - 1], h->weight, (uint64_t)a->V, (uint64_t)h->d, (uint64_t)h->weight_stride, (uint32_t)(wg * kHeadGroup)))
+        return FORK_ERR_INVALID_ARG;
+      have[wg - 1] = true;
+    }
+  }
 
   /* the active set (Algorithm 2, line 3): row list and per-sequence ranges for the select phase */
   SetupParams sp;
@@ -1164,11 +1179,27 @@ extern "C" fork_status fork_step_fused_head(const fork_step_args* a, const fork_
   if (launch(active_set_kernel, dim3(1), dim3(kSetupNT), st, pdl, sp) != cudaSuccess) return FORK_ERR_CUDA;
 
   /* logits tile by tile in tensor memory, reduced to one part per row and vocabulary split */
-  head_gemm_reduce_kernel<<<dim3((unsigned)(hp.m_blocks * hp.n_splits)), dim3(kHeadThreads), kHeadSmemBytes, st>>>(map_h, map_w, hp);
+  head_gemm_reduce_kernel<<<dim3((unsigned)(hp.m_blocks * hp.n_splits)), dim3(kHeadThreads), head_smem, st>>>(maps, hp);
   if (cudaGetLastError() != cudaSuccess) return FORK_ERR_CUDA;
   g_launches.fetch_add(1);
 
-  /* the splits of a row merged like the slices of a vocabulary-parallel step, then the unmask rule */
+  /* the splits of a row merged (ties to the lowest column, like the slices of a vocabulary-parallel step) ... */
+  if ((size_t)hp.m_blocks * kHeadM > (size_t)a->B * a->Lt + 2048) return FORK_ERR_WORKSPACE;
+  {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)((hp.rows + kHeadMergeNT / 32 - 1) / (kHeadMergeNT / 32))); cfg.blockDim = dim3(kHeadMergeNT);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    if (pdl) {
+      attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[0].val.programmaticStreamSerializationAllowed = 1;
+      cfg.attrs = attr; cfg.numAttrs = 1;
+    }
+    if (cudaLaunchKernelEx(&cfg, head_merge_kernel, hp, w.parts) != cudaSuccess) return FORK_ERR_CUDA;
+    g_launches.fetch_add(1);
+  }
+  /* ... then the unmask rule on one record per row */
   ReduceParams rp;
   memset(&rp, 0, sizeof(rp));
   rp.src.pos0 = a->pos0; rp.src.Ll = a->Ll; rp.src.V = a->V;
@@ -1181,9 +1212,9 @@ extern "C" fork_status fork_step_fused_head(const fork_step_args* a, const fork_
   rp.n_unmasked = a->n_unmasked; rp.is_fallback = a->is_fallback; rp.fallback_pos = a->fallback_pos;
   rp.nfe = a->nfe; rp.n_fallback = a->n_fallback;
   rp.fallback_mode = a->fallback_mode; rp.fallback_rand = a->fallback_rand;
-  rp.vp_parts_in = w.head_parts; rp.vp_ranks = hp.n_splits; rp.vp_row_stride = hp.m_blocks * kHeadM;
+  rp.vp_parts_in = w.parts; rp.vp_ranks = 1; rp.vp_row_stride = hp.m_blocks * kHeadM;
   const dim3 grid((unsigned)((a->B + kVpNT / 32 - 1) / (kVpNT / 32)));
-  if (launch(vp_select_kernel<false>, grid, dim3(kVpNT), st, false, rp) != cudaSuccess) return FORK_ERR_CUDA;
+  if (launch(vp_select_kernel<false>, grid, dim3(kVpNT), st, pdl, rp) != cudaSuccess) return FORK_ERR_CUDA;
   return FORK_OK;
 }
 

@@ -4,13 +4,17 @@
  * reach HBM.  (The paper's model "predicts a distribution q_theta^k(.|x_t) for every k in M_t",
  * Section 2; the logits the other kernels read from memory come straight out of this product.)
  *
- * One CTA = one 128-row block of the hidden-state window x one contiguous range of 256-column
- * vocabulary tiles.  Warp roles (192 threads):
- *   warp 0  producer : TMA tensor copies (cp.async.bulk.tensor.2d, no multicast) of a 128 x 64 tile of
- *                      hidden states and a 256 x 64 tile of the weight per k-block into a ring of
- *                      shared-memory stages (128-byte swizzle), full/empty mbarriers;
+ * One CTA = one 128-row block of the hidden-state window x one contiguous range of vocabulary
+ * columns, a whole number of 32-column groups dealt out evenly over the CTAs (so that every SM gets
+ * the same share of the weight whatever V is), walked in tiles of 256 columns with a narrower last
+ * tile.  Warp roles (192 threads):
+ *   warp 0  producer : TMA tensor copies (cp.async.bulk.tensor.2d, no multicast) of a tile of hidden
+ *                      states (64 columns x 128 rows; 32 or 64 rows when the window has no more, which
+ *                      leaves room for more stages) and a 256 x 64 tile of the weight (the narrow last
+ *                      tile in 32-row boxes) per k-block into a ring of shared-memory stages
+ *                      (128-byte swizzle), full/empty mbarriers;
  *   warp 1  MMA      : one elected thread issues tcgen05.mma (kind::f16, bf16 x bf16 -> fp32,
- *                      M = 128, N = 256, K = 16 per instruction) from shared-memory descriptors into
+ *                      M = 128, N = the tile's width, K = 16 per instruction) from shared-memory descriptors into
  *                      one of two 256-column accumulators in tensor memory, frees a stage with
  *                      tcgen05.commit, and hands a finished accumulator to the epilogue the same way;
  *   warps 2-5 epilogue: thread = row (a lane of tensor memory); tcgen05.ld 32 columns at a time,
@@ -33,27 +37,58 @@ namespace forkd {
 constexpr int kHeadM = 128;                 /* rows per CTA (tensor-memory lanes) */
 constexpr int kHeadN = 256;                 /* vocabulary columns per tile (accumulator columns) */
 constexpr int kHeadK = 64;                  /* bf16 elements per k-block: 128 bytes, one swizzle row */
-constexpr int kHeadStages = 4;
+constexpr int kHeadGroup = 32;              /* columns per group: the unit in which the vocabulary is dealt out, and the rows of a small weight box */
+constexpr int kHeadMaxStages = 8;
 constexpr int kHeadThreads = 192;
-constexpr int kHeadABytes = kHeadM * kHeadK * 2;            /* 16 KB */
 constexpr int kHeadBBytes = kHeadN * kHeadK * 2;            /* 32 KB */
-constexpr int kHeadStageBytes = kHeadABytes + kHeadBBytes;
 constexpr uint32_t kHeadSpinLimit = 1u << 24;
-constexpr size_t kHeadSmemBytes = (size_t)kHeadStages * kHeadStageBytes + 1024 /* alignment */ + 256 /* barriers */;
+constexpr size_t kHeadSmemLimit = 227 * 1024;
+constexpr size_t kHeadSmemExtra = 1024 /* alignment */ + 256 /* barriers */;
+
+/* Rows of the hidden-state box: the window's rows rounded up to 32, 64 or 128.  The MMA always reads
+   128 rows (16 KB) from the stage; with a smaller box the rows behind it are whatever the stage holds
+   there (the weight tile), which only reaches accumulator lanes nobody reads. */
+__host__ __device__ constexpr int head_a_box_rows(int rows) { return rows <= 32 ? 32 : rows <= 64 ? 64 : kHeadM; }
+__host__ __device__ constexpr int head_stage_bytes(int a_box_rows) { return a_box_rows * kHeadK * 2 + kHeadBBytes; }
+__host__ __device__ constexpr int head_stages(int a_box_rows) {
+  const int n = (int)((kHeadSmemLimit - kHeadSmemExtra) / (size_t)head_stage_bytes(a_box_rows));
+  return n < kHeadMaxStages ? n : kHeadMaxStages;
+}
 
 struct HeadParams {
   int rows;                  /* B * Ll window rows */
   int V, d;
-  int n_tiles;               /* ceil(V / kHeadN) */
-  int tiles_per_split;       /* vocabulary tiles per CTA */
+  int n_groups;              /* ceil(V / 32) column groups */
+  int unit;                  /* groups per unit of distribution: 1 with a single row block (the CTAs share nothing and the
+                                weight streams from HBM: equal bytes per SM), 8 = whole 256-column tiles otherwise (full-width
+                                MMAs matter more there: measured) */
+  int u_base, u_rem;         /* units per split: u_base, one more for the first u_rem splits */
   int n_splits;
   int m_blocks;
+  int a_box_rows;            /* rows of the hidden-state box: 32, 64 or 128 */
+  int stages;                /* ring depth that fits shared memory with that box */
   float4* parts;             /* [n_splits][m_blocks * kHeadM] */
   WsHeader* hdr;
 };
 
+/* One tensor map of the weight per tile width (box rows = 32, 64, ..., 256): a narrow tile fetched as
+   one box of its own width moves as fast as a full one; fetched as several 32-row boxes it does not
+   (measured: 1.6 x the time when every tile is fetched that way).  Only the widths a launch uses are
+   encoded. */
+struct HeadMaps {
+  CUtensorMap h;
+  CUtensorMap w[kHeadN / kHeadGroup];
+};
+
+/* column groups of split ns: its units, clipped to the end of the vocabulary */
+__host__ __device__ inline int head_split_groups(const HeadParams& p, int ns) {
+  const int g0 = (ns * p.u_base + (ns < p.u_rem ? ns : p.u_rem)) * p.unit;
+  const int g1 = g0 + (p.u_base + (ns < p.u_rem ? 1 : 0)) * p.unit;
+  return (g1 < p.n_groups ? g1 : p.n_groups) - g0;
+}
+
 struct HeadBarriers {
-  unsigned long long full[kHeadStages], empty[kHeadStages], acc_full[2], acc_empty[2];
+  unsigned long long full[kHeadMaxStages], empty[kHeadMaxStages], acc_full[2], acc_empty[2];
   uint32_t tmem_base;
   int abort;
 };
@@ -105,8 +140,8 @@ __device__ __forceinline__ uint64_t head_smem_desc(uint32_t smem_addr) {
 }
 /* Instruction descriptor of tcgen05.mma kind::f16: fp32 accumulator (bits 4-5 = 1), A and B bf16
    (bits 7-9 and 10-12 = 1), both K-major (bits 15, 16 = 0), N / 8 in bits 17-22, M / 16 in bits 24-28. */
-__host__ __device__ constexpr uint32_t head_instr_desc() {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kHeadN >> 3) << 17) | ((uint32_t)(kHeadM >> 4) << 24);
+__host__ __device__ constexpr uint32_t head_instr_desc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kHeadM >> 4) << 24);
 }
 __device__ __forceinline__ void head_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
   asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
@@ -129,19 +164,26 @@ __device__ __forceinline__ void head_tmem_ld32(uint32_t taddr, uint32_t (&v)[32]
 }
 
 __global__ void __launch_bounds__(kHeadThreads, 1)
-head_gemm_reduce_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w, const HeadParams p) {
+head_gemm_reduce_kernel(const __grid_constant__ HeadMaps maps, const HeadParams p) {
   extern __shared__ unsigned char head_smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(head_smem_raw) + 1023) & ~(uintptr_t)1023);
-  HeadBarriers& hb = *reinterpret_cast<HeadBarriers*>(smem + (size_t)kHeadStages * kHeadStageBytes);
+  const int n_stages = p.stages;
+  const int a_bytes = p.a_box_rows * kHeadK * 2, stage_bytes = a_bytes + kHeadBBytes;
+  HeadBarriers& hb = *reinterpret_cast<HeadBarriers*>(smem + (size_t)n_stages * stage_bytes);
   const int warp = (int)threadIdx.x >> 5, lane = (int)threadIdx.x & 31;
   const int mb = (int)blockIdx.x % p.m_blocks, ns = (int)blockIdx.x / p.m_blocks;
-  const int tile0 = ns * p.tiles_per_split;
-  const int tile1 = min(tile0 + p.tiles_per_split, p.n_tiles);
-  const int n_my = tile1 - tile0;                           /* >= 1 by construction of the grid */
+  const int g_cta = head_split_groups(p, ns);                                           /* >= 1 by construction of the grid */
+  const int c_begin = (ns * p.u_base + min(ns, p.u_rem)) * p.unit * kHeadGroup;
+  /* tiles of at most 256 columns, all of (nearly) the same width so that every stage of the ring
+     carries about the same number of bytes: tile t has g_base (+1 for the first g_rem) groups */
+  const int n_my = (g_cta + kHeadN / kHeadGroup - 1) / (kHeadN / kHeadGroup);
+  const int g_base = g_cta / n_my, g_rem = g_cta % n_my;
+  auto tile_col0 = [&](int t) { return c_begin + (t * g_base + min(t, g_rem)) * kHeadGroup; };
+  auto tile_width = [&](int t) { return (g_base + (t < g_rem ? 1 : 0)) * kHeadGroup; };
   const int kblocks = p.d / kHeadK;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kHeadStages; ++s) { head_mbar_init(&hb.full[s], 1); head_mbar_init(&hb.empty[s], 1); }
+    for (int s = 0; s < n_stages; ++s) { head_mbar_init(&hb.full[s], 1); head_mbar_init(&hb.empty[s], 1); }
     for (int a = 0; a < 2; ++a) { head_mbar_init(&hb.acc_full[a], 1); head_mbar_init(&hb.acc_empty[a], 4); }
     hb.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -159,24 +201,24 @@ head_gemm_reduce_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
   if (warp == 0) {
     /* ---------------- producer ---------------- */
     if (lane == 0) {
-      uint32_t n = 0;                                       /* stages issued */
+      uint32_t n = 0, s = 0, ph = 0;                        /* stages issued; ring slot and its phase */
       bool ok = true;
       for (int t = 0; t < n_my && ok; ++t) {
-        const int col0 = (tile0 + t) * kHeadN;
+        const int col0 = tile_col0(t), width = tile_width(t);   /* a multiple of 32 */
         for (int kb = 0; kb < kblocks; ++kb, ++n) {
-          const uint32_t s = n % kHeadStages, ph = (n / kHeadStages) & 1u;
           if (!head_wait(&hb.empty[s], ph ^ 1u, hb, p)) { ok = false; break; }
-          unsigned char* a = smem + (size_t)s * kHeadStageBytes;
-          head_mbar_expect_tx(&hb.full[s], (uint32_t)kHeadStageBytes);
-          head_tma_load_2d(a, &map_h, kb * kHeadK, mb * kHeadM, &hb.full[s]);
-          head_tma_load_2d(a + kHeadABytes, &map_w, kb * kHeadK, col0, &hb.full[s]);
+          unsigned char* a = smem + (size_t)s * stage_bytes;
+          head_mbar_expect_tx(&hb.full[s], (uint32_t)(a_bytes + width * kHeadK * 2));
+          head_tma_load_2d(a, &maps.h, kb * kHeadK, mb * kHeadM, &hb.full[s]);
+          head_tma_load_2d(a + a_bytes, &maps.w[width / kHeadGroup - 1], kb * kHeadK, col0, &hb.full[s]);
+          if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1u; }
         }
       }
       if (!ok) {                                            /* do not leave with copies still landing */
-        const uint32_t first = n > (uint32_t)kHeadStages ? n - (uint32_t)kHeadStages : 0u;
+        const uint32_t first = n > (uint32_t)n_stages ? n - (uint32_t)n_stages : 0u;
         for (uint32_t q = first; q < n; ++q) {
-          unsigned long long* bar = &hb.full[q % kHeadStages];
-          const uint32_t par = (q / kHeadStages) & 1u;
+          unsigned long long* bar = &hb.full[q % (uint32_t)n_stages];
+          const uint32_t par = (q / (uint32_t)n_stages) & 1u;
           for (uint32_t i = 0; i < kHeadSpinLimit && !head_mbar_try(bar, par); ++i) {}
         }
       }
@@ -184,24 +226,24 @@ head_gemm_reduce_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
   } else if (warp == 1) {
     /* ---------------- MMA issuer ---------------- */
     if (lane == 0) {
-      const uint32_t idesc = head_instr_desc();
-      uint32_t n = 0;
+      uint32_t s = 0, ph = 0;
       bool ok = true;
       for (int t = 0; t < n_my && ok; ++t) {
         const uint32_t acc = (uint32_t)t & 1u, use = (uint32_t)t >> 1;
+        const uint32_t idesc = head_instr_desc(tile_width(t));
         if (!head_wait(&hb.acc_empty[acc], (use & 1u) ^ 1u, hb, p)) { ok = false; break; }   /* the epilogue has drained this accumulator */
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t tmem_d = tmem_base + acc * (uint32_t)kHeadN;
-        for (int kb = 0; kb < kblocks; ++kb, ++n) {
-          const uint32_t s = n % kHeadStages, ph = (n / kHeadStages) & 1u;
+        for (int kb = 0; kb < kblocks; ++kb) {
           if (!head_wait(&hb.full[s], ph, hb, p)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t a_addr = head_smem_u32(smem + (size_t)s * kHeadStageBytes);
-          const uint64_t adesc = head_smem_desc(a_addr), bdesc = head_smem_desc(a_addr + kHeadABytes);
+          const uint32_t a_addr = head_smem_u32(smem + (size_t)s * stage_bytes);
+          const uint64_t adesc = head_smem_desc(a_addr), bdesc = head_smem_desc(a_addr + (uint32_t)a_bytes);
 #pragma unroll
           for (int kk = 0; kk < kHeadK / 16; ++kk)          /* 16 bf16 = 32 bytes = 2 descriptor units further along the row */
             head_mma(tmem_d, adesc + (uint64_t)(2 * kk), bdesc + (uint64_t)(2 * kk), idesc, (kb > 0 || kk > 0) ? 1u : 0u);
           head_commit(&hb.empty[s]);                        /* the stage is free once these MMAs have read it */
+          if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1u; }
         }
         if (ok) head_commit(&hb.acc_full[acc]);             /* the accumulator is complete once they have all finished */
       }
@@ -210,6 +252,7 @@ head_gemm_reduce_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
     /* ---------------- epilogue: thread = row ---------------- */
     const int quad = warp & 3;                              /* the 32 tensor-memory lanes this warp may read */
     const int row = mb * kHeadM + quad * 32 + lane;
+    const bool has_rows = mb * kHeadM + quad * 32 < p.rows;  /* a warp whose 32 rows lie beyond the window only hands the accumulator back */
     float m = -INFINITY, s = 0.f, t2 = 0.f;
     int idx = kIdxNone;
     bool ok = true;
@@ -217,10 +260,11 @@ head_gemm_reduce_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
       const uint32_t acc = (uint32_t)t & 1u, use = (uint32_t)t >> 1;
       if (!head_wait(&hb.acc_full[acc], use & 1u, hb, p)) { ok = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const int col0 = (tile0 + t) * kHeadN;
+      const int col0 = tile_col0(t);
+      const int width = has_rows ? tile_width(t) : 0;
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * (uint32_t)kHeadN;
 #pragma unroll 1
-      for (int c = 0; c < kHeadN; c += 32) {
+      for (int c = 0; c < width; c += 32) {
         uint32_t v[32];
         head_tmem_ld32(taddr + (uint32_t)c, v);
         const int cbase = col0 + c;
@@ -263,6 +307,21 @@ head_gemm_reduce_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"(512u) : "memory");
   }
+}
+
+/* The splits of a row merged into one Part: one warp per row, lanes over the splits (independent
+   loads, then one warp reduction), so that the select kernel reads one record per row however many
+   CTAs shared the vocabulary.  Ties keep the lowest column index, as everywhere. */
+constexpr int kHeadMergeNT = 256;
+__global__ void __launch_bounds__(kHeadMergeNT) head_merge_kernel(const HeadParams p, float4* __restrict__ merged) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int row = (int)blockIdx.x * (kHeadMergeNT / 32) + (int)(threadIdx.x >> 5), lane = (int)threadIdx.x & 31;
+  if (row >= p.rows) return;
+  const size_t n = (size_t)p.m_blocks * kHeadM;
+  Part acc = part_empty();
+  for (int j = lane; j < p.n_splits; j += 32) acc = part_merge(acc, part_from(__ldg(p.parts + (size_t)j * n + row)));
+  acc = part_warp_reduce(acc);
+  if (lane == 0) merged[row] = make_float4(acc.m, acc.s, acc.t, __int_as_float(acc.idx));
 }
 
 }  // namespace forkd

@@ -65,7 +65,7 @@ def run_case(B, Ll, Lt, pos0, V, d, lam, n_check, mask_density=1.0, seed=1):
     n0 = pkg.fork_kernel_launches()
     pkg.fork_step_fused_head(st, hid, w_dev, torch.from_numpy(lo).cuda(), torch.from_numpy(hi).cuda(), lam, step=3, pos0=pos0)
     torch.cuda.synchronize()
-    assert pkg.fork_kernel_launches() - n0 == 3
+    assert pkg.fork_kernel_launches() - n0 == 4
     assert pkg.fork_device_status(st) == 0
     g = st.host()
     compare_step_state(g, o, nseq=n_check, rtol=HEAD_RTOL, atol=HEAD_ATOL)
@@ -88,6 +88,8 @@ def test_small_ragged_shapes():
     # V not a multiple of the 256-column tile, rows not a multiple of 128, a window inside a longer buffer
     run_case(B=3, Ll=5, Lt=16, pos0=4, V=1000, d=128, lam=0.9, n_check=3, mask_density=0.8, seed=2)
     run_case(B=5, Ll=40, Lt=40, pos0=0, V=5000, d=256, lam=0.5, n_check=5, mask_density=0.7, seed=3)
+    # 33..64 window rows: the 64-row box of hidden states; a vocabulary that ends inside a 32-column group
+    run_case(B=2, Ll=24, Lt=24, pos0=0, V=3001, d=192, lam=0.7, n_check=2, mask_density=0.9, seed=4)
 
 
 @pytest.mark.parametrize("B,Ll,n_check", [(1, 8, 1), (8, 32, 8), (64, 32, 6)])
