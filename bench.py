@@ -483,18 +483,21 @@ def time_fused_head(device, hbm_peak, shapes=((64, 32), (8, 32), (1, 8))):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
         def timed(fn, reps):
+            """Median over 5 chunks of `reps` back-to-back calls between two events (a call alone between
+            two events would count the host's preparation of its first launch: 30 us of a 190 us call)."""
             for _ in range(3):
                 st.mask.fill_(1)
                 fn()
             torch.cuda.synchronize()
             ts = []
-            for _ in range(reps):
-                st.mask.fill_(1)
+            for _ in range(5):
                 e0.record()
-                fn()
+                for _ in range(reps):
+                    st.mask.fill_(1)
+                    fn()
                 e1.record()
                 torch.cuda.synchronize()
-                ts.append(e0.elapsed_time(e1))
+                ts.append(e0.elapsed_time(e1) / reps)
             return statistics.median(ts)
 
         def fused():

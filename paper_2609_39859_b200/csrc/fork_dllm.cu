@@ -1179,9 +1179,20 @@ extern "C" fork_status fork_step_fused_head(const fork_step_args* a, const fork_
   if (launch(active_set_kernel, dim3(1), dim3(kSetupNT), st, pdl, sp) != cudaSuccess) return FORK_ERR_CUDA;
 
   /* logits tile by tile in tensor memory, reduced to one part per row and vocabulary split */
-  head_gemm_reduce_kernel<<<dim3((unsigned)(hp.m_blocks * hp.n_splits)), dim3(kHeadThreads), head_smem, st>>>(maps, hp);
-  if (cudaGetLastError() != cudaSuccess) return FORK_ERR_CUDA;
-  g_launches.fetch_add(1);
+  {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)(hp.m_blocks * hp.n_splits)); cfg.blockDim = dim3(kHeadThreads);
+    cfg.dynamicSmemBytes = head_smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    if (pdl) {
+      attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[0].val.programmaticStreamSerializationAllowed = 1;
+      cfg.attrs = attr; cfg.numAttrs = 1;
+    }
+    if (cudaLaunchKernelEx(&cfg, head_gemm_reduce_kernel, maps, hp) != cudaSuccess) return FORK_ERR_CUDA;
+    g_launches.fetch_add(1);
+  }
 
   /* the splits of a row merged (ties to the lowest column, like the slices of a vocabulary-parallel step) ... */
   if ((size_t)hp.m_blocks * kHeadM > (size_t)a->B * a->Lt + 2048) return FORK_ERR_WORKSPACE;

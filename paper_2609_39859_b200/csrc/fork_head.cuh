@@ -182,6 +182,12 @@ head_gemm_reduce_kernel(const __grid_constant__ HeadMaps maps, const HeadParams 
   auto tile_width = [&](int t) { return (g_base + (t < g_rem ? 1 : 0)) * kHeadGroup; };
   const int kblocks = p.d / kHeadK;
 
+  /* Nothing here reads what the kernel before it in the stream (the active-set kernel) writes, so
+     under a dependent launch this kernel runs beside it and only waits for it at its very end:
+     whoever comes after this kernel then finds both complete.  Its own dependents may take their
+     places early (they wait at their top). */
+  asm volatile("griddepcontrol.launch_dependents;");
+
   if (threadIdx.x == 0) {
     for (int s = 0; s < n_stages; ++s) { head_mbar_init(&hb.full[s], 1); head_mbar_init(&hb.empty[s], 1); }
     for (int a = 0; a < 2; ++a) { head_mbar_init(&hb.acc_full[a], 1); head_mbar_init(&hb.acc_empty[a], 4); }
@@ -307,6 +313,7 @@ head_gemm_reduce_kernel(const __grid_constant__ HeadMaps maps, const HeadParams 
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"(512u) : "memory");
   }
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 /* The splits of a row merged into one Part: one warp per row, lanes over the splits (independent
@@ -314,6 +321,7 @@ head_gemm_reduce_kernel(const __grid_constant__ HeadMaps maps, const HeadParams 
    CTAs shared the vocabulary.  Ties keep the lowest column index, as everywhere. */
 constexpr int kHeadMergeNT = 256;
 __global__ void __launch_bounds__(kHeadMergeNT) head_merge_kernel(const HeadParams p, float4* __restrict__ merged) {
+  asm volatile("griddepcontrol.launch_dependents;");
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const int row = (int)blockIdx.x * (kHeadMergeNT / 32) + (int)(threadIdx.x >> 5), lane = (int)threadIdx.x & 31;
   if (row >= p.rows) return;
