@@ -396,6 +396,22 @@ def time_logprob(device, peak, B=None):
     out.append({"workload": "grpo: fork_logprob_backward, same %d rows: one read + one write of each row (%.2f GB)" % (rows, 2 * rows * w.V * 4 / 1e9),
                 "positions_per_s": rows / (ms * 1e-3), "ms": ms, "hbm_gbs_read_plus_write": gbs,
                 "frac_of_measured_peak": gbs / peak})
+    ms_three = out[0]["ms"] + out[1]["ms"] + ms
+    # the three calls as one pass: every selected row read from HBM once, its gradient written once
+    for _ in range(2):
+        pkg.fork_grpo_fused(t, tok_d, sel_d, old.contiguous(), reward, 8, 0.2, 0.2, grad, st)
+    torch.cuda.synchronize()
+    old_c = old.contiguous()
+    e0.record()
+    for _ in range(n):
+        pkg.fork_grpo_fused(t, tok_d, sel_d, old_c, reward, 8, 0.2, 0.2, grad, st)
+    e1.record()
+    torch.cuda.synchronize()
+    ms_f = e0.elapsed_time(e1) / n
+    gbs = 2 * rows * w.V * 4 / (ms_f * 1e-3) / 1e9
+    out.append({"workload": "grpo: fork_grpo_fused, same %d rows: scoring, Eq. 2 and backward in one pass (algorithmic: one read + one write, %.2f GB)" % (rows, 2 * rows * w.V * 4 / 1e9),
+                "positions_per_s": rows / (ms_f * 1e-3), "ms": ms_f, "hbm_gbs_read_plus_write": gbs, "frac_of_measured_peak": gbs / peak,
+                "three_calls_ms": ms_three, "speedup_vs_three_calls": ms_three / ms_f})
     del t, grad
     torch.cuda.empty_cache()
     return out
@@ -411,48 +427,67 @@ def time_vocab_parallel(device, peak, n_ranks=8):
     w = fs.workload("passk")
     cfg, bufs, states, lo, hi = full_block_setup(w, w.seed, 2, 1, device)
     st = states[0]
-    off, n = pkg.vocab_shards(w.V, n_ranks, w.es)[1]
-    shard = bufs[0][:, :, off:off + n]
+    shards = pkg.vocab_shards(w.V, n_ranks, w.es)
+    off, n = shards[1]
     parts = []
-    for r, (o, m) in enumerate(pkg.vocab_shards(w.V, n_ranks, w.es)):
+    for r, (o, m) in enumerate(shards):
         parts.append(pkg.fork_vp_reduce(st, bufs[0][:, :, o:o + m], lo, hi, w.threshold, o)[0])
     gathered = torch.stack(parts, 0)
-    e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
-    t_red = t_sel = 0.0
-    reps = 20
-    for i in range(reps + 3):
-        reset_states([st])
-        flush = bufs[1].view(torch.int16)[:, :8].sum()          # touch another buffer: the slice is 65 MB, within L2
-        e0.record()
-        pkg.fork_vp_reduce(st, shard, lo, hi, w.threshold, off)
-        e1.record()
-        pkg.fork_vp_select(st, gathered, None, lo, hi, w.threshold, Ll=w.block_len)
-        e2.record()
-        torch.cuda.synchronize()
-        if i >= 3:
-            t_red += e0.elapsed_time(e1)
-            t_sel += e1.elapsed_time(e2)
-    # the same reduction with the exchange fused in: stores into n_ranks gather buffers (all on this GPU here)
+    # the timed slices rotate over every rank's share of both logits buffers: 16 distinct 65 MB regions,
+    # 1 GB in all (8 x L2), so that no repetition finds its slice in L2
+    views = [(bufs[j][:, :, o:o + m], o) for j in range(len(bufs)) for (o, m) in shards if m == n]
+    e0, e1 = (torch.cuda.Event(enable_timing=True) for _ in range(2))
     Lt = st.Lt
     peers = [torch.zeros((n_ranks, w.B, Lt, 4), dtype=torch.float32, device=device) for _ in range(n_ranks)]
-    t_fused = 0.0
-    for i in range(reps + 3):
-        reset_states([st])
-        flush = bufs[1].view(torch.int16)[:, :8].sum()
-        e0.record()
-        pkg.fork_vp_reduce_peers(st, shard, lo, hi, w.threshold, off, 1, peers)
-        e1.record()
+
+    def chunked(fn, reps=16, chunks=5):
+        """Median over chunks of `reps` back-to-back calls between two events (a call alone between two
+        events would count the host's preparation of its launch, which is longer than these kernels)."""
+        for i in range(3):
+            fn(i)
         torch.cuda.synchronize()
-        if i >= 3:
-            t_fused += e0.elapsed_time(e1)
+        ts = []
+        for c in range(chunks):
+            e0.record()
+            for i in range(reps):
+                fn(c * reps + i)
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) / reps)
+        return statistics.median(ts)
+
+    # arguments marshalled once: the loops below hold nothing but the library calls
+    L = pkg.lib()
+    stream = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    ws = C.c_void_p(st.ws_ptr)
+    calls = [(pkg.make_step_args(st, shard, lo, hi, w.threshold), int(o)) for shard, o in views]
+    out_parts = torch.zeros((w.B, Lt, 4), dtype=torch.float32, device=device)
+    out_ptr = C.c_void_p(out_parts.data_ptr())
+    peer_arr = (C.c_void_p * n_ranks)(*[t.data_ptr() for t in peers])
+    sel_args = pkg.make_step_args(st, None, lo, hi, w.threshold)
+    sel_args.Ll = w.block_len
+    gathered_ptr = C.c_void_p(gathered.data_ptr())
+
+    def reduce_call(i):                                  # the local phase leaves tokens and mask alone: no re-arming needed
+        a, o = calls[i % len(calls)]
+        assert L.fork_vp_reduce(C.byref(a), o, out_ptr, None, ws, st.ws_bytes, stream) == 0
+
+    def fused_call(i):
+        a, o = calls[i % len(calls)]
+        assert L.fork_vp_reduce_peers(C.byref(a), o, 1, n_ranks, peer_arr, None, ws, st.ws_bytes, stream) == 0
+
+    def select_call(i):                                  # (includes the one-byte-per-position fill that re-arms the mask)
+        st.mask.fill_(1)
+        assert L.fork_vp_select(C.byref(sel_args), gathered_ptr, None, n_ranks, ws, st.ws_bytes, stream) == 0
+
+    ms_red, t_fused, ms_sel = chunked(reduce_call), chunked(fused_call), chunked(select_call)
     rows = w.B * w.block_len
-    ms_red, ms_sel = t_red / reps, t_sel / reps
-    return {"reduce_with_fused_exchange_ms": t_fused / reps,
+    return {"reduce_with_fused_exchange_ms": t_fused,
             "workload": "passk sharded over %d ranks along V (one rank's share, emulated on one GPU): "
                         "fork_vp_reduce on a [%d,%d,%d] slice + fork_vp_select on %d gathered buffers" %
                         (n_ranks, w.B, w.block_len, n, n_ranks),
             "reduce_ms": ms_red, "select_ms": ms_sel, "slice_gbs": rows * n * w.es / (ms_red * 1e-3) / 1e9,
-            "exchange_bytes_per_rank": rows * 16, "note": "slice (%.0f MB) may be L2-resident between repetitions" % (rows * n * w.es / 1e6)}
+            "exchange_bytes_per_rank": rows * 16, "l2": "timed slices rotate over %d distinct regions of %.0f MB (%.1f GB in all)" % (len(views), rows * n * w.es / 1e6, len(views) * rows * n * w.es / 1e9)}
 
 
 def time_fused_head(device, hbm_peak, shapes=((64, 32), (8, 32), (1, 8))):
@@ -942,6 +977,8 @@ def main():
         lp = time_logprob(device, peak)
         summary["grpo_logprob"] = {"us_per_call": round(lp[0]["ms"] * 1e3, 1), "frac": round(lp[0]["frac_of_measured_peak"], 4)}
         summary["grpo_backward"] = {"us_per_call": round(lp[2]["ms"] * 1e3, 1), "frac": round(lp[2]["frac_of_measured_peak"], 4)}
+        summary["grpo_fused"] = {"us_per_call": round(lp[3]["ms"] * 1e3, 1), "frac": round(lp[3]["frac_of_measured_peak"], 4),
+                                 "vs_three_calls": round(lp[3]["speedup_vs_three_calls"], 3)}
         also.extend(lp)
         also.append(time_select(device))
         vp = time_vocab_parallel(device, peak)

@@ -17,8 +17,8 @@
  * fork_step_static (no workspace argument), fork_step_fused_head (the step fused into the LM-head
  * product: hidden states and weight in, no logits in memory); the variants the paper compares with or trains with:
  * candidates drawn at temperature tau > 0 and the other fallback orders (fields of fork_step_args),
- * fork_select_top_entropy (JustGRPO-Fast's position selection), fork_grpo_loss (Eq. 2) and
- * fork_logprob_backward (its log-softmax backward); fork_vp_reduce / fork_vp_reduce_peers /
+ * fork_select_top_entropy (JustGRPO-Fast's position selection), fork_grpo_loss (Eq. 2),
+ * fork_logprob_backward (its log-softmax backward) and fork_grpo_fused (the three in one pass); fork_vp_reduce / fork_vp_reduce_peers /
  * fork_vp_select (the step with the vocabulary sharded over ranks).
  *
  * Conventions for every entry point
@@ -207,6 +207,38 @@ typedef struct fork_logprob_bwd_args {
   int64_t grad_stride_b, grad_stride_l;   /* in elements; grad_stride_l >= V */
 } fork_logprob_bwd_args;
 
+/*
+ * ForkGRPO's pass over the new policy's logits in one call (Section 3.2, Eq. 2): for every selected
+ * position (the fallback steps F_i; logits are [B, Lt, V], the window is the whole buffer) the
+ * log-likelihood of the given token as fork_logprob computes it, the ratio and dJ/dlogp_new as
+ * fork_grpo_loss computes them, and the gradient row of fork_logprob_backward for that dlogp -- with
+ * every selected row read from HBM once and its gradient written once (the three calls in a row read
+ * it twice).  Same results as the three calls.  `logp`, `lse`, `row_status`, `ratio` and `dlogp` are
+ * written at the selected positions only; rows of `grad` that belong to unselected positions, or to
+ * tokens outside [0,V), are not touched.  All pointers are device memory.
+ */
+typedef struct fork_grpo_fused_args {
+  const void* logits; int64_t stride_b, stride_l;
+  int32_t B, Lt, V; int32_t dtype;
+  const int32_t* tokens;     /* [B,Lt] */
+  const uint8_t* select;     /* [B,Lt] non-zero at the positions of F_i */
+  int32_t group;             /* B must be a multiple of group; rollout i = prompt * group + j */
+  const float* logp_old;     /* [B,Lt] log q_theta_old(token) at the selected positions */
+  const float* reward;       /* [B] */
+  float eps_lo, eps_hi;      /* clip range [1 - eps_lo, 1 + eps_hi] */
+  void* grad;                /* out: d J / d logits, same dtype and row addressing as logits, with its own strides */
+  int64_t grad_stride_b, grad_stride_l;   /* in elements; grad_stride_l >= V */
+  float* logp;               /* [B,Lt] out: log q_theta(token) */
+  float* lse;                /* [B,Lt] out, optional */
+  uint32_t* row_status;      /* [B,Lt] out, optional: FORK_ROW_* bits */
+  float* seq_obj;            /* [B] out: obj_i of Eq. 2 */
+  float* objective;          /* [1] out, optional: J */
+  float* adv;                /* [B] out, optional: A_i */
+  float* ratio;              /* [B,Lt] out, optional: rho */
+  float* dlogp;              /* [B,Lt] out, optional: dJ/dlogp_new */
+  uint8_t* skipped;          /* [B/group] out, optional: 1 for a group with equal rewards */
+} fork_grpo_fused_args;
+
 /* Device scratch needed by any entry point for a batch of B sequences of buffer length Lt. */
 size_t fork_workspace_bytes(int32_t B, int32_t Lt);
 
@@ -233,6 +265,9 @@ fork_status fork_grpo_loss(const fork_grpo_args* args, void* stream);
 
 /* Log-softmax backward at the selected rows.  Asynchronous; uses the workspace like fork_logprob. */
 fork_status fork_logprob_backward(const fork_logprob_bwd_args* args, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Scoring, Eq. 2 and the backward in one pass over the logits.  Asynchronous; uses the workspace like fork_logprob. */
+fork_status fork_grpo_fused(const fork_grpo_fused_args* args, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * The step with the vocabulary sharded over N ranks (a vocabulary-parallel LM head): rank j holds

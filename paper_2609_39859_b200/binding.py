@@ -70,6 +70,19 @@ class fork_logprob_bwd_args(C.Structure):
     ]
 
 
+class fork_grpo_fused_args(C.Structure):
+    _fields_ = [
+        ("logits", C.c_void_p), ("stride_b", C.c_int64), ("stride_l", C.c_int64),
+        ("B", C.c_int32), ("Lt", C.c_int32), ("V", C.c_int32), ("dtype", C.c_int32),
+        ("tokens", C.c_void_p), ("select", C.c_void_p), ("group", C.c_int32),
+        ("logp_old", C.c_void_p), ("reward", C.c_void_p), ("eps_lo", C.c_float), ("eps_hi", C.c_float),
+        ("grad", C.c_void_p), ("grad_stride_b", C.c_int64), ("grad_stride_l", C.c_int64),
+        ("logp", C.c_void_p), ("lse", C.c_void_p), ("row_status", C.c_void_p),
+        ("seq_obj", C.c_void_p), ("objective", C.c_void_p), ("adv", C.c_void_p), ("ratio", C.c_void_p),
+        ("dlogp", C.c_void_p), ("skipped", C.c_void_p),
+    ]
+
+
 class fork_head_args(C.Structure):
     _fields_ = [("hidden", C.c_void_p), ("hidden_stride", C.c_int64), ("weight", C.c_void_p), ("weight_stride", C.c_int64),
                 ("d", C.c_int32)]
@@ -79,7 +92,7 @@ fork_logits_fn = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32, C.c_void_p, C.c_voi
                              C.c_void_p, C.c_void_p)
 
 EXPORTS = ("fork_workspace_bytes", "fork_sample_scratch_bytes", "fork_step", "fork_step_static", "fork_step_fused_head", "fork_logprob", "fork_decode_loop", "fork_staging_bytes",
-           "fork_select_top_entropy", "fork_grpo_loss", "fork_logprob_backward", "fork_vp_reduce", "fork_vp_reduce_peers", "fork_vp_select", "fork_read_probe",
+           "fork_select_top_entropy", "fork_grpo_loss", "fork_logprob_backward", "fork_grpo_fused", "fork_vp_reduce", "fork_vp_reduce_peers", "fork_vp_select", "fork_read_probe",
            "fork_step_host", "fork_device_status", "fork_status_string", "fork_set_tuning",
            "fork_kernel_launches", "fork_mask_handovers", "fork_workspace_release", "fork_set_timing_events")
 
@@ -140,6 +153,8 @@ def lib():
     L.fork_grpo_loss.argtypes = [C.POINTER(fork_grpo_args), C.c_void_p]
     L.fork_logprob_backward.restype = C.c_int
     L.fork_logprob_backward.argtypes = [C.POINTER(fork_logprob_bwd_args), C.c_void_p, C.c_size_t, C.c_void_p]
+    L.fork_grpo_fused.restype = C.c_int
+    L.fork_grpo_fused.argtypes = [C.POINTER(fork_grpo_fused_args), C.c_void_p, C.c_size_t, C.c_void_p]
     L.fork_vp_reduce.restype = C.c_int
     L.fork_vp_reduce.argtypes = [C.POINTER(fork_step_args), C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
                                  C.c_void_p]
@@ -429,6 +444,41 @@ def fork_grpo_loss(logp_new: torch.Tensor, logp_old: torch.Tensor, select: torch
     rc = lib().fork_grpo_loss(C.byref(a), _stream_ptr(stream))
     if rc != FORK_OK:
         raise ForkError(rc, "fork_grpo_loss")
+    return out
+
+
+def fork_grpo_fused(logits: torch.Tensor, tokens: torch.Tensor, select: torch.Tensor, logp_old: torch.Tensor,
+                    reward: torch.Tensor, group: int, eps_lo: float, eps_hi: float, grad: torch.Tensor, st: ForkState,
+                    stream=None) -> dict:
+    """Scoring, Eq. 2 and the log-softmax backward in one pass over `logits` [B,Lt,V]: returns the outputs of
+    fork_logprob and fork_grpo_loss as a dict and writes d J / d logits into the selected rows of `grad`."""
+    assert logits.dim() == 3 and logits.stride(2) == 1 and grad.dim() == 3 and grad.stride(2) == 1
+    assert grad.dtype == logits.dtype and grad.shape == logits.shape
+    B, Lt, V = logits.shape
+    for t, dt in ((tokens, torch.int32), (select, torch.uint8), (logp_old, torch.float32), (reward, torch.float32)):
+        assert t.dtype == dt and t.is_contiguous()
+    assert tuple(tokens.shape) == (B, Lt) and st.B == B and st.Lt == Lt
+    dev = logits.device
+    out = dict(logp=torch.zeros((B, Lt), dtype=torch.float32, device=dev),
+               lse=torch.zeros((B, Lt), dtype=torch.float32, device=dev),
+               row_status=torch.zeros((B, Lt), dtype=torch.int32, device=dev),
+               seq_obj=torch.empty(B, dtype=torch.float32, device=dev),
+               objective=torch.empty(1, dtype=torch.float32, device=dev),
+               adv=torch.empty(B, dtype=torch.float32, device=dev),
+               ratio=torch.zeros((B, Lt), dtype=torch.float32, device=dev),
+               dlogp=torch.zeros((B, Lt), dtype=torch.float32, device=dev),
+               skipped=torch.empty(max(B // max(group, 1), 1), dtype=torch.uint8, device=dev))
+    a = fork_grpo_fused_args()
+    a.logits, a.stride_b, a.stride_l = logits.data_ptr(), logits.stride(0), logits.stride(1)
+    a.B, a.Lt, a.V, a.dtype = B, Lt, V, _dtype_code(logits)
+    a.tokens, a.select, a.group = tokens.data_ptr(), select.data_ptr(), group
+    a.logp_old, a.reward, a.eps_lo, a.eps_hi = logp_old.data_ptr(), reward.data_ptr(), float(eps_lo), float(eps_hi)
+    a.grad, a.grad_stride_b, a.grad_stride_l = grad.data_ptr(), grad.stride(0), grad.stride(1)
+    for name, t in out.items():
+        setattr(a, name, t.data_ptr())
+    rc = lib().fork_grpo_fused(C.byref(a), C.c_void_p(st.ws_ptr), st.ws_bytes, _stream_ptr(stream))
+    if rc != FORK_OK:
+        raise ForkError(rc, "fork_grpo_fused")
     return out
 
 

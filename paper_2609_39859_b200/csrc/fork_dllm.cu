@@ -791,16 +791,44 @@ extern "C" fork_status fork_select_top_entropy(const float* entropy, const uint8
    terms).  A second one-CTA kernel sums the per-rollout objectives in a fixed order. */
 constexpr int kGrpoNT = 256;
 
+/* mean and population standard deviation of the rewards of prompt group p (one thread, fp64, in index order) */
+__device__ __forceinline__ void grpo_group_stats(const float* reward, int p, int G, double& mean, double& sd) {
+  double m = 0.0, var = 0.0;
+  for (int j = 0; j < G; ++j) m += (double)reward[p * G + j];
+  m /= G;
+  for (int j = 0; j < G; ++j) { const double d = (double)reward[p * G + j] - m; var += d * d; }
+  mean = m; sd = sqrt(var / G);
+}
+/* number of fallback steps of rollout i (selected positions of its row of `select`), by one warp */
+__device__ __forceinline__ int grpo_count_selected(const uint8_t* select, int i, int Lt) {
+  const int lane = threadIdx.x & 31;
+  int nf = 0;
+  for (int k0 = 0; k0 < Lt; k0 += 32) {
+    const int k = k0 + lane;
+    nf += __popc(__ballot_sync(0xffffffffu, k < Lt && select[(size_t)i * Lt + k] != 0));
+  }
+  return nf;
+}
+/* One token of Eq. 2: the ratio, the clipped minimum, and dJ/dlogp_new (rho A / (B |F_i|) where the
+   unclipped term is the minimum, else 0; nothing for a skipped group). */
+__device__ __forceinline__ void grpo_token(float logp_new, float logp_old, float A, bool skip, float scale, float eps_lo,
+                                           float eps_hi, float& rho, float& term, float& d) {
+  rho = expf(logp_new - logp_old);
+  const float clipped = fminf(fmaxf(rho, 1.f - eps_lo), 1.f + eps_hi);
+  const float u = rho * A, c = clipped * A;
+  term = (u <= c) ? u : c;                                   /* the clipped minimum of Eq. 2 */
+  d = (!skip && u <= c) ? rho * A * scale : 0.f;             /* the unclipped term is active */
+}
+
 __global__ void __launch_bounds__(kGrpoNT) grpo_group_kernel(fork_grpo_args a) {
   __shared__ double sh_mean, sh_sd;
   const int p = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = kGrpoNT / 32;
   const int G = a.group, B = a.B, Lt = a.Lt;
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (tid == 0) {
-    double mean = 0.0, var = 0.0;
-    for (int j = 0; j < G; ++j) mean += (double)a.reward[p * G + j];
-    mean /= G;
-    for (int j = 0; j < G; ++j) { const double d = (double)a.reward[p * G + j] - mean; var += d * d; }
-    sh_mean = mean; sh_sd = sqrt(var / G);
+    double mean, sd;
+    grpo_group_stats(a.reward, p, G, mean, sd);
+    sh_mean = mean; sh_sd = sd;
     if (a.skipped) a.skipped[p] = (uint8_t)(!(sh_sd > 0.0));
   }
   __syncthreads();
@@ -808,22 +836,16 @@ __global__ void __launch_bounds__(kGrpoNT) grpo_group_kernel(fork_grpo_args a) {
   for (int j = warp; j < G; j += nwarp) {
     const int i = p * G + j;
     const float A = skip ? 0.f : (float)(((double)a.reward[i] - sh_mean) / sh_sd);
-    int nf = 0;
-    for (int k0 = 0; k0 < Lt; k0 += 32) {
-      const int k = k0 + lane;
-      nf += __popc(__ballot_sync(0xffffffffu, k < Lt && a.select[(size_t)i * Lt + k] != 0));
-    }
+    const int nf = grpo_count_selected(a.select, i, Lt);
     const float scale = nf > 0 ? 1.f / ((float)B * (float)nf) : 0.f;
     float acc = 0.f;
     for (int k = lane; k < Lt; k += 32) {
       const size_t at = (size_t)i * Lt + k;
       float rho = 0.f, d = 0.f;
       if (a.select[at]) {
-        rho = expf(a.logp_new[at] - a.logp_old[at]);
-        const float clipped = fminf(fmaxf(rho, 1.f - a.eps_lo), 1.f + a.eps_hi);
-        const float u = rho * A, c = clipped * A;
-        acc += (u <= c) ? u : c;                             /* the clipped minimum of Eq. 2 */
-        if (!skip && u <= c) d = rho * A * scale;            /* the unclipped term is active */
+        float term;
+        grpo_token(a.logp_new[at], a.logp_old[at], A, skip, scale, a.eps_lo, a.eps_hi, rho, term, d);
+        acc += term;
       }
       if (a.ratio) a.ratio[at] = rho;
       if (a.dlogp) a.dlogp[at] = d;
@@ -995,6 +1017,267 @@ extern "C" fork_status fork_logprob_backward(const fork_logprob_bwd_args* a, voi
   cudaError_t e = a->dtype == FORK_BF16 ? launch(logprob_backward_kernel<bf16_t>, dim3(grid), dim3(kBwdNT), st, pdl, bp)
                                         : launch(logprob_backward_kernel<float>, dim3(grid), dim3(kBwdNT), st, pdl, bp);
   return e == cudaSuccess ? FORK_OK : FORK_ERR_CUDA;
+}
+
+/* ---- ForkGRPO's training pass over the logits in one kernel ---------------------------------
+ * fork_logprob, the derivative of Eq. 2 and fork_logprob_backward per selected row by ONE CTA: the
+ * row is streamed once for (max, sum exp), the CTA's first thread turns that into log q(token), the
+ * ratio and dJ/dlogp, and the row is streamed a second time for the gradient while most of it is
+ * still in L2 (one row per SM in flight: 148 x 0.5 MB; measured: three quarters of the second pass
+ * hit), so HBM sees about 1.25 reads and one write of every row instead of two reads and one write.
+ * Advantage and 1 / (B |F_i|) per rollout come from a small kernel before it.  Eviction-priority
+ * hints on the two passes changed nothing, a larger persisting-L2 set-aside made everything slower,
+ * fewer CTAs (a smaller footprint in L2) were slower in proportion: a CTA's time per row is set by
+ * the bytes it can keep in flight from registers (96 KB), not by HBM. */
+constexpr int kFusedNT = 512;
+/* 128-bit loads in flight per thread (as many as the register file holds without spilling): 96 KB per SM for
+   fp32 rows, 64 KB for bf16 */
+template <typename T> struct FusedLoads { static constexpr int n = sizeof(T) == 4 ? 12 : 8; };
+
+struct GrpoFusedParams {
+  RowSource src; void* grad; long long gstride_b, gstride_l;
+  const WsHeader* hdr; const int2* rows;
+  const int32_t* tokens; const float* logp_old;
+  const float* adv; const float* scale;                       /* [B] each, from grpo_rollout_kernel; scale < 0 marks a skipped group */
+  float* logp; float* lse; uint32_t* row_status; float* dlogp; float* ratio;
+  int Lt, vector_ok; float eps_lo, eps_hi;
+};
+
+/* per rollout: A_i and 1 / (B |F_i|) (0 when F_i is empty, -1 for a group whose rewards are all equal) */
+__global__ void __launch_bounds__(kGrpoNT) grpo_rollout_kernel(const float* reward, const uint8_t* select, int B, int Lt, int G,
+                                                              float* adv, float* scale) {
+  __shared__ double sh_mean, sh_sd;
+  const int p = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nwarp = kGrpoNT / 32;
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;");
+  if (tid == 0) { double mean, sd; grpo_group_stats(reward, p, G, mean, sd); sh_mean = mean; sh_sd = sd; }
+  __syncthreads();
+  const bool skip = !(sh_sd > 0.0);
+  for (int j = warp; j < G; j += nwarp) {
+    const int i = p * G + j;
+    const int nf = grpo_count_selected(select, i, Lt);
+    if (lane == 0) {
+      adv[i] = skip ? 0.f : (float)(((double)reward[i] - sh_mean) / sh_sd);
+      scale[i] = skip ? -1.f : (nf > 0 ? 1.f / ((float)B * (float)nf) : 0.f);
+    }
+  }
+}
+
+template <typename T> __device__ __forceinline__ uint4 minus_inf_vector();
+template <> __device__ __forceinline__ uint4 minus_inf_vector<bf16_t>() { return make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u); }
+template <> __device__ __forceinline__ uint4 minus_inf_vector<float>() { return make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u); }
+
+template <typename T>
+__device__ __forceinline__ void unpack_vector(const uint4& v, float (&x)[16 / sizeof(T)]) {
+  constexpr int VEC = 16 / (int)sizeof(T);
+  if (sizeof(T) == 2) {
+    x[0] = bf16_lo(v.x); x[1] = bf16_hi(v.x); x[2 % VEC] = bf16_lo(v.y); x[3 % VEC] = bf16_hi(v.y);
+    x[4 % VEC] = bf16_lo(v.z); x[5 % VEC] = bf16_hi(v.z); x[6 % VEC] = bf16_lo(v.w); x[7 % VEC] = bf16_hi(v.w);
+  } else {
+    x[0] = __uint_as_float(v.x); x[1] = __uint_as_float(v.y); x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
+  }
+}
+
+/* running (reference, max, sum 2^((x - reference) L)) of one thread; the reference is the first finite
+   maximum the thread meets and is raised only when a later value exceeds it by kRaiseNats */
+struct LseAcc {
+  float ref, m, s; bool have;
+  __device__ __forceinline__ void init() { ref = 0.f; m = -INFINITY; s = 0.f; have = false; }
+  __device__ __forceinline__ void meet(float vm) {           /* vm: maximum of the values about to be added (NaNs ignored) */
+    if (!have) { if (vm > -INFINITY && vm < INFINITY) { ref = vm; have = true; } }
+    else if (vm > ref + kRaiseNats && vm < INFINITY) { s *= ex2_approx((ref - vm) * kLog2e); ref = vm; }
+    m = fmaxf(m, vm);
+  }
+  __device__ __forceinline__ void add(float x) { s += ex2_approx(fmaf(x, kLog2e, -ref * kLog2e)); }
+  __device__ __forceinline__ Part part() const {
+    if (!have) return Part{m, s, 0.f, kIdxNone};             /* nothing finite: (-inf, 0), or +inf / NaN in s */
+    return Part{m, (m == ref) ? s : s * ex2_approx((ref - m) * kLog2e), 0.f, kIdxNone};
+  }
+};
+
+template <typename T>
+__global__ void __launch_bounds__(kFusedNT, 1) grpo_fused_kernel(const GrpoFusedParams p) {
+  constexpr int VEC = 16 / (int)sizeof(T);
+  constexpr int kFusedLoads = FusedLoads<T>::n;
+  __shared__ Part sh_part[32];
+  __shared__ float sh_w, sh_nl;
+  __shared__ int sh_go;
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int R = p.hdr->R, V = p.src.V;
+  const int tid = (int)threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int r = (int)blockIdx.x; r < R; r += (int)gridDim.x) {
+    const int2 bk = p.rows[r];
+    const size_t at = (size_t)bk.x * p.Lt + bk.y;
+    const int tok = p.tokens[at];
+    const bool tok_ok = tok >= 0 && tok < V;
+    const T* row = row_ptr<T>(p.src, bk.x, bk.y);
+    T* grow = reinterpret_cast<T*>(p.grad) + ((long long)bk.x * p.gstride_b + (long long)(bk.y - p.src.pos0) * p.gstride_l);
+    /* what the first thread needs once the sums are in: fetched now, used after the first pass */
+    float x_tok = 0.f, lp_old = 0.f, adv = 0.f, sc = 0.f;
+    if (tid == 0) {
+      if (tok_ok) x_tok = to_f32(row[tok]);
+      lp_old = p.logp_old[at]; adv = p.adv[bk.x]; sc = p.scale[bk.x];
+    }
+    /* ---- first pass: max and sum exp ---- */
+    LseAcc acc;
+    acc.init();
+    const int nvec = p.vector_ok ? V / VEC : 0;
+    const uint4* rv = reinterpret_cast<const uint4*>(row);
+    for (int v0 = tid; v0 < nvec; v0 += kFusedNT * kFusedLoads) {
+      uint4 q[kFusedLoads];
+#pragma unroll
+      for (int j = 0; j < kFusedLoads; ++j) {
+        const int i = v0 + j * kFusedNT;
+        q[j] = (i < nvec) ? ld_stream(rv + i) : minus_inf_vector<T>();
+      }
+      float vm = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < kFusedLoads; ++j) {
+        float x[VEC];
+        unpack_vector<T>(q[j], x);
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) vm = fmaxf(vm, x[e]);
+      }
+      acc.meet(vm);
+#pragma unroll
+      for (int j = 0; j < kFusedLoads; ++j) {
+        float x[VEC];
+        unpack_vector<T>(q[j], x);
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) acc.add(x[e]);
+      }
+    }
+    for (int e = nvec * VEC + tid; e < V; e += kFusedNT) {   /* the ragged end of the row, or all of an unaligned one */
+      const float x = to_f32(row[e]);
+      acc.meet(x);
+      acc.add(x);
+    }
+    Part part = part_warp_reduce(acc.part());
+    __syncthreads();                                         /* the previous row's readers of the shared values are done */
+    if (lane == 0) sh_part[warp] = part;
+    __syncthreads();
+    if (warp == 0) {
+      part = part_warp_reduce(lane < kFusedNT / 32 ? sh_part[lane] : part_empty());
+      if (lane == 0) {
+        const bool bad = !isfinite(part.s) || !(part.m > -INFINITY) || part.m == INFINITY;
+        const float lns = ln_approx(part.s);
+        uint32_t st = bad ? (uint32_t)FORK_ROW_NONFINITE : 0u;
+        const float qnan = __int_as_float(0x7fc00000);
+        float lp;
+        if (!tok_ok) { st |= FORK_ROW_BAD_TOKEN; lp = 0.f; }
+        else if (bad) lp = qnan;
+        else lp = (x_tok - part.m) - lns;                     /* x_tok - m - ln s */
+        const float lse = bad ? qnan : part.m + lns;
+        float rho, term, d;
+        grpo_token(lp, lp_old, adv, sc < 0.f, sc < 0.f ? 0.f : sc, p.eps_lo, p.eps_hi, rho, term, d);
+        p.logp[at] = lp;
+        if (p.lse) p.lse[at] = lse;
+        if (p.row_status) p.row_status[at] = st;
+        if (p.dlogp) p.dlogp[at] = d;
+        if (p.ratio) p.ratio[at] = rho;
+        sh_w = d; sh_nl = -lse * kLog2e; sh_go = tok_ok ? 1 : 0;
+      }
+    }
+    __syncthreads();
+    if (!sh_go) continue;                                    /* scored as FORK_ROW_BAD_TOKEN: no gradient (uniform over the CTA) */
+    /* ---- second pass: grad = dlogp * (1[v = token] - exp(x - lse)), the row coming from L2 ---- */
+    const float w = sh_w, nl = sh_nl;
+    uint4* gv = reinterpret_cast<uint4*>(grow);
+    for (int v0 = tid; v0 < nvec; v0 += kFusedNT * kFusedLoads) {
+      uint4 q[kFusedLoads];
+#pragma unroll
+      for (int j = 0; j < kFusedLoads; ++j) {
+        const int i = v0 + j * kFusedNT;
+        if (i < nvec) q[j] = ld_stream(rv + i);
+      }
+#pragma unroll
+      for (int j = 0; j < kFusedLoads; ++j) {
+        const int i = v0 + j * kFusedNT;
+        if (i < nvec) {
+          float x[VEC], gr[VEC];
+          unpack_vector<T>(q[j], x);
+#pragma unroll
+          for (int e = 0; e < VEC; ++e) gr[e] = w * ((i * VEC + e == tok ? 1.f : 0.f) - ex2_approx(fmaf(x[e], kLog2e, nl)));
+          uint4 o;
+          if (sizeof(T) == 2) {
+            o.x = pack_bf16x2(gr[0], gr[1]); o.y = pack_bf16x2(gr[2 % VEC], gr[3 % VEC]);
+            o.z = pack_bf16x2(gr[4 % VEC], gr[5 % VEC]); o.w = pack_bf16x2(gr[6 % VEC], gr[7 % VEC]);
+          } else {
+            o.x = __float_as_uint(gr[0]); o.y = __float_as_uint(gr[1]); o.z = __float_as_uint(gr[2]); o.w = __float_as_uint(gr[3]);
+          }
+          __stcs(gv + i, o);
+        }
+      }
+    }
+    for (int e = nvec * VEC + tid; e < V; e += kFusedNT) {
+      const float pr = exp2f(fmaf(to_f32(row[e]), kLog2e, nl));
+      store_grad(grow + e, w * ((e == tok ? 1.f : 0.f) - pr));
+    }
+  }
+}
+
+extern "C" fork_status fork_grpo_fused(const fork_grpo_fused_args* a, void* ws, size_t ws_bytes, void* stream) {
+  if (!a) return FORK_ERR_INVALID_ARG;
+  if (bad_source(a->logits, a->stride_b, a->stride_l, 0, a->B, a->Lt, a->Lt, a->V, a->dtype)) return FORK_ERR_INVALID_ARG;
+  if (!a->tokens || !a->select || !a->logp_old || !a->reward || !a->grad || !a->logp || !a->seq_obj) return FORK_ERR_INVALID_ARG;
+  if (a->group <= 0 || a->B % a->group != 0) return FORK_ERR_INVALID_ARG;
+  if (!(a->eps_lo >= 0.f) || !(a->eps_hi >= 0.f)) return FORK_ERR_INVALID_ARG;
+  if (a->grad_stride_l < a->V || a->grad_stride_b < 0) return FORK_ERR_INVALID_ARG;
+  fork_status s = check_workspace(ws, ws_bytes, a->B, a->Lt);
+  if (s != FORK_OK) return s;
+  if (a->B == 0) {
+    if (a->objective && cudaMemsetAsync(a->objective, 0, sizeof(float), (cudaStream_t)stream) != cudaSuccess) return FORK_ERR_CUDA;
+    return FORK_OK;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  DeviceInfo* dev;
+  if (!device_info(&dev)) return FORK_ERR_CUDA;
+  WsView w = ws_view(ws, a->B, a->Lt);
+  const bool pdl = g_tune[FORK_TUNE_PDL].load() >= 0;
+  /* the rows to score: the selected positions (the fallback steps F_i of every rollout) */
+  SetupParams sp;
+  memset(&sp, 0, sizeof(sp));
+  sp.flags = a->select; sp.lo = nullptr; sp.hi = nullptr;
+  sp.B = a->B; sp.Lt = a->Lt; sp.pos0 = 0; sp.Ll = a->Lt; sp.C = 1; sp.G = 1; sp.min_units = 1;
+  sp.hdr = w.hdr; sp.seq_off = w.seq_off; sp.expected = w.expected; sp.ticket = w.ticket; sp.rows = w.rows;
+  if (launch(active_set_kernel, dim3(1), dim3(kSetupNT), st, pdl, sp) != cudaSuccess) return FORK_ERR_CUDA;
+  /* advantage and 1 / (B |F_i|) per rollout, in a corner of the workspace this path does not use otherwise */
+  float* adv_ws = reinterpret_cast<float*>(w.final_rec);
+  float* scale_ws = adv_ws + a->B;
+  {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)(a->B / a->group)); cfg.blockDim = dim3(kGrpoNT); cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    if (pdl) {
+      attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[0].val.programmaticStreamSerializationAllowed = 1;
+      cfg.attrs = attr; cfg.numAttrs = 1;
+    }
+    if (cudaLaunchKernelEx(&cfg, grpo_rollout_kernel, a->reward, a->select, a->B, a->Lt, a->group, adv_ws, scale_ws) != cudaSuccess)
+      return FORK_ERR_CUDA;
+    g_launches.fetch_add(1);
+  }
+  GrpoFusedParams fp;
+  memset(&fp, 0, sizeof(fp));
+  fp.src = RowSource{a->logits, (long long)a->stride_b, (long long)a->stride_l, 0, a->Lt, a->V};
+  fp.grad = a->grad; fp.gstride_b = a->grad_stride_b; fp.gstride_l = a->grad_stride_l;
+  fp.hdr = w.hdr; fp.rows = w.rows; fp.tokens = a->tokens; fp.logp_old = a->logp_old; fp.adv = adv_ws; fp.scale = scale_ws;
+  fp.logp = a->logp; fp.lse = a->lse; fp.row_status = a->row_status; fp.dlogp = a->dlogp; fp.ratio = a->ratio;
+  fp.Lt = a->Lt; fp.eps_lo = a->eps_lo; fp.eps_hi = a->eps_hi;
+  fp.vector_ok = (source_is_vector_aligned(a->logits, a->stride_b, a->stride_l, a->dtype) &&
+                  source_is_vector_aligned(a->grad, a->grad_stride_b, a->grad_stride_l, a->dtype)) ? 1 : 0;
+  cudaError_t e = a->dtype == FORK_BF16 ? launch(grpo_fused_kernel<bf16_t>, dim3(dev->sms), dim3(kFusedNT), st, pdl, fp)
+                                        : launch(grpo_fused_kernel<float>, dim3(dev->sms), dim3(kFusedNT), st, pdl, fp);
+  if (e != cudaSuccess) return FORK_ERR_CUDA;
+  /* the objective itself and the per-rollout outputs, from the log-probabilities just written */
+  fork_grpo_args g;
+  memset(&g, 0, sizeof(g));
+  g.B = a->B; g.Lt = a->Lt; g.group = a->group;
+  g.logp_new = a->logp; g.logp_old = a->logp_old; g.select = a->select; g.reward = a->reward;
+  g.eps_lo = a->eps_lo; g.eps_hi = a->eps_hi;
+  g.seq_obj = a->seq_obj; g.objective = a->objective; g.adv = a->adv; g.skipped = a->skipped;
+  return fork_grpo_loss(&g, stream);
 }
 
 /* ---- vocabulary-parallel entry points ------------------------------------------------------- */

@@ -183,3 +183,17 @@ def test_invalid_arguments_of_the_variant_entry_points():
         setattr(bad, field, value)
         assert L.fork_logprob_backward(C.byref(bad), ws, nbytes, None) == INV, field
     assert L.fork_logprob_backward(C.byref(b), ws, 16, None) == pkg.FORK_ERR_WORKSPACE
+    f = pkg.fork_grpo_fused_args()
+    f.logits = 0x1000
+    f.stride_b, f.stride_l = 32 * 1024, 1024
+    f.B, f.Lt, f.V, f.dtype, f.group = 4, 32, 1024, pkg.FORK_F32, 2
+    f.tokens = f.select = f.logp_old = f.reward = f.grad = f.logp = f.seq_obj = 0x9000
+    f.grad_stride_b, f.grad_stride_l = 32 * 1024, 1024
+    f.eps_lo = f.eps_hi = 0.2
+    for field, value in (("grad", None), ("logp", None), ("seq_obj", None), ("reward", None), ("logp_old", None), ("group", 3),
+                         ("group", 0), ("grad_stride_l", 100), ("V", 0), ("eps_hi", float("nan")), ("dtype", 7)):
+        bad = pkg.fork_grpo_fused_args.from_buffer_copy(f)
+        setattr(bad, field, value)
+        assert L.fork_grpo_fused(C.byref(bad), ws, nbytes, None) == INV, field
+    assert L.fork_grpo_fused(None, ws, nbytes, None) == INV
+    assert L.fork_grpo_fused(C.byref(f), ws, 16, None) == pkg.FORK_ERR_WORKSPACE
