@@ -1216,6 +1216,274 @@ __global__ void __launch_bounds__(kFusedNT, 1) grpo_fused_kernel(const GrpoFused
   }
 }
 
+/* The same pass for 16-byte aligned rows, fed by bulk copies instead of register loads, by a pair
+   of CTAs (a cluster of two) per row, each on one half of it.  A producer lane copies the half row
+   in 16 KB pieces into a ring in shared memory -- first for the sums, then, straight behind, once
+   more for the gradient, then the next row -- and sixteen consumer warps work through the stages in
+   that order.  What is in flight is the ring (192 KB), not what the register file holds; the second
+   pass's pieces arrive while the first pass is still being summed, and the next row's first pass
+   streams in under the gradient stores.  The two CTAs exchange their (max, sum) through each
+   other's shared memory (a 16-byte remote store and a remote mbarrier arrival each way; nothing
+   spins on global memory) and both work out the row's values from the two halves in the same order.
+   Why pairs: with one CTA per row the second pass found only half of the row still in L2 (148 rows of
+   0.5 MB in flight, and the gradient stores pass through L2 too); with half the rows in flight it
+   finds nearly all of it.  Every wait is bounded; the cluster-wide barriers at the two ends of the
+   kernel are reached by every CTA on every path. */
+constexpr int kFrStageBytes = 16384;
+constexpr int kFrStages = 12;
+constexpr int kFrWarps = 16;
+constexpr int kFrPerSm = 1;
+constexpr int kFrConsumers = kFrWarps * 32;
+constexpr int kFrThreads = kFrConsumers + 32;
+constexpr uint32_t kFrSpinLimit = 1u << 24;
+
+constexpr int kFrCluster = 2;
+struct FrSmem {
+  unsigned long long full[kFrStages], empty[kFrStages];
+  unsigned long long red, go;                              /* the warps' sums are in / the row's values are out */
+  unsigned long long xbar;                                 /* both halves' sums are in xpart (one arrival per CTA of the pair) */
+  float4 xpart[2][kFrCluster];                             /* [row parity][rank]: (m, s, -, -) of each half */
+  Part part[kFrWarps];
+  float w, nl;
+  int abort;
+};
+constexpr size_t kFrSmemBytes = (size_t)kFrStages * kFrStageBytes + sizeof(FrSmem) + 128;
+
+__device__ __forceinline__ uint32_t fr_peer_addr(const void* local, uint32_t rank) {
+  uint32_t ra;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(smem_u32(local)), "r"(rank));
+  return ra;
+}
+__device__ __forceinline__ bool fr_try_wait_cluster(unsigned long long* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+template <bool CLUSTER_SCOPE = false>
+__device__ __forceinline__ bool fr_wait(unsigned long long* bar, uint32_t parity, FrSmem& sm, const WsHeader* hdr) {
+  for (uint32_t i = 0; i < kFrSpinLimit; ++i) {
+    if (CLUSTER_SCOPE ? fr_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
+    if ((i & 1023u) == 1023u && *reinterpret_cast<volatile int*>(&sm.abort)) return false;
+  }
+  *reinterpret_cast<volatile int*>(&sm.abort) = 1;
+  atomicOr(const_cast<uint32_t*>(&hdr->dev_status), (uint32_t)FORK_DEV_TIMEOUT);
+  return false;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kFrThreads, kFrPerSm) grpo_fused_ring_kernel(const GrpoFusedParams p) {
+  constexpr int VEC = 16 / (int)sizeof(T);
+  constexpr int kStageVecs = kFrStageBytes / 16;
+  extern __shared__ unsigned char fr_raw[];
+  unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(fr_raw) + 127) & ~(uintptr_t)127);
+  FrSmem& sm = *reinterpret_cast<FrSmem*>(ring + (size_t)kFrStages * kFrStageBytes);
+  const int tid = (int)threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) {
+    for (int s = 0; s < kFrStages; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], kFrWarps); }
+    mbar_init(&sm.red, kFrWarps); mbar_init(&sm.go, 1); mbar_init(&sm.xbar, kFrCluster);
+    sm.abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  /* nobody writes into a peer's shared memory before the peer has set its barriers up */
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int R = p.hdr->R, V = p.src.V;
+  const uint32_t rank = (uint32_t)blockIdx.x % kFrCluster;
+  const int cid = (int)blockIdx.x / kFrCluster, ncl = (int)gridDim.x / kFrCluster;
+  const int nvec_row = V / VEC;                              /* whole 128-bit vectors of a row; the rest by plain loads */
+  const int nv_half = (nvec_row + kFrCluster - 1) / kFrCluster;
+  const int vbase = min((int)rank * nv_half, nvec_row);      /* this CTA's vectors: [vbase, vbase + nvec) */
+  const int nvec = min(nv_half, nvec_row - vbase);
+  const int nchunk = (nvec + kStageVecs - 1) / kStageVecs;
+  const bool has_tail = rank == kFrCluster - 1;              /* the last CTA of the pair takes the ragged end */
+  if (warp == kFrWarps) {
+    /* ---------------- producer ---------------- */
+    if (lane == 0) {
+      uint32_t n = 0;
+      bool ok = true;
+      for (int r = cid; r < R && ok; r += ncl) {
+        const int2 bk = p.rows[r];
+        const int tok = p.tokens[(size_t)bk.x * p.Lt + bk.y];
+        const int passes = (tok >= 0 && tok < V) ? 2 : 1;
+        const unsigned char* row = reinterpret_cast<const unsigned char*>(row_ptr<T>(p.src, bk.x, bk.y)) + (size_t)vbase * 16;
+        for (int pass = 0; pass < passes && ok; ++pass)
+          for (int c = 0; c < nchunk; ++c, ++n) {
+            const uint32_t s = n % kFrStages, ph = (n / kFrStages) & 1u;
+            if (!fr_wait(&sm.empty[s], ph ^ 1u, sm, p.hdr)) { ok = false; break; }
+            const uint32_t bytes = (uint32_t)min(kStageVecs, nvec - c * kStageVecs) * 16u;
+            mbar_arrive_expect_tx(&sm.full[s], bytes);
+            bulk_copy_g2s(ring + (size_t)s * kFrStageBytes, row + (size_t)c * kFrStageBytes, bytes, &sm.full[s]);
+          }
+      }
+      if (!ok) {                                             /* do not leave with copies still landing */
+        const uint32_t first = n > (uint32_t)kFrStages ? n - (uint32_t)kFrStages : 0u;
+        for (uint32_t q = first; q < n; ++q) {
+          unsigned long long* bar = &sm.full[q % kFrStages];
+          const uint32_t par = (q / kFrStages) & 1u;
+          for (uint32_t i = 0; i < kFrSpinLimit && !mbar_try_wait(bar, par); ++i) {}
+        }
+      }
+    }
+  } else {
+    /* ---------------- consumers ---------------- */
+    uint32_t n = 0, rows_done = 0;
+    bool ok = true;
+    for (int r = cid; r < R && ok; r += ncl, ++rows_done) {
+      const int2 bk = p.rows[r];
+      const size_t at = (size_t)bk.x * p.Lt + bk.y;
+      const int tok = p.tokens[at];
+      const bool tok_ok = tok >= 0 && tok < V;
+      const T* row = row_ptr<T>(p.src, bk.x, bk.y);
+      T* grow = reinterpret_cast<T*>(p.grad) + ((long long)bk.x * p.gstride_b + (long long)(bk.y - p.src.pos0) * p.gstride_l);
+      float x_tok = 0.f, lp_old = 0.f, adv = 0.f, sc = 0.f;
+      if (tid == 0) {
+        if (tok_ok) x_tok = to_f32(row[tok]);
+        lp_old = p.logp_old[at]; adv = p.adv[bk.x]; sc = p.scale[bk.x];
+      }
+      /* ---- first pass over this CTA's half ---- */
+      LseAcc acc;
+      acc.init();
+      for (int c = 0; c < nchunk; ++c, ++n) {
+        const uint32_t s = n % kFrStages, ph = (n / kFrStages) & 1u;
+        if (!__all_sync(0xffffffffu, fr_wait(&sm.full[s], ph, sm, p.hdr))) { ok = false; break; }   /* the whole warp stays or goes */
+        const uint4* st = reinterpret_cast<const uint4*>(ring + (size_t)s * kFrStageBytes);
+        const int nv = min(kStageVecs, nvec - c * kStageVecs);
+        uint4 q[kStageVecs / kFrConsumers];
+#pragma unroll
+        for (int j = 0; j < kStageVecs / kFrConsumers; ++j) {
+          const int i = tid + j * kFrConsumers;
+          q[j] = (i < nv) ? st[i] : minus_inf_vector<T>();
+        }
+        float vm = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < kStageVecs / kFrConsumers; ++j) {
+          float x[VEC];
+          unpack_vector<T>(q[j], x);
+#pragma unroll
+          for (int e = 0; e < VEC; ++e) vm = fmaxf(vm, x[e]);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.empty[s]);            /* every loaded word has been used, so the values sit in registers: the stage may be refilled */
+        acc.meet(vm);
+#pragma unroll
+        for (int j = 0; j < kStageVecs / kFrConsumers; ++j) {
+          float x[VEC];
+          unpack_vector<T>(q[j], x);
+#pragma unroll
+          for (int e = 0; e < VEC; ++e) acc.add(x[e]);
+        }
+      }
+      if (!ok) break;
+      if (has_tail)
+        for (int e = nvec_row * VEC + tid; e < V; e += kFrConsumers) {   /* the ragged end of the row */
+          const float x = to_f32(row[e]);
+          acc.meet(x);
+          acc.add(x);
+        }
+      const Part mine = part_warp_reduce(acc.part());
+      if (lane == 0) { sm.part[warp] = mine; mbar_arrive(&sm.red); }
+      if (warp == 0) {
+        if (!__all_sync(0xffffffffu, fr_wait(&sm.red, rows_done & 1u, sm, p.hdr))) { ok = false; break; }
+        const Part half = part_warp_reduce(lane < kFrWarps ? sm.part[lane] : part_empty());
+        if (lane == 0) {
+          /* this half's (m, s) into the same slot of both CTAs, then one arrival on each CTA's barrier;
+             the arrival releases the store, the wait below acquires the peer's */
+          const uint32_t par = rows_done & 1u;
+          const float4 mine4 = make_float4(half.m, half.s, 0.f, 0.f);
+          for (uint32_t j = 0; j < (uint32_t)kFrCluster; ++j) {
+            const uint32_t slot = fr_peer_addr(&sm.xpart[par][rank], j), bar = fr_peer_addr(&sm.xbar, j);
+            asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};"
+                         :: "r"(slot), "f"(mine4.x), "f"(mine4.y), "f"(mine4.z), "f"(mine4.w) : "memory");
+            asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" :: "r"(bar) : "memory");
+          }
+          if (!fr_wait<true>(&sm.xbar, par, sm, p.hdr)) ok = false;
+          Part part = part_empty();
+          for (int j = 0; j < kFrCluster; ++j) {
+            const volatile float* h = reinterpret_cast<const volatile float*>(&sm.xpart[par][j]);
+            part = part_merge(part, Part{h[0], h[1], 0.f, kIdxNone});
+          }
+          const bool bad = !isfinite(part.s) || !(part.m > -INFINITY) || part.m == INFINITY;
+          const float lns = ln_approx(part.s);
+          uint32_t stt = bad ? (uint32_t)FORK_ROW_NONFINITE : 0u;
+          const float qnan = __int_as_float(0x7fc00000);
+          float lp;
+          if (!tok_ok) { stt |= FORK_ROW_BAD_TOKEN; lp = 0.f; }
+          else if (bad) lp = qnan;
+          else lp = (x_tok - part.m) - lns;                   /* x_tok - m - ln s */
+          const float lse = bad ? qnan : part.m + lns;
+          float rho, term, d;
+          grpo_token(lp, lp_old, adv, sc < 0.f, sc < 0.f ? 0.f : sc, p.eps_lo, p.eps_hi, rho, term, d);
+          if (rank == 0 && ok) {
+            p.logp[at] = lp;
+            if (p.lse) p.lse[at] = lse;
+            if (p.row_status) p.row_status[at] = stt;
+            if (p.dlogp) p.dlogp[at] = d;
+            if (p.ratio) p.ratio[at] = rho;
+          }
+          sm.w = d; sm.nl = -lse * kLog2e;
+          if (ok) mbar_arrive(&sm.go);
+        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) break;
+      }
+      if (!__all_sync(0xffffffffu, fr_wait(&sm.go, rows_done & 1u, sm, p.hdr))) { ok = false; break; }
+      if (!tok_ok) continue;                                 /* scored as FORK_ROW_BAD_TOKEN: no gradient, and no second pass was copied */
+      /* ---- second pass ---- */
+      const float w = sm.w, nl = sm.nl;
+      uint4* gv = reinterpret_cast<uint4*>(grow) + vbase;
+      for (int c = 0; c < nchunk; ++c, ++n) {
+        const uint32_t s = n % kFrStages, ph = (n / kFrStages) & 1u;
+        if (!__all_sync(0xffffffffu, fr_wait(&sm.full[s], ph, sm, p.hdr))) { ok = false; break; }
+        const uint4* st = reinterpret_cast<const uint4*>(ring + (size_t)s * kFrStageBytes);
+        const int nv = min(kStageVecs, nvec - c * kStageVecs);
+        uint4 q[kStageVecs / kFrConsumers];
+#pragma unroll
+        for (int j = 0; j < kStageVecs / kFrConsumers; ++j) {
+          const int i = tid + j * kFrConsumers;
+          if (i < nv) q[j] = st[i];
+        }
+        uint4 out[kStageVecs / kFrConsumers];
+#pragma unroll
+        for (int j = 0; j < kStageVecs / kFrConsumers; ++j) {
+          const int i = tid + j * kFrConsumers;
+          if (i < nv) {
+            const int e0 = (vbase + c * kStageVecs + i) * VEC;
+            float x[VEC], gr[VEC];
+            unpack_vector<T>(q[j], x);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) gr[e] = w * ((e0 + e == tok ? 1.f : 0.f) - ex2_approx(fmaf(x[e], kLog2e, nl)));
+            uint4& o = out[j];
+            if (sizeof(T) == 2) {
+              o.x = pack_bf16x2(gr[0], gr[1]); o.y = pack_bf16x2(gr[2 % VEC], gr[3 % VEC]);
+              o.z = pack_bf16x2(gr[4 % VEC], gr[5 % VEC]); o.w = pack_bf16x2(gr[6 % VEC], gr[7 % VEC]);
+            } else {
+              o.x = __float_as_uint(gr[0]); o.y = __float_as_uint(gr[1]); o.z = __float_as_uint(gr[2]); o.w = __float_as_uint(gr[3]);
+            }
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.empty[s]);            /* the gradients are computed: every loaded word has been used */
+#pragma unroll
+        for (int j = 0; j < kStageVecs / kFrConsumers; ++j) {
+          const int i = tid + j * kFrConsumers;
+          if (i < nv) __stcs(gv + (size_t)c * kStageVecs + i, out[j]);
+        }
+      }
+      if (!ok) break;
+      if (has_tail)
+        for (int e = nvec_row * VEC + tid; e < V; e += kFrConsumers) {
+          const float pr = exp2f(fmaf(to_f32(row[e]), kLog2e, nl));
+          store_grad(grow + e, w * ((e == tok ? 1.f : 0.f) - pr));
+        }
+    }
+  }
+  __syncthreads();
+  /* nobody leaves while its peer may still store into its shared memory */
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 extern "C" fork_status fork_grpo_fused(const fork_grpo_fused_args* a, void* ws, size_t ws_bytes, void* stream) {
   if (!a) return FORK_ERR_INVALID_ARG;
   if (bad_source(a->logits, a->stride_b, a->stride_l, 0, a->B, a->Lt, a->Lt, a->V, a->dtype)) return FORK_ERR_INVALID_ARG;
@@ -1267,8 +1535,51 @@ extern "C" fork_status fork_grpo_fused(const fork_grpo_fused_args* a, void* ws, 
   fp.Lt = a->Lt; fp.eps_lo = a->eps_lo; fp.eps_hi = a->eps_hi;
   fp.vector_ok = (source_is_vector_aligned(a->logits, a->stride_b, a->stride_l, a->dtype) &&
                   source_is_vector_aligned(a->grad, a->grad_stride_b, a->grad_stride_l, a->dtype)) ? 1 : 0;
-  cudaError_t e = a->dtype == FORK_BF16 ? launch(grpo_fused_kernel<bf16_t>, dim3(dev->sms), dim3(kFusedNT), st, pdl, fp)
-                                        : launch(grpo_fused_kernel<float>, dim3(dev->sms), dim3(kFusedNT), st, pdl, fp);
+  cudaError_t e;
+  if (fp.vector_ok && g_tune[FORK_TUNE_VARIANT].load() != 1) {
+    static std::once_flag smem_once[64];
+    int di = 0;
+    if (cudaGetDevice(&di) != cudaSuccess || di < 0 || di >= 64) return FORK_ERR_CUDA;
+    std::call_once(smem_once[di], [] {
+      cudaFuncSetAttribute(grpo_fused_ring_kernel<bf16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFrSmemBytes);
+      cudaFuncSetAttribute(grpo_fused_ring_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFrSmemBytes);
+    });
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)(dev->sms * kFrPerSm / kFrCluster * kFrCluster)); cfg.blockDim = dim3(kFrThreads);
+    cfg.dynamicSmemBytes = kFrSmemBytes; cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kFrCluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    {
+      /* a persistent grid: no more clusters than can be resident together (a cluster that had to wait for
+         another to finish would start its share of the rows when the others are done with theirs) */
+      static int max_clusters[64][2];
+      static std::once_flag occ_once[64][2];
+      const int ti = a->dtype == FORK_BF16 ? 0 : 1;
+      std::call_once(occ_once[di][ti], [&] {
+        int n = 0;
+        cudaError_t oe = ti == 0 ? cudaOccupancyMaxActiveClusters(&n, grpo_fused_ring_kernel<bf16_t>, &cfg)
+                                 : cudaOccupancyMaxActiveClusters(&n, grpo_fused_ring_kernel<float>, &cfg);
+        max_clusters[di][ti] = (oe == cudaSuccess && n > 0) ? n : 0;
+      });
+      const int want = dev->sms * kFrPerSm / kFrCluster;
+      const int ncl = max_clusters[di][ti] > 0 && max_clusters[di][ti] < want ? max_clusters[di][ti] : want;
+      cfg.gridDim = dim3((unsigned)(ncl * kFrCluster));
+    }
+    if (pdl) {
+      attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[1].val.programmaticStreamSerializationAllowed = 1;
+      cfg.numAttrs = 2;
+    }
+    e = a->dtype == FORK_BF16 ? cudaLaunchKernelEx(&cfg, grpo_fused_ring_kernel<bf16_t>, fp)
+                              : cudaLaunchKernelEx(&cfg, grpo_fused_ring_kernel<float>, fp);
+    if (e == cudaSuccess) g_launches.fetch_add(1);
+  } else {                                                  /* rows that are not 16-byte aligned (or variant 1): loads from registers */
+    e = a->dtype == FORK_BF16 ? launch(grpo_fused_kernel<bf16_t>, dim3(dev->sms), dim3(kFusedNT), st, pdl, fp)
+                              : launch(grpo_fused_kernel<float>, dim3(dev->sms), dim3(kFusedNT), st, pdl, fp);
+  }
   if (e != cudaSuccess) return FORK_ERR_CUDA;
   /* the objective itself and the per-rollout outputs, from the log-probabilities just written */
   fork_grpo_args g;
