@@ -494,6 +494,19 @@ int64_t fork_kernel_launches(void);
    FORK_TUNE_LATE_CTA).  Synchronises the device; -1 on a CUDA error.  For tests. */
 int64_t fork_mask_handovers(void);
 
+/* For tests: the host-side arithmetic of the work partition as the kernels use it (the paper has no
+   counterpart).  A step's live rows are cut into units of fork_debug_chunk() logits, numbered row by
+   row (C units per row, U in all); fork_debug_effective_grid gives how many of G CTAs take part when
+   every one of them should get at least min_units units; CTA g of those owns the units from
+   fork_debug_part_begin(U, G, g) up to fork_debug_part_begin(U, G, g + 1); fork_debug_part_owner is the
+   CTA that owns unit x, fork_debug_row_parts the number of CTAs that share row r.  Pure functions of
+   their arguments; no GPU is touched. */
+int64_t fork_debug_part_begin(int64_t U, int32_t G, int32_t g);
+int32_t fork_debug_part_owner(int64_t U, int32_t G, int64_t x);
+int32_t fork_debug_row_parts(int64_t U, int32_t G, int32_t C, int64_t r);
+int32_t fork_debug_chunk(void);
+int32_t fork_debug_effective_grid(int64_t U, int32_t G, int32_t min_units);
+
 #ifdef __cplusplus
 }
 #endif
