@@ -94,7 +94,8 @@ fork_logits_fn = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32, C.c_void_p, C.c_voi
 EXPORTS = ("fork_workspace_bytes", "fork_sample_scratch_bytes", "fork_step", "fork_step_static", "fork_step_fused_head", "fork_logprob", "fork_decode_loop", "fork_staging_bytes",
            "fork_select_top_entropy", "fork_grpo_loss", "fork_logprob_backward", "fork_grpo_fused", "fork_vp_reduce", "fork_vp_reduce_peers", "fork_vp_select", "fork_read_probe",
            "fork_step_host", "fork_device_status", "fork_status_string", "fork_set_tuning",
-           "fork_kernel_launches", "fork_mask_handovers", "fork_workspace_release", "fork_set_timing_events")
+           "fork_kernel_launches", "fork_mask_handovers", "fork_workspace_release", "fork_set_timing_events",
+           "fork_debug_part_begin", "fork_debug_part_owner", "fork_debug_row_parts", "fork_debug_chunk", "fork_debug_effective_grid")
 
 _lib = None
 
