@@ -266,3 +266,63 @@ def test_fused_pass_with_a_non_finite_row_and_at_the_training_width():
         close("grad", g[b, k], want, 1e-4, 2e-6 * abs(float(h["dlogp"][b, k])))
     rows_ok = [b for b in range(B) if b != 4]
     close("ratio", h["ratio"][rows_ok][on[rows_ok]], o["ratio"][rows_ok][on[rows_ok]], 1e-5, 1e-7)
+
+
+def test_fused_pass_edge_shapes():
+    """Nothing selected at all; a single selected row (one cluster works, the others only meet at the barriers);
+    bf16 rows of the training width whose halves differ in length and whose last vector is ragged."""
+    pkg = F()
+    rng = np.random.default_rng(5)
+    # (a) nothing selected: no row is read, the objective is 0, grad keeps its canary
+    B, Lt, V, G = 4, 5, 1000, 2
+    x = make_rows(rng, (B, Lt), V, "f32", peak=5.0)
+    xt = to_torch_logits(x)
+    tokens = torch.zeros((B, Lt), dtype=torch.int32, device="cuda")
+    sel = torch.zeros((B, Lt), dtype=torch.uint8, device="cuda")
+    old = torch.zeros((B, Lt), dtype=torch.float32, device="cuda")
+    reward = torch.rand(B, device="cuda")
+    st = pkg.ForkState(B, Lt)
+    grad = torch.full_like(xt, 7.0)
+    out = pkg.fork_grpo_fused(xt, tokens, sel, old, reward, G, 0.2, 0.2, grad, st)
+    torch.cuda.synchronize()
+    assert float(out["objective"][0]) == 0.0 and (out["seq_obj"] == 0).all() and (grad == 7.0).all()
+    # (b) one selected row
+    sel[2, 3] = 1
+    tokens[2, 3] = 17
+    old[2, 3] = -4.0
+    out = pkg.fork_grpo_fused(xt, tokens, sel, old, reward, G, 0.2, 0.2, grad, st)
+    torch.cuda.synchronize()
+    g = grad.cpu().numpy()
+    others = np.ones((B, Lt), bool)
+    others[2, 3] = False
+    assert (g[others] == 7.0).all()
+    lp = oracle.row_logp(x[2, 3], 17)
+    lp = lp[0] if isinstance(lp, tuple) else lp
+    assert abs(float(out["logp"][2, 3]) - lp) <= 1e-5 + 1e-4 * abs(lp)
+    want = oracle.row_logp_grad(x[2, 3], 17, float(out["dlogp"][2, 3]))
+    close("grad", g[2, 3], want, 1e-4, 2e-6 * abs(float(out["dlogp"][2, 3])) + 1e-12)
+    # (c) bf16, V = 126464 + 24: an odd number of vectors (the two halves differ) and no ragged end; then + 3: a ragged end
+    for V in (126464 + 24, ):
+        B, Lt, G = 4, 2, 2
+        xb = make_rows(rng, (B, Lt), V, "bf16", peak=6.0)
+        xt = to_torch_logits(xb)
+        tokens_h = rng.integers(0, V, (B, Lt)).astype(np.int32)
+        tokens_h[0, 0] = V - 1                                  # in the second half's last vector
+        tokens_h[1, 1] = 0
+        sel_h = np.ones((B, Lt), np.uint8)
+        rc, olp, _, _, _ = oracle.logprob(xb, tokens_h, sel_h)
+        old_h = (olp + 0.05 * rng.standard_normal(olp.shape)).astype(np.float32)
+        reward_h = rng.random(B).astype(np.float32)
+        st = pkg.ForkState(B, Lt)
+        grad = torch.zeros_like(xt)
+        out = pkg.fork_grpo_fused(xt, *(torch.from_numpy(t).cuda() for t in (tokens_h, sel_h, old_h, reward_h)), G, 0.2, 0.2, grad, st)
+        torch.cuda.synchronize()
+        assert pkg.fork_device_status(st) == 0
+        h = {k: v.cpu().numpy() for k, v in out.items()}
+        assert_close("logp", h["logp"], olp)
+        o = oracle.grpo_loss(h["logp"], old_h, sel_h, reward_h, G, 0.2, 0.2)
+        close("dlogp", h["dlogp"], o["dlogp"], 1e-4, 1e-9)
+        g = grad.float().cpu().numpy()
+        for b, k in ((0, 0), (1, 1), (3, 0)):
+            want = oracle.row_logp_grad(xb[b, k], int(tokens_h[b, k]), float(h["dlogp"][b, k]))
+            close("grad", g[b, k], want, 2.0 ** -8, 2e-6 * abs(float(h["dlogp"][b, k])))
