@@ -95,3 +95,38 @@ def test_small_ragged_shapes():
 @pytest.mark.parametrize("B,Ll,n_check", [(1, 8, 1), (8, 32, 8), (64, 32, 6)])
 def test_llada_head_shapes(B, Ll, n_check):
     run_case(B=B, Ll=Ll, Lt=256, pos0=32, V=126464, d=4096, lam=0.9, n_check=n_check, seed=10 + B)
+
+
+@pytest.mark.parametrize("mode", ["max_conf", "min_conf", "max_entropy", "random"])
+def test_fallback_orders_on_the_fused_head(mode):
+    """The comparison orders of a fallback step (Algorithm 1's arg-max confidence and the ablations) apply
+    to the fused-head step as to the step on stored logits: with a threshold nothing clears, every live
+    sequence commits exactly the position the oracle picks under that order."""
+    import paper_2609_39859_b200 as pkg
+    code = {"max_conf": pkg.FORK_FALLBACK_MAX_CONF, "min_conf": pkg.FORK_FALLBACK_MIN_CONF,
+            "max_entropy": pkg.FORK_FALLBACK_MAX_ENTROPY, "random": pkg.FORK_FALLBACK_RANDOM}[mode]
+    B, Ll, Lt, V, d = 4, 8, 8, 3000, 256
+    w_bits, w_dev = weight(V, d)
+    rng = np.random.default_rng(40 + code)
+    mask = (rng.random((B, Lt)) < 0.8).astype(np.uint8)
+    mask[:, 0] = 1
+    lo, hi = np.zeros(B, np.int32), np.full(B, Ll, np.int32)
+    rand = rng.integers(0, 2 ** 32, B, dtype=np.uint32) if mode == "random" else None
+    for nonce in range(32):
+        h_bits, _ = fs.head_hidden(w_bits, B * Ll, seed=900 + 32 * code + nonce, h_lo=0.0, h_hi=6.0)
+        logits = oracle.head_logits(h_bits, w_bits).reshape(B, Ll, V)
+        o = oracle.StepState(B, Lt, mask=mask)
+        assert oracle.step(o, logits, lo, hi, 1.0, step_id=0, fallback_mode=code, fallback_rand=rand) == 0
+        if (o.fallback_margin >= (5e-3 if mode == "max_entropy" else 2e-3)).all():   # the order's best and its runner-up are clearly apart
+            break
+    else:
+        raise AssertionError("no draw with clear margins")
+    st = pkg.ForkState(B, Lt, mask=mask)
+    hid = torch.from_numpy(h_bits.view(np.int16)).cuda().view(torch.bfloat16).view(B, Ll, d)
+    pkg.fork_step_fused_head(st, hid, w_dev, torch.from_numpy(lo).cuda(), torch.from_numpy(hi).cuda(), 1.0, step=0,
+                             fallback_mode=code, fallback_rand=None if rand is None else torch.from_numpy(rand.view(np.int32)).cuda())
+    torch.cuda.synchronize()
+    g = st.host()
+    assert (g["is_fallback"] == 1).all() and (g["n_unmasked"] == 1).all()
+    assert (g["fallback_pos"] == o.fallback_pos).all()
+    compare_step_state(g, o, rtol=HEAD_RTOL, atol=HEAD_ATOL)

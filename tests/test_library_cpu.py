@@ -183,6 +183,21 @@ def test_invalid_arguments_of_the_variant_entry_points():
         setattr(bad, field, value)
         assert L.fork_logprob_backward(C.byref(bad), ws, nbytes, None) == INV, field
     assert L.fork_logprob_backward(C.byref(b), ws, 16, None) == pkg.FORK_ERR_WORKSPACE
+    # the step fused into the LM-head product
+    hd = pkg.fork_head_args()
+    hd.hidden, hd.weight, hd.d, hd.hidden_stride, hd.weight_stride = 0x20000, 0x40000, 256, 256, 256
+    a = good_step_args()
+    assert L.fork_step_fused_head(None, C.byref(hd), ws, nbytes, None) == INV
+    assert L.fork_step_fused_head(C.byref(a), None, ws, nbytes, None) == INV
+    for field, value in (("hidden", None), ("weight", None), ("d", 0), ("d", 100), ("hidden_stride", 64), ("weight_stride", 64),
+                         ("hidden_stride", 260), ("hidden", 0x20008)):   # d must be a multiple of 64; rows 16-byte aligned
+        bad = pkg.fork_head_args.from_buffer_copy(hd)
+        setattr(bad, field, value)
+        assert L.fork_step_fused_head(C.byref(a), C.byref(bad), ws, nbytes, None) == INV, field
+    a.temperature = 0.8                                                   # arg-max candidates only
+    assert L.fork_step_fused_head(C.byref(a), C.byref(hd), ws, nbytes, None) == INV
+    a = good_step_args()
+    assert L.fork_step_fused_head(C.byref(a), C.byref(hd), ws, 16, None) == pkg.FORK_ERR_WORKSPACE
     f = pkg.fork_grpo_fused_args()
     f.logits = 0x1000
     f.stride_b, f.stride_l = 32 * 1024, 1024
