@@ -205,14 +205,25 @@ __device__ __noinline__ int row_draw_warp(const ReduceParams& p, const Partition
   };
   float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
   float tail = 0.f;
-  for (int j = 0; j < n; ++j) {
-    const float4* q4 = reinterpret_cast<const float4*>(sq + (size_t)j * kSlotStride) + 2 * lane;
-    const float4 a0 = __ldcg(q4), a1 = __ldcg(q4 + 1);
-    const float tl = __ldcg(sq + (size_t)j * kSlotStride + kSlotTail);
-    const float w = weight(j);
-    v[0] = fmaf(w, a0.x, v[0]); v[1] = fmaf(w, a0.y, v[1]); v[2] = fmaf(w, a0.z, v[2]); v[3] = fmaf(w, a0.w, v[3]);
-    v[4] = fmaf(w, a1.x, v[4]); v[5] = fmaf(w, a1.y, v[5]); v[6] = fmaf(w, a1.z, v[6]); v[7] = fmaf(w, a1.w, v[7]);
-    tail = fmaf(w, tl, tail);
+  for (int j0 = 0; j0 < n; j0 += 4) {                         /* four parts' loads in flight together: one trip for the usual row */
+    float4 a0[4], a1[4];
+    float tl[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int j = min(j0 + i, n - 1);
+      const float4* q4 = reinterpret_cast<const float4*>(sq + (size_t)j * kSlotStride) + 2 * lane;
+      a0[i] = __ldcg(q4); a1[i] = __ldcg(q4 + 1);
+      tl[i] = __ldcg(sq + (size_t)j * kSlotStride + kSlotTail);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (j0 + i < n) {
+        const float w = weight(j0 + i);
+        v[0] = fmaf(w, a0[i].x, v[0]); v[1] = fmaf(w, a0[i].y, v[1]); v[2] = fmaf(w, a0[i].z, v[2]); v[3] = fmaf(w, a0[i].w, v[3]);
+        v[4] = fmaf(w, a1[i].x, v[4]); v[5] = fmaf(w, a1[i].y, v[5]); v[6] = fmaf(w, a1[i].z, v[6]); v[7] = fmaf(w, a1[i].w, v[7]);
+        tail = fmaf(w, tl[i], tail);
+      }
+    }
   }
   const float mine = ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
   const float incl = warp_scan_incl(mine);
@@ -356,8 +367,7 @@ __device__ __forceinline__ void row_part_arrived(const ReduceParams& p, const Pa
   if (last) {
     float xs, total;
     const int tok = row_draw_warp<T>(p, c, r, b, k, xs, total);
-    if (lane == 0) p.row_draw[r] = make_float4(__int_as_float(tok), xs, total, 0.f);
-    __threadfence();
+    if (lane == 0) p.row_draw[r] = make_float4(__int_as_float(tok), xs, total, 0.f);   /* released by this lane's ticket (publish_part) */
     __syncwarp();
   }
 }
@@ -414,7 +424,6 @@ __device__ __forceinline__ RowOut finalize_rows_warp(const ReduceParams& p, cons
     float xs = 0.f;
     if (m.valid && !m.bad) {
       const T* row = row_ptr<T>(p.src, b, k);
-      const int greedy = resolve_index<T>(row, m.merged.idx, p.src.V, m.merged.m);
       float total;
       int tok;
       if (m.reread) {
@@ -424,7 +433,7 @@ __device__ __forceinline__ RowOut finalize_rows_warp(const ReduceParams& p, cons
         const float4 d = __ldcg(p.row_draw + r);             /* left there by the warp that delivered the row's last part */
         tok = __float_as_int(d.x); xs = d.y;
       }
-      if (tok < 0) { tok = greedy; xs = m.merged.m; }
+      if (tok < 0) { tok = resolve_index<T>(row, m.merged.idx, p.src.V, m.merged.m); xs = m.merged.m; }   /* (rare) the arg-max stands in */
       m.merged.idx = tok;
     }
     merged = m.merged;
