@@ -1576,7 +1576,10 @@ extern "C" fork_status fork_grpo_fused(const fork_grpo_fused_args* a, void* ws, 
     e = a->dtype == FORK_BF16 ? cudaLaunchKernelEx(&cfg, grpo_fused_ring_kernel<bf16_t>, fp)
                               : cudaLaunchKernelEx(&cfg, grpo_fused_ring_kernel<float>, fp);
     if (e == cudaSuccess) g_launches.fetch_add(1);
-  } else {                                                  /* rows that are not 16-byte aligned (or variant 1): loads from registers */
+    else (void)cudaGetLastError();                          /* e.g. no room for clusters on this device: the plain kernel below */
+  }
+  if (!(fp.vector_ok && g_tune[FORK_TUNE_VARIANT].load() != 1) || e != cudaSuccess) {
+    /* rows that are not 16-byte aligned (or variant 1): loads from registers */
     e = a->dtype == FORK_BF16 ? launch(grpo_fused_kernel<bf16_t>, dim3(dev->sms), dim3(kFusedNT), st, pdl, fp)
                               : launch(grpo_fused_kernel<float>, dim3(dev->sms), dim3(kFusedNT), st, pdl, fp);
   }
