@@ -359,7 +359,7 @@ fork_status fork_step_fused_head(const fork_step_args* args, const fork_head_arg
  *
  *   - Same arguments, results and asynchrony as fork_step.
  *   - Batches whose scratch need, fork_workspace_bytes(B, Lt), exceeds FORK_STATIC_SCRATCH_BYTES are
- *     rejected with FORK_ERR_WORKSPACE before anything is launched (B*Lt up to about 42,000
+ *     rejected with FORK_ERR_WORKSPACE before anything is launched (B*Lt up to about 30,000
  *     positions fits).
  *   - The first call on each device looks up the array's device address (one cudaGetSymbolAddress,
  *     with that device current) and caches it; make that first call outside any stream capture.
