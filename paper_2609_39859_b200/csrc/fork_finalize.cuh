@@ -596,7 +596,14 @@ __device__ __forceinline__ RowOut gathered_rows_warp(const ReduceParams& p, cons
   const size_t at = p.vp_row_stride > 0 ? (size_t)b * p.src.Ll + (size_t)(k - p.src.pos0) : (size_t)b * p.Lt + k;
   const size_t n = p.vp_row_stride > 0 ? (size_t)p.vp_row_stride : (size_t)p.B * p.Lt;
   Part acc = part_empty();
-  for (int j = 0; j < p.vp_ranks; ++j) acc = part_merge(acc, part_from(__ldg(p.vp_parts_in + j * n + at)));
+  for (int j0 = 0; j0 < p.vp_ranks; j0 += 8) {               /* eight slices' records in flight together, merged in rank order */
+    float4 q[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) q[i] = __ldg(p.vp_parts_in + (size_t)min(j0 + i, p.vp_ranks - 1) * n + at);
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      if (j0 + i < p.vp_ranks) acc = part_merge(acc, part_from(q[i]));
+  }
   const bool bad = !(isfinite(acc.s) && isfinite(acc.t)) || !(acc.m > -INFINITY) || acc.m == INFINITY;
   if (!SAMPLE || bad) return row_out_from(acc, bad);
   /* the slice by inversion with U1 over the slices' tempered totals (each against its own maximum,
