@@ -404,3 +404,59 @@ def test_grpo_training_chain_full_size_sampled_rows():
         assert (np.abs(got - want) <= 2e-6 * abs(float(d[b, k])) + 1e-4 * np.abs(want)).all()
     b, k = map(int, np.argwhere(select == 0)[123])
     assert torch.isnan(grad[b, k]).all()                          # rows of unselected positions keep the canary
+
+
+def test_grpo_fused_pass_full_size_sampled_rows():
+    """fork_grpo_fused in the configuration bench.py times (B=128, Lt=256, V=126464 fp32, 6496 selected rows,
+    16.6 GB of logits and as much gradient): log-probabilities and gradient rows of sampled positions against the
+    oracle, Eq. 2 on the whole batch against the oracle on the call's own log-probabilities, canaries in every
+    sampled row it must not touch."""
+    pkg = F()
+    w = fs.workload("grpo")
+    cfg = w.cfg()
+    tokens, select = fs.scoring_inputs(w, cfg)
+    t = device_logits(w, w.B)
+    sel_d, tok_d = torch.from_numpy(select).cuda(), torch.from_numpy(tokens).cuda()
+    fs.cuda_fill(cfg, 0, sel_d.data_ptr(), None, None, t.data_ptr(), w.Lt * w.V, w.V, 0, w.Lt)
+    st = pkg.ForkState(w.B, w.Lt)
+    rng = np.random.default_rng(6)
+    bs, ks = np.nonzero(select)
+    picks = [(int(bs[i]), int(ks[i])) for i in rng.choice(len(bs), size=24, replace=False)]
+    old_h = np.zeros(select.shape, np.float32)
+    want_lp = {}
+    for b in range(w.B):                                          # old-policy log-probabilities near the new ones
+        for k in np.flatnonzero(select[b]):
+            old_h[b, k] = -2.0
+    for b, k in picks:
+        want_lp[(b, k)] = oracle.row_logp(fs.row_host(cfg, 0, b, k), int(tokens[b, k]))[0]
+        old_h[b, k] = np.float32(want_lp[(b, k)] + 0.05 * rng.standard_normal())
+    gen = torch.Generator(device="cuda").manual_seed(9)
+    reward = (torch.rand(w.B, device="cuda", generator=gen) < 0.4).float()
+    reward[:8] = 1.0                                              # one prompt group with equal rewards
+    grad = torch.empty_like(t)
+    fs.cuda_canary(grad.data_ptr(), grad.numel(), w.dtype, torch.cuda.current_stream().cuda_stream)
+    out = pkg.fork_grpo_fused(t, tok_d, sel_d, torch.from_numpy(old_h).cuda(), reward, 8, 0.2, 0.2, grad, st)
+    torch.cuda.synchronize()
+    assert pkg.fork_device_status(st) == 0
+    h = {k: v.cpu().numpy() for k, v in out.items()}
+    assert (h["row_status"][select != 0] == 0).all()
+    for (b, k), want in want_lp.items():
+        assert_close("logp", h["logp"][b, k], want)
+    o = oracle.grpo_loss(h["logp"], old_h, select, reward.cpu().numpy(), 8, 0.2, 0.2)
+    rho = o["ratio"][select != 0]
+    near = (np.abs(rho - 0.8) < 1e-4) | (np.abs(rho - 1.2) < 1e-4)
+    ok = np.abs(h["dlogp"] - o["dlogp"]) <= 1e-9 + 1e-4 * np.abs(o["dlogp"])
+    assert ok[select != 0][~near].all() and (h["dlogp"][:8][select[:8] != 0] == 0).all()
+    assert abs(float(h["objective"][0]) - o["objective"]) <= 1e-6 + 1e-4 * abs(o["objective"])
+    assert o["skipped"][0] == 1 and h["skipped"][0] == 1
+    for b, k in picks:
+        row = fs.row_host(cfg, 0, b, k)
+        d = float(h["dlogp"][b, k])
+        want = oracle.row_logp_grad(row, int(tokens[b, k]), d)
+        got = grad[b, k].cpu().numpy().astype(np.float64)
+        assert (np.abs(got - want) <= 2e-6 * abs(d) + 1e-4 * np.abs(want)).all(), (b, k)
+        assert abs(float(h["lse"][b, k]) - oracle.row_lse(row)) <= 1e-5 + 1e-5 * abs(float(h["lse"][b, k]))
+    # rows of unselected positions keep the canary (NaN for fp32)
+    ub, uk = np.nonzero(select == 0)
+    for i in rng.choice(len(ub), size=6, replace=False):
+        assert torch.isnan(grad[int(ub[i]), int(uk[i])]).all()
