@@ -335,7 +335,11 @@ fork_status fork_vp_reduce_peers(const fork_step_args* args, int32_t vocab_offse
  *   - The logits are the fp32-accumulated products themselves (not rounded to bf16 on the way), so
  *     results agree with fork_step on materialised bf16 logits only up to that rounding.  A row whose
  *     logits hold NaN or an infinity is flagged FORK_ROW_NONFINITE.
- * Asynchronous on `stream`; three kernels (active set, product + reduction, merge + unmask rule).
+ *   - row_pos0 (optional): the window of every sequence starts at its own position, row b * Ll + l is
+ *     position row_pos0[b] + l of sequence b (args->pos0 is then ignored).  This is how a caller whose
+ *     sequences sit in different blocks hands over just each sequence's active block.
+ * Asynchronous on `stream`; four kernels (active set, product + reduction, merge of the column
+ * splits, unmask rule).
  */
 typedef struct fork_head_args {
   const void* hidden;        /* [B*Ll, d] bf16 */
@@ -343,6 +347,7 @@ typedef struct fork_head_args {
   const void* weight;        /* [V, d] bf16 */
   int64_t weight_stride;     /* elements between rows, >= d */
   int32_t d;                 /* hidden size */
+  const int32_t* row_pos0;   /* device [B], optional: first position of each sequence's window */
 } fork_head_args;
 fork_status fork_step_fused_head(const fork_step_args* args, const fork_head_args* head, void* workspace,
                                  size_t workspace_bytes, void* stream);
@@ -407,6 +412,20 @@ typedef int (*fork_logits_fn)(void* ctx, int32_t step, const int32_t* tokens, co
 fork_status fork_decode_loop(const fork_step_args* proto, int32_t block_len, int32_t gen_lo, int32_t gen_hi,
                              fork_logits_fn provider, void* ctx, int32_t max_steps, int32_t* steps_taken,
                              void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * fork_decode_loop on hidden states: every step, `provider` fills head->hidden with the final hidden
+ * states of each sequence's ACTIVE BLOCK -- row b * Ll + l is position blk_lo[b] + l of sequence b,
+ * where blk_lo is the cursor array the provider is called with (Ll = proto->Ll >= block_len) -- and
+ * the step is fork_step_fused_head on them; the logits are never stored.  Everything else (cursors
+ * advanced on the device, outcomes read from pinned host memory, FORK_TUNE_LOOP_AHEAD, steps_taken,
+ * the error codes) is as for fork_decode_loop.  head->row_pos0 is ignored (the loop supplies its
+ * cursors); proto->pos0, logits, strides and dtype are ignored; temperature must be 0.
+ */
+fork_status fork_decode_loop_fused_head(const fork_step_args* proto, const fork_head_args* head, int32_t block_len,
+                                        int32_t gen_lo, int32_t gen_hi, fork_logits_fn provider, void* ctx,
+                                        int32_t max_steps, int32_t* steps_taken, void* workspace,
+                                        size_t workspace_bytes, void* stream);
 
 /*
  * fork_step for callers whose buffers live in HOST memory (pinned memory recommended): every

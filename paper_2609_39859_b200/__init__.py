@@ -8,5 +8,5 @@ from .binding import (  # noqa: F401
     FORK_FALLBACK_LEFTMOST, FORK_FALLBACK_MAX_CONF, FORK_FALLBACK_MAX_ENTROPY, FORK_FALLBACK_MIN_CONF,
     FORK_FALLBACK_RANDOM, fork_select_top_entropy, fork_grpo_loss, fork_grpo_args, fork_logprob_backward, fork_grpo_fused, fork_grpo_fused_args,
     fork_logprob_bwd_args, fork_vp_reduce, fork_vp_reduce_peers, fork_vp_select, fork_step_vocab_parallel, gather_rank_major, vocab_shards,
-    fork_status_string, fork_step, fork_step_args, fork_step_static, fork_step_fused_head, fork_head_args, FORK_STATIC_SCRATCH_BYTES, fork_workspace_bytes, lib, make_step_args,
+    fork_status_string, fork_step, fork_step_args, fork_step_static, fork_step_fused_head, fork_decode_loop_fused_head, fork_head_args, FORK_STATIC_SCRATCH_BYTES, fork_workspace_bytes, lib, make_step_args,
 )

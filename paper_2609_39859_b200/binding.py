@@ -85,13 +85,13 @@ class fork_grpo_fused_args(C.Structure):
 
 class fork_head_args(C.Structure):
     _fields_ = [("hidden", C.c_void_p), ("hidden_stride", C.c_int64), ("weight", C.c_void_p), ("weight_stride", C.c_int64),
-                ("d", C.c_int32)]
+                ("d", C.c_int32), ("row_pos0", C.c_void_p)]
 
 
 fork_logits_fn = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                              C.c_void_p, C.c_void_p)
 
-EXPORTS = ("fork_workspace_bytes", "fork_sample_scratch_bytes", "fork_step", "fork_step_static", "fork_step_fused_head", "fork_logprob", "fork_decode_loop", "fork_staging_bytes",
+EXPORTS = ("fork_workspace_bytes", "fork_sample_scratch_bytes", "fork_step", "fork_step_static", "fork_step_fused_head", "fork_logprob", "fork_decode_loop", "fork_decode_loop_fused_head", "fork_staging_bytes",
            "fork_select_top_entropy", "fork_grpo_loss", "fork_logprob_backward", "fork_grpo_fused", "fork_vp_reduce", "fork_vp_reduce_peers", "fork_vp_select", "fork_read_probe",
            "fork_step_host", "fork_device_status", "fork_status_string", "fork_set_tuning",
            "fork_kernel_launches", "fork_mask_handovers", "fork_workspace_release", "fork_set_timing_events",
@@ -154,6 +154,9 @@ def lib():
     L.fork_grpo_loss.argtypes = [C.POINTER(fork_grpo_args), C.c_void_p]
     L.fork_logprob_backward.restype = C.c_int
     L.fork_logprob_backward.argtypes = [C.POINTER(fork_logprob_bwd_args), C.c_void_p, C.c_size_t, C.c_void_p]
+    L.fork_decode_loop_fused_head.restype = C.c_int
+    L.fork_decode_loop_fused_head.argtypes = [C.POINTER(fork_step_args), C.POINTER(fork_head_args), C.c_int32, C.c_int32, C.c_int32,
+                                              C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(C.c_int32), C.c_void_p, C.c_size_t, C.c_void_p]
     L.fork_grpo_fused.restype = C.c_int
     L.fork_grpo_fused.argtypes = [C.POINTER(fork_grpo_fused_args), C.c_void_p, C.c_size_t, C.c_void_p]
     L.fork_vp_reduce.restype = C.c_int
@@ -320,10 +323,58 @@ def fork_step_static(st: ForkState, logits: torch.Tensor, blk_lo: torch.Tensor, 
         raise ForkError(rc, "fork_step_static")
 
 
+def _head_args(hidden: torch.Tensor, weight: torch.Tensor, row_pos0=None) -> fork_head_args:
+    assert hidden.dtype == torch.bfloat16 and weight.dtype == torch.bfloat16
+    assert hidden.dim() == 3 and hidden.stride(2) == 1 and hidden.stride(0) == hidden.shape[1] * hidden.stride(1)
+    assert weight.dim() == 2 and weight.stride(1) == 1 and weight.shape[1] == hidden.shape[2]
+    h = fork_head_args()
+    h.hidden, h.hidden_stride, h.weight, h.weight_stride, h.d = hidden.data_ptr(), hidden.stride(1), weight.data_ptr(), weight.stride(0), hidden.shape[2]
+    if row_pos0 is not None:
+        assert row_pos0.dtype == torch.int32 and row_pos0.is_contiguous() and row_pos0.numel() == hidden.shape[0]
+        h.row_pos0 = row_pos0.data_ptr()
+    return h
+
+
+def fork_decode_loop_fused_head(st: ForkState, hidden: torch.Tensor, weight: torch.Tensor, block_len: int, gen_lo: int, gen_hi: int,
+                                provider, ctx, threshold: float, max_steps: int, step0: int = 0, stream=None,
+                                raise_on_error: bool = True, **variant):
+    """fork_decode_loop on hidden states: `provider` (as for fork_decode_loop) fills `hidden` [B, Ll, d] with each
+    sequence's active block (row l of sequence b = position lo[b] + l); the step is the fused LM-head step.
+    Returns (status, steps_taken)."""
+    B, Ll, d = hidden.shape
+    assert B == st.B
+    a = make_step_args(st, None, None, None, threshold, step0, 0, **variant)
+    a.Ll, a.V = Ll, weight.shape[0]
+    h = _head_args(hidden, weight)
+    keep = None
+    if callable(provider) and not isinstance(provider, (int, C._CFuncPtr)):
+        def _tramp(_ctx, step, _tok, _mask, lo, hi, _out, stream_p):
+            try:
+                return int(provider(int(step), lo, hi, stream_p) or 0)
+            except Exception:
+                import traceback
+                traceback.print_exc()
+                return 1
+        keep = fork_logits_fn(_tramp)
+        fn_ptr = C.cast(keep, C.c_void_p)
+    elif isinstance(provider, int):
+        fn_ptr = C.c_void_p(provider)
+    else:
+        fn_ptr = C.cast(provider, C.c_void_p)
+    steps = C.c_int32(0)
+    rc = lib().fork_decode_loop_fused_head(C.byref(a), C.byref(h), block_len, gen_lo, gen_hi, fn_ptr, C.c_void_p(ctx or 0), max_steps,
+                                           C.byref(steps), C.c_void_p(st.ws_ptr), st.ws_bytes, _stream_ptr(stream))
+    del keep
+    if rc != FORK_OK and raise_on_error:
+        raise ForkError(rc, "fork_decode_loop_fused_head")
+    return int(rc), int(steps.value)
+
+
 def fork_step_fused_head(st: ForkState, hidden: torch.Tensor, weight: torch.Tensor, blk_lo: torch.Tensor, blk_hi: torch.Tensor,
-                         threshold: float, step: int = 0, pos0: int = 0, stream=None, **variant) -> None:
+                         threshold: float, step: int = 0, pos0: int = 0, stream=None, row_pos0=None, **variant) -> None:
     """One sampling step from hidden states [B, Ll, d] (bf16) and the LM-head weight [V, d] (bf16): the
-    logits are formed and reduced on the fly, never stored.  Asynchronous on the stream."""
+    logits are formed and reduced on the fly, never stored.  `row_pos0` [B] int32 (optional): every sequence's
+    window starts at its own position.  Asynchronous on the stream."""
     assert hidden.dtype == torch.bfloat16 and weight.dtype == torch.bfloat16
     assert hidden.dim() == 3 and hidden.stride(2) == 1 and hidden.stride(0) == hidden.shape[1] * hidden.stride(1)
     assert weight.dim() == 2 and weight.stride(1) == 1 and weight.shape[1] == hidden.shape[2]
@@ -331,8 +382,7 @@ def fork_step_fused_head(st: ForkState, hidden: torch.Tensor, weight: torch.Tens
     assert B == st.B
     a = make_step_args(st, None, blk_lo, blk_hi, threshold, step, pos0, **variant)
     a.Ll, a.V = Ll, weight.shape[0]
-    h = fork_head_args()
-    h.hidden, h.hidden_stride, h.weight, h.weight_stride, h.d = hidden.data_ptr(), hidden.stride(1), weight.data_ptr(), weight.stride(0), d
+    h = _head_args(hidden, weight, row_pos0)
     rc = lib().fork_step_fused_head(C.byref(a), C.byref(h), C.c_void_p(st.ws_ptr), st.ws_bytes, _stream_ptr(stream))
     if rc != FORK_OK:
         raise ForkError(rc, "fork_step_fused_head")

@@ -554,17 +554,12 @@ static int loop_wait_flag(const volatile unsigned long long* word, uint32_t tick
   }
 }
 
-extern "C" fork_status fork_decode_loop(const fork_step_args* proto, int32_t block_len, int32_t gen_lo,
-                                        int32_t gen_hi, fork_logits_fn provider, void* ctx, int32_t max_steps,
-                                        int32_t* steps_taken, void* ws, size_t ws_bytes, void* stream) {
-  if (steps_taken) *steps_taken = 0;
-  fork_status s = check_step_args(proto, false);
-  if (s != FORK_OK) return s;
-  if (!provider || block_len <= 0 || gen_lo < 0 || gen_hi > proto->Lt || gen_lo > gen_hi || max_steps < 0)
-    return FORK_ERR_INVALID_ARG;
-  s = check_workspace(ws, ws_bytes, proto->B, proto->Lt);
-  if (s != FORK_OK) return s;
-  if (proto->B == 0) return FORK_OK;
+/* The loop itself; `buffer` is what the provider fills (logits, or hidden states), `enqueue` puts one
+   step on the stream for the cursors it is given. */
+template <typename StepFn>
+static fork_status decode_loop_impl(const fork_step_args* proto, void* buffer, int32_t block_len, int32_t gen_lo, int32_t gen_hi,
+                                    fork_logits_fn provider, void* ctx, int32_t max_steps, int32_t* steps_taken,
+                                    void* ws, void* stream, StepFn enqueue) {
   cudaStream_t st = (cudaStream_t)stream;
   WsView w = ws_view(ws, proto->B, proto->Lt);
   int ahead = g_tune[FORK_TUNE_LOOP_AHEAD].load();
@@ -612,13 +607,13 @@ extern "C" fork_status fork_decode_loop(const fork_step_args* proto, int32_t blo
     if (issued >= max_steps) { rc = FORK_ERR_MAX_STEPS; break; }      /* every report is in: something is still masked */
     const int32_t* lo = w.loop_lo[issued & 1];
     const int32_t* hi = w.loop_hi[issued & 1];
-    if (provider(ctx, proto->step + issued, proto->tokens, proto->mask, lo, hi, const_cast<void*>(proto->logits), stream) != 0) {
+    if (provider(ctx, proto->step + issued, proto->tokens, proto->mask, lo, hi, buffer, stream) != 0) {
       rc = FORK_ERR_PROVIDER;
       break;
     }
     fork_step_args a = *proto;
     a.step = proto->step + issued;
-    rc = step_impl(&a, lo, hi, ws, st, nullptr, false, w.loop);
+    rc = enqueue(a, lo, hi, w.loop);
     if (rc != FORK_OK) break;
     ++issued;
   }
@@ -634,6 +629,24 @@ extern "C" fork_status fork_decode_loop(const fork_step_args* proto, int32_t blo
   loop_ring_release(ring);
   if (steps_taken) *steps_taken = done_at >= 0 ? done_at : issued;
   return rc;
+}
+
+extern "C" fork_status fork_decode_loop(const fork_step_args* proto, int32_t block_len, int32_t gen_lo,
+                                        int32_t gen_hi, fork_logits_fn provider, void* ctx, int32_t max_steps,
+                                        int32_t* steps_taken, void* ws, size_t ws_bytes, void* stream) {
+  if (steps_taken) *steps_taken = 0;
+  fork_status s = check_step_args(proto, false);
+  if (s != FORK_OK) return s;
+  if (!provider || block_len <= 0 || gen_lo < 0 || gen_hi > proto->Lt || gen_lo > gen_hi || max_steps < 0)
+    return FORK_ERR_INVALID_ARG;
+  s = check_workspace(ws, ws_bytes, proto->B, proto->Lt);
+  if (s != FORK_OK) return s;
+  if (proto->B == 0) return FORK_OK;
+  cudaStream_t st = (cudaStream_t)stream;
+  return decode_loop_impl(proto, const_cast<void*>(proto->logits), block_len, gen_lo, gen_hi, provider, ctx, max_steps, steps_taken,
+                          ws, stream, [&](const fork_step_args& a, const int32_t* lo, const int32_t* hi, LoopCtl* loop) {
+                            return step_impl(&a, lo, hi, ws, st, nullptr, false, loop);
+                          });
 }
 
 extern "C" fork_status fork_workspace_release(const void* ws) {
@@ -1701,12 +1714,12 @@ static bool head_tensor_map(CUtensorMap* map, const void* base, uint64_t rows, u
                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-extern "C" fork_status fork_step_fused_head(const fork_step_args* a, const fork_head_args* h, void* ws, size_t ws_bytes,
-                                            void* stream) {
+static fork_status check_head_args(const fork_step_args* a, const fork_head_args* h, bool need_bounds) {
   if (!a || !h) return FORK_ERR_INVALID_ARG;
-  if (a->B < 0 || a->Lt <= 0 || a->Ll <= 0 || a->V <= 0 || a->pos0 < 0 || !a->tokens || !a->mask || !a->blk_lo || !a->blk_hi)
-    return FORK_ERR_INVALID_ARG;
-  if ((int64_t)a->B * a->Lt > (int64_t)1 << 30 || a->pos0 + (int64_t)a->Ll > a->Lt) return FORK_ERR_INVALID_ARG;
+  if (a->B < 0 || a->Lt <= 0 || a->Ll <= 0 || a->V <= 0 || a->pos0 < 0 || !a->tokens || !a->mask) return FORK_ERR_INVALID_ARG;
+  if (need_bounds && (!a->blk_lo || !a->blk_hi)) return FORK_ERR_INVALID_ARG;
+  if ((int64_t)a->B * a->Lt > (int64_t)1 << 30) return FORK_ERR_INVALID_ARG;
+  if (need_bounds && !h->row_pos0 && a->pos0 + (int64_t)a->Ll > a->Lt) return FORK_ERR_INVALID_ARG;
   if (a->threshold != a->threshold) return FORK_ERR_INVALID_ARG;
   if (a->fallback_mode < FORK_FALLBACK_LEFTMOST || a->fallback_mode > FORK_FALLBACK_RANDOM) return FORK_ERR_INVALID_ARG;
   if (a->fallback_mode == FORK_FALLBACK_RANDOM && !a->fallback_rand) return FORK_ERR_INVALID_ARG;
@@ -1715,9 +1728,12 @@ extern "C" fork_status fork_step_fused_head(const fork_step_args* a, const fork_
   if (h->hidden_stride < h->d || h->weight_stride < h->d) return FORK_ERR_INVALID_ARG;
   if (((uintptr_t)h->hidden % 16) != 0 || ((uintptr_t)h->weight % 16) != 0 || (h->hidden_stride % 8) != 0 ||
       (h->weight_stride % 8) != 0) return FORK_ERR_INVALID_ARG;        /* tensor copies need 16-byte aligned rows */
-  fork_status s = check_workspace(ws, ws_bytes, a->B, a->Lt);
-  if (s != FORK_OK) return s;
-  if (a->B == 0) return FORK_OK;
+  return FORK_OK;
+}
+
+/* one fused-head step on the stream: windows [row_pos0[b] (or pos0), + Ll) of every sequence, blocks lo / hi */
+static fork_status head_step_impl(const fork_step_args* a, const fork_head_args* h, const int32_t* lo, const int32_t* hi,
+                                  const int32_t* row_pos0, void* ws, cudaStream_t st, LoopCtl* loop) {
   DeviceInfo* dev;
   if (!device_info(&dev)) return FORK_ERR_CUDA;
   std::call_once(g_head_once, head_init);
@@ -1730,7 +1746,6 @@ extern "C" fork_status fork_step_fused_head(const fork_step_args* a, const fork_
       cudaFuncSetAttribute(head_gemm_reduce_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHeadSmemLimit);
     });
   }
-  cudaStream_t st = (cudaStream_t)stream;
   WsView w = ws_view(ws, a->B, a->Lt);
   const bool pdl = g_tune[FORK_TUNE_PDL].load() >= 0;
 
@@ -1769,10 +1784,12 @@ extern "C" fork_status fork_step_fused_head(const fork_step_args* a, const fork_
   /* the active set (Algorithm 2, line 3): row list and per-sequence ranges for the select phase */
   SetupParams sp;
   memset(&sp, 0, sizeof(sp));
-  sp.flags = a->mask; sp.lo = a->blk_lo; sp.hi = a->blk_hi;
+  sp.flags = a->mask; sp.lo = lo; sp.hi = hi;
   sp.B = a->B; sp.Lt = a->Lt; sp.pos0 = a->pos0; sp.Ll = a->Ll; sp.C = 1; sp.G = 1; sp.min_units = 1;
+  sp.pos0_seq = row_pos0;
   sp.hdr = w.hdr; sp.seq_off = w.seq_off; sp.expected = w.expected; sp.ticket = w.ticket; sp.rows = w.rows;
   sp.n_unmasked = a->n_unmasked; sp.is_fallback = a->is_fallback; sp.fallback_pos = a->fallback_pos;
+  sp.loop = loop; sp.step = a->step;
   if (launch(active_set_kernel, dim3(1), dim3(kSetupNT), st, pdl, sp) != cudaSuccess) return FORK_ERR_CUDA;
 
   /* logits tile by tile in tensor memory, reduced to one part per row and vocabulary split */
@@ -1821,9 +1838,41 @@ extern "C" fork_status fork_step_fused_head(const fork_step_args* a, const fork_
   rp.nfe = a->nfe; rp.n_fallback = a->n_fallback;
   rp.fallback_mode = a->fallback_mode; rp.fallback_rand = a->fallback_rand;
   rp.vp_parts_in = w.parts; rp.vp_ranks = 1; rp.vp_row_stride = hp.m_blocks * kHeadM;
+  rp.vp_pos0_seq = row_pos0;
+  rp.loop = loop; rp.blk_lo = lo; rp.blk_hi = hi;
   const dim3 grid((unsigned)((a->B + kVpNT / 32 - 1) / (kVpNT / 32)));
   if (launch(vp_select_kernel<false>, grid, dim3(kVpNT), st, pdl, rp) != cudaSuccess) return FORK_ERR_CUDA;
   return FORK_OK;
+}
+
+extern "C" fork_status fork_step_fused_head(const fork_step_args* a, const fork_head_args* h, void* ws, size_t ws_bytes,
+                                            void* stream) {
+  fork_status s = check_head_args(a, h, true);
+  if (s != FORK_OK) return s;
+  s = check_workspace(ws, ws_bytes, a->B, a->Lt);
+  if (s != FORK_OK) return s;
+  if (a->B == 0) return FORK_OK;
+  return head_step_impl(a, h, a->blk_lo, a->blk_hi, h->row_pos0, ws, (cudaStream_t)stream, nullptr);
+}
+
+extern "C" fork_status fork_decode_loop_fused_head(const fork_step_args* proto, const fork_head_args* head, int32_t block_len,
+                                                   int32_t gen_lo, int32_t gen_hi, fork_logits_fn provider, void* ctx,
+                                                   int32_t max_steps, int32_t* steps_taken, void* ws, size_t ws_bytes,
+                                                   void* stream) {
+  if (steps_taken) *steps_taken = 0;
+  fork_status s = check_head_args(proto, head, false);
+  if (s != FORK_OK) return s;
+  if (!provider || block_len <= 0 || block_len > proto->Ll || gen_lo < 0 || gen_hi > proto->Lt || gen_lo > gen_hi || max_steps < 0)
+    return FORK_ERR_INVALID_ARG;
+  s = check_workspace(ws, ws_bytes, proto->B, proto->Lt);
+  if (s != FORK_OK) return s;
+  if (proto->B == 0) return FORK_OK;
+  cudaStream_t st = (cudaStream_t)stream;
+  /* every sequence's window is its own block: row 0 of sequence b is position lo[b] of the step's cursors */
+  return decode_loop_impl(proto, const_cast<void*>(head->hidden), block_len, gen_lo, gen_hi, provider, ctx, max_steps, steps_taken,
+                          ws, stream, [&](const fork_step_args& a, const int32_t* lo, const int32_t* hi, LoopCtl* loop) {
+                            return head_step_impl(&a, head, lo, hi, lo, ws, st, loop);
+                          });
 }
 
 /* ---- host-buffer entry point --------------------------------------------------------------- */

@@ -468,7 +468,8 @@ __device__ __forceinline__ SeqHint load_seq_hint(const ReduceParams& p, const Ro
     h.cur_lo = lo; h.cur_hi = hi;
     /* a window that reaches outside the logits buffer keeps masked positions the steps cannot see:
        its cursor never moves on (the loop then ends at its step limit) */
-    const bool whole = lo >= 0 && hi <= p.Lt && lo >= p.src.pos0 && hi <= p.src.pos0 + p.src.Ll;
+    const int pos0 = p.vp_pos0_seq ? p.vp_pos0_seq[b] : p.src.pos0;
+    const bool whole = lo >= 0 && hi <= p.Lt && lo >= pos0 && hi <= pos0 + p.src.Ll;
     h.nxt_lo = h.nxt_hi = whole ? gen_hi : -1;
     if (whole) {
       for (int s = lo + bl; s < gen_hi; s += bl) {
@@ -593,7 +594,8 @@ __device__ __forceinline__ RowOut gathered_rows_warp(const ReduceParams& p, cons
   k = 0;
   if (r >= r1) return row_out_from(part_empty(), true);
   k = (k_hint >= 0) ? k_hint : rm.k_of(b, r);
-  const size_t at = p.vp_row_stride > 0 ? (size_t)b * p.src.Ll + (size_t)(k - p.src.pos0) : (size_t)b * p.Lt + k;
+  const size_t at = p.vp_row_stride > 0 ? (size_t)b * p.src.Ll + (size_t)(k - (p.vp_pos0_seq ? p.vp_pos0_seq[b] : p.src.pos0))
+                                        : (size_t)b * p.Lt + k;
   const size_t n = p.vp_row_stride > 0 ? (size_t)p.vp_row_stride : (size_t)p.B * p.Lt;
   Part acc = part_empty();
   for (int j0 = 0; j0 < p.vp_ranks; j0 += 8) {               /* eight slices' records in flight together, merged in rank order */

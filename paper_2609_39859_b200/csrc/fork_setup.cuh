@@ -19,6 +19,7 @@ struct SetupParams {
   int32_t* n_unmasked; uint8_t* is_fallback; int32_t* fallback_pos;   /* step mode */
   float* seq_sum; int32_t* seq_cnt;                                   /* log-probability mode */
   LoopCtl* loop; int step;                                            /* a step of fork_decode_loop (else NULL) */
+  const int32_t* pos0_seq;           /* NULL, or [B]: the position of row 0 of each sequence's window (instead of pos0) */
 };
 
 __device__ __forceinline__ void seq_window(const SetupParams& p, int b, int& lo, int& hi, bool& clipped) {
@@ -26,8 +27,9 @@ __device__ __forceinline__ void seq_window(const SetupParams& p, int b, int& lo,
   lo = l0; hi = h0;
   if (lo < 0) lo = 0;
   if (hi > p.Lt) hi = p.Lt;
-  if (lo < p.pos0) lo = p.pos0;
-  if (hi > p.pos0 + p.Ll) hi = p.pos0 + p.Ll;
+  const int pos0 = p.pos0_seq ? p.pos0_seq[b] : p.pos0;
+  if (lo < pos0) lo = pos0;
+  if (hi > pos0 + p.Ll) hi = pos0 + p.Ll;
   clipped = (h0 > l0) && (lo != l0 || hi != h0);
   if (hi < lo) hi = lo;
 }

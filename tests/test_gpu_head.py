@@ -130,3 +130,58 @@ def test_fallback_orders_on_the_fused_head(mode):
     assert (g["is_fallback"] == 1).all() and (g["n_unmasked"] == 1).all()
     assert (g["fallback_pos"] == o.fallback_pos).all()
     compare_step_state(g, o, rtol=HEAD_RTOL, atol=HEAD_ATOL)
+
+
+def test_decode_loop_on_hidden_states():
+    """fork_decode_loop_fused_head: every step the provider hands over the hidden states of each sequence's own
+    active block (row l of sequence b = position lo[b] + l) and the step runs on the product with the head; the
+    whole loop against the oracle's loop on the same products, sequences drifting apart in their blocks."""
+    import paper_2609_39859_b200 as pkg
+    from helpers import live_mask
+    B, Lt, BL, V, d, lam = 3, 24, 8, 3000, 256, 0.6
+    w_bits, w_dev = weight(V, d)
+    o = oracle.StepState(B, Lt)
+    lo, hi = oracle.block_cursors(o.mask, 0, Lt, BL)
+    hidden_steps = []
+    step = 0
+    while (lo < hi).any():
+        assert step < 200
+        live = live_mask(o.mask, lo, hi)
+        for nonce in range(64):
+            h_bits, _ = fs.head_hidden(w_bits, B * BL, seed=7000 + 64 * step + nonce, h_lo=0.0, h_hi=9.0)
+            blocks = oracle.head_logits(h_bits, w_bits).reshape(B, BL, V)
+            full = np.full((B, Lt, V), np.nan, np.float32)      # rows outside a sequence's block must not be read
+            for b in range(B):
+                n = max(0, min(BL, Lt - int(lo[b])))
+                full[b, lo[b]:lo[b] + n] = blocks[b, :n]
+            import copy
+            trial = copy.deepcopy(o)
+            assert oracle.step(trial, full, lo, hi, lam, step_id=step) == 0
+            rows = full[live]
+            top2 = np.partition(rows, V - 2, axis=1)[:, V - 2:]
+            if (np.abs(trial.conf[live] - np.float64(np.float32(lam))) >= 2e-3).all() and ((top2[:, 1] - top2[:, 0]) >= 5e-3).all():
+                break
+        else:
+            raise AssertionError("no draw with clear margins at step %d" % step)
+        o = trial
+        hidden_steps.append(torch.from_numpy(h_bits.view(np.int16)).view(torch.bfloat16).view(B, BL, d).pin_memory())
+        step += 1
+        lo, hi = oracle.block_cursors(o.mask, 0, Lt, BL, lo, hi)
+    assert step > Lt // BL                                       # more than one step per block: thresholds and fallbacks both occur
+    st = pkg.ForkState(B, Lt)
+    hid = torch.zeros((B, BL, d), dtype=torch.bfloat16, device="cuda")
+    calls = []
+
+    def model(s_, lo_ptr, hi_ptr, stream_ptr):
+        calls.append(s_)
+        hid.copy_(hidden_steps[min(s_, len(hidden_steps) - 1)], non_blocking=True)
+        return 0
+
+    rc, steps = pkg.fork_decode_loop_fused_head(st, hid, w_dev, BL, 0, Lt, model, None, lam, max_steps=200)
+    torch.cuda.synchronize()
+    assert rc == 0 and steps == step and calls == list(range(step))
+    assert pkg.fork_device_status(st) == 0
+    g = st.host()
+    assert g["mask"].sum() == 0
+    compare_step_state(g, o, rtol=HEAD_RTOL, atol=HEAD_ATOL)
+    assert (g["nfe"] == o.nfe).all() and g["n_fallback"].sum() > 0

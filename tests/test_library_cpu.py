@@ -197,6 +197,18 @@ def test_invalid_arguments_of_the_variant_entry_points():
     a.temperature = 0.8                                                   # arg-max candidates only
     assert L.fork_step_fused_head(C.byref(a), C.byref(hd), ws, nbytes, None) == INV
     a = good_step_args()
+    cb = pkg.binding.fork_logits_fn(lambda *x: 0)
+    fn = C.cast(cb, C.c_void_p)
+    n = C.c_int32(7)
+    loop = L.fork_decode_loop_fused_head
+    assert loop(C.byref(a), C.byref(hd), 8, 0, 32, None, None, 10, C.byref(n), ws, nbytes, None) == INV and n.value == 0   # no provider
+    assert loop(C.byref(a), None, 8, 0, 32, fn, None, 10, C.byref(n), ws, nbytes, None) == INV
+    assert loop(C.byref(a), C.byref(hd), 0, 0, 32, fn, None, 10, C.byref(n), ws, nbytes, None) == INV          # block length
+    assert loop(C.byref(a), C.byref(hd), a.Ll + 1, 0, 32, fn, None, 10, C.byref(n), ws, nbytes, None) == INV   # block longer than the window
+    assert loop(C.byref(a), C.byref(hd), 8, 0, a.Lt + 1, fn, None, 10, C.byref(n), ws, nbytes, None) == INV
+    assert loop(C.byref(a), C.byref(hd), 8, 0, 32, fn, None, -1, C.byref(n), ws, nbytes, None) == INV
+    assert loop(C.byref(a), C.byref(hd), 8, 0, 32, fn, None, 10, C.byref(n), ws, 16, None) == pkg.FORK_ERR_WORKSPACE
+    a = good_step_args()
     assert L.fork_step_fused_head(C.byref(a), C.byref(hd), ws, 16, None) == pkg.FORK_ERR_WORKSPACE
     f = pkg.fork_grpo_fused_args()
     f.logits = 0x1000
