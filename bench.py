@@ -24,6 +24,7 @@ from __future__ import annotations
 import argparse
 import ctypes as C
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -718,6 +719,72 @@ def loop_stats(device, names=("b8", "passk")):
     return out
 
 
+def head_loop_stats(device, B=8, Lt=256, block_len=32, threshold=0.9):
+    """The decode loop on hidden states (fork_decode_loop_fused_head) at the B=8 shape and the LLaDA-8B head, beside the
+    same loop with the logits materialised (library GEMM into a bf16 buffer, then fork_decode_loop): the "model" is a
+    pool of seeded hidden-state blocks with a planted peak per row (height h ~ U(0,12) above the row's log-sum-exp, as in
+    the logits workloads), one block per step.  Whole loops by the host's clock."""
+    import torch
+    import paper_2609_39859_b200 as pkg
+    d, V = 4096, 126464
+    gen = torch.Generator(device=device).manual_seed(4321)
+    W = torch.randn((V, d), device=device, generator=gen, dtype=torch.float32).to(torch.bfloat16)
+    pool = []
+    for i in range(16):
+        hid = torch.randn((B, block_len, d), device=device, generator=gen, dtype=torch.float32) * (3.0 / d ** 0.5)
+        tok = torch.randint(0, V, (B, block_len), device=device, generator=gen)
+        height = (math.log(V) + 4.5 - 1.4) + 12.0 * torch.rand((B, block_len, 1), device=device, generator=gen)
+        pool.append((hid + (height / d) * W[tok].float()).to(torch.bfloat16))
+    hid_buf = torch.empty((B, block_len, d), dtype=torch.bfloat16, device=device)
+    logits = torch.empty((B, Lt, V), dtype=torch.bfloat16, device=device)
+
+    class DeviceInts:                                  # the loop's cursor array (a raw device address) as a tensor
+        def __init__(self, ptr, n):
+            self.__cuda_array_interface__ = {"shape": (n,), "typestr": "<i4", "data": (int(ptr), False), "version": 2}
+
+    rows_b = torch.arange(B, device=device).view(B, 1)
+    cols_l = torch.arange(block_len, device=device).view(1, block_len)
+
+    def model_hidden(step, lo_ptr, hi_ptr, stream_p):
+        hid_buf.copy_(pool[step % len(pool)])
+        return 0
+
+    def model_logits(step, lo_ptr, hi_ptr, stream_p):
+        # the same hidden states through the library GEMM, written to each sequence's block of the logits buffer
+        out = torch.matmul(pool[step % len(pool)].view(B * block_len, d), W.t()).view(B, block_len, V)
+        lo = torch.as_tensor(DeviceInts(lo_ptr, B), device=device)
+        logits[rows_b, lo.long().clamp(max=Lt - block_len).view(B, 1) + cols_l] = out
+        return 0
+
+    res = {}
+    for kind in ("fused", "unfused"):
+        best, steps_taken = 1e30, 0
+        for rep in range(3):
+            st = pkg.ForkState(B, Lt, device=device)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            if kind == "fused":
+                rc, steps = pkg.fork_decode_loop_fused_head(st, hid_buf, W, block_len, 0, Lt, model_hidden, None, threshold, Lt + 8)
+            else:
+                rc, steps = pkg.fork_decode_loop(st, logits, block_len, 0, Lt, model_logits, None, threshold, Lt + 8)
+            torch.cuda.synchronize()
+            ms = (time.perf_counter() - t0) * 1e3
+            assert rc == 0 and int(st.mask.sum()) == 0
+            if rep > 0:
+                best = min(best, ms)
+            steps_taken = steps
+            st.close()
+        res[kind] = (best, steps_taken)
+    del W, logits, pool
+    torch.cuda.empty_cache()
+    return {"workload": "decode loop on hidden states: B=%d, %d tokens per sequence in blocks of %d, d=%d, V=%d bf16, threshold %.2f"
+                        % (B, Lt, block_len, d, V, threshold),
+            "steps_taken": res["fused"][1], "loop_wall_ms": res["fused"][0], "wall_us_per_step": res["fused"][0] * 1e3 / max(res["fused"][1], 1),
+            "unfused_steps_taken": res["unfused"][1], "unfused_loop_wall_ms": res["unfused"][0],
+            "unfused_wall_us_per_step": res["unfused"][0] * 1e3 / max(res["unfused"][1], 1),
+            "unfused": "library GEMM of the same hidden states into a bf16 logits buffer, then fork_decode_loop"}
+
+
 def cpu_baseline(w, seed, target_cpu_seconds=12.0):
     """The oracle, as it stands, on one full-block step's rows generated on the host."""
     import fork_synth as fs
@@ -861,7 +928,10 @@ def main():
 
     if args.loops_only:                                        # a profiling aid, not the benchmark line
         if rank == 0:
-            print(json.dumps({"loops": loop_stats(device, tuple(args.loops_only.split(",")))}))
+            if args.loops_only == "head":
+                print(json.dumps({"loops": [head_loop_stats(device)]}))
+            else:
+                print(json.dumps({"loops": loop_stats(device, tuple(args.loops_only.split(",")))}))
         return 0
     if args.head_only:                                         # a profiling aid, not the benchmark line
         if rank == 0:
@@ -999,6 +1069,10 @@ def main():
             summary["loop_" + q["workload"].split(":")[0]] = {"steps": q["steps_taken"], "kernel_us_per_step": round(q["mean_us_per_step"], 2),
                                                               "hbm_gbs": round(q["hbm_gbs"], 1),
                                                               "wall_us_per_step_incl_generator": round(q["wall_us_per_step"], 1)}
+        hl = head_loop_stats(device)
+        summary["loop_b8_hidden_states"] = {"steps": hl["steps_taken"], "wall_us_per_step": round(hl["wall_us_per_step"], 1),
+                                            "unfused_wall_us_per_step": round(hl["unfused_wall_us_per_step"], 1)}
+        loops.append(hl)
         out["cpu_baseline"] = cpu_baseline(w, seed)
         # what a truncated copy of this line must still carry comes first: every shape as (time, fraction of the peak)
         head = {k: out[k] for k in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better",
