@@ -15,7 +15,8 @@
  * Entry points: fork_step (one step), fork_decode_loop (steps until nothing is masked),
  * fork_logprob (log-likelihood scoring of Section 3.2), fork_step_host (host buffers),
  * fork_step_static (no workspace argument), fork_step_fused_head (the step fused into the LM-head
- * product: hidden states and weight in, no logits in memory); the variants the paper compares with or trains with:
+ * product: hidden states and weight in, no logits in memory) and fork_decode_loop_fused_head (the
+ * loop on hidden states); the variants the paper compares with or trains with:
  * candidates drawn at temperature tau > 0 and the other fallback orders (fields of fork_step_args),
  * fork_select_top_entropy (JustGRPO-Fast's position selection), fork_grpo_loss (Eq. 2),
  * fork_logprob_backward (its log-softmax backward) and fork_grpo_fused (the three in one pass); fork_vp_reduce / fork_vp_reduce_peers /
