@@ -543,15 +543,18 @@ def time_fused_head(device, hbm_peak, shapes=((64, 32), (8, 32), (1, 8))):
             logits = torch.matmul(hid.view(R, d), W.t()).view(B, Ll, V)
             pkg.fork_step(st, logits, lo, hi, 0.9)
 
+        def fused_drawn():
+            pkg.fork_step_fused_head(st, hid, W, lo, hi, 0.9, temperature=0.8, sample_seed=11)
+
         reps = 10 if R >= 1024 else 20
-        ms_f, ms_u = timed(fused, reps), timed(unfused, reps)
+        ms_f, ms_u, ms_fd = timed(fused, reps), timed(unfused, reps), timed(fused_drawn, reps)
         flops = 2.0 * R * V * d
         out.append({"workload": "fused LM-head step: %d window rows (B=%d, block %d), d=%d, V=%d, bf16 x bf16 -> fp32" % (R, B, Ll, d, V),
                     "fused_ms": ms_f, "unfused_gemm_plus_fork_step_ms": ms_u, "speedup_vs_unfused": ms_u / ms_f,
                     "tflops": flops / (ms_f * 1e-3) / 1e12, "frac_of_bf16_peak": flops / (ms_f * 1e-3) / 1e12 / tf_peak,
                     "bf16_peak_tflops": tf_peak, "peak_source": tf_src,
                     "weight_read_gbs": V * d * 2 / (ms_f * 1e-3) / 1e9, "weight_read_frac_of_hbm_peak": V * d * 2 / (ms_f * 1e-3) / 1e9 / hbm_peak,
-                    "hbm_bytes_not_moved": 2 * R * V * 2,
+                    "hbm_bytes_not_moved": 2 * R * V * 2, "fused_ms_candidates_drawn_tau0.8": ms_fd,
                     "bound": "tensor" if flops / (tf_peak * 1e12) > V * d * 2 / (hbm_peak * 1e9) else "hbm (one read of the weight)"})
         del st, hid
     del W

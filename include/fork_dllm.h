@@ -332,7 +332,13 @@ fork_status fork_vp_reduce_peers(const fork_step_args* args, int32_t vocab_offse
  *     k of sequence b (every position of the window, masked or not), rows hidden_stride elements apart.
  *   - weight: device, bf16, [V, d], rows weight_stride elements apart: logit v = <hidden row, weight row v>.
  *   - d a multiple of 64; both base addresses 16-byte aligned and both strides multiples of 8 elements.
- *   - args->logits, stride_b, stride_l and dtype are ignored; temperature must be 0.
+ *   - args->logits, stride_b, stride_l and dtype are ignored.
+ *   - temperature > 0 draws the candidates (Algorithm 2 line 4) in two stages, with the two uniforms of the
+ *     row that fork_step uses: the vocabulary is cut into chunks of 32 consecutive entries; the chunk is
+ *     drawn with probability proportional to its tempered weight (by inversion, chunks ascending), and the
+ *     token inside it by inversion in index order -- i.e. the draw fork_step_vocab_parallel makes with one
+ *     slice per chunk.  args->sample_scratch must then hold fork_head_sample_scratch_bytes(B, Ll, V) bytes
+ *     (device, 256-byte aligned; it needs no initialisation).
  *   - The logits are the fp32-accumulated products themselves (not rounded to bf16 on the way), so
  *     results agree with fork_step on materialised bf16 logits only up to that rounding.  A row whose
  *     logits hold NaN or an infinity is flagged FORK_ROW_NONFINITE.
@@ -352,6 +358,7 @@ typedef struct fork_head_args {
 } fork_head_args;
 fork_status fork_step_fused_head(const fork_step_args* args, const fork_head_args* head, void* workspace,
                                  size_t workspace_bytes, void* stream);
+size_t fork_head_sample_scratch_bytes(int32_t B, int32_t Ll, int32_t V);
 
 /*
  * fork_step without a workspace argument, for callers that have no device memory to give and
@@ -421,7 +428,7 @@ fork_status fork_decode_loop(const fork_step_args* proto, int32_t block_len, int
  * the step is fork_step_fused_head on them; the logits are never stored.  Everything else (cursors
  * advanced on the device, outcomes read from pinned host memory, FORK_TUNE_LOOP_AHEAD, steps_taken,
  * the error codes) is as for fork_decode_loop.  head->row_pos0 is ignored (the loop supplies its
- * cursors); proto->pos0, logits, strides and dtype are ignored; temperature must be 0.
+ * cursors); proto->pos0, logits, strides and dtype are ignored.
  */
 fork_status fork_decode_loop_fused_head(const fork_step_args* proto, const fork_head_args* head, int32_t block_len,
                                         int32_t gen_lo, int32_t gen_hi, fork_logits_fn provider, void* ctx,

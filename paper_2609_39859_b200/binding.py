@@ -91,7 +91,7 @@ class fork_head_args(C.Structure):
 fork_logits_fn = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                              C.c_void_p, C.c_void_p)
 
-EXPORTS = ("fork_workspace_bytes", "fork_sample_scratch_bytes", "fork_step", "fork_step_static", "fork_step_fused_head", "fork_logprob", "fork_decode_loop", "fork_decode_loop_fused_head", "fork_staging_bytes",
+EXPORTS = ("fork_workspace_bytes", "fork_sample_scratch_bytes", "fork_step", "fork_step_static", "fork_step_fused_head", "fork_head_sample_scratch_bytes", "fork_logprob", "fork_decode_loop", "fork_decode_loop_fused_head", "fork_staging_bytes",
            "fork_select_top_entropy", "fork_grpo_loss", "fork_logprob_backward", "fork_grpo_fused", "fork_vp_reduce", "fork_vp_reduce_peers", "fork_vp_select", "fork_read_probe",
            "fork_step_host", "fork_device_status", "fork_status_string", "fork_set_tuning",
            "fork_kernel_launches", "fork_mask_handovers", "fork_workspace_release", "fork_set_timing_events",
@@ -154,6 +154,8 @@ def lib():
     L.fork_grpo_loss.argtypes = [C.POINTER(fork_grpo_args), C.c_void_p]
     L.fork_logprob_backward.restype = C.c_int
     L.fork_logprob_backward.argtypes = [C.POINTER(fork_logprob_bwd_args), C.c_void_p, C.c_size_t, C.c_void_p]
+    L.fork_head_sample_scratch_bytes.restype = C.c_size_t
+    L.fork_head_sample_scratch_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32]
     L.fork_decode_loop_fused_head.restype = C.c_int
     L.fork_decode_loop_fused_head.argtypes = [C.POINTER(fork_step_args), C.POINTER(fork_head_args), C.c_int32, C.c_int32, C.c_int32,
                                               C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(C.c_int32), C.c_void_p, C.c_size_t, C.c_void_p]
@@ -294,7 +296,7 @@ def make_step_args(st: ForkState, logits: torch.Tensor, blk_lo, blk_hi, threshol
         setattr(a, name, getattr(st, name).data_ptr())
     a.fallback_mode, a.fallback_rand = int(fallback_mode), _p(fallback_rand)
     a.temperature, a.sample_seed = float(temperature), int(sample_seed)
-    if temperature > 0:
+    if temperature > 0 and logits is not None:           # (the fused-head step brings its own scratch; the select phase needs none)
         a.sample_scratch, a.sample_scratch_bytes = st.sample_scratch_ptr()
     return a
 
@@ -323,6 +325,19 @@ def fork_step_static(st: ForkState, logits: torch.Tensor, blk_lo: torch.Tensor, 
         raise ForkError(rc, "fork_step_static")
 
 
+def _head_sample_scratch(st: ForkState, a: fork_step_args, B: int, Ll: int, V: int, device) -> None:
+    """Scratch of a fused-head step that draws its candidates; kept on the state and reused while it is large enough."""
+    if not a.temperature > 0:
+        return
+    n = int(lib().fork_head_sample_scratch_bytes(B, Ll, V))
+    buf = getattr(st, "_head_scratch", None)
+    if buf is None or buf.numel() < n + 256:
+        buf = torch.empty(n + 256, dtype=torch.uint8, device=device)
+        st._head_scratch = buf
+    off = (-buf.data_ptr()) % 256
+    a.sample_scratch, a.sample_scratch_bytes = buf.data_ptr() + off, n
+
+
 def _head_args(hidden: torch.Tensor, weight: torch.Tensor, row_pos0=None) -> fork_head_args:
     assert hidden.dtype == torch.bfloat16 and weight.dtype == torch.bfloat16
     assert hidden.dim() == 3 and hidden.stride(2) == 1 and hidden.stride(0) == hidden.shape[1] * hidden.stride(1)
@@ -345,6 +360,7 @@ def fork_decode_loop_fused_head(st: ForkState, hidden: torch.Tensor, weight: tor
     assert B == st.B
     a = make_step_args(st, None, None, None, threshold, step0, 0, **variant)
     a.Ll, a.V = Ll, weight.shape[0]
+    _head_sample_scratch(st, a, B, Ll, a.V, hidden.device)
     h = _head_args(hidden, weight)
     keep = None
     if callable(provider) and not isinstance(provider, (int, C._CFuncPtr)):
@@ -382,6 +398,7 @@ def fork_step_fused_head(st: ForkState, hidden: torch.Tensor, weight: torch.Tens
     assert B == st.B
     a = make_step_args(st, None, blk_lo, blk_hi, threshold, step, pos0, **variant)
     a.Ll, a.V = Ll, weight.shape[0]
+    _head_sample_scratch(st, a, B, Ll, a.V, hidden.device)
     h = _head_args(hidden, weight, row_pos0)
     rc = lib().fork_step_fused_head(C.byref(a), C.byref(h), C.c_void_p(st.ws_ptr), st.ws_bytes, _stream_ptr(stream))
     if rc != FORK_OK:

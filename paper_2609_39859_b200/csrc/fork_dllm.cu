@@ -1714,6 +1714,13 @@ static bool head_tensor_map(CUtensorMap* map, const void* base, uint64_t rows, u
                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+extern "C" size_t fork_head_sample_scratch_bytes(int32_t B, int32_t Ll, int32_t V) {
+  if (B < 0 || Ll <= 0 || V <= 0) return 0;
+  const size_t rows_pad = (((size_t)(B > 0 ? B : 1) * (size_t)Ll + kHeadM - 1) / kHeadM) * kHeadM;
+  const size_t cells = (size_t)((V + kHeadGroup - 1) / kHeadGroup) * rows_pad;
+  return 2 * align_up(cells * 4, 256) + align_up(cells, 256) + align_up(rows_pad * sizeof(float4), 256);
+}
+
 static fork_status check_head_args(const fork_step_args* a, const fork_head_args* h, bool need_bounds) {
   if (!a || !h) return FORK_ERR_INVALID_ARG;
   if (a->B < 0 || a->Lt <= 0 || a->Ll <= 0 || a->V <= 0 || a->pos0 < 0 || !a->tokens || !a->mask) return FORK_ERR_INVALID_ARG;
@@ -1723,11 +1730,14 @@ static fork_status check_head_args(const fork_step_args* a, const fork_head_args
   if (a->threshold != a->threshold) return FORK_ERR_INVALID_ARG;
   if (a->fallback_mode < FORK_FALLBACK_LEFTMOST || a->fallback_mode > FORK_FALLBACK_RANDOM) return FORK_ERR_INVALID_ARG;
   if (a->fallback_mode == FORK_FALLBACK_RANDOM && !a->fallback_rand) return FORK_ERR_INVALID_ARG;
-  if (a->temperature != 0.f) return FORK_ERR_INVALID_ARG;              /* arg-max candidates only */
+  if (!(a->temperature >= 0.f) || a->temperature > 3.0e38f) return FORK_ERR_INVALID_ARG;
   if (!h->hidden || !h->weight || h->d <= 0 || h->d % kHeadK != 0) return FORK_ERR_INVALID_ARG;
   if (h->hidden_stride < h->d || h->weight_stride < h->d) return FORK_ERR_INVALID_ARG;
   if (((uintptr_t)h->hidden % 16) != 0 || ((uintptr_t)h->weight % 16) != 0 || (h->hidden_stride % 8) != 0 ||
       (h->weight_stride % 8) != 0) return FORK_ERR_INVALID_ARG;        /* tensor copies need 16-byte aligned rows */
+  if (a->temperature > 0.f && (!a->sample_scratch || ((uintptr_t)a->sample_scratch % 256) != 0 ||
+                               a->sample_scratch_bytes < fork_head_sample_scratch_bytes(a->B, a->Ll, a->V)))
+    return FORK_ERR_WORKSPACE;                                         /* drawn candidates need their scratch */
   return FORK_OK;
 }
 
@@ -1743,7 +1753,8 @@ static fork_status head_step_impl(const fork_step_args* a, const fork_head_args*
     int di = 0;
     if (cudaGetDevice(&di) != cudaSuccess || di < 0 || di >= 64) return FORK_ERR_CUDA;
     std::call_once(smem_once[di], [] {
-      cudaFuncSetAttribute(head_gemm_reduce_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHeadSmemLimit);
+      cudaFuncSetAttribute(head_gemm_reduce_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHeadSmemLimit);
+      cudaFuncSetAttribute(head_gemm_reduce_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHeadSmemLimit);
     });
   }
   WsView w = ws_view(ws, a->B, a->Lt);
@@ -1766,6 +1777,19 @@ static fork_status head_step_impl(const fork_step_args* a, const fork_head_args*
   const size_t head_smem = (size_t)hp.stages * head_stage_bytes(hp.a_box_rows) + kHeadSmemExtra;
   if ((size_t)hp.n_splits * hp.m_blocks * kHeadM > (size_t)a->B * a->Lt + kHeadPartsExtra) return FORK_ERR_WORKSPACE;
   hp.parts = w.head_parts; hp.hdr = w.hdr;
+  const bool drawn = a->temperature > 0.f;
+  if (drawn) {
+    /* per 32-column chunk and window row: log2-weight, drawn logit, drawn index; then a draw record per row */
+    const size_t cells = (size_t)hp.n_groups * hp.m_blocks * kHeadM;
+    char* base = (char*)a->sample_scratch;
+    hp.lw = (float*)base;
+    hp.xt = (float*)(base + align_up(cells * 4, 256));
+    hp.jt = (unsigned char*)(base + 2 * align_up(cells * 4, 256));
+    hp.draw = (float4*)(base + 2 * align_up(cells * 4, 256) + align_up(cells, 256));
+    hp.merged = w.parts;
+    hp.c_tau = (float)(1.4426950408889634 / (double)a->temperature);
+    hp.seed = a->sample_seed; hp.step = a->step; hp.Ll = a->Ll; hp.pos0 = a->pos0; hp.row_pos0 = row_pos0;
+  }
   HeadMaps maps;
   memset(&maps, 0, sizeof(maps));
   if (!head_tensor_map(&maps.h, h->hidden, (uint64_t)hp.rows, (uint64_t)h->d, (uint64_t)h->hidden_stride, (uint32_t)hp.a_box_rows))
@@ -1804,7 +1828,8 @@ static fork_status head_step_impl(const fork_step_args* a, const fork_head_args*
       attr[0].val.programmaticStreamSerializationAllowed = 1;
       cfg.attrs = attr; cfg.numAttrs = 1;
     }
-    if (cudaLaunchKernelEx(&cfg, head_gemm_reduce_kernel, maps, hp) != cudaSuccess) return FORK_ERR_CUDA;
+    if ((drawn ? cudaLaunchKernelEx(&cfg, head_gemm_reduce_kernel<true>, maps, hp)
+               : cudaLaunchKernelEx(&cfg, head_gemm_reduce_kernel<false>, maps, hp)) != cudaSuccess) return FORK_ERR_CUDA;
     g_launches.fetch_add(1);
   }
 
@@ -1823,6 +1848,11 @@ static fork_status head_step_impl(const fork_step_args* a, const fork_head_args*
     }
     if (cudaLaunchKernelEx(&cfg, head_merge_kernel, hp, w.parts) != cudaSuccess) return FORK_ERR_CUDA;
     g_launches.fetch_add(1);
+    if (drawn) {                                             /* the chunk of every row, now that the rows' maxima are known */
+      cfg.gridDim = dim3((unsigned)((hp.rows + 31) / 32)); cfg.blockDim = dim3(kHeadDrawNT);
+      if (cudaLaunchKernelEx(&cfg, head_draw_kernel, hp) != cudaSuccess) return FORK_ERR_CUDA;
+      g_launches.fetch_add(1);
+    }
   }
   /* ... then the unmask rule on one record per row */
   ReduceParams rp;
@@ -1840,8 +1870,10 @@ static fork_status head_step_impl(const fork_step_args* a, const fork_head_args*
   rp.vp_parts_in = w.parts; rp.vp_ranks = 1; rp.vp_row_stride = hp.m_blocks * kHeadM;
   rp.vp_pos0_seq = row_pos0;
   rp.loop = loop; rp.blk_lo = lo; rp.blk_hi = hi;
+  if (drawn) { rp.head_draw = hp.draw; rp.sample_seed = a->sample_seed; rp.noise_c = hp.c_tau; }
   const dim3 grid((unsigned)((a->B + kVpNT / 32 - 1) / (kVpNT / 32)));
-  if (launch(vp_select_kernel<false>, grid, dim3(kVpNT), st, pdl, rp) != cudaSuccess) return FORK_ERR_CUDA;
+  if ((drawn ? launch(vp_select_kernel<true>, grid, dim3(kVpNT), st, pdl, rp)
+             : launch(vp_select_kernel<false>, grid, dim3(kVpNT), st, pdl, rp)) != cudaSuccess) return FORK_ERR_CUDA;
   return FORK_OK;
 }
 

@@ -608,6 +608,13 @@ __device__ __forceinline__ RowOut gathered_rows_warp(const ReduceParams& p, cons
   }
   const bool bad = !(isfinite(acc.s) && isfinite(acc.t)) || !(acc.m > -INFINITY) || acc.m == INFINITY;
   if (!SAMPLE || bad) return row_out_from(acc, bad);
+  if (p.head_draw) {                                         /* fused LM-head step: the row's draw was made by head_draw_kernel */
+    const float4 d = __ldg(p.head_draw + at);
+    const int tok = __float_as_int(d.x);
+    if (tok < 0) return row_out_from(acc, false);            /* nothing had weight: the arg-max stands in */
+    acc.idx = tok;
+    return row_out_sampled(acc, false, d.y);
+  }
   /* the slice by inversion with U1 over the slices' tempered totals (each against its own maximum,
      re-weighted to the row's), in rank order; the token is that slice's own draw */
   const float u1 = sample_uniform_slice(sample_row_key(p.sample_seed, p.step, b, k));

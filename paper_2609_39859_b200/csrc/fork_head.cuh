@@ -69,6 +69,16 @@ struct HeadParams {
   int stages;                /* ring depth that fits shared memory with that box */
   float4* parts;             /* [n_splits][m_blocks * kHeadM] */
   WsHeader* hdr;
+  /* candidates drawn at a temperature (Algorithm 2 line 4): per row and 32-column chunk the log2 of the chunk's
+     tempered weight, and the chunk's own draw (with the row's entry uniform, in index order) */
+  float c_tau;               /* log2(e) / tau */
+  unsigned long long seed; int step;
+  int Ll, pos0; const int32_t* row_pos0;   /* row -> (sequence, position), for the row's uniforms */
+  float* lw;                 /* [n_groups][m_blocks * kHeadM] */
+  float* xt;                 /* [n_groups][m_blocks * kHeadM] the logit of the chunk's drawn entry */
+  unsigned char* jt;         /* [n_groups][m_blocks * kHeadM] its index inside the chunk (255: the chunk has no weight) */
+  const float4* merged;      /* head_draw_kernel: [m_blocks * kHeadM] the rows' merged records */
+  float4* draw;              /* head_draw_kernel: [m_blocks * kHeadM] out (token, its logit, total, 0) */
 };
 
 /* One tensor map of the weight per tile width (box rows = 32, 64, ..., 256): a narrow tile fetched as
@@ -163,6 +173,7 @@ __device__ __forceinline__ void head_tmem_ld32(uint32_t taddr, uint32_t (&v)[32]
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+template <bool TEMP>
 __global__ void __launch_bounds__(kHeadThreads, 1)
 head_gemm_reduce_kernel(const __grid_constant__ HeadMaps maps, const HeadParams p) {
   extern __shared__ unsigned char head_smem_raw[];
@@ -259,6 +270,12 @@ head_gemm_reduce_kernel(const __grid_constant__ HeadMaps maps, const HeadParams 
     const int quad = warp & 3;                              /* the 32 tensor-memory lanes this warp may read */
     const int row = mb * kHeadM + quad * 32 + lane;
     const bool has_rows = mb * kHeadM + quad * 32 < p.rows;  /* a warp whose 32 rows lie beyond the window only hands the accumulator back */
+    float u_tok = 0.5f;                                      /* TEMP: the uniform that draws inside a chunk, the same for every chunk of the row */
+    if (TEMP && row < p.rows) {
+      const int b = row / p.Ll, k = (p.row_pos0 ? p.row_pos0[b] : p.pos0) + (row - b * p.Ll);
+      u_tok = sample_uniform_token(sample_row_key(p.seed, p.step, b, k));
+    }
+    const size_t rows_pad = (size_t)p.m_blocks * kHeadM;
     float m = -INFINITY, s = 0.f, t2 = 0.f;
     int idx = kIdxNone;
     bool ok = true;
@@ -278,6 +295,40 @@ head_gemm_reduce_kernel(const __grid_constant__ HeadMaps maps, const HeadParams 
 #pragma unroll
           for (int j = 0; j < 32; ++j)
             if (cbase + j >= p.V) v[j] = __float_as_uint(-1.0e30f);
+        }
+        if (TEMP) {
+          /* the chunk as a slice of the vocabulary: its tempered weight (as a log2, against nothing: the
+             rows' maxima are not known yet) and its own draw by inversion in index order */
+          float cmax = -INFINITY;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) cmax = fmaxf(cmax, __uint_as_float(v[j]));
+          const float nref = -cmax * p.c_tau;
+          float wj[32];
+          float cs = 0.f;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            wj[j] = ex2_approx(fmaf(__uint_as_float(v[j]), p.c_tau, nref));   /* -inf and the columns that do not exist: 0 */
+            cs += wj[j];
+          }
+          const float target = u_tok * cs;
+          float run = 0.f;
+          int jt = 255;
+          bool found = false;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            if (!found && wj[j] > 0.f) { run += wj[j]; jt = j; found = run >= target; }   /* (the last entry with weight stands if rounding leaves the sum short) */
+          }
+          float xsel = cmax;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) xsel = (j == jt) ? __uint_as_float(v[j]) : xsel;
+          float lg;
+          asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(lg) : "f"(cs));
+          const size_t at = (size_t)(cbase >> 5) * rows_pad + (size_t)row;
+          if (row < (int)rows_pad) {
+            p.lw[at] = (cs > 0.f && cmax > -1.0e29f) ? lg + cmax * p.c_tau : -INFINITY;
+            p.xt[at] = xsel;
+            p.jt[at] = (unsigned char)jt;
+          }
         }
         /* the exact running maximum and its first index (columns ascend: strict > keeps the lowest) */
         const float m_old = m;
@@ -330,6 +381,79 @@ __global__ void __launch_bounds__(kHeadMergeNT) head_merge_kernel(const HeadPara
   for (int j = lane; j < p.n_splits; j += 32) acc = part_merge(acc, part_from(__ldg(p.parts + (size_t)j * n + row)));
   acc = part_warp_reduce(acc);
   if (lane == 0) merged[row] = make_float4(acc.m, acc.s, acc.t, __int_as_float(acc.idx));
+}
+
+/* Drawn candidates, second stage: the chunk of every window row by inversion with the row's slice uniform
+   over the chunks' tempered weights (now against the row's maximum), in ascending order; the token is
+   that chunk's own draw.  One CTA per 32 rows, lane = row, the chunks dealt to the warps in consecutive
+   ranges (reads of 32 consecutive rows are one line). */
+constexpr int kHeadDrawNT = 1024;
+constexpr int kHeadDrawBatch = 8;           /* loads in flight per thread: the loop is a chain of trips to L2 otherwise */
+__global__ void __launch_bounds__(kHeadDrawNT) head_draw_kernel(const HeadParams p) {
+  __shared__ float part[kHeadDrawNT / 32][32];
+  asm volatile("griddepcontrol.launch_dependents;");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int lane = (int)threadIdx.x & 31, warp = (int)threadIdx.x >> 5, nw = kHeadDrawNT / 32;
+  const int row = (int)blockIdx.x * 32 + lane;
+  const size_t rows_pad = (size_t)p.m_blocks * kHeadM;
+  const bool valid = row < p.rows;
+  const float M = valid ? p.merged[row].x : 0.f;
+  const float nM = -M * p.c_tau;
+  const int per = (p.n_groups + nw - 1) / nw, c0 = warp * per, c1 = min(c0 + per, p.n_groups);
+  float sum = 0.f;
+  if (valid)
+    for (int c = c0; c < c1; c += kHeadDrawBatch) {
+      float l[kHeadDrawBatch];
+#pragma unroll
+      for (int i = 0; i < kHeadDrawBatch; ++i) l[i] = (c + i < c1) ? __ldg(p.lw + (size_t)(c + i) * rows_pad + row) : -INFINITY;
+#pragma unroll
+      for (int i = 0; i < kHeadDrawBatch; ++i) sum += ex2_approx(l[i] + nM);   /* in ascending order, as the second look below */
+    }
+  part[warp][lane] = sum;
+  __syncthreads();
+  float total = 0.f;
+#pragma unroll
+  for (int w = 0; w < nw; ++w) total += part[w][lane];
+  float u_slice = 0.5f;
+  if (valid) {
+    const int b = row / p.Ll, k = (p.row_pos0 ? p.row_pos0[b] : p.pos0) + (row - b * p.Ll);
+    u_slice = sample_uniform_slice(sample_row_key(p.seed, p.step, b, k));
+  }
+  const float target = u_slice * total;
+  int ws = -1;                                               /* the range that holds the target (the last one with weight if rounding leaves the sum short) */
+  float before = 0.f, run = 0.f;
+  bool found = false;
+#pragma unroll
+  for (int w = 0; w < nw; ++w) {
+    const float pw = part[w][lane];
+    if (!found && pw > 0.f) { before = run; run += pw; ws = w; found = run >= target; }
+  }
+  if (valid && ws == warp) {
+    const float rest = target - before;
+    float acc = 0.f;
+    int pick = -1;
+    bool got = false;
+    for (int c = c0; c < c1 && !got; c += kHeadDrawBatch) {
+      float l[kHeadDrawBatch];
+#pragma unroll
+      for (int i = 0; i < kHeadDrawBatch; ++i) l[i] = (c + i < c1) ? __ldg(p.lw + (size_t)(c + i) * rows_pad + row) : -INFINITY;
+#pragma unroll
+      for (int i = 0; i < kHeadDrawBatch; ++i) {
+        const float w = ex2_approx(l[i] + nM);
+        if (!got && w > 0.f) { acc += w; pick = c + i; got = acc >= rest; }
+      }
+    }
+    int tok = -1;
+    float xs = M;
+    if (pick >= 0) {
+      const size_t at = (size_t)pick * rows_pad + row;
+      const int j = (int)p.jt[at];
+      if (j < 32) { tok = pick * 32 + j; xs = p.xt[at]; }
+    }
+    p.draw[row] = make_float4(__int_as_float(tok), xs, total, 0.f);
+  } else if (valid && ws < 0 && warp == 0) {
+    p.draw[row] = make_float4(__int_as_float(-1), M, total, 0.f);   /* nothing with weight: the arg-max stands in */
+  }
 }
 
 }  // namespace forkd

@@ -149,6 +149,7 @@ struct ReduceParams {
                                         instance of the kernel alone; 0 = none) */
   int l2_evict_first;                /* bulk copies of logits carry the L2 "evict first" hint */
   const int32_t* vp_pos0_seq;        /* fused LM-head step: NULL, or [B] the position of row 0 of each sequence's window */
+  const float4* head_draw;           /* fused LM-head step with drawn candidates: [window rows] (token, its logit, total, 0) */
   int min_units;                     /* small steps: units per participating CTA (fork_effective_grid) */
   LoopCtl* loop;                     /* a step of fork_decode_loop: where the cursors of the next step go (else NULL) */
   int vocab_offset;                  /* vocabulary-parallel slices: global index of entry 0 of this buffer */

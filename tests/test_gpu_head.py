@@ -132,7 +132,8 @@ def test_fallback_orders_on_the_fused_head(mode):
     compare_step_state(g, o, rtol=HEAD_RTOL, atol=HEAD_ATOL)
 
 
-def test_decode_loop_on_hidden_states():
+@pytest.mark.parametrize("tau", [0.0, 0.8])
+def test_decode_loop_on_hidden_states(tau):
     """fork_decode_loop_fused_head: every step the provider hands over the hidden states of each sequence's own
     active block (row l of sequence b = position lo[b] + l) and the step runs on the product with the head; the
     whole loop against the oracle's loop on the same products, sequences drifting apart in their blocks."""
@@ -140,6 +141,8 @@ def test_decode_loop_on_hidden_states():
     from helpers import live_mask
     B, Lt, BL, V, d, lam = 3, 24, 8, 3000, 256, 0.6
     w_bits, w_dev = weight(V, d)
+    slices = np.append(np.arange(0, V, 32), V).astype(np.int32)
+    draw = dict(temperature=tau, sample_seed=99, slices=slices) if tau > 0 else {}
     o = oracle.StepState(B, Lt)
     lo, hi = oracle.block_cursors(o.mask, 0, Lt, BL)
     hidden_steps = []
@@ -148,7 +151,7 @@ def test_decode_loop_on_hidden_states():
         assert step < 200
         live = live_mask(o.mask, lo, hi)
         for nonce in range(64):
-            h_bits, _ = fs.head_hidden(w_bits, B * BL, seed=7000 + 64 * step + nonce, h_lo=0.0, h_hi=9.0)
+            h_bits, _ = fs.head_hidden(w_bits, B * BL, seed=7000 + 64 * step + nonce, h_lo=0.0 if tau == 0 else 3.0, h_hi=9.0 if tau == 0 else 12.0)
             blocks = oracle.head_logits(h_bits, w_bits).reshape(B, BL, V)
             full = np.full((B, Lt, V), np.nan, np.float32)      # rows outside a sequence's block must not be read
             for b in range(B):
@@ -156,10 +159,11 @@ def test_decode_loop_on_hidden_states():
                 full[b, lo[b]:lo[b] + n] = blocks[b, :n]
             import copy
             trial = copy.deepcopy(o)
-            assert oracle.step(trial, full, lo, hi, lam, step_id=step) == 0
+            assert oracle.step(trial, full, lo, hi, lam, step_id=step, **draw) == 0
             rows = full[live]
             top2 = np.partition(rows, V - 2, axis=1)[:, V - 2:]
-            if (np.abs(trial.conf[live] - np.float64(np.float32(lam))) >= 2e-3).all() and ((top2[:, 1] - top2[:, 0]) >= 5e-3).all():
+            if (np.abs(trial.conf[live] - np.float64(np.float32(lam))) >= 2e-3).all() and ((top2[:, 1] - top2[:, 0]) >= 5e-3).all() \
+                    and (tau == 0 or (trial.sample_margin[live] >= 5e-4).all()):
                 break
         else:
             raise AssertionError("no draw with clear margins at step %d" % step)
@@ -167,7 +171,7 @@ def test_decode_loop_on_hidden_states():
         hidden_steps.append(torch.from_numpy(h_bits.view(np.int16)).view(torch.bfloat16).view(B, BL, d).pin_memory())
         step += 1
         lo, hi = oracle.block_cursors(o.mask, 0, Lt, BL, lo, hi)
-    assert step > Lt // BL                                       # more than one step per block: thresholds and fallbacks both occur
+    assert tau > 0 or step > Lt // BL                            # more than one step per block: thresholds and fallbacks both occur
     st = pkg.ForkState(B, Lt)
     hid = torch.zeros((B, BL, d), dtype=torch.bfloat16, device="cuda")
     calls = []
@@ -177,11 +181,109 @@ def test_decode_loop_on_hidden_states():
         hid.copy_(hidden_steps[min(s_, len(hidden_steps) - 1)], non_blocking=True)
         return 0
 
-    rc, steps = pkg.fork_decode_loop_fused_head(st, hid, w_dev, BL, 0, Lt, model, None, lam, max_steps=200)
+    rc, steps = pkg.fork_decode_loop_fused_head(st, hid, w_dev, BL, 0, Lt, model, None, lam, max_steps=200,
+                                                **({"temperature": tau, "sample_seed": 99} if tau > 0 else {}))
     torch.cuda.synchronize()
     assert rc == 0 and steps == step and calls == list(range(step))
     assert pkg.fork_device_status(st) == 0
     g = st.host()
     assert g["mask"].sum() == 0
     compare_step_state(g, o, rtol=HEAD_RTOL, atol=HEAD_ATOL)
-    assert (g["nfe"] == o.nfe).all() and g["n_fallback"].sum() > 0
+    assert (g["nfe"] == o.nfe).all() and (g["n_fallback"] == o.n_fallback).all()
+    assert tau > 0 or g["n_fallback"].sum() > 0                # (the drawn case plants high peaks to keep its draws clear: no fallbacks there)
+
+
+@pytest.mark.parametrize("B,Ll,V,d,tau", [(3, 7, 1000, 128, 0.8), (4, 8, 40000, 256, 0.8), (2, 16, 5003, 192, 1.3)])
+def test_drawn_candidates_on_the_fused_head(B, Ll, V, d, tau):
+    """Candidates at a temperature on the fused-head step: the two-stage draw (a chunk of 32 consecutive entries by
+    the row's slice uniform, the token inside it by its entry uniform, both by inversion in ascending order) is the
+    oracle's draw with the vocabulary in slices of 32; tokens are compared exactly on inputs whose draws keep clear of
+    the boundaries of the running sums, confidence and log-probability are the untempered ones of the drawn token."""
+    import paper_2609_39859_b200 as pkg
+    Lt, lam, seed = Ll, 0.9, 77
+    w_bits, w_dev = weight(V, d)
+    rng = np.random.default_rng(3 * V + B)
+    mask = (rng.random((B, Lt)) < 0.9).astype(np.uint8)
+    lo, hi = np.zeros(B, np.int32), np.full(B, Ll, np.int32)
+    slices = np.append(np.arange(0, V, 32), V).astype(np.int32)
+    for nonce in range(48):
+        h_bits, _ = fs.head_hidden(w_bits, B * Ll, seed=31000 + 48 * (V % 97) + nonce, h_lo=3.0, h_hi=12.0)
+        logits = oracle.head_logits(h_bits, w_bits).reshape(B, Ll, V)
+        o = oracle.StepState(B, Lt, mask=mask)
+        assert oracle.step(o, logits, lo, hi, lam, step_id=4, temperature=tau, sample_seed=seed, slices=slices) == 0
+        live = (mask != 0)
+        # (with a chunk per 32 entries the running sum over the chunks has a boundary every 1/1250 of a flat row's
+        # mass: the margin is what the draws of these few rows keep, not a bound on the kernels' error)
+        if (np.abs(o.conf[live] - np.float64(np.float32(lam))) >= 2e-3).all() and (o.sample_margin[live] >= 5e-4).all():
+            break
+    else:
+        raise AssertionError("no draw with clear margins")
+    st = pkg.ForkState(B, Lt, mask=mask)
+    hid = torch.from_numpy(h_bits.view(np.int16)).cuda().view(torch.bfloat16).view(B, Ll, d)
+    n0 = pkg.fork_kernel_launches()
+    pkg.fork_step_fused_head(st, hid, w_dev, torch.from_numpy(lo).cuda(), torch.from_numpy(hi).cuda(), lam, step=4,
+                             temperature=tau, sample_seed=seed)
+    torch.cuda.synchronize()
+    assert pkg.fork_kernel_launches() - n0 == 5               # active set, product + reduction, merge, draw, unmask rule
+    assert pkg.fork_device_status(st) == 0
+    g = st.host()
+    compare_step_state(g, o, rtol=HEAD_RTOL, atol=HEAD_ATOL)
+
+
+def test_drawn_candidates_on_the_fused_head_at_a_block_of_eight_sequences():
+    """256 window rows, V = 40000: per position, the drawn token is the oracle's wherever the oracle's draw keeps
+    clear of the boundaries of its running sums (and nearly everywhere else), and confidence, log-probability and
+    entropy of every position with the same token agree; it is a draw, not the arg-max."""
+    import paper_2609_39859_b200 as pkg
+    B, Ll, V, d, tau, seed = 8, 32, 40000, 256, 0.8, 78
+    w_bits, w_dev = weight(V, d)
+    mask = np.ones((B, Ll), np.uint8)
+    lo, hi = np.zeros(B, np.int32), np.full(B, Ll, np.int32)
+    slices = np.append(np.arange(0, V, 32), V).astype(np.int32)
+    h_bits, _ = fs.head_hidden(w_bits, B * Ll, seed=4242, h_lo=0.0, h_hi=10.0)
+    logits = oracle.head_logits(h_bits, w_bits).reshape(B, Ll, V)
+    o = oracle.StepState(B, Ll, mask=mask)
+    assert oracle.step(o, logits, lo, hi, 2.0, step_id=1, temperature=tau, sample_seed=seed, slices=slices) == 0
+    st = pkg.ForkState(B, Ll, mask=mask)
+    hid = torch.from_numpy(h_bits.view(np.int16)).cuda().view(torch.bfloat16).view(B, Ll, d)
+    pkg.fork_step_fused_head(st, hid, w_dev, torch.from_numpy(lo).cuda(), torch.from_numpy(hi).cuda(), 2.0, step=1,
+                             temperature=tau, sample_seed=seed)
+    torch.cuda.synchronize()
+    g = st.host()
+    same = g["cand"] == o.cand
+    clear = o.sample_margin >= 2e-3
+    assert same[clear].all() and clear.mean() > 0.5
+    assert same.mean() > 0.97
+    for name in ("conf", "logp", "entropy"):
+        got, want = g[name][same].astype(np.float64), getattr(o, name)[same]
+        assert (np.abs(got - want) <= HEAD_ATOL + HEAD_RTOL * np.abs(want)).all(), name
+    assert (g["cand"] != logits.argmax(-1)).mean() > 0.05       # it is a draw, not the arg-max
+    assert (g["n_unmasked"] == 1).all() and (g["is_fallback"] == 1).all()   # threshold 2: every sequence commits its leftmost position
+
+
+def test_drawn_candidates_on_the_fused_head_follow_the_tempered_softmax():
+    """Distribution: one row's hidden state repeated over many positions and seeds; the drawn tokens against
+    softmax(logits / tau) by chi-square on the likeliest tokens."""
+    import paper_2609_39859_b200 as pkg
+    from scipy import stats
+    B, Ll, V, d, tau = 16, 32, 1000, 128, 0.9
+    w_bits, w_dev = weight(V, d)
+    h_bits, _ = fs.head_hidden(w_bits, 1, seed=5, sigma=2.0, h_lo=1.0, h_hi=1.0)
+    logits = oracle.head_logits(h_bits, w_bits)[0].astype(np.float64)
+    prob = np.exp((logits - logits.max()) / tau)
+    prob /= prob.sum()
+    hid = torch.from_numpy(np.repeat(h_bits, B * Ll, 0).view(np.int16)).cuda().view(torch.bfloat16).view(B, Ll, d)
+    lo = torch.zeros(B, dtype=torch.int32, device="cuda")
+    hi = torch.full((B,), Ll, dtype=torch.int32, device="cuda")
+    counts = np.zeros(V, np.int64)
+    for seed in range(24):
+        st = pkg.ForkState(B, Ll)
+        pkg.fork_step_fused_head(st, hid, w_dev, lo, hi, 2.0, step=seed, temperature=tau, sample_seed=1000 + seed)
+        torch.cuda.synchronize()
+        counts += np.bincount(st.host()["cand"].ravel(), minlength=V)
+    n = counts.sum()
+    top = np.flatnonzero(prob * n >= 8)                          # the tokens likely enough for a chi-square cell of their own
+    obs = np.append(counts[top], n - counts[top].sum())
+    exp = np.append(prob[top], 1 - prob[top].sum()) * n
+    assert len(top) >= 20 and exp.min() > 5
+    assert stats.chisquare(obs, exp).pvalue > 1e-4

@@ -194,8 +194,13 @@ def test_invalid_arguments_of_the_variant_entry_points():
         bad = pkg.fork_head_args.from_buffer_copy(hd)
         setattr(bad, field, value)
         assert L.fork_step_fused_head(C.byref(a), C.byref(bad), ws, nbytes, None) == INV, field
-    a.temperature = 0.8                                                   # arg-max candidates only
+    a.temperature = 0.8                                                   # drawn candidates need their scratch
+    assert L.fork_step_fused_head(C.byref(a), C.byref(hd), ws, nbytes, None) == pkg.FORK_ERR_WORKSPACE
+    a.sample_scratch, a.sample_scratch_bytes = 0x80000, L.fork_head_sample_scratch_bytes(a.B, a.Ll, a.V) - 1
+    assert L.fork_step_fused_head(C.byref(a), C.byref(hd), ws, nbytes, None) == pkg.FORK_ERR_WORKSPACE
+    a.temperature = -1.0
     assert L.fork_step_fused_head(C.byref(a), C.byref(hd), ws, nbytes, None) == INV
+    assert L.fork_head_sample_scratch_bytes(8, 32, 126464) == 2 * 3952 * 256 * 4 + 3952 * 256 + 256 * 16
     a = good_step_args()
     cb = pkg.binding.fork_logits_fn(lambda *x: 0)
     fn = C.cast(cb, C.c_void_p)
