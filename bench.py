@@ -1062,7 +1062,8 @@ def main():
                                        "vs_unfused": round(fh[0]["speedup_vs_unfused"], 3)}
         summary["fused_head_R256"] = {"us_per_step": round(fh[1]["fused_ms"] * 1e3, 1),
                                       "weight_read_frac_of_hbm_peak": round(fh[1]["weight_read_frac_of_hbm_peak"], 4),
-                                      "vs_unfused": round(fh[1]["speedup_vs_unfused"], 3)}
+                                      "vs_unfused": round(fh[1]["speedup_vs_unfused"], 3),
+                                      "us_per_step_candidates_drawn_tau0.8": round(fh[1]["fused_ms_candidates_drawn_tau0.8"] * 1e3, 1)}
         also.extend(fh)
         ro = read_only_ceiling(device)
         out["roofline"]["read_only_ceiling_gbs"] = ro          # the library's own read-only streaming probe, same run
