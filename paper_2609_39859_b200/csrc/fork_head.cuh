@@ -388,7 +388,7 @@ __global__ void __launch_bounds__(kHeadMergeNT) head_merge_kernel(const HeadPara
    that chunk's own draw.  One CTA per 32 rows, lane = row, the chunks dealt to the warps in consecutive
    ranges (reads of 32 consecutive rows are one line). */
 constexpr int kHeadDrawNT = 1024;
-constexpr int kHeadDrawBatch = 8;           /* loads in flight per thread: the loop is a chain of trips to L2 otherwise */
+constexpr int kHeadDrawBatch = 16;          /* loads in flight per thread: the loop is a chain of trips to L2 otherwise */
 __global__ void __launch_bounds__(kHeadDrawNT) head_draw_kernel(const HeadParams p) {
   __shared__ float part[kHeadDrawNT / 32][32];
   asm volatile("griddepcontrol.launch_dependents;");
