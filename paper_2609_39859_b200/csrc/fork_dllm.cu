@@ -1704,6 +1704,7 @@ static void head_init() {
 }
 
 /* a [rows, d] bf16 matrix, d contiguous, row stride `ld` elements, cut into boxes of box_rows x 64 with the 128-byte swizzle */
+constexpr int FORK_HEAD_MAX_SPLITS = 256;                   /* column ranges (CTAs along the vocabulary) of a launch: at most the SM count */
 static bool head_tensor_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t d, uint64_t ld, uint32_t box_rows) {
   const cuuint64_t dims[2] = {d, rows};
   const cuuint64_t strides[1] = {ld * 2};
@@ -1718,7 +1719,8 @@ extern "C" size_t fork_head_sample_scratch_bytes(int32_t B, int32_t Ll, int32_t 
   if (B < 0 || Ll <= 0 || V <= 0) return 0;
   const size_t rows_pad = (((size_t)(B > 0 ? B : 1) * (size_t)Ll + kHeadM - 1) / kHeadM) * kHeadM;
   const size_t cells = (size_t)((V + kHeadGroup - 1) / kHeadGroup) * rows_pad;
-  return 2 * align_up(cells * 4, 256) + align_up(cells, 256) + align_up(rows_pad * sizeof(float4), 256);
+  return 2 * align_up(cells * 4, 256) + align_up(cells, 256) + align_up(rows_pad * sizeof(float4), 256) +
+         align_up((size_t)FORK_HEAD_MAX_SPLITS * rows_pad * sizeof(float), 256);
 }
 
 static fork_status check_head_args(const fork_step_args* a, const fork_head_args* h, bool need_bounds) {
@@ -1769,6 +1771,7 @@ static fork_status head_step_impl(const fork_step_args* a, const fork_head_args*
   const int n_units = (hp.n_groups + hp.unit - 1) / hp.unit;
   int splits = dev->sms / hp.m_blocks;
   if (splits < 1) splits = 1;
+  if (splits > FORK_HEAD_MAX_SPLITS) splits = FORK_HEAD_MAX_SPLITS;   /* (what the sample scratch has room for) */
   if (splits > n_units) splits = n_units;
   hp.n_splits = splits;
   hp.u_base = n_units / splits; hp.u_rem = n_units % splits;
@@ -1786,6 +1789,7 @@ static fork_status head_step_impl(const fork_step_args* a, const fork_head_args*
     hp.xt = (float*)(base + align_up(cells * 4, 256));
     hp.jt = (unsigned char*)(base + 2 * align_up(cells * 4, 256));
     hp.draw = (float4*)(base + 2 * align_up(cells * 4, 256) + align_up(cells, 256));
+    hp.lws = (float*)(base + 2 * align_up(cells * 4, 256) + align_up(cells, 256) + align_up((size_t)hp.m_blocks * kHeadM * sizeof(float4), 256));
     hp.merged = w.parts;
     hp.c_tau = (float)(1.4426950408889634 / (double)a->temperature);
     hp.seed = a->sample_seed; hp.step = a->step; hp.Ll = a->Ll; hp.pos0 = a->pos0; hp.row_pos0 = row_pos0;
@@ -1850,7 +1854,10 @@ static fork_status head_step_impl(const fork_step_args* a, const fork_head_args*
     g_launches.fetch_add(1);
     if (drawn) {                                             /* the chunk of every row, now that the rows' maxima are known */
       cfg.gridDim = dim3((unsigned)((hp.rows + 31) / 32)); cfg.blockDim = dim3(kHeadDrawNT);
-      if (cudaLaunchKernelEx(&cfg, head_draw_kernel, hp) != cudaSuccess) return FORK_ERR_CUDA;
+      /* many short column ranges (few window rows): the range first, then its chunks; else all chunks in two passes */
+      const bool by_ranges = hp.n_splits <= 256 && (hp.u_base + 1) * hp.unit <= kHeadDrawMaxRangeChunks;
+      if ((by_ranges ? cudaLaunchKernelEx(&cfg, head_draw_ranges_kernel, hp)
+                     : cudaLaunchKernelEx(&cfg, head_draw_kernel, hp)) != cudaSuccess) return FORK_ERR_CUDA;
       g_launches.fetch_add(1);
     }
   }

@@ -77,6 +77,7 @@ struct HeadParams {
   float* lw;                 /* [n_groups][m_blocks * kHeadM] */
   float* xt;                 /* [n_groups][m_blocks * kHeadM] the logit of the chunk's drawn entry */
   unsigned char* jt;         /* [n_groups][m_blocks * kHeadM] its index inside the chunk (255: the chunk has no weight) */
+  float* lws;                /* [n_splits][m_blocks * kHeadM] log2 of the tempered weight of a CTA's whole column range */
   const float4* merged;      /* head_draw_kernel: [m_blocks * kHeadM] the rows' merged records */
   float4* draw;              /* head_draw_kernel: [m_blocks * kHeadM] out (token, its logit, total, 0) */
 };
@@ -276,6 +277,7 @@ head_gemm_reduce_kernel(const __grid_constant__ HeadMaps maps, const HeadParams 
       u_tok = sample_uniform_token(sample_row_key(p.seed, p.step, b, k));
     }
     const size_t rows_pad = (size_t)p.m_blocks * kHeadM;
+    float st_run = 0.f;                                      /* TEMP: tempered weight of the columns so far, against the running maximum */
     float m = -INFINITY, s = 0.f, t2 = 0.f;
     int idx = kIdxNone;
     bool ok = true;
@@ -296,15 +298,14 @@ head_gemm_reduce_kernel(const __grid_constant__ HeadMaps maps, const HeadParams 
           for (int j = 0; j < 32; ++j)
             if (cbase + j >= p.V) v[j] = __float_as_uint(-1.0e30f);
         }
+        float cmax = -INFINITY, cs = 0.f;                    /* TEMP: the chunk's maximum and its tempered weight against it */
         if (TEMP) {
           /* the chunk as a slice of the vocabulary: its tempered weight (as a log2, against nothing: the
              rows' maxima are not known yet) and its own draw by inversion in index order */
-          float cmax = -INFINITY;
 #pragma unroll
           for (int j = 0; j < 32; ++j) cmax = fmaxf(cmax, __uint_as_float(v[j]));
           const float nref = -cmax * p.c_tau;
           float wj[32];
-          float cs = 0.f;
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
             wj[j] = ex2_approx(fmaf(__uint_as_float(v[j]), p.c_tau, nref));   /* -inf and the columns that do not exist: 0 */
@@ -338,6 +339,11 @@ head_gemm_reduce_kernel(const __grid_constant__ HeadMaps maps, const HeadParams 
           if (x > m) { m = x; idx = cbase + j; }
         }
         /* (s, t2) re-expressed against the new maximum, then this chunk's terms */
+        if (TEMP) {                                          /* the range's weight so far, re-expressed against the new maximum */
+          const float keep = (m_old > -INFINITY) ? ex2_approx((m_old - m) * p.c_tau) : 0.f;
+          const float add = (cs > 0.f && cmax > -1.0e29f) ? cs * ex2_approx((cmax - m) * p.c_tau) : 0.f;
+          st_run = fmaf(st_run, keep, add);
+        }
         const float dd = (m_old > -INFINITY) ? (m_old - m) * kLog2e : 0.f;
         const float w = (m_old > -INFINITY) ? ex2_approx(dd) : 0.f;
         t2 = w * fmaf(dd, s, t2);
@@ -355,8 +361,14 @@ head_gemm_reduce_kernel(const __grid_constant__ HeadMaps maps, const HeadParams 
       __syncwarp();
       if (lane == 0) head_mbar_arrive(&hb.acc_empty[acc]);
     }
-    if (ok && row < p.m_blocks * kHeadM)
+    if (ok && row < p.m_blocks * kHeadM) {
       p.parts[(size_t)ns * ((size_t)p.m_blocks * kHeadM) + row] = make_float4(m, s, t2, __int_as_float(idx));
+      if (TEMP) {
+        float lg;
+        asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(lg) : "f"(st_run));
+        p.lws[(size_t)ns * rows_pad + row] = (st_run > 0.f && m > -1.0e29f) ? lg + m * p.c_tau : -INFINITY;
+      }
+    }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
@@ -453,6 +465,85 @@ __global__ void __launch_bounds__(kHeadDrawNT) head_draw_kernel(const HeadParams
     p.draw[row] = make_float4(__int_as_float(tok), xs, total, 0.f);
   } else if (valid && ws < 0 && warp == 0) {
     p.draw[row] = make_float4(__int_as_float(-1), M, total, 0.f);   /* nothing with weight: the arg-max stands in */
+  }
+}
+
+/* The same when a CTA's column range is short (few window rows, many CTAs along the vocabulary): first the CTA
+   range by its weight (one value per range and row, written by the GEMM's epilogue), then the chunk inside
+   that range only -- two short looks instead of two passes over all of a row's chunks. */
+constexpr int kHeadDrawMaxRangeChunks = 32;     /* measured: with 54 chunks per range (256 window rows) the two passes over everything are faster */
+__global__ void __launch_bounds__(kHeadDrawNT) head_draw_ranges_kernel(const HeadParams p) {
+  __shared__ float part[kHeadDrawNT / 32][32];
+  asm volatile("griddepcontrol.launch_dependents;");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int lane = (int)threadIdx.x & 31, warp = (int)threadIdx.x >> 5, nw = kHeadDrawNT / 32;
+  const int row = (int)blockIdx.x * 32 + lane;
+  const size_t rows_pad = (size_t)p.m_blocks * kHeadM;
+  const bool valid = row < p.rows;
+  const float M = valid ? p.merged[row].x : 0.f;
+  const float nM = -M * p.c_tau;
+  constexpr int kPer = 8;                                    /* ranges per warp: 32 warps x 8 covers every grid this kernel is used for */
+  const int s0 = warp * kPer;
+  float wr[kPer];
+  float sum = 0.f;
+#pragma unroll
+  for (int i = 0; i < kPer; ++i) {
+    const float l = (valid && s0 + i < p.n_splits) ? __ldg(p.lws + (size_t)(s0 + i) * rows_pad + row) : -INFINITY;
+    wr[i] = ex2_approx(l + nM);
+    sum += wr[i];
+  }
+  part[warp][lane] = sum;
+  __syncthreads();
+  float total = 0.f;
+#pragma unroll
+  for (int w = 0; w < nw; ++w) total += part[w][lane];
+  float u_slice = 0.5f;
+  if (valid) {
+    const int b = row / p.Ll, k = (p.row_pos0 ? p.row_pos0[b] : p.pos0) + (row - b * p.Ll);
+    u_slice = sample_uniform_slice(sample_row_key(p.seed, p.step, b, k));
+  }
+  const float target = u_slice * total;
+  int ws = -1;
+  float before = 0.f, run = 0.f;
+  bool found = false;
+#pragma unroll
+  for (int w = 0; w < nw; ++w) {
+    const float pw = part[w][lane];
+    if (!found && pw > 0.f) { before = run; run += pw; ws = w; found = run >= target; }
+  }
+  if (valid && ws == warp) {
+    /* the range among this warp's eight, then the chunk among the range's */
+    int ns = -1;
+    float acc = before, acc_before = before;
+    bool got = false;
+#pragma unroll
+    for (int i = 0; i < kPer; ++i)
+      if (!got && wr[i] > 0.f) { acc_before = acc; acc += wr[i]; ns = s0 + i; got = acc >= target; }
+    const float rest = target - acc_before;
+    const int c0 = (ns * p.u_base + min(ns, p.u_rem)) * p.unit, c1 = c0 + head_split_groups(p, ns);
+    float a2 = 0.f;
+    int pick = -1;
+    bool got2 = false;
+    for (int c = c0; c < c1 && !got2; c += kHeadDrawBatch) {
+      float l[kHeadDrawBatch];
+#pragma unroll
+      for (int i = 0; i < kHeadDrawBatch; ++i) l[i] = (c + i < c1) ? __ldg(p.lw + (size_t)(c + i) * rows_pad + row) : -INFINITY;
+#pragma unroll
+      for (int i = 0; i < kHeadDrawBatch; ++i) {
+        const float w = ex2_approx(l[i] + nM);
+        if (!got2 && w > 0.f) { a2 += w; pick = c + i; got2 = a2 >= rest; }
+      }
+    }
+    int tok = -1;
+    float xs = M;
+    if (pick >= 0) {
+      const size_t at = (size_t)pick * rows_pad + row;
+      const int j = (int)p.jt[at];
+      if (j < 32) { tok = pick * 32 + j; xs = p.xt[at]; }
+    }
+    p.draw[row] = make_float4(__int_as_float(tok), xs, total, 0.f);
+  } else if (valid && ws < 0 && warp == 0) {
+    p.draw[row] = make_float4(__int_as_float(-1), M, total, 0.f);
   }
 }
 

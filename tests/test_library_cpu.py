@@ -200,7 +200,7 @@ def test_invalid_arguments_of_the_variant_entry_points():
     assert L.fork_step_fused_head(C.byref(a), C.byref(hd), ws, nbytes, None) == pkg.FORK_ERR_WORKSPACE
     a.temperature = -1.0
     assert L.fork_step_fused_head(C.byref(a), C.byref(hd), ws, nbytes, None) == INV
-    assert L.fork_head_sample_scratch_bytes(8, 32, 126464) == 2 * 3952 * 256 * 4 + 3952 * 256 + 256 * 16
+    assert L.fork_head_sample_scratch_bytes(8, 32, 126464) == 2 * 3952 * 256 * 4 + 3952 * 256 + 256 * 16 + 256 * 256 * 4
     a = good_step_args()
     cb = pkg.binding.fork_logits_fn(lambda *x: 0)
     fn = C.cast(cb, C.c_void_p)
