@@ -287,3 +287,32 @@ def test_drawn_candidates_on_the_fused_head_follow_the_tempered_softmax():
     exp = np.append(prob[top], 1 - prob[top].sum()) * n
     assert len(top) >= 20 and exp.min() > 5
     assert stats.chisquare(obs, exp).pvalue > 1e-4
+
+
+def test_drawn_candidates_at_the_llada_head_shape():
+    """d = 4096, V = 126464, 256 window rows (the shape at which every row's chunks are gone through in two passes
+    rather than range by range): the first two sequences' positions against the oracle, as above."""
+    import paper_2609_39859_b200 as pkg
+    B, Ll, V, d, tau, seed, n_check = 8, 32, 126464, 4096, 0.8, 5, 2
+    w_bits, w_dev = weight(V, d)
+    mask = np.ones((B, Ll), np.uint8)
+    lo, hi = np.zeros(B, np.int32), np.full(B, Ll, np.int32)
+    slices = np.append(np.arange(0, V, 32), V).astype(np.int32)
+    h_bits, _ = fs.head_hidden(w_bits, B * Ll, seed=99)
+    logits = oracle.head_logits(h_bits[:n_check * Ll], w_bits).reshape(n_check, Ll, V)
+    o = oracle.StepState(n_check, Ll, mask=mask[:n_check])
+    assert oracle.step(o, logits, lo[:n_check], hi[:n_check], 2.0, step_id=1, temperature=tau, sample_seed=seed, slices=slices) == 0
+    st = pkg.ForkState(B, Ll, mask=mask)
+    hid = torch.from_numpy(h_bits.view(np.int16)).cuda().view(torch.bfloat16).view(B, Ll, d)
+    pkg.fork_step_fused_head(st, hid, w_dev, torch.from_numpy(lo).cuda(), torch.from_numpy(hi).cuda(), 2.0, step=1,
+                             temperature=tau, sample_seed=seed)
+    torch.cuda.synchronize()
+    assert pkg.fork_device_status(st) == 0
+    g = st.host()
+    same = g["cand"][:n_check] == o.cand
+    clear = o.sample_margin >= 2e-3
+    assert same[clear].all() and clear.mean() > 0.4 and same.mean() > 0.9
+    for name in ("conf", "logp", "entropy"):
+        got, want = g[name][:n_check][same].astype(np.float64), getattr(o, name)[same]
+        assert (np.abs(got - want) <= HEAD_ATOL + HEAD_RTOL * np.abs(want)).all(), name
+    assert (g["cand"][:n_check] != logits.argmax(-1)).mean() > 0.05
