@@ -354,6 +354,24 @@ def test_grpo_advantages_and_skipped_groups():
     assert np.allclose(r["adv"], np.array([0.75, -0.25, -0.25, -0.25]) / (math.sqrt(3) / 4))
 
 
+def test_every_position_selected_is_the_justgrpo_objective():
+    """Eq. 1 (JustGRPO) is Eq. 2 with F_i = all L positions: the same call with every position selected against the
+    formula of Eq. 1 written out with numpy (one group statistic per prompt, a mean over positions, a mean over rollouts)."""
+    rng = np.random.default_rng(11)
+    P, G, L, eps = 3, 4, 7, float(np.float32(0.2))            # (the clip range is passed in fp32)
+    B = P * G
+    old = rng.normal(-1.5, 0.5, (B, L)).astype(np.float32)
+    new = (old + rng.normal(0, 0.3, (B, L))).astype(np.float32)
+    reward = rng.random(B).astype(np.float32)
+    r = oracle.grpo_loss(new, old, np.ones((B, L), np.uint8), reward, G, eps, eps)
+    rho = np.exp(new.astype(np.float64) - old.astype(np.float64))
+    rg = reward.astype(np.float64).reshape(P, G)
+    adv = ((rg - rg.mean(1, keepdims=True)) / rg.std(1, keepdims=True)).reshape(B, 1)
+    want = np.minimum(rho * adv, np.clip(rho, 1 - eps, 1 + eps) * adv).mean(1).mean()
+    assert abs(r["objective"] - want) <= 1e-12 * max(1.0, abs(want))
+    assert np.allclose(r["seq_obj"], np.minimum(rho * adv, np.clip(rho, 1 - eps, 1 + eps) * adv).mean(1), rtol=1e-12, atol=1e-14)
+
+
 def test_grpo_clipping_cases_and_fallback_count_average():
     B, Lt, G = 2, 3, 2
     old = np.zeros((B, Lt), np.float32)
