@@ -21,9 +21,11 @@
  *                      online soft-max statistics in registers (exact running maximum with its
  *                      first index, s and t2 rescaled when the maximum rises), while the MMA warp
  *                      already fills the other accumulator.
- * At the end every row's Part goes to head_parts[split][row]; the select kernel of the
- * vocabulary-parallel step merges the splits of a row (they are slices of the vocabulary, exactly
- * like ranks) and applies the unmask rule.
+ * At the end every row's Part goes to head_parts[split][row]; head_merge_kernel merges the splits of
+ * a row (they are slices of the vocabulary, exactly like the ranks of a vocabulary-parallel step) and
+ * the select kernel of that step applies the unmask rule.  With candidates drawn at a temperature
+ * the epilogue also treats every 32-column chunk as a slice of its own (its tempered weight and its
+ * own draw), and a draw kernel picks the chunk once the rows' maxima are known.
  * Every mbarrier wait is bounded; a wait that runs out sets FORK_DEV_TIMEOUT, all roles leave their
  * loops, in-flight copies are waited for, tensor memory is given back.
  */
