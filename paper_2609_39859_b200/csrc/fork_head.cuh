@@ -8,7 +8,7 @@
  * columns, a whole number of 32-column groups dealt out evenly over the CTAs (so that every SM gets
  * the same share of the weight whatever V is), walked in tiles of 256 columns with a narrower last
  * tile.  Warp roles (192 threads):
- *   warp 0  producer : TMA tensor copies (cp.async.bulk.tensor.2d, no multicast) of a tile of hidden
+ *   warp 0  producer : TMA tensor copies (cp.async.bulk.tensor.2d, every CTA fetching for itself) of a tile of hidden
  *                      states (64 columns x 128 rows; 32 or 64 rows when the window has no more, which
  *                      leaves room for more stages) and a 256 x 64 tile of the weight (the narrow last
  *                      tile in 32-row boxes) per k-block into a ring of shared-memory stages
