@@ -316,3 +316,35 @@ def test_drawn_candidates_at_the_llada_head_shape():
         got, want = g[name][:n_check][same].astype(np.float64), getattr(o, name)[same]
         assert (np.abs(got - want) <= HEAD_ATOL + HEAD_RTOL * np.abs(want)).all(), name
     assert (g["cand"][:n_check] != logits.argmax(-1)).mean() > 0.05
+
+
+def test_decode_loop_on_hidden_states_error_paths():
+    """The loop's own outcomes on the hidden-state form: the step limit, a failing provider, and a clean restart
+    from the buffers as they were left."""
+    import paper_2609_39859_b200 as pkg
+    B, Lt, BL, V, d = 2, 16, 8, 1000, 128
+    w_bits, w_dev = weight(V, d)
+    h_bits, _ = fs.head_hidden(w_bits, B * BL, seed=3)
+    hid = torch.from_numpy(h_bits.view(np.int16)).cuda().view(torch.bfloat16).view(B, BL, d)
+    st = pkg.ForkState(B, Lt)
+    rc, steps = pkg.fork_decode_loop_fused_head(st, hid, w_dev, BL, 0, Lt, lambda *a: 0, None, 2.0, max_steps=3, raise_on_error=False)
+    torch.cuda.synchronize()
+    assert rc == pkg.FORK_ERR_MAX_STEPS and steps == 3
+    g = st.host()
+    assert (g["mask"].sum(1) == Lt - 3).all() and g["commit_step"][0, :3].tolist() == [0, 1, 2]   # threshold 2: left to right
+    calls = []
+
+    def failing(step, lo, hi, stream_p):
+        calls.append(step)
+        return 1 if step == 5 else 0
+
+    rc, steps = pkg.fork_decode_loop_fused_head(st, hid, w_dev, BL, 0, Lt, failing, None, 2.0, max_steps=100, step0=3, raise_on_error=False)
+    torch.cuda.synchronize()
+    assert rc == pkg.FORK_ERR_PROVIDER and steps == 2 and calls == [3, 4, 5]
+    rc, steps = pkg.fork_decode_loop_fused_head(st, hid, w_dev, BL, 0, Lt, lambda *a: 0, None, 2.0, max_steps=100, step0=5)
+    torch.cuda.synchronize()
+    g = st.host()
+    assert rc == 0 and steps == Lt - 5 and g["mask"].sum() == 0
+    assert (g["commit_step"] == np.arange(Lt)[None, :]).all() and (g["nfe"] == Lt).all()
+    with pytest.raises(pkg.ForkError):
+        pkg.fork_decode_loop_fused_head(pkg.ForkState(B, Lt), hid, w_dev, BL, 0, Lt, lambda *a: 0, None, 2.0, max_steps=1)
