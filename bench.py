@@ -46,8 +46,8 @@ NOMINAL_HBM_GBS = 8000.0
 # from one ncu capture of that workload; `source` names the summary that holds it.  A shape without a
 # capture of its own reports null.
 NCU_TRAFFIC = {
-    "b8": {"bytes": 64_888_064, "source": "ncu capture of this workload: profiles/reduce_select_ring_bf16_b8_and_passk.md, section 0"},
-    "passk": {"bytes": 522_807_040, "source": "ncu capture of this workload: profiles/reduce_select_ring_bf16_b8_and_passk.md, section 0"},
+    "b8": {"bytes": 64_888_064, "source": "ncu capture of this workload on 2026-11-25 (kernel as of the commit that added the L2 evict-first hint): profiles/reduce_select_ring_bf16_b8_and_passk.md, section 0"},
+    "passk": {"bytes": 522_807_040, "source": "ncu capture of this workload on 2026-11-25 (kernel as of the commit that added the L2 evict-first hint): profiles/reduce_select_ring_bf16_b8_and_passk.md, section 0"},
 }
 FALLBACK_HBM_GBS = 6650.0
 
