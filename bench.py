@@ -502,8 +502,10 @@ def time_fused_head(device, hbm_peak, shapes=((64, 32), (8, 32), (1, 8))):
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
             mp = json.load(f)
         tf_peak, tf_src = float(mp["bf16_tflops"]), "measured (MEASURED_PEAKS.json, cuBLAS bf16 burst)"
+        tf_sustained = float(mp.get("bf16_tflops_sustained", 0.0)) or None
     except Exception:
         tf_peak, tf_src = 1590.0, "fallback (earlier measurement on this pool)"
+        tf_sustained = 1400.0
     gen = torch.Generator(device=device).manual_seed(1234)
     W = torch.randn((V, d), device=device, generator=gen, dtype=torch.float32).to(torch.bfloat16)
     out = []
@@ -553,6 +555,8 @@ def time_fused_head(device, hbm_peak, shapes=((64, 32), (8, 32), (1, 8))):
                     "fused_ms": ms_f, "unfused_gemm_plus_fork_step_ms": ms_u, "speedup_vs_unfused": ms_u / ms_f,
                     "tflops": flops / (ms_f * 1e-3) / 1e12, "frac_of_bf16_peak": flops / (ms_f * 1e-3) / 1e12 / tf_peak,
                     "bf16_peak_tflops": tf_peak, "peak_source": tf_src,
+                    # (these chunks last some ten milliseconds: a burst; the library's own rate under seconds of load beside it)
+                    "frac_of_bf16_sustained_peak": (flops / (ms_f * 1e-3) / 1e12 / tf_sustained) if tf_sustained else None,
                     "weight_read_gbs": V * d * 2 / (ms_f * 1e-3) / 1e9, "weight_read_frac_of_hbm_peak": V * d * 2 / (ms_f * 1e-3) / 1e9 / hbm_peak,
                     "hbm_bytes_not_moved": 2 * R * V * 2, "fused_ms_candidates_drawn_tau0.8": ms_fd,
                     "bound": "tensor" if flops / (tf_peak * 1e12) > V * d * 2 / (hbm_peak * 1e9) else "hbm (one read of the weight)"})
